@@ -1,0 +1,147 @@
+/*
+ * llvq.h -- C ABI of the B200 (sm_100a) LLVQ dequantization library.
+ *
+ * LLVQ stores every block of 24 weights as one integer index into a union of
+ * Leech-lattice shells plus a per-block gain.  This library maps the stored
+ * index stream back to weights on the GPU, with no materialised codebook, and
+ * fuses that with the decode-time matrix-vector / small-batch matrix product.
+ *
+ * Conventions common to all entry points
+ *   - Pointers named d_* are DEVICE pointers owned by the caller; the library
+ *     never allocates, frees or retains them.  `stream` is a cudaStream_t
+ *     passed as void* (NULL = default stream).  Work is enqueued on that
+ *     stream and the call returns without synchronising, unless stated.
+ *   - Every function returns a status code (LLVQ_OK = 0).  Bad arguments are
+ *     rejected on the host before anything is launched.  Nothing throws,
+ *     aborts or traps.
+ *   - Index stream (App. A: the global integer index I; Sec. 2.2: an index
+ *     takes W = ceil(log2 N) bits): field b occupies bits [b*W, (b+1)*W) of a
+ *     little-endian bit stream (stream bit t = bit t%8 of byte t/8).  Indices
+ *     are 0-based, I in [0, N).  The buffer is 16-byte aligned and
+ *     llvq_index_bytes() long (padded with zeros to a multiple of 16 bytes).
+ *   - Gains: one IEEE binary16 bit pattern per block (uint16_t), finite.
+ *   - A field with I >= N decodes to the zero vector and is counted in a
+ *     device-side error counter (see llvq_last_error); it never faults.
+ *   - Block layouts of a rows x cols matrix:
+ *       LLVQ_LAYOUT_FLAT     block b holds elements 24b .. 24b+23 of the
+ *                            row-major flattened matrix; the unused tail of the
+ *                            last block is dropped.
+ *       LLVQ_LAYOUT_ROWWISE  every row has ceil(cols/24) blocks of its own;
+ *                            block r*ceil(cols/24)+c holds columns 24c..24c+23
+ *                            of row r; the unused tail of a row's last block is
+ *                            dropped (App. C pads K the same way).
+ */
+#ifndef LLVQ_H
+#define LLVQ_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct llvq_ctx llvq_ctx;   /* opaque: host + device tables of one code; immutable after create */
+
+enum {
+    LLVQ_OK = 0,
+    LLVQ_EINVAL = 1,        /* null pointer, negative or zero size, unknown enum value    */
+    LLVQ_EALIGN = 2,        /* a pointer or leading dimension violates the stated alignment */
+    LLVQ_EUNSUPPORTED = 3,  /* a size or code outside what the kernels support            */
+    LLVQ_ECUDA = 4,         /* a CUDA runtime call failed                                 */
+    LLVQ_EINDEX = 5,        /* reserved: invalid indices are counted, see llvq_last_error */
+    LLVQ_ETIMEOUT = 6       /* a bounded device-side wait ran out (flag in llvq_last_error) */
+};
+enum { LLVQ_LAYOUT_FLAT = 0, LLVQ_LAYOUT_ROWWISE = 1 };
+enum { LLVQ_F32 = 0, LLVQ_BF16 = 1 };
+enum { LLVQ_FLAG_WAIT_TIMEOUT = 1u };   /* bit in llvq_last_error's flags */
+
+/*
+ * Build the tables of the code  union of Shell(m), m_lo <= m <= m_hi  (Sec. 2.2:
+ * Shell(m) = lattice points of squared norm 2m; m_lo = 2 gives the ball cut
+ * Lambda_24(m_hi)) and upload them to CUDA device `device`.  Classes, their
+ * order, cardinalities A * 2^B * P and cumulative offsets follow Sec. 2.4-2.5
+ * and Sec. 3.2.  Supported: 2 <= m_lo <= m_hi <= 53 with N <= 2^72; (2,2),
+ * (3,3), (2,13) and (2,53) are the codes the benchmarks use.
+ * Allocates the library's own host and device tables; *out is freed by
+ * llvq_destroy.  Synchronous.  device < 0 builds a host-only context: the
+ * query functions work, every function that would launch returns LLVQ_EINVAL.
+ */
+int llvq_create(llvq_ctx** out, int m_lo, int m_hi, int device);
+void llvq_destroy(llvq_ctx* ctx);
+
+/* W = ceil(log2 N): 18 for (2,2), 24 for (3,3), 48 for (2,13), 72 for (2,53) (Sec. 2.2, Table 1). */
+int llvq_index_bits(const llvq_ctx* ctx);
+/* N = number of points of the code, as lo_hi[0] + 2^64 * lo_hi[1]. */
+int llvq_num_points(const llvq_ctx* ctx, uint64_t lo_hi[2]);
+/* Number of classes (Sec. 2.4): 3, 4, 383, 114976 for the four codes above. */
+int llvq_num_classes(const llvq_ctx* ctx);
+/* Bytes of an index stream of nblocks fields: ceil(nblocks*W/8) rounded up to 16. */
+size_t llvq_index_bytes(const llvq_ctx* ctx, uint64_t nblocks);
+
+/*
+ * Host-side introspection of the tables (no device work; used to cross-check the
+ * table generator).  Class j in global order (Sec. 3.2 (1)-(2)):
+ * info = {m, parity (0 even / 1 odd), Golay weight w, sign bits B, number of distinct values};
+ * *A, card and offset (as lo, hi) are the quantities of Sec. 2.5 / App. A step 2;
+ * values[] / mults[] = distinct absolute values, descending, with multiplicities (24 entries of room).
+ */
+int llvq_class_info(const llvq_ctx* ctx, int j, int info[5], uint64_t* A, uint64_t card[2], uint64_t offset[2],
+                    int values[24], int mults[24]);
+/* The 4096 extended-Golay codewords (Sec. 2.3) in table order: by weight, then by value; bit i = coordinate i. */
+int llvq_golay_table(const llvq_ctx* ctx, uint32_t out[4096]);
+
+/*
+ * Dequantizer, App. A steps 1-4: d_points[b][0..23] = the integer lattice point
+ * (coordinates of L^int, |x_i| <= 28) of field b, b < nblocks.
+ * d_idx: device, 16-byte aligned.  d_points: device, int8 [nblocks][24], 4-byte aligned.
+ */
+int llvq_decode_blocks(const llvq_ctx* ctx, const void* d_idx, uint64_t nblocks,
+                       int8_t* d_points, void* stream);
+
+/*
+ * Shape-gain reconstruction w = g * s (App. E, "Shape-gain"; App. A for s):
+ * d_w[r*ld + c] = bf16_rn( float(gain[b]) * float(x[b][j]) ) for the block b and
+ * lane j that hold element (r, c) under `layout`; one rounding, to nearest even.
+ * d_gain_f16: device, [nblocks] binary16 bits.  d_w_bf16: device, bf16 bits,
+ * rows x cols with leading dimension ld >= cols (elements), 2-byte aligned
+ * (16-byte aligned base and ld % 8 == 0 select the vectorised store path).
+ * FLAT requires ld == cols.
+ */
+int llvq_dequant_matrix(const llvq_ctx* ctx, const void* d_idx, const uint16_t* d_gain_f16,
+                        int64_t rows, int64_t cols, int layout,
+                        uint16_t* d_w_bf16, int64_t ld, void* stream);
+
+/*
+ * Fused dequantization + matrix-vector product of App. C: y = W x with
+ * W (n_out x k_in, ROWWISE blocks) never written to memory.  The weights are
+ * the bf16-rounded values llvq_dequant_matrix would produce; products are
+ * accumulated in binary32.  d_x_bf16: device, [k_in] bf16 bits.
+ * d_y: device, [n_out], float (y_dtype = LLVQ_F32) or bf16 bits (LLVQ_BF16).
+ */
+int llvq_gemv(const llvq_ctx* ctx, const void* d_idx, const uint16_t* d_gain_f16,
+              int64_t n_out, int64_t k_in, const uint16_t* d_x_bf16,
+              void* d_y, int y_dtype, void* stream);
+
+/*
+ * The same product for a small batch, Y[b][i] = sum_k X[b][k] W[i][k]
+ * (App. C's kernel generalised to batch <= 64): the dequantized bf16 tile is
+ * fed to the tensor cores, accumulation in binary32.
+ * d_x_bf16: device, [batch][k_in] bf16 bits, 16-byte aligned, k_in % 8 == 0.
+ * d_y_bf16: device, [batch][n_out] bf16 bits.  1 <= batch <= 64.
+ */
+int llvq_gemm_small_batch(const llvq_ctx* ctx, const void* d_idx, const uint16_t* d_gain_f16,
+                          int64_t n_out, int64_t k_in, const uint16_t* d_x_bf16,
+                          int batch, uint16_t* d_y_bf16, void* stream);
+
+/*
+ * Synchronises `stream`, then reports and clears the device-side error state:
+ * *n_bad_index = number of fields with I >= N seen since the last call,
+ * *flags = OR of LLVQ_FLAG_* bits.  Either output pointer may be NULL.
+ */
+int llvq_last_error(llvq_ctx* ctx, void* stream, uint64_t* n_bad_index, uint32_t* flags);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* LLVQ_H */

@@ -1,0 +1,202 @@
+"""Python binding of the LLVQ CUDA library (``include/llvq.h``).
+
+Argument marshalling only: every step of the dequantization path runs in the
+CUDA kernels of ``libllvq.so``.  PyTorch is used for device memory and streams.
+There is no CPU fallback: if the library is missing or the device is not a CUDA
+device, calls raise.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+
+import torch
+
+from .build import LIB
+
+__all__ = [
+    "Context", "llvq_decode_blocks", "llvq_dequant_matrix", "llvq_gemv", "llvq_gemm_small_batch",
+    "llvq_last_error", "LlvqError", "EXPORTS", "load_library",
+    "LLVQ_LAYOUT_FLAT", "LLVQ_LAYOUT_ROWWISE", "LLVQ_F32", "LLVQ_BF16",
+]
+
+LLVQ_LAYOUT_FLAT, LLVQ_LAYOUT_ROWWISE = 0, 1
+LLVQ_F32, LLVQ_BF16 = 0, 1
+_STATUS = {0: "LLVQ_OK", 1: "LLVQ_EINVAL", 2: "LLVQ_EALIGN", 3: "LLVQ_EUNSUPPORTED", 4: "LLVQ_ECUDA",
+           5: "LLVQ_EINDEX", 6: "LLVQ_ETIMEOUT"}
+
+# every symbol include/llvq.h declares
+EXPORTS = [
+    "llvq_create", "llvq_destroy", "llvq_index_bits", "llvq_num_points", "llvq_num_classes", "llvq_index_bytes",
+    "llvq_decode_blocks", "llvq_dequant_matrix", "llvq_gemv", "llvq_gemm_small_batch", "llvq_last_error",
+]
+
+
+class LlvqError(RuntimeError):
+    def __init__(self, call: str, status: int):
+        super().__init__(f"{call} failed: {_STATUS.get(status, status)}")
+        self.status = status
+
+
+_lib = None
+
+
+def load_library() -> ctypes.CDLL:
+    """Load libllvq.so (built in-tree by ``paper_2603_11021_b200.build``); raises if it is missing."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(LIB):
+        raise ImportError(f"{LIB} not found: run `python -m paper_2603_11021_b200.build` (needs nvcc); there is no fallback path")
+    lib = ctypes.CDLL(LIB)
+    vp, i64, u64 = ctypes.c_void_p, ctypes.c_int64, ctypes.c_uint64
+    lib.llvq_create.argtypes = [ctypes.POINTER(vp), ctypes.c_int, ctypes.c_int, ctypes.c_int]
+    lib.llvq_destroy.argtypes = [vp]
+    lib.llvq_destroy.restype = None
+    lib.llvq_index_bits.argtypes = [vp]
+    lib.llvq_num_points.argtypes = [vp, ctypes.POINTER(u64)]
+    lib.llvq_num_classes.argtypes = [vp]
+    lib.llvq_index_bytes.argtypes = [vp, u64]
+    lib.llvq_index_bytes.restype = ctypes.c_size_t
+    lib.llvq_decode_blocks.argtypes = [vp, vp, u64, vp, vp]
+    lib.llvq_dequant_matrix.argtypes = [vp, vp, vp, i64, i64, ctypes.c_int, vp, i64, vp]
+    lib.llvq_gemv.argtypes = [vp, vp, vp, i64, i64, vp, vp, ctypes.c_int, vp]
+    lib.llvq_gemm_small_batch.argtypes = [vp, vp, vp, i64, i64, vp, ctypes.c_int, vp, vp]
+    lib.llvq_last_error.argtypes = [vp, vp, ctypes.POINTER(u64), ctypes.POINTER(ctypes.c_uint32)]
+    lib.llvq_class_info.argtypes = [vp, ctypes.c_int, vp, vp, vp, vp, vp, vp]
+    lib.llvq_golay_table.argtypes = [vp, vp]
+    _lib = lib
+    return lib
+
+
+def _check(call: str, status: int) -> None:
+    if status != 0:
+        raise LlvqError(call, status)
+
+
+def _stream_ptr(stream) -> int:
+    if stream is None:
+        stream = torch.cuda.current_stream()
+    return int(stream.cuda_stream)
+
+
+def _dev(t: torch.Tensor, name: str) -> int:
+    if not (isinstance(t, torch.Tensor) and t.is_cuda and t.is_contiguous()):
+        raise TypeError(f"{name} must be a contiguous CUDA tensor")
+    return t.data_ptr()
+
+
+class Context:
+    """Tables of the code  union of Shell(m), m_lo <= m <= m_hi,  on one CUDA device."""
+
+    def __init__(self, m_lo: int, m_hi: int, device: int = 0):
+        self._lib = load_library()
+        h = ctypes.c_void_p()
+        _check("llvq_create", self._lib.llvq_create(ctypes.byref(h), m_lo, m_hi, device))
+        self._h = h
+        self.device = device
+        self.m_lo, self.m_hi = m_lo, m_hi
+        self.index_bits = int(self._lib.llvq_index_bits(h))
+        out = (ctypes.c_uint64 * 2)()
+        _check("llvq_num_points", self._lib.llvq_num_points(h, out))
+        self.num_points = (int(out[1]) << 64) | int(out[0])
+        self.num_classes = int(self._lib.llvq_num_classes(h))
+
+    def index_bytes(self, nblocks: int) -> int:
+        return int(self._lib.llvq_index_bytes(self._h, nblocks))
+
+    def class_info(self, j: int) -> dict:
+        """Host-side description of class j as the library's own table generator built it."""
+        import numpy as np
+        info = np.zeros(5, dtype=np.int32)
+        A = np.zeros(1, dtype=np.uint64)
+        card = np.zeros(2, dtype=np.uint64)
+        off = np.zeros(2, dtype=np.uint64)
+        vals = np.zeros(24, dtype=np.int32)
+        mults = np.zeros(24, dtype=np.int32)
+        p = lambda a: a.ctypes.data_as(ctypes.c_void_p)
+        _check("llvq_class_info", self._lib.llvq_class_info(self._h, j, p(info), p(A), p(card), p(off), p(vals), p(mults)))
+        nv = int(info[4])
+        return {"m": int(info[0]), "parity": int(info[1]), "w": int(info[2]), "B": int(info[3]), "A": int(A[0]),
+                "card": (int(card[1]) << 64) | int(card[0]), "offset": (int(off[1]) << 64) | int(off[0]),
+                "values": [int(v) for v in vals[:nv]], "mults": [int(v) for v in mults[:nv]]}
+
+    def golay_table(self):
+        import numpy as np
+        out = np.zeros(4096, dtype=np.uint32)
+        _check("llvq_golay_table", self._lib.llvq_golay_table(self._h, out.ctypes.data_as(ctypes.c_void_p)))
+        return out
+
+    def close(self) -> None:
+        if getattr(self, "_h", None):
+            self._lib.llvq_destroy(self._h)
+            self._h = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+
+def llvq_decode_blocks(ctx: Context, d_idx: torch.Tensor, nblocks: int, d_points: torch.Tensor | None = None, stream=None):
+    """int8 [nblocks, 24] lattice points of the fields of the index stream ``d_idx`` (uint8, CUDA)."""
+    if d_points is None:
+        d_points = torch.empty((nblocks, 24), dtype=torch.int8, device=d_idx.device)
+    assert d_points.dtype == torch.int8 and d_points.numel() >= nblocks * 24
+    assert d_idx.numel() * d_idx.element_size() >= ctx.index_bytes(nblocks)
+    _check("llvq_decode_blocks", ctx._lib.llvq_decode_blocks(ctx._h, _dev(d_idx, "d_idx"), nblocks, _dev(d_points, "d_points"), _stream_ptr(stream)))
+    return d_points
+
+
+def llvq_dequant_matrix(ctx: Context, d_idx: torch.Tensor, d_gain: torch.Tensor, rows: int, cols: int, layout: int,
+                        d_w: torch.Tensor | None = None, ld: int | None = None, stream=None):
+    """bf16 [rows, cols] dequantized weights; ``d_gain`` is float16 [nblocks]."""
+    ld = cols if ld is None else ld
+    if d_w is None:
+        d_w = torch.empty((rows, ld), dtype=torch.bfloat16, device=d_idx.device)
+    assert d_w.dtype == torch.bfloat16 and d_gain.dtype == torch.float16
+    nblocks = (rows * cols + 23) // 24 if layout == LLVQ_LAYOUT_FLAT else rows * ((cols + 23) // 24)
+    assert d_gain.numel() >= nblocks and d_idx.numel() * d_idx.element_size() >= ctx.index_bytes(nblocks)
+    assert d_w.numel() >= (rows - 1) * ld + cols if rows else True
+    _check("llvq_dequant_matrix", ctx._lib.llvq_dequant_matrix(
+        ctx._h, _dev(d_idx, "d_idx"), _dev(d_gain, "d_gain"), rows, cols, layout, _dev(d_w, "d_w"), ld, _stream_ptr(stream)))
+    return d_w
+
+
+def llvq_gemv(ctx: Context, d_idx: torch.Tensor, d_gain: torch.Tensor, n_out: int, k_in: int, d_x: torch.Tensor,
+              d_y: torch.Tensor | None = None, y_dtype: torch.dtype = torch.float32, stream=None):
+    """y = W x with W given by (index stream, gains), ROWWISE blocks; x bf16 [k_in]; y float32 or bf16 [n_out]."""
+    if d_y is None:
+        d_y = torch.empty(n_out, dtype=y_dtype, device=d_idx.device)
+    assert d_x.dtype == torch.bfloat16 and d_x.numel() >= k_in and d_gain.dtype == torch.float16
+    assert d_y.dtype in (torch.float32, torch.bfloat16) and d_y.numel() >= n_out
+    nblocks = n_out * ((k_in + 23) // 24)
+    assert d_gain.numel() >= nblocks and d_idx.numel() * d_idx.element_size() >= ctx.index_bytes(nblocks)
+    code = LLVQ_F32 if d_y.dtype == torch.float32 else LLVQ_BF16
+    _check("llvq_gemv", ctx._lib.llvq_gemv(ctx._h, _dev(d_idx, "d_idx"), _dev(d_gain, "d_gain"), n_out, k_in,
+                                           _dev(d_x, "d_x"), _dev(d_y, "d_y"), code, _stream_ptr(stream)))
+    return d_y
+
+
+def llvq_gemm_small_batch(ctx: Context, d_idx: torch.Tensor, d_gain: torch.Tensor, n_out: int, k_in: int,
+                          d_x: torch.Tensor, d_y: torch.Tensor | None = None, stream=None):
+    """Y[b, i] = sum_k X[b, k] W[i, k]; X bf16 [batch, k_in], Y bf16 [batch, n_out], batch <= 64."""
+    assert d_x.dtype == torch.bfloat16 and d_x.dim() == 2 and d_x.shape[1] == k_in and d_gain.dtype == torch.float16
+    batch = d_x.shape[0]
+    if d_y is None:
+        d_y = torch.empty((batch, n_out), dtype=torch.bfloat16, device=d_idx.device)
+    assert d_y.dtype == torch.bfloat16 and d_y.numel() >= batch * n_out
+    nblocks = n_out * ((k_in + 23) // 24)
+    assert d_gain.numel() >= nblocks and d_idx.numel() * d_idx.element_size() >= ctx.index_bytes(nblocks)
+    _check("llvq_gemm_small_batch", ctx._lib.llvq_gemm_small_batch(
+        ctx._h, _dev(d_idx, "d_idx"), _dev(d_gain, "d_gain"), n_out, k_in, _dev(d_x, "d_x"), batch, _dev(d_y, "d_y"), _stream_ptr(stream)))
+    return d_y
+
+
+def llvq_last_error(ctx: Context, stream=None) -> tuple[int, int]:
+    """(number of out-of-range fields since the last call, error flags); synchronises the stream."""
+    n = ctypes.c_uint64(0)
+    f = ctypes.c_uint32(0)
+    _check("llvq_last_error", ctx._lib.llvq_last_error(ctx._h, _stream_ptr(stream), ctypes.byref(n), ctypes.byref(f)))
+    return int(n.value), int(f.value)

@@ -1,0 +1,391 @@
+// C ABI and kernels of the LLVQ dequantization library (see include/llvq.h).
+#include "llvq.h"
+
+#include <cuda_runtime.h>
+
+#include <cstdio>
+#include <cstring>
+#include <new>
+#include <vector>
+
+#include "decode.cuh"
+#include "tables.h"
+
+using namespace llvq;
+
+struct llvq_ctx {
+    int device = 0;
+    HostTables host;
+    DevCode dev{};
+    void* d_blob = nullptr;          // one allocation holding every device table
+    unsigned long long* d_err = nullptr;
+    int sm_count = 0;
+};
+
+namespace {
+
+constexpr int kThreads = 256;
+
+struct DeviceGuard {
+    int prev = -1; bool ok = false;
+    explicit DeviceGuard(int dev) {
+        if (cudaGetDevice(&prev) != cudaSuccess) return;
+        ok = (prev == dev) || cudaSetDevice(dev) == cudaSuccess;
+    }
+    ~DeviceGuard() { if (ok && prev >= 0) cudaSetDevice(prev); }
+};
+
+inline bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) & (a - 1)) == 0; }
+
+// ---------------------------------------------------------------------------
+// llvq_decode_blocks: one thread per field; the 24 bytes of a point are staged
+// through shared memory so that the stores to global memory are coalesced.
+// ---------------------------------------------------------------------------
+__global__ void __launch_bounds__(kThreads)
+decode_blocks_kernel(DevCode dc, const uint32_t* __restrict__ stream, uint64_t nblocks, uint32_t* __restrict__ out)
+{
+    __shared__ uint32_t stage[kThreads * 6];
+    const uint64_t base = (uint64_t)blockIdx.x * kThreads;
+    const uint64_t b = base + threadIdx.x;
+    Point pt;
+    if (b < nblocks) {
+        decode_field(dc, stream, b, pt);
+#pragma unroll
+        for (int i = 0; i < 6; ++i) stage[threadIdx.x * 6 + i] = pt.w[i];
+    }
+    __syncthreads();
+    const uint64_t nvalid = min((uint64_t)kThreads, nblocks - base) * 6;
+    for (uint32_t i = threadIdx.x; i < nvalid; i += kThreads) out[base * 6 + i] = stage[i];
+}
+
+// ---------------------------------------------------------------------------
+// llvq_dequant_matrix
+// ---------------------------------------------------------------------------
+// FLAT layout: block b -> elements 24b..24b+23 of the flattened matrix.
+__global__ void __launch_bounds__(kThreads)
+dequant_flat_kernel(DevCode dc, const uint32_t* __restrict__ stream, const uint16_t* __restrict__ gain,
+                    uint64_t nblocks, uint64_t total, __nv_bfloat16* __restrict__ out, int vec_ok)
+{
+    __shared__ uint32_t stage[kThreads * 12];
+    const uint64_t base = (uint64_t)blockIdx.x * kThreads;
+    const uint64_t b = base + threadIdx.x;
+    if (b < nblocks) {
+        Point pt;
+        decode_field(dc, stream, b, pt);
+        const float g = gain_to_float(__ldg(gain + b));
+#pragma unroll
+        for (int j = 0; j < 12; ++j) {
+            __nv_bfloat162 v = __halves2bfloat162(dequant(g, pt, 2 * j), dequant(g, pt, 2 * j + 1));
+            stage[threadIdx.x * 12 + j] = *reinterpret_cast<uint32_t*>(&v);
+        }
+    }
+    __syncthreads();
+    const uint64_t first = base * 24;                          // first element of this CTA
+    const uint64_t count = min((uint64_t)kThreads * 24, total - first);
+    if (vec_ok && count == (uint64_t)kThreads * 24) {
+        uint4* dst = reinterpret_cast<uint4*>(out + first);    // first*2 bytes = base*48: 16-byte aligned
+        const uint4* src = reinterpret_cast<const uint4*>(stage);
+        for (uint32_t i = threadIdx.x; i < kThreads * 3; i += kThreads) dst[i] = src[i];
+    } else {
+        const __nv_bfloat16* src = reinterpret_cast<const __nv_bfloat16*>(stage);
+        for (uint64_t i = threadIdx.x; i < count; i += kThreads) out[first + i] = src[i];
+    }
+}
+
+// ROWWISE layout: block (r, cb) -> columns 24cb..24cb+23 of row r; leading dimension ld.
+__global__ void __launch_bounds__(kThreads)
+dequant_rowwise_kernel(DevCode dc, const uint32_t* __restrict__ stream, const uint16_t* __restrict__ gain,
+                       int64_t rows, int64_t cols, int64_t bpr, __nv_bfloat16* __restrict__ out, int64_t ld)
+{
+    const uint64_t b = (uint64_t)blockIdx.x * kThreads + threadIdx.x;
+    if (b >= (uint64_t)(rows * bpr)) return;
+    const int64_t r = (int64_t)(b / (uint64_t)bpr), cb = (int64_t)(b % (uint64_t)bpr);
+    Point pt;
+    decode_field(dc, stream, b, pt);
+    const float g = gain_to_float(__ldg(gain + b));
+    __nv_bfloat16* dst = out + r * ld + cb * 24;
+    const int64_t left = cols - cb * 24;
+    if (left >= 24 && (reinterpret_cast<uintptr_t>(dst) & 15) == 0) {
+        uint32_t v[12];
+#pragma unroll
+        for (int j = 0; j < 12; ++j) {
+            __nv_bfloat162 h = __halves2bfloat162(dequant(g, pt, 2 * j), dequant(g, pt, 2 * j + 1));
+            v[j] = *reinterpret_cast<uint32_t*>(&h);
+        }
+        uint4* d4 = reinterpret_cast<uint4*>(dst);
+        d4[0] = make_uint4(v[0], v[1], v[2], v[3]);
+        d4[1] = make_uint4(v[4], v[5], v[6], v[7]);
+        d4[2] = make_uint4(v[8], v[9], v[10], v[11]);
+    } else {
+#pragma unroll
+        for (int j = 0; j < 24; ++j)
+            if (j < left) dst[j] = dequant(g, pt, j);
+    }
+}
+
+// ---------------------------------------------------------------------------
+// llvq_gemv: one warp per output row; lanes stride over the row's blocks; x is
+// staged in shared memory as binary32, 25 words per block of 24 to keep the
+// lanes of a warp on distinct banks.
+// ---------------------------------------------------------------------------
+constexpr int kGemvWarps = 8;
+
+template <bool kOutBf16>
+__global__ void __launch_bounds__(kGemvWarps * 32)
+gemv_kernel(DevCode dc, const uint32_t* __restrict__ stream, const uint16_t* __restrict__ gain,
+            int64_t n_out, int64_t k_in, int64_t bpr, const uint16_t* __restrict__ x, void* __restrict__ y)
+{
+    extern __shared__ float xs[];                              // [bpr][25]
+    for (int64_t i = threadIdx.x; i < bpr * 24; i += blockDim.x) {
+        float v = 0.f;
+        if (i < k_in) v = __bfloat162float(__ushort_as_bfloat16(__ldg(x + i)));
+        xs[(i / 24) * 25 + (i % 24)] = v;
+    }
+    __syncthreads();
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int64_t row = (int64_t)blockIdx.x * kGemvWarps + warp;
+    if (row >= n_out) return;
+    float acc = 0.f;
+    for (int64_t cb = lane; cb < bpr; cb += 32) {
+        const uint64_t b = (uint64_t)(row * bpr + cb);
+        Point pt;
+        decode_field(dc, stream, b, pt);
+        const float g = gain_to_float(__ldg(gain + b));
+        const float* xb = xs + cb * 25;
+        float part = 0.f;
+#pragma unroll
+        for (int j = 0; j < 24; ++j) part = fmaf(__bfloat162float(dequant(g, pt, j)), xb[j], part);
+        acc += part;
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
+    if (lane == 0) {
+        if (kOutBf16) reinterpret_cast<__nv_bfloat16*>(y)[row] = __float2bfloat16_rn(acc);
+        else reinterpret_cast<float*>(y)[row] = acc;
+    }
+}
+
+int check_common(const llvq_ctx* ctx, const void* d_idx)
+{
+    if (!ctx || !d_idx || ctx->device < 0) return LLVQ_EINVAL;
+    if (!aligned(d_idx, 16)) return LLVQ_EALIGN;
+    return LLVQ_OK;
+}
+
+int launch_status()
+{
+    return cudaGetLastError() == cudaSuccess ? LLVQ_OK : LLVQ_ECUDA;
+}
+
+}  // namespace
+
+extern "C" {
+
+int llvq_create(llvq_ctx** out, int m_lo, int m_hi, int device)
+{
+    if (!out) return LLVQ_EINVAL;
+    *out = nullptr;
+    llvq_ctx* ctx = new (std::nothrow) llvq_ctx();
+    if (!ctx) return LLVQ_ECUDA;
+    if (!build_tables(m_lo, m_hi, ctx->host)) { delete ctx; return LLVQ_EUNSUPPORTED; }
+    ctx->device = device;
+    if (device < 0) { *out = ctx; return LLVQ_OK; }      // host-only context: table queries, no kernels
+    DeviceGuard guard(device);
+    if (!guard.ok) { delete ctx; return LLVQ_ECUDA; }
+    cudaDeviceProp prop;
+    if (cudaGetDeviceProperties(&prop, device) != cudaSuccess) { delete ctx; return LLVQ_ECUDA; }
+    ctx->sm_count = prop.multiProcessorCount;
+
+    const HostTables& h = ctx->host;
+    const size_t ncls = h.desc.size();
+    std::vector<uint64_t> off_lo(ncls + 1);
+    std::vector<uint32_t> off_hi(ncls + 1);
+    for (size_t j = 0; j <= ncls; ++j) { off_lo[j] = (uint64_t)h.offset[j]; off_hi[j] = (uint32_t)(h.offset[j] >> 64); }
+
+    // one blob: [golay | pascal | off_hi | off_lo | classes | error words], each part 256-byte aligned
+    auto up = [](size_t v) { return (v + 255) & ~size_t(255); };
+    size_t o_golay = 0;
+    size_t o_pascal = up(o_golay + 4096 * 4);
+    size_t o_offhi = up(o_pascal + sizeof(h.pascal));
+    size_t o_offlo = up(o_offhi + (ncls + 1) * 4);
+    size_t o_cls = up(o_offlo + (ncls + 1) * 8);
+    size_t o_err = up(o_cls + ncls * sizeof(ClassDesc));
+    size_t total = o_err + 256;
+    std::vector<uint8_t> blob(total, 0);
+    std::memcpy(blob.data() + o_golay, h.golay.data(), 4096 * 4);
+    std::memcpy(blob.data() + o_pascal, h.pascal, sizeof(h.pascal));
+    std::memcpy(blob.data() + o_offhi, off_hi.data(), (ncls + 1) * 4);
+    std::memcpy(blob.data() + o_offlo, off_lo.data(), (ncls + 1) * 8);
+    std::memcpy(blob.data() + o_cls, h.desc.data(), ncls * sizeof(ClassDesc));
+    if (cudaMalloc(&ctx->d_blob, total) != cudaSuccess) { delete ctx; return LLVQ_ECUDA; }
+    if (cudaMemcpy(ctx->d_blob, blob.data(), total, cudaMemcpyHostToDevice) != cudaSuccess) {
+        cudaFree(ctx->d_blob); delete ctx; return LLVQ_ECUDA;
+    }
+    uint8_t* d = static_cast<uint8_t*>(ctx->d_blob);
+    ctx->dev.golay = reinterpret_cast<const uint32_t*>(d + o_golay);
+    ctx->dev.pascal = reinterpret_cast<const uint32_t*>(d + o_pascal);
+    ctx->dev.off_hi = reinterpret_cast<const uint32_t*>(d + o_offhi);
+    ctx->dev.off_lo = reinterpret_cast<const uint64_t*>(d + o_offlo);
+    ctx->dev.cls = reinterpret_cast<const ClassDesc*>(d + o_cls);
+    ctx->d_err = reinterpret_cast<unsigned long long*>(d + o_err);
+    ctx->dev.bad_index = ctx->d_err;
+    ctx->dev.flags = reinterpret_cast<uint32_t*>(d + o_err + 8);
+    ctx->dev.n_lo = (uint64_t)h.N; ctx->dev.n_hi = (uint64_t)(h.N >> 64);
+    ctx->dev.nclasses = (int)ncls;
+    ctx->dev.W = h.W;
+    *out = ctx;
+    return LLVQ_OK;
+}
+
+void llvq_destroy(llvq_ctx* ctx)
+{
+    if (!ctx) return;
+    if (ctx->d_blob) {
+        DeviceGuard guard(ctx->device);
+        cudaFree(ctx->d_blob);
+    }
+    delete ctx;
+}
+
+int llvq_index_bits(const llvq_ctx* ctx) { return ctx ? ctx->host.W : -1; }
+
+int llvq_num_points(const llvq_ctx* ctx, uint64_t lo_hi[2])
+{
+    if (!ctx || !lo_hi) return LLVQ_EINVAL;
+    lo_hi[0] = (uint64_t)ctx->host.N; lo_hi[1] = (uint64_t)(ctx->host.N >> 64);
+    return LLVQ_OK;
+}
+
+int llvq_num_classes(const llvq_ctx* ctx) { return ctx ? (int)ctx->host.desc.size() : -1; }
+
+size_t llvq_index_bytes(const llvq_ctx* ctx, uint64_t nblocks)
+{
+    if (!ctx) return 0;
+    unsigned __int128 bits = (unsigned __int128)nblocks * (unsigned)ctx->host.W;
+    unsigned __int128 bytes = (bits + 7) / 8;
+    return (size_t)((bytes + 15) / 16 * 16);
+}
+
+// Host-only: description of class j (for tests of the table generator).
+// info = {m, parity, w, B, nvalues}; values/mults hold up to 24 entries.
+int llvq_class_info(const llvq_ctx* ctx, int j, int info[5], uint64_t* A, uint64_t card[2], uint64_t offset[2],
+                    int values[24], int mults[24])
+{
+    if (!ctx || j < 0 || j >= (int)ctx->host.info.size() || !info || !A || !card || !offset || !values || !mults) return LLVQ_EINVAL;
+    const ClassInfo& c = ctx->host.info[j];
+    info[0] = c.m; info[1] = c.parity; info[2] = c.w; info[3] = c.B; info[4] = (int)c.values.size();
+    *A = c.A;
+    card[0] = (uint64_t)c.card; card[1] = (uint64_t)(c.card >> 64);
+    offset[0] = (uint64_t)c.offset; offset[1] = (uint64_t)(c.offset >> 64);
+    for (size_t i = 0; i < c.values.size(); ++i) { values[i] = c.values[i]; mults[i] = c.mults[i]; }
+    return LLVQ_OK;
+}
+
+// Host-only: copy of the sorted Golay table (4096 words).
+int llvq_golay_table(const llvq_ctx* ctx, uint32_t out[4096])
+{
+    if (!ctx || !out) return LLVQ_EINVAL;
+    std::memcpy(out, ctx->host.golay.data(), 4096 * 4);
+    return LLVQ_OK;
+}
+
+int llvq_decode_blocks(const llvq_ctx* ctx, const void* d_idx, uint64_t nblocks, int8_t* d_points, void* stream)
+{
+    if (int e = check_common(ctx, d_idx)) return e;
+    if (!d_points) return LLVQ_EINVAL;
+    if (!aligned(d_points, 4)) return LLVQ_EALIGN;
+    if (nblocks == 0) return LLVQ_OK;
+    if (nblocks > (1ull << 40)) return LLVQ_EUNSUPPORTED;
+    DeviceGuard guard(ctx->device);
+    if (!guard.ok) return LLVQ_ECUDA;
+    uint64_t grid = (nblocks + kThreads - 1) / kThreads;
+    if (grid > 0x7fffffffull) return LLVQ_EUNSUPPORTED;
+    decode_blocks_kernel<<<(unsigned)grid, kThreads, 0, (cudaStream_t)stream>>>(
+        ctx->dev, static_cast<const uint32_t*>(d_idx), nblocks, reinterpret_cast<uint32_t*>(d_points));
+    return launch_status();
+}
+
+int llvq_dequant_matrix(const llvq_ctx* ctx, const void* d_idx, const uint16_t* d_gain_f16,
+                        int64_t rows, int64_t cols, int layout, uint16_t* d_w_bf16, int64_t ld, void* stream)
+{
+    if (int e = check_common(ctx, d_idx)) return e;
+    if (!d_gain_f16 || !d_w_bf16 || rows < 0 || cols < 0 || ld < cols) return LLVQ_EINVAL;
+    if (layout != LLVQ_LAYOUT_FLAT && layout != LLVQ_LAYOUT_ROWWISE) return LLVQ_EINVAL;
+    if (!aligned(d_gain_f16, 2) || !aligned(d_w_bf16, 2)) return LLVQ_EALIGN;
+    if (rows == 0 || cols == 0) return LLVQ_OK;
+    if (rows > (1ll << 31) || cols > (1ll << 31)) return LLVQ_EUNSUPPORTED;
+    DeviceGuard guard(ctx->device);
+    if (!guard.ok) return LLVQ_ECUDA;
+    cudaStream_t st = (cudaStream_t)stream;
+    if (layout == LLVQ_LAYOUT_FLAT) {
+        if (ld != cols) return LLVQ_EINVAL;
+        uint64_t total = (uint64_t)rows * (uint64_t)cols, nblocks = (total + 23) / 24;
+        uint64_t grid = (nblocks + kThreads - 1) / kThreads;
+        if (grid > 0x7fffffffull) return LLVQ_EUNSUPPORTED;
+        dequant_flat_kernel<<<(unsigned)grid, kThreads, 0, st>>>(
+            ctx->dev, static_cast<const uint32_t*>(d_idx), d_gain_f16, nblocks, total,
+            reinterpret_cast<__nv_bfloat16*>(d_w_bf16), aligned(d_w_bf16, 16) ? 1 : 0);
+    } else {
+        int64_t bpr = (cols + 23) / 24;
+        uint64_t nblocks = (uint64_t)rows * (uint64_t)bpr;
+        uint64_t grid = (nblocks + kThreads - 1) / kThreads;
+        if (grid > 0x7fffffffull) return LLVQ_EUNSUPPORTED;
+        dequant_rowwise_kernel<<<(unsigned)grid, kThreads, 0, st>>>(
+            ctx->dev, static_cast<const uint32_t*>(d_idx), d_gain_f16, rows, cols, bpr,
+            reinterpret_cast<__nv_bfloat16*>(d_w_bf16), ld);
+    }
+    return launch_status();
+}
+
+int llvq_gemv(const llvq_ctx* ctx, const void* d_idx, const uint16_t* d_gain_f16, int64_t n_out, int64_t k_in,
+              const uint16_t* d_x_bf16, void* d_y, int y_dtype, void* stream)
+{
+    if (int e = check_common(ctx, d_idx)) return e;
+    if (!d_gain_f16 || !d_x_bf16 || !d_y || n_out < 0 || k_in < 0) return LLVQ_EINVAL;
+    if (y_dtype != LLVQ_F32 && y_dtype != LLVQ_BF16) return LLVQ_EINVAL;
+    if (!aligned(d_gain_f16, 2) || !aligned(d_x_bf16, 2) || !aligned(d_y, y_dtype == LLVQ_F32 ? 4 : 2)) return LLVQ_EALIGN;
+    if (n_out == 0) return LLVQ_OK;
+    DeviceGuard guard(ctx->device);
+    if (!guard.ok) return LLVQ_ECUDA;
+    cudaStream_t st = (cudaStream_t)stream;
+    if (k_in == 0) {
+        return cudaMemsetAsync(d_y, 0, (size_t)n_out * (y_dtype == LLVQ_F32 ? 4 : 2), st) == cudaSuccess ? LLVQ_OK : LLVQ_ECUDA;
+    }
+    int64_t bpr = (k_in + 23) / 24;
+    size_t smem = (size_t)bpr * 25 * sizeof(float);
+    if (smem > 200 * 1024 || n_out > (1ll << 31)) return LLVQ_EUNSUPPORTED;
+    unsigned grid = (unsigned)((n_out + kGemvWarps - 1) / kGemvWarps);
+    const uint32_t* idx = static_cast<const uint32_t*>(d_idx);
+    if (y_dtype == LLVQ_BF16) {
+        if (cudaFuncSetAttribute(gemv_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return LLVQ_ECUDA;
+        gemv_kernel<true><<<grid, kGemvWarps * 32, smem, st>>>(ctx->dev, idx, d_gain_f16, n_out, k_in, bpr, d_x_bf16, d_y);
+    } else {
+        if (cudaFuncSetAttribute(gemv_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return LLVQ_ECUDA;
+        gemv_kernel<false><<<grid, kGemvWarps * 32, smem, st>>>(ctx->dev, idx, d_gain_f16, n_out, k_in, bpr, d_x_bf16, d_y);
+    }
+    return launch_status();
+}
+
+int llvq_gemm_small_batch(const llvq_ctx* ctx, const void* d_idx, const uint16_t* d_gain_f16, int64_t n_out, int64_t k_in,
+                          const uint16_t* d_x_bf16, int batch, uint16_t* d_y_bf16, void* stream)
+{
+    (void)ctx; (void)d_idx; (void)d_gain_f16; (void)n_out; (void)k_in; (void)d_x_bf16; (void)batch; (void)d_y_bf16; (void)stream;
+    return LLVQ_EUNSUPPORTED;
+}
+
+int llvq_last_error(llvq_ctx* ctx, void* stream, uint64_t* n_bad_index, uint32_t* flags)
+{
+    if (!ctx || ctx->device < 0) return LLVQ_EINVAL;
+    DeviceGuard guard(ctx->device);
+    if (!guard.ok) return LLVQ_ECUDA;
+    cudaStream_t st = (cudaStream_t)stream;
+    unsigned long long host[2] = {0, 0};
+    if (cudaMemcpyAsync(host, ctx->d_err, 16, cudaMemcpyDeviceToHost, st) != cudaSuccess) return LLVQ_ECUDA;
+    if (cudaMemsetAsync(ctx->d_err, 0, 16, st) != cudaSuccess) return LLVQ_ECUDA;
+    if (cudaStreamSynchronize(st) != cudaSuccess) return LLVQ_ECUDA;
+    if (n_bad_index) *n_bad_index = host[0];
+    if (flags) *flags = (uint32_t)host[1];
+    return LLVQ_OK;
+}
+
+}  // extern "C"

@@ -1,0 +1,209 @@
+// Host-side table generator (see tables.h).
+#include "tables.h"
+
+#include <algorithm>
+#include <array>
+#include <cmath>
+#include <cstring>
+
+namespace llvq {
+namespace {
+
+inline int popc(uint32_t v) { return __builtin_popcount(v); }
+
+// Extended Golay code (Sec. 2.3).  Basis: the 12 shifts of the generator
+// polynomial x^11+x^10+x^6+x^5+x^4+x^2+1 of the cyclic [23,12,7] code, each
+// extended by an overall parity bit at coordinate 23; all 4096 sums are walked
+// in Gray-code order.
+void make_golay(HostTables& t)
+{
+    uint32_t basis[12];
+    for (int i = 0; i < 12; ++i) {
+        uint32_t row = 0xC75u << i;
+        if (popc(row) & 1) row |= 1u << 23;
+        basis[i] = row;
+    }
+    t.golay.resize(4096);
+    uint32_t word = 0;
+    t.golay[0] = 0;
+    for (uint32_t g = 1; g < 4096; ++g) {
+        word ^= basis[__builtin_ctz(g)];     // Gray code: flip one basis vector per step
+        t.golay[g] = word;
+    }
+    std::sort(t.golay.begin(), t.golay.end(), [](uint32_t a, uint32_t b) {
+        int wa = popc(a), wb = popc(b);
+        return wa != wb ? wa < wb : a < b;
+    });
+    for (uint32_t c : t.golay) t.wcnt[popc(c)]++;
+    int acc = 0;
+    for (int w = 0; w <= 24; ++w) { t.woff[w] = acc; acc += t.wcnt[w]; }
+}
+
+void make_pascal(HostTables& t)
+{
+    for (int n = 0; n < 25; ++n) {
+        t.pascal[n * 25] = 1;
+        for (int k = 1; k <= n; ++k)
+            t.pascal[n * 25 + k] = (n ? t.pascal[(n - 1) * 25 + k - 1] : 0) + (k <= n - 1 ? t.pascal[(n - 1) * 25 + k] : 0);
+    }
+}
+
+struct Multiset {
+    int parity;
+    std::array<int, 32> cnt;     // cnt[v] = multiplicity of absolute value v
+};
+
+// All multisets of 24 values of one parity with squared norm `norm`,
+// generated from the smallest value upwards.
+void gen_multisets(int parity, int v, int left, int norm, Multiset& cur, std::vector<Multiset>& out)
+{
+    if (left == 0) { if (norm == 0) out.push_back(cur); return; }
+    if (v * v * left > norm && v > 0) return;      // even the smallest remaining value overshoots
+    if (v > 31 || v * v > norm) return;
+    int maxc = v == 0 ? left : std::min(left, norm / (v * v));
+    for (int c = maxc; c >= 0; --c) {
+        cur.cnt[v] = c;
+        gen_multisets(parity, v + 2, left - c, norm - c * v * v, cur, out);
+    }
+    cur.cnt[v] = 0;
+}
+
+u128 choose(const HostTables& t, int n, int k) { return (k < 0 || k > n) ? 0 : (u128)t.pascal[n * 25 + k]; }
+
+bool admissible(const Multiset& s, int& w)
+{
+    int n2 = 0, n4 = 0, n35 = 0;
+    for (int v = 0; v < 32; ++v) {
+        if (v % 4 == 2) n2 += s.cnt[v];
+        if (v % 8 == 4) n4 += s.cnt[v];
+        if (v % 8 == 3 || v % 8 == 5) n35 += s.cnt[v];
+    }
+    if (s.parity) { w = 0; return (n35 % 2) == 1; }            // coordinate sum = 4 mod 8
+    w = n2;
+    if (!(w == 0 || w == 8 || w == 12 || w == 16 || w == 24)) return false;
+    return w != 0 || n4 % 2 == 0;                              // coordinate sum = 0 mod 8
+}
+
+std::array<int, 24> leader(const ClassInfo& c)
+{
+    std::array<int, 24> l{};
+    int p = 0;
+    for (size_t i = 0; i < c.values.size(); ++i)
+        for (int j = 0; j < c.mults[i]; ++j) l[p++] = c.values[i];
+    return l;
+}
+
+// Fixed class order inside a shell (Sec. 3.2 (2)): even classes by ascending
+// Golay weight then ascending leader; then odd classes by descending leader.
+bool class_before(const ClassInfo& a, const ClassInfo& b)
+{
+    if (a.parity != b.parity) return a.parity < b.parity;
+    auto la = leader(a), lb = leader(b);
+    if (a.parity == 0) {
+        if (a.w != b.w) return a.w < b.w;
+        return la < lb;
+    }
+    return la > lb;
+}
+
+bool fill_descriptor(const HostTables& t, const ClassInfo& c, ClassDesc& d, int& nlev)
+{
+    std::memset(&d, 0, sizeof d);
+    d.parity = (uint8_t)c.parity; d.w = (uint8_t)c.w; d.B = (uint8_t)c.B; d.m = (uint32_t)c.m;
+    d.A = (uint16_t)c.A;
+    d.goff = (uint16_t)(c.parity ? 0 : t.woff[c.w]);
+    d.magicA = ~0ull / c.A;
+    int n46 = 0;
+    for (size_t i = 0; i < c.values.size(); ++i)
+        if (c.values[i] % 8 == 4 || c.values[i] % 8 == 6) n46 += c.mults[i];
+    d.signpar = (uint8_t)(n46 & 1);
+    nlev = 0;
+    for (int group = 1; group >= 0; --group) {
+        std::vector<int> gv, gm;
+        for (size_t i = 0; i < c.values.size(); ++i) {
+            bool in1 = !c.parity && c.values[i] % 4 == 2;
+            if ((group == 1) == in1) { gv.push_back(c.values[i]); gm.push_back(c.mults[i]); }
+        }
+        int n = group == 1 ? c.w : 24 - c.w;
+        if (c.parity) n = group == 1 ? 0 : 24;
+        int steps = 0;
+        for (size_t i = 0; i + 1 < gv.size(); ++i) {
+            if (nlev >= kMaxLevels) return false;
+            LevelDesc& l = d.lev[nlev++];
+            l.radix = t.pascal[n * 25 + gm[i]];
+            l.k = (uint8_t)gm[i]; l.val = (uint8_t)gv[i]; l.n = (uint8_t)n; l.pad = 0;
+            l.magic = ~0ull / l.radix;
+            n -= gm[i];
+            ++steps;
+        }
+        uint8_t fill = gv.empty() ? 0 : (uint8_t)gv.back();
+        if (group == 1) { d.nlev1 = (uint8_t)steps; d.fill1 = fill; }
+        else            { d.nlev0 = (uint8_t)steps; d.fill0 = fill; }
+    }
+    return true;
+}
+
+}  // namespace
+
+bool build_tables(int m_lo, int m_hi, HostTables& t)
+{
+    if (m_lo < 2 || m_hi < m_lo || m_hi > 53) return false;
+    t = HostTables();
+    t.m_lo = m_lo; t.m_hi = m_hi;
+    make_golay(t);
+    make_pascal(t);
+    u128 running = 0;
+    for (int m = m_lo; m <= m_hi; ++m) {
+        std::vector<ClassInfo> shell;
+        for (int parity = 0; parity <= 1; ++parity) {
+            std::vector<Multiset> sets;
+            Multiset cur; cur.parity = parity; cur.cnt.fill(0);
+            gen_multisets(parity, parity, 24, 16 * m, cur, sets);
+            for (const Multiset& s : sets) {
+                int w;
+                if (!admissible(s, w)) continue;
+                ClassInfo c;
+                c.m = m; c.parity = parity; c.w = w;
+                for (int v = 31; v >= 0; --v)
+                    if (s.cnt[v]) { c.values.push_back(v); c.mults.push_back(s.cnt[v]); }
+                // cardinality A * 2^B * P (Sec. 2.5)
+                u128 P = 1;
+                if (parity) {
+                    c.A = 4096; c.B = 0;
+                    int left = 24;
+                    for (int k : c.mults) { P *= choose(t, left, k); left -= k; }
+                } else {
+                    c.A = (uint64_t)t.wcnt[w];
+                    int left1 = w, left0 = 24 - w, nz0 = 0;
+                    for (size_t i = 0; i < c.values.size(); ++i) {
+                        if (c.values[i] % 4 == 2) { P *= choose(t, left1, c.mults[i]); left1 -= c.mults[i]; }
+                        else { P *= choose(t, left0, c.mults[i]); left0 -= c.mults[i]; if (c.values[i]) nz0 += c.mults[i]; }
+                    }
+                    c.B = nz0 + (w > 0 ? w - 1 : 0);
+                }
+                c.card = (u128)c.A * ((u128)1 << c.B) * P;
+                c.offset = 0;
+                shell.push_back(c);
+            }
+        }
+        std::sort(shell.begin(), shell.end(), class_before);
+        for (ClassInfo& c : shell) { c.offset = running; running += c.card; t.info.push_back(c); }
+    }
+    t.N = running;
+    t.W = 0;
+    while (t.W < 100 && ((u128)1 << t.W) < t.N) ++t.W;
+    if (t.W > 72) return false;
+    t.desc.resize(t.info.size());
+    t.offset.resize(t.info.size() + 1);
+    for (size_t j = 0; j < t.info.size(); ++j) {
+        int nlev;
+        if (!fill_descriptor(t, t.info[j], t.desc[j], nlev)) return false;
+        if (t.info[j].card >> 63) return false;          // class-local indices must fit 63 bits
+        t.max_levels = std::max(t.max_levels, nlev);
+        t.offset[j] = t.info[j].offset;
+    }
+    t.offset[t.info.size()] = t.N;
+    return true;
+}
+
+}  // namespace llvq

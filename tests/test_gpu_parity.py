@@ -1,0 +1,232 @@
+"""Parity of the CUDA library against the CPU oracle, through the C ABI.
+
+Integer work (lattice points, bf16 weights) must be bit-exact.  Fused products
+accumulate in binary32 and are compared with the oracle's binary64 result:
+max relative error <= 1e-3 with the denominator floored at 1e-3 * max|y|; bf16
+outputs are additionally allowed the half-ulp of their own rounding (2^-9).
+"""
+import numpy as np
+import pytest
+import torch
+
+import llvq_inputs as gen
+from gpu_util import bf16_bits, gemv_error, to_dev_bf16, to_dev_f16, to_dev_u8
+
+pytestmark = pytest.mark.gpu
+
+TOL = 1e-3
+TOL_BF16_OUT = 1e-3 + 2.0 ** -8
+
+
+@pytest.fixture(scope="module")
+def lib():
+    import paper_2603_11021_b200 as P
+    assert torch.cuda.is_available(), "these tests need a CUDA device; there is no CPU path"
+    return P
+
+
+@pytest.fixture(scope="module")
+def ctxs(lib):
+    return {code: lib.Context(*code, device=0) for code in [(2, 2), (3, 3), (2, 13), (2, 53)]}
+
+
+def _oracle(oracle_mod, cache={}):
+    def get(code):
+        if code not in cache:
+            cache[code] = oracle_mod.Code(*code)
+        return cache[code]
+    return get
+
+
+def _decode_gpu(lib, ctx, lo, hi):
+    stream = gen.pack_indices(lo, hi, ctx.index_bits)
+    assert stream.size == ctx.index_bytes(len(lo))
+    pts = lib.llvq_decode_blocks(ctx, to_dev_u8(stream), len(lo))
+    torch.cuda.synchronize()
+    return pts.cpu().numpy()
+
+
+def test_context_matches_oracle_tables(lib, ctxs, oracle_mod):
+    for code, ctx in ctxs.items():
+        o = _oracle(oracle_mod)(code)
+        assert (ctx.index_bits, ctx.num_points, ctx.num_classes) == (o.W, o.N, o.num_classes)
+
+
+def test_decode_exhaustive_minimal_shell(lib, ctxs, oracle_mod):
+    o = _oracle(oracle_mod)((2, 2))
+    lo = np.arange(o.N, dtype=np.uint64)
+    got = _decode_gpu(lib, ctxs[(2, 2)], lo, np.zeros_like(lo))
+    assert np.array_equal(got, o.unrank_arrays(lo, np.zeros_like(lo)))
+    assert lib.llvq_last_error(ctxs[(2, 2)]) == (0, 0)
+
+
+@pytest.mark.parametrize("code,nrand", [((2, 2), 8192), ((3, 3), 200003), ((2, 13), 300007), ((2, 53), 100001)])
+def test_decode_random_and_class_edges(lib, ctxs, oracle_mod, code, nrand):
+    o = _oracle(oracle_mod)(code)
+    ctx = ctxs[code]
+    lo, hi = gen.random_indices(o.N, o.W, nrand, seed=0)
+    edges = []
+    for k in o.classes():
+        edges += [k["offset"], k["offset"] + k["card"] - 1, k["offset"] + k["card"] // 2]
+    elo, ehi = gen.indices_to_arrays(edges)
+    lo, hi = np.concatenate([lo, elo]), np.concatenate([hi, ehi])
+    got = _decode_gpu(lib, ctx, lo, hi)
+    want = o.unrank_arrays(lo, hi)
+    bad = np.nonzero((got != want).any(axis=1))[0]
+    assert bad.size == 0, (bad[:5], got[bad[:2]], want[bad[:2]])
+    assert lib.llvq_last_error(ctx) == (0, 0)
+
+
+@pytest.mark.parametrize("code", [(2, 2), (2, 13), (2, 53)])
+def test_decode_out_of_range_fields_are_zero_and_counted(lib, ctxs, oracle_mod, code):
+    o = _oracle(oracle_mod)(code)
+    ctx = ctxs[code]
+    idx = [0, o.N, o.N - 1, (1 << o.W) - 1, o.N + 12345, 5]
+    lo, hi = gen.indices_to_arrays(idx)
+    got = _decode_gpu(lib, ctx, lo, hi)
+    want = o.unrank(idx)
+    assert np.array_equal(got, want)
+    assert not got[1].any() and not got[3].any() and got[2].any()
+    assert lib.llvq_last_error(ctx) == (3, 0)
+    assert lib.llvq_last_error(ctx) == (0, 0)          # cleared by the read
+
+
+def test_decode_empty_and_single(lib, ctxs, oracle_mod):
+    ctx = ctxs[(2, 13)]
+    o = _oracle(oracle_mod)((2, 13))
+    out = lib.llvq_decode_blocks(ctx, torch.zeros(16, dtype=torch.uint8, device="cuda"), 0)
+    assert out.shape == (0, 24)
+    lo, hi = gen.indices_to_arrays([o.N - 1])
+    assert np.array_equal(_decode_gpu(lib, ctx, lo, hi), o.unrank([o.N - 1]))
+
+
+@pytest.mark.parametrize("code,rows,cols,layout", [
+    ((2, 2), 256, 768, 1),           # config 1 shape
+    ((2, 13), 37, 1000, 0),          # FLAT, 37000 elements = 1541 blocks + 16 elements
+    ((2, 13), 301, 4096, 1),         # ROWWISE, 171 blocks per row, 8 pad lanes per row
+    ((2, 13), 64, 24, 1),
+    ((2, 13), 1, 7, 0),
+    ((2, 53), 129, 520, 1),
+    ((2, 53), 100, 333, 0),
+    ((3, 3), 50, 4104, 1),           # the shape of the paper's own kernel timing
+])
+def test_dequant_matrix_bit_exact(lib, ctxs, oracle_mod, code, rows, cols, layout):
+    o = _oracle(oracle_mod)(code)
+    ctx = ctxs[code]
+    stream, gain, nblocks = gen.make_layer(o.N, o.W, rows, cols, layout, seed=1)
+    want = o.dequant_matrix(stream, gain, rows, cols, layout)
+    got = lib.llvq_dequant_matrix(ctx, to_dev_u8(stream), to_dev_f16(gain), rows, cols, layout)
+    torch.cuda.synchronize()
+    assert np.array_equal(bf16_bits(got), want)
+    assert lib.llvq_last_error(ctx) == (0, 0)
+
+
+def test_dequant_matrix_leading_dimension_and_unaligned_rows(lib, ctxs, oracle_mod):
+    o = _oracle(oracle_mod)((2, 13))
+    ctx = ctxs[(2, 13)]
+    rows, cols, ld = 33, 100, 107                       # odd ld: rows start at 2-byte aligned addresses only
+    stream, gain, _ = gen.make_layer(o.N, o.W, rows, cols, 1, seed=2)
+    want = o.dequant_matrix(stream, gain, rows, cols, 1)
+    buf = torch.full((rows, ld), -7.0, dtype=torch.bfloat16, device="cuda")
+    lib.llvq_dequant_matrix(ctx, to_dev_u8(stream), to_dev_f16(gain), rows, cols, 1, d_w=buf, ld=ld)
+    torch.cuda.synchronize()
+    out = bf16_bits(buf)
+    assert np.array_equal(out[:, :cols], want)
+    assert (buf[:, cols:].float().cpu().numpy() == -7.0).all()      # padding untouched
+
+
+def test_dequant_signed_zero_and_special_gains(lib, ctxs, oracle_mod):
+    o = _oracle(oracle_mod)((2, 13))
+    ctx = ctxs[(2, 13)]
+    rows, cols = 16, 240
+    stream, gain, nblocks = gen.make_layer(o.N, o.W, rows, cols, 1, seed=3)
+    special = np.array([0x0000, 0x8000, 0x0001, 0x03FF, 0x0400, 0x7BFF, 0xFBFF, 0x3C00, 0xBC00, 0x3555], dtype=np.uint16)
+    gain[: special.size * 4] = np.tile(special, 4)
+    want = o.dequant_matrix(stream, gain, rows, cols, 1)
+    got = lib.llvq_dequant_matrix(ctx, to_dev_u8(stream), to_dev_f16(gain), rows, cols, 1)
+    torch.cuda.synchronize()
+    assert np.array_equal(bf16_bits(got), want)
+
+
+def test_gemv_config1_tiny(lib, ctxs, oracle_mod):
+    # 256 x 768, minimal shell only, 18-bit fields, fp32 output
+    o = _oracle(oracle_mod)((2, 2))
+    ctx = ctxs[(2, 2)]
+    n_out, k_in = 256, 768
+    stream, gain, nblocks = gen.make_layer(o.N, o.W, n_out, k_in, 1, seed=0)
+    assert nblocks == 8192
+    x = gen.normal_bf16(k_in, seed=0)
+    want = o.gemv(stream, gain, n_out, k_in, x)
+    got = lib.llvq_gemv(ctx, to_dev_u8(stream), to_dev_f16(gain), n_out, k_in, to_dev_bf16(x))
+    torch.cuda.synchronize()
+    assert gemv_error(got.cpu().numpy(), want) <= TOL
+
+
+@pytest.mark.parametrize("code,n_out,k_in", [((2, 13), 67, 4096), ((2, 13), 8, 24), ((2, 13), 129, 1000),
+                                             ((2, 53), 40, 2048), ((3, 3), 33, 4104)])
+def test_gemv_small_shapes_both_output_types(lib, ctxs, oracle_mod, code, n_out, k_in):
+    o = _oracle(oracle_mod)(code)
+    ctx = ctxs[code]
+    stream, gain, _ = gen.make_layer(o.N, o.W, n_out, k_in, 1, seed=4)
+    x = gen.normal_bf16(k_in, seed=4)
+    want = o.gemv(stream, gain, n_out, k_in, x)
+    d = (to_dev_u8(stream), to_dev_f16(gain))
+    y32 = lib.llvq_gemv(ctx, *d, n_out, k_in, to_dev_bf16(x))
+    y16 = lib.llvq_gemv(ctx, *d, n_out, k_in, to_dev_bf16(x), y_dtype=torch.bfloat16)
+    torch.cuda.synchronize()
+    assert gemv_error(y32.cpu().numpy(), want) <= TOL
+    assert gemv_error(y16.float().cpu().numpy(), want) <= TOL_BF16_OUT
+    # the bf16 output is the rounding of the fp32 one
+    assert torch.equal(y32.to(torch.bfloat16), y16)
+
+
+def test_gemv_exact_integer_cases(lib, ctxs, oracle_mod):
+    # gains = 1 and x = e_k / all-ones: results are small integers, exact in binary32
+    o = _oracle(oracle_mod)((2, 13))
+    ctx = ctxs[(2, 13)]
+    n_out, k_in = 50, 500
+    stream, _, nblocks = gen.make_layer(o.N, o.W, n_out, k_in, 1, seed=5)
+    ones = np.full(nblocks, 0x3C00, dtype=np.uint16)
+    pts, _ = o.decode_stream(stream, nblocks)
+    Wint = pts.reshape(n_out, -1)[:, :k_in].astype(np.int64)
+    for xv in (np.ones(k_in, dtype=np.float32), np.eye(k_in, dtype=np.float32)[499], np.eye(k_in, dtype=np.float32)[24]):
+        y = lib.llvq_gemv(ctx, to_dev_u8(stream), to_dev_f16(ones), n_out, k_in, to_dev_bf16(gen.f32_to_bf16_bits(xv)))
+        torch.cuda.synchronize()
+        assert np.array_equal(y.cpu().numpy().astype(np.int64), (Wint * xv.astype(np.int64)).sum(axis=1))
+
+
+@pytest.mark.parametrize("n_out,k_in", [(4096, 4096), (11008, 4096), (4096, 11008)])
+def test_gemv_full_size_layers_sampled_rows(lib, ctxs, oracle_mod, n_out, k_in):
+    # the 7B-shaped layers the benchmark times, in the same launch configuration; the oracle
+    # recomputes a sample of output rows one by one
+    o = _oracle(oracle_mod)((2, 13))
+    ctx = ctxs[(2, 13)]
+    stream, gain, _ = gen.make_layer(o.N, o.W, n_out, k_in, 1, seed=0)
+    x = gen.normal_bf16(k_in, seed=0)
+    y = lib.llvq_gemv(ctx, to_dev_u8(stream), to_dev_f16(gain), n_out, k_in, to_dev_bf16(x), y_dtype=torch.bfloat16)
+    torch.cuda.synchronize()
+    y = y.float().cpu().numpy()
+    rows = sorted(set([0, 1, 7, 8, n_out // 2, n_out - 9, n_out - 1] + list(range(5, n_out, n_out // 23))))
+    ref = np.array([o.gemv(stream, gain, n_out, k_in, x, rows=(r, 1))[r] for r in rows])
+    scale = float(np.abs(ref).max())
+    err = np.abs(y[rows] - ref) / np.maximum(np.abs(ref), 1e-3 * scale)
+    assert err.max() <= TOL_BF16_OUT
+    assert np.isfinite(y).all()
+    assert lib.llvq_last_error(ctx) == (0, 0)
+
+
+def test_argument_checks(lib, ctxs):
+    ctx = ctxs[(2, 13)]
+    idx = torch.zeros(64, dtype=torch.uint8, device="cuda")
+    pts = torch.zeros((4, 24), dtype=torch.int8, device="cuda")
+    L = ctx._lib
+    assert L.llvq_decode_blocks(ctx._h, None, 4, pts.data_ptr(), None) == 1           # EINVAL
+    assert L.llvq_decode_blocks(ctx._h, idx.data_ptr() + 4, 4, pts.data_ptr(), None) == 2   # EALIGN
+    assert L.llvq_decode_blocks(ctx._h, idx.data_ptr(), 4, pts.data_ptr() + 1, None) == 2
+    g = torch.zeros(8, dtype=torch.float16, device="cuda")
+    w = torch.zeros(64, dtype=torch.bfloat16, device="cuda")
+    assert L.llvq_dequant_matrix(ctx._h, idx.data_ptr(), g.data_ptr(), 2, 24, 7, w.data_ptr(), 24, None) == 1
+    assert L.llvq_dequant_matrix(ctx._h, idx.data_ptr(), g.data_ptr(), 2, 24, 1, w.data_ptr(), 8, None) == 1
+    assert L.llvq_gemv(ctx._h, idx.data_ptr(), g.data_ptr(), 2, 24, w.data_ptr(), w.data_ptr(), 9, None) == 1
+    assert L.llvq_gemv(ctx._h, idx.data_ptr(), g.data_ptr(), 2, 10_000_000, w.data_ptr(), w.data_ptr(), 0, None) == 3
+    torch.cuda.synchronize()
