@@ -1,0 +1,342 @@
+#!/usr/bin/env python
+"""Benchmark of the LLVQ dequantization hot path on B200.
+
+A "step" is one pass of the fused dequant+GEMV (batch 1) over the three
+7B-shaped layers of the headline workload -- 4096x4096, 11008x4096 and
+4096x11008 at ~2 bits/weight (48-bit indices over the union of shells 2..13,
+fp16 gain per block of 24), bf16 activations, fp32 accumulation, bf16 output.
+Inputs are seeded and synthetic (uniform indices, |N(0,1)|*0.02 gains, N(0,1)
+activations).  The metric is algorithmic GB/s: compressed index + gain +
+activation + output bytes per second, the numerator of the HBM roofline.
+
+Timing: CUDA events on the launching stream; the step rotates over several
+distinct copies of the layers whose total size exceeds L2, so no timed
+iteration re-reads weights from cache.  One JSON line on stdout.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import llvq_inputs as gen  # noqa: E402
+
+CODE = (2, 13)                      # Lambda_24(13): 48-bit indices, 2.000 bits/weight + gain
+CODE_N = 280974212784720            # Table 1, N(13)
+CODE_W = 48
+LAYERS = [(4096, 4096), (11008, 4096), (4096, 11008)]      # (n_out, k_in)
+L2_BYTES = 126 * 1024 * 1024
+METRIC = "fused dequant+GEMV algorithmic GB/s (index+gain+activation+output bytes / s), 7B-shaped layers, ~2 bits/weight"
+UNIT = "GB/s"
+WORKLOAD = "configs[2]: fused dequant+GEMV batch 1 on W 4096x4096, 11008x4096, 4096x11008, 48-bit indices (shells 2..13), fp16 gain per 24 weights"
+
+# dram bytes (read + write) of one gemv launch on the 11008x4096 layer, from the ncu capture summarised
+# in profiles/; None until a capture exists
+NCU_TRAFFIC_BYTES_11008x4096 = None
+
+
+def layer_bytes(n_out: int, k_in: int) -> dict:
+    bpr = (k_in + 23) // 24
+    nblocks = n_out * bpr
+    return {"nblocks": nblocks, "idx": nblocks * CODE_W // 8, "gain": nblocks * 2, "x": k_in * 2, "y": n_out * 2}
+
+
+def algorithmic_bytes(n_out: int, k_in: int) -> int:
+    b = layer_bytes(n_out, k_in)
+    return b["idx"] + b["gain"] + b["x"] + b["y"]
+
+
+def host_layer(n_out: int, k_in: int, seed: int):
+    stream, gain, nblocks = gen.make_layer(CODE_N, CODE_W, n_out, k_in, 1, seed)
+    x = gen.normal_bf16(k_in, seed)
+    return stream, gain, x, nblocks
+
+
+def measured_peaks() -> tuple[float, str]:
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured"
+    except Exception:
+        return 6650.0, "fallback"
+
+
+class ClockSampler:
+    """Polls SM clock and throttle reasons through NVML (read-only) while the timed region runs."""
+
+    def __init__(self, index: int):
+        self.samples, self.reasons, self.max_mhz = [], set(), None
+        self._stop = threading.Event()
+        self._thread = None
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self._nv = pynvml
+            self._h = pynvml.nvmlDeviceGetHandleByIndex(index)
+            self.max_mhz = int(pynvml.nvmlDeviceGetMaxClockInfo(self._h, pynvml.NVML_CLOCK_SM))
+        except Exception:
+            self._nv = None
+
+    def _run(self):
+        nv = self._nv
+        names = {
+            "hw_slowdown": getattr(nv, "nvmlClocksEventReasonHwSlowdown", 0x8),
+            "hw_thermal_slowdown": getattr(nv, "nvmlClocksEventReasonHwThermalSlowdown", 0x40),
+            "sw_thermal_slowdown": getattr(nv, "nvmlClocksEventReasonSwThermalSlowdown", 0x20),
+            "sw_power_cap": getattr(nv, "nvmlClocksEventReasonSwPowerCap", 0x4),
+        }
+        while not self._stop.is_set():
+            try:
+                self.samples.append(int(nv.nvmlDeviceGetClockInfo(self._h, nv.NVML_CLOCK_SM)))
+                try:
+                    mask = int(nv.nvmlDeviceGetCurrentClocksEventReasons(self._h))
+                except Exception:
+                    mask = int(nv.nvmlDeviceGetCurrentClocksThrottleReasons(self._h))
+                for k, bit in names.items():
+                    if mask & bit:
+                        self.reasons.add(k)
+            except Exception:
+                pass
+            time.sleep(0.002)
+
+    def __enter__(self):
+        if self._nv is not None:
+            self._thread = threading.Thread(target=self._run, daemon=True)
+            self._thread.start()
+        return self
+
+    def __exit__(self, *exc):
+        self._stop.set()
+        if self._thread is not None:
+            self._thread.join()
+
+    def summary(self) -> dict:
+        med = int(np.median(self.samples)) if self.samples else None
+        return {"sm_mhz": med, "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons), "samples": len(self.samples)}
+
+
+def run_reference(args) -> None:
+    """The CPU oracle, as it stands, on the host cores: the slow baseline arm."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    import oracle
+    code = oracle.Code(*CODE)
+    cores = os.cpu_count() or 1
+    rows_per_layer = 256                                   # bounded sample: 256 output rows of each layer per step
+    data = [host_layer(n, k, seed=0) for n, k in LAYERS]
+    sample_bytes = sum(algorithmic_bytes(n, k) * rows_per_layer / n for n, k in LAYERS)
+
+    def step():
+        for (n, k), (stream, gain, x, _) in zip(LAYERS, data):
+            code.gemv(stream, gain, n, k, x, rows=(0, rows_per_layer), threads=cores)
+
+    for _ in range(args.warmup):
+        step()
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        step()
+    dt = time.perf_counter() - t0
+    value = sample_bytes * args.steps / dt / 1e9
+    sample = f"{rows_per_layer} output rows of each of the 3 layers per step"
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": dt / args.steps * 1e3, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": WORKLOAD, "sample": sample},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }))
+
+
+def cpu_baseline() -> dict:
+    """Times the oracle on a bounded sample of the same workload on the host cores (rank 0, N = 1 only)."""
+    import oracle
+    code = oracle.Code(*CODE)
+    cores = os.cpu_count() or 1
+    n_out, k_in = LAYERS[0]
+    stream, gain, x, nblocks = host_layer(n_out, k_in, seed=0)
+    code.gemv(stream, gain, n_out, k_in, x, rows=(0, 64), threads=cores)      # touch
+    reps, t0 = 0, time.perf_counter()
+    while time.perf_counter() - t0 < 10.0 and reps < 20:
+        code.gemv(stream, gain, n_out, k_in, x, threads=cores)
+        reps += 1
+    dt = time.perf_counter() - t0
+    gbs = algorithmic_bytes(n_out, k_in) * reps / dt / 1e9
+    return {"value": gbs, "unit": UNIT, "cores": cores, "kind": "oracle",
+            "sample": f"{reps} x the 4096x4096 layer ({nblocks} blocks each), fp64 GEMV", "blocks_per_s": nblocks * reps / dt}
+
+
+def main() -> None:
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--warmup", type=int, default=20)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+
+    if args.impl == "reference":
+        run_reference(args)
+        return
+
+    import torch
+    import paper_2603_11021_b200 as P
+
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: there is no CPU path")
+    torch.cuda.set_device(local_rank)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+
+    ctx = P.Context(*CODE, device=local_rank)
+    assert ctx.num_points == CODE_N and ctx.index_bits == CODE_W
+
+    # distinct copies of the three layers, more than twice L2 in total, visited round robin
+    step_bytes = sum(algorithmic_bytes(n, k) for n, k in LAYERS)
+    copies = max(2, -(-2 * L2_BYTES // step_bytes))
+    sets, host_sets = [], []
+    for c in range(copies):
+        dev, host = [], []
+        for li, (n, k) in enumerate(LAYERS):
+            stream, gain, x, nblocks = host_layer(n, k, seed=1000 * rank + 10 * c + li)
+            h = (torch.from_numpy(stream).pin_memory(), torch.from_numpy(gain.view(np.float16)).pin_memory(),
+                 torch.from_numpy(x.view(np.int16)).view(torch.bfloat16).pin_memory())
+            host.append(h)
+            dev.append(tuple(t.cuda() for t in h) + (torch.empty(n, dtype=torch.bfloat16, device="cuda"),))
+        sets.append(dev)
+        host_sets.append(host)
+    torch.cuda.synchronize()
+
+    launches = 0
+
+    def step(i: int) -> None:
+        nonlocal launches
+        for (n, k), (d_idx, d_gain, d_x, d_y) in zip(LAYERS, sets[i % copies]):
+            P.llvq_gemv(ctx, d_idx, d_gain, n, k, d_x, d_y=d_y)
+            launches += 1
+
+    def barrier():
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for i in range(args.warmup):
+        step(i)
+    barrier()
+    launches = 0
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    with ClockSampler(local_rank) as clocks:
+        ev0.record()
+        for i in range(args.steps):
+            step(i)
+        ev1.record()
+        barrier()
+    ms_total = ev0.elapsed_time(ev1)
+    if dist is not None:
+        t = torch.tensor([ms_total], device="cuda")
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms_total = float(t.item())
+    ms_per_step = ms_total / args.steps
+    value = world * step_bytes / (ms_per_step * 1e-3) / 1e9
+    timed_launches = launches
+
+    # per-layer device time of the kernel (events around each launch, same rotation)
+    per_layer = []
+    for li, (n, k) in enumerate(LAYERS):
+        tot = 0.0
+        reps = max(10, min(args.steps, 100))
+        for i in range(reps):
+            d_idx, d_gain, d_x, d_y = sets[i % copies][li]
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record()
+            P.llvq_gemv(ctx, d_idx, d_gain, n, k, d_x, d_y=d_y)
+            b.record()
+            b.synchronize()
+            tot += a.elapsed_time(b)
+        us = tot / reps * 1e3
+        by = algorithmic_bytes(n, k)
+        per_layer.append({"n_out": n, "k_in": k, "us": us, "GBps": by / us / 1e3,
+                          "weights_per_s": n * k / (us * 1e-6)})
+
+    # end to end: inputs start in pinned host memory, the result is read back to the host, every step
+    h2d = sum(layer_bytes(n, k)["idx"] + layer_bytes(n, k)["gain"] + layer_bytes(n, k)["x"] for n, k in LAYERS)
+    d2h = sum(layer_bytes(n, k)["y"] for n, k in LAYERS)
+    y_host = [torch.empty(n, dtype=torch.bfloat16).pin_memory() for n, _ in LAYERS]
+    e2e_steps = max(3, min(args.steps, 20))
+
+    def e2e_step(i: int) -> None:
+        for li, (n, k) in enumerate(LAYERS):
+            h_idx, h_gain, h_x = host_sets[i % copies][li]
+            d_idx, d_gain, d_x, d_y = sets[i % copies][li]
+            d_idx.copy_(h_idx, non_blocking=True)
+            d_gain.copy_(h_gain, non_blocking=True)
+            d_x.copy_(h_x, non_blocking=True)
+            P.llvq_gemv(ctx, d_idx, d_gain, n, k, d_x, d_y=d_y)
+            y_host[li].copy_(d_y, non_blocking=True)
+        torch.cuda.current_stream().synchronize()
+
+    for i in range(3):
+        e2e_step(i)
+    barrier()
+    ev0.record()
+    for i in range(e2e_steps):
+        e2e_step(i)
+    ev1.record()
+    barrier()
+    e2e_ms = ev0.elapsed_time(ev1) / e2e_steps
+    if dist is not None:
+        t = torch.tensor([e2e_ms], device="cuda")
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        e2e_ms = float(t.item())
+    e2e_value = world * step_bytes / (e2e_ms * 1e-3) / 1e9
+
+    bad, flags = P.llvq_last_error(ctx)
+    if bad or flags:
+        raise SystemExit(f"device error state: {bad} invalid fields, flags {flags}")
+
+    if rank == 0:
+        peak, which = measured_peaks()
+        dom = per_layer[1]                                   # the 11008x4096 launch: largest share of the step
+        dom_bytes = algorithmic_bytes(*LAYERS[1])
+        achieved = dom_bytes / dom["us"] / 1e3
+        out = {
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+            "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": "bf16 weights x bf16 activations, f32 accumulate", "data": "synthetic",
+            "config": {"workload": WORKLOAD, "l2": f"rotation over {copies} distinct copies of the layers ({copies * step_bytes / 1e6:.0f} MB > 2 x L2)",
+                       "bytes_per_step": step_bytes, "blocks_per_step": sum(layer_bytes(n, k)["nblocks"] for n, k in LAYERS)},
+            "weights_per_s": world * sum(n * k for n, k in LAYERS) / (ms_per_step * 1e-3),
+            "frac_of_hbm_peak": value / world / peak,
+            "layers": per_layer,
+            "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
+                         "traffic": NCU_TRAFFIC_BYTES_11008x4096, "kernel": "gemv_kernel on 11008x4096",
+                         "algorithmic_bytes_per_launch": dom_bytes, "peak_source": f"of {which}", "frac_of_nominal_8TBps": achieved / 8000.0},
+            "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "ms_per_step": e2e_ms},
+            "gpu_launches": timed_launches,
+            "clocks": clocks.summary(),
+        }
+        if world == 1 and not args.no_cpu_baseline:
+            out["cpu_baseline"] = cpu_baseline()
+        print(json.dumps(out))
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

@@ -291,10 +291,10 @@ int llvq_golay_table(const llvq_ctx* ctx, uint32_t out[4096])
 
 int llvq_decode_blocks(const llvq_ctx* ctx, const void* d_idx, uint64_t nblocks, int8_t* d_points, void* stream)
 {
+    if (ctx && ctx->device >= 0 && nblocks == 0) return LLVQ_OK;      // nothing to do: pointers may be null
     if (int e = check_common(ctx, d_idx)) return e;
     if (!d_points) return LLVQ_EINVAL;
     if (!aligned(d_points, 4)) return LLVQ_EALIGN;
-    if (nblocks == 0) return LLVQ_OK;
     if (nblocks > (1ull << 40)) return LLVQ_EUNSUPPORTED;
     DeviceGuard guard(ctx->device);
     if (!guard.ok) return LLVQ_ECUDA;
