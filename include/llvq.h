@@ -94,7 +94,7 @@ int llvq_golay_table(const llvq_ctx* ctx, uint32_t out[4096]);
 /*
  * Dequantizer, App. A steps 1-4: d_points[b][0..23] = the integer lattice point
  * (coordinates of L^int, |x_i| <= 28) of field b, b < nblocks.
- * d_idx: device, 16-byte aligned.  d_points: device, int8 [nblocks][24], 4-byte aligned.
+ * d_idx: device, 16-byte aligned.  d_points: device, int8 [nblocks][24], 8-byte aligned.
  */
 int llvq_decode_blocks(const llvq_ctx* ctx, const void* d_idx, uint64_t nblocks,
                        int8_t* d_points, void* stream);

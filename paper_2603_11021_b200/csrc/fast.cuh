@@ -1,0 +1,272 @@
+// Fast dequantizer for codes whose tables fit in shared memory (few classes,
+// indices up to 64 bits): App. A steps 1-4 with every table lookup served from
+// shared memory, one thread per block of 24 weights.
+#pragma once
+#include <cstdint>
+#include <cuda_bf16.h>
+#include <cuda_fp16.h>
+
+#include "tables.h"
+
+namespace llvq {
+
+constexpr uint32_t kFullMask = 0xffffffffu;
+
+// Pointers into the CTA's copy of the table image.
+struct FastSmem {
+    const uint32_t* golay;
+    const uint16_t* lut;
+    const uint32_t* pascal;
+    const uint32_t* base16;
+    const uint16_t* r16;
+    const uint8_t* pd6;
+    const uint64_t* off;
+    const uint32_t* desc;
+    uint32_t lut_shift;
+};
+
+__device__ __forceinline__ FastSmem fast_view(const uint8_t* smem, const FastLayout& L)
+{
+    FastSmem T;
+    T.golay = reinterpret_cast<const uint32_t*>(smem + L.golay);
+    T.lut = reinterpret_cast<const uint16_t*>(smem + L.lut);
+    T.pascal = reinterpret_cast<const uint32_t*>(smem + L.pascal);
+    T.base16 = reinterpret_cast<const uint32_t*>(smem + L.base16);
+    T.r16 = reinterpret_cast<const uint16_t*>(smem + L.r16);
+    T.pd6 = smem + L.pd6;
+    T.off = reinterpret_cast<const uint64_t*>(smem + L.off);
+    T.desc = reinterpret_cast<const uint32_t*>(smem + L.desc);
+    T.lut_shift = L.lut_shift;
+    return T;
+}
+
+__device__ __forceinline__ uint32_t smem_addr(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+// Copy the table image into shared memory with bulk asynchronous copies (TMA,
+// no multicast) tracked by one mbarrier.  Every thread of the CTA must call this.
+// Returns false (for the whole CTA) if the copy did not complete within the
+// wait limit; the error flag is then set and the caller must return.
+__device__ __forceinline__ bool fast_load_image(uint8_t* dst, const uint8_t* __restrict__ src, uint32_t bytes,
+                                                uint64_t* bar, uint32_t* err_flags)
+{
+    const uint32_t bar_a = smem_addr(bar);
+    if (threadIdx.x == 0) {
+        asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(bar_a));
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar_a), "r"(bytes) : "memory");
+        constexpr uint32_t kChunk = 32768;
+        for (uint32_t o = 0; o < bytes; o += kChunk) {
+            uint32_t n = bytes - o < kChunk ? bytes - o : kChunk;
+            asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                         ::"r"(smem_addr(dst + o)), "l"(src + o), "r"(n), "r"(bar_a) : "memory");
+        }
+    }
+    uint32_t done = 0;
+    for (uint32_t it = 0; it < (1u << 20) && !done; ++it) {
+        asm volatile("{\n .reg .pred p;\n mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n selp.u32 %0, 1, 0, p;\n}"
+                     : "=r"(done) : "r"(bar_a), "r"(0u) : "memory");
+    }
+    if (!done) atomicOr(err_flags, 1u);
+    return __syncthreads_and((int)done) != 0;
+}
+
+// Deposit the low bits of src into the set bits of mask, lowest first (24-bit masks, 6 bits per lookup).
+__device__ __forceinline__ uint32_t deposit24(const uint8_t* pd6, uint32_t src, uint32_t mask)
+{
+    uint32_t out = 0;
+#pragma unroll
+    for (int g = 0; g < 4; ++g) {
+        const uint32_t f = (mask >> (6 * g)) & 63u;
+        out |= (uint32_t)pd6[(f << 6) | (src & 63u)] << (6 * g);
+        src >>= __popc(f);
+    }
+    return out;
+}
+
+// The rho-th k-subset of the slots {0..n-1} in combinatorial-number-system order (numeric
+// order of the bit masks).  Slots >= 16 are decided one at a time against C(slot, t); the
+// remaining t-subset of the low 16 slots is one table entry.  `top` = largest n in the warp.
+__device__ __forceinline__ uint32_t nth_subset(const FastSmem& T, uint32_t k, uint32_t rho, int top)
+{
+    uint32_t m = 0, t = k;
+    for (int pos = top - 1; pos >= 16; --pos) {
+        const uint32_t cnt = T.pascal[pos * 25 + t];
+        if (t > 0 && rho >= cnt) { rho -= cnt; m |= 1u << pos; --t; }
+    }
+    uint32_t idx, flip;
+    if (t <= 8) { idx = T.base16[t] + rho; flip = 0u; }
+    else        { idx = T.base16[16 - t] + (T.base16[16 + t] - 1u - rho); flip = 0xffffu; }
+    return m | ((uint32_t)T.r16[idx] ^ flip);
+}
+
+// Result of the index -> point map in a form the consumers expand cheaply:
+// three bit planes giving each position a value id (0..7), the table of
+// absolute values per id, and the mask of negative positions.
+struct Decoded {
+    uint32_t p0, p1, p2;
+    uint32_t neg;
+    uint32_t vals_lo, vals_hi;     // absolute value of id 0..3 / 4..7, one byte each
+};
+
+__device__ __forceinline__ void fast_decode(const FastSmem& T, uint64_t I, bool valid, Decoded& d)
+{
+    // S2: class lookup
+    uint32_t cls = valid ? T.lut[(uint32_t)(I >> T.lut_shift)] : 0u;
+    if (valid) while (I >= T.off[cls + 1]) ++cls;
+    const uint64_t local = valid ? I - T.off[cls] : 0ull;
+    const uint4* D = reinterpret_cast<const uint4*>(T.desc + cls * kFastDescWords);
+    const uint4 h = D[0], v = D[1], lw = D[2], mg = D[3];
+    const uint32_t w = h.x & 0xff, B = (h.x >> 8) & 0xff, flags = (h.x >> 16) & 0xff;
+    const uint32_t nlev1 = (h.x >> 24) & 0xf, nlev = valid ? h.x >> 28 : 0u;
+    const uint32_t goff = h.y & 0xffff, A = h.y >> 16;
+    const bool odd = flags & 1u;
+
+    // S3: r fastest, then the sign word s, then the arrangement rank p
+    uint64_t q;
+    uint32_t r;
+    if (A == 4096u) { r = (uint32_t)local & 4095u; q = local >> 12; }
+    else {
+        q = __umul64hi(local, ((uint64_t)h.w << 32) | h.z);
+        uint64_t rem = local - q * A;
+        if (rem >= A) { rem -= A; ++q; }
+        r = (uint32_t)rem;
+    }
+    const uint32_t s = (uint32_t)q & ((1u << B) - 1u);
+    const uint64_t p = q >> B;
+
+    // S4: Golay codeword
+    const uint32_t c = T.golay[goff + r];
+
+    // S5: arrangement.  Group 1 lives on F1(c), group 0 on F0(c); an odd class is one group 0 on all positions.
+    const uint32_t F1 = odd ? 0u : c;
+    const uint32_t F0 = ~F1 & 0xffffffu;
+    uint32_t freem = F1;
+    bool in_group0 = false;
+    uint32_t p0 = 0, p1 = 0, p2 = 0, bit1 = 0, nz0 = 0;
+    uint32_t p32 = 0;
+    const uint32_t lwords[4] = {lw.x, lw.y, lw.z, lw.w};
+    const uint32_t magics[4] = {0u, mg.x, mg.y, mg.z};
+    const int maxlev = __reduce_max_sync(kFullMask, nlev);
+#pragma unroll
+    for (int l = 0; l < kFastMaxLevels; ++l) {
+        if (l < maxlev) {
+            if (!in_group0 && (uint32_t)l >= nlev1) {           // group 1 done: its filler gets id 1
+                p0 |= freem;
+                if (flags & 8u) bit1 |= freem;
+                freem = F0; in_group0 = true;
+            }
+            const bool active = (uint32_t)l < nlev;
+            const uint32_t word = lwords[l];
+            const uint32_t radix = word & 0x3fffffu;
+            const uint32_t k = active ? (word >> 22) & 31u : 0u;
+            uint32_t rho;
+            if (l == 0) {
+                uint64_t qq = __umul64hi(p, ((uint64_t)v.w << 32) | v.z);
+                uint64_t rem = p - qq * radix;
+                if (rem >= radix) { rem -= radix; ++qq; }
+                p32 = (uint32_t)qq; rho = (uint32_t)rem;
+            } else {
+                uint32_t qq = __umulhi(p32, magics[l]);
+                uint32_t rem = p32 - qq * radix;
+                if (rem >= radix) { rem -= radix; ++qq; }
+                p32 = qq; rho = rem;
+            }
+            if (!active) rho = 0u;
+            const uint32_t n = active ? (mg.w >> (8 * l)) & 0xffu : 0u;
+            const int top = __reduce_max_sync(kFullMask, n);
+            const uint32_t rel = nth_subset(T, k, rho, top);
+            const uint32_t a = deposit24(T.pd6, rel, freem);
+            freem ^= a;
+            if (word & (1u << 27)) p0 |= a;
+            if (word & (1u << 28)) p1 |= a;
+            if (word & (1u << 29)) p2 |= a;
+            if (word & (1u << 30)) bit1 |= a;
+            if (in_group0 && (word >> 31)) nz0 |= a;
+        }
+    }
+    if (!in_group0) {
+        p0 |= freem;
+        if (flags & 8u) bit1 |= freem;
+        freem = F0;
+    }
+    if (flags & 16u) bit1 |= freem;                             // filler of group 0 keeps id 0
+    if (flags & 4u) nz0 |= freem;
+
+    // S6: signs
+    const uint32_t nf1 = w ? w - 1u : 0u;                       // free sign bits on F1
+    const uint32_t s1 = s & ((1u << nf1) - 1u);
+    const uint32_t src1 = s1 | (((__popc(s1) + (flags >> 1)) & 1u) << nf1);   // last F1 position: sum = 0 mod 8
+    const uint32_t neg_even = deposit24(T.pd6, src1, F1) | deposit24(T.pd6, s >> nf1, odd ? 0u : nz0);
+    uint32_t neg = odd ? (c ^ bit1) : neg_even;                 // odd: 1 mod 4 on F0, 3 mod 4 on F1
+    if (!valid) { p0 = p1 = p2 = 0; neg = 0; }
+    d.p0 = p0; d.p1 = p1; d.p2 = p2; d.neg = neg;
+    d.vals_lo = valid ? v.x : 0u; d.vals_hi = valid ? v.y : 0u;
+}
+
+// ---- expansion helpers -------------------------------------------------------
+// 8 mask bits -> 8 nibbles (bit i -> bit 4i).
+__device__ __forceinline__ uint32_t nibspread8(uint32_t b)
+{
+    uint32_t x = (b | (b << 12)) & 0x000f000fu;
+    x = (x | (x << 6)) & 0x03030303u;
+    x = (x | (x << 3)) & 0x11111111u;
+    return x;
+}
+
+// Value id of each position as a nibble string: sel[r] holds positions 8r..8r+7.
+__device__ __forceinline__ void id_nibbles(const Decoded& d, uint32_t sel[3])
+{
+#pragma unroll
+    for (int r = 0; r < 3; ++r)
+        sel[r] = nibspread8((d.p0 >> (8 * r)) & 0xffu) | (nibspread8((d.p1 >> (8 * r)) & 0xffu) << 1) |
+                 (nibspread8((d.p2 >> (8 * r)) & 0xffu) << 2);
+}
+
+// 4 mask bits -> the most significant bits of 4 bytes.
+__device__ __forceinline__ uint32_t msbspread4(uint32_t nib) { return (nib * 0x10204080u) & 0x80808080u; }
+
+// The 24 coordinates as signed bytes, coordinate i in byte (i & 3) of word (i >> 2).
+__device__ __forceinline__ void expand_bytes(const Decoded& d, uint32_t out[6])
+{
+    uint32_t sel[3];
+    id_nibbles(d, sel);
+#pragma unroll
+    for (int j = 0; j < 6; ++j) {
+        const uint32_t s16 = (j & 1) ? sel[j >> 1] >> 16 : sel[j >> 1];
+        const uint32_t a = __byte_perm(d.vals_lo, d.vals_hi, s16);
+        const uint32_t sm = msbspread4((d.neg >> (4 * j)) & 15u) >> 7;     // bytes 0 / 1
+        out[j] = (a ^ (sm * 0xffu)) + sm;                                     // negated bytes are never zero
+    }
+}
+
+// The 24 dequantized weights bf16_rn(gain * x_i) as 12 packed pairs (weight 2j in the low half of w[j]).
+__device__ __forceinline__ void expand_bf16(const Decoded& d, float gain, uint32_t w[12])
+{
+    // bf16(gain * a) for the eight value ids; float(a) by the 2^23 trick (a <= 28)
+    uint32_t packed[4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        const uint32_t src = i < 2 ? d.vals_lo : d.vals_hi;
+        const float a0 = __uint_as_float(__byte_perm(src, 0x4b000000u, (i & 1) ? 0x7442 : 0x7440)) - 8388608.f;
+        const float a1 = __uint_as_float(__byte_perm(src, 0x4b000000u, (i & 1) ? 0x7443 : 0x7441)) - 8388608.f;
+        __nv_bfloat162 b = __floats2bfloat162_rn(gain * a0, gain * a1);
+        packed[i] = *reinterpret_cast<uint32_t*>(&b);
+    }
+    const uint32_t lo03 = __byte_perm(packed[0], packed[1], 0x6420), hi03 = __byte_perm(packed[0], packed[1], 0x7531);
+    const uint32_t lo47 = __byte_perm(packed[2], packed[3], 0x6420), hi47 = __byte_perm(packed[2], packed[3], 0x7531);
+    uint32_t sel[3];
+    id_nibbles(d, sel);
+#pragma unroll
+    for (int j = 0; j < 6; ++j) {
+        const uint32_t s16 = (j & 1) ? sel[j >> 1] >> 16 : sel[j >> 1];
+        const uint32_t lob = __byte_perm(lo03, lo47, s16);
+        const uint32_t hib = __byte_perm(hi03, hi47, s16) ^ msbspread4((d.neg >> (4 * j)) & 15u);
+        w[2 * j] = __byte_perm(lob, hib, 0x5140);
+        w[2 * j + 1] = __byte_perm(lob, hib, 0x7362);
+    }
+}
+
+}  // namespace llvq

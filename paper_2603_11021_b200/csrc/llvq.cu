@@ -3,12 +3,14 @@
 
 #include <cuda_runtime.h>
 
+#include <algorithm>
 #include <cstdio>
 #include <cstring>
 #include <new>
 #include <vector>
 
 #include "decode.cuh"
+#include "fast.cuh"
 #include "tables.h"
 
 using namespace llvq;
@@ -20,6 +22,9 @@ struct llvq_ctx {
     void* d_blob = nullptr;          // one allocation holding every device table
     unsigned long long* d_err = nullptr;
     int sm_count = 0;
+    bool fast = false;               // tables fit shared memory: the fast kernels are used
+    FastLayout fl{};
+    const uint8_t* d_image = nullptr;
 };
 
 namespace {
@@ -165,6 +170,184 @@ gemv_kernel(DevCode dc, const uint32_t* __restrict__ stream, const uint16_t* __r
     }
 }
 
+
+// ===========================================================================
+// Fast path (tables in shared memory).  Dynamic shared memory of every fast
+// kernel: [table image | mbarrier (16 bytes) | kernel-specific staging].
+// Persistent CTAs, one per SM.
+// ===========================================================================
+constexpr int kFastThreads = 512;
+
+struct FastArgs {
+    FastLayout L;
+    const uint8_t* image;
+    uint32_t* flags;
+    unsigned long long* bad_index;
+    uint64_t n_points;              // N (fits 64 bits on the fast path)
+};
+
+__device__ __forceinline__ uint64_t load_field(const uint32_t* __restrict__ stream, uint64_t b, int W)
+{
+    uint64_t lo, hi;
+    load_index(stream, b, W, lo, hi);
+    return lo;
+}
+
+#define FAST_PROLOGUE()                                                                         \
+    extern __shared__ __align__(128) uint8_t smem[];                                            \
+    uint64_t* bar = reinterpret_cast<uint64_t*>(smem + fa.L.total);                              \
+    uint8_t* staging = smem + fa.L.total + 16;                                                  \
+    (void)staging;                                                                              \
+    if (!fast_load_image(smem, fa.image, fa.L.total, bar, fa.flags)) return;                    \
+    const FastSmem T = fast_view(smem, fa.L);
+
+__global__ void __launch_bounds__(kFastThreads, 1)
+decode_blocks_fast_kernel(FastArgs fa, const uint32_t* __restrict__ stream, uint64_t nblocks, uint2* __restrict__ out)
+{
+    FAST_PROLOGUE();
+    const uint64_t ntiles = (nblocks + kFastThreads - 1) / kFastThreads;
+    for (uint64_t tile = blockIdx.x; tile < ntiles; tile += gridDim.x) {
+        const uint64_t b = tile * kFastThreads + threadIdx.x;
+        const bool in = b < nblocks;
+        const uint64_t I = in ? load_field(stream, b, (int)fa.L.W) : 0ull;
+        const bool valid = in && I < fa.n_points;
+        if (in && !valid) atomicAdd(fa.bad_index, 1ull);
+        Decoded d;
+        fast_decode(T, I, valid, d);
+        if (in) {
+            uint32_t w[6];
+            expand_bytes(d, w);
+            out[b * 3 + 0] = make_uint2(w[0], w[1]);
+            out[b * 3 + 1] = make_uint2(w[2], w[3]);
+            out[b * 3 + 2] = make_uint2(w[4], w[5]);
+        }
+    }
+}
+
+// FLAT (bpr == 0): block b covers elements 24b.. of the flattened matrix.
+// ROWWISE: block b = r * bpr + cb covers columns 24cb.. of row r.
+__global__ void __launch_bounds__(kFastThreads, 1)
+dequant_fast_kernel(FastArgs fa, const uint32_t* __restrict__ stream, const uint16_t* __restrict__ gain, uint64_t nblocks,
+                    int64_t rows, int64_t cols, int64_t bpr, __nv_bfloat16* __restrict__ out, int64_t ld)
+{
+    FAST_PROLOGUE();
+    const uint64_t ntiles = (nblocks + kFastThreads - 1) / kFastThreads;
+    const uint64_t total = (uint64_t)rows * (uint64_t)cols;
+    for (uint64_t tile = blockIdx.x; tile < ntiles; tile += gridDim.x) {
+        const uint64_t b = tile * kFastThreads + threadIdx.x;
+        const bool in = b < nblocks;
+        const uint64_t I = in ? load_field(stream, b, (int)fa.L.W) : 0ull;
+        const bool valid = in && I < fa.n_points;
+        if (in && !valid) atomicAdd(fa.bad_index, 1ull);
+        Decoded d;
+        fast_decode(T, I, valid, d);
+        if (!in) continue;
+        uint32_t w[12];
+        expand_bf16(d, gain_to_float(__ldg(gain + b)), w);
+        __nv_bfloat16* dst;
+        int64_t left;
+        if (bpr == 0) { dst = out + b * 24; left = (int64_t)(total - b * 24); }
+        else { const int64_t r = (int64_t)(b / (uint64_t)bpr), cb = (int64_t)(b % (uint64_t)bpr); dst = out + r * ld + cb * 24; left = cols - cb * 24; }
+        if (left >= 24 && (reinterpret_cast<uintptr_t>(dst) & 15) == 0) {
+            uint4* d4 = reinterpret_cast<uint4*>(dst);
+            d4[0] = make_uint4(w[0], w[1], w[2], w[3]);
+            d4[1] = make_uint4(w[4], w[5], w[6], w[7]);
+            d4[2] = make_uint4(w[8], w[9], w[10], w[11]);
+        } else {
+#pragma unroll
+            for (int j = 0; j < 24; ++j)
+                if (j < left) dst[j] = __ushort_as_bfloat16((unsigned short)(w[j >> 1] >> (16 * (j & 1))));
+        }
+    }
+}
+
+// Fused dequant + GEMV.  A warp owns units of 16 rows x 4 column blocks: lane (g, t) = (lane / 4, lane % 4)
+// decodes the blocks (row g, column block 4q + t) and (row g + 8, same column block); their 2 x 12 packed bf16
+// pairs are the A fragments of six m16n8k16 tensor-core MMAs whose B fragment carries the matching 4 x 24
+// activations (the same in all 8 columns), accumulating in binary32.
+constexpr int kGemvRows = 32;           // output rows per CTA tile
+
+__device__ __forceinline__ void mma_bf16_16816(float c[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0, uint32_t b1)
+{
+    asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+                 : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3]) : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+
+template <bool kOutBf16>
+__global__ void __launch_bounds__(kFastThreads, 1)
+gemv_fast_kernel(FastArgs fa, const uint32_t* __restrict__ stream, const uint16_t* __restrict__ gain,
+                 int64_t n_out, int64_t k_in, int64_t bpr, const uint16_t* __restrict__ x, void* __restrict__ y)
+{
+    FAST_PROLOGUE();
+    const int64_t nq = (bpr + 3) / 4;                               // units along K
+    uint32_t* xs = reinterpret_cast<uint32_t*>(staging);            // [nq * 4][12] packed bf16 pairs of x
+    float* acc = reinterpret_cast<float*>(xs + nq * 48);            // [kGemvRows]
+    for (int64_t i = threadIdx.x; i < nq * 48; i += kFastThreads) {
+        const int64_t e = 2 * i;
+        const uint32_t lo = e < k_in ? __ldg(x + e) : 0u, hi = e + 1 < k_in ? __ldg(x + e + 1) : 0u;
+        xs[i] = lo | hi << 16;
+    }
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, g = lane >> 2, t = lane & 3;
+    constexpr int kWarps = kFastThreads / 32;
+    const int64_t ntiles = (n_out + kGemvRows - 1) / kGemvRows;
+    for (int64_t tile = blockIdx.x; tile < ntiles; tile += gridDim.x) {
+        if (threadIdx.x < kGemvRows) acc[threadIdx.x] = 0.f;
+        __syncthreads();
+        const int64_t row0 = tile * kGemvRows;
+        const int64_t units = (kGemvRows / 16) * nq;
+        for (int64_t u = warp; u < units; u += kWarps) {
+            const int64_t rg = u / nq, kq = u % nq;
+            const int64_t cb = kq * 4 + t;
+            const int64_t rowA = row0 + rg * 16 + g, rowB = rowA + 8;
+            const bool inA = rowA < n_out && cb < bpr, inB = rowB < n_out && cb < bpr;
+            const uint64_t bA = (uint64_t)(rowA * bpr + cb), bB = (uint64_t)(rowB * bpr + cb);
+            const uint64_t IA = inA ? load_field(stream, bA, (int)fa.L.W) : 0ull;
+            const uint64_t IB = inB ? load_field(stream, bB, (int)fa.L.W) : 0ull;
+            const float gA = inA ? gain_to_float(__ldg(gain + bA)) : 0.f;
+            const float gB = inB ? gain_to_float(__ldg(gain + bB)) : 0.f;
+            const bool vA = inA && IA < fa.n_points, vB = inB && IB < fa.n_points;
+            if ((inA && !vA) || (inB && !vB)) atomicAdd(fa.bad_index, (unsigned long long)((inA && !vA) + (inB && !vB)));
+            Decoded dA, dB;
+            fast_decode(T, IA, vA, dA);
+            fast_decode(T, IB, vB, dB);
+            uint32_t wA[12], wB[12];
+            expand_bf16(dA, gA, wA);
+            expand_bf16(dB, gB, wB);
+            const uint4* xb = reinterpret_cast<const uint4*>(xs + cb * 12);
+            const uint4 x0 = xb[0], x1 = xb[1], x2 = xb[2];
+            const uint32_t xv[12] = {x0.x, x0.y, x0.z, x0.w, x1.x, x1.y, x1.z, x1.w, x2.x, x2.y, x2.z, x2.w};
+            float c[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+            for (int q = 0; q < 6; ++q)
+                mma_bf16_16816(c, wA[2 * q], wB[2 * q], wA[2 * q + 1], wB[2 * q + 1], xv[2 * q], xv[2 * q + 1]);
+            if (t == 0) {
+                atomicAdd(&acc[rg * 16 + g], c[0]);
+                atomicAdd(&acc[rg * 16 + g + 8], c[2]);
+            }
+        }
+        __syncthreads();
+        if (threadIdx.x < kGemvRows && row0 + threadIdx.x < n_out) {
+            if (kOutBf16) reinterpret_cast<__nv_bfloat16*>(y)[row0 + threadIdx.x] = __float2bfloat16_rn(acc[threadIdx.x]);
+            else reinterpret_cast<float*>(y)[row0 + threadIdx.x] = acc[threadIdx.x];
+        }
+        __syncthreads();
+    }
+}
+
+FastArgs fast_args(const llvq_ctx* ctx)
+{
+    FastArgs fa;
+    fa.L = ctx->fl; fa.image = ctx->d_image; fa.flags = ctx->dev.flags; fa.bad_index = ctx->dev.bad_index;
+    fa.n_points = ctx->dev.n_lo;
+    return fa;
+}
+
+template <typename K>
+bool set_smem(K kernel, size_t bytes)
+{
+    return cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes) == cudaSuccess;
+}
+
 int check_common(const llvq_ctx* ctx, const void* d_idx)
 {
     if (!ctx || !d_idx || ctx->device < 0) return LLVQ_EINVAL;
@@ -210,8 +393,12 @@ int llvq_create(llvq_ctx** out, int m_lo, int m_hi, int device)
     size_t o_offlo = up(o_offhi + (ncls + 1) * 4);
     size_t o_cls = up(o_offlo + (ncls + 1) * 8);
     size_t o_err = up(o_cls + ncls * sizeof(ClassDesc));
-    size_t total = o_err + 256;
+    std::vector<uint8_t> image;
+    ctx->fast = build_fast_image(h, ctx->fl, image);
+    size_t o_img = up(o_err + 256);
+    size_t total = o_img + (ctx->fast ? image.size() : 0);
     std::vector<uint8_t> blob(total, 0);
+    if (ctx->fast) std::memcpy(blob.data() + o_img, image.data(), image.size());
     std::memcpy(blob.data() + o_golay, h.golay.data(), 4096 * 4);
     std::memcpy(blob.data() + o_pascal, h.pascal, sizeof(h.pascal));
     std::memcpy(blob.data() + o_offhi, off_hi.data(), (ncls + 1) * 4);
@@ -233,6 +420,7 @@ int llvq_create(llvq_ctx** out, int m_lo, int m_hi, int device)
     ctx->dev.n_lo = (uint64_t)h.N; ctx->dev.n_hi = (uint64_t)(h.N >> 64);
     ctx->dev.nclasses = (int)ncls;
     ctx->dev.W = h.W;
+    ctx->d_image = d + o_img;
     *out = ctx;
     return LLVQ_OK;
 }
@@ -294,10 +482,19 @@ int llvq_decode_blocks(const llvq_ctx* ctx, const void* d_idx, uint64_t nblocks,
     if (ctx && ctx->device >= 0 && nblocks == 0) return LLVQ_OK;      // nothing to do: pointers may be null
     if (int e = check_common(ctx, d_idx)) return e;
     if (!d_points) return LLVQ_EINVAL;
-    if (!aligned(d_points, 4)) return LLVQ_EALIGN;
+    if (!aligned(d_points, 8)) return LLVQ_EALIGN;
     if (nblocks > (1ull << 40)) return LLVQ_EUNSUPPORTED;
     DeviceGuard guard(ctx->device);
     if (!guard.ok) return LLVQ_ECUDA;
+    if (ctx->fast) {
+        const size_t smem = ctx->fl.total + 16;
+        if (!set_smem(decode_blocks_fast_kernel, smem)) return LLVQ_ECUDA;
+        uint64_t tiles = (nblocks + kFastThreads - 1) / kFastThreads;
+        unsigned g = (unsigned)std::min<uint64_t>(tiles, (uint64_t)ctx->sm_count);
+        decode_blocks_fast_kernel<<<g, kFastThreads, smem, (cudaStream_t)stream>>>(
+            fast_args(ctx), static_cast<const uint32_t*>(d_idx), nblocks, reinterpret_cast<uint2*>(d_points));
+        return launch_status();
+    }
     uint64_t grid = (nblocks + kThreads - 1) / kThreads;
     if (grid > 0x7fffffffull) return LLVQ_EUNSUPPORTED;
     decode_blocks_kernel<<<(unsigned)grid, kThreads, 0, (cudaStream_t)stream>>>(
@@ -317,8 +514,19 @@ int llvq_dequant_matrix(const llvq_ctx* ctx, const void* d_idx, const uint16_t* 
     DeviceGuard guard(ctx->device);
     if (!guard.ok) return LLVQ_ECUDA;
     cudaStream_t st = (cudaStream_t)stream;
+    if (layout == LLVQ_LAYOUT_FLAT && ld != cols) return LLVQ_EINVAL;
+    if (ctx->fast) {
+        const int64_t bpr = layout == LLVQ_LAYOUT_FLAT ? 0 : (cols + 23) / 24;
+        const uint64_t nblocks = layout == LLVQ_LAYOUT_FLAT ? ((uint64_t)rows * (uint64_t)cols + 23) / 24 : (uint64_t)rows * (uint64_t)bpr;
+        const size_t smem = ctx->fl.total + 16;
+        if (!set_smem(dequant_fast_kernel, smem)) return LLVQ_ECUDA;
+        uint64_t tiles = (nblocks + kFastThreads - 1) / kFastThreads;
+        unsigned g = (unsigned)std::min<uint64_t>(tiles, (uint64_t)ctx->sm_count);
+        dequant_fast_kernel<<<g, kFastThreads, smem, st>>>(fast_args(ctx), static_cast<const uint32_t*>(d_idx), d_gain_f16, nblocks,
+                                                           rows, cols, bpr, reinterpret_cast<__nv_bfloat16*>(d_w_bf16), ld);
+        return launch_status();
+    }
     if (layout == LLVQ_LAYOUT_FLAT) {
-        if (ld != cols) return LLVQ_EINVAL;
         uint64_t total = (uint64_t)rows * (uint64_t)cols, nblocks = (total + 23) / 24;
         uint64_t grid = (nblocks + kThreads - 1) / kThreads;
         if (grid > 0x7fffffffull) return LLVQ_EUNSUPPORTED;
@@ -352,6 +560,22 @@ int llvq_gemv(const llvq_ctx* ctx, const void* d_idx, const uint16_t* d_gain_f16
         return cudaMemsetAsync(d_y, 0, (size_t)n_out * (y_dtype == LLVQ_F32 ? 4 : 2), st) == cudaSuccess ? LLVQ_OK : LLVQ_ECUDA;
     }
     int64_t bpr = (k_in + 23) / 24;
+    if (ctx->fast) {
+        const int64_t nq = (bpr + 3) / 4;
+        const size_t smem = ctx->fl.total + 16 + (size_t)nq * 48 * 4 + kGemvRows * 4;
+        if (smem > 227 * 1024 || n_out > (1ll << 31)) return LLVQ_EUNSUPPORTED;
+        const int64_t tiles = (n_out + kGemvRows - 1) / kGemvRows;
+        unsigned g = (unsigned)std::min<int64_t>(tiles, ctx->sm_count);
+        const uint32_t* idx = static_cast<const uint32_t*>(d_idx);
+        if (y_dtype == LLVQ_BF16) {
+            if (!set_smem(gemv_fast_kernel<true>, smem)) return LLVQ_ECUDA;
+            gemv_fast_kernel<true><<<g, kFastThreads, smem, st>>>(fast_args(ctx), idx, d_gain_f16, n_out, k_in, bpr, d_x_bf16, d_y);
+        } else {
+            if (!set_smem(gemv_fast_kernel<false>, smem)) return LLVQ_ECUDA;
+            gemv_fast_kernel<false><<<g, kFastThreads, smem, st>>>(fast_args(ctx), idx, d_gain_f16, n_out, k_in, bpr, d_x_bf16, d_y);
+        }
+        return launch_status();
+    }
     size_t smem = (size_t)bpr * 25 * sizeof(float);
     if (smem > 200 * 1024 || n_out > (1ll << 31)) return LLVQ_EUNSUPPORTED;
     unsigned grid = (unsigned)((n_out + kGemvWarps - 1) / kGemvWarps);

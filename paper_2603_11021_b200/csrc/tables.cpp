@@ -207,3 +207,88 @@ bool build_tables(int m_lo, int m_hi, HostTables& t)
 }
 
 }  // namespace llvq
+
+namespace llvq {
+
+bool build_fast_image(const HostTables& t, FastLayout& L, std::vector<uint8_t>& img)
+{
+    const size_t ncls = t.desc.size();
+    if (t.W > 64 || t.W < 12 || ncls > 1024 || t.max_levels > kFastMaxLevels) return false;
+    auto up16 = [](size_t v) { return (uint32_t)((v + 15) & ~size_t(15)); };
+    // r16: k-subsets of 16 slots, k = 0..8
+    std::vector<uint16_t> r16;
+    uint32_t base16[48] = {0};
+    for (int k = 0; k <= 8; ++k) {
+        base16[k] = (uint32_t)r16.size();
+        for (uint32_t m = 0; m < 65536; ++m)
+            if (__builtin_popcount(m) == k) r16.push_back((uint16_t)m);
+    }
+    for (int k = 0; k <= 16; ++k) base16[16 + k] = t.pascal[16 * 25 + k];   // C(16, k)
+    L.golay = 0;
+    L.lut = up16(L.golay + 4096 * 4);
+    L.pascal = up16(L.lut + 4096 * 2);
+    L.base16 = up16(L.pascal + 625 * 4);
+    L.r16 = up16(L.base16 + 48 * 4);
+    L.pd6 = up16(L.r16 + r16.size() * 2);
+    L.off = up16(L.pd6 + 4096);
+    L.desc = up16(L.off + (ncls + 1) * 8);
+    L.total = up16(L.desc + ncls * kFastDescWords * 4);
+    L.lut_shift = (uint32_t)(t.W - 12);
+    L.ncls = (uint32_t)ncls;
+    L.W = (uint32_t)t.W;
+    img.assign(L.total, 0);
+    std::memcpy(img.data() + L.golay, t.golay.data(), 4096 * 4);
+    std::memcpy(img.data() + L.pascal, t.pascal, 625 * 4);
+    std::memcpy(img.data() + L.base16, base16, sizeof base16);
+    std::memcpy(img.data() + L.r16, r16.data(), r16.size() * 2);
+    // pd6
+    for (uint32_t f = 0; f < 64; ++f)
+        for (uint32_t s = 0; s < 64; ++s) {
+            uint32_t out = 0, src = s;
+            for (int b = 0; b < 6; ++b)
+                if ((f >> b) & 1u) { if (src & 1u) out |= 1u << b; src >>= 1; }
+            img[L.pd6 + (f << 6 | s)] = (uint8_t)out;
+        }
+    // class lookup by the top 12 bits of the index
+    uint16_t* lut = reinterpret_cast<uint16_t*>(img.data() + L.lut);
+    size_t c = 0;
+    for (uint32_t b = 0; b < 4096; ++b) {
+        u128 first = (u128)b << L.lut_shift;
+        while (c + 1 < ncls && t.offset[c + 1] <= first) ++c;
+        lut[b] = (uint16_t)c;
+    }
+    uint64_t* off = reinterpret_cast<uint64_t*>(img.data() + L.off);
+    for (size_t j = 0; j <= ncls; ++j) off[j] = (uint64_t)t.offset[j];
+    uint32_t* dw = reinterpret_cast<uint32_t*>(img.data() + L.desc);
+    for (size_t j = 0; j < ncls; ++j) {
+        const ClassDesc& d = t.desc[j];
+        uint32_t* w = dw + j * kFastDescWords;
+        const int nlev = d.nlev1 + d.nlev0;
+        if (nlev > kFastMaxLevels || nlev + 2 > 8) return false;
+        uint32_t flags = (d.parity ? 1u : 0u) | (d.signpar ? 2u : 0u) | (d.fill0 ? 4u : 0u) |
+                         ((d.fill1 & 2) ? 8u : 0u) | ((d.fill0 & 2) ? 16u : 0u);
+        w[0] = d.w | (uint32_t)d.B << 8 | flags << 16 | (uint32_t)d.nlev1 << 24 | (uint32_t)nlev << 28;
+        w[1] = d.goff | (uint32_t)d.A << 16;
+        w[2] = (uint32_t)d.magicA; w[3] = (uint32_t)(d.magicA >> 32);
+        uint8_t vals[8] = {d.fill0, d.fill1, 0, 0, 0, 0, 0, 0};
+        uint32_t nbytes = 0;
+        u128 p_after = t.info[j].card / ((u128)d.A << d.B);        // number of arrangements P
+        for (int l = 0; l < nlev; ++l) {
+            const LevelDesc& lv = d.lev[l];
+            if (lv.radix >= (1u << 22)) return false;
+            vals[2 + l] = lv.val;
+            w[8 + l] = lv.radix | (uint32_t)lv.k << 22 | (uint32_t)(2 + l) << 27 | ((lv.val & 2) ? 1u << 30 : 0u) | (lv.val ? 1u << 31 : 0u);
+            nbytes |= (uint32_t)lv.n << (8 * l);
+            if (l == 0) { w[6] = (uint32_t)lv.magic; w[7] = (uint32_t)(lv.magic >> 32); p_after = (p_after + lv.radix - 1) / lv.radix; }
+            else {
+                if (p_after >> 32) return false;                     // 32-bit quotient chain after the first step
+                w[11 + l] = (uint32_t)((1ull << 32) / lv.radix);
+            }
+        }
+        std::memcpy(&w[4], vals, 8);
+        w[15] = nbytes;
+    }
+    return true;
+}
+
+}  // namespace llvq

@@ -69,3 +69,43 @@ struct HostTables {
 bool build_tables(int m_lo, int m_hi, HostTables& out);
 
 }  // namespace llvq
+
+// ---------------------------------------------------------------------------
+// Shared-memory table image for codes with few classes ("fast path"): one
+// contiguous blob, copied into every CTA's shared memory by bulk copies.
+// ---------------------------------------------------------------------------
+namespace llvq {
+
+constexpr int kFastMaxLevels = 4;      // unranking steps per class on the fast path
+constexpr int kFastDescWords = 16;     // 64-byte class descriptor
+constexpr int kLowBits = 16;           // slots resolved by one table lookup in the subset unranking
+
+// Byte offsets of the parts of the image (all 16-byte aligned) and scalars the kernels need.
+struct FastLayout {
+    uint32_t golay;       // u32[4096]
+    uint32_t lut;         // u16[4096]  class of the first index of bucket (I >> lut_shift)
+    uint32_t pascal;      // u32[25*25]
+    uint32_t base16;      // u32[48]: [k] = first entry of the k-subsets in r16 (k <= 8); [16 + k] = C(16, k), k <= 16
+    uint32_t r16;         // u16[]: the k-subsets of 16 slots as bit masks, k = 0..8, each in numeric order
+    uint32_t pd6;         // u8[4096]: [f << 6 | s] = low bits of s deposited into the set bits of f
+    uint32_t off;         // u64[ncls + 1]
+    uint32_t desc;        // u32[ncls][kFastDescWords]
+    uint32_t total;       // bytes, multiple of 16
+    uint32_t lut_shift;
+    uint32_t ncls;
+    uint32_t W;
+};
+
+// Word layout of a fast descriptor:
+//  0: w | B << 8 | flags << 16 | nlev1 << 24 | nlev << 28
+//       flags: bit0 parity, bit1 signpar, bit2 fill0 is nonzero, bit3 fill1 has value bit 1, bit4 fill0 has value bit 1
+//  1: goff | A << 16
+//  2,3: magicA = floor((2^64-1)/A)
+//  4,5: absolute value of id 0..7 (one byte each): id 0 = fill0, id 1 = fill1, ids 2.. = levels in order
+//  6,7: magic of level 0 = floor((2^64-1)/radix0)
+//  8..11: level l: radix | k << 22 | id << 27 | (value bit 1) << 30 | (value nonzero) << 31
+//  12..14: floor(2^32 / radix) of levels 1..3
+//  15: n (free slots before the step) of levels 0..3, one byte each
+bool build_fast_image(const HostTables& t, FastLayout& layout, std::vector<uint8_t>& image);
+
+}  // namespace llvq
