@@ -91,11 +91,16 @@ __device__ __forceinline__ uint32_t deposit24(const uint8_t* pd6, uint32_t src, 
 // remaining t-subset of the low 16 slots is one table entry.  `top` = largest n in the warp.
 __device__ __forceinline__ uint32_t nth_subset(const FastSmem& T, uint32_t k, uint32_t rho, int top)
 {
-    uint32_t m = 0, t = k;
-    for (int pos = top - 1; pos >= 16; --pos) {
-        const uint32_t cnt = T.pascal[pos * 25 + t];
-        if (t > 0 && rho >= cnt) { rho -= cnt; m |= 1u << pos; --t; }
+    uint32_t m = 0;
+    const uint32_t* col = T.pascal + k;                 // column t of the table, walked down as elements are taken
+#pragma unroll
+    for (int pos = 23; pos >= 16; --pos) {
+        if (pos < top) {                                // warp-uniform
+            const uint32_t cnt = col[pos * 25];         // C(pos, t); column 0 is stored as 0xffffffff: never taken
+            if (rho >= cnt) { rho -= cnt; m |= 1u << pos; --col; }
+        }
     }
+    const uint32_t t = (uint32_t)(col - T.pascal);
     uint32_t idx, flip;
     if (t <= 8) { idx = T.base16[t] + rho; flip = 0u; }
     else        { idx = T.base16[16 - t] + (T.base16[16 + t] - 1u - rho); flip = 0xffffu; }

@@ -176,7 +176,8 @@ gemv_kernel(DevCode dc, const uint32_t* __restrict__ stream, const uint16_t* __r
 // kernel: [table image | mbarrier (16 bytes) | kernel-specific staging].
 // Persistent CTAs, one per SM.
 // ===========================================================================
-constexpr int kFastThreads = 512;
+constexpr int kFastThreads = 1024;      // decode / dequant kernels
+constexpr int kGemvThreads = 768;
 
 struct FastArgs {
     FastLayout L;
@@ -186,11 +187,19 @@ struct FastArgs {
     uint64_t n_points;              // N (fits 64 bits on the fast path)
 };
 
+// Field b of a stream of W-bit fields, W <= 64: at most three 32-bit words, the third only when the field reaches it.
 __device__ __forceinline__ uint64_t load_field(const uint32_t* __restrict__ stream, uint64_t b, int W)
 {
-    uint64_t lo, hi;
-    load_index(stream, b, W, lo, hi);
-    return lo;
+    const uint64_t bp = b * (uint64_t)W;
+    const uint32_t* p = stream + (bp >> 5);
+    const int sh = (int)(bp & 31);
+    const int last = sh + W;                                     // bits of the field counted from the first word
+    const uint32_t w0 = __ldg(p);
+    const uint32_t w1 = last > 32 ? __ldg(p + 1) : 0u;
+    const uint32_t w2 = last > 64 ? __ldg(p + 2) : 0u;
+    uint64_t v = (((uint64_t)w1 << 32) | w0) >> sh;
+    if (sh) v |= (uint64_t)w2 << (64 - sh);
+    return W < 64 ? v & ((1ull << W) - 1) : v;
 }
 
 #define FAST_PROLOGUE()                                                                         \
@@ -274,7 +283,7 @@ __device__ __forceinline__ void mma_bf16_16816(float c[4], uint32_t a0, uint32_t
 }
 
 template <bool kOutBf16>
-__global__ void __launch_bounds__(kFastThreads, 1)
+__global__ void __launch_bounds__(kGemvThreads, 1)
 gemv_fast_kernel(FastArgs fa, const uint32_t* __restrict__ stream, const uint16_t* __restrict__ gain,
                  int64_t n_out, int64_t k_in, int64_t bpr, const uint16_t* __restrict__ x, void* __restrict__ y)
 {
@@ -282,13 +291,13 @@ gemv_fast_kernel(FastArgs fa, const uint32_t* __restrict__ stream, const uint16_
     const int64_t nq = (bpr + 3) / 4;                               // units along K
     uint32_t* xs = reinterpret_cast<uint32_t*>(staging);            // [nq * 4][12] packed bf16 pairs of x
     float* acc = reinterpret_cast<float*>(xs + nq * 48);            // [kGemvRows]
-    for (int64_t i = threadIdx.x; i < nq * 48; i += kFastThreads) {
+    for (int64_t i = threadIdx.x; i < nq * 48; i += kGemvThreads) {
         const int64_t e = 2 * i;
         const uint32_t lo = e < k_in ? __ldg(x + e) : 0u, hi = e + 1 < k_in ? __ldg(x + e + 1) : 0u;
         xs[i] = lo | hi << 16;
     }
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, g = lane >> 2, t = lane & 3;
-    constexpr int kWarps = kFastThreads / 32;
+    constexpr int kWarps = kGemvThreads / 32;
     const int64_t ntiles = (n_out + kGemvRows - 1) / kGemvRows;
     for (int64_t tile = blockIdx.x; tile < ntiles; tile += gridDim.x) {
         if (threadIdx.x < kGemvRows) acc[threadIdx.x] = 0.f;
@@ -569,10 +578,10 @@ int llvq_gemv(const llvq_ctx* ctx, const void* d_idx, const uint16_t* d_gain_f16
         const uint32_t* idx = static_cast<const uint32_t*>(d_idx);
         if (y_dtype == LLVQ_BF16) {
             if (!set_smem(gemv_fast_kernel<true>, smem)) return LLVQ_ECUDA;
-            gemv_fast_kernel<true><<<g, kFastThreads, smem, st>>>(fast_args(ctx), idx, d_gain_f16, n_out, k_in, bpr, d_x_bf16, d_y);
+            gemv_fast_kernel<true><<<g, kGemvThreads, smem, st>>>(fast_args(ctx), idx, d_gain_f16, n_out, k_in, bpr, d_x_bf16, d_y);
         } else {
             if (!set_smem(gemv_fast_kernel<false>, smem)) return LLVQ_ECUDA;
-            gemv_fast_kernel<false><<<g, kFastThreads, smem, st>>>(fast_args(ctx), idx, d_gain_f16, n_out, k_in, bpr, d_x_bf16, d_y);
+            gemv_fast_kernel<false><<<g, kGemvThreads, smem, st>>>(fast_args(ctx), idx, d_gain_f16, n_out, k_in, bpr, d_x_bf16, d_y);
         }
         return launch_status();
     }

@@ -239,6 +239,8 @@ bool build_fast_image(const HostTables& t, FastLayout& L, std::vector<uint8_t>& 
     img.assign(L.total, 0);
     std::memcpy(img.data() + L.golay, t.golay.data(), 4096 * 4);
     std::memcpy(img.data() + L.pascal, t.pascal, 625 * 4);
+    for (int n = 0; n < 25; ++n)                           // column 0 is a sentinel in the image: "no element left to place"
+        reinterpret_cast<uint32_t*>(img.data() + L.pascal)[n * 25] = 0xffffffffu;
     std::memcpy(img.data() + L.base16, base16, sizeof base16);
     std::memcpy(img.data() + L.r16, r16.data(), r16.size() * 2);
     // pd6
