@@ -11,6 +11,7 @@
 
 #include "decode.cuh"
 #include "fast.cuh"
+#include "umma.cuh"
 #include "tables.h"
 
 using namespace llvq;
@@ -22,6 +23,8 @@ struct llvq_ctx {
     void* d_blob = nullptr;          // one allocation holding every device table
     unsigned long long* d_err = nullptr;
     int sm_count = 0;
+    float* d_scratch = nullptr;      // split-K accumulation buffer of the small-batch GEMM, kept all-zero between calls
+    uint32_t* d_counters = nullptr;  // per row tile arrival counters, kept zero between calls
     bool fast = false;               // tables fit shared memory: the fast kernels are used
     FastLayout fl{};
     const uint8_t* d_image = nullptr;
@@ -343,6 +346,183 @@ gemv_fast_kernel(FastArgs fa, const uint32_t* __restrict__ stream, const uint16_
     }
 }
 
+// ===========================================================================
+// llvq_gemm_small_batch: Y[b][i] = sum_k X[b][k] W[i][k] on the tensor cores.
+// A work item is a tile of 128 output rows x a range of K stages (96 columns = 4 blocks of 24 per row).
+// Per stage every thread dequantizes one block into the shared-memory A tile (bf16, K-major core-matrix
+// layout), the matching slice of X goes into the B tile, and one thread issues six tcgen05 MMAs
+// (M = 128, N = padded batch, K = 16) accumulating in tensor memory.  Two stages are in flight.
+// Split-K partial sums are added into a zero-initialised binary32 scratch [npad][n_out]; the last item
+// of a row tile converts it to bf16 and clears it again.
+// ===========================================================================
+constexpr int kGemmThreads = 512;
+constexpr int kGemmRows = 128;
+constexpr int kStageBlocks = 4;                       // column blocks per stage
+constexpr int kStageK = kStageBlocks * 24;            // 96
+constexpr int kMaxScratchRows = 65536;
+constexpr uint32_t kTmemCols = 64;
+
+struct GemmArgs {
+    int64_t n_out, k_in, bpr;
+    int batch, npad;
+    int nstages, split;
+    const uint16_t* x;
+    uint16_t* y;
+    float* scratch;            // [npad][scratch_ld] binary32, all zero on entry and on exit
+    int64_t scratch_ld;        // row tiles * 128
+    uint32_t* counters;        // [row tiles], zero on entry and on exit
+};
+
+template <bool kFast>
+__global__ void __launch_bounds__(kGemmThreads, 1)
+gemm_kernel(FastArgs fa, DevCode dc, const uint32_t* __restrict__ stream, const uint16_t* __restrict__ gain, GemmArgs ga)
+{
+    extern __shared__ __align__(128) uint8_t smem[];
+    const uint32_t img_bytes = kFast ? fa.L.total : 0u;
+    uint64_t* bar_img = reinterpret_cast<uint64_t*>(smem + img_bytes);
+    uint64_t* bar_free = bar_img + 1;                                     // [2]
+    uint64_t* bar_done = bar_img + 3;
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bar_img + 4);
+    uint32_t* last_flag = tmem_slot + 1;
+    const uint32_t a_off = (img_bytes + 64 + 1023) & ~1023u;
+    uint8_t* a_buf = smem + a_off;                                        // 2 x 24576
+    uint8_t* b_buf = a_buf + 2 * kGemmRows * kStageK * 2;                  // 2 x npad * 192
+    const uint32_t b_stage = (uint32_t)ga.npad * kStageK * 2;
+
+    FastSmem T{};
+    if (kFast) {
+        if (!fast_load_image(smem, fa.image, fa.L.total, bar_img, fa.flags)) return;
+        T = fast_view(smem, fa.L);
+    }
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    if (threadIdx.x == 0) {
+        mbar_init(&bar_free[0], 1); mbar_init(&bar_free[1], 1); mbar_init(bar_done, 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 0) tmem_alloc(tmem_slot, kTmemCols);
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = *tmem_slot;
+    const uint32_t idesc = instr_desc_bf16_m128((uint32_t)ga.npad);
+
+    const int64_t row_tiles = (ga.n_out + kGemmRows - 1) / kGemmRows;
+    const int64_t items = row_tiles * ga.split;
+    uint32_t gstage = 0, gitem = 0;
+    bool failed = false;
+    for (int64_t item = blockIdx.x; item < items && !failed; item += gridDim.x, ++gitem) {
+        const int64_t rt = item / ga.split;
+        const int f = (int)(item % ga.split);
+        const int s_begin = (int)((int64_t)f * ga.nstages / ga.split), s_end = (int)((int64_t)(f + 1) * ga.nstages / ga.split);
+        const int64_t row = rt * kGemmRows + warp * 8 + (lane & 7);
+        for (int s = s_begin; s < s_end; ++s, ++gstage) {
+            const uint32_t buf = gstage & 1u;
+            bool ok = true;
+            if (gstage >= 2) ok = mbar_wait(&bar_free[buf], ((gstage >> 1) - 1u) & 1u);     // the MMAs that read this buffer are done
+            if (__syncthreads_or(!ok)) { failed = true; break; }
+            // ---- A: dequantize one block of 24 weights
+            const int64_t cb = (int64_t)s * kStageBlocks + (lane >> 3);
+            const bool in = row < ga.n_out && cb < ga.bpr;
+            const uint64_t b = in ? (uint64_t)(row * ga.bpr + cb) : 0ull;
+            uint32_t w[12];
+            if (kFast) {
+                const uint64_t I = in ? load_field(stream, b, (int)fa.L.W) : 0ull;
+                const bool valid = in && I < fa.n_points;
+                if (in && !valid) atomicAdd(fa.bad_index, 1ull);
+                Decoded d;
+                fast_decode(T, I, valid, d);
+                expand_bf16(d, in ? gain_to_float(__ldg(gain + b)) : 0.f, w);
+            } else {
+                Point pt;
+#pragma unroll
+                for (int i = 0; i < 6; ++i) pt.w[i] = 0;
+                if (in) decode_field(dc, stream, b, pt);
+                const float g = in ? gain_to_float(__ldg(gain + b)) : 0.f;
+#pragma unroll
+                for (int j = 0; j < 12; ++j) {
+                    __nv_bfloat162 h = __halves2bfloat162(dequant(g, pt, 2 * j), dequant(g, pt, 2 * j + 1));
+                    w[j] = *reinterpret_cast<uint32_t*>(&h);
+                }
+            }
+            uint8_t* a_dst = a_buf + buf * (kGemmRows * kStageK * 2) + warp * 128 + (lane & 7) * 16;
+#pragma unroll
+            for (int j = 0; j < 3; ++j)
+                *reinterpret_cast<uint4*>(a_dst + (3 * (lane >> 3) + j) * 2048) = make_uint4(w[4 * j], w[4 * j + 1], w[4 * j + 2], w[4 * j + 3]);
+            // ---- B: the slice of X, 16-byte chunks (8 values along K)
+            for (int i = threadIdx.x; i < ga.npad * (kStageK / 8); i += kGemmThreads) {
+                const int kc = i / ga.npad, n = i % ga.npad;
+                const int64_t k = (int64_t)s * kStageK + kc * 8;
+                uint4 v = make_uint4(0, 0, 0, 0);
+                if (n < ga.batch && k < ga.k_in) v = __ldg(reinterpret_cast<const uint4*>(ga.x + (int64_t)n * ga.k_in + k));
+                *reinterpret_cast<uint4*>(b_buf + buf * b_stage + (uint32_t)kc * ga.npad * 16 + n * 16) = v;
+            }
+            fence_async_smem();
+            __syncthreads();
+            if (threadIdx.x == 0) {
+                tc_fence_after();
+                const uint32_t a_addr = smem_u32(a_buf + buf * (kGemmRows * kStageK * 2));
+                const uint32_t b_addr = smem_u32(b_buf + buf * b_stage);
+#pragma unroll
+                for (int j = 0; j < kStageK / 16; ++j)
+                    umma_bf16(tmem, smem_desc(a_addr + j * 4096, 2048, 128), smem_desc(b_addr + j * 2 * ga.npad * 16, ga.npad * 16, 128),
+                              idesc, (s > s_begin || j > 0) ? 1u : 0u);
+                umma_commit(&bar_free[buf]);
+                if (s == s_end - 1) umma_commit(bar_done);
+            }
+        }
+        if (failed) break;
+        // ---- epilogue: accumulator -> scratch (split-K) or Y
+        if (s_end > s_begin) {
+            const bool ok = mbar_wait(bar_done, gitem & 1u);
+            if (__syncthreads_or(!ok)) { failed = true; break; }
+            tc_fence_after();
+            if (warp < 4) {
+                const int64_t orow = rt * kGemmRows + warp * 32 + lane;
+                for (int c0 = 0; c0 < ga.npad; c0 += 16) {
+                    float v[16];
+                    tmem_ld16(tmem + ((uint32_t)(warp * 32) << 16) + (uint32_t)c0, v);
+                    if (orow < ga.n_out) {
+#pragma unroll
+                        for (int i = 0; i < 16; ++i) {
+                            const int n = c0 + i;
+                            if (n < ga.batch) {
+                                if (ga.split == 1) reinterpret_cast<__nv_bfloat16*>(ga.y)[(int64_t)n * ga.n_out + orow] = __float2bfloat16_rn(v[i]);
+                                else atomicAdd(ga.scratch + (int64_t)n * ga.scratch_ld + orow, v[i]);
+                            }
+                        }
+                    }
+                }
+            }
+            tc_fence_before();
+        } else {
+            --gitem;                                        // no MMA was committed for this item
+        }
+        if (ga.split > 1) {
+            __threadfence();
+            __syncthreads();
+            if (threadIdx.x == 0) *last_flag = (atomicAdd(ga.counters + rt, 1u) == (uint32_t)ga.split - 1u);
+            __syncthreads();
+            if (*last_flag) {
+                __threadfence();
+                for (int i = threadIdx.x; i < kGemmRows * ga.batch; i += kGemmThreads) {
+                    const int n = i / kGemmRows;
+                    const int64_t orow = rt * kGemmRows + (i % kGemmRows);
+                    if (orow < ga.n_out) {
+                        float* sp = ga.scratch + (int64_t)n * ga.scratch_ld + orow;
+                        reinterpret_cast<__nv_bfloat16*>(ga.y)[(int64_t)n * ga.n_out + orow] = __float2bfloat16_rn(__ldcg(sp));
+                        __stcg(sp, 0.f);
+                    }
+                }
+                if (threadIdx.x == 0) ga.counters[rt] = 0u;
+            }
+        }
+        __syncthreads();
+    }
+    if (failed && threadIdx.x == 0) atomicOr(fa.flags, 1u);
+    __syncthreads();
+    if (warp == 0) tmem_dealloc(tmem, kTmemCols);
+}
+
 FastArgs fast_args(const llvq_ctx* ctx)
 {
     FastArgs fa;
@@ -362,6 +542,58 @@ int check_common(const llvq_ctx* ctx, const void* d_idx)
     if (!ctx || !d_idx || ctx->device < 0) return LLVQ_EINVAL;
     if (!aligned(d_idx, 16)) return LLVQ_EALIGN;
     return LLVQ_OK;
+}
+
+int launch_status();
+
+int check_gemm_args(const llvq_ctx* ctx, const void* d_idx, const uint16_t* d_gain_f16, int64_t n_out, int64_t k_in,
+                    const uint16_t* d_x_bf16, int batch, const uint16_t* d_y_bf16)
+{
+    if (int e = check_common(ctx, d_idx)) return e;
+    if (!d_gain_f16 || !d_x_bf16 || !d_y_bf16 || n_out < 0 || k_in < 0 || batch < 1 || batch > 64) return LLVQ_EINVAL;
+    if (!aligned(d_gain_f16, 2) || !aligned(d_x_bf16, 16) || !aligned(d_y_bf16, 2) || (k_in & 7)) return LLVQ_EALIGN;
+    return LLVQ_OK;
+}
+
+// Enqueue the small-batch GEMM with the given split-K scratch ([npad][row tiles * 128] floats) and counters
+// ([row tiles]); both must be zero when the kernel starts and are zero again when it ends.
+int launch_gemm(const llvq_ctx* ctx, const void* d_idx, const uint16_t* d_gain_f16, int64_t n_out, int64_t k_in,
+                const uint16_t* d_x_bf16, int batch, uint16_t* d_y_bf16, float* scratch, uint32_t* counters, void* stream)
+{
+    if (n_out == 0) return LLVQ_OK;
+    DeviceGuard guard(ctx->device);
+    if (!guard.ok) return LLVQ_ECUDA;
+    cudaStream_t st = (cudaStream_t)stream;
+    if (k_in == 0) return cudaMemsetAsync(d_y_bf16, 0, (size_t)n_out * batch * 2, st) == cudaSuccess ? LLVQ_OK : LLVQ_ECUDA;
+    GemmArgs ga;
+    ga.n_out = n_out; ga.k_in = k_in; ga.bpr = (k_in + 23) / 24;
+    ga.batch = batch; ga.npad = (batch + 15) / 16 * 16;
+    ga.nstages = (int)((ga.bpr + kStageBlocks - 1) / kStageBlocks);
+    ga.x = d_x_bf16; ga.y = d_y_bf16; ga.scratch = scratch; ga.counters = counters;
+    // split K so that the work items fill the SMs evenly, keeping at least four stages per item
+    const int64_t row_tiles = (n_out + kGemmRows - 1) / kGemmRows;
+    ga.scratch_ld = row_tiles * kGemmRows;
+    int best = 1; double best_eff = 0.0;
+    for (int f = 1; f <= 64 && f * 4 <= std::max(ga.nstages, 4); ++f) {
+        const int64_t items = row_tiles * f;
+        const double eff = (double)items / (double)(((items + ctx->sm_count - 1) / ctx->sm_count) * ctx->sm_count);
+        if (eff > best_eff + 1e-9) { best_eff = eff; best = f; }
+    }
+    ga.split = best;
+    const int64_t items = row_tiles * ga.split;
+    const unsigned grid = (unsigned)std::min<int64_t>(items, ctx->sm_count);
+    const size_t img = ctx->fast ? ctx->fl.total : 0;
+    const size_t smem = ((img + 64 + 1023) & ~size_t(1023)) + 2 * kGemmRows * kStageK * 2 + 2 * (size_t)ga.npad * kStageK * 2;
+    if (smem > 227 * 1024) return LLVQ_EUNSUPPORTED;
+    const uint32_t* idx = static_cast<const uint32_t*>(d_idx);
+    if (ctx->fast) {
+        if (!set_smem(gemm_kernel<true>, smem)) return LLVQ_ECUDA;
+        gemm_kernel<true><<<grid, kGemmThreads, smem, st>>>(fast_args(ctx), ctx->dev, idx, d_gain_f16, ga);
+    } else {
+        if (!set_smem(gemm_kernel<false>, smem)) return LLVQ_ECUDA;
+        gemm_kernel<false><<<grid, kGemmThreads, smem, st>>>(fast_args(ctx), ctx->dev, idx, d_gain_f16, ga);
+    }
+    return launch_status();
 }
 
 int launch_status()
@@ -405,7 +637,9 @@ int llvq_create(llvq_ctx** out, int m_lo, int m_hi, int device)
     std::vector<uint8_t> image;
     ctx->fast = build_fast_image(h, ctx->fl, image);
     size_t o_img = up(o_err + 256);
-    size_t total = o_img + (ctx->fast ? image.size() : 0);
+    size_t o_cnt = up(o_img + (ctx->fast ? image.size() : 0));
+    size_t o_scr = up(o_cnt + (kMaxScratchRows / kGemmRows) * 4);
+    size_t total = o_scr + (size_t)64 * kMaxScratchRows * 4;
     std::vector<uint8_t> blob(total, 0);
     if (ctx->fast) std::memcpy(blob.data() + o_img, image.data(), image.size());
     std::memcpy(blob.data() + o_golay, h.golay.data(), 4096 * 4);
@@ -430,6 +664,8 @@ int llvq_create(llvq_ctx** out, int m_lo, int m_hi, int device)
     ctx->dev.nclasses = (int)ncls;
     ctx->dev.W = h.W;
     ctx->d_image = d + o_img;
+    ctx->d_counters = reinterpret_cast<uint32_t*>(d + o_cnt);
+    ctx->d_scratch = reinterpret_cast<float*>(d + o_scr);
     *out = ctx;
     return LLVQ_OK;
 }
@@ -602,8 +838,9 @@ int llvq_gemv(const llvq_ctx* ctx, const void* d_idx, const uint16_t* d_gain_f16
 int llvq_gemm_small_batch(const llvq_ctx* ctx, const void* d_idx, const uint16_t* d_gain_f16, int64_t n_out, int64_t k_in,
                           const uint16_t* d_x_bf16, int batch, uint16_t* d_y_bf16, void* stream)
 {
-    (void)ctx; (void)d_idx; (void)d_gain_f16; (void)n_out; (void)k_in; (void)d_x_bf16; (void)batch; (void)d_y_bf16; (void)stream;
-    return LLVQ_EUNSUPPORTED;
+    if (int e = check_gemm_args(ctx, d_idx, d_gain_f16, n_out, k_in, d_x_bf16, batch, d_y_bf16)) return e;
+    if (n_out > kMaxScratchRows) return LLVQ_EUNSUPPORTED;
+    return launch_gemm(ctx, d_idx, d_gain_f16, n_out, k_in, d_x_bf16, batch, d_y_bf16, ctx->d_scratch, ctx->d_counters, stream);
 }
 
 int llvq_last_error(llvq_ctx* ctx, void* stream, uint64_t* n_bad_index, uint32_t* flags)

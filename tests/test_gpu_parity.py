@@ -230,3 +230,66 @@ def test_argument_checks(lib, ctxs):
     assert L.llvq_gemv(ctx._h, idx.data_ptr(), g.data_ptr(), 2, 24, w.data_ptr(), w.data_ptr(), 9, None) == 1
     assert L.llvq_gemv(ctx._h, idx.data_ptr(), g.data_ptr(), 2, 10_000_000, w.data_ptr(), w.data_ptr(), 0, None) == 3
     torch.cuda.synchronize()
+
+
+# --------------------------------------------------------------------------
+# small-batch GEMM on the tensor cores
+# --------------------------------------------------------------------------
+def _gemm_check(lib, ctx, o, n_out, k_in, batch, seed, repeat=1):
+    stream, gain, _ = gen.make_layer(o.N, o.W, n_out, k_in, 1, seed=seed)
+    X = gen.normal_bf16((batch, k_in), seed=seed)
+    want = o.gemm(stream, gain, n_out, k_in, X, threads=8)
+    d_idx, d_gain, d_x = to_dev_u8(stream), to_dev_f16(gain), to_dev_bf16(X)
+    for _ in range(repeat):
+        y = lib.llvq_gemm_small_batch(ctx, d_idx, d_gain, n_out, k_in, d_x)
+        torch.cuda.synchronize()
+        assert lib.llvq_last_error(ctx) == (0, 0)
+        got = y.float().cpu().numpy()
+        assert got.shape == (batch, n_out)
+        scale = np.abs(want).max()
+        err = np.abs(got - want) / np.maximum(np.abs(want), 1e-3 * scale)
+        assert err.max() <= TOL_BF16_OUT, (err.max(), np.unravel_index(err.argmax(), err.shape))
+
+
+@pytest.mark.parametrize("n_out,k_in,batch", [(128, 96, 16), (300, 1000, 16), (300, 1000, 64), (129, 192, 1),
+                                              (257, 4104, 7), (640, 2048, 33), (100, 24, 64)])
+def test_gemm_small_batch_2bit(lib, ctxs, oracle_mod, n_out, k_in, batch):
+    _gemm_check(lib, ctxs[(2, 13)], _oracle(oracle_mod)((2, 13)), n_out, k_in, batch, seed=7, repeat=2)
+
+
+@pytest.mark.parametrize("code,n_out,k_in,batch", [((2, 53), 200, 1000, 16), ((2, 53), 130, 480, 64), ((2, 2), 256, 768, 5)])
+def test_gemm_small_batch_other_codes(lib, ctxs, oracle_mod, code, n_out, k_in, batch):
+    _gemm_check(lib, ctxs[code], _oracle(oracle_mod)(code), n_out, k_in, batch, seed=8)
+
+
+def test_gemm_exact_integer_case(lib, ctxs, oracle_mod):
+    # gains = 1, X = 0/1 patterns: every partial sum is a small integer, exact in binary32 and in bf16
+    o = _oracle(oracle_mod)((2, 13))
+    ctx = ctxs[(2, 13)]
+    n_out, k_in, batch = 200, 480, 16
+    stream, _, nblocks = gen.make_layer(o.N, o.W, n_out, k_in, 1, seed=9)
+    ones = np.full(nblocks, 0x3C00, dtype=np.uint16)
+    pts, _ = o.decode_stream(stream, nblocks)
+    Wint = pts.reshape(n_out, -1)[:, :k_in].astype(np.int64)
+    X = np.zeros((batch, k_in), dtype=np.float32)
+    for b in range(batch):
+        X[b, b * 30:(b + 1) * 30:3] = 1.0
+    y = lib.llvq_gemm_small_batch(ctx, to_dev_u8(stream), to_dev_f16(ones), n_out, k_in, to_dev_bf16(gen.f32_to_bf16_bits(X)))
+    torch.cuda.synchronize()
+    assert np.array_equal(y.float().cpu().numpy().astype(np.int64), X.astype(np.int64) @ Wint.T)
+
+
+def test_gemm_matches_gemv_rows(lib, ctxs, oracle_mod):
+    # batch rows are independent: row b of the GEMM equals the GEMV with x = X[b] up to accumulation order
+    o = _oracle(oracle_mod)((2, 13))
+    ctx = ctxs[(2, 13)]
+    n_out, k_in, batch = 384, 1536, 16
+    stream, gain, _ = gen.make_layer(o.N, o.W, n_out, k_in, 1, seed=10)
+    X = gen.normal_bf16((batch, k_in), seed=10)
+    d = (to_dev_u8(stream), to_dev_f16(gain))
+    Y = lib.llvq_gemm_small_batch(ctx, *d, n_out, k_in, to_dev_bf16(X)).float()
+    for b in (0, 7, 15):
+        y = lib.llvq_gemv(ctx, *d, n_out, k_in, to_dev_bf16(X[b]))
+        torch.cuda.synchronize()
+        ref = y.cpu().numpy().astype(np.float64)
+        assert gemv_error(Y[b].cpu().numpy(), ref) <= 2.0 ** -8 + 1e-4
