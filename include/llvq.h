@@ -135,6 +135,31 @@ int llvq_gemm_small_batch(const llvq_ctx* ctx, const void* d_idx, const uint16_t
                           int batch, uint16_t* d_y_bf16, void* stream);
 
 /*
+ * llvq_gemm_small_batch for callers that cannot allocate device memory.  (The paper has no
+ * counterpart: this is a packaging variant of the call above, same arguments, same result.)
+ *
+ * Who needs it: code that runs after the application has handed all device memory to its own
+ * pool, code inside a latency-critical decode loop where the implicit device synchronisation of
+ * cudaMalloc / cudaFree is not acceptable, and plug-ins whose host only lets them launch work.
+ * llvq_gemm_small_batch itself takes its split-K scratch from a buffer the context allocated at
+ * llvq_create; this variant instead uses a fixed array compiled into the library (1 MiB + 512
+ * bytes of device memory on every GPU that loads the library, held until the process exits), and
+ * calls no allocating routine at all.
+ *
+ * Limits: ceil(n_out / 128) <= 128 and  roundup(batch, 16) * roundup(n_out, 128) <= 262144
+ * (for example 4096 rows at batch 64, or 16384 rows at batch 16); larger problems return
+ * LLVQ_EUNSUPPORTED and launch nothing.
+ * The first call on a device looks up the array's device address (cudaGetSymbolAddress with that
+ * device current); make that first call outside any stream capture.
+ * All calls share the one array: each call clears the part it uses on `stream` before the kernel
+ * runs, so calls must be ordered on the GPU (same stream, or dependent streams); calls that
+ * overlap in time race on the array and give wrong results.
+ */
+int llvq_gemm_small_batch_noalloc(const llvq_ctx* ctx, const void* d_idx, const uint16_t* d_gain_f16,
+                                  int64_t n_out, int64_t k_in, const uint16_t* d_x_bf16,
+                                  int batch, uint16_t* d_y_bf16, void* stream);
+
+/*
  * Synchronises `stream`, then reports and clears the device-side error state:
  * *n_bad_index = number of fields with I >= N seen since the last call,
  * *flags = OR of LLVQ_FLAG_* bits.  Either output pointer may be NULL.

@@ -15,7 +15,7 @@ import torch
 from .build import LIB
 
 __all__ = [
-    "Context", "llvq_decode_blocks", "llvq_dequant_matrix", "llvq_gemv", "llvq_gemm_small_batch",
+    "Context", "llvq_decode_blocks", "llvq_dequant_matrix", "llvq_gemv", "llvq_gemm_small_batch", "llvq_gemm_small_batch_noalloc",
     "llvq_last_error", "LlvqError", "EXPORTS", "load_library",
     "LLVQ_LAYOUT_FLAT", "LLVQ_LAYOUT_ROWWISE", "LLVQ_F32", "LLVQ_BF16",
 ]
@@ -28,7 +28,8 @@ _STATUS = {0: "LLVQ_OK", 1: "LLVQ_EINVAL", 2: "LLVQ_EALIGN", 3: "LLVQ_EUNSUPPORT
 # every symbol include/llvq.h declares
 EXPORTS = [
     "llvq_create", "llvq_destroy", "llvq_index_bits", "llvq_num_points", "llvq_num_classes", "llvq_index_bytes",
-    "llvq_decode_blocks", "llvq_dequant_matrix", "llvq_gemv", "llvq_gemm_small_batch", "llvq_last_error",
+    "llvq_decode_blocks", "llvq_dequant_matrix", "llvq_gemv", "llvq_gemm_small_batch", "llvq_gemm_small_batch_noalloc",
+    "llvq_last_error",
 ]
 
 
@@ -62,6 +63,7 @@ def load_library() -> ctypes.CDLL:
     lib.llvq_dequant_matrix.argtypes = [vp, vp, vp, i64, i64, ctypes.c_int, vp, i64, vp]
     lib.llvq_gemv.argtypes = [vp, vp, vp, i64, i64, vp, vp, ctypes.c_int, vp]
     lib.llvq_gemm_small_batch.argtypes = [vp, vp, vp, i64, i64, vp, ctypes.c_int, vp, vp]
+    lib.llvq_gemm_small_batch_noalloc.argtypes = [vp, vp, vp, i64, i64, vp, ctypes.c_int, vp, vp]
     lib.llvq_last_error.argtypes = [vp, vp, ctypes.POINTER(u64), ctypes.POINTER(ctypes.c_uint32)]
     lib.llvq_class_info.argtypes = [vp, ctypes.c_int, vp, vp, vp, vp, vp, vp]
     lib.llvq_golay_table.argtypes = [vp, vp]
@@ -190,6 +192,20 @@ def llvq_gemm_small_batch(ctx: Context, d_idx: torch.Tensor, d_gain: torch.Tenso
     nblocks = n_out * ((k_in + 23) // 24)
     assert d_gain.numel() >= nblocks and d_idx.numel() * d_idx.element_size() >= ctx.index_bytes(nblocks)
     _check("llvq_gemm_small_batch", ctx._lib.llvq_gemm_small_batch(
+        ctx._h, _dev(d_idx, "d_idx"), _dev(d_gain, "d_gain"), n_out, k_in, _dev(d_x, "d_x"), batch, _dev(d_y, "d_y"), _stream_ptr(stream)))
+    return d_y
+
+
+def llvq_gemm_small_batch_noalloc(ctx: Context, d_idx: torch.Tensor, d_gain: torch.Tensor, n_out: int, k_in: int,
+                                  d_x: torch.Tensor, d_y: torch.Tensor, stream=None):
+    """Same product as ``llvq_gemm_small_batch`` for callers that must not allocate device memory: the
+    library uses a fixed built-in scratch array instead of allocated memory, and this wrapper does not allocate
+    either, so the output tensor ``d_y`` (bf16 [batch, n_out]) has to be passed in.  Sizes beyond the built-in
+    array (see ``include/llvq.h``) raise ``LlvqError`` with LLVQ_EUNSUPPORTED.  Calls must not overlap on the GPU."""
+    assert d_x.dtype == torch.bfloat16 and d_x.dim() == 2 and d_x.shape[1] == k_in and d_gain.dtype == torch.float16
+    batch = d_x.shape[0]
+    assert d_y.dtype == torch.bfloat16 and d_y.numel() >= batch * n_out
+    _check("llvq_gemm_small_batch_noalloc", ctx._lib.llvq_gemm_small_batch_noalloc(
         ctx._h, _dev(d_idx, "d_idx"), _dev(d_gain, "d_gain"), n_out, k_in, _dev(d_x, "d_x"), batch, _dev(d_y, "d_y"), _stream_ptr(stream)))
     return d_y
 

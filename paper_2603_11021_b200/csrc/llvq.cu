@@ -6,6 +6,7 @@
 #include <algorithm>
 #include <cstdio>
 #include <cstring>
+#include <mutex>
 #include <new>
 #include <vector>
 
@@ -841,6 +842,49 @@ int llvq_gemm_small_batch(const llvq_ctx* ctx, const void* d_idx, const uint16_t
     if (int e = check_gemm_args(ctx, d_idx, d_gain_f16, n_out, k_in, d_x_bf16, batch, d_y_bf16)) return e;
     if (n_out > kMaxScratchRows) return LLVQ_EUNSUPPORTED;
     return launch_gemm(ctx, d_idx, d_gain_f16, n_out, k_in, d_x_bf16, batch, d_y_bf16, ctx->d_scratch, ctx->d_counters, stream);
+}
+
+
+// ---------------------------------------------------------------------------
+// llvq_gemm_small_batch_noalloc: the small-batch GEMM for callers that must not allocate.
+// Its split-K scratch is this fixed array, which every GPU that loads the library carries
+// until the process exits.  Layout: [row-tile counters: 512 bytes][binary32 partial sums: 1 MiB].
+// ---------------------------------------------------------------------------
+constexpr int kNoallocMaxRowTiles = 128;                          // 128 tiles x 128 rows = 16384 output rows
+constexpr size_t kNoallocCounterBytes = kNoallocMaxRowTiles * sizeof(uint32_t);
+constexpr size_t kNoallocScratchFloats = 262144;                  // padded batch x padded rows must fit: 1 MiB
+static __device__ __align__(256) unsigned char g_noalloc_scratch[kNoallocCounterBytes + kNoallocScratchFloats * sizeof(float)];
+
+int llvq_gemm_small_batch_noalloc(const llvq_ctx* ctx, const void* d_idx, const uint16_t* d_gain_f16, int64_t n_out, int64_t k_in,
+                                  const uint16_t* d_x_bf16, int batch, uint16_t* d_y_bf16, void* stream)
+{
+    if (int e = check_gemm_args(ctx, d_idx, d_gain_f16, n_out, k_in, d_x_bf16, batch, d_y_bf16)) return e;
+    const int64_t row_tiles = (n_out + kGemmRows - 1) / kGemmRows;
+    const int64_t npad = (batch + 15) / 16 * 16;
+    if (row_tiles > kNoallocMaxRowTiles || npad * row_tiles * kGemmRows > (int64_t)kNoallocScratchFloats) return LLVQ_EUNSUPPORTED;
+    if (n_out == 0) return LLVQ_OK;
+    if (ctx->device >= 64) return LLVQ_EUNSUPPORTED;
+    DeviceGuard guard(ctx->device);
+    if (!guard.ok) return LLVQ_ECUDA;
+    // The array's name is only a host-side handle: ask the runtime, once per device and with that device
+    // current, for the address the kernels can use.
+    static std::mutex lock;
+    static unsigned char* device_ptr[64] = {nullptr};
+    unsigned char* base;
+    {
+        std::lock_guard<std::mutex> hold(lock);
+        if (!device_ptr[ctx->device]) {
+            void* p = nullptr;
+            if (cudaGetSymbolAddress(&p, g_noalloc_scratch) != cudaSuccess || !p) return LLVQ_ECUDA;
+            device_ptr[ctx->device] = static_cast<unsigned char*>(p);
+        }
+        base = device_ptr[ctx->device];
+    }
+    // The array keeps whatever the previous call (or an aborted one) left: clear the part this call uses.
+    const size_t used = kNoallocCounterBytes + (size_t)(npad * row_tiles * kGemmRows) * sizeof(float);
+    if (cudaMemsetAsync(base, 0, used, (cudaStream_t)stream) != cudaSuccess) return LLVQ_ECUDA;
+    return launch_gemm(ctx, d_idx, d_gain_f16, n_out, k_in, d_x_bf16, batch, d_y_bf16,
+                       reinterpret_cast<float*>(base + kNoallocCounterBytes), reinterpret_cast<uint32_t*>(base), stream);
 }
 
 int llvq_last_error(llvq_ctx* ctx, void* stream, uint64_t* n_bad_index, uint32_t* flags)
