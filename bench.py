@@ -124,6 +124,26 @@ class ClockSampler:
         return {"sm_mhz": med, "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons), "samples": len(self.samples)}
 
 
+def max_over_ranks(value: float, dist, device) -> float:
+    """Max of a per-rank scalar over all ranks (identity without a process group)."""
+    if dist is None:
+        return float(value)
+    import torch
+    t = torch.tensor([float(value)], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def whole_job_value(world: int, bytes_per_rank_step: int, ms_per_step: float) -> float:
+    """Weak scaling: every rank moves the same algorithmic bytes per step; GB/s of the whole job."""
+    return world * bytes_per_rank_step / (ms_per_step * 1e-3) / 1e9
+
+
+def rank_seed(rank: int, copy: int, layer: int) -> int:
+    """Distinct synthetic layers per rank / copy / layer."""
+    return 1000 * rank + 10 * copy + layer
+
+
 def run_reference(args) -> None:
     """The CPU oracle, as it stands, on the host cores: the slow baseline arm."""
     rank = int(os.environ.get("RANK", "0"))
@@ -214,7 +234,7 @@ def main() -> None:
     for c in range(copies):
         dev, host = [], []
         for li, (n, k) in enumerate(LAYERS):
-            stream, gain, x, nblocks = host_layer(n, k, seed=1000 * rank + 10 * c + li)
+            stream, gain, x, nblocks = host_layer(n, k, seed=rank_seed(rank, c, li))
             h = (torch.from_numpy(stream).pin_memory(), torch.from_numpy(gain.view(np.float16)).pin_memory(),
                  torch.from_numpy(x.view(np.int16)).view(torch.bfloat16).pin_memory())
             host.append(h)
@@ -247,13 +267,9 @@ def main() -> None:
             step(i)
         ev1.record()
         barrier()
-    ms_total = ev0.elapsed_time(ev1)
-    if dist is not None:
-        t = torch.tensor([ms_total], device="cuda")
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms_total = float(t.item())
+    ms_total = max_over_ranks(ev0.elapsed_time(ev1), dist, "cuda")
     ms_per_step = ms_total / args.steps
-    value = world * step_bytes / (ms_per_step * 1e-3) / 1e9
+    value = whole_job_value(world, step_bytes, ms_per_step)
     timed_launches = launches
 
     # per-layer device time of the kernel (events around each launch, same rotation)
@@ -299,12 +315,8 @@ def main() -> None:
         e2e_step(i)
     ev1.record()
     barrier()
-    e2e_ms = ev0.elapsed_time(ev1) / e2e_steps
-    if dist is not None:
-        t = torch.tensor([e2e_ms], device="cuda")
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        e2e_ms = float(t.item())
-    e2e_value = world * step_bytes / (e2e_ms * 1e-3) / 1e9
+    e2e_ms = max_over_ranks(ev0.elapsed_time(ev1) / e2e_steps, dist, "cuda")
+    e2e_value = whole_job_value(world, step_bytes, e2e_ms)
 
     bad, flags = P.llvq_last_error(ctx)
     if bad or flags:
