@@ -11,14 +11,15 @@
 namespace llvq {
 
 constexpr uint32_t kFullMask = 0xffffffffu;
+constexpr int kPascalToBase14 = 2512;     // byte distance from pascal[t] to base14[t] in the table image
 
 // Pointers into the CTA's copy of the table image.
 struct FastSmem {
     const uint32_t* golay;
     const uint16_t* lut;
     const uint32_t* pascal;
-    const uint32_t* base16;
-    const uint16_t* r16;
+    const uint32_t* base14;
+    const uint16_t* r14;
     const uint8_t* pd6;
     const uint64_t* off;
     const uint32_t* desc;
@@ -31,8 +32,8 @@ __device__ __forceinline__ FastSmem fast_view(const uint8_t* smem, const FastLay
     T.golay = reinterpret_cast<const uint32_t*>(smem + L.golay);
     T.lut = reinterpret_cast<const uint16_t*>(smem + L.lut);
     T.pascal = reinterpret_cast<const uint32_t*>(smem + L.pascal);
-    T.base16 = reinterpret_cast<const uint32_t*>(smem + L.base16);
-    T.r16 = reinterpret_cast<const uint16_t*>(smem + L.r16);
+    T.base14 = reinterpret_cast<const uint32_t*>(smem + L.base14);
+    T.r14 = reinterpret_cast<const uint16_t*>(smem + L.r14);
     T.pd6 = smem + L.pd6;
     T.off = reinterpret_cast<const uint64_t*>(smem + L.off);
     T.desc = reinterpret_cast<const uint32_t*>(smem + L.desc);
@@ -87,24 +88,38 @@ __device__ __forceinline__ uint32_t deposit24(const uint8_t* pd6, uint32_t src, 
 }
 
 // The rho-th k-subset of the slots {0..n-1} in combinatorial-number-system order (numeric
-// order of the bit masks).  Slots >= 16 are decided one at a time against C(slot, t); the
-// remaining t-subset of the low 16 slots is one table entry.  `top` = largest n in the warp.
+// order of the bit masks).  Slots >= 14 are decided one at a time against C(slot, t); the
+// remaining t-subset of the low 14 slots is one table entry.  `top` (warp-uniform) bounds n.
+template <int kOff>
+__device__ __forceinline__ uint32_t lds_at(uint32_t addr)
+{
+    uint32_t v;
+    asm volatile("ld.shared.u32 %0, [%1+%2];" : "=r"(v) : "r"(addr), "n"(kOff));
+    return v;
+}
+
+// One slot decision: take slot kPos iff at least C(kPos, t) subsets come before (t = elements still to place).
+template <int kPos>
+__device__ __forceinline__ void subset_step(uint32_t& col, uint32_t& rho, uint32_t& m, int top)
+{
+    if (kPos < top) {                                   // warp-uniform
+        const uint32_t cnt = lds_at<kPos * 100>(col);   // C(kPos, t); column 0 is stored as 0xffffffff: never taken
+        if (rho >= cnt) { rho -= cnt; m |= 1u << kPos; col -= 4u; }
+    }
+}
+
 __device__ __forceinline__ uint32_t nth_subset(const FastSmem& T, uint32_t k, uint32_t rho, int top)
 {
+    static_assert(kLowBits == 14, "the slot decisions below cover slots 23..14");
     uint32_t m = 0;
-    const uint32_t* col = T.pascal + k;                 // column t of the table, walked down as elements are taken
-#pragma unroll
-    for (int pos = 23; pos >= 16; --pos) {
-        if (pos < top) {                                // warp-uniform
-            const uint32_t cnt = col[pos * 25];         // C(pos, t); column 0 is stored as 0xffffffff: never taken
-            if (rho >= cnt) { rho -= cnt; m |= 1u << pos; --col; }
-        }
-    }
-    const uint32_t t = (uint32_t)(col - T.pascal);
-    uint32_t idx, flip;
-    if (t <= 8) { idx = T.base16[t] + rho; flip = 0u; }
-    else        { idx = T.base16[16 - t] + (T.base16[16 + t] - 1u - rho); flip = 0xffffu; }
-    return m | ((uint32_t)T.r16[idx] ^ flip);
+    // byte address (shared window) of C(0, t); it walks down one column each time an element is taken
+    uint32_t col = smem_addr(T.pascal) + k * 4u;
+    subset_step<23>(col, rho, m, top); subset_step<22>(col, rho, m, top); subset_step<21>(col, rho, m, top);
+    subset_step<20>(col, rho, m, top); subset_step<19>(col, rho, m, top); subset_step<18>(col, rho, m, top);
+    subset_step<17>(col, rho, m, top); subset_step<16>(col, rho, m, top); subset_step<15>(col, rho, m, top);
+    subset_step<14>(col, rho, m, top);
+    const uint32_t first = lds_at<kPascalToBase14>(col);   // base14[t] sits right after the 625-entry Pascal table
+    return m | (uint32_t)T.r14[first + rho];
 }
 
 // Result of the index -> point map in a form the consumers expand cheaply:
@@ -116,12 +131,18 @@ struct Decoded {
     uint32_t vals_lo, vals_hi;     // absolute value of id 0..3 / 4..7, one byte each
 };
 
-__device__ __forceinline__ void fast_decode(const FastSmem& T, uint64_t I, bool valid, Decoded& d)
+// S2: class of index I (< N) and its class-local index.
+__device__ __forceinline__ uint32_t fast_find_class(const FastSmem& T, uint64_t I, uint64_t& local)
 {
-    // S2: class lookup
-    uint32_t cls = valid ? T.lut[(uint32_t)(I >> T.lut_shift)] : 0u;
-    if (valid) while (I >= T.off[cls + 1]) ++cls;
-    const uint64_t local = valid ? I - T.off[cls] : 0ull;
+    uint32_t cls = T.lut[(uint32_t)(I >> T.lut_shift)];
+    while (I >= T.off[cls + 1]) ++cls;
+    local = I - T.off[cls];
+    return cls;
+}
+
+// S3-S6 for any class; `mask` = the lanes of the warp that call this together.
+__device__ __forceinline__ void fast_decode_local(const FastSmem& T, uint32_t cls, uint64_t local, bool valid, uint32_t mask, Decoded& d)
+{
     const uint4* D = reinterpret_cast<const uint4*>(T.desc + cls * kFastDescWords);
     const uint4 h = D[0], v = D[1], lw = D[2], mg = D[3];
     const uint32_t w = h.x & 0xff, B = (h.x >> 8) & 0xff, flags = (h.x >> 16) & 0xff;
@@ -154,7 +175,7 @@ __device__ __forceinline__ void fast_decode(const FastSmem& T, uint64_t I, bool 
     uint32_t p32 = 0;
     const uint32_t lwords[4] = {lw.x, lw.y, lw.z, lw.w};
     const uint32_t magics[4] = {0u, mg.x, mg.y, mg.z};
-    const int maxlev = __reduce_max_sync(kFullMask, nlev);
+    const int maxlev = __reduce_max_sync(mask, nlev);
 #pragma unroll
     for (int l = 0; l < kFastMaxLevels; ++l) {
         if (l < maxlev) {
@@ -181,7 +202,7 @@ __device__ __forceinline__ void fast_decode(const FastSmem& T, uint64_t I, bool 
             }
             if (!active) rho = 0u;
             const uint32_t n = active ? (mg.w >> (8 * l)) & 0xffu : 0u;
-            const int top = __reduce_max_sync(kFullMask, n);
+            const int top = __reduce_max_sync(mask, n);
             const uint32_t rel = nth_subset(T, k, rho, top);
             const uint32_t a = deposit24(T.pd6, rel, freem);
             freem ^= a;
@@ -209,6 +230,13 @@ __device__ __forceinline__ void fast_decode(const FastSmem& T, uint64_t I, bool 
     if (!valid) { p0 = p1 = p2 = 0; neg = 0; }
     d.p0 = p0; d.p1 = p1; d.p2 = p2; d.neg = neg;
     d.vals_lo = valid ? v.x : 0u; d.vals_hi = valid ? v.y : 0u;
+}
+
+__device__ __forceinline__ void fast_decode(const FastSmem& T, uint64_t I, bool valid, Decoded& d)
+{
+    uint64_t local = 0;
+    const uint32_t cls = valid ? fast_find_class(T, I, local) : 0u;
+    fast_decode_local(T, cls, local, valid, kFullMask, d);
 }
 
 // ---- expansion helpers -------------------------------------------------------

@@ -215,21 +215,21 @@ bool build_fast_image(const HostTables& t, FastLayout& L, std::vector<uint8_t>& 
     const size_t ncls = t.desc.size();
     if (t.W > 64 || t.W < 12 || ncls > 1024 || t.max_levels > kFastMaxLevels) return false;
     auto up16 = [](size_t v) { return (uint32_t)((v + 15) & ~size_t(15)); };
-    // r16: k-subsets of 16 slots, k = 0..8
-    std::vector<uint16_t> r16;
-    uint32_t base16[48] = {0};
-    for (int k = 0; k <= 8; ++k) {
-        base16[k] = (uint32_t)r16.size();
-        for (uint32_t m = 0; m < 65536; ++m)
-            if (__builtin_popcount(m) == k) r16.push_back((uint16_t)m);
+    // r14: all k-subsets of 14 slots, grouped by k, each group in numeric order
+    std::vector<uint16_t> r14;
+    uint32_t base14[16] = {0};
+    for (int k = 0; k <= kLowBits; ++k) {
+        base14[k] = (uint32_t)r14.size();
+        for (uint32_t m = 0; m < (1u << kLowBits); ++m)
+            if (__builtin_popcount(m) == k) r14.push_back((uint16_t)m);
     }
-    for (int k = 0; k <= 16; ++k) base16[16 + k] = t.pascal[16 * 25 + k];   // C(16, k)
     L.golay = 0;
     L.lut = up16(L.golay + 4096 * 4);
     L.pascal = up16(L.lut + 4096 * 2);
-    L.base16 = up16(L.pascal + 625 * 4);
-    L.r16 = up16(L.base16 + 48 * 4);
-    L.pd6 = up16(L.r16 + r16.size() * 2);
+    L.base14 = up16(L.pascal + 625 * 4);
+    if (L.base14 - L.pascal != 2512) return false;                      // the kernels address base14 relative to pascal
+    L.r14 = up16(L.base14 + 16 * 4);
+    L.pd6 = up16(L.r14 + r14.size() * 2);
     L.off = up16(L.pd6 + 4096);
     L.desc = up16(L.off + (ncls + 1) * 8);
     L.total = up16(L.desc + ncls * kFastDescWords * 4);
@@ -241,8 +241,8 @@ bool build_fast_image(const HostTables& t, FastLayout& L, std::vector<uint8_t>& 
     std::memcpy(img.data() + L.pascal, t.pascal, 625 * 4);
     for (int n = 0; n < 25; ++n)                           // column 0 is a sentinel in the image: "no element left to place"
         reinterpret_cast<uint32_t*>(img.data() + L.pascal)[n * 25] = 0xffffffffu;
-    std::memcpy(img.data() + L.base16, base16, sizeof base16);
-    std::memcpy(img.data() + L.r16, r16.data(), r16.size() * 2);
+    std::memcpy(img.data() + L.base14, base14, sizeof base14);
+    std::memcpy(img.data() + L.r14, r14.data(), r14.size() * 2);
     // pd6
     for (uint32_t f = 0; f < 64; ++f)
         for (uint32_t s = 0; s < 64; ++s) {

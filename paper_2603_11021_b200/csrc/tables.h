@@ -78,15 +78,16 @@ namespace llvq {
 
 constexpr int kFastMaxLevels = 4;      // unranking steps per class on the fast path
 constexpr int kFastDescWords = 16;     // 64-byte class descriptor
-constexpr int kLowBits = 16;           // slots resolved by one table lookup in the subset unranking
+constexpr int kLowBits = 14;           // slots resolved by one table lookup in the subset unranking
+
 
 // Byte offsets of the parts of the image (all 16-byte aligned) and scalars the kernels need.
 struct FastLayout {
     uint32_t golay;       // u32[4096]
     uint32_t lut;         // u16[4096]  class of the first index of bucket (I >> lut_shift)
     uint32_t pascal;      // u32[25*25]
-    uint32_t base16;      // u32[48]: [k] = first entry of the k-subsets in r16 (k <= 8); [16 + k] = C(16, k), k <= 16
-    uint32_t r16;         // u16[]: the k-subsets of 16 slots as bit masks, k = 0..8, each in numeric order
+    uint32_t base14;      // u32[16]: [k] = first entry of the k-subsets of 14 slots in r14
+    uint32_t r14;         // u16[16384]: the k-subsets of 14 slots as bit masks, k = 0..14, each in numeric order
     uint32_t pd6;         // u8[4096]: [f << 6 | s] = low bits of s deposited into the set bits of f
     uint32_t off;         // u64[ncls + 1]
     uint32_t desc;        // u32[ncls][kFastDescWords]

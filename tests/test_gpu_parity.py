@@ -228,7 +228,7 @@ def test_argument_checks(lib, ctxs):
     assert L.llvq_dequant_matrix(ctx._h, idx.data_ptr(), g.data_ptr(), 2, 24, 7, w.data_ptr(), 24, None) == 1
     assert L.llvq_dequant_matrix(ctx._h, idx.data_ptr(), g.data_ptr(), 2, 24, 1, w.data_ptr(), 8, None) == 1
     assert L.llvq_gemv(ctx._h, idx.data_ptr(), g.data_ptr(), 2, 24, w.data_ptr(), w.data_ptr(), 9, None) == 1
-    assert L.llvq_gemv(ctx._h, idx.data_ptr(), g.data_ptr(), 2, 10_000_000, w.data_ptr(), w.data_ptr(), 0, None) == 3
+    assert L.llvq_gemv(ctx._h, idx.data_ptr(), g.data_ptr(), 2, 10_000_000, w.data_ptr(), w.data_ptr(), 0, None) == 3   # x does not fit shared memory
     torch.cuda.synchronize()
 
 
