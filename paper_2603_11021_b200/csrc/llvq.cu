@@ -181,7 +181,7 @@ gemv_kernel(DevCode dc, const uint32_t* __restrict__ stream, const uint16_t* __r
 // Persistent CTAs, one per SM.
 // ===========================================================================
 constexpr int kFastThreads = 1024;      // decode / dequant kernels
-constexpr int kGemvThreads = 768;
+constexpr int kGemvThreads = 1024;     // upper bound; the launch picks the warp count that divides the units per CTA best
 
 struct FastArgs {
     FastLayout L;
@@ -274,11 +274,13 @@ dequant_fast_kernel(FastArgs fa, const uint32_t* __restrict__ stream, const uint
     }
 }
 
-// Fused dequant + GEMV.  A warp owns units of 16 rows x 4 column blocks: lane (g, t) = (lane / 4, lane % 4)
-// decodes the blocks (row g, column block 4q + t) and (row g + 8, same column block); their 2 x 12 packed bf16
-// pairs are the A fragments of six m16n8k16 tensor-core MMAs whose B fragment carries the matching 4 x 24
-// activations (the same in all 8 columns), accumulating in binary32.
-constexpr int kGemvRows = 32;           // output rows per CTA tile
+// Fused dequant + GEMV.  The work is cut into units of 16 rows x 4 column blocks, numbered row group major, and
+// every CTA takes an equal contiguous range of units.  In a unit lane (g, t) = (lane / 4, lane % 4) decodes the
+// blocks (row g, column block 4q + t) and (row g + 8, same column block); their 2 x 12 packed bf16 pairs are
+// the A fragments of six m16n8k16 tensor-core MMAs whose B fragment carries the matching 4 x 24 activations
+// (the same in all 8 columns), accumulating in binary32.  Row sums are collected in shared memory; a row
+// group that is split between CTAs is finished through a zero-kept global scratch and an arrival counter.
+constexpr int kGemvGroupsPerPass = 64;   // row groups (of 16 rows) whose sums a CTA keeps in shared memory at a time
 
 __device__ __forceinline__ void mma_bf16_16816(float c[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0, uint32_t b1)
 {
@@ -286,32 +288,41 @@ __device__ __forceinline__ void mma_bf16_16816(float c[4], uint32_t a0, uint32_t
                  : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3]) : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
 }
 
+// CTA that owns unit u when G CTAs split U units into ranges [c*U/G, (c+1)*U/G).
+__device__ __forceinline__ int64_t unit_owner(int64_t u, int64_t U, int64_t G) { return ((u + 1) * G - 1) / U; }
+
 template <bool kOutBf16>
 __global__ void __launch_bounds__(kGemvThreads, 1)
 gemv_fast_kernel(FastArgs fa, const uint32_t* __restrict__ stream, const uint16_t* __restrict__ gain,
-                 int64_t n_out, int64_t k_in, int64_t bpr, const uint16_t* __restrict__ x, void* __restrict__ y)
+                 int64_t n_out, int64_t k_in, int64_t bpr, const uint16_t* __restrict__ x, void* __restrict__ y,
+                 float* __restrict__ scratch, uint32_t* __restrict__ counters)
 {
     FAST_PROLOGUE();
     const int64_t nq = (bpr + 3) / 4;                               // units along K
     uint32_t* xs = reinterpret_cast<uint32_t*>(staging);            // [nq * 4][12] packed bf16 pairs of x
-    float* acc = reinterpret_cast<float*>(xs + nq * 48);            // [kGemvRows]
-    for (int64_t i = threadIdx.x; i < nq * 48; i += kGemvThreads) {
+    float* acc = reinterpret_cast<float*>(xs + nq * 48);            // [kGemvGroupsPerPass][16]
+    uint32_t* last_flag = reinterpret_cast<uint32_t*>(acc + kGemvGroupsPerPass * 16);
+    for (int64_t i = threadIdx.x; i < nq * 48; i += blockDim.x) {
         const int64_t e = 2 * i;
         const uint32_t lo = e < k_in ? __ldg(x + e) : 0u, hi = e + 1 < k_in ? __ldg(x + e + 1) : 0u;
         xs[i] = lo | hi << 16;
     }
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, g = lane >> 2, t = lane & 3;
-    constexpr int kWarps = kGemvThreads / 32;
-    const int64_t ntiles = (n_out + kGemvRows - 1) / kGemvRows;
-    for (int64_t tile = blockIdx.x; tile < ntiles; tile += gridDim.x) {
-        if (threadIdx.x < kGemvRows) acc[threadIdx.x] = 0.f;
+    const int kWarps = (int)(blockDim.x >> 5);
+    const int64_t groups = (n_out + 15) / 16;
+    const int64_t U = groups * nq, G = gridDim.x;
+    const int64_t u_begin = blockIdx.x * U / G, u_end = (blockIdx.x + 1) * U / G;
+    if (u_begin >= u_end) return;
+    const int64_t rg_first = u_begin / nq, rg_last = (u_end - 1) / nq;
+    for (int64_t rg0 = rg_first; rg0 <= rg_last; rg0 += kGemvGroupsPerPass) {
+        const int64_t rg1 = min(rg0 + kGemvGroupsPerPass - 1, rg_last);
+        for (int i = threadIdx.x; i < kGemvGroupsPerPass * 16; i += (int)blockDim.x) acc[i] = 0.f;
         __syncthreads();
-        const int64_t row0 = tile * kGemvRows;
-        const int64_t units = (kGemvRows / 16) * nq;
-        for (int64_t u = warp; u < units; u += kWarps) {
-            const int64_t rg = u / nq, kq = u % nq;
+        const int64_t p_begin = max(u_begin, rg0 * nq), p_end = min(u_end, (rg1 + 1) * nq);
+        for (int64_t u = p_begin + warp; u < p_end; u += kWarps) {
+            const int64_t rg = u / nq, kq = u - rg * nq;
             const int64_t cb = kq * 4 + t;
-            const int64_t rowA = row0 + rg * 16 + g, rowB = rowA + 8;
+            const int64_t rowA = rg * 16 + g, rowB = rowA + 8;
             const bool inA = rowA < n_out && cb < bpr, inB = rowB < n_out && cb < bpr;
             const uint64_t bA = (uint64_t)(rowA * bpr + cb), bB = (uint64_t)(rowB * bpr + cb);
             const uint64_t IA = inA ? load_field(stream, bA, (int)fa.L.W) : 0ull;
@@ -334,16 +345,44 @@ gemv_fast_kernel(FastArgs fa, const uint32_t* __restrict__ stream, const uint16_
             for (int q = 0; q < 6; ++q)
                 mma_bf16_16816(c, wA[2 * q], wB[2 * q], wA[2 * q + 1], wB[2 * q + 1], xv[2 * q], xv[2 * q + 1]);
             if (t == 0) {
-                atomicAdd(&acc[rg * 16 + g], c[0]);
-                atomicAdd(&acc[rg * 16 + g + 8], c[2]);
+                atomicAdd(&acc[(rg - rg0) * 16 + g], c[0]);
+                atomicAdd(&acc[(rg - rg0) * 16 + g + 8], c[2]);
             }
         }
         __syncthreads();
-        if (threadIdx.x < kGemvRows && row0 + threadIdx.x < n_out) {
-            if (kOutBf16) reinterpret_cast<__nv_bfloat16*>(y)[row0 + threadIdx.x] = __float2bfloat16_rn(acc[threadIdx.x]);
-            else reinterpret_cast<float*>(y)[row0 + threadIdx.x] = acc[threadIdx.x];
+        // row groups this CTA covers completely are final; the (at most two) split ones go through the scratch
+        for (int64_t rg = rg0; rg <= rg1; ++rg) {
+            const bool whole = u_begin <= rg * nq && (rg + 1) * nq <= u_end;
+            const int64_t row = rg * 16 + threadIdx.x;
+            const bool mine = threadIdx.x < 16 && row < n_out;
+            if (whole) {
+                if (mine) {
+                    const float v = acc[(rg - rg0) * 16 + threadIdx.x];
+                    if (kOutBf16) reinterpret_cast<__nv_bfloat16*>(y)[row] = __float2bfloat16_rn(v);
+                    else reinterpret_cast<float*>(y)[row] = v;
+                }
+                continue;
+            }
+            if (mine) atomicAdd(scratch + row, acc[(rg - rg0) * 16 + threadIdx.x]);
+            __threadfence();
+            __syncthreads();
+            if (threadIdx.x == 0) {
+                const uint32_t parts = (uint32_t)(unit_owner((rg + 1) * nq - 1, U, G) - unit_owner(rg * nq, U, G) + 1);
+                *last_flag = atomicAdd(counters + rg, 1u) == parts - 1u;
+            }
+            __syncthreads();
+            if (*last_flag) {
+                __threadfence();
+                if (mine) {
+                    const float v = __ldcg(scratch + row);
+                    if (kOutBf16) reinterpret_cast<__nv_bfloat16*>(y)[row] = __float2bfloat16_rn(v);
+                    else reinterpret_cast<float*>(y)[row] = v;
+                    __stcg(scratch + row, 0.f);
+                }
+                if (threadIdx.x == 0) counters[rg] = 0u;
+            }
+            __syncthreads();
         }
-        __syncthreads();
     }
 }
 
@@ -639,7 +678,7 @@ int llvq_create(llvq_ctx** out, int m_lo, int m_hi, int device)
     ctx->fast = build_fast_image(h, ctx->fl, image);
     size_t o_img = up(o_err + 256);
     size_t o_cnt = up(o_img + (ctx->fast ? image.size() : 0));
-    size_t o_scr = up(o_cnt + (kMaxScratchRows / kGemmRows) * 4);
+    size_t o_scr = up(o_cnt + (size_t)(64 * kMaxScratchRows / 16) * 4);   // one counter per group of 16 rows (GEMV) / per 128-row tile (GEMM)
     size_t total = o_scr + (size_t)64 * kMaxScratchRows * 4;
     std::vector<uint8_t> blob(total, 0);
     if (ctx->fast) std::memcpy(blob.data() + o_img, image.data(), image.size());
@@ -808,17 +847,25 @@ int llvq_gemv(const llvq_ctx* ctx, const void* d_idx, const uint16_t* d_gain_f16
     int64_t bpr = (k_in + 23) / 24;
     if (ctx->fast) {
         const int64_t nq = (bpr + 3) / 4;
-        const size_t smem = ctx->fl.total + 16 + (size_t)nq * 48 * 4 + kGemvRows * 4;
-        if (smem > 227 * 1024 || n_out > (1ll << 31)) return LLVQ_EUNSUPPORTED;
-        const int64_t tiles = (n_out + kGemvRows - 1) / kGemvRows;
-        unsigned g = (unsigned)std::min<int64_t>(tiles, ctx->sm_count);
+        const size_t smem = ctx->fl.total + 16 + (size_t)nq * 48 * 4 + kGemvGroupsPerPass * 16 * 4 + 16;
+        if (smem > 227 * 1024 || n_out > 64ll * kMaxScratchRows) return LLVQ_EUNSUPPORTED;
+        const int64_t units = ((n_out + 15) / 16) * nq;
+        unsigned g = (unsigned)std::min<int64_t>(units, ctx->sm_count);
+        // warps per CTA: the count in [20, 32] that wastes the fewest warp slots on the units of one CTA
+        const int64_t upc = (units + g - 1) / g;
+        int warps = 32; double best_eff = 0.0;
+        for (int w = 32; w >= 20; --w) {
+            const double eff = (double)upc / (double)(((upc + w - 1) / w) * w);
+            if (eff > best_eff + 1e-9) { best_eff = eff; warps = w; }
+        }
+        const unsigned threads = 32u * (unsigned)warps;
         const uint32_t* idx = static_cast<const uint32_t*>(d_idx);
         if (y_dtype == LLVQ_BF16) {
             if (!set_smem(gemv_fast_kernel<true>, smem)) return LLVQ_ECUDA;
-            gemv_fast_kernel<true><<<g, kGemvThreads, smem, st>>>(fast_args(ctx), idx, d_gain_f16, n_out, k_in, bpr, d_x_bf16, d_y);
+            gemv_fast_kernel<true><<<g, threads, smem, st>>>(fast_args(ctx), idx, d_gain_f16, n_out, k_in, bpr, d_x_bf16, d_y, ctx->d_scratch, ctx->d_counters);
         } else {
             if (!set_smem(gemv_fast_kernel<false>, smem)) return LLVQ_ECUDA;
-            gemv_fast_kernel<false><<<g, kGemvThreads, smem, st>>>(fast_args(ctx), idx, d_gain_f16, n_out, k_in, bpr, d_x_bf16, d_y);
+            gemv_fast_kernel<false><<<g, threads, smem, st>>>(fast_args(ctx), idx, d_gain_f16, n_out, k_in, bpr, d_x_bf16, d_y, ctx->d_scratch, ctx->d_counters);
         }
         return launch_status();
     }
