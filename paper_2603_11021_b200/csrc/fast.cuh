@@ -143,7 +143,7 @@ __device__ __forceinline__ uint32_t fast_find_class(const FastSmem& T, uint64_t 
 // S3-S6 for any class; `mask` = the lanes of the warp that call this together.
 __device__ __forceinline__ void fast_decode_local(const FastSmem& T, uint32_t cls, uint64_t local, bool valid, uint32_t mask, Decoded& d)
 {
-    const uint4* D = reinterpret_cast<const uint4*>(T.desc + cls * kFastDescWords);
+    const uint4* D = reinterpret_cast<const uint4*>(T.desc + cls * kFastDescStride);
     const uint4 h = D[0], v = D[1], lw = D[2], mg = D[3];
     const uint32_t w = h.x & 0xff, B = (h.x >> 8) & 0xff, flags = (h.x >> 16) & 0xff;
     const uint32_t nlev1 = (h.x >> 24) & 0xf, nlev = valid ? h.x >> 28 : 0u;

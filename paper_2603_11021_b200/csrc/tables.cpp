@@ -232,7 +232,7 @@ bool build_fast_image(const HostTables& t, FastLayout& L, std::vector<uint8_t>& 
     L.pd6 = up16(L.r14 + r14.size() * 2);
     L.off = up16(L.pd6 + 4096);
     L.desc = up16(L.off + (ncls + 1) * 8);
-    L.total = up16(L.desc + ncls * kFastDescWords * 4);
+    L.total = up16(L.desc + ncls * kFastDescStride * 4);
     L.lut_shift = (uint32_t)(t.W - 12);
     L.ncls = (uint32_t)ncls;
     L.W = (uint32_t)t.W;
@@ -264,7 +264,7 @@ bool build_fast_image(const HostTables& t, FastLayout& L, std::vector<uint8_t>& 
     uint32_t* dw = reinterpret_cast<uint32_t*>(img.data() + L.desc);
     for (size_t j = 0; j < ncls; ++j) {
         const ClassDesc& d = t.desc[j];
-        uint32_t* w = dw + j * kFastDescWords;
+        uint32_t* w = dw + j * kFastDescStride;
         const int nlev = d.nlev1 + d.nlev0;
         if (nlev > kFastMaxLevels || nlev + 2 > 8) return false;
         uint32_t flags = (d.parity ? 1u : 0u) | (d.signpar ? 2u : 0u) | (d.fill0 ? 4u : 0u) |

@@ -77,7 +77,8 @@ bool build_tables(int m_lo, int m_hi, HostTables& out);
 namespace llvq {
 
 constexpr int kFastMaxLevels = 4;      // unranking steps per class on the fast path
-constexpr int kFastDescWords = 16;     // 64-byte class descriptor
+constexpr int kFastDescWords = 16;     // words of a class descriptor that carry data
+constexpr int kFastDescStride = 20;    // words between descriptors: 80 bytes spread consecutive classes over all bank groups
 constexpr int kLowBits = 14;           // slots resolved by one table lookup in the subset unranking
 
 
@@ -90,7 +91,7 @@ struct FastLayout {
     uint32_t r14;         // u16[16384]: the k-subsets of 14 slots as bit masks, k = 0..14, each in numeric order
     uint32_t pd6;         // u8[4096]: [f << 6 | s] = low bits of s deposited into the set bits of f
     uint32_t off;         // u64[ncls + 1]
-    uint32_t desc;        // u32[ncls][kFastDescWords]
+    uint32_t desc;        // u32[ncls][kFastDescStride]
     uint32_t total;       // bytes, multiple of 16
     uint32_t lut_shift;
     uint32_t ncls;
