@@ -589,6 +589,7 @@ int launch_status();
 int check_gemm_args(const llvq_ctx* ctx, const void* d_idx, const uint16_t* d_gain_f16, int64_t n_out, int64_t k_in,
                     const uint16_t* d_x_bf16, int batch, const uint16_t* d_y_bf16)
 {
+    if (ctx && ctx->device >= 0 && n_out == 0 && batch >= 1 && batch <= 64) return LLVQ_OK;   // nothing to do: pointers may be null
     if (int e = check_common(ctx, d_idx)) return e;
     if (!d_gain_f16 || !d_x_bf16 || !d_y_bf16 || n_out < 0 || k_in < 0 || batch < 1 || batch > 64) return LLVQ_EINVAL;
     if (!aligned(d_gain_f16, 2) || !aligned(d_x_bf16, 16) || !aligned(d_y_bf16, 2) || (k_in & 7)) return LLVQ_EALIGN;
@@ -790,6 +791,7 @@ int llvq_decode_blocks(const llvq_ctx* ctx, const void* d_idx, uint64_t nblocks,
 int llvq_dequant_matrix(const llvq_ctx* ctx, const void* d_idx, const uint16_t* d_gain_f16,
                         int64_t rows, int64_t cols, int layout, uint16_t* d_w_bf16, int64_t ld, void* stream)
 {
+    if (ctx && ctx->device >= 0 && (rows == 0 || cols == 0)) return LLVQ_OK;      // nothing to do: pointers may be null
     if (int e = check_common(ctx, d_idx)) return e;
     if (!d_gain_f16 || !d_w_bf16 || rows < 0 || cols < 0 || ld < cols) return LLVQ_EINVAL;
     if (layout != LLVQ_LAYOUT_FLAT && layout != LLVQ_LAYOUT_ROWWISE) return LLVQ_EINVAL;
@@ -833,6 +835,7 @@ int llvq_dequant_matrix(const llvq_ctx* ctx, const void* d_idx, const uint16_t* 
 int llvq_gemv(const llvq_ctx* ctx, const void* d_idx, const uint16_t* d_gain_f16, int64_t n_out, int64_t k_in,
               const uint16_t* d_x_bf16, void* d_y, int y_dtype, void* stream)
 {
+    if (ctx && ctx->device >= 0 && n_out == 0) return LLVQ_OK;                     // nothing to do: pointers may be null
     if (int e = check_common(ctx, d_idx)) return e;
     if (!d_gain_f16 || !d_x_bf16 || !d_y || n_out < 0 || k_in < 0) return LLVQ_EINVAL;
     if (y_dtype != LLVQ_F32 && y_dtype != LLVQ_BF16) return LLVQ_EINVAL;

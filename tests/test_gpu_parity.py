@@ -293,3 +293,58 @@ def test_gemm_matches_gemv_rows(lib, ctxs, oracle_mod):
         torch.cuda.synchronize()
         ref = y.cpu().numpy().astype(np.float64)
         assert gemv_error(Y[b].cpu().numpy(), ref) <= 2.0 ** -8 + 1e-4
+
+
+# --------------------------------------------------------------------------
+# full benchmark sizes, in the launch configuration bench.py times
+# --------------------------------------------------------------------------
+def test_dequant_full_size_config2(lib, ctxs, oracle_mod):
+    # 4096 x 4096 FLAT, 699051 blocks (the last one holds 16 real weights), 48-bit indices: every element compared
+    o = _oracle(oracle_mod)((2, 13))
+    ctx = ctxs[(2, 13)]
+    rows = cols = 4096
+    stream, gain, nblocks = gen.make_layer(o.N, o.W, rows, cols, 0, seed=0)
+    assert nblocks == 699051
+    got = lib.llvq_dequant_matrix(ctx, to_dev_u8(stream), to_dev_f16(gain), rows, cols, 0)
+    torch.cuda.synchronize()
+    want = o.dequant_matrix(stream, gain, rows, cols, 0)
+    assert np.array_equal(bf16_bits(got), want)
+    assert lib.llvq_last_error(ctx) == (0, 0)
+
+
+@pytest.mark.parametrize("code,n_out,k_in,batch", [((2, 13), 8192, 8192, 16), ((2, 13), 8192, 8192, 64), ((2, 13), 28672, 8192, 16),
+                                                   ((2, 13), 8192, 28672, 64), ((2, 53), 8192, 8192, 16)])
+def test_gemm_full_size_config4_sampled_rows(lib, ctxs, oracle_mod, code, n_out, k_in, batch):
+    o = _oracle(oracle_mod)(code)
+    ctx = ctxs[code]
+    stream, gain, _ = gen.make_layer(o.N, o.W, n_out, k_in, 1, seed=0)
+    X = gen.normal_bf16((batch, k_in), seed=0)
+    Y = lib.llvq_gemm_small_batch(ctx, to_dev_u8(stream), to_dev_f16(gain), n_out, k_in, to_dev_bf16(X))
+    torch.cuda.synchronize()
+    Y = Y.float().cpu().numpy()
+    assert np.isfinite(Y).all()
+    rows = sorted(set([0, 127, 128, n_out // 2 + 1, n_out - 129, n_out - 1] + list(range(17, n_out, n_out // 11))))
+    ref = np.stack([o.gemm(stream, gain, n_out, k_in, X, rows=(r, 1))[:, r] for r in rows], axis=1)      # [batch, len(rows)]
+    scale = float(np.abs(ref).max())
+    err = np.abs(Y[:, rows] - ref) / np.maximum(np.abs(ref), 1e-3 * scale)
+    assert err.max() <= TOL_BF16_OUT, err.max()
+    assert lib.llvq_last_error(ctx) == (0, 0)
+
+
+def test_smallest_and_odd_shapes(lib, ctxs, oracle_mod):
+    o = _oracle(oracle_mod)((2, 13))
+    ctx = ctxs[(2, 13)]
+    for n_out, k_in, batch in [(1, 8, 1), (1, 24, 64), (17, 40, 3), (2049, 72, 2)]:
+        stream, gain, _ = gen.make_layer(o.N, o.W, n_out, k_in, 1, seed=12)
+        X = gen.normal_bf16((batch, k_in), seed=12)
+        want = o.gemm(stream, gain, n_out, k_in, X)
+        d = (to_dev_u8(stream), to_dev_f16(gain))
+        Y = lib.llvq_gemm_small_batch(ctx, *d, n_out, k_in, to_dev_bf16(X)).float().cpu().numpy()
+        y = lib.llvq_gemv(ctx, *d, n_out, k_in, to_dev_bf16(X[0])).cpu().numpy()
+        torch.cuda.synchronize()
+        scale = np.abs(want).max()
+        assert (np.abs(Y - want) / np.maximum(np.abs(want), 1e-3 * scale)).max() <= TOL_BF16_OUT
+        assert gemv_error(y, want[0]) <= TOL
+    # zero-sized calls are accepted and touch nothing
+    assert lib.llvq_dequant_matrix(ctx, torch.zeros(16, dtype=torch.uint8, device="cuda"), torch.zeros(1, dtype=torch.float16, device="cuda"),
+                                   0, 24, 1).numel() == 0
