@@ -39,9 +39,9 @@ METRIC = "fused dequant+GEMV algorithmic GB/s (index+gain+activation+output byte
 UNIT = "GB/s"
 WORKLOAD = "configs[2]: fused dequant+GEMV batch 1 on W 4096x4096, 11008x4096, 4096x11008, 48-bit indices (shells 2..13), fp16 gain per 24 weights"
 
-# dram bytes (read + write) of one gemv launch on the 11008x4096 layer, from the ncu capture summarised
-# in profiles/; None until a capture exists
-NCU_TRAFFIC_BYTES_11008x4096 = None
+# dram__bytes_read.sum + dram__bytes_write.sum of one gemv_fast_kernel launch on the 11008x4096 layer, from the
+# ncu capture summarised in profiles/gemv_fast_kernel_7B_layers.md (algorithmic bytes: 15 089 152)
+NCU_TRAFFIC_BYTES_11008x4096 = 15237888
 
 
 def layer_bytes(n_out: int, k_in: int) -> dict:
@@ -223,6 +223,76 @@ def profile_run(P, ctx, args) -> None:
     print(json.dumps({"profile": args.profile, "launches": args.warmup + args.steps, "copies": copies, "errors": P.llvq_last_error(ctx)}))
 
 
+def _event_us(torch, fn, reps: int) -> float:
+    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    a.record()
+    for i in range(reps):
+        fn(i)
+    b.record()
+    b.synchronize()
+    return a.elapsed_time(b) / reps * 1e3
+
+
+def extras(P, ctx) -> dict:
+    """Other configurations of the same path, each on rotating buffers larger than L2 (reported, not the headline):
+    standalone dequant 4096x4096 FLAT, small-batch GEMM 8192x8192 at batch 16/64, and the GEMV sweep over the
+    linear layers of an 8B Llama-3-shaped decoder (tokens/s of the quantized-weight decode step)."""
+    import torch
+    out = {}
+    dev = lambda a, view=None: torch.from_numpy(a if view is None else a.view(view)).cuda()
+    # --- dequant, 4096 x 4096 FLAT
+    rows = cols = 4096
+    bufs = []
+    for c in range(4):
+        stream, gain, nb = gen.make_layer(CODE_N, CODE_W, rows, cols, 0, seed=100 + c)
+        bufs.append((dev(stream), dev(gain, np.float16), torch.empty((rows, cols), dtype=torch.bfloat16, device="cuda")))
+    fn = lambda i: P.llvq_dequant_matrix(ctx, bufs[i % 4][0], bufs[i % 4][1], rows, cols, 0, d_w=bufs[i % 4][2])
+    _event_us(torch, fn, 8)
+    us = _event_us(torch, fn, 40)
+    by = nb * (CODE_W // 8 + 2) + rows * cols * 2
+    out["dequant_4096x4096_flat"] = {"us": us, "GBps": by / us / 1e3, "weights_per_s": rows * cols / (us * 1e-6), "algorithmic_bytes": by}
+    del bufs
+    # --- GEMM, 8192 x 8192
+    n, k = 8192, 8192
+    bufs = []
+    for c in range(12):
+        stream, gain, nb = gen.make_layer(CODE_N, CODE_W, n, k, 1, seed=200 + c)
+        bufs.append((dev(stream), dev(gain, np.float16)))
+    for batch in (16, 64):
+        x = dev(gen.normal_bf16((batch, k), seed=batch), np.int16).view(torch.bfloat16)
+        y = torch.empty((batch, n), dtype=torch.bfloat16, device="cuda")
+        fn = lambda i: P.llvq_gemm_small_batch(ctx, bufs[i % 12][0], bufs[i % 12][1], n, k, x, d_y=y)
+        _event_us(torch, fn, 4)
+        us = _event_us(torch, fn, 24)
+        by = nb * (CODE_W // 8 + 2) + batch * k * 2 + batch * n * 2
+        out[f"gemm_8192x8192_b{batch}"] = {"us": us, "GBps": by / us / 1e3, "TFLOPs": 2.0 * n * k * batch / us / 1e6, "algorithmic_bytes": by}
+    del bufs
+    # --- decoder sweep: q, k, v, o, gate, up, down of one layer; 32 layers; 4 distinct layer sets (> 2 x L2)
+    shapes = [(4096, 4096), (1024, 4096), (1024, 4096), (4096, 4096), (14336, 4096), (14336, 4096), (4096, 14336)]
+    sets = []
+    for c in range(4):
+        layer = []
+        for li, (n, k) in enumerate(shapes):
+            stream, gain, nb = gen.make_layer(CODE_N, CODE_W, n, k, 1, seed=300 + 10 * c + li)
+            layer.append((dev(stream), dev(gain, np.float16)))
+        sets.append(layer)
+    xs = {k: dev(gen.normal_bf16(k, seed=k), np.int16).view(torch.bfloat16) for k in (4096, 14336)}
+    ys = {n: torch.empty(n, dtype=torch.bfloat16, device="cuda") for n in (4096, 1024, 14336)}
+
+    def token(i):
+        for layer in range(32):
+            for (n, k), (d_idx, d_gain) in zip(shapes, sets[(i * 32 + layer) % 4]):
+                P.llvq_gemv(ctx, d_idx, d_gain, n, k, xs[k], d_y=ys[n])
+    token(0)
+    torch.cuda.synchronize()
+    us = _event_us(torch, token, 3)
+    blocks = 32 * sum(n * ((k + 23) // 24) for n, k in shapes)
+    by = blocks * (CODE_W // 8 + 2) + 32 * sum(2 * k + 2 * n for n, k in shapes)
+    out["llama3_8b_linear_sweep"] = {"us_per_token": us, "tokens_per_s": 1e6 / us, "GBps": by / us / 1e3, "blocks_per_token": blocks,
+                                     "launches_per_token": 32 * len(shapes), "algorithmic_bytes": by}
+    return out
+
+
 def main() -> None:
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -230,6 +300,7 @@ def main() -> None:
     ap.add_argument("--warmup", type=int, default=20)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-extras", action="store_true", help="skip the secondary configurations (dequant, GEMM, decoder sweep)")
     ap.add_argument("--profile", default=None, choices=["gemv", "dequant", "gemm"],
                     help="run only a few launches of one kernel over rotating buffers (for ncu captures); no timing line")
     args = ap.parse_args()
@@ -369,12 +440,16 @@ def main() -> None:
             "frac_of_hbm_peak": value / world / peak,
             "layers": per_layer,
             "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
-                         "traffic": NCU_TRAFFIC_BYTES_11008x4096, "kernel": "gemv_kernel on 11008x4096",
+                         "traffic": NCU_TRAFFIC_BYTES_11008x4096, "kernel": "gemv_fast_kernel on 11008x4096",
                          "algorithmic_bytes_per_launch": dom_bytes, "peak_source": f"of {which}", "frac_of_nominal_8TBps": achieved / 8000.0},
             "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "ms_per_step": e2e_ms},
             "gpu_launches": timed_launches,
             "clocks": clocks.summary(),
         }
+        if world == 1 and not args.no_extras:
+            del sets, host_sets
+            torch.cuda.empty_cache()
+            out["extras"] = extras(P, ctx)
         if world == 1 and not args.no_cpu_baseline:
             out["cpu_baseline"] = cpu_baseline()
         print(json.dumps(out))
