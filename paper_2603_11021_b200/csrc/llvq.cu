@@ -389,18 +389,20 @@ gemv_fast_kernel(FastArgs fa, const uint32_t* __restrict__ stream, const uint16_
 // ===========================================================================
 // llvq_gemm_small_batch: Y[b][i] = sum_k X[b][k] W[i][k] on the tensor cores.
 // A work item is a tile of 128 output rows x a range of K stages (96 columns = 4 blocks of 24 per row).
-// Per stage every thread dequantizes one block into the shared-memory A tile (bf16, K-major core-matrix
-// layout), the matching slice of X goes into the B tile, and one thread issues six tcgen05 MMAs
-// (M = 128, N = padded batch, K = 16) accumulating in tensor memory.  Two stages are in flight.
+// Per stage every thread of a 512-thread group dequantizes one block into the group's shared-memory A tile
+// (bf16, K-major core-matrix layout), the matching slice of X goes into its B tile, and one thread issues
+// six tcgen05 MMAs (M = 128, N = padded batch, K = 16) into the group's accumulator in tensor memory.
+// The two groups of a CTA take alternate stages, so two stages are in flight.
 // Split-K partial sums are added into a zero-initialised binary32 scratch [npad][n_out]; the last item
 // of a row tile converts it to bf16 and clears it again.
 // ===========================================================================
-constexpr int kGemmThreads = 512;
+constexpr int kGemmThreads = 1024;
+constexpr int kGemmGroupThreads = 512;
 constexpr int kGemmRows = 128;
 constexpr int kStageBlocks = 4;                       // column blocks per stage
 constexpr int kStageK = kStageBlocks * 24;            // 96
 constexpr int kMaxScratchRows = 65536;
-constexpr uint32_t kTmemCols = 64;
+constexpr uint32_t kTmemCols = 128;
 
 struct GemmArgs {
     int64_t n_out, k_in, bpr;
@@ -413,6 +415,11 @@ struct GemmArgs {
     uint32_t* counters;        // [row tiles], zero on entry and on exit
 };
 
+__device__ __forceinline__ void group_barrier(int group)
+{
+    asm volatile("bar.sync %0, %1;" ::"r"(1 + group), "n"(kGemmGroupThreads) : "memory");
+}
+
 template <bool kFast>
 __global__ void __launch_bounds__(kGemmThreads, 1)
 gemm_kernel(FastArgs fa, DevCode dc, const uint32_t* __restrict__ stream, const uint16_t* __restrict__ gain, GemmArgs ga)
@@ -420,13 +427,13 @@ gemm_kernel(FastArgs fa, DevCode dc, const uint32_t* __restrict__ stream, const 
     extern __shared__ __align__(128) uint8_t smem[];
     const uint32_t img_bytes = kFast ? fa.L.total : 0u;
     uint64_t* bar_img = reinterpret_cast<uint64_t*>(smem + img_bytes);
-    uint64_t* bar_free = bar_img + 1;                                     // [2]
-    uint64_t* bar_done = bar_img + 3;
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bar_img + 4);
+    uint64_t* bar_free = bar_img + 1;                                     // [2]: the MMAs reading group h's buffers are done
+    uint64_t* bar_done = bar_img + 3;                                     // [2]: group h's accumulator of this item is complete
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bar_img + 5);
     uint32_t* last_flag = tmem_slot + 1;
     const uint32_t a_off = (img_bytes + 64 + 1023) & ~1023u;
-    uint8_t* a_buf = smem + a_off;                                        // 2 x 24576
-    uint8_t* b_buf = a_buf + 2 * kGemmRows * kStageK * 2;                  // 2 x npad * 192
+    uint8_t* a_buf = smem + a_off;                                        // [2 groups] x 24576
+    uint8_t* b_buf = a_buf + 2 * kGemmRows * kStageK * 2;                  // [2 groups] x npad * 192
     const uint32_t b_stage = (uint32_t)ga.npad * kStageK * 2;
 
     FastSmem T{};
@@ -434,9 +441,12 @@ gemm_kernel(FastArgs fa, DevCode dc, const uint32_t* __restrict__ stream, const 
         if (!fast_load_image(smem, fa.image, fa.L.total, bar_img, fa.flags)) return;
         T = fast_view(smem, fa.L);
     }
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    // Two groups of 512 threads fill alternate stages, each into its own buffers and its own accumulator
+    // (TMEM columns [64 h, 64 h + npad)); the epilogue adds the two accumulators.
+    const int group = threadIdx.x / kGemmGroupThreads, gtid = threadIdx.x % kGemmGroupThreads;
+    const int gwarp = gtid >> 5, lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     if (threadIdx.x == 0) {
-        mbar_init(&bar_free[0], 1); mbar_init(&bar_free[1], 1); mbar_init(bar_done, 1);
+        mbar_init(&bar_free[0], 1); mbar_init(&bar_free[1], 1); mbar_init(&bar_done[0], 1); mbar_init(&bar_done[1], 1);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     if (warp == 0) tmem_alloc(tmem_slot, kTmemCols);
@@ -445,21 +455,21 @@ gemm_kernel(FastArgs fa, DevCode dc, const uint32_t* __restrict__ stream, const 
     tc_fence_after();
     const uint32_t tmem = *tmem_slot;
     const uint32_t idesc = instr_desc_bf16_m128((uint32_t)ga.npad);
+    uint8_t* const a_mine = a_buf + group * (kGemmRows * kStageK * 2);
+    uint8_t* const b_mine = b_buf + group * b_stage;
 
     const int64_t row_tiles = (ga.n_out + kGemmRows - 1) / kGemmRows;
     const int64_t items = row_tiles * ga.split;
-    uint32_t gstage = 0, gitem = 0;
-    bool failed = false;
-    for (int64_t item = blockIdx.x; item < items && !failed; item += gridDim.x, ++gitem) {
+    uint32_t uses = 0;                                  // stages this group has filled so far
+    uint32_t done[2] = {0, 0};                          // completed accumulations per group
+    bool timeout = false;
+    for (int64_t item = blockIdx.x; item < items; item += gridDim.x) {
         const int64_t rt = item / ga.split;
         const int f = (int)(item % ga.split);
         const int s_begin = (int)((int64_t)f * ga.nstages / ga.split), s_end = (int)((int64_t)(f + 1) * ga.nstages / ga.split);
-        const int64_t row = rt * kGemmRows + warp * 8 + (lane & 7);
-        for (int s = s_begin; s < s_end; ++s, ++gstage) {
-            const uint32_t buf = gstage & 1u;
-            bool ok = true;
-            if (gstage >= 2) ok = mbar_wait(&bar_free[buf], ((gstage >> 1) - 1u) & 1u);     // the MMAs that read this buffer are done
-            if (__syncthreads_or(!ok)) { failed = true; break; }
+        const int64_t row = rt * kGemmRows + gwarp * 8 + (lane & 7);
+        for (int s = s_begin + group; s < s_end; s += 2, ++uses) {
+            if (uses > 0 && !mbar_wait(&bar_free[group], (uses - 1u) & 1u)) timeout = true;   // the MMAs of the previous stage read these buffers
             // ---- A: dequantize one block of 24 weights
             const int64_t cb = (int64_t)s * kStageBlocks + (lane >> 3);
             const bool in = row < ga.n_out && cb < ga.bpr;
@@ -484,59 +494,60 @@ gemm_kernel(FastArgs fa, DevCode dc, const uint32_t* __restrict__ stream, const 
                     w[j] = *reinterpret_cast<uint32_t*>(&h);
                 }
             }
-            uint8_t* a_dst = a_buf + buf * (kGemmRows * kStageK * 2) + warp * 128 + (lane & 7) * 16;
+            uint8_t* a_dst = a_mine + gwarp * 128 + (lane & 7) * 16;
 #pragma unroll
             for (int j = 0; j < 3; ++j)
                 *reinterpret_cast<uint4*>(a_dst + (3 * (lane >> 3) + j) * 2048) = make_uint4(w[4 * j], w[4 * j + 1], w[4 * j + 2], w[4 * j + 3]);
             // ---- B: the slice of X, 16-byte chunks (8 values along K)
-            for (int i = threadIdx.x; i < ga.npad * (kStageK / 8); i += kGemmThreads) {
+            for (int i = gtid; i < ga.npad * (kStageK / 8); i += kGemmGroupThreads) {
                 const int kc = i / ga.npad, n = i % ga.npad;
                 const int64_t k = (int64_t)s * kStageK + kc * 8;
                 uint4 v = make_uint4(0, 0, 0, 0);
                 if (n < ga.batch && k < ga.k_in) v = __ldg(reinterpret_cast<const uint4*>(ga.x + (int64_t)n * ga.k_in + k));
-                *reinterpret_cast<uint4*>(b_buf + buf * b_stage + (uint32_t)kc * ga.npad * 16 + n * 16) = v;
+                *reinterpret_cast<uint4*>(b_mine + (uint32_t)kc * ga.npad * 16 + n * 16) = v;
             }
             fence_async_smem();
-            __syncthreads();
-            if (threadIdx.x == 0) {
+            group_barrier(group);
+            if (gtid == 0) {
                 tc_fence_after();
-                const uint32_t a_addr = smem_u32(a_buf + buf * (kGemmRows * kStageK * 2));
-                const uint32_t b_addr = smem_u32(b_buf + buf * b_stage);
+                const uint32_t a_addr = smem_u32(a_mine), b_addr = smem_u32(b_mine);
 #pragma unroll
                 for (int j = 0; j < kStageK / 16; ++j)
-                    umma_bf16(tmem, smem_desc(a_addr + j * 4096, 2048, 128), smem_desc(b_addr + j * 2 * ga.npad * 16, ga.npad * 16, 128),
-                              idesc, (s > s_begin || j > 0) ? 1u : 0u);
-                umma_commit(&bar_free[buf]);
-                if (s == s_end - 1) umma_commit(bar_done);
+                    umma_bf16(tmem + 64u * group, smem_desc(a_addr + j * 4096, 2048, 128),
+                              smem_desc(b_addr + j * 2 * ga.npad * 16, ga.npad * 16, 128), idesc, (s > s_begin + group || j > 0) ? 1u : 0u);
+                umma_commit(&bar_free[group]);
+                if (s + 2 >= s_end) umma_commit(&bar_done[group]);
             }
         }
-        if (failed) break;
-        // ---- epilogue: accumulator -> scratch (split-K) or Y
-        if (s_end > s_begin) {
-            const bool ok = mbar_wait(bar_done, gitem & 1u);
-            if (__syncthreads_or(!ok)) { failed = true; break; }
+        // ---- epilogue: accumulators -> scratch (split-K) or Y
+        const bool has0 = s_end > s_begin, has1 = s_end > s_begin + 1;
+        if (warp < 4) {
+            if (has0 && !mbar_wait(&bar_done[0], done[0] & 1u)) timeout = true;
+            if (has1 && !mbar_wait(&bar_done[1], done[1] & 1u)) timeout = true;
             tc_fence_after();
-            if (warp < 4) {
-                const int64_t orow = rt * kGemmRows + warp * 32 + lane;
-                for (int c0 = 0; c0 < ga.npad; c0 += 16) {
-                    float v[16];
-                    tmem_ld16(tmem + ((uint32_t)(warp * 32) << 16) + (uint32_t)c0, v);
-                    if (orow < ga.n_out) {
+            const int64_t orow = rt * kGemmRows + warp * 32 + lane;
+            for (int c0 = 0; c0 < ga.npad && has0; c0 += 16) {
+                float v[16], v1[16];
+                tmem_ld16(tmem + ((uint32_t)(warp * 32) << 16) + (uint32_t)c0, v);
+                if (has1) {
+                    tmem_ld16(tmem + ((uint32_t)(warp * 32) << 16) + 64u + (uint32_t)c0, v1);
 #pragma unroll
-                        for (int i = 0; i < 16; ++i) {
-                            const int n = c0 + i;
-                            if (n < ga.batch) {
-                                if (ga.split == 1) reinterpret_cast<__nv_bfloat16*>(ga.y)[(int64_t)n * ga.n_out + orow] = __float2bfloat16_rn(v[i]);
-                                else atomicAdd(ga.scratch + (int64_t)n * ga.scratch_ld + orow, v[i]);
-                            }
+                    for (int i = 0; i < 16; ++i) v[i] += v1[i];
+                }
+                if (orow < ga.n_out) {
+#pragma unroll
+                    for (int i = 0; i < 16; ++i) {
+                        const int n = c0 + i;
+                        if (n < ga.batch) {
+                            if (ga.split == 1) reinterpret_cast<__nv_bfloat16*>(ga.y)[(int64_t)n * ga.n_out + orow] = __float2bfloat16_rn(v[i]);
+                            else atomicAdd(ga.scratch + (int64_t)n * ga.scratch_ld + orow, v[i]);
                         }
                     }
                 }
             }
             tc_fence_before();
-        } else {
-            --gitem;                                        // no MMA was committed for this item
         }
+        done[0] += has0; done[1] += has1;
         if (ga.split > 1) {
             __threadfence();
             __syncthreads();
@@ -558,7 +569,7 @@ gemm_kernel(FastArgs fa, DevCode dc, const uint32_t* __restrict__ stream, const 
         }
         __syncthreads();
     }
-    if (failed && threadIdx.x == 0) atomicOr(fa.flags, 1u);
+    if (timeout) atomicOr(fa.flags, 1u);
     __syncthreads();
     if (warp == 0) tmem_dealloc(tmem, kTmemCols);
 }
