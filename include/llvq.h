@@ -160,6 +160,15 @@ int llvq_gemm_small_batch_noalloc(const llvq_ctx* ctx, const void* d_idx, const 
                                   int batch, uint16_t* d_y_bf16, void* stream);
 
 /*
+ * Self-test of the error path every kernel of this library uses for its device-side waits (table copy,
+ * tensor-core completion): launches a one-warp kernel that waits, with a small iteration limit, on a barrier
+ * nothing arrives at, sees the limit run out, sets LLVQ_FLAG_WAIT_TIMEOUT and returns normally.  Nothing
+ * faults or hangs; the context stays usable.  llvq_last_error then reports the flag.  (No counterpart in the
+ * paper.)
+ */
+int llvq_selftest_wait_timeout(llvq_ctx* ctx, void* stream);
+
+/*
  * Synchronises `stream`, then reports and clears the device-side error state:
  * *n_bad_index = number of fields with I >= N seen since the last call,
  * *flags = OR of LLVQ_FLAG_* bits.  Either output pointer may be NULL.

@@ -29,7 +29,7 @@ _STATUS = {0: "LLVQ_OK", 1: "LLVQ_EINVAL", 2: "LLVQ_EALIGN", 3: "LLVQ_EUNSUPPORT
 EXPORTS = [
     "llvq_create", "llvq_destroy", "llvq_index_bits", "llvq_num_points", "llvq_num_classes", "llvq_index_bytes",
     "llvq_decode_blocks", "llvq_dequant_matrix", "llvq_gemv", "llvq_gemm_small_batch", "llvq_gemm_small_batch_noalloc",
-    "llvq_last_error",
+    "llvq_selftest_wait_timeout", "llvq_last_error",
 ]
 
 
@@ -64,6 +64,7 @@ def load_library() -> ctypes.CDLL:
     lib.llvq_gemv.argtypes = [vp, vp, vp, i64, i64, vp, vp, ctypes.c_int, vp]
     lib.llvq_gemm_small_batch.argtypes = [vp, vp, vp, i64, i64, vp, ctypes.c_int, vp, vp]
     lib.llvq_gemm_small_batch_noalloc.argtypes = [vp, vp, vp, i64, i64, vp, ctypes.c_int, vp, vp]
+    lib.llvq_selftest_wait_timeout.argtypes = [vp, vp]
     lib.llvq_last_error.argtypes = [vp, vp, ctypes.POINTER(u64), ctypes.POINTER(ctypes.c_uint32)]
     lib.llvq_class_info.argtypes = [vp, ctypes.c_int, vp, vp, vp, vp, vp, vp]
     lib.llvq_golay_table.argtypes = [vp, vp]
@@ -208,6 +209,11 @@ def llvq_gemm_small_batch_noalloc(ctx: Context, d_idx: torch.Tensor, d_gain: tor
     _check("llvq_gemm_small_batch_noalloc", ctx._lib.llvq_gemm_small_batch_noalloc(
         ctx._h, _dev(d_idx, "d_idx"), _dev(d_gain, "d_gain"), n_out, k_in, _dev(d_x, "d_x"), batch, _dev(d_y, "d_y"), _stream_ptr(stream)))
     return d_y
+
+
+def llvq_selftest_wait_timeout(ctx: Context, stream=None) -> None:
+    """Run the bounded-wait self-test kernel: afterwards ``llvq_last_error`` reports LLVQ_FLAG_WAIT_TIMEOUT."""
+    _check("llvq_selftest_wait_timeout", ctx._lib.llvq_selftest_wait_timeout(ctx._h, _stream_ptr(stream)))
 
 
 def llvq_last_error(ctx: Context, stream=None) -> tuple[int, int]:

@@ -274,13 +274,14 @@ dequant_fast_kernel(FastArgs fa, const uint32_t* __restrict__ stream, const uint
     }
 }
 
-// Fused dequant + GEMV.  The work is cut into units of 16 rows x 4 column blocks, numbered row group major, and
+// Fused dequant + GEMV.  The work is cut into units of 8 rows x 4 column blocks, numbered row group major, and
 // every CTA takes an equal contiguous range of units.  In a unit lane (g, t) = (lane / 4, lane % 4) decodes the
-// blocks (row g, column block 4q + t) and (row g + 8, same column block); their 2 x 12 packed bf16 pairs are
-// the A fragments of six m16n8k16 tensor-core MMAs whose B fragment carries the matching 4 x 24 activations
-// (the same in all 8 columns), accumulating in binary32.  Row sums are collected in shared memory; a row
-// group that is split between CTAs is finished through a zero-kept global scratch and an arrival counter.
-constexpr int kGemvGroupsPerPass = 64;   // row groups (of 16 rows) whose sums a CTA keeps in shared memory at a time
+// block (row g, column block 4q + t); its 12 packed bf16 pairs are the A fragments (rows 0..7; rows 8..15 are
+// zero) of six m16n8k16 tensor-core MMAs whose B fragment carries the matching 4 x 24 activations (the same in
+// all 8 columns), accumulating in binary32.  Row sums are collected in shared memory; a row group that is
+// split between CTAs is finished through a zero-kept global scratch and an arrival counter.
+constexpr int kGemvGroupRows = 8;        // rows per unit
+constexpr int kGemvGroupsPerPass = 128;  // row groups whose sums a CTA keeps in shared memory at a time
 
 __device__ __forceinline__ void mma_bf16_16816(float c[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0, uint32_t b1)
 {
@@ -300,8 +301,8 @@ gemv_fast_kernel(FastArgs fa, const uint32_t* __restrict__ stream, const uint16_
     FAST_PROLOGUE();
     const int64_t nq = (bpr + 3) / 4;                               // units along K
     uint32_t* xs = reinterpret_cast<uint32_t*>(staging);            // [nq * 4][12] packed bf16 pairs of x
-    float* acc = reinterpret_cast<float*>(xs + nq * 48);            // [kGemvGroupsPerPass][16]
-    uint32_t* last_flag = reinterpret_cast<uint32_t*>(acc + kGemvGroupsPerPass * 16);
+    float* acc = reinterpret_cast<float*>(xs + nq * 48);            // [kGemvGroupsPerPass][8]
+    uint32_t* last_flag = reinterpret_cast<uint32_t*>(acc + kGemvGroupsPerPass * kGemvGroupRows);
     for (int64_t i = threadIdx.x; i < nq * 48; i += blockDim.x) {
         const int64_t e = 2 * i;
         const uint32_t lo = e < k_in ? __ldg(x + e) : 0u, hi = e + 1 < k_in ? __ldg(x + e + 1) : 0u;
@@ -309,61 +310,54 @@ gemv_fast_kernel(FastArgs fa, const uint32_t* __restrict__ stream, const uint16_
     }
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, g = lane >> 2, t = lane & 3;
     const int kWarps = (int)(blockDim.x >> 5);
-    const int64_t groups = (n_out + 15) / 16;
+    const int64_t groups = (n_out + kGemvGroupRows - 1) / kGemvGroupRows;
     const int64_t U = groups * nq, G = gridDim.x;
     const int64_t u_begin = blockIdx.x * U / G, u_end = (blockIdx.x + 1) * U / G;
     if (u_begin >= u_end) return;
     const int64_t rg_first = u_begin / nq, rg_last = (u_end - 1) / nq;
     for (int64_t rg0 = rg_first; rg0 <= rg_last; rg0 += kGemvGroupsPerPass) {
         const int64_t rg1 = min(rg0 + kGemvGroupsPerPass - 1, rg_last);
-        for (int i = threadIdx.x; i < kGemvGroupsPerPass * 16; i += (int)blockDim.x) acc[i] = 0.f;
+        for (int i = threadIdx.x; i < kGemvGroupsPerPass * kGemvGroupRows; i += (int)blockDim.x) acc[i] = 0.f;
         __syncthreads();
         const int64_t p_begin = max(u_begin, rg0 * nq), p_end = min(u_end, (rg1 + 1) * nq);
         for (int64_t u = p_begin + warp; u < p_end; u += kWarps) {
             const int64_t rg = u / nq, kq = u - rg * nq;
             const int64_t cb = kq * 4 + t;
-            const int64_t rowA = rg * 16 + g, rowB = rowA + 8;
-            const bool inA = rowA < n_out && cb < bpr, inB = rowB < n_out && cb < bpr;
-            const uint64_t bA = (uint64_t)(rowA * bpr + cb), bB = (uint64_t)(rowB * bpr + cb);
-            const uint64_t IA = inA ? load_field(stream, bA, (int)fa.L.W) : 0ull;
-            const uint64_t IB = inB ? load_field(stream, bB, (int)fa.L.W) : 0ull;
-            const float gA = inA ? gain_to_float(__ldg(gain + bA)) : 0.f;
-            const float gB = inB ? gain_to_float(__ldg(gain + bB)) : 0.f;
-            const bool vA = inA && IA < fa.n_points, vB = inB && IB < fa.n_points;
-            if ((inA && !vA) || (inB && !vB)) atomicAdd(fa.bad_index, (unsigned long long)((inA && !vA) + (inB && !vB)));
-            Decoded dA, dB;
-            fast_decode(T, IA, vA, dA);
-            fast_decode(T, IB, vB, dB);
-            uint32_t wA[12], wB[12];
-            expand_bf16(dA, gA, wA);
-            expand_bf16(dB, gB, wB);
+            const int64_t row = rg * kGemvGroupRows + g;
+            const bool in = row < n_out && cb < bpr;
+            const uint64_t b = (uint64_t)(row * bpr + cb);
+            const uint64_t I = in ? load_field(stream, b, (int)fa.L.W) : 0ull;
+            const float gn = in ? gain_to_float(__ldg(gain + b)) : 0.f;
+            const bool valid = in && I < fa.n_points;
+            if (in && !valid) atomicAdd(fa.bad_index, 1ull);
+            Decoded d;
+            fast_decode(T, I, valid, d);
+            uint32_t w[12];
+            expand_bf16(d, gn, w);
             const uint4* xb = reinterpret_cast<const uint4*>(xs + cb * 12);
             const uint4 x0 = xb[0], x1 = xb[1], x2 = xb[2];
             const uint32_t xv[12] = {x0.x, x0.y, x0.z, x0.w, x1.x, x1.y, x1.z, x1.w, x2.x, x2.y, x2.z, x2.w};
             float c[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
             for (int q = 0; q < 6; ++q)
-                mma_bf16_16816(c, wA[2 * q], wB[2 * q], wA[2 * q + 1], wB[2 * q + 1], xv[2 * q], xv[2 * q + 1]);
-            if (t == 0) {
-                atomicAdd(&acc[(rg - rg0) * 16 + g], c[0]);
-                atomicAdd(&acc[(rg - rg0) * 16 + g + 8], c[2]);
-            }
+                mma_bf16_16816(c, w[2 * q], 0u, w[2 * q + 1], 0u, xv[2 * q], xv[2 * q + 1]);
+            if (t == 0) atomicAdd(&acc[(rg - rg0) * kGemvGroupRows + g], c[0]);
         }
         __syncthreads();
         // row groups this CTA covers completely are final; the (at most two) split ones go through the scratch
         for (int64_t rg = rg0; rg <= rg1; ++rg) {
             const bool whole = u_begin <= rg * nq && (rg + 1) * nq <= u_end;
-            const int64_t row = rg * 16 + threadIdx.x;
-            const bool mine = threadIdx.x < 16 && row < n_out;
+            const int64_t row = rg * kGemvGroupRows + threadIdx.x;
+            const bool mine = threadIdx.x < kGemvGroupRows && row < n_out;
             if (whole) {
                 if (mine) {
-                    const float v = acc[(rg - rg0) * 16 + threadIdx.x];
+                    const float v = acc[(rg - rg0) * kGemvGroupRows + threadIdx.x];
                     if (kOutBf16) reinterpret_cast<__nv_bfloat16*>(y)[row] = __float2bfloat16_rn(v);
                     else reinterpret_cast<float*>(y)[row] = v;
                 }
                 continue;
             }
-            if (mine) atomicAdd(scratch + row, acc[(rg - rg0) * 16 + threadIdx.x]);
+            if (mine) atomicAdd(scratch + row, acc[(rg - rg0) * kGemvGroupRows + threadIdx.x]);
             __threadfence();
             __syncthreads();
             if (threadIdx.x == 0) {
@@ -690,7 +684,7 @@ int llvq_create(llvq_ctx** out, int m_lo, int m_hi, int device)
     ctx->fast = build_fast_image(h, ctx->fl, image);
     size_t o_img = up(o_err + 256);
     size_t o_cnt = up(o_img + (ctx->fast ? image.size() : 0));
-    size_t o_scr = up(o_cnt + (size_t)(64 * kMaxScratchRows / 16) * 4);   // one counter per group of 16 rows (GEMV) / per 128-row tile (GEMM)
+    size_t o_scr = up(o_cnt + (size_t)(64 * kMaxScratchRows / 8) * 4);    // one counter per group of 8 rows (GEMV) / per 128-row tile (GEMM)
     size_t total = o_scr + (size_t)64 * kMaxScratchRows * 4;
     std::vector<uint8_t> blob(total, 0);
     if (ctx->fast) std::memcpy(blob.data() + o_img, image.data(), image.size());
@@ -861,9 +855,9 @@ int llvq_gemv(const llvq_ctx* ctx, const void* d_idx, const uint16_t* d_gain_f16
     int64_t bpr = (k_in + 23) / 24;
     if (ctx->fast) {
         const int64_t nq = (bpr + 3) / 4;
-        const size_t smem = ctx->fl.total + 16 + (size_t)nq * 48 * 4 + kGemvGroupsPerPass * 16 * 4 + 16;
+        const size_t smem = ctx->fl.total + 16 + (size_t)nq * 48 * 4 + kGemvGroupsPerPass * kGemvGroupRows * 4 + 16;
         if (smem > 227 * 1024 || n_out > 64ll * kMaxScratchRows) return LLVQ_EUNSUPPORTED;
-        const int64_t units = ((n_out + 15) / 16) * nq;
+        const int64_t units = ((n_out + kGemvGroupRows - 1) / kGemvGroupRows) * nq;
         unsigned g = (unsigned)std::min<int64_t>(units, ctx->sm_count);
         // warps per CTA: the count in [20, 32] that wastes the fewest warp slots on the units of one CTA
         const int64_t upc = (units + g - 1) / g;
@@ -946,6 +940,34 @@ int llvq_gemm_small_batch_noalloc(const llvq_ctx* ctx, const void* d_idx, const 
     if (cudaMemsetAsync(base, 0, used, (cudaStream_t)stream) != cudaSuccess) return LLVQ_ECUDA;
     return launch_gemm(ctx, d_idx, d_gain_f16, n_out, k_in, d_x_bf16, batch, d_y_bf16,
                        reinterpret_cast<float*>(base + kNoallocCounterBytes), reinterpret_cast<uint32_t*>(base), stream);
+}
+
+// Waits, with a small iteration limit, on an mbarrier that nothing ever arrives at, then records the expiry the
+// same way the real kernels do.  Exercises the "bounded wait -> error flag -> normal return" path without any fault.
+__global__ void selftest_wait_kernel(uint32_t* flags)
+{
+    __shared__ uint64_t bar;
+    if (threadIdx.x == 0) {
+        mbar_init(&bar, 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    __syncthreads();
+    const uint32_t a = smem_u32(&bar);
+    uint32_t done = 0;
+    for (uint32_t it = 0; it < 64u && !done; ++it) {
+        asm volatile("{\n .reg .pred p;\n mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n selp.u32 %0, 1, 0, p;\n}"
+                     : "=r"(done) : "r"(a), "r"(0u) : "memory");
+    }
+    if (!done && threadIdx.x == 0) atomicOr(flags, (uint32_t)LLVQ_FLAG_WAIT_TIMEOUT);
+}
+
+int llvq_selftest_wait_timeout(llvq_ctx* ctx, void* stream)
+{
+    if (!ctx || ctx->device < 0) return LLVQ_EINVAL;
+    DeviceGuard guard(ctx->device);
+    if (!guard.ok) return LLVQ_ECUDA;
+    selftest_wait_kernel<<<1, 32, 0, (cudaStream_t)stream>>>(ctx->dev.flags);
+    return launch_status();
 }
 
 int llvq_last_error(llvq_ctx* ctx, void* stream, uint64_t* n_bad_index, uint32_t* flags)

@@ -348,3 +348,15 @@ def test_smallest_and_odd_shapes(lib, ctxs, oracle_mod):
     # zero-sized calls are accepted and touch nothing
     assert lib.llvq_dequant_matrix(ctx, torch.zeros(16, dtype=torch.uint8, device="cuda"), torch.zeros(1, dtype=torch.float16, device="cuda"),
                                    0, 24, 1).numel() == 0
+
+
+def test_bounded_wait_reports_timeout_and_context_stays_usable(lib, ctxs, oracle_mod):
+    # a wait nothing satisfies runs into its iteration limit: the kernel returns, the flag is set, later calls work
+    ctx = ctxs[(2, 2)]
+    assert lib.llvq_last_error(ctx) == (0, 0)
+    lib.llvq_selftest_wait_timeout(ctx)
+    assert lib.llvq_last_error(ctx) == (0, 1)            # LLVQ_FLAG_WAIT_TIMEOUT
+    assert lib.llvq_last_error(ctx) == (0, 0)            # cleared by the read
+    o = _oracle(oracle_mod)((2, 2))
+    lo = np.arange(100, dtype=np.uint64)
+    assert np.array_equal(_decode_gpu(lib, ctx, lo, np.zeros_like(lo)), o.unrank_arrays(lo, np.zeros_like(lo)))
