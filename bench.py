@@ -288,6 +288,22 @@ def extras(P, ctx) -> dict:
     us = _event_us(torch, token, 3)
     blocks = 32 * sum(n * ((k + 23) // 24) for n, k in shapes)
     by = blocks * (CODE_W // 8 + 2) + 32 * sum(2 * k + 2 * n for n, k in shapes)
+    # --- the one shape the paper timed (App. C): (4096 x 4104) . (4104 x 1), single shell M = 3 (24-bit indices, 1 bit/weight)
+    ctx3 = P.Context(3, 3, device=torch.cuda.current_device())
+    n, k = 4096, 4104
+    bufs3 = []
+    for c in range(64):                                   # 64 x 2.8 MB > L2
+        stream, gain, nb3 = gen.make_layer(ctx3.num_points, ctx3.index_bits, n, k, 1, seed=400 + c)
+        bufs3.append((dev(stream), dev(gain, np.float16)))
+    x3 = dev(gen.normal_bf16(k, seed=3), np.int16).view(torch.bfloat16)
+    y3 = torch.empty(n, dtype=torch.bfloat16, device="cuda")
+    fn = lambda i: P.llvq_gemv(ctx3, bufs3[i % 64][0], bufs3[i % 64][1], n, k, x3, d_y=y3)
+    _event_us(torch, fn, 16)
+    us3 = _event_us(torch, fn, 128)
+    by3 = nb3 * (24 // 8 + 2) + 2 * k + 2 * n
+    out["paper_shape_shell3_4096x4104_gemv"] = {"us": us3, "GBps": by3 / us3 / 1e3, "weights_per_s": n * k / (us3 * 1e-6),
+                                                "paper_us_fp16_unnamed_gpu": 11.94, "algorithmic_bytes": by3}
+    del bufs3
     out["llama3_8b_linear_sweep"] = {"us_per_token": us, "tokens_per_s": 1e6 / us, "GBps": by / us / 1e3, "blocks_per_token": blocks,
                                      "launches_per_token": 32 * len(shapes), "algorithmic_bytes": by}
     return out

@@ -276,22 +276,31 @@ __device__ __forceinline__ void expand_bytes(const Decoded& d, uint32_t out[6])
 }
 
 // The 24 dequantized weights bf16_rn(gain * x_i) as 12 packed pairs (weight 2j in the low half of w[j]).
+// All lanes of the warp must call this together: when no lane uses a value id above 3 (codes with few distinct
+// values per class) the third bit plane and the upper half of the value table are skipped.
 __device__ __forceinline__ void expand_bf16(const Decoded& d, float gain, uint32_t w[12])
 {
-    // bf16(gain * a) for the eight value ids; float(a) by the 2^23 trick (a <= 28)
-    uint32_t packed[4];
+    const bool wide = __any_sync(kFullMask, d.p2 != 0u);
+    // bf16(gain * a) for the value ids; float(a) by the 2^23 trick (a <= 28)
+    uint32_t packed[4] = {0u, 0u, 0u, 0u};
 #pragma unroll
     for (int i = 0; i < 4; ++i) {
-        const uint32_t src = i < 2 ? d.vals_lo : d.vals_hi;
-        const float a0 = __uint_as_float(__byte_perm(src, 0x4b000000u, (i & 1) ? 0x7442 : 0x7440)) - 8388608.f;
-        const float a1 = __uint_as_float(__byte_perm(src, 0x4b000000u, (i & 1) ? 0x7443 : 0x7441)) - 8388608.f;
-        __nv_bfloat162 b = __floats2bfloat162_rn(gain * a0, gain * a1);
-        packed[i] = *reinterpret_cast<uint32_t*>(&b);
+        if (i < 2 || wide) {
+            const uint32_t src = i < 2 ? d.vals_lo : d.vals_hi;
+            const float a0 = __uint_as_float(__byte_perm(src, 0x4b000000u, (i & 1) ? 0x7442 : 0x7440)) - 8388608.f;
+            const float a1 = __uint_as_float(__byte_perm(src, 0x4b000000u, (i & 1) ? 0x7443 : 0x7441)) - 8388608.f;
+            __nv_bfloat162 b = __floats2bfloat162_rn(gain * a0, gain * a1);
+            packed[i] = *reinterpret_cast<uint32_t*>(&b);
+        }
     }
     const uint32_t lo03 = __byte_perm(packed[0], packed[1], 0x6420), hi03 = __byte_perm(packed[0], packed[1], 0x7531);
     const uint32_t lo47 = __byte_perm(packed[2], packed[3], 0x6420), hi47 = __byte_perm(packed[2], packed[3], 0x7531);
     uint32_t sel[3];
-    id_nibbles(d, sel);
+#pragma unroll
+    for (int r = 0; r < 3; ++r) {
+        sel[r] = nibspread8((d.p0 >> (8 * r)) & 0xffu) | (nibspread8((d.p1 >> (8 * r)) & 0xffu) << 1);
+        if (wide) sel[r] |= nibspread8((d.p2 >> (8 * r)) & 0xffu) << 2;
+    }
 #pragma unroll
     for (int j = 0; j < 6; ++j) {
         const uint32_t s16 = (j & 1) ? sel[j >> 1] >> 16 : sel[j >> 1];

@@ -254,9 +254,9 @@ dequant_fast_kernel(FastArgs fa, const uint32_t* __restrict__ stream, const uint
         if (in && !valid) atomicAdd(fa.bad_index, 1ull);
         Decoded d;
         fast_decode(T, I, valid, d);
-        if (!in) continue;
         uint32_t w[12];
-        expand_bf16(d, gain_to_float(__ldg(gain + b)), w);
+        expand_bf16(d, in ? gain_to_float(__ldg(gain + b)) : 0.f, w);      // whole warp: the expansion votes
+        if (!in) continue;
         __nv_bfloat16* dst;
         int64_t left;
         if (bpr == 0) { dst = out + b * 24; left = (int64_t)(total - b * 24); }
