@@ -267,6 +267,22 @@ def extras(P, ctx) -> dict:
         by = nb * (CODE_W // 8 + 2) + batch * k * 2 + batch * n * 2
         out[f"gemm_8192x8192_b{batch}"] = {"us": us, "GBps": by / us / 1e3, "TFLOPs": 2.0 * n * k * batch / us / 1e6, "algorithmic_bytes": by}
     del bufs
+    # --- GEMM, 8192 x 8192 at ~3 bits/weight: 72-bit indices over shells 2..53
+    ctx53 = P.Context(2, 53, device=torch.cuda.current_device())
+    bufs = []
+    for c in range(8):
+        stream, gain, nb = gen.make_layer(ctx53.num_points, ctx53.index_bits, n, k, 1, seed=250 + c)
+        bufs.append((dev(stream), dev(gain, np.float16)))
+    for batch in (16, 64):
+        x = dev(gen.normal_bf16((batch, k), seed=batch), np.int16).view(torch.bfloat16)
+        y = torch.empty((batch, n), dtype=torch.bfloat16, device="cuda")
+        fn = lambda i: P.llvq_gemm_small_batch(ctx53, bufs[i % 8][0], bufs[i % 8][1], n, k, x, d_y=y)
+        _event_us(torch, fn, 4)
+        us = _event_us(torch, fn, 16)
+        by = nb * (72 // 8 + 2) + batch * k * 2 + batch * n * 2
+        out[f"gemm_8192x8192_b{batch}_72bit"] = {"us": us, "GBps": by / us / 1e3, "TFLOPs": 2.0 * n * k * batch / us / 1e6, "algorithmic_bytes": by}
+    assert P.llvq_last_error(ctx53) == (0, 0)
+    del bufs, ctx53
     # --- decoder sweep: q, k, v, o, gate, up, down of one layer; 32 layers; 4 distinct layer sets (> 2 x L2)
     shapes = [(4096, 4096), (1024, 4096), (1024, 4096), (4096, 4096), (14336, 4096), (14336, 4096), (4096, 14336)]
     sets = []

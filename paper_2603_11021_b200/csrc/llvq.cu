@@ -12,6 +12,7 @@
 
 #include "decode.cuh"
 #include "fast.cuh"
+#include "big.cuh"
 #include "umma.cuh"
 #include "tables.h"
 
@@ -26,14 +27,12 @@ struct llvq_ctx {
     int sm_count = 0;
     float* d_scratch = nullptr;      // split-K accumulation buffer of the small-batch GEMM, kept all-zero between calls
     uint32_t* d_counters = nullptr;  // per row tile arrival counters, kept zero between calls
-    bool fast = false;               // tables fit shared memory: the fast kernels are used
+    bool fast = false;               // class tables fit the shared-memory image; otherwise they are read from global memory
     FastLayout fl{};
     const uint8_t* d_image = nullptr;
 };
 
 namespace {
-
-constexpr int kThreads = 256;
 
 struct DeviceGuard {
     int prev = -1; bool ok = false;
@@ -45,135 +44,6 @@ struct DeviceGuard {
 };
 
 inline bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) & (a - 1)) == 0; }
-
-// ---------------------------------------------------------------------------
-// llvq_decode_blocks: one thread per field; the 24 bytes of a point are staged
-// through shared memory so that the stores to global memory are coalesced.
-// ---------------------------------------------------------------------------
-__global__ void __launch_bounds__(kThreads)
-decode_blocks_kernel(DevCode dc, const uint32_t* __restrict__ stream, uint64_t nblocks, uint32_t* __restrict__ out)
-{
-    __shared__ uint32_t stage[kThreads * 6];
-    const uint64_t base = (uint64_t)blockIdx.x * kThreads;
-    const uint64_t b = base + threadIdx.x;
-    Point pt;
-    if (b < nblocks) {
-        decode_field(dc, stream, b, pt);
-#pragma unroll
-        for (int i = 0; i < 6; ++i) stage[threadIdx.x * 6 + i] = pt.w[i];
-    }
-    __syncthreads();
-    const uint64_t nvalid = min((uint64_t)kThreads, nblocks - base) * 6;
-    for (uint32_t i = threadIdx.x; i < nvalid; i += kThreads) out[base * 6 + i] = stage[i];
-}
-
-// ---------------------------------------------------------------------------
-// llvq_dequant_matrix
-// ---------------------------------------------------------------------------
-// FLAT layout: block b -> elements 24b..24b+23 of the flattened matrix.
-__global__ void __launch_bounds__(kThreads)
-dequant_flat_kernel(DevCode dc, const uint32_t* __restrict__ stream, const uint16_t* __restrict__ gain,
-                    uint64_t nblocks, uint64_t total, __nv_bfloat16* __restrict__ out, int vec_ok)
-{
-    __shared__ uint32_t stage[kThreads * 12];
-    const uint64_t base = (uint64_t)blockIdx.x * kThreads;
-    const uint64_t b = base + threadIdx.x;
-    if (b < nblocks) {
-        Point pt;
-        decode_field(dc, stream, b, pt);
-        const float g = gain_to_float(__ldg(gain + b));
-#pragma unroll
-        for (int j = 0; j < 12; ++j) {
-            __nv_bfloat162 v = __halves2bfloat162(dequant(g, pt, 2 * j), dequant(g, pt, 2 * j + 1));
-            stage[threadIdx.x * 12 + j] = *reinterpret_cast<uint32_t*>(&v);
-        }
-    }
-    __syncthreads();
-    const uint64_t first = base * 24;                          // first element of this CTA
-    const uint64_t count = min((uint64_t)kThreads * 24, total - first);
-    if (vec_ok && count == (uint64_t)kThreads * 24) {
-        uint4* dst = reinterpret_cast<uint4*>(out + first);    // first*2 bytes = base*48: 16-byte aligned
-        const uint4* src = reinterpret_cast<const uint4*>(stage);
-        for (uint32_t i = threadIdx.x; i < kThreads * 3; i += kThreads) dst[i] = src[i];
-    } else {
-        const __nv_bfloat16* src = reinterpret_cast<const __nv_bfloat16*>(stage);
-        for (uint64_t i = threadIdx.x; i < count; i += kThreads) out[first + i] = src[i];
-    }
-}
-
-// ROWWISE layout: block (r, cb) -> columns 24cb..24cb+23 of row r; leading dimension ld.
-__global__ void __launch_bounds__(kThreads)
-dequant_rowwise_kernel(DevCode dc, const uint32_t* __restrict__ stream, const uint16_t* __restrict__ gain,
-                       int64_t rows, int64_t cols, int64_t bpr, __nv_bfloat16* __restrict__ out, int64_t ld)
-{
-    const uint64_t b = (uint64_t)blockIdx.x * kThreads + threadIdx.x;
-    if (b >= (uint64_t)(rows * bpr)) return;
-    const int64_t r = (int64_t)(b / (uint64_t)bpr), cb = (int64_t)(b % (uint64_t)bpr);
-    Point pt;
-    decode_field(dc, stream, b, pt);
-    const float g = gain_to_float(__ldg(gain + b));
-    __nv_bfloat16* dst = out + r * ld + cb * 24;
-    const int64_t left = cols - cb * 24;
-    if (left >= 24 && (reinterpret_cast<uintptr_t>(dst) & 15) == 0) {
-        uint32_t v[12];
-#pragma unroll
-        for (int j = 0; j < 12; ++j) {
-            __nv_bfloat162 h = __halves2bfloat162(dequant(g, pt, 2 * j), dequant(g, pt, 2 * j + 1));
-            v[j] = *reinterpret_cast<uint32_t*>(&h);
-        }
-        uint4* d4 = reinterpret_cast<uint4*>(dst);
-        d4[0] = make_uint4(v[0], v[1], v[2], v[3]);
-        d4[1] = make_uint4(v[4], v[5], v[6], v[7]);
-        d4[2] = make_uint4(v[8], v[9], v[10], v[11]);
-    } else {
-#pragma unroll
-        for (int j = 0; j < 24; ++j)
-            if (j < left) dst[j] = dequant(g, pt, j);
-    }
-}
-
-// ---------------------------------------------------------------------------
-// llvq_gemv: one warp per output row; lanes stride over the row's blocks; x is
-// staged in shared memory as binary32, 25 words per block of 24 to keep the
-// lanes of a warp on distinct banks.
-// ---------------------------------------------------------------------------
-constexpr int kGemvWarps = 8;
-
-template <bool kOutBf16>
-__global__ void __launch_bounds__(kGemvWarps * 32)
-gemv_kernel(DevCode dc, const uint32_t* __restrict__ stream, const uint16_t* __restrict__ gain,
-            int64_t n_out, int64_t k_in, int64_t bpr, const uint16_t* __restrict__ x, void* __restrict__ y)
-{
-    extern __shared__ float xs[];                              // [bpr][25]
-    for (int64_t i = threadIdx.x; i < bpr * 24; i += blockDim.x) {
-        float v = 0.f;
-        if (i < k_in) v = __bfloat162float(__ushort_as_bfloat16(__ldg(x + i)));
-        xs[(i / 24) * 25 + (i % 24)] = v;
-    }
-    __syncthreads();
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int64_t row = (int64_t)blockIdx.x * kGemvWarps + warp;
-    if (row >= n_out) return;
-    float acc = 0.f;
-    for (int64_t cb = lane; cb < bpr; cb += 32) {
-        const uint64_t b = (uint64_t)(row * bpr + cb);
-        Point pt;
-        decode_field(dc, stream, b, pt);
-        const float g = gain_to_float(__ldg(gain + b));
-        const float* xb = xs + cb * 25;
-        float part = 0.f;
-#pragma unroll
-        for (int j = 0; j < 24; ++j) part = fmaf(__bfloat162float(dequant(g, pt, j)), xb[j], part);
-        acc += part;
-    }
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
-    if (lane == 0) {
-        if (kOutBf16) reinterpret_cast<__nv_bfloat16*>(y)[row] = __float2bfloat16_rn(acc);
-        else reinterpret_cast<float*>(y)[row] = acc;
-    }
-}
-
 
 // ===========================================================================
 // Fast path (tables in shared memory).  Dynamic shared memory of every fast
@@ -188,22 +58,66 @@ struct FastArgs {
     const uint8_t* image;
     uint32_t* flags;
     unsigned long long* bad_index;
-    uint64_t n_points;              // N (fits 64 bits on the fast path)
+    uint64_t n_points;              // N when it fits 64 bits (fast path)
+    DevCode dc;                     // class tables in global memory (big codes)
 };
 
-// Field b of a stream of W-bit fields, W <= 64: at most three 32-bit words, the third only when the field reaches it.
-__device__ __forceinline__ uint64_t load_field(const uint32_t* __restrict__ stream, uint64_t b, int W)
+// One block of 24 weights, end to end, in the two forms the consumers use.  kBig selects the decoder for codes
+// whose class tables live in global memory; otherwise everything is served from the shared-memory image.
+// All 32 lanes of a warp call these together; `in` = the block exists.
+template <bool kBig>
+__device__ __forceinline__ void block_point(const FastArgs& fa, const FastSmem& T, const uint32_t* __restrict__ stream,
+                                            uint64_t b, bool in, Point& pt)
 {
-    const uint64_t bp = b * (uint64_t)W;
-    const uint32_t* p = stream + (bp >> 5);
-    const int sh = (int)(bp & 31);
-    const int last = sh + W;                                     // bits of the field counted from the first word
-    const uint32_t w0 = __ldg(p);
-    const uint32_t w1 = last > 32 ? __ldg(p + 1) : 0u;
-    const uint32_t w2 = last > 64 ? __ldg(p + 2) : 0u;
-    uint64_t v = (((uint64_t)w1 << 32) | w0) >> sh;
-    if (sh) v |= (uint64_t)w2 << (64 - sh);
-    return W < 64 ? v & ((1ull << W) - 1) : v;
+    uint64_t lo = 0, hi = 0;
+    if (in) load_index(stream, b, fa.dc.W, lo, hi);
+    const bool valid = in && (hi < fa.dc.n_hi || (hi == fa.dc.n_hi && lo < fa.dc.n_lo));
+    if (in && !valid) atomicAdd(fa.bad_index, 1ull);
+    uint64_t local = 0;
+    const int cls = valid ? big_find_class(fa.dc, lo, hi, local) : 0;
+    big_decode_local(T, fa.dc, cls, local, valid, pt);
+}
+
+template <bool kBig>
+__device__ __forceinline__ void block_bytes(const FastArgs& fa, const FastSmem& T, const uint32_t* __restrict__ stream,
+                                            uint64_t b, bool in, uint32_t w[6])
+{
+    if (kBig) {
+        Point pt;
+        block_point<kBig>(fa, T, stream, b, in, pt);
+#pragma unroll
+        for (int i = 0; i < 6; ++i) w[i] = pt.w[i];
+    } else {
+        const uint64_t I = in ? load_field(stream, b, (int)fa.L.W) : 0ull;
+        const bool valid = in && I < fa.n_points;
+        if (in && !valid) atomicAdd(fa.bad_index, 1ull);
+        Decoded d;
+        fast_decode(T, I, valid, d);
+        expand_bytes(d, w);
+    }
+}
+
+template <bool kBig>
+__device__ __forceinline__ void block_pairs(const FastArgs& fa, const FastSmem& T, const uint32_t* __restrict__ stream,
+                                            const uint16_t* __restrict__ gain, uint64_t b, bool in, uint32_t w[12])
+{
+    const float g = in ? gain_to_float(__ldg(gain + b)) : 0.f;
+    if (kBig) {
+        Point pt;
+        block_point<kBig>(fa, T, stream, b, in, pt);
+#pragma unroll
+        for (int j = 0; j < 12; ++j) {
+            __nv_bfloat162 h = __halves2bfloat162(dequant(g, pt, 2 * j), dequant(g, pt, 2 * j + 1));
+            w[j] = *reinterpret_cast<uint32_t*>(&h);
+        }
+    } else {
+        const uint64_t I = in ? load_field(stream, b, (int)fa.L.W) : 0ull;
+        const bool valid = in && I < fa.n_points;
+        if (in && !valid) atomicAdd(fa.bad_index, 1ull);
+        Decoded d;
+        fast_decode(T, I, valid, d);
+        expand_bf16(d, g, w);
+    }
 }
 
 #define FAST_PROLOGUE()                                                                         \
@@ -214,6 +128,7 @@ __device__ __forceinline__ uint64_t load_field(const uint32_t* __restrict__ stre
     if (!fast_load_image(smem, fa.image, fa.L.total, bar, fa.flags)) return;                    \
     const FastSmem T = fast_view(smem, fa.L);
 
+template <bool kBig>
 __global__ void __launch_bounds__(kFastThreads, 1)
 decode_blocks_fast_kernel(FastArgs fa, const uint32_t* __restrict__ stream, uint64_t nblocks, uint2* __restrict__ out)
 {
@@ -222,14 +137,9 @@ decode_blocks_fast_kernel(FastArgs fa, const uint32_t* __restrict__ stream, uint
     for (uint64_t tile = blockIdx.x; tile < ntiles; tile += gridDim.x) {
         const uint64_t b = tile * kFastThreads + threadIdx.x;
         const bool in = b < nblocks;
-        const uint64_t I = in ? load_field(stream, b, (int)fa.L.W) : 0ull;
-        const bool valid = in && I < fa.n_points;
-        if (in && !valid) atomicAdd(fa.bad_index, 1ull);
-        Decoded d;
-        fast_decode(T, I, valid, d);
+        uint32_t w[6];
+        block_bytes<kBig>(fa, T, stream, b, in, w);
         if (in) {
-            uint32_t w[6];
-            expand_bytes(d, w);
             out[b * 3 + 0] = make_uint2(w[0], w[1]);
             out[b * 3 + 1] = make_uint2(w[2], w[3]);
             out[b * 3 + 2] = make_uint2(w[4], w[5]);
@@ -239,6 +149,7 @@ decode_blocks_fast_kernel(FastArgs fa, const uint32_t* __restrict__ stream, uint
 
 // FLAT (bpr == 0): block b covers elements 24b.. of the flattened matrix.
 // ROWWISE: block b = r * bpr + cb covers columns 24cb.. of row r.
+template <bool kBig>
 __global__ void __launch_bounds__(kFastThreads, 1)
 dequant_fast_kernel(FastArgs fa, const uint32_t* __restrict__ stream, const uint16_t* __restrict__ gain, uint64_t nblocks,
                     int64_t rows, int64_t cols, int64_t bpr, __nv_bfloat16* __restrict__ out, int64_t ld)
@@ -249,13 +160,8 @@ dequant_fast_kernel(FastArgs fa, const uint32_t* __restrict__ stream, const uint
     for (uint64_t tile = blockIdx.x; tile < ntiles; tile += gridDim.x) {
         const uint64_t b = tile * kFastThreads + threadIdx.x;
         const bool in = b < nblocks;
-        const uint64_t I = in ? load_field(stream, b, (int)fa.L.W) : 0ull;
-        const bool valid = in && I < fa.n_points;
-        if (in && !valid) atomicAdd(fa.bad_index, 1ull);
-        Decoded d;
-        fast_decode(T, I, valid, d);
         uint32_t w[12];
-        expand_bf16(d, in ? gain_to_float(__ldg(gain + b)) : 0.f, w);      // whole warp: the expansion votes
+        block_pairs<kBig>(fa, T, stream, gain, b, in, w);             // whole warp: the decoders vote
         if (!in) continue;
         __nv_bfloat16* dst;
         int64_t left;
@@ -292,7 +198,7 @@ __device__ __forceinline__ void mma_bf16_16816(float c[4], uint32_t a0, uint32_t
 // CTA that owns unit u when G CTAs split U units into ranges [c*U/G, (c+1)*U/G).
 __device__ __forceinline__ int64_t unit_owner(int64_t u, int64_t U, int64_t G) { return ((u + 1) * G - 1) / U; }
 
-template <bool kOutBf16>
+template <bool kBig, bool kOutBf16>
 __global__ void __launch_bounds__(kGemvThreads, 1)
 gemv_fast_kernel(FastArgs fa, const uint32_t* __restrict__ stream, const uint16_t* __restrict__ gain,
                  int64_t n_out, int64_t k_in, int64_t bpr, const uint16_t* __restrict__ x, void* __restrict__ y,
@@ -326,14 +232,8 @@ gemv_fast_kernel(FastArgs fa, const uint32_t* __restrict__ stream, const uint16_
             const int64_t row = rg * kGemvGroupRows + g;
             const bool in = row < n_out && cb < bpr;
             const uint64_t b = (uint64_t)(row * bpr + cb);
-            const uint64_t I = in ? load_field(stream, b, (int)fa.L.W) : 0ull;
-            const float gn = in ? gain_to_float(__ldg(gain + b)) : 0.f;
-            const bool valid = in && I < fa.n_points;
-            if (in && !valid) atomicAdd(fa.bad_index, 1ull);
-            Decoded d;
-            fast_decode(T, I, valid, d);
             uint32_t w[12];
-            expand_bf16(d, gn, w);
+            block_pairs<kBig>(fa, T, stream, gain, b, in, w);
             const uint4* xb = reinterpret_cast<const uint4*>(xs + cb * 12);
             const uint4 x0 = xb[0], x1 = xb[1], x2 = xb[2];
             const uint32_t xv[12] = {x0.x, x0.y, x0.z, x0.w, x1.x, x1.y, x1.z, x1.w, x2.x, x2.y, x2.z, x2.w};
@@ -414,12 +314,12 @@ __device__ __forceinline__ void group_barrier(int group)
     asm volatile("bar.sync %0, %1;" ::"r"(1 + group), "n"(kGemmGroupThreads) : "memory");
 }
 
-template <bool kFast>
+template <bool kBig>
 __global__ void __launch_bounds__(kGemmThreads, 1)
-gemm_kernel(FastArgs fa, DevCode dc, const uint32_t* __restrict__ stream, const uint16_t* __restrict__ gain, GemmArgs ga)
+gemm_kernel(FastArgs fa, const uint32_t* __restrict__ stream, const uint16_t* __restrict__ gain, GemmArgs ga)
 {
     extern __shared__ __align__(128) uint8_t smem[];
-    const uint32_t img_bytes = kFast ? fa.L.total : 0u;
+    const uint32_t img_bytes = fa.L.total;
     uint64_t* bar_img = reinterpret_cast<uint64_t*>(smem + img_bytes);
     uint64_t* bar_free = bar_img + 1;                                     // [2]: the MMAs reading group h's buffers are done
     uint64_t* bar_done = bar_img + 3;                                     // [2]: group h's accumulator of this item is complete
@@ -430,11 +330,8 @@ gemm_kernel(FastArgs fa, DevCode dc, const uint32_t* __restrict__ stream, const 
     uint8_t* b_buf = a_buf + 2 * kGemmRows * kStageK * 2;                  // [2 groups] x npad * 192
     const uint32_t b_stage = (uint32_t)ga.npad * kStageK * 2;
 
-    FastSmem T{};
-    if (kFast) {
-        if (!fast_load_image(smem, fa.image, fa.L.total, bar_img, fa.flags)) return;
-        T = fast_view(smem, fa.L);
-    }
+    if (!fast_load_image(smem, fa.image, fa.L.total, bar_img, fa.flags)) return;
+    const FastSmem T = fast_view(smem, fa.L);
     // Two groups of 512 threads fill alternate stages, each into its own buffers and its own accumulator
     // (TMEM columns [64 h, 64 h + npad)); the epilogue adds the two accumulators.
     const int group = threadIdx.x / kGemmGroupThreads, gtid = threadIdx.x % kGemmGroupThreads;
@@ -469,25 +366,7 @@ gemm_kernel(FastArgs fa, DevCode dc, const uint32_t* __restrict__ stream, const 
             const bool in = row < ga.n_out && cb < ga.bpr;
             const uint64_t b = in ? (uint64_t)(row * ga.bpr + cb) : 0ull;
             uint32_t w[12];
-            if (kFast) {
-                const uint64_t I = in ? load_field(stream, b, (int)fa.L.W) : 0ull;
-                const bool valid = in && I < fa.n_points;
-                if (in && !valid) atomicAdd(fa.bad_index, 1ull);
-                Decoded d;
-                fast_decode(T, I, valid, d);
-                expand_bf16(d, in ? gain_to_float(__ldg(gain + b)) : 0.f, w);
-            } else {
-                Point pt;
-#pragma unroll
-                for (int i = 0; i < 6; ++i) pt.w[i] = 0;
-                if (in) decode_field(dc, stream, b, pt);
-                const float g = in ? gain_to_float(__ldg(gain + b)) : 0.f;
-#pragma unroll
-                for (int j = 0; j < 12; ++j) {
-                    __nv_bfloat162 h = __halves2bfloat162(dequant(g, pt, 2 * j), dequant(g, pt, 2 * j + 1));
-                    w[j] = *reinterpret_cast<uint32_t*>(&h);
-                }
-            }
+            block_pairs<kBig>(fa, T, stream, gain, b, in, w);
             uint8_t* a_dst = a_mine + gwarp * 128 + (lane & 7) * 16;
 #pragma unroll
             for (int j = 0; j < 3; ++j)
@@ -573,6 +452,7 @@ FastArgs fast_args(const llvq_ctx* ctx)
     FastArgs fa;
     fa.L = ctx->fl; fa.image = ctx->d_image; fa.flags = ctx->dev.flags; fa.bad_index = ctx->dev.bad_index;
     fa.n_points = ctx->dev.n_lo;
+    fa.dc = ctx->dev;
     return fa;
 }
 
@@ -628,16 +508,16 @@ int launch_gemm(const llvq_ctx* ctx, const void* d_idx, const uint16_t* d_gain_f
     ga.split = best;
     const int64_t items = row_tiles * ga.split;
     const unsigned grid = (unsigned)std::min<int64_t>(items, ctx->sm_count);
-    const size_t img = ctx->fast ? ctx->fl.total : 0;
+    const size_t img = ctx->fl.total;
     const size_t smem = ((img + 64 + 1023) & ~size_t(1023)) + 2 * kGemmRows * kStageK * 2 + 2 * (size_t)ga.npad * kStageK * 2;
     if (smem > 227 * 1024) return LLVQ_EUNSUPPORTED;
     const uint32_t* idx = static_cast<const uint32_t*>(d_idx);
     if (ctx->fast) {
-        if (!set_smem(gemm_kernel<true>, smem)) return LLVQ_ECUDA;
-        gemm_kernel<true><<<grid, kGemmThreads, smem, st>>>(fast_args(ctx), ctx->dev, idx, d_gain_f16, ga);
-    } else {
         if (!set_smem(gemm_kernel<false>, smem)) return LLVQ_ECUDA;
-        gemm_kernel<false><<<grid, kGemmThreads, smem, st>>>(fast_args(ctx), ctx->dev, idx, d_gain_f16, ga);
+        gemm_kernel<false><<<grid, kGemmThreads, smem, st>>>(fast_args(ctx), idx, d_gain_f16, ga);
+    } else {
+        if (!set_smem(gemm_kernel<true>, smem)) return LLVQ_ECUDA;
+        gemm_kernel<true><<<grid, kGemmThreads, smem, st>>>(fast_args(ctx), idx, d_gain_f16, ga);
     }
     return launch_status();
 }
@@ -671,38 +551,39 @@ int llvq_create(llvq_ctx** out, int m_lo, int m_hi, int device)
     std::vector<uint64_t> off_lo(ncls + 1);
     std::vector<uint32_t> off_hi(ncls + 1);
     for (size_t j = 0; j <= ncls; ++j) { off_lo[j] = (uint64_t)h.offset[j]; off_hi[j] = (uint32_t)(h.offset[j] >> 64); }
+    std::vector<uint8_t> image;
+    ctx->fast = build_fast_image(h, ctx->fl, image, true);
+    if (!ctx->fast && !build_fast_image(h, ctx->fl, image, false)) { delete ctx; return LLVQ_EUNSUPPORTED; }
+    std::vector<uint32_t> lut16;
+    build_bucket_table(h, lut16);
 
-    // one blob: [golay | pascal | off_hi | off_lo | classes | error words], each part 256-byte aligned
+    // one blob: [off_hi | off_lo | classes | bucket table | error words | table image | counters | scratch], 256-byte aligned parts
     auto up = [](size_t v) { return (v + 255) & ~size_t(255); };
-    size_t o_golay = 0;
-    size_t o_pascal = up(o_golay + 4096 * 4);
-    size_t o_offhi = up(o_pascal + sizeof(h.pascal));
+    size_t o_offhi = 0;
     size_t o_offlo = up(o_offhi + (ncls + 1) * 4);
     size_t o_cls = up(o_offlo + (ncls + 1) * 8);
-    size_t o_err = up(o_cls + ncls * sizeof(ClassDesc));
-    std::vector<uint8_t> image;
-    ctx->fast = build_fast_image(h, ctx->fl, image);
+    size_t o_lut = up(o_cls + ncls * sizeof(ClassDesc));
+    size_t o_err = up(o_lut + lut16.size() * 4);
     size_t o_img = up(o_err + 256);
-    size_t o_cnt = up(o_img + (ctx->fast ? image.size() : 0));
+    size_t o_cnt = up(o_img + image.size());
     size_t o_scr = up(o_cnt + (size_t)(64 * kMaxScratchRows / 8) * 4);    // one counter per group of 8 rows (GEMV) / per 128-row tile (GEMM)
     size_t total = o_scr + (size_t)64 * kMaxScratchRows * 4;
-    std::vector<uint8_t> blob(total, 0);
-    if (ctx->fast) std::memcpy(blob.data() + o_img, image.data(), image.size());
-    std::memcpy(blob.data() + o_golay, h.golay.data(), 4096 * 4);
-    std::memcpy(blob.data() + o_pascal, h.pascal, sizeof(h.pascal));
+    std::vector<uint8_t> blob(o_cnt, 0);
     std::memcpy(blob.data() + o_offhi, off_hi.data(), (ncls + 1) * 4);
     std::memcpy(blob.data() + o_offlo, off_lo.data(), (ncls + 1) * 8);
     std::memcpy(blob.data() + o_cls, h.desc.data(), ncls * sizeof(ClassDesc));
+    std::memcpy(blob.data() + o_lut, lut16.data(), lut16.size() * 4);
+    std::memcpy(blob.data() + o_img, image.data(), image.size());
     if (cudaMalloc(&ctx->d_blob, total) != cudaSuccess) { delete ctx; return LLVQ_ECUDA; }
-    if (cudaMemcpy(ctx->d_blob, blob.data(), total, cudaMemcpyHostToDevice) != cudaSuccess) {
+    if (cudaMemcpy(ctx->d_blob, blob.data(), blob.size(), cudaMemcpyHostToDevice) != cudaSuccess ||
+        cudaMemset(static_cast<uint8_t*>(ctx->d_blob) + o_cnt, 0, total - o_cnt) != cudaSuccess) {
         cudaFree(ctx->d_blob); delete ctx; return LLVQ_ECUDA;
     }
     uint8_t* d = static_cast<uint8_t*>(ctx->d_blob);
-    ctx->dev.golay = reinterpret_cast<const uint32_t*>(d + o_golay);
-    ctx->dev.pascal = reinterpret_cast<const uint32_t*>(d + o_pascal);
     ctx->dev.off_hi = reinterpret_cast<const uint32_t*>(d + o_offhi);
     ctx->dev.off_lo = reinterpret_cast<const uint64_t*>(d + o_offlo);
     ctx->dev.cls = reinterpret_cast<const ClassDesc*>(d + o_cls);
+    ctx->dev.lut16 = reinterpret_cast<const uint32_t*>(d + o_lut);
     ctx->d_err = reinterpret_cast<unsigned long long*>(d + o_err);
     ctx->dev.bad_index = ctx->d_err;
     ctx->dev.flags = reinterpret_cast<uint32_t*>(d + o_err + 8);
@@ -777,19 +658,17 @@ int llvq_decode_blocks(const llvq_ctx* ctx, const void* d_idx, uint64_t nblocks,
     if (nblocks > (1ull << 40)) return LLVQ_EUNSUPPORTED;
     DeviceGuard guard(ctx->device);
     if (!guard.ok) return LLVQ_ECUDA;
+    const size_t smem = ctx->fl.total + 16;
+    const uint64_t tiles = (nblocks + kFastThreads - 1) / kFastThreads;
+    const unsigned g = (unsigned)std::min<uint64_t>(tiles, (uint64_t)ctx->sm_count);
+    const uint32_t* idx = static_cast<const uint32_t*>(d_idx);
     if (ctx->fast) {
-        const size_t smem = ctx->fl.total + 16;
-        if (!set_smem(decode_blocks_fast_kernel, smem)) return LLVQ_ECUDA;
-        uint64_t tiles = (nblocks + kFastThreads - 1) / kFastThreads;
-        unsigned g = (unsigned)std::min<uint64_t>(tiles, (uint64_t)ctx->sm_count);
-        decode_blocks_fast_kernel<<<g, kFastThreads, smem, (cudaStream_t)stream>>>(
-            fast_args(ctx), static_cast<const uint32_t*>(d_idx), nblocks, reinterpret_cast<uint2*>(d_points));
-        return launch_status();
+        if (!set_smem(decode_blocks_fast_kernel<false>, smem)) return LLVQ_ECUDA;
+        decode_blocks_fast_kernel<false><<<g, kFastThreads, smem, (cudaStream_t)stream>>>(fast_args(ctx), idx, nblocks, reinterpret_cast<uint2*>(d_points));
+    } else {
+        if (!set_smem(decode_blocks_fast_kernel<true>, smem)) return LLVQ_ECUDA;
+        decode_blocks_fast_kernel<true><<<g, kFastThreads, smem, (cudaStream_t)stream>>>(fast_args(ctx), idx, nblocks, reinterpret_cast<uint2*>(d_points));
     }
-    uint64_t grid = (nblocks + kThreads - 1) / kThreads;
-    if (grid > 0x7fffffffull) return LLVQ_EUNSUPPORTED;
-    decode_blocks_kernel<<<(unsigned)grid, kThreads, 0, (cudaStream_t)stream>>>(
-        ctx->dev, static_cast<const uint32_t*>(d_idx), nblocks, reinterpret_cast<uint32_t*>(d_points));
     return launch_status();
 }
 
@@ -807,32 +686,19 @@ int llvq_dequant_matrix(const llvq_ctx* ctx, const void* d_idx, const uint16_t* 
     if (!guard.ok) return LLVQ_ECUDA;
     cudaStream_t st = (cudaStream_t)stream;
     if (layout == LLVQ_LAYOUT_FLAT && ld != cols) return LLVQ_EINVAL;
+    const int64_t bpr = layout == LLVQ_LAYOUT_FLAT ? 0 : (cols + 23) / 24;
+    const uint64_t nblocks = layout == LLVQ_LAYOUT_FLAT ? ((uint64_t)rows * (uint64_t)cols + 23) / 24 : (uint64_t)rows * (uint64_t)bpr;
+    const size_t smem = ctx->fl.total + 16;
+    const uint64_t tiles = (nblocks + kFastThreads - 1) / kFastThreads;
+    const unsigned g = (unsigned)std::min<uint64_t>(tiles, (uint64_t)ctx->sm_count);
+    const uint32_t* idx = static_cast<const uint32_t*>(d_idx);
+    __nv_bfloat16* w = reinterpret_cast<__nv_bfloat16*>(d_w_bf16);
     if (ctx->fast) {
-        const int64_t bpr = layout == LLVQ_LAYOUT_FLAT ? 0 : (cols + 23) / 24;
-        const uint64_t nblocks = layout == LLVQ_LAYOUT_FLAT ? ((uint64_t)rows * (uint64_t)cols + 23) / 24 : (uint64_t)rows * (uint64_t)bpr;
-        const size_t smem = ctx->fl.total + 16;
-        if (!set_smem(dequant_fast_kernel, smem)) return LLVQ_ECUDA;
-        uint64_t tiles = (nblocks + kFastThreads - 1) / kFastThreads;
-        unsigned g = (unsigned)std::min<uint64_t>(tiles, (uint64_t)ctx->sm_count);
-        dequant_fast_kernel<<<g, kFastThreads, smem, st>>>(fast_args(ctx), static_cast<const uint32_t*>(d_idx), d_gain_f16, nblocks,
-                                                           rows, cols, bpr, reinterpret_cast<__nv_bfloat16*>(d_w_bf16), ld);
-        return launch_status();
-    }
-    if (layout == LLVQ_LAYOUT_FLAT) {
-        uint64_t total = (uint64_t)rows * (uint64_t)cols, nblocks = (total + 23) / 24;
-        uint64_t grid = (nblocks + kThreads - 1) / kThreads;
-        if (grid > 0x7fffffffull) return LLVQ_EUNSUPPORTED;
-        dequant_flat_kernel<<<(unsigned)grid, kThreads, 0, st>>>(
-            ctx->dev, static_cast<const uint32_t*>(d_idx), d_gain_f16, nblocks, total,
-            reinterpret_cast<__nv_bfloat16*>(d_w_bf16), aligned(d_w_bf16, 16) ? 1 : 0);
+        if (!set_smem(dequant_fast_kernel<false>, smem)) return LLVQ_ECUDA;
+        dequant_fast_kernel<false><<<g, kFastThreads, smem, st>>>(fast_args(ctx), idx, d_gain_f16, nblocks, rows, cols, bpr, w, ld);
     } else {
-        int64_t bpr = (cols + 23) / 24;
-        uint64_t nblocks = (uint64_t)rows * (uint64_t)bpr;
-        uint64_t grid = (nblocks + kThreads - 1) / kThreads;
-        if (grid > 0x7fffffffull) return LLVQ_EUNSUPPORTED;
-        dequant_rowwise_kernel<<<(unsigned)grid, kThreads, 0, st>>>(
-            ctx->dev, static_cast<const uint32_t*>(d_idx), d_gain_f16, rows, cols, bpr,
-            reinterpret_cast<__nv_bfloat16*>(d_w_bf16), ld);
+        if (!set_smem(dequant_fast_kernel<true>, smem)) return LLVQ_ECUDA;
+        dequant_fast_kernel<true><<<g, kFastThreads, smem, st>>>(fast_args(ctx), idx, d_gain_f16, nblocks, rows, cols, bpr, w, ld);
     }
     return launch_status();
 }
@@ -852,42 +718,31 @@ int llvq_gemv(const llvq_ctx* ctx, const void* d_idx, const uint16_t* d_gain_f16
     if (k_in == 0) {
         return cudaMemsetAsync(d_y, 0, (size_t)n_out * (y_dtype == LLVQ_F32 ? 4 : 2), st) == cudaSuccess ? LLVQ_OK : LLVQ_ECUDA;
     }
-    int64_t bpr = (k_in + 23) / 24;
-    if (ctx->fast) {
-        const int64_t nq = (bpr + 3) / 4;
-        const size_t smem = ctx->fl.total + 16 + (size_t)nq * 48 * 4 + kGemvGroupsPerPass * kGemvGroupRows * 4 + 16;
-        if (smem > 227 * 1024 || n_out > 64ll * kMaxScratchRows) return LLVQ_EUNSUPPORTED;
-        const int64_t units = ((n_out + kGemvGroupRows - 1) / kGemvGroupRows) * nq;
-        unsigned g = (unsigned)std::min<int64_t>(units, ctx->sm_count);
-        // warps per CTA: the count in [20, 32] that wastes the fewest warp slots on the units of one CTA
-        const int64_t upc = (units + g - 1) / g;
-        int warps = 32; double best_eff = 0.0;
-        for (int w = 32; w >= 20; --w) {
-            const double eff = (double)upc / (double)(((upc + w - 1) / w) * w);
-            if (eff > best_eff + 1e-9) { best_eff = eff; warps = w; }
-        }
-        const unsigned threads = 32u * (unsigned)warps;
-        const uint32_t* idx = static_cast<const uint32_t*>(d_idx);
-        if (y_dtype == LLVQ_BF16) {
-            if (!set_smem(gemv_fast_kernel<true>, smem)) return LLVQ_ECUDA;
-            gemv_fast_kernel<true><<<g, threads, smem, st>>>(fast_args(ctx), idx, d_gain_f16, n_out, k_in, bpr, d_x_bf16, d_y, ctx->d_scratch, ctx->d_counters);
-        } else {
-            if (!set_smem(gemv_fast_kernel<false>, smem)) return LLVQ_ECUDA;
-            gemv_fast_kernel<false><<<g, threads, smem, st>>>(fast_args(ctx), idx, d_gain_f16, n_out, k_in, bpr, d_x_bf16, d_y, ctx->d_scratch, ctx->d_counters);
-        }
-        return launch_status();
+    const int64_t bpr = (k_in + 23) / 24;
+    const int64_t nq = (bpr + 3) / 4;
+    const size_t smem = ctx->fl.total + 16 + (size_t)nq * 48 * 4 + kGemvGroupsPerPass * kGemvGroupRows * 4 + 16;
+    if (smem > 227 * 1024 || n_out > 64ll * kMaxScratchRows) return LLVQ_EUNSUPPORTED;
+    const int64_t units = ((n_out + kGemvGroupRows - 1) / kGemvGroupRows) * nq;
+    const unsigned g = (unsigned)std::min<int64_t>(units, ctx->sm_count);
+    // warps per CTA: the count in [20, 32] that wastes the fewest warp slots on the units of one CTA
+    const int64_t upc = (units + g - 1) / g;
+    int warps = 32; double best_eff = 0.0;
+    for (int w = 32; w >= 20; --w) {
+        const double eff = (double)upc / (double)(((upc + w - 1) / w) * w);
+        if (eff > best_eff + 1e-9) { best_eff = eff; warps = w; }
     }
-    size_t smem = (size_t)bpr * 25 * sizeof(float);
-    if (smem > 200 * 1024 || n_out > (1ll << 31)) return LLVQ_EUNSUPPORTED;
-    unsigned grid = (unsigned)((n_out + kGemvWarps - 1) / kGemvWarps);
+    const unsigned threads = 32u * (unsigned)warps;
     const uint32_t* idx = static_cast<const uint32_t*>(d_idx);
-    if (y_dtype == LLVQ_BF16) {
-        if (cudaFuncSetAttribute(gemv_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return LLVQ_ECUDA;
-        gemv_kernel<true><<<grid, kGemvWarps * 32, smem, st>>>(ctx->dev, idx, d_gain_f16, n_out, k_in, bpr, d_x_bf16, d_y);
-    } else {
-        if (cudaFuncSetAttribute(gemv_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return LLVQ_ECUDA;
-        gemv_kernel<false><<<grid, kGemvWarps * 32, smem, st>>>(ctx->dev, idx, d_gain_f16, n_out, k_in, bpr, d_x_bf16, d_y);
-    }
+    const FastArgs fa = fast_args(ctx);
+#define LLVQ_LAUNCH_GEMV(BIG, BF16)                                                                           \
+    do {                                                                                                      \
+        if (!set_smem(gemv_fast_kernel<BIG, BF16>, smem)) return LLVQ_ECUDA;                                  \
+        gemv_fast_kernel<BIG, BF16><<<g, threads, smem, st>>>(fa, idx, d_gain_f16, n_out, k_in, bpr, d_x_bf16, d_y, \
+                                                              ctx->d_scratch, ctx->d_counters);               \
+    } while (0)
+    if (ctx->fast) { if (y_dtype == LLVQ_BF16) LLVQ_LAUNCH_GEMV(false, true); else LLVQ_LAUNCH_GEMV(false, false); }
+    else           { if (y_dtype == LLVQ_BF16) LLVQ_LAUNCH_GEMV(true, true);  else LLVQ_LAUNCH_GEMV(true, false); }
+#undef LLVQ_LAUNCH_GEMV
     return launch_status();
 }
 

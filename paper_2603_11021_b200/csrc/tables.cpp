@@ -210,10 +210,10 @@ bool build_tables(int m_lo, int m_hi, HostTables& t)
 
 namespace llvq {
 
-bool build_fast_image(const HostTables& t, FastLayout& L, std::vector<uint8_t>& img)
+bool build_fast_image(const HostTables& t, FastLayout& L, std::vector<uint8_t>& img, bool with_classes)
 {
-    const size_t ncls = t.desc.size();
-    if (t.W > 64 || t.W < 12 || ncls > 1024 || t.max_levels > kFastMaxLevels) return false;
+    const size_t ncls = with_classes ? t.desc.size() : 0;
+    if (with_classes && (t.W > 64 || t.W < 12 || ncls > 1024 || t.max_levels > kFastMaxLevels)) return false;
     auto up16 = [](size_t v) { return (uint32_t)((v + 15) & ~size_t(15)); };
     // r14: all k-subsets of 14 slots, grouped by k, each group in numeric order
     std::vector<uint16_t> r14;
@@ -225,15 +225,15 @@ bool build_fast_image(const HostTables& t, FastLayout& L, std::vector<uint8_t>& 
     }
     L.golay = 0;
     L.lut = up16(L.golay + 4096 * 4);
-    L.pascal = up16(L.lut + 4096 * 2);
+    L.pascal = up16(L.lut + (with_classes ? 4096 * 2 : 0));
     L.base14 = up16(L.pascal + 625 * 4);
     if (L.base14 - L.pascal != 2512) return false;                      // the kernels address base14 relative to pascal
     L.r14 = up16(L.base14 + 16 * 4);
     L.pd6 = up16(L.r14 + r14.size() * 2);
     L.off = up16(L.pd6 + 4096);
-    L.desc = up16(L.off + (ncls + 1) * 8);
+    L.desc = up16(L.off + (with_classes ? (ncls + 1) * 8 : 0));
     L.total = up16(L.desc + ncls * kFastDescStride * 4);
-    L.lut_shift = (uint32_t)(t.W - 12);
+    L.lut_shift = (uint32_t)(t.W >= 12 ? t.W - 12 : 0);
     L.ncls = (uint32_t)ncls;
     L.W = (uint32_t)t.W;
     img.assign(L.total, 0);
@@ -251,6 +251,7 @@ bool build_fast_image(const HostTables& t, FastLayout& L, std::vector<uint8_t>& 
                 if ((f >> b) & 1u) { if (src & 1u) out |= 1u << b; src >>= 1; }
             img[L.pd6 + (f << 6 | s)] = (uint8_t)out;
         }
+    if (!with_classes) return true;                        // small tables only: the class tables stay in global memory
     // class lookup by the top 12 bits of the index
     uint16_t* lut = reinterpret_cast<uint16_t*>(img.data() + L.lut);
     size_t c = 0;
@@ -291,6 +292,22 @@ bool build_fast_image(const HostTables& t, FastLayout& L, std::vector<uint8_t>& 
         w[15] = nbytes;
     }
     return true;
+}
+
+// Class of the first index of every bucket (I >> (W - 16)), plus a final entry = last class: the class of an
+// index lies between the entries of its bucket and of the next one.
+void build_bucket_table(const HostTables& t, std::vector<uint32_t>& lut)
+{
+    const size_t ncls = t.desc.size();
+    const int shift = t.W > 16 ? t.W - 16 : 0;
+    lut.assign(65537, (uint32_t)(ncls - 1));
+    size_t c = 0;
+    for (uint32_t b = 0; b < 65536; ++b) {
+        u128 first = (u128)b << shift;
+        if (first >= t.N) break;
+        while (c + 1 < ncls && t.offset[c + 1] <= first) ++c;
+        lut[b] = (uint32_t)c;
+    }
 }
 
 }  // namespace llvq

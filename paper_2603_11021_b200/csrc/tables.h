@@ -108,6 +108,9 @@ struct FastLayout {
 //  8..11: level l: radix | k << 22 | id << 27 | (value bit 1) << 30 | (value nonzero) << 31
 //  12..14: floor(2^32 / radix) of levels 1..3
 //  15: n (free slots before the step) of levels 0..3, one byte each
-bool build_fast_image(const HostTables& t, FastLayout& layout, std::vector<uint8_t>& image);
+// with_classes = false builds only the class-independent tables (Golay, Pascal, subsets, deposit): codes whose class
+// tables do not fit shared memory keep those in global memory.
+bool build_fast_image(const HostTables& t, FastLayout& layout, std::vector<uint8_t>& image, bool with_classes = true);
+void build_bucket_table(const HostTables& t, std::vector<uint32_t>& lut);   // u32[65537], see tables.cpp
 
 }  // namespace llvq
