@@ -77,19 +77,15 @@ __device__ __forceinline__ bool fast_load_image(uint8_t* dst, const uint8_t* __r
 // Deposit the low bits of src into the set bits of mask, lowest first (24-bit masks, 6 bits per lookup).
 __device__ __forceinline__ uint32_t deposit24(const uint8_t* pd6, uint32_t src, uint32_t mask)
 {
-    uint32_t out = 0;
-#pragma unroll
-    for (int g = 0; g < 4; ++g) {
-        const uint32_t f = (mask >> (6 * g)) & 63u;
-        out |= (uint32_t)pd6[(f << 6) | (src & 63u)] << (6 * g);
-        src >>= __popc(f);
-    }
-    return out;
+    // how many source bits the lower groups consume: known from the mask alone, so the four lookups are independent
+    const uint32_t c1 = __popc(mask & 0x3fu), c2 = __popc(mask & 0xfffu), c3 = __popc(mask & 0x3ffffu);
+    const uint32_t r0 = pd6[((mask & 0x3fu) << 6) | (src & 63u)];
+    const uint32_t r1 = pd6[(((mask >> 6) & 0x3fu) << 6) | ((src >> c1) & 63u)];
+    const uint32_t r2 = pd6[(((mask >> 12) & 0x3fu) << 6) | ((src >> c2) & 63u)];
+    const uint32_t r3 = pd6[(((mask >> 18) & 0x3fu) << 6) | ((src >> c3) & 63u)];
+    return r0 | r1 << 6 | r2 << 12 | r3 << 18;
 }
 
-// The rho-th k-subset of the slots {0..n-1} in combinatorial-number-system order (numeric
-// order of the bit masks).  Slots >= 14 are decided one at a time against C(slot, t); the
-// remaining t-subset of the low 14 slots is one table entry.  `top` (warp-uniform) bounds n.
 template <int kOff>
 __device__ __forceinline__ uint32_t lds_at(uint32_t addr)
 {

@@ -724,10 +724,10 @@ int llvq_gemv(const llvq_ctx* ctx, const void* d_idx, const uint16_t* d_gain_f16
     if (smem > 227 * 1024 || n_out > 64ll * kMaxScratchRows) return LLVQ_EUNSUPPORTED;
     const int64_t units = ((n_out + kGemvGroupRows - 1) / kGemvGroupRows) * nq;
     const unsigned g = (unsigned)std::min<int64_t>(units, ctx->sm_count);
-    // warps per CTA: the count in [20, 32] that wastes the fewest warp slots on the units of one CTA
+    // warps per CTA: the count in [28, 32] that wastes the fewest warp slots on the units of one CTA
     const int64_t upc = (units + g - 1) / g;
     int warps = 32; double best_eff = 0.0;
-    for (int w = 32; w >= 20; --w) {
+    for (int w = 32; w >= 28; --w) {
         const double eff = (double)upc / (double)(((upc + w - 1) / w) * w);
         if (eff > best_eff + 1e-9) { best_eff = eff; warps = w; }
     }
