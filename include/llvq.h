@@ -124,6 +124,24 @@ int llvq_gemv(const llvq_ctx* ctx, const void* d_idx, const uint16_t* d_gain_f16
               void* d_y, int y_dtype, void* stream);
 
 /*
+ * Kernel-private packed layout for the fused GEMV (preprocessing at load time; the paper describes no storage
+ * layout beyond "a compact integer index" per block, Sec. 1, and App. A step 5 notes that blocks are independent,
+ * which is what makes reordering them legitimate).  llvq_repack rewrites a ROWWISE index stream once: the class
+ * lookup of App. A steps 1-2 is done here, and inside tiles of 8 rows x 16 column blocks the blocks are grouped
+ * by the form of steps 3-4 their class needs (odd classes / even classes of Golay weight 8, 12, 16 / others), each
+ * block becoming a 64-bit entry (class-local index, class, position in the tile).  llvq_gemv_packed computes the
+ * same y = W x as llvq_gemv from the packed stream and the unchanged gain array.
+ * The packed stream takes llvq_packed_bytes() bytes (8 per block, tiles padded; 0 if the code is not
+ * supported: it must have at most 512 classes of at most 2^45 points, which holds for (2,2), (3,3), (2,13)).
+ * d_packed: device, 16-byte aligned.  Out-of-range fields are counted at repack time and decode to zero.
+ */
+size_t llvq_packed_bytes(const llvq_ctx* ctx, int64_t n_out, int64_t k_in);
+int llvq_repack(const llvq_ctx* ctx, const void* d_idx, int64_t n_out, int64_t k_in, void* d_packed, void* stream);
+int llvq_gemv_packed(const llvq_ctx* ctx, const void* d_packed, const uint16_t* d_gain_f16,
+                     int64_t n_out, int64_t k_in, const uint16_t* d_x_bf16,
+                     void* d_y, int y_dtype, void* stream);
+
+/*
  * The same product for a small batch, Y[b][i] = sum_k X[b][k] W[i][k]
  * (App. C's kernel generalised to batch <= 64): the dequantized bf16 tile is
  * fed to the tensor cores, accumulation in binary32.

@@ -136,28 +136,31 @@ __device__ __forceinline__ uint32_t fast_find_class(const FastSmem& T, uint64_t 
     return cls;
 }
 
-// S3-S6 for any class; `mask` = the lanes of the warp that call this together.
+// S3-S6.  `mask` = the lanes of the warp that call this together.  kPar = -1: any class.  kPar = 1: all calling lanes
+// hold odd classes.  kPar = 0: all calling lanes hold even classes of Golay weight 8, 12 or 16 (both slot groups have
+// at most 16 slots).  The specialised forms drop the work the other parity needs (slot decisions above 16, sign deposits).
+template <int kPar>
 __device__ __forceinline__ void fast_decode_local(const FastSmem& T, uint32_t cls, uint64_t local, bool valid, uint32_t mask, Decoded& d)
 {
     const uint4* D = reinterpret_cast<const uint4*>(T.desc + cls * kFastDescStride);
     const uint4 h = D[0], v = D[1], lw = D[2], mg = D[3];
     const uint32_t w = h.x & 0xff, B = (h.x >> 8) & 0xff, flags = (h.x >> 16) & 0xff;
-    const uint32_t nlev1 = (h.x >> 24) & 0xf, nlev = valid ? h.x >> 28 : 0u;
+    const uint32_t nlev1 = kPar == 1 ? 0u : (h.x >> 24) & 0xf, nlev = valid ? h.x >> 28 : 0u;
     const uint32_t goff = h.y & 0xffff, A = h.y >> 16;
-    const bool odd = flags & 1u;
+    const bool odd = kPar == 1 || (kPar == -1 && (flags & 1u));
 
     // S3: r fastest, then the sign word s, then the arrangement rank p
     uint64_t q;
     uint32_t r;
-    if (A == 4096u) { r = (uint32_t)local & 4095u; q = local >> 12; }
+    if (kPar == 1 || (kPar == -1 && A == 4096u)) { r = (uint32_t)local & 4095u; q = local >> 12; }
     else {
         q = __umul64hi(local, ((uint64_t)h.w << 32) | h.z);
         uint64_t rem = local - q * A;
         if (rem >= A) { rem -= A; ++q; }
         r = (uint32_t)rem;
     }
-    const uint32_t s = (uint32_t)q & ((1u << B) - 1u);
-    const uint64_t p = q >> B;
+    const uint32_t s = kPar == 1 ? 0u : (uint32_t)q & ((1u << B) - 1u);
+    const uint64_t p = kPar == 1 ? q : q >> B;
 
     // S4: Golay codeword
     const uint32_t c = T.golay[goff + r];
@@ -165,8 +168,8 @@ __device__ __forceinline__ void fast_decode_local(const FastSmem& T, uint32_t cl
     // S5: arrangement.  Group 1 lives on F1(c), group 0 on F0(c); an odd class is one group 0 on all positions.
     const uint32_t F1 = odd ? 0u : c;
     const uint32_t F0 = ~F1 & 0xffffffu;
-    uint32_t freem = F1;
-    bool in_group0 = false;
+    uint32_t freem = kPar == 1 ? 0xffffffu : F1;
+    bool in_group0 = kPar == 1;
     uint32_t p0 = 0, p1 = 0, p2 = 0, bit1 = 0, nz0 = 0;
     uint32_t p32 = 0;
     const uint32_t lwords[4] = {lw.x, lw.y, lw.z, lw.w};
@@ -175,9 +178,9 @@ __device__ __forceinline__ void fast_decode_local(const FastSmem& T, uint32_t cl
 #pragma unroll
     for (int l = 0; l < kFastMaxLevels; ++l) {
         if (l < maxlev) {
-            if (!in_group0 && (uint32_t)l >= nlev1) {           // group 1 done: its filler gets id 1
+            if (kPar != 1 && !in_group0 && (uint32_t)l >= nlev1) {     // group 1 done: its filler gets id 1
                 p0 |= freem;
-                if (flags & 8u) bit1 |= freem;
+                if (kPar == -1 && (flags & 8u)) bit1 |= freem;
                 freem = F0; in_group0 = true;
             }
             const bool active = (uint32_t)l < nlev;
@@ -197,32 +200,39 @@ __device__ __forceinline__ void fast_decode_local(const FastSmem& T, uint32_t cl
                 p32 = qq; rho = rem;
             }
             if (!active) rho = 0u;
-            const uint32_t n = active ? (mg.w >> (8 * l)) & 0xffu : 0u;
-            const int top = __reduce_max_sync(mask, n);
+            int top;
+            if (kPar == 0) top = 16;
+            else if (kPar == 1 && l == 0) top = 24;
+            else top = __reduce_max_sync(mask, active ? (mg.w >> (8 * l)) & 0xffu : 0u);
             const uint32_t rel = nth_subset(T, k, rho, top);
-            const uint32_t a = deposit24(T.pd6, rel, freem);
+            const uint32_t a = (kPar == 1 && l == 0) ? rel : deposit24(T.pd6, rel, freem);   // odd, first step: every position is free
             freem ^= a;
             if (word & (1u << 27)) p0 |= a;
             if (word & (1u << 28)) p1 |= a;
             if (word & (1u << 29)) p2 |= a;
-            if (word & (1u << 30)) bit1 |= a;
-            if (in_group0 && (word >> 31)) nz0 |= a;
+            if (kPar != 0 && (word & (1u << 30))) bit1 |= a;
+            if (kPar != 1 && in_group0 && (word >> 31)) nz0 |= a;
         }
     }
-    if (!in_group0) {
+    if (kPar != 1 && !in_group0) {
         p0 |= freem;
-        if (flags & 8u) bit1 |= freem;
+        if (kPar == -1 && (flags & 8u)) bit1 |= freem;
         freem = F0;
     }
-    if (flags & 16u) bit1 |= freem;                             // filler of group 0 keeps id 0
-    if (flags & 4u) nz0 |= freem;
+    if (kPar != 0 && (flags & 16u)) bit1 |= freem;              // filler of group 0 keeps id 0
+    if (kPar != 1 && (flags & 4u)) nz0 |= freem;
 
     // S6: signs
-    const uint32_t nf1 = w ? w - 1u : 0u;                       // free sign bits on F1
-    const uint32_t s1 = s & ((1u << nf1) - 1u);
-    const uint32_t src1 = s1 | (((__popc(s1) + (flags >> 1)) & 1u) << nf1);   // last F1 position: sum = 0 mod 8
-    const uint32_t neg_even = deposit24(T.pd6, src1, F1) | deposit24(T.pd6, s >> nf1, odd ? 0u : nz0);
-    uint32_t neg = odd ? (c ^ bit1) : neg_even;                 // odd: 1 mod 4 on F0, 3 mod 4 on F1
+    uint32_t neg;
+    if (kPar == 1) {
+        neg = c ^ bit1;                                         // 1 mod 4 on F0, 3 mod 4 on F1
+    } else {
+        const uint32_t nf1 = w ? w - 1u : 0u;                   // free sign bits on F1
+        const uint32_t s1 = s & ((1u << nf1) - 1u);
+        const uint32_t src1 = s1 | (((__popc(s1) + (flags >> 1)) & 1u) << nf1);   // last F1 position: sum = 0 mod 8
+        const uint32_t neg_even = deposit24(T.pd6, src1, F1) | deposit24(T.pd6, s >> nf1, odd ? 0u : nz0);
+        neg = odd ? (c ^ bit1) : neg_even;
+    }
     if (!valid) { p0 = p1 = p2 = 0; neg = 0; }
     d.p0 = p0; d.p1 = p1; d.p2 = p2; d.neg = neg;
     d.vals_lo = valid ? v.x : 0u; d.vals_hi = valid ? v.y : 0u;
@@ -232,7 +242,7 @@ __device__ __forceinline__ void fast_decode(const FastSmem& T, uint64_t I, bool 
 {
     uint64_t local = 0;
     const uint32_t cls = valid ? fast_find_class(T, I, local) : 0u;
-    fast_decode_local(T, cls, local, valid, kFullMask, d);
+    fast_decode_local<-1>(T, cls, local, valid, kFullMask, d);
 }
 
 // ---- expansion helpers -------------------------------------------------------

@@ -281,6 +281,192 @@ gemv_fast_kernel(FastArgs fa, const uint32_t* __restrict__ stream, const uint16_
 }
 
 // ===========================================================================
+// Kernel-private packed layout for the fused GEMV (llvq_repack / llvq_gemv_packed).
+// The matrix is cut into tiles of 8 rows x 16 column blocks (128 blocks).  Inside a tile the blocks are
+// reordered so that blocks whose classes need the same decoder form are adjacent: first the odd classes, then
+// the even classes of Golay weight 8/12/16, then all others, then padding.  Each block becomes one 64-bit
+// entry: class-local index (45 bits) | class (9 bits) << 45 | position in the tile (8 bits) << 54 | kind << 62.
+// The class lookup (S2) is done once, by llvq_repack; the GEMV then runs one decoder form per group of 32
+// entries (both forms only for the group that straddles a boundary) instead of the any-class form for all.
+// Gains stay in their ROWWISE array.  Tiles are stored row-tile major, 1024 bytes each.
+// ===========================================================================
+constexpr int kPackRows = 8, kPackCols = 16, kPackTile = kPackRows * kPackCols;
+constexpr uint32_t kKindEven = 0u, kKindOdd = 1u, kKindOther = 2u, kKindNull = 3u;
+
+__global__ void __launch_bounds__(256, 1)
+repack_kernel(FastArgs fa, const uint32_t* __restrict__ stream, int64_t n_out, int64_t bpr, int64_t col_tiles, int64_t ntiles,
+              unsigned long long* __restrict__ out)
+{
+    FAST_PROLOGUE();
+    const int lane = threadIdx.x & 31;
+    const int64_t warps = (int64_t)gridDim.x * (blockDim.x >> 5);
+    for (int64_t tile = (int64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5); tile < ntiles; tile += warps) {
+        const int64_t rt = tile / col_tiles, ct = tile - rt * col_tiles;
+        unsigned long long e[kPackTile / 32];
+        uint32_t count[4] = {0, 0, 0, 0};
+#pragma unroll
+        for (int j = 0; j < kPackTile / 32; ++j) {
+            const uint32_t pos = (uint32_t)(j * 32 + lane);
+            const int64_t row = rt * kPackRows + pos / kPackCols, cb = ct * kPackCols + pos % kPackCols;
+            const bool in = row < n_out && cb < bpr;
+            const uint64_t I = in ? load_field(stream, (uint64_t)(row * bpr + cb), (int)fa.L.W) : 0ull;
+            const bool valid = in && I < fa.n_points;
+            if (in && !valid) atomicAdd(fa.bad_index, 1ull);
+            uint32_t kind = kKindNull;
+            uint64_t local = 0; uint32_t cls = 0;
+            if (valid) {
+                cls = fast_find_class(T, I, local);
+                const uint32_t h = T.desc[cls * kFastDescStride];
+                const uint32_t w = h & 0xffu;
+                kind = (h & (1u << 16)) ? kKindOdd : ((w == 8u || w == 12u || w == 16u) ? kKindEven : kKindOther);
+            }
+            e[j] = local | (unsigned long long)cls << 45 | (unsigned long long)pos << 54 | (unsigned long long)kind << 62;
+#pragma unroll
+            for (uint32_t k = 0; k < 4; ++k) count[k] += __popc(__ballot_sync(kFullMask, kind == k));
+        }
+        // order of the groups in the tile: odd, even, other, null
+        const uint32_t first[4] = {count[kKindOdd], 0u, count[kKindOdd] + count[kKindEven], count[kKindOdd] + count[kKindEven] + count[kKindOther]};
+        uint32_t seen[4] = {0, 0, 0, 0};
+#pragma unroll
+        for (int j = 0; j < kPackTile / 32; ++j) {
+            const uint32_t kind = (uint32_t)(e[j] >> 62);
+            uint32_t slot = 0;
+#pragma unroll
+            for (uint32_t k = 0; k < 4; ++k) {
+                const uint32_t m = __ballot_sync(kFullMask, kind == k);
+                if (kind == k) slot = (k == kKindOdd ? 0u : first[k]) + seen[k] + __popc(m & ((1u << lane) - 1u));
+                seen[k] += __popc(m);
+            }
+            out[tile * kPackTile + slot] = e[j];
+        }
+    }
+}
+
+constexpr int kPackedThreads = 1024;
+constexpr int kPackedWarps = kPackedThreads / 32;
+constexpr int kPackedGroups = 128;         // row groups of 8 rows whose sums a CTA keeps in shared memory at a time
+
+template <bool kOutBf16>
+__global__ void __launch_bounds__(kPackedThreads, 1)
+gemv_packed_kernel(FastArgs fa, const unsigned long long* __restrict__ packed, const uint16_t* __restrict__ gain,
+                   int64_t n_out, int64_t k_in, int64_t bpr, int64_t col_tiles, const uint16_t* __restrict__ x, void* __restrict__ y,
+                   float* __restrict__ scratch, uint32_t* __restrict__ counters)
+{
+    FAST_PROLOGUE();
+    const int64_t nx = col_tiles * kPackCols * 12;                           // packed bf16 pairs of x, zero padded
+    uint32_t* xs = reinterpret_cast<uint32_t*>(staging);
+    float* acc = reinterpret_cast<float*>(xs + nx);                          // [kPackedGroups][16]
+    uint32_t* last_flag = reinterpret_cast<uint32_t*>(acc + kPackedGroups * kPackRows);
+    uint32_t* recs = last_flag + 4;                                          // [warps][256][6]: records of the warp's tile
+    for (int64_t i = threadIdx.x; i < nx; i += kPackedThreads) {
+        const int64_t e = 2 * i;
+        const uint32_t lo = e < k_in ? __ldg(x + e) : 0u, hi = e + 1 < k_in ? __ldg(x + e + 1) : 0u;
+        xs[i] = lo | hi << 16;
+    }
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, g = lane >> 2, t = lane & 3;
+    uint32_t* rec = recs + warp * (kPackTile * 6);
+    const int64_t groups = (n_out + kPackRows - 1) / kPackRows;
+    const int64_t U = groups * col_tiles, G = gridDim.x;                     // units = tiles, row-tile major
+    const int64_t u_begin = blockIdx.x * U / G, u_end = (blockIdx.x + 1) * U / G;
+    if (u_begin >= u_end) return;
+    const int64_t rg_first = u_begin / col_tiles, rg_last = (u_end - 1) / col_tiles;
+    for (int64_t rg0 = rg_first; rg0 <= rg_last; rg0 += kPackedGroups) {
+        const int64_t rg1 = min(rg0 + kPackedGroups - 1, rg_last);
+        for (int i = threadIdx.x; i < kPackedGroups * kPackRows; i += kPackedThreads) acc[i] = 0.f;
+        __syncthreads();
+        const int64_t p_begin = max(u_begin, rg0 * col_tiles), p_end = min(u_end, (rg1 + 1) * col_tiles);
+        for (int64_t u = p_begin + warp; u < p_end; u += kPackedWarps) {
+            const int64_t rg = u / col_tiles, ct = u - rg * col_tiles;
+            // ---- unrank the entries of the tile, 32 at a time, one decoder form per kind present
+#pragma unroll 1
+            for (int j = 0; j < kPackTile / 32; ++j) {
+                const unsigned long long e = __ldg(packed + u * kPackTile + j * 32 + lane);
+                const uint32_t kind = (uint32_t)(e >> 62), pos = (uint32_t)(e >> 54) & 0xffu, cls = (uint32_t)(e >> 45) & 0x1ffu;
+                const uint64_t local = e & ((1ull << 45) - 1);
+                Decoded d, r;
+                r.p0 = r.p1 = r.p2 = r.neg = r.vals_lo = r.vals_hi = 0u;
+                if (__any_sync(kFullMask, kind == kKindOdd)) {
+                    const bool mine = kind == kKindOdd;
+                    fast_decode_local<1>(T, mine ? cls : 0u, mine ? local : 0ull, mine, kFullMask, d);
+                    if (mine) r = d;
+                }
+                if (__any_sync(kFullMask, kind == kKindEven)) {
+                    const bool mine = kind == kKindEven;
+                    fast_decode_local<0>(T, mine ? cls : 0u, mine ? local : 0ull, mine, kFullMask, d);
+                    if (mine) r = d;
+                }
+                if (__any_sync(kFullMask, kind == kKindOther)) {
+                    const bool mine = kind == kKindOther;
+                    fast_decode_local<-1>(T, mine ? cls : 0u, mine ? local : 0ull, mine, kFullMask, d);
+                    if (mine) r = d;
+                }
+                uint2* o = reinterpret_cast<uint2*>(rec + pos * 6);
+                o[0] = make_uint2(r.p0, r.p1); o[1] = make_uint2(r.p2, r.neg); o[2] = make_uint2(r.vals_lo, r.vals_hi);
+            }
+            __syncwarp();
+            // ---- consume: 4 units of 8 rows x 4 column blocks (rows 8..15 of the MMA tile are zero)
+            float c[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll 1
+            for (int q4 = 0; q4 < kPackCols / 4; ++q4) {
+                const int cbl = q4 * 4 + t;
+                const int64_t cb = ct * kPackCols + cbl;
+                const int64_t row = rg * kPackRows + g;
+                const bool in = row < n_out && cb < bpr;
+                const float gn = in ? gain_to_float(__ldg(gain + row * bpr + cb)) : 0.f;
+                Decoded d;
+                const uint2* ia = reinterpret_cast<const uint2*>(rec + (g * kPackCols + cbl) * 6);
+                const uint2 a0 = ia[0], a1 = ia[1], a2 = ia[2];
+                d.p0 = a0.x; d.p1 = a0.y; d.p2 = a1.x; d.neg = a1.y; d.vals_lo = a2.x; d.vals_hi = a2.y;
+                uint32_t w[12];
+                expand_bf16(d, gn, w);
+                const uint4* xb = reinterpret_cast<const uint4*>(xs + cb * 12);
+                const uint4 x0 = xb[0], x1 = xb[1], x2 = xb[2];
+                const uint32_t xv[12] = {x0.x, x0.y, x0.z, x0.w, x1.x, x1.y, x1.z, x1.w, x2.x, x2.y, x2.z, x2.w};
+#pragma unroll
+                for (int q = 0; q < 6; ++q)
+                    mma_bf16_16816(c, w[2 * q], 0u, w[2 * q + 1], 0u, xv[2 * q], xv[2 * q + 1]);
+            }
+            if (t == 0) atomicAdd(&acc[(rg - rg0) * kPackRows + g], c[0]);
+            __syncwarp();
+        }
+        __syncthreads();
+        // row groups this CTA covers completely are final; the (at most two) split ones go through the scratch
+        for (int64_t rg = rg0; rg <= rg1; ++rg) {
+            const bool whole = u_begin <= rg * col_tiles && (rg + 1) * col_tiles <= u_end;
+            const int64_t row = rg * kPackRows + threadIdx.x;
+            const bool mine = threadIdx.x < kPackRows && row < n_out;
+            if (whole) {
+                if (mine) {
+                    const float v = acc[(rg - rg0) * kPackRows + threadIdx.x];
+                    if (kOutBf16) reinterpret_cast<__nv_bfloat16*>(y)[row] = __float2bfloat16_rn(v);
+                    else reinterpret_cast<float*>(y)[row] = v;
+                }
+                continue;
+            }
+            if (mine) atomicAdd(scratch + row, acc[(rg - rg0) * kPackRows + threadIdx.x]);
+            __threadfence();
+            __syncthreads();
+            if (threadIdx.x == 0) {
+                const uint32_t parts = (uint32_t)(unit_owner((rg + 1) * col_tiles - 1, U, G) - unit_owner(rg * col_tiles, U, G) + 1);
+                *last_flag = atomicAdd(counters + rg, 1u) == parts - 1u;
+            }
+            __syncthreads();
+            if (*last_flag) {
+                __threadfence();
+                if (mine) {
+                    const float v = __ldcg(scratch + row);
+                    if (kOutBf16) reinterpret_cast<__nv_bfloat16*>(y)[row] = __float2bfloat16_rn(v);
+                    else reinterpret_cast<float*>(y)[row] = v;
+                    __stcg(scratch + row, 0.f);
+                }
+                if (threadIdx.x == 0) counters[rg] = 0u;
+            }
+            __syncthreads();
+        }
+    }
+}
+
+// ===========================================================================
 // llvq_gemm_small_batch: Y[b][i] = sum_k X[b][k] W[i][k] on the tensor cores.
 // A work item is a tile of 128 output rows x a range of K stages (96 columns = 4 blocks of 24 per row).
 // Per stage every thread of a 512-thread group dequantizes one block into the group's shared-memory A tile
@@ -743,6 +929,72 @@ int llvq_gemv(const llvq_ctx* ctx, const void* d_idx, const uint16_t* d_gain_f16
     if (ctx->fast) { if (y_dtype == LLVQ_BF16) LLVQ_LAUNCH_GEMV(false, true); else LLVQ_LAUNCH_GEMV(false, false); }
     else           { if (y_dtype == LLVQ_BF16) LLVQ_LAUNCH_GEMV(true, true);  else LLVQ_LAUNCH_GEMV(true, false); }
 #undef LLVQ_LAUNCH_GEMV
+    return launch_status();
+}
+
+// Kernel-private packed layout (see the comment at repack_kernel).  Available for codes whose classes fit the
+// 64-bit entry: at most 512 classes of at most 2^45 points each.
+static bool packable(const llvq_ctx* ctx)
+{
+    if (!ctx->fast || ctx->host.desc.size() > 512) return false;
+    for (const ClassInfo& c : ctx->host.info) if (c.card >> 45) return false;
+    return true;
+}
+
+size_t llvq_packed_bytes(const llvq_ctx* ctx, int64_t n_out, int64_t k_in)
+{
+    if (!ctx || n_out <= 0 || k_in <= 0 || !packable(ctx)) return 0;
+    const int64_t bpr = (k_in + 23) / 24;
+    const int64_t tiles = ((n_out + kPackRows - 1) / kPackRows) * ((bpr + kPackCols - 1) / kPackCols);
+    return (size_t)tiles * kPackTile * 8;
+}
+
+int llvq_repack(const llvq_ctx* ctx, const void* d_idx, int64_t n_out, int64_t k_in, void* d_packed, void* stream)
+{
+    if (int e = check_common(ctx, d_idx)) return e;
+    if (!d_packed || n_out <= 0 || k_in <= 0) return LLVQ_EINVAL;
+    if (!aligned(d_packed, 16)) return LLVQ_EALIGN;
+    if (!packable(ctx)) return LLVQ_EUNSUPPORTED;
+    DeviceGuard guard(ctx->device);
+    if (!guard.ok) return LLVQ_ECUDA;
+    const int64_t bpr = (k_in + 23) / 24, col_tiles = (bpr + kPackCols - 1) / kPackCols;
+    const int64_t ntiles = ((n_out + kPackRows - 1) / kPackRows) * col_tiles;
+    const size_t smem = ctx->fl.total + 16;
+    if (!set_smem(repack_kernel, smem)) return LLVQ_ECUDA;
+    const unsigned g = (unsigned)std::min<int64_t>((ntiles + 7) / 8, ctx->sm_count);
+    repack_kernel<<<g, 256, smem, (cudaStream_t)stream>>>(fast_args(ctx), static_cast<const uint32_t*>(d_idx), n_out, bpr, col_tiles, ntiles,
+                                                         static_cast<unsigned long long*>(d_packed));
+    return launch_status();
+}
+
+int llvq_gemv_packed(const llvq_ctx* ctx, const void* d_packed, const uint16_t* d_gain_f16, int64_t n_out, int64_t k_in,
+                     const uint16_t* d_x_bf16, void* d_y, int y_dtype, void* stream)
+{
+    if (ctx && ctx->device >= 0 && n_out == 0) return LLVQ_OK;
+    if (int e = check_common(ctx, d_packed)) return e;
+    if (!d_gain_f16 || !d_x_bf16 || !d_y || n_out < 0 || k_in <= 0) return LLVQ_EINVAL;
+    if (y_dtype != LLVQ_F32 && y_dtype != LLVQ_BF16) return LLVQ_EINVAL;
+    if (!aligned(d_gain_f16, 2) || !aligned(d_x_bf16, 2) || !aligned(d_y, y_dtype == LLVQ_F32 ? 4 : 2)) return LLVQ_EALIGN;
+    if (!packable(ctx)) return LLVQ_EUNSUPPORTED;
+    DeviceGuard guard(ctx->device);
+    if (!guard.ok) return LLVQ_ECUDA;
+    cudaStream_t st = (cudaStream_t)stream;
+    const int64_t bpr = (k_in + 23) / 24, col_tiles = (bpr + kPackCols - 1) / kPackCols;
+    const int64_t groups = (n_out + kPackRows - 1) / kPackRows;
+    const size_t smem = ctx->fl.total + 16 + (size_t)col_tiles * kPackCols * 48 + kPackedGroups * kPackRows * 4 + 16 +
+                        (size_t)kPackedWarps * kPackTile * 24;
+    if (smem > 227 * 1024 || n_out > 64ll * kMaxScratchRows) return LLVQ_EUNSUPPORTED;
+    const unsigned g = (unsigned)std::min<int64_t>(groups * col_tiles, ctx->sm_count);
+    const unsigned long long* pk = static_cast<const unsigned long long*>(d_packed);
+    if (y_dtype == LLVQ_BF16) {
+        if (!set_smem(gemv_packed_kernel<true>, smem)) return LLVQ_ECUDA;
+        gemv_packed_kernel<true><<<g, kPackedThreads, smem, st>>>(fast_args(ctx), pk, d_gain_f16, n_out, k_in, bpr, col_tiles, d_x_bf16, d_y,
+                                                                   ctx->d_scratch, ctx->d_counters);
+    } else {
+        if (!set_smem(gemv_packed_kernel<false>, smem)) return LLVQ_ECUDA;
+        gemv_packed_kernel<false><<<g, kPackedThreads, smem, st>>>(fast_args(ctx), pk, d_gain_f16, n_out, k_in, bpr, col_tiles, d_x_bf16, d_y,
+                                                                    ctx->d_scratch, ctx->d_counters);
+    }
     return launch_status();
 }
 

@@ -360,3 +360,84 @@ def test_bounded_wait_reports_timeout_and_context_stays_usable(lib, ctxs, oracle
     o = _oracle(oracle_mod)((2, 2))
     lo = np.arange(100, dtype=np.uint64)
     assert np.array_equal(_decode_gpu(lib, ctx, lo, np.zeros_like(lo)), o.unrank_arrays(lo, np.zeros_like(lo)))
+
+
+# --------------------------------------------------------------------------
+# packed layout: repack once, then the fused GEMV on the packed stream
+# --------------------------------------------------------------------------
+@pytest.mark.parametrize("code,n_out,k_in", [((2, 13), 67, 4096), ((2, 13), 16, 384), ((2, 13), 129, 1000), ((2, 13), 1, 24),
+                                             ((2, 2), 256, 768), ((3, 3), 33, 4104)])
+def test_gemv_packed_small_shapes(lib, ctxs, oracle_mod, code, n_out, k_in):
+    o = _oracle(oracle_mod)(code)
+    ctx = ctxs[code]
+    stream, gain, _ = gen.make_layer(o.N, o.W, n_out, k_in, 1, seed=14)
+    x = gen.normal_bf16(k_in, seed=14)
+    want = o.gemv(stream, gain, n_out, k_in, x)
+    packed = lib.llvq_repack(ctx, to_dev_u8(stream), n_out, k_in)
+    assert packed.numel() == 1024 * ((n_out + 7) // 8) * (((k_in + 23) // 24 + 15) // 16)
+    y32 = lib.llvq_gemv_packed(ctx, packed, to_dev_f16(gain), n_out, k_in, to_dev_bf16(x))
+    y16 = lib.llvq_gemv_packed(ctx, packed, to_dev_f16(gain), n_out, k_in, to_dev_bf16(x), y_dtype=torch.bfloat16)
+    torch.cuda.synchronize()
+    assert gemv_error(y32.cpu().numpy(), want) <= TOL
+    assert gemv_error(y16.float().cpu().numpy(), want) <= TOL_BF16_OUT
+    assert lib.llvq_last_error(ctx) == (0, 0)
+
+
+def test_repack_is_a_permutation_of_the_blocks(lib, ctxs, oracle_mod):
+    # every block of the matrix appears exactly once with its own class-local index; padding entries are marked
+    o = _oracle(oracle_mod)((2, 13))
+    ctx = ctxs[(2, 13)]
+    n_out, k_in = 37, 1000                                  # 42 blocks per row: 5 x 3 tiles, ragged in both directions
+    bpr = 42
+    stream, _, nblocks = gen.make_layer(o.N, o.W, n_out, k_in, 1, seed=15)
+    packed = lib.llvq_repack(ctx, to_dev_u8(stream), n_out, k_in)
+    torch.cuda.synchronize()
+    e = packed.cpu().numpy().view(np.uint64).reshape(-1, 128)
+    assert e.shape[0] == 15
+    offsets = [k["offset"] for k in o.classes()]
+    parity = [k["parity"] for k in o.classes()]
+    idx = o.unpack(stream, nblocks)
+    seen = set()
+    for t in range(15):
+        rt, ct = divmod(t, 3)
+        kinds = (e[t] >> np.uint64(62)).astype(int)
+        order = [{1: 0, 0: 1, 2: 2, 3: 3}[k] for k in kinds]           # odd, even, other, padding
+        assert order == sorted(order)
+        for ent in e[t].tolist():
+            kind, pos, cls, local = ent >> 62, (ent >> 54) & 255, (ent >> 45) & 511, ent & ((1 << 45) - 1)
+            row, cb = rt * 8 + pos // 16, ct * 16 + pos % 16
+            if kind == 3:
+                assert row >= n_out or cb >= bpr
+                continue
+            b = row * bpr + cb
+            assert idx[b] == offsets[cls] + local and b not in seen
+            assert (kind == 1) == (parity[cls] == 1)
+            seen.add(b)
+    assert len(seen) == nblocks
+
+
+@pytest.mark.parametrize("n_out,k_in", [(4096, 4096), (11008, 4096), (4096, 11008)])
+def test_gemv_packed_full_size_layers_sampled_rows(lib, ctxs, oracle_mod, n_out, k_in):
+    o = _oracle(oracle_mod)((2, 13))
+    ctx = ctxs[(2, 13)]
+    stream, gain, _ = gen.make_layer(o.N, o.W, n_out, k_in, 1, seed=0)
+    x = gen.normal_bf16(k_in, seed=0)
+    packed = lib.llvq_repack(ctx, to_dev_u8(stream), n_out, k_in)
+    y = lib.llvq_gemv_packed(ctx, packed, to_dev_f16(gain), n_out, k_in, to_dev_bf16(x), y_dtype=torch.bfloat16)
+    y2 = lib.llvq_gemv(ctx, to_dev_u8(stream), to_dev_f16(gain), n_out, k_in, to_dev_bf16(x), y_dtype=torch.bfloat16)
+    torch.cuda.synchronize()
+    y = y.float().cpu().numpy()
+    rows = sorted(set([0, 1, 15, 16, n_out // 2, n_out - 17, n_out - 1] + list(range(5, n_out, n_out // 23))))
+    ref = np.array([o.gemv(stream, gain, n_out, k_in, x, rows=(r, 1))[r] for r in rows])
+    scale = float(np.abs(ref).max())
+    assert (np.abs(y[rows] - ref) / np.maximum(np.abs(ref), 1e-3 * scale)).max() <= TOL_BF16_OUT
+    # and all rows against the unpacked kernel (same weights, different summation order)
+    assert gemv_error(y, y2.float().cpu().numpy().astype(np.float64)) <= 2.0 ** -7
+    assert lib.llvq_last_error(ctx) == (0, 0)
+
+
+def test_packed_layout_unsupported_for_the_72_bit_code(lib, ctxs):
+    ctx = ctxs[(2, 53)]
+    assert ctx._lib.llvq_packed_bytes(ctx._h, 64, 96) == 0
+    buf = torch.zeros(4096, dtype=torch.uint8, device="cuda")
+    assert ctx._lib.llvq_repack(ctx._h, buf.data_ptr(), 16, 96, buf.data_ptr(), None) == 3
