@@ -343,7 +343,7 @@ repack_kernel(FastArgs fa, const uint32_t* __restrict__ stream, int64_t n_out, i
 }
 
 constexpr int kPackedThreads = 1024;
-constexpr int kPackedWarps = kPackedThreads / 32;
+constexpr int kPackedWarps = kPackedThreads / 32;   // upper bound; the launch picks the count that divides the tiles per CTA best
 constexpr int kPackedGroups = 128;         // row groups of 8 rows whose sums a CTA keeps in shared memory at a time
 
 template <bool kOutBf16>
@@ -358,7 +358,7 @@ gemv_packed_kernel(FastArgs fa, const unsigned long long* __restrict__ packed, c
     float* acc = reinterpret_cast<float*>(xs + nx);                          // [kPackedGroups][16]
     uint32_t* last_flag = reinterpret_cast<uint32_t*>(acc + kPackedGroups * kPackRows);
     uint32_t* recs = last_flag + 4;                                          // [warps][256][6]: records of the warp's tile
-    for (int64_t i = threadIdx.x; i < nx; i += kPackedThreads) {
+    for (int64_t i = threadIdx.x; i < nx; i += blockDim.x) {
         const int64_t e = 2 * i;
         const uint32_t lo = e < k_in ? __ldg(x + e) : 0u, hi = e + 1 < k_in ? __ldg(x + e + 1) : 0u;
         xs[i] = lo | hi << 16;
@@ -372,10 +372,10 @@ gemv_packed_kernel(FastArgs fa, const unsigned long long* __restrict__ packed, c
     const int64_t rg_first = u_begin / col_tiles, rg_last = (u_end - 1) / col_tiles;
     for (int64_t rg0 = rg_first; rg0 <= rg_last; rg0 += kPackedGroups) {
         const int64_t rg1 = min(rg0 + kPackedGroups - 1, rg_last);
-        for (int i = threadIdx.x; i < kPackedGroups * kPackRows; i += kPackedThreads) acc[i] = 0.f;
+        for (int i = threadIdx.x; i < kPackedGroups * kPackRows; i += (int)blockDim.x) acc[i] = 0.f;
         __syncthreads();
         const int64_t p_begin = max(u_begin, rg0 * col_tiles), p_end = min(u_end, (rg1 + 1) * col_tiles);
-        for (int64_t u = p_begin + warp; u < p_end; u += kPackedWarps) {
+        for (int64_t u = p_begin + warp; u < p_end; u += (int64_t)(blockDim.x >> 5)) {
             const int64_t rg = u / col_tiles, ct = u - rg * col_tiles;
             // ---- unrank the entries of the tile, 32 at a time, one decoder form per kind present
 #pragma unroll 1
@@ -985,14 +985,22 @@ int llvq_gemv_packed(const llvq_ctx* ctx, const void* d_packed, const uint16_t* 
                         (size_t)kPackedWarps * kPackTile * 24;
     if (smem > 227 * 1024 || n_out > 64ll * kMaxScratchRows) return LLVQ_EUNSUPPORTED;
     const unsigned g = (unsigned)std::min<int64_t>(groups * col_tiles, ctx->sm_count);
+    // warps per CTA: the count in [22, 32] that wastes the fewest warp slots on the tiles of one CTA
+    const int64_t upc = (groups * col_tiles + g - 1) / g;
+    int warps = kPackedWarps; double best_eff = 0.0;
+    for (int w = kPackedWarps; w >= 22; --w) {
+        const double eff = (double)upc / (double)(((upc + w - 1) / w) * w);
+        if (eff > best_eff + 1e-9) { best_eff = eff; warps = w; }
+    }
+    const unsigned threads = 32u * (unsigned)warps;
     const unsigned long long* pk = static_cast<const unsigned long long*>(d_packed);
     if (y_dtype == LLVQ_BF16) {
         if (!set_smem(gemv_packed_kernel<true>, smem)) return LLVQ_ECUDA;
-        gemv_packed_kernel<true><<<g, kPackedThreads, smem, st>>>(fast_args(ctx), pk, d_gain_f16, n_out, k_in, bpr, col_tiles, d_x_bf16, d_y,
+        gemv_packed_kernel<true><<<g, threads, smem, st>>>(fast_args(ctx), pk, d_gain_f16, n_out, k_in, bpr, col_tiles, d_x_bf16, d_y,
                                                                    ctx->d_scratch, ctx->d_counters);
     } else {
         if (!set_smem(gemv_packed_kernel<false>, smem)) return LLVQ_ECUDA;
-        gemv_packed_kernel<false><<<g, kPackedThreads, smem, st>>>(fast_args(ctx), pk, d_gain_f16, n_out, k_in, bpr, col_tiles, d_x_bf16, d_y,
+        gemv_packed_kernel<false><<<g, threads, smem, st>>>(fast_args(ctx), pk, d_gain_f16, n_out, k_in, bpr, col_tiles, d_x_bf16, d_y,
                                                                     ctx->d_scratch, ctx->d_counters);
     }
     return launch_status();
