@@ -249,9 +249,11 @@ __device__ __forceinline__ void fast_decode(const FastSmem& T, uint64_t I, bool 
 // 8 mask bits -> 8 nibbles (bit i -> bit 4i).
 __device__ __forceinline__ uint32_t nibspread8(uint32_t b)
 {
-    uint32_t x = (b | (b << 12)) & 0x000f000fu;
-    x = (x | (x << 6)) & 0x03030303u;
-    x = (x | (x << 3)) & 0x11111111u;
+    // each "x | x << s" is written as a multiplication (the two copies never overlap): it runs on the FMA pipe,
+    // the integer ALU pipe is the busy one
+    uint32_t x = (b * 0x1001u) & 0x000f000fu;
+    x = (x * 65u) & 0x03030303u;
+    x = (x * 9u) & 0x11111111u;
     return x;
 }
 
