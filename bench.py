@@ -40,8 +40,8 @@ UNIT = "GB/s"
 WORKLOAD = "configs[2]: fused dequant+GEMV batch 1 on W 4096x4096, 11008x4096, 4096x11008, 48-bit indices (shells 2..13), fp16 gain per 24 weights"
 
 # dram__bytes_read.sum + dram__bytes_write.sum of one gemv_fast_kernel launch on the 11008x4096 layer, from the
-# ncu capture summarised in profiles/gemv_fast_kernel_7B_layers.md (algorithmic bytes: 15 089 152)
-NCU_TRAFFIC_BYTES_11008x4096 = 15237888
+# ncu capture summarised under profiles/ (algorithmic bytes: 15 089 152)
+NCU_TRAFFIC_BYTES_11008x4096 = 15228160
 
 
 def layer_bytes(n_out: int, k_in: int) -> dict:
