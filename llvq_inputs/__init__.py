@@ -127,3 +127,27 @@ def make_layer(N: int, W: int, rows: int, cols: int, layout: int, seed: int = 0)
     nblocks = (rows * cols + 23) // 24 if layout == 0 else rows * ((cols + 23) // 24)
     lo, hi = random_indices(N, W, nblocks, seed)
     return pack_indices(lo, hi, W), gains_f16(nblocks, seed), nblocks
+
+
+def gain_indices(nblocks: int, gain_bits: int, seed: int = 0) -> np.ndarray:
+    """Uniform gain-codebook indices in [0, 2**gain_bits), one per block (uint64)."""
+    if gain_bits == 0:
+        return np.zeros(nblocks, dtype=np.uint64)
+    blocks = np.arange(nblocks, dtype=np.uint64)
+    return _draw(seed ^ 0x6A09E667, blocks, 0, 7) >> np.uint64(64 - gain_bits)
+
+
+def row_scales_f32(rows: int, seed: int = 0, scale: float = 0.02) -> np.ndarray:
+    """One positive binary32 scale per output row: scale * (1 + 0.1 z), z ~ N(0,1) clipped to +-3."""
+    rng = np.random.default_rng(seed + 0x5CA1E)
+    z = np.clip(rng.standard_normal(rows), -3.0, 3.0)
+    return (scale * (1.0 + 0.1 * z)).astype(np.float32)
+
+
+def make_layer_sg(N: int, W: int, gain_bits: int, rows: int, cols: int, seed: int = 0):
+    """(stream, nblocks) of a ROWWISE layer whose fields are W + gain_bits wide: shape index | gain index << W."""
+    assert W + gain_bits <= 64
+    nblocks = rows * ((cols + 23) // 24)
+    lo, hi = random_indices(N, W, nblocks, seed)
+    lo = lo | (gain_indices(nblocks, gain_bits, seed) << np.uint64(W)) if gain_bits else lo
+    return pack_indices(lo, hi, W + gain_bits), nblocks

@@ -60,6 +60,10 @@ def _load():
             lib.oc_dequant_matrix.argtypes = [vp, vp, vp, i64, i64, ctypes.c_int, vp]
             lib.oc_gemm_rows.restype = i64
             lib.oc_gemm_rows.argtypes = [vp, vp, vp, i64, i64, vp, ctypes.c_int, i64, i64, vp]
+            lib.oc_dequant_matrix_sg.restype = i64
+            lib.oc_dequant_matrix_sg.argtypes = [vp, vp, ctypes.c_int, vp, vp, i64, i64, vp]
+            lib.oc_gemm_rows_sg.restype = i64
+            lib.oc_gemm_rows_sg.argtypes = [vp, vp, ctypes.c_int, vp, vp, i64, i64, vp, ctypes.c_int, i64, i64, vp]
             lib.oc_nearest_angular.argtypes = [vp, vp, vp]
             lib.oc_is_member.argtypes = [vp]
             lib.oc_shell_size.argtypes = [ctypes.c_int, u64p]
@@ -233,6 +237,45 @@ class Code:
 
     def gemv(self, stream, gain_f16, n_out: int, k_in: int, x_bf16, **kw) -> np.ndarray:
         return self.gemm(stream, gain_f16, n_out, k_in, np.asarray(x_bf16).reshape(-1), **kw)
+
+    # -- shape-gain with a gain codebook and an optional scale per row ------
+    def dequant_matrix_sg(self, stream, gain_bits: int, codebook, row_scale, rows: int, cols: int) -> np.ndarray:
+        """bf16 bit patterns of gain * x / |x| (ROWWISE fields of W + gain_bits bits); row_scale may be None."""
+        stream = np.ascontiguousarray(stream, dtype=np.uint8)
+        cb = np.ascontiguousarray(codebook, dtype=np.float32)
+        assert cb.size == 1 << gain_bits
+        rs = None if row_scale is None else np.ascontiguousarray(row_scale, dtype=np.float32)
+        out = np.zeros((rows, cols), dtype=np.uint16)
+        self._lib.oc_dequant_matrix_sg(self._h, _ptr(stream), gain_bits, _ptr(cb), None if rs is None else _ptr(rs),
+                                       rows, cols, _ptr(out))
+        return out
+
+    def gemm_sg(self, stream, gain_bits: int, codebook, row_scale, n_out: int, k_in: int, x_bf16, rows=None,
+                threads: int = 1) -> np.ndarray:
+        stream = np.ascontiguousarray(stream, dtype=np.uint8)
+        cb = np.ascontiguousarray(codebook, dtype=np.float32)
+        assert cb.size == 1 << gain_bits
+        rs = None if row_scale is None else np.ascontiguousarray(row_scale, dtype=np.float32)
+        x = np.ascontiguousarray(x_bf16, dtype=np.uint16)
+        vec = x.ndim == 1
+        x2 = x.reshape(1, -1) if vec else x
+        batch = x2.shape[0]
+        assert x2.shape[1] == k_in
+        y = np.zeros((batch, n_out), dtype=np.float64)
+        first, count = rows if rows is not None else (0, n_out)
+
+        def run(job):
+            self._lib.oc_gemm_rows_sg(self._h, _ptr(stream), gain_bits, _ptr(cb), None if rs is None else _ptr(rs),
+                                      n_out, k_in, _ptr(x2), batch, job[0], job[1], _ptr(y))
+
+        if threads <= 1:
+            run((first, count))
+        else:
+            step = -(-count // threads)
+            jobs = [(first + s, min(step, count - s)) for s in range(0, count, step)]
+            with ThreadPoolExecutor(threads) as ex:
+                list(ex.map(run, jobs))
+        return y[0] if vec else y
 
     def nearest_angular(self, x) -> int:
         v = np.ascontiguousarray(np.asarray(x, dtype=np.float64))

@@ -741,6 +741,84 @@ int64_t oc_gemm_rows(const oc_code* code, const uint8_t* stream, const uint16_t*
 }
 
 /* ------------------------------------------------------------------------- */
+/* Shape-gain with a projected spherical code and a scalar gain code (App. E   */
+/* "Shape-gain"; App. "spherical shaping or shape-gain": C_shape = {x/|x|},    */
+/* C_gain a small codebook, reconstruction = gain * shape), optionally times a */
+/* high-precision scale per output row ("0 bit gain": the scale alone).       */
+/* Stored field of W + gain_bits bits: shape index I in the low W bits, gain   */
+/* index k above it (the paper only says the pair is one integer; this is the */
+/* convention).  Arithmetic, all in binary32, each operation rounded once:    */
+/*   rn = (float)(1 / sqrt(sum x_i^2))      (formed in binary64, then rounded) */
+/*   g  = (row_scale * codebook[k]) * rn                                        */
+/*   w_j = bf16_rne(g * (float)x_j)                                            */
+/* row_scale == NULL means 1.  An index I >= N decodes to zeros (rn = 0).     */
+/* ------------------------------------------------------------------------- */
+static u128 stream_field(const uint8_t* stream, int width, int64_t b) { return stream_index(stream, width, b); }
+
+static float sg_block_gain(const int8_t x[OC_DIM], float row_scale, float cb)
+{
+    long norm = 0;
+    for (int i = 0; i < OC_DIM; ++i) norm += (long)x[i] * x[i];
+    volatile float rn = norm ? (float)(1.0 / sqrt((double)norm)) : 0.0f;
+    volatile float sc = row_scale * cb;
+    volatile float g = sc * rn;
+    return g;
+}
+
+static uint16_t sg_weight(float g, int x)
+{
+    volatile float prod = g * (float)x;
+    return float_to_bf16_rne(prod);
+}
+
+/* ROWWISE blocks only (a row scale has no meaning for a block that spans rows). */
+int64_t oc_dequant_matrix_sg(const oc_code* code, const uint8_t* stream, int gain_bits, const float* codebook,
+                             const float* row_scale, int64_t rows, int64_t cols, uint16_t* out)
+{
+    int64_t bad = 0, bpr = (cols + OC_DIM - 1) / OC_DIM;
+    int8_t x[OC_DIM];
+    for (int64_t r = 0; r < rows; ++r)
+        for (int64_t cb = 0; cb < bpr; ++cb) {
+            u128 field = stream_field(stream, code->W + gain_bits, r * bpr + cb);
+            u128 I = field & (((u128)1 << code->W) - 1);
+            int k = (int)(field >> code->W);
+            bad += unrank_point(code, I, x);
+            float g = sg_block_gain(x, row_scale ? row_scale[r] : 1.0f, codebook[k]);
+            for (int j = 0; j < OC_DIM; ++j) {
+                int64_t col = cb * OC_DIM + j;
+                if (col < cols) out[r * cols + col] = sg_weight(g, x[j]);
+            }
+        }
+    return bad;
+}
+
+int64_t oc_gemm_rows_sg(const oc_code* code, const uint8_t* stream, int gain_bits, const float* codebook,
+                        const float* row_scale, int64_t n_out, int64_t k_in, const uint16_t* x_bf16, int batch,
+                        int64_t row_first, int64_t row_count, double* y)
+{
+    int64_t bad = 0, bpr = (k_in + OC_DIM - 1) / OC_DIM;
+    int8_t pt[OC_DIM];
+    for (int64_t r = row_first; r < row_first + row_count && r < n_out; ++r) {
+        for (int bb = 0; bb < batch; ++bb) y[(int64_t)bb * n_out + r] = 0.0;
+        for (int64_t cb = 0; cb < bpr; ++cb) {
+            u128 field = stream_field(stream, code->W + gain_bits, r * bpr + cb);
+            u128 I = field & (((u128)1 << code->W) - 1);
+            int k = (int)(field >> code->W);
+            bad += unrank_point(code, I, pt);
+            float g = sg_block_gain(pt, row_scale ? row_scale[r] : 1.0f, codebook[k]);
+            for (int j = 0; j < OC_DIM; ++j) {
+                int64_t col = cb * OC_DIM + j;
+                if (col >= k_in) break;
+                double w = bf16_bits_to_double(sg_weight(g, pt[j]));
+                for (int bb = 0; bb < batch; ++bb)
+                    y[(int64_t)bb * n_out + r] += w * bf16_bits_to_double(x_bf16[(int64_t)bb * k_in + col]);
+            }
+        }
+    }
+    return bad;
+}
+
+/* ------------------------------------------------------------------------- */
 /* Angular nearest point (Sec. 3.1): argmax over all points v of the code of   */
 /* <x, v> / |v|, by brute force.  Lowest index wins ties.  Tiny codes only.   */
 /* ------------------------------------------------------------------------- */
