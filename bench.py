@@ -306,7 +306,7 @@ def extras(P, ctx) -> dict:
                 P.llvq_gemv(ctx, d_idx, d_gain, n, k, xs[k], d_y=ys[n])
     token(0)
     torch.cuda.synchronize()
-    us = _event_us(torch, token, 3)
+    sweep_us = _event_us(torch, token, 3)
     blocks = 32 * sum(n * ((k + 23) // 24) for n, k in shapes)
     by = blocks * (CODE_W // 8 + 2) + 32 * sum(2 * k + 2 * n for n, k in shapes)
     # --- the headline layers through the kernel-private packed layout (repacked once, outside the timed loop)
@@ -343,7 +343,27 @@ def extras(P, ctx) -> dict:
     out["paper_shape_shell3_4096x4104_gemv"] = {"us": us3, "GBps": by3 / us3 / 1e3, "weights_per_s": n * k / (us3 * 1e-6),
                                                 "paper_us_fp16_unnamed_gpu": 11.94, "algorithmic_bytes": by3}
     del bufs3
-    out["llama3_8b_linear_sweep"] = {"us_per_token": us, "tokens_per_s": 1e6 / us, "GBps": by / us / 1e3, "blocks_per_token": blocks,
+    # --- shape-gain form at the same 48 bits per block: shells 2..12 (47-bit shape index) + 1 gain bit, row scales
+    ctx12 = P.Context(2, 12, device=torch.cuda.current_device())
+    from_codebook = np.array([4.3157, 5.4413], dtype=np.float32)       # Lloyd-Max levels of chi(24) at one bit
+    d_cb = dev(from_codebook)
+    n, k = 11008, 4096
+    bufs12 = []
+    for c in range(20):                                   # 20 x 15.1 MB > 2 x L2
+        stream, nb12 = gen.make_layer_sg(ctx12.num_points, ctx12.index_bits, 1, n, k, seed=600 + c)
+        bufs12.append(dev(stream))
+    d_rs = dev(gen.row_scales_f32(n, seed=6))
+    x12 = dev(gen.normal_bf16(k, seed=12), np.int16).view(torch.bfloat16)
+    y12 = torch.empty(n, dtype=torch.bfloat16, device="cuda")
+    fn = lambda i: P.llvq_gemv_sg(ctx12, bufs12[i % 20], 1, d_cb, d_rs, n, k, x12, d_y=y12)
+    _event_us(torch, fn, 8)
+    us12 = _event_us(torch, fn, 60)
+    by12 = nb12 * 6 + 4 * n + 2 * k + 2 * n
+    out["gemv_shape_gain_47p1_11008x4096"] = {"us": us12, "GBps": by12 / us12 / 1e3, "algorithmic_bytes": by12,
+                                              "bits_per_weight": 48 * nb12 / (n * k)}
+    assert P.llvq_last_error(ctx12) == (0, 0)
+    del bufs12, ctx12
+    out["llama3_8b_linear_sweep"] = {"us_per_token": sweep_us, "tokens_per_s": 1e6 / sweep_us, "GBps": by / sweep_us / 1e3, "blocks_per_token": blocks,
                                      "launches_per_token": 32 * len(shapes), "algorithmic_bytes": by}
     return out
 

@@ -124,6 +124,35 @@ int llvq_gemv(const llvq_ctx* ctx, const void* d_idx, const uint16_t* d_gain_f16
               void* d_y, int y_dtype, void* stream);
 
 /*
+ * Shape-gain with a projected spherical shape code and a scalar gain codebook (App. E "Shape-gain"; the
+ * appendix comparing spherical shaping with shape-gain: C_shape = { x / |x| }, C_gain a small chi(24)-matched
+ * codebook, reconstruction = gain * shape), optionally times a high-precision scale per output row (the
+ * "0 bit gain" setting: gain_bits = 0, a one-entry codebook and the row scale alone).
+ *
+ * Stored format: ROWWISE fields of llvq_index_bits(ctx) + gain_bits bits (at most 64 in all), packed like the
+ * index stream: the shape index I in the low bits, the gain index k in the gain_bits bits above it.
+ * llvq_field_bytes gives the stream length (rounded up to 16 bytes; 0 on bad arguments).
+ *
+ * Arithmetic, every operation in binary32 and rounded once:
+ *     rn  = float( 1 / sqrt(16 m) )           m = shell of the point, |x|^2 = 16 m; formed in binary64
+ *     g   = (row_scale[r] * codebook[k]) * rn  row_scale == NULL means 1
+ *     w_j = bf16_rn( g * float(x_j) )
+ * A field with I >= N decodes to zeros and is counted (see llvq_last_error).
+ *
+ * d_fields: device, 16-byte aligned.  d_codebook_f32: device, [1 << gain_bits] floats, 0 <= gain_bits <= 8.
+ * d_row_scale_f32: device, [rows] ([n_out]) floats, or NULL.  Other arguments as in llvq_dequant_matrix (layout
+ * is always ROWWISE) and llvq_gemv.  Codes whose class tables do not fit shared memory ((2,53)) return
+ * LLVQ_EUNSUPPORTED.
+ */
+size_t llvq_field_bytes(const llvq_ctx* ctx, uint64_t nblocks, int gain_bits);
+int llvq_dequant_matrix_sg(const llvq_ctx* ctx, const void* d_fields, int gain_bits, const float* d_codebook_f32,
+                           const float* d_row_scale_f32, int64_t rows, int64_t cols,
+                           uint16_t* d_w_bf16, int64_t ld, void* stream);
+int llvq_gemv_sg(const llvq_ctx* ctx, const void* d_fields, int gain_bits, const float* d_codebook_f32,
+                 const float* d_row_scale_f32, int64_t n_out, int64_t k_in, const uint16_t* d_x_bf16,
+                 void* d_y, int y_dtype, void* stream);
+
+/*
  * Kernel-private packed layout for the fused GEMV (preprocessing at load time; the paper describes no storage
  * layout beyond "a compact integer index" per block, Sec. 1, and App. A step 5 notes that blocks are independent,
  * which is what makes reordering them legitimate).  llvq_repack rewrites a ROWWISE index stream once: the class

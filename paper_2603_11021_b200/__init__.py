@@ -16,6 +16,7 @@ from .build import LIB
 
 __all__ = [
     "Context", "llvq_decode_blocks", "llvq_dequant_matrix", "llvq_gemv", "llvq_gemm_small_batch", "llvq_gemm_small_batch_noalloc",
+    "llvq_dequant_matrix_sg", "llvq_gemv_sg", "llvq_repack", "llvq_gemv_packed",
     "llvq_last_error", "LlvqError", "EXPORTS", "load_library",
     "LLVQ_LAYOUT_FLAT", "LLVQ_LAYOUT_ROWWISE", "LLVQ_F32", "LLVQ_BF16",
 ]
@@ -30,6 +31,7 @@ EXPORTS = [
     "llvq_create", "llvq_destroy", "llvq_index_bits", "llvq_num_points", "llvq_num_classes", "llvq_index_bytes",
     "llvq_decode_blocks", "llvq_dequant_matrix", "llvq_gemv", "llvq_gemm_small_batch", "llvq_gemm_small_batch_noalloc",
     "llvq_packed_bytes", "llvq_repack", "llvq_gemv_packed", "llvq_selftest_wait_timeout", "llvq_last_error",
+    "llvq_field_bytes", "llvq_dequant_matrix_sg", "llvq_gemv_sg", "llvq_class_info", "llvq_golay_table",
 ]
 
 
@@ -69,6 +71,10 @@ def load_library() -> ctypes.CDLL:
     lib.llvq_packed_bytes.restype = ctypes.c_size_t
     lib.llvq_repack.argtypes = [vp, vp, i64, i64, vp, vp]
     lib.llvq_gemv_packed.argtypes = [vp, vp, vp, i64, i64, vp, vp, ctypes.c_int, vp]
+    lib.llvq_field_bytes.argtypes = [vp, u64, ctypes.c_int]
+    lib.llvq_field_bytes.restype = ctypes.c_size_t
+    lib.llvq_dequant_matrix_sg.argtypes = [vp, vp, ctypes.c_int, vp, vp, i64, i64, vp, i64, vp]
+    lib.llvq_gemv_sg.argtypes = [vp, vp, ctypes.c_int, vp, vp, i64, i64, vp, vp, ctypes.c_int, vp]
     lib.llvq_last_error.argtypes = [vp, vp, ctypes.POINTER(u64), ctypes.POINTER(ctypes.c_uint32)]
     lib.llvq_class_info.argtypes = [vp, ctypes.c_int, vp, vp, vp, vp, vp, vp]
     lib.llvq_golay_table.argtypes = [vp, vp]
@@ -183,6 +189,44 @@ def llvq_gemv(ctx: Context, d_idx: torch.Tensor, d_gain: torch.Tensor, n_out: in
     code = LLVQ_F32 if d_y.dtype == torch.float32 else LLVQ_BF16
     _check("llvq_gemv", ctx._lib.llvq_gemv(ctx._h, _dev(d_idx, "d_idx"), _dev(d_gain, "d_gain"), n_out, k_in,
                                            _dev(d_x, "d_x"), _dev(d_y, "d_y"), code, _stream_ptr(stream)))
+    return d_y
+
+
+def _sg_args(ctx: Context, d_fields, gain_bits: int, d_codebook, d_row_scale, rows: int, nblocks: int):
+    assert d_codebook.dtype == torch.float32 and d_codebook.numel() >= (1 << gain_bits)
+    assert d_row_scale is None or (d_row_scale.dtype == torch.float32 and d_row_scale.numel() >= rows)
+    assert d_fields.numel() * d_fields.element_size() >= int(ctx._lib.llvq_field_bytes(ctx._h, nblocks, gain_bits))
+    return _dev(d_codebook, "d_codebook"), (None if d_row_scale is None else _dev(d_row_scale, "d_row_scale"))
+
+
+def llvq_dequant_matrix_sg(ctx: Context, d_fields: torch.Tensor, gain_bits: int, d_codebook: torch.Tensor,
+                           d_row_scale: torch.Tensor | None, rows: int, cols: int,
+                           d_w: torch.Tensor | None = None, ld: int | None = None, stream=None):
+    """bf16 [rows, cols] weights of the shape-gain form: (row_scale * codebook[k]) * x / |x|, ROWWISE fields
+    (shape index | gain index << index_bits); ``d_row_scale`` may be None."""
+    ld = cols if ld is None else ld
+    if d_w is None:
+        d_w = torch.empty((rows, ld), dtype=torch.bfloat16, device=d_fields.device)
+    assert d_w.dtype == torch.bfloat16
+    assert d_w.numel() >= (rows - 1) * ld + cols if rows else True
+    cb, rs = _sg_args(ctx, d_fields, gain_bits, d_codebook, d_row_scale, rows, rows * ((cols + 23) // 24))
+    _check("llvq_dequant_matrix_sg", ctx._lib.llvq_dequant_matrix_sg(
+        ctx._h, _dev(d_fields, "d_fields"), gain_bits, cb, rs, rows, cols, _dev(d_w, "d_w"), ld, _stream_ptr(stream)))
+    return d_w
+
+
+def llvq_gemv_sg(ctx: Context, d_fields: torch.Tensor, gain_bits: int, d_codebook: torch.Tensor,
+                 d_row_scale: torch.Tensor | None, n_out: int, k_in: int, d_x: torch.Tensor,
+                 d_y: torch.Tensor | None = None, y_dtype: torch.dtype = torch.float32, stream=None):
+    """y = W x with W in the shape-gain form of ``llvq_dequant_matrix_sg``."""
+    if d_y is None:
+        d_y = torch.empty(n_out, dtype=y_dtype, device=d_fields.device)
+    assert d_x.dtype == torch.bfloat16 and d_x.numel() >= k_in
+    assert d_y.dtype in (torch.float32, torch.bfloat16) and d_y.numel() >= n_out
+    cb, rs = _sg_args(ctx, d_fields, gain_bits, d_codebook, d_row_scale, n_out, n_out * ((k_in + 23) // 24))
+    code = LLVQ_F32 if d_y.dtype == torch.float32 else LLVQ_BF16
+    _check("llvq_gemv_sg", ctx._lib.llvq_gemv_sg(ctx._h, _dev(d_fields, "d_fields"), gain_bits, cb, rs, n_out, k_in,
+                                                 _dev(d_x, "d_x"), _dev(d_y, "d_y"), code, _stream_ptr(stream)))
     return d_y
 
 

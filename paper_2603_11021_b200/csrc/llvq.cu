@@ -120,6 +120,35 @@ __device__ __forceinline__ void block_pairs(const FastArgs& fa, const FastSmem& 
     }
 }
 
+// Shape-gain form of the gain step (App. E "Shape-gain" with a scalar gain codebook): the stored field carries the
+// shape index in its low W bits and a gain index above; the block gain is
+// (row_scale * codebook[k]) / |x|, each operation in binary32, 1/|x| = 1/sqrt(16 m) taken from the class descriptor.
+struct SgArgs {
+    const float* codebook;      // [1 << bits]
+    const float* row_scale;     // [rows] or null (= 1)
+    int bits;
+};
+
+__device__ __forceinline__ void block_pairs_sg(const FastArgs& fa, const FastSmem& T, const uint32_t* __restrict__ stream,
+                                               const SgArgs& sg, uint64_t b, int64_t row, bool in, uint32_t w[12])
+{
+    const uint64_t f = in ? load_field(stream, b, (int)fa.L.W + sg.bits) : 0ull;
+    const uint64_t I = f & ((1ull << fa.L.W) - 1ull);                 // W < 64 whenever gain bits are present or not: checked on the host
+    const uint32_t k = (uint32_t)(f >> fa.L.W);
+    const bool valid = in && I < fa.n_points;
+    if (in && !valid) atomicAdd(fa.bad_index, 1ull);
+    uint64_t local = 0;
+    const uint32_t cls = valid ? fast_find_class(T, I, local) : 0u;
+    Decoded d;
+    fast_decode_local<-1>(T, cls, local, valid, kFullMask, d);
+    float g = 0.f;
+    if (in) {
+        const float scale = sg.row_scale ? __ldg(sg.row_scale + row) : 1.f;
+        g = __fmul_rn(__fmul_rn(scale, __ldg(sg.codebook + k)), __uint_as_float(T.desc[cls * kFastDescStride + kFastDescRnorm]));
+    }
+    expand_bf16(d, g, w);
+}
+
 #define FAST_PROLOGUE()                                                                         \
     extern __shared__ __align__(128) uint8_t smem[];                                            \
     uint64_t* bar = reinterpret_cast<uint64_t*>(smem + fa.L.total);                              \
@@ -149,9 +178,9 @@ decode_blocks_fast_kernel(FastArgs fa, const uint32_t* __restrict__ stream, uint
 
 // FLAT (bpr == 0): block b covers elements 24b.. of the flattened matrix.
 // ROWWISE: block b = r * bpr + cb covers columns 24cb.. of row r.
-template <bool kBig>
+template <bool kBig, bool kSg = false>
 __global__ void __launch_bounds__(kFastThreads, 1)
-dequant_fast_kernel(FastArgs fa, const uint32_t* __restrict__ stream, const uint16_t* __restrict__ gain, uint64_t nblocks,
+dequant_fast_kernel(FastArgs fa, const uint32_t* __restrict__ stream, const uint16_t* __restrict__ gain, SgArgs sg, uint64_t nblocks,
                     int64_t rows, int64_t cols, int64_t bpr, __nv_bfloat16* __restrict__ out, int64_t ld)
 {
     FAST_PROLOGUE();
@@ -161,7 +190,8 @@ dequant_fast_kernel(FastArgs fa, const uint32_t* __restrict__ stream, const uint
         const uint64_t b = tile * kFastThreads + threadIdx.x;
         const bool in = b < nblocks;
         uint32_t w[12];
-        block_pairs<kBig>(fa, T, stream, gain, b, in, w);             // whole warp: the decoders vote
+        if (kSg) block_pairs_sg(fa, T, stream, sg, b, in ? (int64_t)(b / (uint64_t)bpr) : 0, in, w);   // ROWWISE only
+        else block_pairs<kBig>(fa, T, stream, gain, b, in, w);        // whole warp: the decoders vote
         if (!in) continue;
         __nv_bfloat16* dst;
         int64_t left;
@@ -198,9 +228,9 @@ __device__ __forceinline__ void mma_bf16_16816(float c[4], uint32_t a0, uint32_t
 // CTA that owns unit u when G CTAs split U units into ranges [c*U/G, (c+1)*U/G).
 __device__ __forceinline__ int64_t unit_owner(int64_t u, int64_t U, int64_t G) { return ((u + 1) * G - 1) / U; }
 
-template <bool kBig, bool kOutBf16>
+template <bool kBig, bool kOutBf16, bool kSg = false>
 __global__ void __launch_bounds__(kGemvThreads, 1)
-gemv_fast_kernel(FastArgs fa, const uint32_t* __restrict__ stream, const uint16_t* __restrict__ gain,
+gemv_fast_kernel(FastArgs fa, const uint32_t* __restrict__ stream, const uint16_t* __restrict__ gain, SgArgs sg,
                  int64_t n_out, int64_t k_in, int64_t bpr, const uint16_t* __restrict__ x, void* __restrict__ y,
                  float* __restrict__ scratch, uint32_t* __restrict__ counters)
 {
@@ -233,7 +263,8 @@ gemv_fast_kernel(FastArgs fa, const uint32_t* __restrict__ stream, const uint16_
             const bool in = row < n_out && cb < bpr;
             const uint64_t b = (uint64_t)(row * bpr + cb);
             uint32_t w[12];
-            block_pairs<kBig>(fa, T, stream, gain, b, in, w);
+            if (kSg) block_pairs_sg(fa, T, stream, sg, b, row, in, w);
+            else block_pairs<kBig>(fa, T, stream, gain, b, in, w);
             const uint4* xb = reinterpret_cast<const uint4*>(xs + cb * 12);
             const uint4 x0 = xb[0], x1 = xb[1], x2 = xb[2];
             const uint32_t xv[12] = {x0.x, x0.y, x0.z, x0.w, x1.x, x1.y, x1.z, x1.w, x2.x, x2.y, x2.z, x2.w};
@@ -881,22 +912,21 @@ int llvq_dequant_matrix(const llvq_ctx* ctx, const void* d_idx, const uint16_t* 
     __nv_bfloat16* w = reinterpret_cast<__nv_bfloat16*>(d_w_bf16);
     if (ctx->fast) {
         if (!set_smem(dequant_fast_kernel<false>, smem)) return LLVQ_ECUDA;
-        dequant_fast_kernel<false><<<g, kFastThreads, smem, st>>>(fast_args(ctx), idx, d_gain_f16, nblocks, rows, cols, bpr, w, ld);
+        dequant_fast_kernel<false><<<g, kFastThreads, smem, st>>>(fast_args(ctx), idx, d_gain_f16, SgArgs{}, nblocks, rows, cols, bpr, w, ld);
     } else {
         if (!set_smem(dequant_fast_kernel<true>, smem)) return LLVQ_ECUDA;
-        dequant_fast_kernel<true><<<g, kFastThreads, smem, st>>>(fast_args(ctx), idx, d_gain_f16, nblocks, rows, cols, bpr, w, ld);
+        dequant_fast_kernel<true><<<g, kFastThreads, smem, st>>>(fast_args(ctx), idx, d_gain_f16, SgArgs{}, nblocks, rows, cols, bpr, w, ld);
     }
     return launch_status();
 }
 
-int llvq_gemv(const llvq_ctx* ctx, const void* d_idx, const uint16_t* d_gain_f16, int64_t n_out, int64_t k_in,
-              const uint16_t* d_x_bf16, void* d_y, int y_dtype, void* stream)
+// Shared by llvq_gemv and llvq_gemv_sg: exactly one of d_gain_f16 / sg is used.
+static int gemv_common(const llvq_ctx* ctx, const void* d_idx, const uint16_t* d_gain_f16, const SgArgs* sg, int64_t n_out, int64_t k_in,
+                       const uint16_t* d_x_bf16, void* d_y, int y_dtype, void* stream)
 {
-    if (ctx && ctx->device >= 0 && n_out == 0) return LLVQ_OK;                     // nothing to do: pointers may be null
-    if (int e = check_common(ctx, d_idx)) return e;
-    if (!d_gain_f16 || !d_x_bf16 || !d_y || n_out < 0 || k_in < 0) return LLVQ_EINVAL;
+    if (!d_x_bf16 || !d_y || n_out < 0 || k_in < 0) return LLVQ_EINVAL;
     if (y_dtype != LLVQ_F32 && y_dtype != LLVQ_BF16) return LLVQ_EINVAL;
-    if (!aligned(d_gain_f16, 2) || !aligned(d_x_bf16, 2) || !aligned(d_y, y_dtype == LLVQ_F32 ? 4 : 2)) return LLVQ_EALIGN;
+    if (!aligned(d_x_bf16, 2) || !aligned(d_y, y_dtype == LLVQ_F32 ? 4 : 2)) return LLVQ_EALIGN;
     if (n_out == 0) return LLVQ_OK;
     DeviceGuard guard(ctx->device);
     if (!guard.ok) return LLVQ_ECUDA;
@@ -920,16 +950,76 @@ int llvq_gemv(const llvq_ctx* ctx, const void* d_idx, const uint16_t* d_gain_f16
     const unsigned threads = 32u * (unsigned)warps;
     const uint32_t* idx = static_cast<const uint32_t*>(d_idx);
     const FastArgs fa = fast_args(ctx);
-#define LLVQ_LAUNCH_GEMV(BIG, BF16)                                                                           \
-    do {                                                                                                      \
-        if (!set_smem(gemv_fast_kernel<BIG, BF16>, smem)) return LLVQ_ECUDA;                                  \
-        gemv_fast_kernel<BIG, BF16><<<g, threads, smem, st>>>(fa, idx, d_gain_f16, n_out, k_in, bpr, d_x_bf16, d_y, \
-                                                              ctx->d_scratch, ctx->d_counters);               \
+    const SgArgs sga = sg ? *sg : SgArgs{};
+#define LLVQ_LAUNCH_GEMV(BIG, BF16, SG)                                                                            \
+    do {                                                                                                           \
+        if (!set_smem(gemv_fast_kernel<BIG, BF16, SG>, smem)) return LLVQ_ECUDA;                                   \
+        gemv_fast_kernel<BIG, BF16, SG><<<g, threads, smem, st>>>(fa, idx, d_gain_f16, sga, n_out, k_in, bpr, d_x_bf16, d_y, \
+                                                                  ctx->d_scratch, ctx->d_counters);                \
     } while (0)
-    if (ctx->fast) { if (y_dtype == LLVQ_BF16) LLVQ_LAUNCH_GEMV(false, true); else LLVQ_LAUNCH_GEMV(false, false); }
-    else           { if (y_dtype == LLVQ_BF16) LLVQ_LAUNCH_GEMV(true, true);  else LLVQ_LAUNCH_GEMV(true, false); }
+    if (sg)             { if (y_dtype == LLVQ_BF16) LLVQ_LAUNCH_GEMV(false, true, true);  else LLVQ_LAUNCH_GEMV(false, false, true); }
+    else if (ctx->fast) { if (y_dtype == LLVQ_BF16) LLVQ_LAUNCH_GEMV(false, true, false); else LLVQ_LAUNCH_GEMV(false, false, false); }
+    else                { if (y_dtype == LLVQ_BF16) LLVQ_LAUNCH_GEMV(true, true, false);  else LLVQ_LAUNCH_GEMV(true, false, false); }
 #undef LLVQ_LAUNCH_GEMV
     return launch_status();
+}
+
+int llvq_gemv(const llvq_ctx* ctx, const void* d_idx, const uint16_t* d_gain_f16, int64_t n_out, int64_t k_in,
+              const uint16_t* d_x_bf16, void* d_y, int y_dtype, void* stream)
+{
+    if (ctx && ctx->device >= 0 && n_out == 0) return LLVQ_OK;                     // nothing to do: pointers may be null
+    if (int e = check_common(ctx, d_idx)) return e;
+    if (!d_gain_f16) return LLVQ_EINVAL;
+    if (!aligned(d_gain_f16, 2)) return LLVQ_EALIGN;
+    return gemv_common(ctx, d_idx, d_gain_f16, nullptr, n_out, k_in, d_x_bf16, d_y, y_dtype, stream);
+}
+
+// Argument checks of the shape-gain entry points.
+static int check_sg(const llvq_ctx* ctx, const void* d_fields, int gain_bits, const float* d_codebook, const float* d_row_scale)
+{
+    if (int e = check_common(ctx, d_fields)) return e;
+    if (gain_bits < 0 || gain_bits > 8 || !d_codebook) return LLVQ_EINVAL;
+    if (!aligned(d_codebook, 4) || !aligned(d_row_scale, 4)) return LLVQ_EALIGN;
+    if (!ctx->fast || ctx->host.W + gain_bits > 64 || ctx->host.W > 63) return LLVQ_EUNSUPPORTED;
+    return LLVQ_OK;
+}
+
+size_t llvq_field_bytes(const llvq_ctx* ctx, uint64_t nblocks, int gain_bits)
+{
+    if (!ctx || gain_bits < 0 || gain_bits > 8) return 0;
+    unsigned __int128 bits = (unsigned __int128)nblocks * (unsigned)(ctx->host.W + gain_bits);
+    return (size_t)(((bits + 7) / 8 + 15) / 16 * 16);
+}
+
+int llvq_dequant_matrix_sg(const llvq_ctx* ctx, const void* d_fields, int gain_bits, const float* d_codebook_f32,
+                           const float* d_row_scale_f32, int64_t rows, int64_t cols, uint16_t* d_w_bf16, int64_t ld, void* stream)
+{
+    if (ctx && ctx->device >= 0 && (rows == 0 || cols == 0)) return LLVQ_OK;      // nothing to do: pointers may be null
+    if (int e = check_sg(ctx, d_fields, gain_bits, d_codebook_f32, d_row_scale_f32)) return e;
+    if (!d_w_bf16 || rows < 0 || cols < 0 || ld < cols) return LLVQ_EINVAL;
+    if (!aligned(d_w_bf16, 2)) return LLVQ_EALIGN;
+    if (rows > (1ll << 31) || cols > (1ll << 31)) return LLVQ_EUNSUPPORTED;
+    DeviceGuard guard(ctx->device);
+    if (!guard.ok) return LLVQ_ECUDA;
+    const int64_t bpr = (cols + 23) / 24;
+    const uint64_t nblocks = (uint64_t)rows * (uint64_t)bpr;
+    const size_t smem = ctx->fl.total + 16;
+    const uint64_t tiles = (nblocks + kFastThreads - 1) / kFastThreads;
+    const unsigned g = (unsigned)std::min<uint64_t>(tiles, (uint64_t)ctx->sm_count);
+    if (!set_smem(dequant_fast_kernel<false, true>, smem)) return LLVQ_ECUDA;
+    dequant_fast_kernel<false, true><<<g, kFastThreads, smem, (cudaStream_t)stream>>>(
+        fast_args(ctx), static_cast<const uint32_t*>(d_fields), nullptr, SgArgs{d_codebook_f32, d_row_scale_f32, gain_bits},
+        nblocks, rows, cols, bpr, reinterpret_cast<__nv_bfloat16*>(d_w_bf16), ld);
+    return launch_status();
+}
+
+int llvq_gemv_sg(const llvq_ctx* ctx, const void* d_fields, int gain_bits, const float* d_codebook_f32, const float* d_row_scale_f32,
+                 int64_t n_out, int64_t k_in, const uint16_t* d_x_bf16, void* d_y, int y_dtype, void* stream)
+{
+    if (ctx && ctx->device >= 0 && n_out == 0) return LLVQ_OK;                     // nothing to do: pointers may be null
+    if (int e = check_sg(ctx, d_fields, gain_bits, d_codebook_f32, d_row_scale_f32)) return e;
+    const SgArgs sg{d_codebook_f32, d_row_scale_f32, gain_bits};
+    return gemv_common(ctx, d_fields, nullptr, &sg, n_out, k_in, d_x_bf16, d_y, y_dtype, stream);
 }
 
 // Kernel-private packed layout (see the comment at repack_kernel).  Available for codes whose classes fit the

@@ -290,6 +290,8 @@ bool build_fast_image(const HostTables& t, FastLayout& L, std::vector<uint8_t>& 
         }
         std::memcpy(&w[4], vals, 8);
         w[15] = nbytes;
+        const float rnorm = (float)(1.0 / std::sqrt(16.0 * (double)d.m));
+        std::memcpy(&w[kFastDescRnorm], &rnorm, 4);
     }
     return true;
 }

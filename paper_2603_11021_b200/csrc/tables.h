@@ -77,7 +77,8 @@ bool build_tables(int m_lo, int m_hi, HostTables& out);
 namespace llvq {
 
 constexpr int kFastMaxLevels = 4;      // unranking steps per class on the fast path
-constexpr int kFastDescWords = 16;     // words of a class descriptor that carry data
+constexpr int kFastDescWords = 17;     // words of a class descriptor that carry data
+constexpr int kFastDescRnorm = 16;     // word holding 1 / sqrt(16 m) as binary32
 constexpr int kFastDescStride = 20;    // words between descriptors: 80 bytes spread consecutive classes over all bank groups
 constexpr int kLowBits = 14;           // slots resolved by one table lookup in the subset unranking
 
@@ -108,6 +109,7 @@ struct FastLayout {
 //  8..11: level l: radix | k << 22 | id << 27 | (value bit 1) << 30 | (value nonzero) << 31
 //  12..14: floor(2^32 / radix) of levels 1..3
 //  15: n (free slots before the step) of levels 0..3, one byte each
+//  16: binary32 bits of 1 / |x| = 1 / sqrt(16 m) (formed in binary64, rounded once), for the shape-gain form
 // with_classes = false builds only the class-independent tables (Golay, Pascal, subsets, deposit): codes whose class
 // tables do not fit shared memory keep those in global memory.
 bool build_fast_image(const HostTables& t, FastLayout& layout, std::vector<uint8_t>& image, bool with_classes = true);
