@@ -65,6 +65,9 @@ def _load():
             lib.oc_gemm_rows_sg.restype = i64
             lib.oc_gemm_rows_sg.argtypes = [vp, vp, ctypes.c_int, vp, vp, i64, i64, vp, ctypes.c_int, i64, i64, vp]
             lib.oc_nearest_angular.argtypes = [vp, vp, vp]
+            lib.oc_encode.restype = i64
+            lib.oc_encode.argtypes = [vp, vp, i64, ctypes.c_int, vp, vp, vp]
+            lib.oc_nearest_lattice_point.argtypes = [vp, i64, vp, vp]
             lib.oc_is_member.argtypes = [vp]
             lib.oc_shell_size.argtypes = [ctypes.c_int, u64p]
             lib.oc_golay_table.argtypes = [vp]
@@ -109,6 +112,18 @@ def is_member(x) -> int:
 
 def dequant_scalar(gain_f16_bits: int, x: int) -> int:
     return int(_load().oc_dequant_scalar(int(gain_f16_bits), int(x)))
+
+
+def nearest_lattice_point(v) -> tuple[np.ndarray, np.ndarray]:
+    """Nearest point of the unbounded lattice (integer coordinates) to each row of v, and the squared distances."""
+    a = np.ascontiguousarray(np.asarray(v, dtype=np.float64)).reshape(-1, 24)
+    pts = np.zeros((len(a), 24), dtype=np.int32)
+    d2 = np.zeros(len(a), dtype=np.float64)
+    _load().oc_nearest_lattice_point(_ptr(a), len(a), _ptr(pts), _ptr(d2))
+    return pts, d2
+
+
+EUCLIDEAN, ANGULAR = 0, 1
 
 
 class Code:
@@ -276,6 +291,28 @@ class Code:
             with ThreadPoolExecutor(threads) as ex:
                 list(ex.map(run, jobs))
         return y[0] if vec else y
+
+    def encode(self, v, metric: int, threads: int = 1) -> tuple[np.ndarray, list[int]]:
+        """Nearest points of the code to the rows of v (integer-coordinate units) and their indices."""
+        a = np.ascontiguousarray(np.asarray(v, dtype=np.float64)).reshape(-1, 24)
+        n = len(a)
+        pts = np.zeros((n, 24), dtype=np.int8)
+        lo = np.zeros(n, dtype=np.uint64)
+        hi = np.zeros(n, dtype=np.uint64)
+
+        def run(job):
+            f, c = job
+            return int(self._lib.oc_encode(self._h, _ptr(a[f:f + c]), c, metric, _ptr(pts[f:f + c]), _ptr(lo[f:f + c]), _ptr(hi[f:f + c])))
+
+        if threads <= 1 or n < 2 * threads:
+            bad = run((0, n))
+        else:
+            step = -(-n // threads)
+            with ThreadPoolExecutor(threads) as ex:
+                bad = sum(ex.map(run, [(s, min(step, n - s)) for s in range(0, n, step)]))
+        if bad:
+            raise ValueError(f"the search gave up on {bad} vectors (unsupported code?)")
+        return pts, _join(lo, hi)
 
     def nearest_angular(self, x) -> int:
         v = np.ascontiguousarray(np.asarray(x, dtype=np.float64))

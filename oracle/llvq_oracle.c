@@ -819,6 +819,129 @@ int64_t oc_gemm_rows_sg(const oc_code* code, const uint8_t* stream, int gain_bit
 }
 
 /* ------------------------------------------------------------------------- */
+/* Encoder: nearest point of the code to a real vector (Sec. 3.1, "Extending to */
+/* spherical search": Euclidean scoring for spherical shaping, angular scoring */
+/* for shape-gain).  The paper defers the search itself to the literature; the */
+/* search used here is coset decoding of the whole lattice, which is exact for */
+/* the unbounded lattice: every lattice point is pi + 2c + 4z with pi the      */
+/* parity, c a Golay codeword and z integer, subject to the sum rule of        */
+/* Sec. 2.4; for fixed (pi, c) the nearest z is found by rounding each          */
+/* coordinate and, if the sum rule fails, moving the coordinate with the       */
+/* largest rounding error to its other neighbour.  The best of the 2 x 4096     */
+/* cosets is the nearest lattice point.  Ties: lowest parity, then lowest      */
+/* codeword position in T; inside a coset the first coordinate with the        */
+/* largest error.  Inputs are in integer-coordinate units (|x|^2 = 16 m).      */
+/*                                                                           */
+/* Restriction to the shells m_lo..m_hi of the code (m_lo must be 2, m_hi >= 6):*/
+/* EUCLIDEAN (metric 0): the input is projected into the ball of radius        */
+/*   sqrt(16 m_hi) (App. E "Spherical shaping"); while the nearest lattice      */
+/*   point of the working vector lies beyond the last shell the working vector  */
+/*   is shrunk by 2 %; if the nearest point is the origin the input is scaled   */
+/*   to the radius of the first shell and decoded once more.                   */
+/* ANGULAR (metric 1): for every shell radius sqrt(16 m) the input direction    */
+/*   scaled to that radius is decoded; of the candidates that lie in the code   */
+/*   the one with the largest cosine wins (first radius on ties).              */
+/* A zero input encodes to index 0.  This is a practical search, exact for the */
+/* unbounded lattice and near-optimal on the cut; what is pinned is the exact  */
+/* part (brute force over small shells) and the distortion it reaches.        */
+/* ------------------------------------------------------------------------- */
+static double nearest_in_lattice(const double v[OC_DIM], int best_x[OC_DIM])
+{
+    oc_golay_init();
+    double best = INFINITY;
+    for (int pi = 0; pi < 2; ++pi)
+        for (int j = 0; j < 4096; ++j) {
+            uint32_t c = g_T[j];
+            int x[OC_DIM]; double err[OC_DIM]; long sum = 0; double d2 = 0;
+            for (int i = 0; i < OC_DIM; ++i) {
+                int base = pi + 2 * (int)((c >> i) & 1u);
+                double t = (v[i] - base) / 4.0;
+                double z = rint(t);                       /* ties to even */
+                err[i] = t - z;
+                x[i] = base + 4 * (int)z;
+                sum += x[i];
+            }
+            long want = pi ? 4 : 0;
+            if (((sum % 8) + 8) % 8 != want) {            /* sum rule violated: one coordinate moves by 4 */
+                int k = 0;
+                for (int i = 1; i < OC_DIM; ++i) if (fabs(err[i]) > fabs(err[k])) k = i;
+                x[k] += err[k] > 0 ? 4 : (err[k] < 0 ? -4 : 4);
+            }
+            for (int i = 0; i < OC_DIM; ++i) { double d = v[i] - x[i]; d2 += d * d; }
+            if (d2 < best) { best = d2; memcpy(best_x, x, sizeof x); }
+        }
+    return best;
+}
+
+static int shell_of(const int x[OC_DIM])
+{
+    long n = 0;
+    for (int i = 0; i < OC_DIM; ++i) n += (long)x[i] * x[i];
+    return (int)(n / 16);
+}
+
+/* Returns 0 and the point, or 1 if the code is not one the encoder supports / the search gave up (point = index 0). */
+static int encode_point(const oc_code* code, const double v[OC_DIM], int metric, int8_t out[OC_DIM])
+{
+    int x[OC_DIM], bestx[OC_DIM];
+    double n2 = 0;
+    for (int i = 0; i < OC_DIM; ++i) n2 += v[i] * v[i];
+    int ok = 0;
+    if (code->m_lo != 2 || code->m_hi < 6) { unrank_point(code, 0, out); return 1; }
+    if (n2 == 0) { unrank_point(code, 0, out); return 0; }
+    if (metric == 0) {
+        double R2 = 16.0 * code->m_hi, u[OC_DIM], f = n2 > R2 ? sqrt(R2 / n2) : 1.0;
+        for (int i = 0; i < OC_DIM; ++i) u[i] = v[i] * f;
+        for (int it = 0; it < 64 && !ok; ++it) {
+            nearest_in_lattice(u, x);
+            int m = shell_of(x);
+            if (m > code->m_hi) { for (int i = 0; i < OC_DIM; ++i) u[i] *= 0.98; }
+            else if (m < 2) { double g = sqrt(32.0 / n2); for (int i = 0; i < OC_DIM; ++i) u[i] = v[i] * g; }
+            else { ok = 1; memcpy(bestx, x, sizeof x); }
+        }
+    } else {
+        double best = -INFINITY, rn = 1.0 / sqrt(n2);
+        for (int m = code->m_lo; m <= code->m_hi; ++m) {
+            double u[OC_DIM], rad = sqrt(16.0 * m);
+            for (int i = 0; i < OC_DIM; ++i) u[i] = v[i] * rn * rad;
+            nearest_in_lattice(u, x);
+            int mx = shell_of(x);
+            if (mx < code->m_lo || mx > code->m_hi) continue;
+            double dot = 0, xx = 0;
+            for (int i = 0; i < OC_DIM; ++i) { dot += v[i] * rn * x[i]; xx += (double)x[i] * x[i]; }
+            double score = dot / sqrt(xx);
+            if (score > best) { best = score; ok = 1; memcpy(bestx, x, sizeof x); }
+        }
+    }
+    if (!ok) { unrank_point(code, 0, out); return 1; }
+    for (int i = 0; i < OC_DIM; ++i) out[i] = (int8_t)bestx[i];
+    return 0;
+}
+
+/* v: n x 24 doubles.  points: n x 24 int8; lo/hi: the indices.  Returns the number of vectors the search gave up on. */
+int64_t oc_encode(const oc_code* code, const double* v, int64_t n, int metric, int8_t* points, uint64_t* lo, uint64_t* hi)
+{
+    int64_t bad = 0;
+    for (int64_t b = 0; b < n; ++b) {
+        bad += encode_point(code, v + b * OC_DIM, metric, points + b * OC_DIM);
+        u128 I = 0;
+        rank_point(code, points + b * OC_DIM, &I);
+        lo[b] = (uint64_t)I; hi[b] = (uint64_t)(I >> 64);
+    }
+    return bad;
+}
+
+/* The exact part alone: nearest point of the unbounded lattice (points may have any norm, the origin included). */
+void oc_nearest_lattice_point(const double* v, int64_t n, int32_t* points, double* dist2)
+{
+    for (int64_t b = 0; b < n; ++b) {
+        int x[OC_DIM];
+        dist2[b] = nearest_in_lattice(v + b * OC_DIM, x);
+        for (int i = 0; i < OC_DIM; ++i) points[b * OC_DIM + i] = x[i];
+    }
+}
+
+/* ------------------------------------------------------------------------- */
 /* Angular nearest point (Sec. 3.1): argmax over all points v of the code of   */
 /* <x, v> / |v|, by brute force.  Lowest index wins ties.  Tiny codes only.   */
 /* ------------------------------------------------------------------------- */
