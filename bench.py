@@ -363,6 +363,19 @@ def extras(P, ctx) -> dict:
                                               "bits_per_weight": 48 * nb12 / (n * k)}
     assert P.llvq_last_error(ctx12) == (0, 0)
     del bufs12, ctx12
+    # --- encoder: nearest-point search + indexing of a 4096 x 4096 matrix worth of Gaussian blocks (offline step)
+    nb_enc = 4096 * 4096 // 24
+    torch.manual_seed(0)
+    v_enc = torch.randn((nb_enc, 24), device="cuda", dtype=torch.float32) * 2.5
+    p_enc = torch.empty((nb_enc, 24), dtype=torch.int8, device="cuda")
+    i_enc = torch.empty(nb_enc, dtype=torch.int64, device="cuda")
+    for name, metric, reps in (("euclidean", P.LLVQ_EUCLIDEAN, 3), ("angular", P.LLVQ_ANGULAR, 1)):
+        fn = lambda i: P.llvq_encode_blocks(ctx, v_enc, metric, d_points=p_enc, d_index=i_enc)
+        fn(0)
+        us_enc = _event_us(torch, fn, reps)
+        out[f"encode_{name}_4096x4096"] = {"ms": us_enc / 1e3, "blocks_per_s": nb_enc / (us_enc * 1e-6), "weights_per_s": 24 * nb_enc / (us_enc * 1e-6)}
+    assert P.llvq_last_error(ctx) == (0, 0)
+    del v_enc, p_enc, i_enc
     out["llama3_8b_linear_sweep"] = {"us_per_token": sweep_us, "tokens_per_s": 1e6 / sweep_us, "GBps": by / sweep_us / 1e3, "blocks_per_token": blocks,
                                      "launches_per_token": 32 * len(shapes), "algorithmic_bytes": by}
     return out

@@ -54,7 +54,9 @@ enum {
 };
 enum { LLVQ_LAYOUT_FLAT = 0, LLVQ_LAYOUT_ROWWISE = 1 };
 enum { LLVQ_F32 = 0, LLVQ_BF16 = 1 };
-enum { LLVQ_FLAG_WAIT_TIMEOUT = 1u };   /* bit in llvq_last_error's flags */
+enum { LLVQ_FLAG_WAIT_TIMEOUT = 1u,     /* bits in llvq_last_error's flags */
+       LLVQ_FLAG_SEARCH_GAVE_UP = 4u }; /* the encoder's search found no point of the code for some input (non-finite input) */
+enum { LLVQ_EUCLIDEAN = 0, LLVQ_ANGULAR = 1 };   /* scoring of the encoder's search (Sec. 3.1) */
 
 /*
  * Build the tables of the code  union of Shell(m), m_lo <= m <= m_hi  (Sec. 2.2:
@@ -205,6 +207,37 @@ int llvq_gemm_small_batch(const llvq_ctx* ctx, const void* d_idx, const uint16_t
 int llvq_gemm_small_batch_noalloc(const llvq_ctx* ctx, const void* d_idx, const uint16_t* d_gain_f16,
                                   int64_t n_out, int64_t k_in, const uint16_t* d_x_bf16,
                                   int batch, uint16_t* d_y_bf16, void* stream);
+
+/*
+ * Encoder (Sec. 3.1 "Extending to spherical search", Sec. 3.2 "Indexing scheme"): nearest point of the code to
+ * each real vector, and its index.  d_v_f32: device, [nblocks][24] floats in units of the integer coordinates
+ * (a point of Shell(m) has squared norm 16 m; the caller applies its own scale).  Outputs: d_points, device,
+ * int8 [nblocks][24] (the chosen lattice points) and d_index, device, uint64 [nblocks], 8-byte aligned (their
+ * indices, ready for llvq_pack_fields).
+ *
+ * The paper defers the search itself to the literature.  Here the nearest point of the unbounded lattice is found
+ * exactly by decoding all 2 x 4096 cosets (parity, Golay codeword) + 4 Z^24 under the sum rules of Sec. 2.4;
+ * the restriction to the shells of the code is a policy:
+ *   LLVQ_EUCLIDEAN (spherical shaping, App. E): the input is projected into the ball of radius sqrt(16 m_hi); while
+ *     the nearest lattice point lies beyond the last shell the working vector is shrunk by 2 %; if it is the
+ *     origin the input is scaled to the radius of the first shell and decoded again.
+ *   LLVQ_ANGULAR (shape-gain, App. E): the input direction is decoded at every shell radius sqrt(16 m),
+ *     m_lo <= m <= m_hi; of the candidates that lie in the code the one with the largest cosine wins.
+ * A zero vector encodes to index 0.  Non-finite inputs encode to index 0 and set LLVQ_FLAG_SEARCH_GAVE_UP.
+ * Supported codes: m_lo == 2, m_hi >= 6, indices of at most 64 bits; others return LLVQ_EUNSUPPORTED.
+ *
+ * llvq_rank_blocks is the indexing step alone (point -> index, the inverse of llvq_decode_blocks): a point that
+ * is not in the code gets index 0 and is counted like an out-of-range field (llvq_last_error).
+ *
+ * llvq_pack_fields writes the stored stream from the indices: field b = d_index[b] | d_gain_index[b] << W
+ * (gain_bits = 0: the plain index stream of llvq_index_bytes() bytes, d_gain_index ignored; otherwise the
+ * shape-gain fields of llvq_field_bytes() bytes).  d_fields: device, 16-byte aligned.
+ */
+int llvq_encode_blocks(const llvq_ctx* ctx, const float* d_v_f32, uint64_t nblocks, int metric,
+                       int8_t* d_points, uint64_t* d_index, void* stream);
+int llvq_rank_blocks(const llvq_ctx* ctx, const int8_t* d_points, uint64_t nblocks, uint64_t* d_index, void* stream);
+int llvq_pack_fields(const llvq_ctx* ctx, const uint64_t* d_index, const uint8_t* d_gain_index, int gain_bits,
+                     uint64_t nblocks, void* d_fields, void* stream);
 
 /*
  * Self-test of the error path every kernel of this library uses for its device-side waits (table copy,

@@ -17,12 +17,15 @@ from .build import LIB
 __all__ = [
     "Context", "llvq_decode_blocks", "llvq_dequant_matrix", "llvq_gemv", "llvq_gemm_small_batch", "llvq_gemm_small_batch_noalloc",
     "llvq_dequant_matrix_sg", "llvq_gemv_sg", "llvq_repack", "llvq_gemv_packed",
+    "llvq_encode_blocks", "llvq_rank_blocks", "llvq_pack_fields", "LLVQ_EUCLIDEAN", "LLVQ_ANGULAR",
     "llvq_last_error", "LlvqError", "EXPORTS", "load_library",
     "LLVQ_LAYOUT_FLAT", "LLVQ_LAYOUT_ROWWISE", "LLVQ_F32", "LLVQ_BF16",
 ]
 
 LLVQ_LAYOUT_FLAT, LLVQ_LAYOUT_ROWWISE = 0, 1
 LLVQ_F32, LLVQ_BF16 = 0, 1
+LLVQ_EUCLIDEAN, LLVQ_ANGULAR = 0, 1
+LLVQ_FLAG_WAIT_TIMEOUT, LLVQ_FLAG_SEARCH_GAVE_UP = 1, 4
 _STATUS = {0: "LLVQ_OK", 1: "LLVQ_EINVAL", 2: "LLVQ_EALIGN", 3: "LLVQ_EUNSUPPORTED", 4: "LLVQ_ECUDA",
            5: "LLVQ_EINDEX", 6: "LLVQ_ETIMEOUT"}
 
@@ -32,6 +35,7 @@ EXPORTS = [
     "llvq_decode_blocks", "llvq_dequant_matrix", "llvq_gemv", "llvq_gemm_small_batch", "llvq_gemm_small_batch_noalloc",
     "llvq_packed_bytes", "llvq_repack", "llvq_gemv_packed", "llvq_selftest_wait_timeout", "llvq_last_error",
     "llvq_field_bytes", "llvq_dequant_matrix_sg", "llvq_gemv_sg", "llvq_class_info", "llvq_golay_table",
+    "llvq_encode_blocks", "llvq_rank_blocks", "llvq_pack_fields",
 ]
 
 
@@ -75,6 +79,9 @@ def load_library() -> ctypes.CDLL:
     lib.llvq_field_bytes.restype = ctypes.c_size_t
     lib.llvq_dequant_matrix_sg.argtypes = [vp, vp, ctypes.c_int, vp, vp, i64, i64, vp, i64, vp]
     lib.llvq_gemv_sg.argtypes = [vp, vp, ctypes.c_int, vp, vp, i64, i64, vp, vp, ctypes.c_int, vp]
+    lib.llvq_encode_blocks.argtypes = [vp, vp, u64, ctypes.c_int, vp, vp, vp]
+    lib.llvq_rank_blocks.argtypes = [vp, vp, u64, vp, vp]
+    lib.llvq_pack_fields.argtypes = [vp, vp, vp, ctypes.c_int, u64, vp, vp]
     lib.llvq_last_error.argtypes = [vp, vp, ctypes.POINTER(u64), ctypes.POINTER(ctypes.c_uint32)]
     lib.llvq_class_info.argtypes = [vp, ctypes.c_int, vp, vp, vp, vp, vp, vp]
     lib.llvq_golay_table.argtypes = [vp, vp]
@@ -285,6 +292,49 @@ def llvq_gemv_packed(ctx: Context, d_packed: torch.Tensor, d_gain: torch.Tensor,
     _check("llvq_gemv_packed", ctx._lib.llvq_gemv_packed(ctx._h, _dev(d_packed, "d_packed"), _dev(d_gain, "d_gain"), n_out, k_in,
                                                          _dev(d_x, "d_x"), _dev(d_y, "d_y"), code, _stream_ptr(stream)))
     return d_y
+
+
+def llvq_encode_blocks(ctx: Context, d_v: torch.Tensor, metric: int, d_points: torch.Tensor | None = None,
+                       d_index: torch.Tensor | None = None, stream=None):
+    """(points int8 [n, 24], indices int64 [n]) of the code points nearest to the rows of ``d_v`` (float32 [n, 24],
+    integer-coordinate units) under LLVQ_EUCLIDEAN or LLVQ_ANGULAR scoring."""
+    assert d_v.dtype == torch.float32 and d_v.dim() == 2 and d_v.shape[1] == 24
+    n = d_v.shape[0]
+    if d_points is None:
+        d_points = torch.empty((n, 24), dtype=torch.int8, device=d_v.device)
+    if d_index is None:
+        d_index = torch.empty(n, dtype=torch.int64, device=d_v.device)
+    assert d_points.dtype == torch.int8 and d_points.numel() >= n * 24 and d_index.dtype == torch.int64 and d_index.numel() >= n
+    _check("llvq_encode_blocks", ctx._lib.llvq_encode_blocks(ctx._h, _dev(d_v, "d_v"), n, metric, _dev(d_points, "d_points"),
+                                                             _dev(d_index, "d_index"), _stream_ptr(stream)))
+    return d_points, d_index
+
+
+def llvq_rank_blocks(ctx: Context, d_points: torch.Tensor, d_index: torch.Tensor | None = None, stream=None):
+    """Indices (int64 [n]) of the lattice points ``d_points`` (int8 [n, 24]); the inverse of ``llvq_decode_blocks``."""
+    assert d_points.dtype == torch.int8 and d_points.dim() == 2 and d_points.shape[1] == 24
+    n = d_points.shape[0]
+    if d_index is None:
+        d_index = torch.empty(n, dtype=torch.int64, device=d_points.device)
+    assert d_index.dtype == torch.int64 and d_index.numel() >= n
+    _check("llvq_rank_blocks", ctx._lib.llvq_rank_blocks(ctx._h, _dev(d_points, "d_points"), n, _dev(d_index, "d_index"), _stream_ptr(stream)))
+    return d_index
+
+
+def llvq_pack_fields(ctx: Context, d_index: torch.Tensor, d_gain_index: torch.Tensor | None = None, gain_bits: int = 0,
+                     d_fields: torch.Tensor | None = None, stream=None):
+    """The stored stream (uint8) of the fields index | gain index << index_bits."""
+    assert d_index.dtype == torch.int64
+    n = d_index.numel()
+    nbytes = int(ctx._lib.llvq_field_bytes(ctx._h, n, gain_bits))
+    if d_fields is None:
+        d_fields = torch.empty(nbytes, dtype=torch.uint8, device=d_index.device)
+    assert d_fields.numel() * d_fields.element_size() >= nbytes
+    assert gain_bits == 0 or (d_gain_index is not None and d_gain_index.dtype == torch.uint8 and d_gain_index.numel() >= n)
+    _check("llvq_pack_fields", ctx._lib.llvq_pack_fields(
+        ctx._h, _dev(d_index, "d_index"), None if d_gain_index is None or gain_bits == 0 else _dev(d_gain_index, "d_gain_index"),
+        gain_bits, n, _dev(d_fields, "d_fields"), _stream_ptr(stream)))
+    return d_fields
 
 
 def llvq_selftest_wait_timeout(ctx: Context, stream=None) -> None:

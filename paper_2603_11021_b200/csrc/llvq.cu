@@ -15,35 +15,12 @@
 #include "big.cuh"
 #include "umma.cuh"
 #include "tables.h"
+#include "ctx.h"
 
 using namespace llvq;
 
-struct llvq_ctx {
-    int device = 0;
-    HostTables host;
-    DevCode dev{};
-    void* d_blob = nullptr;          // one allocation holding every device table
-    unsigned long long* d_err = nullptr;
-    int sm_count = 0;
-    float* d_scratch = nullptr;      // split-K accumulation buffer of the small-batch GEMM, kept all-zero between calls
-    uint32_t* d_counters = nullptr;  // per row tile arrival counters, kept zero between calls
-    bool fast = false;               // class tables fit the shared-memory image; otherwise they are read from global memory
-    FastLayout fl{};
-    const uint8_t* d_image = nullptr;
-};
-
 namespace {
 
-struct DeviceGuard {
-    int prev = -1; bool ok = false;
-    explicit DeviceGuard(int dev) {
-        if (cudaGetDevice(&prev) != cudaSuccess) return;
-        ok = (prev == dev) || cudaSetDevice(dev) == cudaSuccess;
-    }
-    ~DeviceGuard() { if (ok && prev >= 0) cudaSetDevice(prev); }
-};
-
-inline bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) & (a - 1)) == 0; }
 
 // ===========================================================================
 // Fast path (tables in shared memory).  Dynamic shared memory of every fast
@@ -774,7 +751,22 @@ int llvq_create(llvq_ctx** out, int m_lo, int m_hi, int device)
     std::vector<uint32_t> lut16;
     build_bucket_table(h, lut16);
 
-    // one blob: [off_hi | off_lo | classes | bucket table | error words | table image | counters | scratch], 256-byte aligned parts
+    // encoder tables (point -> index), for codes the encoder supports
+    std::vector<uint64_t> hkeys; std::vector<uint32_t> hcls;
+    std::vector<uint16_t> pos12(4096, 0xffff);
+    ctx->can_encode = m_lo == 2 && m_hi >= 6 && h.W <= 64 && build_class_hash(h, hkeys, hcls);
+    if (ctx->can_encode) {
+        for (uint32_t j = 0; j < 4096; ++j) {
+            uint16_t& slot = pos12[h.golay[j] & 0xfffu];
+            if (slot != 0xffff) ctx->can_encode = false;       // the low 12 bits must identify the codeword
+            slot = (uint16_t)j;
+        }
+    }
+    if (!ctx->can_encode) { hkeys.clear(); hcls.clear(); }
+    uint64_t sigs[64];
+    for (int a = 0; a < 64; ++a) sigs[a] = sig_of_value(a);
+
+    // one blob: [off_hi | off_lo | classes | bucket table | error words | table image | encoder tables | counters | scratch], 256-byte aligned parts
     auto up = [](size_t v) { return (v + 255) & ~size_t(255); };
     size_t o_offhi = 0;
     size_t o_offlo = up(o_offhi + (ncls + 1) * 4);
@@ -782,7 +774,12 @@ int llvq_create(llvq_ctx** out, int m_lo, int m_hi, int device)
     size_t o_lut = up(o_cls + ncls * sizeof(ClassDesc));
     size_t o_err = up(o_lut + lut16.size() * 4);
     size_t o_img = up(o_err + 256);
-    size_t o_cnt = up(o_img + image.size());
+    size_t o_gol = up(o_img + image.size());
+    size_t o_p12 = up(o_gol + 4096 * 4);
+    size_t o_sig = up(o_p12 + 4096 * 2);
+    size_t o_hk = up(o_sig + sizeof sigs);
+    size_t o_hc = up(o_hk + hkeys.size() * 8);
+    size_t o_cnt = up(o_hc + hcls.size() * 4);
     size_t o_scr = up(o_cnt + (size_t)(64 * kMaxScratchRows / 8) * 4);    // one counter per group of 8 rows (GEMV) / per 128-row tile (GEMM)
     size_t total = o_scr + (size_t)64 * kMaxScratchRows * 4;
     std::vector<uint8_t> blob(o_cnt, 0);
@@ -791,6 +788,13 @@ int llvq_create(llvq_ctx** out, int m_lo, int m_hi, int device)
     std::memcpy(blob.data() + o_cls, h.desc.data(), ncls * sizeof(ClassDesc));
     std::memcpy(blob.data() + o_lut, lut16.data(), lut16.size() * 4);
     std::memcpy(blob.data() + o_img, image.data(), image.size());
+    std::memcpy(blob.data() + o_gol, h.golay.data(), 4096 * 4);
+    std::memcpy(blob.data() + o_p12, pos12.data(), 4096 * 2);
+    std::memcpy(blob.data() + o_sig, sigs, sizeof sigs);
+    if (!hkeys.empty()) {
+        std::memcpy(blob.data() + o_hk, hkeys.data(), hkeys.size() * 8);
+        std::memcpy(blob.data() + o_hc, hcls.data(), hcls.size() * 4);
+    }
     if (cudaMalloc(&ctx->d_blob, total) != cudaSuccess) { delete ctx; return LLVQ_ECUDA; }
     if (cudaMemcpy(ctx->d_blob, blob.data(), blob.size(), cudaMemcpyHostToDevice) != cudaSuccess ||
         cudaMemset(static_cast<uint8_t*>(ctx->d_blob) + o_cnt, 0, total - o_cnt) != cudaSuccess) {
@@ -808,6 +812,12 @@ int llvq_create(llvq_ctx** out, int m_lo, int m_hi, int device)
     ctx->dev.nclasses = (int)ncls;
     ctx->dev.W = h.W;
     ctx->d_image = d + o_img;
+    ctx->d_golay = reinterpret_cast<const uint32_t*>(d + o_gol);
+    ctx->enc.pos_by_low12 = reinterpret_cast<const uint16_t*>(d + o_p12);
+    ctx->enc.sig_of_value = reinterpret_cast<const uint64_t*>(d + o_sig);
+    ctx->enc.hash_key = reinterpret_cast<const uint64_t*>(d + o_hk);
+    ctx->enc.hash_cls = reinterpret_cast<const uint32_t*>(d + o_hc);
+    ctx->enc.hash_mask = hkeys.empty() ? 0u : (uint32_t)(hkeys.size() - 1);
     ctx->d_counters = reinterpret_cast<uint32_t*>(d + o_cnt);
     ctx->d_scratch = reinterpret_cast<float*>(d + o_scr);
     *out = ctx;

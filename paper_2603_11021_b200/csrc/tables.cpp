@@ -313,3 +313,38 @@ void build_bucket_table(const HostTables& t, std::vector<uint32_t>& lut)
 }
 
 }  // namespace llvq
+
+namespace llvq {
+
+// splitmix64 of (a + 1): fixed, well-mixed 64-bit numbers
+uint64_t sig_of_value(int a)
+{
+    uint64_t z = (uint64_t)(a + 1) * 0x9E3779B97F4A7C15ull;
+    z = (z ^ (z >> 30)) * 0xBF58476D1CE4E5B9ull;
+    z = (z ^ (z >> 27)) * 0x94D049BB133111EBull;
+    return z ^ (z >> 31);
+}
+
+// Open-addressing table (linear probing) from class signature to class number, at most 25 % full.
+bool build_class_hash(const HostTables& t, std::vector<uint64_t>& keys, std::vector<uint32_t>& cls)
+{
+    size_t size = 64;
+    while (size < 4 * t.info.size()) size *= 2;
+    keys.assign(size, 0);
+    cls.assign(size, 0);
+    for (size_t j = 0; j < t.info.size(); ++j) {
+        const ClassInfo& c = t.info[j];
+        uint64_t sig = 0;
+        for (size_t i = 0; i < c.values.size(); ++i) sig += (uint64_t)c.mults[i] * sig_of_value(c.values[i]);
+        if (sig == 0) return false;
+        size_t slot = (size_t)(sig >> 20) & (size - 1);
+        while (keys[slot]) {
+            if (keys[slot] == sig) return false;             // two classes with one signature
+            slot = (slot + 1) & (size - 1);
+        }
+        keys[slot] = sig; cls[slot] = (uint32_t)j;
+    }
+    return true;
+}
+
+}  // namespace llvq

@@ -115,4 +115,11 @@ struct FastLayout {
 bool build_fast_image(const HostTables& t, FastLayout& layout, std::vector<uint8_t>& image, bool with_classes = true);
 void build_bucket_table(const HostTables& t, std::vector<uint32_t>& lut);   // u32[65537], see tables.cpp
 
+// Encoder side (point -> class).  Signature of a class: sum over its 24 absolute values of a fixed pseudo-random
+// 64-bit number per value (the multiset fixes shell and parity).  build_class_hash() fills an open-addressing
+// table (linear probing from (signature >> 20) & (size - 1), key 0 = empty) and returns false if two classes of the
+// code share a signature.
+uint64_t sig_of_value(int a);
+bool build_class_hash(const HostTables& t, std::vector<uint64_t>& keys, std::vector<uint32_t>& cls);
+
 }  // namespace llvq
