@@ -155,20 +155,24 @@ int llvq_gemv_sg(const llvq_ctx* ctx, const void* d_fields, int gain_bits, const
                  void* d_y, int y_dtype, void* stream);
 
 /*
- * Kernel-private packed layout for the fused GEMV (preprocessing at load time; the paper describes no storage
- * layout beyond "a compact integer index" per block, Sec. 1, and App. A step 5 notes that blocks are independent,
- * which is what makes reordering them legitimate).  llvq_repack rewrites a ROWWISE index stream once: the class
- * lookup of App. A steps 1-2 is done here, and inside tiles of 8 rows x 16 column blocks the blocks are grouped
- * by the form of steps 3-4 their class needs (odd classes / even classes of Golay weight 8, 12, 16 / others), each
- * block becoming a 64-bit entry (class-local index, class, position in the tile).  llvq_gemv_packed computes the
- * same y = W x as llvq_gemv from the packed stream and the unchanged gain array.
- * The packed stream takes llvq_packed_bytes() bytes (8 per block, tiles padded; 0 if the code is not
- * supported: it must have at most 512 classes of at most 2^45 points, which holds for (2,2), (3,3), (2,13)).
- * d_packed: device, 16-byte aligned.  Out-of-range fields are counted at repack time and decode to zero.
+ * Sorted layout for the fused GEMV: a kernel-private arrangement of the same blocks, made once at load time (the
+ * paper describes no storage layout beyond "a compact integer index" per block, Sec. 1, and App. A step 5 notes
+ * that blocks are independent, which is what makes reordering them legitimate).  llvq_sort_blocks rewrites a
+ * ROWWISE index stream for the GPU of this context: the blocks each thread block of the GEMV will own are stored,
+ * in segments of up to 65536 blocks, ordered by the form of App. A steps 3-4 their class needs (odd / even with
+ * Golay weight 8, 12, 16 / other), its number of unranking steps and the class, every block as a 64-bit entry
+ * holding the stored index unchanged (low 48 bits) and its position in the segment (high 16 bits).
+ * llvq_gemv_sorted computes the same y = W x as llvq_gemv: all of App. A steps 1-4 still run in the kernel, but the
+ * 32 lanes of a warp now execute one form with one trip count and read one class descriptor.
+ * The sorted stream takes llvq_sorted_bytes() bytes (8 per block of the 8-row x 4-block units the matrix is padded
+ * to; 0 if unsupported: the code must have its class tables in shared memory, at most 1023 classes and fewer than
+ * 2^48 - 1 points, which holds for (2,2), (3,3) and (2,13), not for (2,53)).  The layout depends on the SM count of
+ * the device; use it with the context that produced it.  d_sorted: device, 16-byte aligned.  Out-of-range fields
+ * are counted when sorting and decode to zero.  Gains stay in their ROWWISE array.
  */
-size_t llvq_packed_bytes(const llvq_ctx* ctx, int64_t n_out, int64_t k_in);
-int llvq_repack(const llvq_ctx* ctx, const void* d_idx, int64_t n_out, int64_t k_in, void* d_packed, void* stream);
-int llvq_gemv_packed(const llvq_ctx* ctx, const void* d_packed, const uint16_t* d_gain_f16,
+size_t llvq_sorted_bytes(const llvq_ctx* ctx, int64_t n_out, int64_t k_in);
+int llvq_sort_blocks(const llvq_ctx* ctx, const void* d_idx, int64_t n_out, int64_t k_in, void* d_sorted, void* stream);
+int llvq_gemv_sorted(const llvq_ctx* ctx, const void* d_sorted, const uint16_t* d_gain_f16,
                      int64_t n_out, int64_t k_in, const uint16_t* d_x_bf16,
                      void* d_y, int y_dtype, void* stream);
 

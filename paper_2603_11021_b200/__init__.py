@@ -16,8 +16,9 @@ from .build import LIB
 
 __all__ = [
     "Context", "llvq_decode_blocks", "llvq_dequant_matrix", "llvq_gemv", "llvq_gemm_small_batch", "llvq_gemm_small_batch_noalloc",
-    "llvq_dequant_matrix_sg", "llvq_gemv_sg", "llvq_repack", "llvq_gemv_packed",
+    "llvq_dequant_matrix_sg", "llvq_gemv_sg",
     "llvq_encode_blocks", "llvq_rank_blocks", "llvq_pack_fields", "LLVQ_EUCLIDEAN", "LLVQ_ANGULAR",
+    "llvq_sort_blocks", "llvq_gemv_sorted",
     "llvq_last_error", "LlvqError", "EXPORTS", "load_library",
     "LLVQ_LAYOUT_FLAT", "LLVQ_LAYOUT_ROWWISE", "LLVQ_F32", "LLVQ_BF16",
 ]
@@ -33,9 +34,10 @@ _STATUS = {0: "LLVQ_OK", 1: "LLVQ_EINVAL", 2: "LLVQ_EALIGN", 3: "LLVQ_EUNSUPPORT
 EXPORTS = [
     "llvq_create", "llvq_destroy", "llvq_index_bits", "llvq_num_points", "llvq_num_classes", "llvq_index_bytes",
     "llvq_decode_blocks", "llvq_dequant_matrix", "llvq_gemv", "llvq_gemm_small_batch", "llvq_gemm_small_batch_noalloc",
-    "llvq_packed_bytes", "llvq_repack", "llvq_gemv_packed", "llvq_selftest_wait_timeout", "llvq_last_error",
+    "llvq_selftest_wait_timeout", "llvq_last_error",
     "llvq_field_bytes", "llvq_dequant_matrix_sg", "llvq_gemv_sg", "llvq_class_info", "llvq_golay_table",
     "llvq_encode_blocks", "llvq_rank_blocks", "llvq_pack_fields",
+    "llvq_sorted_bytes", "llvq_sort_blocks", "llvq_gemv_sorted",
 ]
 
 
@@ -71,14 +73,14 @@ def load_library() -> ctypes.CDLL:
     lib.llvq_gemm_small_batch.argtypes = [vp, vp, vp, i64, i64, vp, ctypes.c_int, vp, vp]
     lib.llvq_gemm_small_batch_noalloc.argtypes = [vp, vp, vp, i64, i64, vp, ctypes.c_int, vp, vp]
     lib.llvq_selftest_wait_timeout.argtypes = [vp, vp]
-    lib.llvq_packed_bytes.argtypes = [vp, i64, i64]
-    lib.llvq_packed_bytes.restype = ctypes.c_size_t
-    lib.llvq_repack.argtypes = [vp, vp, i64, i64, vp, vp]
-    lib.llvq_gemv_packed.argtypes = [vp, vp, vp, i64, i64, vp, vp, ctypes.c_int, vp]
     lib.llvq_field_bytes.argtypes = [vp, u64, ctypes.c_int]
     lib.llvq_field_bytes.restype = ctypes.c_size_t
     lib.llvq_dequant_matrix_sg.argtypes = [vp, vp, ctypes.c_int, vp, vp, i64, i64, vp, i64, vp]
     lib.llvq_gemv_sg.argtypes = [vp, vp, ctypes.c_int, vp, vp, i64, i64, vp, vp, ctypes.c_int, vp]
+    lib.llvq_sorted_bytes.argtypes = [vp, i64, i64]
+    lib.llvq_sorted_bytes.restype = ctypes.c_size_t
+    lib.llvq_sort_blocks.argtypes = [vp, vp, i64, i64, vp, vp]
+    lib.llvq_gemv_sorted.argtypes = [vp, vp, vp, i64, i64, vp, vp, ctypes.c_int, vp]
     lib.llvq_encode_blocks.argtypes = [vp, vp, u64, ctypes.c_int, vp, vp, vp]
     lib.llvq_rank_blocks.argtypes = [vp, vp, u64, vp, vp]
     lib.llvq_pack_fields.argtypes = [vp, vp, vp, ctypes.c_int, u64, vp, vp]
@@ -266,30 +268,30 @@ def llvq_gemm_small_batch_noalloc(ctx: Context, d_idx: torch.Tensor, d_gain: tor
     return d_y
 
 
-def llvq_repack(ctx: Context, d_idx: torch.Tensor, n_out: int, k_in: int, d_packed: torch.Tensor | None = None, stream=None):
-    """Rewrite a ROWWISE index stream into the kernel-private packed layout of ``llvq_gemv_packed`` (done once per matrix)."""
-    nbytes = int(ctx._lib.llvq_packed_bytes(ctx._h, n_out, k_in))
+def llvq_sort_blocks(ctx: Context, d_idx: torch.Tensor, n_out: int, k_in: int, d_sorted: torch.Tensor | None = None, stream=None):
+    """Rewrite a ROWWISE index stream into the sorted layout of ``llvq_gemv_sorted`` (done once per matrix, per device)."""
+    nbytes = int(ctx._lib.llvq_sorted_bytes(ctx._h, n_out, k_in))
     if nbytes == 0:
-        raise LlvqError("llvq_packed_bytes", 3)
-    if d_packed is None:
-        d_packed = torch.empty(nbytes, dtype=torch.uint8, device=d_idx.device)
-    assert d_packed.numel() * d_packed.element_size() >= nbytes
+        raise LlvqError("llvq_sorted_bytes", 3)
+    if d_sorted is None:
+        d_sorted = torch.empty(nbytes, dtype=torch.uint8, device=d_idx.device)
+    assert d_sorted.numel() * d_sorted.element_size() >= nbytes
     assert d_idx.numel() * d_idx.element_size() >= ctx.index_bytes(n_out * ((k_in + 23) // 24))
-    _check("llvq_repack", ctx._lib.llvq_repack(ctx._h, _dev(d_idx, "d_idx"), n_out, k_in, _dev(d_packed, "d_packed"), _stream_ptr(stream)))
-    return d_packed
+    _check("llvq_sort_blocks", ctx._lib.llvq_sort_blocks(ctx._h, _dev(d_idx, "d_idx"), n_out, k_in, _dev(d_sorted, "d_sorted"), _stream_ptr(stream)))
+    return d_sorted
 
 
-def llvq_gemv_packed(ctx: Context, d_packed: torch.Tensor, d_gain: torch.Tensor, n_out: int, k_in: int, d_x: torch.Tensor,
+def llvq_gemv_sorted(ctx: Context, d_sorted: torch.Tensor, d_gain: torch.Tensor, n_out: int, k_in: int, d_x: torch.Tensor,
                      d_y: torch.Tensor | None = None, y_dtype: torch.dtype = torch.float32, stream=None):
-    """y = W x from the packed stream of ``llvq_repack`` and the ROWWISE gains; same result as ``llvq_gemv``."""
+    """y = W x from the sorted stream of ``llvq_sort_blocks`` and the ROWWISE gains; same result as ``llvq_gemv``."""
     if d_y is None:
-        d_y = torch.empty(n_out, dtype=y_dtype, device=d_packed.device)
+        d_y = torch.empty(n_out, dtype=y_dtype, device=d_sorted.device)
     assert d_x.dtype == torch.bfloat16 and d_x.numel() >= k_in and d_gain.dtype == torch.float16
     assert d_y.dtype in (torch.float32, torch.bfloat16) and d_y.numel() >= n_out
     assert d_gain.numel() >= n_out * ((k_in + 23) // 24)
-    assert d_packed.numel() * d_packed.element_size() >= int(ctx._lib.llvq_packed_bytes(ctx._h, n_out, k_in))
+    assert d_sorted.numel() * d_sorted.element_size() >= int(ctx._lib.llvq_sorted_bytes(ctx._h, n_out, k_in))
     code = LLVQ_F32 if d_y.dtype == torch.float32 else LLVQ_BF16
-    _check("llvq_gemv_packed", ctx._lib.llvq_gemv_packed(ctx._h, _dev(d_packed, "d_packed"), _dev(d_gain, "d_gain"), n_out, k_in,
+    _check("llvq_gemv_sorted", ctx._lib.llvq_gemv_sorted(ctx._h, _dev(d_sorted, "d_sorted"), _dev(d_gain, "d_gain"), n_out, k_in,
                                                          _dev(d_x, "d_x"), _dev(d_y, "d_y"), code, _stream_ptr(stream)))
     return d_y
 

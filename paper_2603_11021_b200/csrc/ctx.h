@@ -31,6 +31,7 @@ struct llvq_ctx {
     bool can_encode = false;         // m_lo == 2, m_hi >= 6, indices fit 64 bits
     EncTables enc{};
     const uint32_t* d_golay = nullptr;   // [4096] sorted codewords in global memory
+    const uint16_t* d_sort_rank = nullptr;   // [nclasses] (fast codes with at most 1023 classes) position of a class in the order of the sorted layout
 };
 
 namespace llvq {

@@ -233,8 +233,9 @@ gemv_fast_kernel(FastArgs fa, const uint32_t* __restrict__ stream, const uint16_
         for (int i = threadIdx.x; i < kGemvGroupsPerPass * kGemvGroupRows; i += (int)blockDim.x) acc[i] = 0.f;
         __syncthreads();
         const int64_t p_begin = max(u_begin, rg0 * nq), p_end = min(u_end, (rg1 + 1) * nq);
-        for (int64_t u = p_begin + warp; u < p_end; u += kWarps) {
-            const int64_t rg = u / nq, kq = u - rg * nq;
+        int64_t rg = (p_begin + warp) / nq, kq = (p_begin + warp) - rg * nq;      // walked along with u: no division per unit
+        for (int64_t u = p_begin + warp; u < p_end; u += kWarps, kq += kWarps) {
+            while (kq >= nq) { kq -= nq; ++rg; }
             const int64_t cb = kq * 4 + t;
             const int64_t row = rg * kGemvGroupRows + g;
             const bool in = row < n_out && cb < bpr;
@@ -285,177 +286,205 @@ gemv_fast_kernel(FastArgs fa, const uint32_t* __restrict__ stream, const uint16_
             }
             __syncthreads();
         }
+        __syncthreads();                                   // the sums are read above: the next pass may clear them only now
     }
 }
 
-// ===========================================================================
-// Kernel-private packed layout for the fused GEMV (llvq_repack / llvq_gemv_packed).
-// The matrix is cut into tiles of 8 rows x 16 column blocks (128 blocks).  Inside a tile the blocks are
-// reordered so that blocks whose classes need the same decoder form are adjacent: first the odd classes, then
-// the even classes of Golay weight 8/12/16, then all others, then padding.  Each block becomes one 64-bit
-// entry: class-local index (45 bits) | class (9 bits) << 45 | position in the tile (8 bits) << 54 | kind << 62.
-// The class lookup (S2) is done once, by llvq_repack; the GEMV then runs one decoder form per group of 32
-// entries (both forms only for the group that straddles a boundary) instead of the any-class form for all.
-// Gains stay in their ROWWISE array.  Tiles are stored row-tile major, 1024 bytes each.
-// ===========================================================================
-constexpr int kPackRows = 8, kPackCols = 16, kPackTile = kPackRows * kPackCols;
-constexpr uint32_t kKindEven = 0u, kKindOdd = 1u, kKindOther = 2u, kKindNull = 3u;
+constexpr uint32_t kKindEven = 0u, kKindOdd = 1u, kKindOther = 2u, kKindNull = 3u;   // decoder form a class needs
 
-__global__ void __launch_bounds__(256, 1)
-repack_kernel(FastArgs fa, const uint32_t* __restrict__ stream, int64_t n_out, int64_t bpr, int64_t col_tiles, int64_t ntiles,
-              unsigned long long* __restrict__ out)
+// ===========================================================================
+// Sorted layout for the fused GEMV (llvq_sort_blocks / llvq_gemv_sorted).
+// The work is cut exactly as in gemv_fast_kernel: units of 8 rows x 4 column blocks, row group major, an equal
+// contiguous range of units per CTA (for the CTA count of this device).  Inside a CTA's range the units are taken
+// in segments of up to kSortSegUnits units, and the blocks of a segment are stored sorted by the decoder form
+// their class needs (odd / even with Golay weight 8, 12, 16 / other) and its number of unranking steps (most
+// expensive first), so that the 32 lanes of a warp run the same form with the same trip count.  Each block is a
+// 64-bit entry: the stored index I unchanged in the low 48 bits, its position in the segment (unit * 32 + lane)
+// in the high 16 bits; entries that do not exist (ragged edges) or are out of range carry I = 2^48 - 1.
+// All of App. A runs in the GEMV kernel.  A warp takes 32 consecutive entries, each lane unranks its block and
+// multiplies it with its own slice of x (binary32 FMAs), and adds the partial row sum to the CTA's row sums.
+// ===========================================================================
+constexpr int kSortSegUnits = 2048;                  // 65536 blocks
+constexpr int kSortThreads = 1024;
+constexpr int kSortAccCopies = 4;                    // copies of the row sums in shared memory (a power of two)
+constexpr unsigned long long kSortIndexMask = (1ull << 48) - 1ull;
+
+// Calls f(tu0, tu1, rg0, rg1, first, last) for every segment [tu0, tu1) of CTA `cta` (of G) in order; rg0..rg1 = row
+// groups of the pass the segment belongs to (a pass covers at most kGemvGroupsPerPass row groups); first / last =
+// the segment opens / closes its pass.
+template <typename F>
+__device__ __forceinline__ void for_each_sorted_segment(int64_t U, int64_t G, int64_t nq, int64_t cta, F f)
+{
+    const int64_t u_begin = cta * U / G, u_end = (cta + 1) * U / G;
+    if (u_begin >= u_end) return;
+    const int64_t rg_first = u_begin / nq, rg_last = (u_end - 1) / nq;
+    for (int64_t rg0 = rg_first; rg0 <= rg_last; rg0 += kGemvGroupsPerPass) {
+        const int64_t rg1 = min(rg0 + kGemvGroupsPerPass - 1, rg_last);
+        const int64_t p_begin = max(u_begin, rg0 * nq), p_end = min(u_end, (rg1 + 1) * nq);
+        for (int64_t tu0 = p_begin; tu0 < p_end; tu0 += kSortSegUnits)
+            f(tu0, min(tu0 + (int64_t)kSortSegUnits, p_end), rg0, rg1, tu0 == p_begin, tu0 + kSortSegUnits >= p_end);
+    }
+}
+
+__global__ void __launch_bounds__(kSortThreads, 1)
+sort_blocks_kernel(FastArgs fa, const uint32_t* __restrict__ stream, const uint16_t* __restrict__ sort_rank, int64_t n_out, int64_t bpr,
+                   unsigned long long* __restrict__ out)
 {
     FAST_PROLOGUE();
-    const int lane = threadIdx.x & 31;
-    const int64_t warps = (int64_t)gridDim.x * (blockDim.x >> 5);
-    for (int64_t tile = (int64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5); tile < ntiles; tile += warps) {
-        const int64_t rt = tile / col_tiles, ct = tile - rt * col_tiles;
-        unsigned long long e[kPackTile / 32];
-        uint32_t count[4] = {0, 0, 0, 0};
-#pragma unroll
-        for (int j = 0; j < kPackTile / 32; ++j) {
-            const uint32_t pos = (uint32_t)(j * 32 + lane);
-            const int64_t row = rt * kPackRows + pos / kPackCols, cb = ct * kPackCols + pos % kPackCols;
-            const bool in = row < n_out && cb < bpr;
-            const uint64_t I = in ? load_field(stream, (uint64_t)(row * bpr + cb), (int)fa.L.W) : 0ull;
-            const bool valid = in && I < fa.n_points;
-            if (in && !valid) atomicAdd(fa.bad_index, 1ull);
-            uint32_t kind = kKindNull;
-            uint64_t local = 0; uint32_t cls = 0;
-            if (valid) {
-                cls = fast_find_class(T, I, local);
-                const uint32_t h = T.desc[cls * kFastDescStride];
-                const uint32_t w = h & 0xffu;
-                kind = (h & (1u << 16)) ? kKindOdd : ((w == 8u || w == 12u || w == 16u) ? kKindEven : kKindOther);
-            }
-            e[j] = local | (unsigned long long)cls << 45 | (unsigned long long)pos << 54 | (unsigned long long)kind << 62;
-#pragma unroll
-            for (uint32_t k = 0; k < 4; ++k) count[k] += __popc(__ballot_sync(kFullMask, kind == k));
+    __shared__ uint32_t hist[1024], cursor[1024];                  // one bin per class, in sort order; bin 1023 = no block
+    const int64_t nq = (bpr + 3) / 4;
+    const int64_t groups = (n_out + kGemvGroupRows - 1) / kGemvGroupRows;
+    const int64_t U = groups * nq, G = gridDim.x;
+    for_each_sorted_segment(U, G, nq, blockIdx.x, [&](int64_t tu0, int64_t tu1, int64_t, int64_t, bool, bool) {
+        const int entries = (int)(tu1 - tu0) * 32;
+        hist[threadIdx.x] = 0; cursor[threadIdx.x] = 0;
+        __syncthreads();
+        // key and field of entry i of the segment; count = the first pass (out-of-range fields are counted once)
+        auto entry_of = [&](int i, bool count, unsigned long long& field) {
+            const int64_t u = tu0 + (i >> 5);
+            const int lane = i & 31;
+            const int64_t rg = u / nq, kq = u - rg * nq;
+            const int64_t row = rg * kGemvGroupRows + (lane >> 2), cb = kq * 4 + (lane & 3);
+            field = kSortIndexMask;
+            if (row >= n_out || cb >= bpr) return 1023u;
+            const uint64_t I = load_field(stream, (uint64_t)(row * bpr + cb), (int)fa.L.W);
+            if (I >= fa.n_points) { if (count) atomicAdd(fa.bad_index, 1ull); return 1023u; }
+            uint64_t local;
+            field = I;
+            return (uint32_t)__ldg(sort_rank + fast_find_class(T, I, local));
+        };
+        for (int i = threadIdx.x; i < entries; i += kSortThreads) {
+            unsigned long long field;
+            atomicAdd(&hist[entry_of(i, true, field)], 1u);
         }
-        // order of the groups in the tile: odd, even, other, null
-        const uint32_t first[4] = {count[kKindOdd], 0u, count[kKindOdd] + count[kKindEven], count[kKindOdd] + count[kKindEven] + count[kKindOther]};
-        uint32_t seen[4] = {0, 0, 0, 0};
-#pragma unroll
-        for (int j = 0; j < kPackTile / 32; ++j) {
-            const uint32_t kind = (uint32_t)(e[j] >> 62);
-            uint32_t slot = 0;
-#pragma unroll
-            for (uint32_t k = 0; k < 4; ++k) {
-                const uint32_t m = __ballot_sync(kFullMask, kind == k);
-                if (kind == k) slot = (k == kKindOdd ? 0u : first[k]) + seen[k] + __popc(m & ((1u << lane) - 1u));
-                seen[k] += __popc(m);
-            }
-            out[tile * kPackTile + slot] = e[j];
+        __syncthreads();
+        if (threadIdx.x == 0) {
+            uint32_t run = 0;
+            for (int k = 0; k < 1024; ++k) { const uint32_t c = hist[k]; hist[k] = run; run += c; }
         }
-    }
+        __syncthreads();
+        for (int i = threadIdx.x; i < entries; i += kSortThreads) {
+            unsigned long long field;
+            const uint32_t key = entry_of(i, false, field);
+            const uint32_t slot = hist[key] + atomicAdd(&cursor[key], 1u);
+            out[tu0 * 32 + slot] = field | (unsigned long long)i << 48;
+        }
+        __syncthreads();
+    });
 }
 
-constexpr int kPackedThreads = 1024;
-constexpr int kPackedWarps = kPackedThreads / 32;   // upper bound; the launch picks the count that divides the tiles per CTA best
-constexpr int kPackedGroups = 128;         // row groups of 8 rows whose sums a CTA keeps in shared memory at a time
-
 template <bool kOutBf16>
-__global__ void __launch_bounds__(kPackedThreads, 1)
-gemv_packed_kernel(FastArgs fa, const unsigned long long* __restrict__ packed, const uint16_t* __restrict__ gain,
-                   int64_t n_out, int64_t k_in, int64_t bpr, int64_t col_tiles, const uint16_t* __restrict__ x, void* __restrict__ y,
+__global__ void __launch_bounds__(kSortThreads, 1)
+gemv_sorted_kernel(FastArgs fa, const unsigned long long* __restrict__ sorted, const uint16_t* __restrict__ gain,
+                   int64_t n_out, int64_t k_in, int64_t bpr, uint32_t nq_magic, const uint16_t* __restrict__ x, void* __restrict__ y,
                    float* __restrict__ scratch, uint32_t* __restrict__ counters)
 {
     FAST_PROLOGUE();
-    const int64_t nx = col_tiles * kPackCols * 12;                           // packed bf16 pairs of x, zero padded
-    uint32_t* xs = reinterpret_cast<uint32_t*>(staging);
-    float* acc = reinterpret_cast<float*>(xs + nx);                          // [kPackedGroups][16]
-    uint32_t* last_flag = reinterpret_cast<uint32_t*>(acc + kPackedGroups * kPackRows);
-    uint32_t* recs = last_flag + 4;                                          // [warps][256][6]: records of the warp's tile
-    for (int64_t i = threadIdx.x; i < nx; i += blockDim.x) {
+    const int64_t nq = (bpr + 3) / 4;
+    uint32_t* xs = reinterpret_cast<uint32_t*>(staging);            // [nq * 4][12] packed bf16 pairs of x
+    float* acc = reinterpret_cast<float*>(xs + nq * 48);            // [kSortAccCopies][kGemvGroupsPerPass][8]: warps spread their adds over the copies
+    uint32_t* last_flag = reinterpret_cast<uint32_t*>(acc + kSortAccCopies * kGemvGroupsPerPass * kGemvGroupRows);
+    uint32_t* next_chunk = last_flag + 1;
+    for (int64_t i = threadIdx.x; i < nq * 48; i += blockDim.x) {
         const int64_t e = 2 * i;
         const uint32_t lo = e < k_in ? __ldg(x + e) : 0u, hi = e + 1 < k_in ? __ldg(x + e + 1) : 0u;
         xs[i] = lo | hi << 16;
     }
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, g = lane >> 2, t = lane & 3;
-    uint32_t* rec = recs + warp * (kPackTile * 6);
-    const int64_t groups = (n_out + kPackRows - 1) / kPackRows;
-    const int64_t U = groups * col_tiles, G = gridDim.x;                     // units = tiles, row-tile major
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const uint32_t kWarps = blockDim.x >> 5;
+    const int64_t groups = (n_out + kGemvGroupRows - 1) / kGemvGroupRows;
+    const int64_t U = groups * nq, G = gridDim.x;
     const int64_t u_begin = blockIdx.x * U / G, u_end = (blockIdx.x + 1) * U / G;
-    if (u_begin >= u_end) return;
-    const int64_t rg_first = u_begin / col_tiles, rg_last = (u_end - 1) / col_tiles;
-    for (int64_t rg0 = rg_first; rg0 <= rg_last; rg0 += kPackedGroups) {
-        const int64_t rg1 = min(rg0 + kPackedGroups - 1, rg_last);
-        for (int i = threadIdx.x; i < kPackedGroups * kPackRows; i += (int)blockDim.x) acc[i] = 0.f;
+    const uint32_t nq32 = (uint32_t)nq;
+    for_each_sorted_segment(U, G, nq, blockIdx.x, [&](int64_t tu0, int64_t tu1, int64_t rg0, int64_t rg1, bool first, bool last) {
+        if (first)
+            for (int i = threadIdx.x; i < kSortAccCopies * kGemvGroupsPerPass * kGemvGroupRows; i += (int)blockDim.x) acc[i] = 0.f;
+        if (threadIdx.x == 0) *next_chunk = kWarps;
         __syncthreads();
-        const int64_t p_begin = max(u_begin, rg0 * col_tiles), p_end = min(u_end, (rg1 + 1) * col_tiles);
-        for (int64_t u = p_begin + warp; u < p_end; u += (int64_t)(blockDim.x >> 5)) {
-            const int64_t rg = u / col_tiles, ct = u - rg * col_tiles;
-            // ---- unrank the entries of the tile, 32 at a time, one decoder form per kind present
-#pragma unroll 1
-            for (int j = 0; j < kPackTile / 32; ++j) {
-                const unsigned long long e = __ldg(packed + u * kPackTile + j * 32 + lane);
-                const uint32_t kind = (uint32_t)(e >> 62), pos = (uint32_t)(e >> 54) & 0xffu, cls = (uint32_t)(e >> 45) & 0x1ffu;
-                const uint64_t local = e & ((1ull << 45) - 1);
-                Decoded d, r;
-                r.p0 = r.p1 = r.p2 = r.neg = r.vals_lo = r.vals_hi = 0u;
-                if (__any_sync(kFullMask, kind == kKindOdd)) {
-                    const bool mine = kind == kKindOdd;
-                    fast_decode_local<1>(T, mine ? cls : 0u, mine ? local : 0ull, mine, kFullMask, d);
-                    if (mine) r = d;
-                }
-                if (__any_sync(kFullMask, kind == kKindEven)) {
-                    const bool mine = kind == kKindEven;
-                    fast_decode_local<0>(T, mine ? cls : 0u, mine ? local : 0ull, mine, kFullMask, d);
-                    if (mine) r = d;
-                }
-                if (__any_sync(kFullMask, kind == kKindOther)) {
-                    const bool mine = kind == kKindOther;
-                    fast_decode_local<-1>(T, mine ? cls : 0u, mine ? local : 0ull, mine, kFullMask, d);
-                    if (mine) r = d;
-                }
-                uint2* o = reinterpret_cast<uint2*>(rec + pos * 6);
-                o[0] = make_uint2(r.p0, r.p1); o[1] = make_uint2(r.p2, r.neg); o[2] = make_uint2(r.vals_lo, r.vals_hi);
+        const int64_t rg_a = tu0 / nq;
+        const uint32_t kq_a = (uint32_t)(tu0 - rg_a * nq), rg_off = (uint32_t)(rg_a - rg0);
+        const uint32_t nchunks = (uint32_t)(tu1 - tu0);
+        const unsigned long long* seg = sorted + tu0 * 32 + lane;
+        uint32_t ch = (uint32_t)warp;
+        unsigned long long e = ch < nchunks ? __ldg(seg + (uint64_t)ch * 32) : 0ull;
+        while (ch < nchunks) {
+            // chunks are handed out dynamically (their cost depends on the form); the next entry is fetched ahead
+            uint32_t nxt = 0;
+            if (lane == 0) nxt = atomicAdd(next_chunk, 1u);
+            nxt = __shfl_sync(kFullMask, nxt, 0);
+            const unsigned long long e_next = nxt < nchunks ? __ldg(seg + (uint64_t)nxt * 32) : 0ull;
+            const uint64_t I = e & kSortIndexMask;
+            const uint32_t pos = (uint32_t)(e >> 48);
+            const bool valid = I < fa.n_points;
+            // where the block sits: unit = pos / 32 of the segment, (row, column block) = lane of the unit
+            const uint32_t v = kq_a + (pos >> 5);
+            uint32_t q = __umulhi(v, nq_magic), kq = v - q * nq32;
+            if (kq >= nq32) { kq -= nq32; ++q; }
+            const uint32_t rloc = (rg_off + q) * kGemvGroupRows + ((pos >> 2) & 7u);      // row inside the pass
+            const uint32_t cb = kq * 4u + (pos & 3u);
+            const float gn = valid ? gain_to_float(__ldg(gain + ((int64_t)rg0 * kGemvGroupRows + rloc) * bpr + cb)) : 0.f;
+            uint64_t local = 0;
+            const uint32_t cls = valid ? fast_find_class(T, I, local) : 0u;
+            const uint32_t h = T.desc[cls * kFastDescStride];
+            const uint32_t w8 = h & 0xffu;
+            const uint32_t kind = !valid ? kKindNull : ((h & (1u << 16)) ? kKindOdd : ((w8 == 8u || w8 == 12u || w8 == 16u) ? kKindEven : kKindOther));
+            Decoded d, r;
+            r.p0 = r.p1 = r.p2 = r.neg = r.vals_lo = r.vals_hi = 0u;
+            if (__any_sync(kFullMask, kind == kKindOdd)) {
+                const bool mine = kind == kKindOdd;
+                fast_decode_local<1>(T, mine ? cls : 0u, mine ? local : 0ull, mine, kFullMask, d);
+                if (mine) r = d;
             }
-            __syncwarp();
-            // ---- consume: 4 units of 8 rows x 4 column blocks (rows 8..15 of the MMA tile are zero)
-            float c[4] = {0.f, 0.f, 0.f, 0.f};
-#pragma unroll 1
-            for (int q4 = 0; q4 < kPackCols / 4; ++q4) {
-                const int cbl = q4 * 4 + t;
-                const int64_t cb = ct * kPackCols + cbl;
-                const int64_t row = rg * kPackRows + g;
-                const bool in = row < n_out && cb < bpr;
-                const float gn = in ? gain_to_float(__ldg(gain + row * bpr + cb)) : 0.f;
-                Decoded d;
-                const uint2* ia = reinterpret_cast<const uint2*>(rec + (g * kPackCols + cbl) * 6);
-                const uint2 a0 = ia[0], a1 = ia[1], a2 = ia[2];
-                d.p0 = a0.x; d.p1 = a0.y; d.p2 = a1.x; d.neg = a1.y; d.vals_lo = a2.x; d.vals_hi = a2.y;
-                uint32_t w[12];
-                expand_bf16(d, gn, w);
-                const uint4* xb = reinterpret_cast<const uint4*>(xs + cb * 12);
-                const uint4 x0 = xb[0], x1 = xb[1], x2 = xb[2];
-                const uint32_t xv[12] = {x0.x, x0.y, x0.z, x0.w, x1.x, x1.y, x1.z, x1.w, x2.x, x2.y, x2.z, x2.w};
+            if (__any_sync(kFullMask, kind == kKindEven)) {
+                const bool mine = kind == kKindEven;
+                fast_decode_local<0>(T, mine ? cls : 0u, mine ? local : 0ull, mine, kFullMask, d);
+                if (mine) r = d;
+            }
+            if (__any_sync(kFullMask, kind == kKindOther)) {
+                const bool mine = kind == kKindOther;
+                fast_decode_local<-1>(T, mine ? cls : 0u, mine ? local : 0ull, mine, kFullMask, d);
+                if (mine) r = d;
+            }
+            uint32_t w[12];
+            expand_bf16(r, gn, w);
+            const uint4* xb = reinterpret_cast<const uint4*>(xs + cb * 12u);
+            const uint4 x0 = xb[0], x1 = xb[1], x2 = xb[2];
+            const uint32_t xv[12] = {x0.x, x0.y, x0.z, x0.w, x1.x, x1.y, x1.z, x1.w, x2.x, x2.y, x2.z, x2.w};
+            float s0 = 0.f, s1 = 0.f;
 #pragma unroll
-                for (int q = 0; q < 6; ++q)
-                    mma_bf16_16816(c, w[2 * q], 0u, w[2 * q + 1], 0u, xv[2 * q], xv[2 * q + 1]);
+            for (int j = 0; j < 12; ++j) {                        // bf16 x bf16 products are exact in binary32
+                s0 = fmaf(__uint_as_float(w[j] << 16), __uint_as_float(xv[j] << 16), s0);
+                s1 = fmaf(__uint_as_float(w[j] & 0xffff0000u), __uint_as_float(xv[j] & 0xffff0000u), s1);
             }
-            if (t == 0) atomicAdd(&acc[(rg - rg0) * kPackRows + g], c[0]);
-            __syncwarp();
+            if (valid) atomicAdd(&acc[(warp & (kSortAccCopies - 1)) * (kGemvGroupsPerPass * kGemvGroupRows) + rloc], s0 + s1);
+            ch = nxt; e = e_next;
         }
         __syncthreads();
-        // row groups this CTA covers completely are final; the (at most two) split ones go through the scratch
+        if (!last) return;
+        // end of the pass: row groups this CTA covers completely are final; the split ones go through the scratch
+        auto row_sum = [&](int64_t r) {
+            float v = 0.f;
+#pragma unroll
+            for (int c = 0; c < kSortAccCopies; ++c) v += acc[c * (kGemvGroupsPerPass * kGemvGroupRows) + r];
+            return v;
+        };
         for (int64_t rg = rg0; rg <= rg1; ++rg) {
-            const bool whole = u_begin <= rg * col_tiles && (rg + 1) * col_tiles <= u_end;
-            const int64_t row = rg * kPackRows + threadIdx.x;
-            const bool mine = threadIdx.x < kPackRows && row < n_out;
+            const bool whole = u_begin <= rg * nq && (rg + 1) * nq <= u_end;
+            const int64_t row = rg * kGemvGroupRows + threadIdx.x;
+            const bool mine = threadIdx.x < kGemvGroupRows && row < n_out;
             if (whole) {
                 if (mine) {
-                    const float v = acc[(rg - rg0) * kPackRows + threadIdx.x];
+                    const float v = row_sum((rg - rg0) * kGemvGroupRows + threadIdx.x);
                     if (kOutBf16) reinterpret_cast<__nv_bfloat16*>(y)[row] = __float2bfloat16_rn(v);
                     else reinterpret_cast<float*>(y)[row] = v;
                 }
                 continue;
             }
-            if (mine) atomicAdd(scratch + row, acc[(rg - rg0) * kPackRows + threadIdx.x]);
+            if (mine) atomicAdd(scratch + row, row_sum((rg - rg0) * kGemvGroupRows + threadIdx.x));
             __threadfence();
             __syncthreads();
             if (threadIdx.x == 0) {
-                const uint32_t parts = (uint32_t)(unit_owner((rg + 1) * col_tiles - 1, U, G) - unit_owner(rg * col_tiles, U, G) + 1);
+                const uint32_t parts = (uint32_t)(unit_owner((rg + 1) * nq - 1, U, G) - unit_owner(rg * nq, U, G) + 1);
                 *last_flag = atomicAdd(counters + rg, 1u) == parts - 1u;
             }
             __syncthreads();
@@ -471,7 +500,8 @@ gemv_packed_kernel(FastArgs fa, const unsigned long long* __restrict__ packed, c
             }
             __syncthreads();
         }
-    }
+        __syncthreads();                                   // the sums are read above: the next pass may clear them only now
+    });
 }
 
 // ===========================================================================
@@ -779,7 +809,22 @@ int llvq_create(llvq_ctx** out, int m_lo, int m_hi, int device)
     size_t o_sig = up(o_p12 + 4096 * 2);
     size_t o_hk = up(o_sig + sizeof sigs);
     size_t o_hc = up(o_hk + hkeys.size() * 8);
-    size_t o_cnt = up(o_hc + hcls.size() * 4);
+    size_t o_srk = up(o_hc + hcls.size() * 4);
+    // order of the classes in the sorted GEMV layout: decoder form, then unranking steps (most first), then class
+    std::vector<uint16_t> sort_rank;
+    if (ctx->fast && ncls <= 1023) {
+        std::vector<uint32_t> order(ncls);
+        auto form_key = [&](uint32_t j) {
+            const ClassDesc& d = h.desc[j];
+            const uint32_t kind = d.parity ? 0u : ((d.w == 8 || d.w == 12 || d.w == 16) ? 1u : 2u);
+            return kind * 16u + (15u - (uint32_t)(d.nlev1 + d.nlev0));
+        };
+        for (uint32_t j = 0; j < ncls; ++j) order[j] = j;
+        std::stable_sort(order.begin(), order.end(), [&](uint32_t a, uint32_t b) { return form_key(a) < form_key(b); });
+        sort_rank.resize(ncls);
+        for (uint32_t r = 0; r < ncls; ++r) sort_rank[order[r]] = (uint16_t)r;
+    }
+    size_t o_cnt = up(o_srk + sort_rank.size() * 2);
     size_t o_scr = up(o_cnt + (size_t)(64 * kMaxScratchRows / 8) * 4);    // one counter per group of 8 rows (GEMV) / per 128-row tile (GEMM)
     size_t total = o_scr + (size_t)64 * kMaxScratchRows * 4;
     std::vector<uint8_t> blob(o_cnt, 0);
@@ -795,6 +840,7 @@ int llvq_create(llvq_ctx** out, int m_lo, int m_hi, int device)
         std::memcpy(blob.data() + o_hk, hkeys.data(), hkeys.size() * 8);
         std::memcpy(blob.data() + o_hc, hcls.data(), hcls.size() * 4);
     }
+    if (!sort_rank.empty()) std::memcpy(blob.data() + o_srk, sort_rank.data(), sort_rank.size() * 2);
     if (cudaMalloc(&ctx->d_blob, total) != cudaSuccess) { delete ctx; return LLVQ_ECUDA; }
     if (cudaMemcpy(ctx->d_blob, blob.data(), blob.size(), cudaMemcpyHostToDevice) != cudaSuccess ||
         cudaMemset(static_cast<uint8_t*>(ctx->d_blob) + o_cnt, 0, total - o_cnt) != cudaSuccess) {
@@ -813,6 +859,7 @@ int llvq_create(llvq_ctx** out, int m_lo, int m_hi, int device)
     ctx->dev.W = h.W;
     ctx->d_image = d + o_img;
     ctx->d_golay = reinterpret_cast<const uint32_t*>(d + o_gol);
+    ctx->d_sort_rank = sort_rank.empty() ? nullptr : reinterpret_cast<const uint16_t*>(d + o_srk);
     ctx->enc.pos_by_low12 = reinterpret_cast<const uint16_t*>(d + o_p12);
     ctx->enc.sig_of_value = reinterpret_cast<const uint64_t*>(d + o_sig);
     ctx->enc.hash_key = reinterpret_cast<const uint64_t*>(d + o_hk);
@@ -1032,76 +1079,67 @@ int llvq_gemv_sg(const llvq_ctx* ctx, const void* d_fields, int gain_bits, const
     return gemv_common(ctx, d_fields, nullptr, &sg, n_out, k_in, d_x_bf16, d_y, y_dtype, stream);
 }
 
-// Kernel-private packed layout (see the comment at repack_kernel).  Available for codes whose classes fit the
-// 64-bit entry: at most 512 classes of at most 2^45 points each.
-static bool packable(const llvq_ctx* ctx)
+// Sorted layout (see the comment at sort_blocks_kernel).  Available for fast-path codes whose indices fit 48 bits
+// with 2^48 - 1 left over as the "no block" marker.
+static bool sortable(const llvq_ctx* ctx, int64_t k_in)
 {
-    if (!ctx->fast || ctx->host.desc.size() > 512) return false;
-    for (const ClassInfo& c : ctx->host.info) if (c.card >> 45) return false;
-    return true;
+    if (!ctx->fast || !ctx->d_sort_rank || ctx->host.W > 48 || ctx->host.N >= (u128)kSortIndexMask) return false;
+    const int64_t nq = ((k_in + 23) / 24 + 3) / 4;
+    const size_t smem = ctx->fl.total + 16 + (size_t)nq * 48 * 4 + kSortAccCopies * kGemvGroupsPerPass * kGemvGroupRows * 4 + 16;
+    return smem <= 227 * 1024 && nq < (1ll << 24);
 }
 
-size_t llvq_packed_bytes(const llvq_ctx* ctx, int64_t n_out, int64_t k_in)
+size_t llvq_sorted_bytes(const llvq_ctx* ctx, int64_t n_out, int64_t k_in)
 {
-    if (!ctx || n_out <= 0 || k_in <= 0 || !packable(ctx)) return 0;
-    const int64_t bpr = (k_in + 23) / 24;
-    const int64_t tiles = ((n_out + kPackRows - 1) / kPackRows) * ((bpr + kPackCols - 1) / kPackCols);
-    return (size_t)tiles * kPackTile * 8;
+    if (!ctx || ctx->device < 0 || n_out <= 0 || k_in <= 0 || !sortable(ctx, k_in)) return 0;
+    const int64_t nq = ((k_in + 23) / 24 + 3) / 4;
+    return (size_t)(((n_out + kGemvGroupRows - 1) / kGemvGroupRows) * nq) * 32 * 8;
 }
 
-int llvq_repack(const llvq_ctx* ctx, const void* d_idx, int64_t n_out, int64_t k_in, void* d_packed, void* stream)
+int llvq_sort_blocks(const llvq_ctx* ctx, const void* d_idx, int64_t n_out, int64_t k_in, void* d_sorted, void* stream)
 {
     if (int e = check_common(ctx, d_idx)) return e;
-    if (!d_packed || n_out <= 0 || k_in <= 0) return LLVQ_EINVAL;
-    if (!aligned(d_packed, 16)) return LLVQ_EALIGN;
-    if (!packable(ctx)) return LLVQ_EUNSUPPORTED;
+    if (!d_sorted || n_out <= 0 || k_in <= 0) return LLVQ_EINVAL;
+    if (!aligned(d_sorted, 16)) return LLVQ_EALIGN;
+    if (!sortable(ctx, k_in) || n_out > 64ll * kMaxScratchRows) return LLVQ_EUNSUPPORTED;
     DeviceGuard guard(ctx->device);
     if (!guard.ok) return LLVQ_ECUDA;
-    const int64_t bpr = (k_in + 23) / 24, col_tiles = (bpr + kPackCols - 1) / kPackCols;
-    const int64_t ntiles = ((n_out + kPackRows - 1) / kPackRows) * col_tiles;
+    const int64_t bpr = (k_in + 23) / 24, nq = (bpr + 3) / 4;
+    const int64_t units = ((n_out + kGemvGroupRows - 1) / kGemvGroupRows) * nq;
+    const unsigned g = (unsigned)std::min<int64_t>(units, ctx->sm_count);
     const size_t smem = ctx->fl.total + 16;
-    if (!set_smem(repack_kernel, smem)) return LLVQ_ECUDA;
-    const unsigned g = (unsigned)std::min<int64_t>((ntiles + 7) / 8, ctx->sm_count);
-    repack_kernel<<<g, 256, smem, (cudaStream_t)stream>>>(fast_args(ctx), static_cast<const uint32_t*>(d_idx), n_out, bpr, col_tiles, ntiles,
-                                                         static_cast<unsigned long long*>(d_packed));
+    if (!set_smem(sort_blocks_kernel, smem)) return LLVQ_ECUDA;
+    sort_blocks_kernel<<<g, kSortThreads, smem, (cudaStream_t)stream>>>(fast_args(ctx), static_cast<const uint32_t*>(d_idx), ctx->d_sort_rank, n_out, bpr,
+                                                                       static_cast<unsigned long long*>(d_sorted));
     return launch_status();
 }
 
-int llvq_gemv_packed(const llvq_ctx* ctx, const void* d_packed, const uint16_t* d_gain_f16, int64_t n_out, int64_t k_in,
+int llvq_gemv_sorted(const llvq_ctx* ctx, const void* d_sorted, const uint16_t* d_gain_f16, int64_t n_out, int64_t k_in,
                      const uint16_t* d_x_bf16, void* d_y, int y_dtype, void* stream)
 {
     if (ctx && ctx->device >= 0 && n_out == 0) return LLVQ_OK;
-    if (int e = check_common(ctx, d_packed)) return e;
+    if (int e = check_common(ctx, d_sorted)) return e;
     if (!d_gain_f16 || !d_x_bf16 || !d_y || n_out < 0 || k_in <= 0) return LLVQ_EINVAL;
     if (y_dtype != LLVQ_F32 && y_dtype != LLVQ_BF16) return LLVQ_EINVAL;
     if (!aligned(d_gain_f16, 2) || !aligned(d_x_bf16, 2) || !aligned(d_y, y_dtype == LLVQ_F32 ? 4 : 2)) return LLVQ_EALIGN;
-    if (!packable(ctx)) return LLVQ_EUNSUPPORTED;
+    if (!sortable(ctx, k_in) || n_out > 64ll * kMaxScratchRows) return LLVQ_EUNSUPPORTED;
     DeviceGuard guard(ctx->device);
     if (!guard.ok) return LLVQ_ECUDA;
     cudaStream_t st = (cudaStream_t)stream;
-    const int64_t bpr = (k_in + 23) / 24, col_tiles = (bpr + kPackCols - 1) / kPackCols;
-    const int64_t groups = (n_out + kPackRows - 1) / kPackRows;
-    const size_t smem = ctx->fl.total + 16 + (size_t)col_tiles * kPackCols * 48 + kPackedGroups * kPackRows * 4 + 16 +
-                        (size_t)kPackedWarps * kPackTile * 24;
-    if (smem > 227 * 1024 || n_out > 64ll * kMaxScratchRows) return LLVQ_EUNSUPPORTED;
-    const unsigned g = (unsigned)std::min<int64_t>(groups * col_tiles, ctx->sm_count);
-    // warps per CTA: the count in [22, 32] that wastes the fewest warp slots on the tiles of one CTA
-    const int64_t upc = (groups * col_tiles + g - 1) / g;
-    int warps = kPackedWarps; double best_eff = 0.0;
-    for (int w = kPackedWarps; w >= 22; --w) {
-        const double eff = (double)upc / (double)(((upc + w - 1) / w) * w);
-        if (eff > best_eff + 1e-9) { best_eff = eff; warps = w; }
-    }
-    const unsigned threads = 32u * (unsigned)warps;
-    const unsigned long long* pk = static_cast<const unsigned long long*>(d_packed);
+    const int64_t bpr = (k_in + 23) / 24, nq = (bpr + 3) / 4;
+    const int64_t units = ((n_out + kGemvGroupRows - 1) / kGemvGroupRows) * nq;
+    const unsigned g = (unsigned)std::min<int64_t>(units, ctx->sm_count);
+    const size_t smem = ctx->fl.total + 16 + (size_t)nq * 48 * 4 + kSortAccCopies * kGemvGroupsPerPass * kGemvGroupRows * 4 + 16;
+    const uint32_t magic = nq == 1 ? 0xffffffffu : (uint32_t)((1ull << 32) / (uint64_t)nq);
+    const unsigned long long* sp = static_cast<const unsigned long long*>(d_sorted);
     if (y_dtype == LLVQ_BF16) {
-        if (!set_smem(gemv_packed_kernel<true>, smem)) return LLVQ_ECUDA;
-        gemv_packed_kernel<true><<<g, threads, smem, st>>>(fast_args(ctx), pk, d_gain_f16, n_out, k_in, bpr, col_tiles, d_x_bf16, d_y,
-                                                                   ctx->d_scratch, ctx->d_counters);
+        if (!set_smem(gemv_sorted_kernel<true>, smem)) return LLVQ_ECUDA;
+        gemv_sorted_kernel<true><<<g, kSortThreads, smem, st>>>(fast_args(ctx), sp, d_gain_f16, n_out, k_in, bpr, magic, d_x_bf16, d_y,
+                                                                ctx->d_scratch, ctx->d_counters);
     } else {
-        if (!set_smem(gemv_packed_kernel<false>, smem)) return LLVQ_ECUDA;
-        gemv_packed_kernel<false><<<g, threads, smem, st>>>(fast_args(ctx), pk, d_gain_f16, n_out, k_in, bpr, col_tiles, d_x_bf16, d_y,
-                                                                    ctx->d_scratch, ctx->d_counters);
+        if (!set_smem(gemv_sorted_kernel<false>, smem)) return LLVQ_ECUDA;
+        gemv_sorted_kernel<false><<<g, kSortThreads, smem, st>>>(fast_args(ctx), sp, d_gain_f16, n_out, k_in, bpr, magic, d_x_bf16, d_y,
+                                                                 ctx->d_scratch, ctx->d_counters);
     }
     return launch_status();
 }

@@ -363,67 +363,90 @@ def test_bounded_wait_reports_timeout_and_context_stays_usable(lib, ctxs, oracle
 
 
 # --------------------------------------------------------------------------
-# packed layout: repack once, then the fused GEMV on the packed stream
+# sorted layout: rearrange once, then the fused GEMV on the sorted stream
 # --------------------------------------------------------------------------
+def _sm_count():
+    return torch.cuda.get_device_properties(0).multi_processor_count
+
+
 @pytest.mark.parametrize("code,n_out,k_in", [((2, 13), 67, 4096), ((2, 13), 16, 384), ((2, 13), 129, 1000), ((2, 13), 1, 24),
-                                             ((2, 2), 256, 768), ((3, 3), 33, 4104)])
-def test_gemv_packed_small_shapes(lib, ctxs, oracle_mod, code, n_out, k_in):
+                                             ((2, 13), 3000, 96), ((2, 2), 256, 768), ((3, 3), 33, 4104)])
+def test_gemv_sorted_small_shapes(lib, ctxs, oracle_mod, code, n_out, k_in):
     o = _oracle(oracle_mod)(code)
     ctx = ctxs[code]
     stream, gain, _ = gen.make_layer(o.N, o.W, n_out, k_in, 1, seed=14)
     x = gen.normal_bf16(k_in, seed=14)
     want = o.gemv(stream, gain, n_out, k_in, x)
-    packed = lib.llvq_repack(ctx, to_dev_u8(stream), n_out, k_in)
-    assert packed.numel() == 1024 * ((n_out + 7) // 8) * (((k_in + 23) // 24 + 15) // 16)
-    y32 = lib.llvq_gemv_packed(ctx, packed, to_dev_f16(gain), n_out, k_in, to_dev_bf16(x))
-    y16 = lib.llvq_gemv_packed(ctx, packed, to_dev_f16(gain), n_out, k_in, to_dev_bf16(x), y_dtype=torch.bfloat16)
+    srt = lib.llvq_sort_blocks(ctx, to_dev_u8(stream), n_out, k_in)
+    assert srt.numel() == 256 * ((n_out + 7) // 8) * (((k_in + 23) // 24 + 3) // 4)
+    y32 = lib.llvq_gemv_sorted(ctx, srt, to_dev_f16(gain), n_out, k_in, to_dev_bf16(x))
+    y16 = lib.llvq_gemv_sorted(ctx, srt, to_dev_f16(gain), n_out, k_in, to_dev_bf16(x), y_dtype=torch.bfloat16)
     torch.cuda.synchronize()
     assert gemv_error(y32.cpu().numpy(), want) <= TOL
     assert gemv_error(y16.float().cpu().numpy(), want) <= TOL_BF16_OUT
     assert lib.llvq_last_error(ctx) == (0, 0)
 
 
-def test_repack_is_a_permutation_of_the_blocks(lib, ctxs, oracle_mod):
-    # every block of the matrix appears exactly once with its own class-local index; padding entries are marked
+def test_sort_blocks_is_a_permutation_of_the_blocks(lib, ctxs, oracle_mod):
+    # every block of the matrix appears exactly once, with its stored index unchanged, inside the range of units of
+    # the thread block that owns it; entries of one range are ordered by decoder form, unranking steps and class
     o = _oracle(oracle_mod)((2, 13))
     ctx = ctxs[(2, 13)]
-    n_out, k_in = 37, 1000                                  # 42 blocks per row: 5 x 3 tiles, ragged in both directions
-    bpr = 42
+    n_out, k_in = 523, 1000                                 # 42 blocks per row, 11 units per row group, ragged in both directions
+    bpr, nq, groups = 42, 11, 66
     stream, _, nblocks = gen.make_layer(o.N, o.W, n_out, k_in, 1, seed=15)
-    packed = lib.llvq_repack(ctx, to_dev_u8(stream), n_out, k_in)
-    torch.cuda.synchronize()
-    e = packed.cpu().numpy().view(np.uint64).reshape(-1, 128)
-    assert e.shape[0] == 15
-    offsets = [k["offset"] for k in o.classes()]
-    parity = [k["parity"] for k in o.classes()]
     idx = o.unpack(stream, nblocks)
+    idx[7] = o.N                                            # one out-of-range field
+    lo, hi = gen.indices_to_arrays(idx)
+    stream = gen.pack_indices(lo, hi, o.W)
+    srt = lib.llvq_sort_blocks(ctx, to_dev_u8(stream), n_out, k_in)
+    torch.cuda.synchronize()
+    assert lib.llvq_last_error(ctx) == (1, 0)
+    e = srt.cpu().numpy().view(np.uint64)
+    U, G = groups * nq, min(groups * nq, _sm_count())
+    assert e.size == U * 32
+    cls = o.classes()
+    offs = np.array([c["offset"] for c in cls] + [o.N], dtype=np.uint64)
+
+    def form(c):
+        k = cls[c]
+        if k["parity"]:
+            return (0, -(len(k["values"]) - 1), c)
+        g1 = sum(1 for v in k["values"] if v % 4 == 2)
+        g0 = len(k["values"]) - g1
+        return (1 if k["w"] in (8, 12, 16) else 2, -(max(g1 - 1, 0) + max(g0 - 1, 0)), c)
+
     seen = set()
-    for t in range(15):
-        rt, ct = divmod(t, 3)
-        kinds = (e[t] >> np.uint64(62)).astype(int)
-        order = [{1: 0, 0: 1, 2: 2, 3: 3}[k] for k in kinds]           # odd, even, other, padding
-        assert order == sorted(order)
-        for ent in e[t].tolist():
-            kind, pos, cls, local = ent >> 62, (ent >> 54) & 255, (ent >> 45) & 511, ent & ((1 << 45) - 1)
-            row, cb = rt * 8 + pos // 16, ct * 16 + pos % 16
-            if kind == 3:
-                assert row >= n_out or cb >= bpr
+    for cta in range(G):
+        u0, u1 = cta * U // G, (cta + 1) * U // G
+        seg = e[u0 * 32:u1 * 32]                             # a single segment and a single pass at this size
+        keys = []
+        for ent in seg.tolist():
+            I, pos = ent & ((1 << 48) - 1), ent >> 48
+            u, lane = u0 + pos // 32, pos % 32
+            rg, kq = divmod(u, nq)
+            row, cb = rg * 8 + lane // 4, kq * 4 + lane % 4
+            assert u < u1
+            if I == (1 << 48) - 1:
+                assert row >= n_out or cb >= bpr or row * bpr + cb == 7
+                keys.append((3, 0, 0))
                 continue
             b = row * bpr + cb
-            assert idx[b] == offsets[cls] + local and b not in seen
-            assert (kind == 1) == (parity[cls] == 1)
+            assert idx[b] == I and b not in seen
             seen.add(b)
-    assert len(seen) == nblocks
+            keys.append(form(int(np.searchsorted(offs, np.uint64(I), side="right")) - 1))
+        assert keys == sorted(keys)
+    assert len(seen) == nblocks - 1
 
 
 @pytest.mark.parametrize("n_out,k_in", [(4096, 4096), (11008, 4096), (4096, 11008)])
-def test_gemv_packed_full_size_layers_sampled_rows(lib, ctxs, oracle_mod, n_out, k_in):
+def test_gemv_sorted_full_size_layers_sampled_rows(lib, ctxs, oracle_mod, n_out, k_in):
     o = _oracle(oracle_mod)((2, 13))
     ctx = ctxs[(2, 13)]
     stream, gain, _ = gen.make_layer(o.N, o.W, n_out, k_in, 1, seed=0)
     x = gen.normal_bf16(k_in, seed=0)
-    packed = lib.llvq_repack(ctx, to_dev_u8(stream), n_out, k_in)
-    y = lib.llvq_gemv_packed(ctx, packed, to_dev_f16(gain), n_out, k_in, to_dev_bf16(x), y_dtype=torch.bfloat16)
+    srt = lib.llvq_sort_blocks(ctx, to_dev_u8(stream), n_out, k_in)
+    y = lib.llvq_gemv_sorted(ctx, srt, to_dev_f16(gain), n_out, k_in, to_dev_bf16(x), y_dtype=torch.bfloat16)
     y2 = lib.llvq_gemv(ctx, to_dev_u8(stream), to_dev_f16(gain), n_out, k_in, to_dev_bf16(x), y_dtype=torch.bfloat16)
     torch.cuda.synchronize()
     y = y.float().cpu().numpy()
@@ -431,13 +454,32 @@ def test_gemv_packed_full_size_layers_sampled_rows(lib, ctxs, oracle_mod, n_out,
     ref = np.array([o.gemv(stream, gain, n_out, k_in, x, rows=(r, 1))[r] for r in rows])
     scale = float(np.abs(ref).max())
     assert (np.abs(y[rows] - ref) / np.maximum(np.abs(ref), 1e-3 * scale)).max() <= TOL_BF16_OUT
-    # and all rows against the unpacked kernel (same weights, different summation order)
+    # and all rows against the kernel on the stored stream (same weights, different summation order)
     assert gemv_error(y, y2.float().cpu().numpy().astype(np.float64)) <= 2.0 ** -7
     assert lib.llvq_last_error(ctx) == (0, 0)
 
 
-def test_packed_layout_unsupported_for_the_72_bit_code(lib, ctxs):
+def test_gemv_sorted_many_row_groups_per_thread_block(lib, ctxs, oracle_mod):
+    # narrow and tall: every thread block owns more row groups than it keeps sums for at a time (several passes)
+    o = _oracle(oracle_mod)((2, 13))
+    ctx = ctxs[(2, 13)]
+    n_out, k_in = 8 * 130 * _sm_count() + 5, 48
+    stream, gain, _ = gen.make_layer(o.N, o.W, n_out, k_in, 1, seed=3)
+    x = gen.normal_bf16(k_in, seed=3)
+    srt = lib.llvq_sort_blocks(ctx, to_dev_u8(stream), n_out, k_in)
+    y = lib.llvq_gemv_sorted(ctx, srt, to_dev_f16(gain), n_out, k_in, to_dev_bf16(x))
+    y2 = lib.llvq_gemv(ctx, to_dev_u8(stream), to_dev_f16(gain), n_out, k_in, to_dev_bf16(x))
+    torch.cuda.synchronize()
+    ref = o.gemv(stream, gain, n_out, k_in, x, threads=4)                     # all rows: two blocks each
+    assert gemv_error(y.cpu().numpy(), ref) <= TOL
+    assert gemv_error(y2.cpu().numpy(), ref) <= TOL                           # the kernel on the stored stream takes several passes too
+    assert lib.llvq_last_error(ctx) == (0, 0)
+    assert lib.llvq_last_error(ctx) == (0, 0)
+
+
+def test_sorted_layout_unsupported_for_the_72_bit_code(lib, ctxs):
     ctx = ctxs[(2, 53)]
-    assert ctx._lib.llvq_packed_bytes(ctx._h, 64, 96) == 0
+    assert ctx._lib.llvq_sorted_bytes(ctx._h, 64, 96) == 0
     buf = torch.zeros(4096, dtype=torch.uint8, device="cuda")
-    assert ctx._lib.llvq_repack(ctx._h, buf.data_ptr(), 16, 96, buf.data_ptr(), None) == 3
+    assert ctx._lib.llvq_sort_blocks(ctx._h, buf.data_ptr(), 16, 96, buf.data_ptr(), None) == 3
+    assert ctx._lib.llvq_gemv_sorted(ctx._h, buf.data_ptr(), buf.data_ptr(), 16, 96, buf.data_ptr(), buf.data_ptr(), 0, None) == 3
