@@ -126,6 +126,12 @@ __device__ __forceinline__ void block_pairs_sg(const FastArgs& fa, const FastSme
     expand_bf16(d, g, w);
 }
 
+// Programmatic dependent launch: a GEMV kernel lets the next kernel of the stream start early (its thread blocks
+// move in as soon as this kernel's finish) and itself waits for the previous kernel to complete only after it has
+// loaded its table image, before it reads anything a predecessor may have written (x, the scratch, the counters).
+__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
 #define FAST_PROLOGUE()                                                                         \
     extern __shared__ __align__(128) uint8_t smem[];                                            \
     uint64_t* bar = reinterpret_cast<uint64_t*>(smem + fa.L.total);                              \
@@ -211,7 +217,9 @@ gemv_fast_kernel(FastArgs fa, const uint32_t* __restrict__ stream, const uint16_
                  int64_t n_out, int64_t k_in, int64_t bpr, const uint16_t* __restrict__ x, void* __restrict__ y,
                  float* __restrict__ scratch, uint32_t* __restrict__ counters)
 {
+    pdl_launch_dependents();
     FAST_PROLOGUE();
+    pdl_wait();
     const int64_t nq = (bpr + 3) / 4;                               // units along K
     uint32_t* xs = reinterpret_cast<uint32_t*>(staging);            // [nq * 4][12] packed bf16 pairs of x
     float* acc = reinterpret_cast<float*>(xs + nq * 48);            // [kGemvGroupsPerPass][8]
@@ -379,7 +387,9 @@ gemv_sorted_kernel(FastArgs fa, const unsigned long long* __restrict__ sorted, c
                    int64_t n_out, int64_t k_in, int64_t bpr, uint32_t nq_magic, const uint16_t* __restrict__ x, void* __restrict__ y,
                    float* __restrict__ scratch, uint32_t* __restrict__ counters)
 {
+    pdl_launch_dependents();
     FAST_PROLOGUE();
+    pdl_wait();
     const int64_t nq = (bpr + 3) / 4;
     uint32_t* xs = reinterpret_cast<uint32_t*>(staging);            // [nq * 4][12] packed bf16 pairs of x
     float* acc = reinterpret_cast<float*>(xs + nq * 48);            // [kSortAccCopies][kGemvGroupsPerPass][8]: warps spread their adds over the copies
@@ -678,6 +688,19 @@ FastArgs fast_args(const llvq_ctx* ctx)
     fa.n_points = ctx->dev.n_lo;
     fa.dc = ctx->dev;
     return fa;
+}
+
+// Launch with programmatic stream serialization allowed (see pdl_wait above).
+template <typename... KArgs, typename... Args>
+cudaError_t launch_pdl(void (*kernel)(KArgs...), unsigned grid, unsigned block, size_t smem, cudaStream_t st, Args... args)
+{
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(grid); cfg.blockDim = dim3(block); cfg.dynamicSmemBytes = smem; cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr; cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kernel, KArgs(args)...);
 }
 
 template <typename K>
@@ -1011,8 +1034,8 @@ static int gemv_common(const llvq_ctx* ctx, const void* d_idx, const uint16_t* d
 #define LLVQ_LAUNCH_GEMV(BIG, BF16, SG)                                                                            \
     do {                                                                                                           \
         if (!set_smem(gemv_fast_kernel<BIG, BF16, SG>, smem)) return LLVQ_ECUDA;                                   \
-        gemv_fast_kernel<BIG, BF16, SG><<<g, threads, smem, st>>>(fa, idx, d_gain_f16, sga, n_out, k_in, bpr, d_x_bf16, d_y, \
-                                                                  ctx->d_scratch, ctx->d_counters);                \
+        if (launch_pdl(gemv_fast_kernel<BIG, BF16, SG>, g, threads, smem, st, fa, idx, d_gain_f16, sga, n_out, k_in, bpr, d_x_bf16, d_y, \
+                       ctx->d_scratch, ctx->d_counters) != cudaSuccess) return LLVQ_ECUDA;                         \
     } while (0)
     if (sg)             { if (y_dtype == LLVQ_BF16) LLVQ_LAUNCH_GEMV(false, true, true);  else LLVQ_LAUNCH_GEMV(false, false, true); }
     else if (ctx->fast) { if (y_dtype == LLVQ_BF16) LLVQ_LAUNCH_GEMV(false, true, false); else LLVQ_LAUNCH_GEMV(false, false, false); }
@@ -1134,12 +1157,12 @@ int llvq_gemv_sorted(const llvq_ctx* ctx, const void* d_sorted, const uint16_t* 
     const unsigned long long* sp = static_cast<const unsigned long long*>(d_sorted);
     if (y_dtype == LLVQ_BF16) {
         if (!set_smem(gemv_sorted_kernel<true>, smem)) return LLVQ_ECUDA;
-        gemv_sorted_kernel<true><<<g, kSortThreads, smem, st>>>(fast_args(ctx), sp, d_gain_f16, n_out, k_in, bpr, magic, d_x_bf16, d_y,
-                                                                ctx->d_scratch, ctx->d_counters);
+        if (launch_pdl(gemv_sorted_kernel<true>, g, (unsigned)kSortThreads, smem, st, fast_args(ctx), sp, d_gain_f16, n_out, k_in, bpr, magic,
+                       d_x_bf16, d_y, ctx->d_scratch, ctx->d_counters) != cudaSuccess) return LLVQ_ECUDA;
     } else {
         if (!set_smem(gemv_sorted_kernel<false>, smem)) return LLVQ_ECUDA;
-        gemv_sorted_kernel<false><<<g, kSortThreads, smem, st>>>(fast_args(ctx), sp, d_gain_f16, n_out, k_in, bpr, magic, d_x_bf16, d_y,
-                                                                 ctx->d_scratch, ctx->d_counters);
+        if (launch_pdl(gemv_sorted_kernel<false>, g, (unsigned)kSortThreads, smem, st, fast_args(ctx), sp, d_gain_f16, n_out, k_in, bpr, magic,
+                       d_x_bf16, d_y, ctx->d_scratch, ctx->d_counters) != cudaSuccess) return LLVQ_ECUDA;
     }
     return launch_status();
 }
