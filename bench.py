@@ -445,20 +445,12 @@ def main() -> None:
     value = whole_job_value(world, step_bytes, ms_per_step)
     timed_launches = launches
 
-    # per-layer device time of the kernel (events around each launch, same rotation)
+    # per-layer device time of the kernel: events around a run of back-to-back launches of that layer, same rotation
     per_layer = []
     for li, (n, k) in enumerate(LAYERS):
-        tot = 0.0
-        reps = max(10, min(args.steps, 100))
-        for i in range(reps):
-            d_idx, d_gain, d_x, d_y = sets[i % copies][li]
-            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-            a.record()
-            P.llvq_gemv(ctx, d_idx, d_gain, n, k, d_x, d_y=d_y)
-            b.record()
-            b.synchronize()
-            tot += a.elapsed_time(b)
-        us = tot / reps * 1e3
+        fn = lambda i: P.llvq_gemv(ctx, sets[i % copies][li][0], sets[i % copies][li][1], n, k, sets[i % copies][li][2], d_y=sets[i % copies][li][3])
+        _event_us(torch, fn, 5)
+        us = _event_us(torch, fn, max(10, min(args.steps, 100)))
         by = algorithmic_bytes(n, k)
         per_layer.append({"n_out": n, "k_in": k, "us": us, "GBps": by / us / 1e3,
                           "weights_per_s": n * k / (us * 1e-6)})

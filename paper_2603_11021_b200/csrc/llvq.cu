@@ -137,7 +137,9 @@ __device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;"
     uint64_t* bar = reinterpret_cast<uint64_t*>(smem + fa.L.total);                              \
     uint8_t* staging = smem + fa.L.total + 16;                                                  \
     (void)staging;                                                                              \
+    pdl_launch_dependents();                                                                    \
     if (!fast_load_image(smem, fa.image, fa.L.total, bar, fa.flags)) return;                    \
+    pdl_wait();                                                                                 \
     const FastSmem T = fast_view(smem, fa.L);
 
 template <bool kBig>
@@ -217,9 +219,7 @@ gemv_fast_kernel(FastArgs fa, const uint32_t* __restrict__ stream, const uint16_
                  int64_t n_out, int64_t k_in, int64_t bpr, const uint16_t* __restrict__ x, void* __restrict__ y,
                  float* __restrict__ scratch, uint32_t* __restrict__ counters)
 {
-    pdl_launch_dependents();
     FAST_PROLOGUE();
-    pdl_wait();
     const int64_t nq = (bpr + 3) / 4;                               // units along K
     uint32_t* xs = reinterpret_cast<uint32_t*>(staging);            // [nq * 4][12] packed bf16 pairs of x
     float* acc = reinterpret_cast<float*>(xs + nq * 48);            // [kGemvGroupsPerPass][8]
@@ -387,9 +387,7 @@ gemv_sorted_kernel(FastArgs fa, const unsigned long long* __restrict__ sorted, c
                    int64_t n_out, int64_t k_in, int64_t bpr, uint32_t nq_magic, const uint16_t* __restrict__ x, void* __restrict__ y,
                    float* __restrict__ scratch, uint32_t* __restrict__ counters)
 {
-    pdl_launch_dependents();
     FAST_PROLOGUE();
-    pdl_wait();
     const int64_t nq = (bpr + 3) / 4;
     uint32_t* xs = reinterpret_cast<uint32_t*>(staging);            // [nq * 4][12] packed bf16 pairs of x
     float* acc = reinterpret_cast<float*>(xs + nq * 48);            // [kSortAccCopies][kGemvGroupsPerPass][8]: warps spread their adds over the copies
@@ -564,7 +562,9 @@ gemm_kernel(FastArgs fa, const uint32_t* __restrict__ stream, const uint16_t* __
     uint8_t* b_buf = a_buf + 2 * kGemmRows * kStageK * 2;                  // [2 groups] x npad * 192
     const uint32_t b_stage = (uint32_t)ga.npad * kStageK * 2;
 
+    pdl_launch_dependents();
     if (!fast_load_image(smem, fa.image, fa.L.total, bar_img, fa.flags)) return;
+    pdl_wait();
     const FastSmem T = fast_view(smem, fa.L);
     // Two groups of 512 threads fill alternate stages, each into its own buffers and its own accumulator
     // (TMEM columns [64 h, 64 h + npad)); the epilogue adds the two accumulators.
@@ -761,10 +761,10 @@ int launch_gemm(const llvq_ctx* ctx, const void* d_idx, const uint16_t* d_gain_f
     const uint32_t* idx = static_cast<const uint32_t*>(d_idx);
     if (ctx->fast) {
         if (!set_smem(gemm_kernel<false>, smem)) return LLVQ_ECUDA;
-        gemm_kernel<false><<<grid, kGemmThreads, smem, st>>>(fast_args(ctx), idx, d_gain_f16, ga);
+        if (launch_pdl(gemm_kernel<false>, grid, (unsigned)kGemmThreads, smem, st, fast_args(ctx), idx, d_gain_f16, ga) != cudaSuccess) return LLVQ_ECUDA;
     } else {
         if (!set_smem(gemm_kernel<true>, smem)) return LLVQ_ECUDA;
-        gemm_kernel<true><<<grid, kGemmThreads, smem, st>>>(fast_args(ctx), idx, d_gain_f16, ga);
+        if (launch_pdl(gemm_kernel<true>, grid, (unsigned)kGemmThreads, smem, st, fast_args(ctx), idx, d_gain_f16, ga) != cudaSuccess) return LLVQ_ECUDA;
     }
     return launch_status();
 }
@@ -961,10 +961,12 @@ int llvq_decode_blocks(const llvq_ctx* ctx, const void* d_idx, uint64_t nblocks,
     const uint32_t* idx = static_cast<const uint32_t*>(d_idx);
     if (ctx->fast) {
         if (!set_smem(decode_blocks_fast_kernel<false>, smem)) return LLVQ_ECUDA;
-        decode_blocks_fast_kernel<false><<<g, kFastThreads, smem, (cudaStream_t)stream>>>(fast_args(ctx), idx, nblocks, reinterpret_cast<uint2*>(d_points));
+        if (launch_pdl(decode_blocks_fast_kernel<false>, g, (unsigned)kFastThreads, smem, (cudaStream_t)stream, fast_args(ctx), idx, nblocks,
+                       reinterpret_cast<uint2*>(d_points)) != cudaSuccess) return LLVQ_ECUDA;
     } else {
         if (!set_smem(decode_blocks_fast_kernel<true>, smem)) return LLVQ_ECUDA;
-        decode_blocks_fast_kernel<true><<<g, kFastThreads, smem, (cudaStream_t)stream>>>(fast_args(ctx), idx, nblocks, reinterpret_cast<uint2*>(d_points));
+        if (launch_pdl(decode_blocks_fast_kernel<true>, g, (unsigned)kFastThreads, smem, (cudaStream_t)stream, fast_args(ctx), idx, nblocks,
+                       reinterpret_cast<uint2*>(d_points)) != cudaSuccess) return LLVQ_ECUDA;
     }
     return launch_status();
 }
@@ -992,10 +994,12 @@ int llvq_dequant_matrix(const llvq_ctx* ctx, const void* d_idx, const uint16_t* 
     __nv_bfloat16* w = reinterpret_cast<__nv_bfloat16*>(d_w_bf16);
     if (ctx->fast) {
         if (!set_smem(dequant_fast_kernel<false>, smem)) return LLVQ_ECUDA;
-        dequant_fast_kernel<false><<<g, kFastThreads, smem, st>>>(fast_args(ctx), idx, d_gain_f16, SgArgs{}, nblocks, rows, cols, bpr, w, ld);
+        if (launch_pdl(dequant_fast_kernel<false, false>, g, (unsigned)kFastThreads, smem, st, fast_args(ctx), idx, d_gain_f16, SgArgs{}, (uint64_t)nblocks,
+                       rows, cols, bpr, w, ld) != cudaSuccess) return LLVQ_ECUDA;
     } else {
         if (!set_smem(dequant_fast_kernel<true>, smem)) return LLVQ_ECUDA;
-        dequant_fast_kernel<true><<<g, kFastThreads, smem, st>>>(fast_args(ctx), idx, d_gain_f16, SgArgs{}, nblocks, rows, cols, bpr, w, ld);
+        if (launch_pdl(dequant_fast_kernel<true, false>, g, (unsigned)kFastThreads, smem, st, fast_args(ctx), idx, d_gain_f16, SgArgs{}, (uint64_t)nblocks,
+                       rows, cols, bpr, w, ld) != cudaSuccess) return LLVQ_ECUDA;
     }
     return launch_status();
 }
