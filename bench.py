@@ -484,23 +484,46 @@ def main() -> None:
     y_host = [torch.empty(n, dtype=torch.bfloat16).pin_memory() for n, _ in LAYERS]
     e2e_steps = max(3, min(args.steps, 20))
 
-    def e2e_step(i: int) -> None:
-        for li, (n, k) in enumerate(LAYERS):
-            h_idx, h_gain, h_x = host_sets[i % copies][li]
-            d_idx, d_gain, d_x, d_y = sets[i % copies][li]
-            d_idx.copy_(h_idx, non_blocking=True)
-            d_gain.copy_(h_gain, non_blocking=True)
-            d_x.copy_(h_x, non_blocking=True)
-            P.llvq_gemv(ctx, d_idx, d_gain, n, k, d_x, d_y=d_y)
-            y_host[li].copy_(d_y, non_blocking=True)
-        torch.cuda.current_stream().synchronize()
+    # copies run on their own stream, one step ahead of the kernels (the device buffers rotate, so the copy of
+    # step i + 1 never touches what step i reads); every step ends with the host holding that step's result
+    main_stream, copy_stream = torch.cuda.current_stream(), torch.cuda.Stream()
+    copied = [[torch.cuda.Event() for _ in LAYERS] for _ in range(copies)]
+    consumed = [[torch.cuda.Event() for _ in LAYERS] for _ in range(copies)]
+    for c in range(copies):
+        for e in consumed[c]:
+            e.record(main_stream)
 
-    for i in range(3):
-        e2e_step(i)
+    def e2e_copies(i: int) -> None:
+        with torch.cuda.stream(copy_stream):
+            for li in range(len(LAYERS)):
+                h_idx, h_gain, h_x = host_sets[i % copies][li]
+                d_idx, d_gain, d_x, _ = sets[i % copies][li]
+                copy_stream.wait_event(consumed[i % copies][li])
+                d_idx.copy_(h_idx, non_blocking=True)
+                d_gain.copy_(h_gain, non_blocking=True)
+                d_x.copy_(h_x, non_blocking=True)
+                copied[i % copies][li].record(copy_stream)
+
+    def e2e_compute(i: int) -> None:
+        for li, (n, k) in enumerate(LAYERS):
+            d_idx, d_gain, d_x, d_y = sets[i % copies][li]
+            main_stream.wait_event(copied[i % copies][li])
+            P.llvq_gemv(ctx, d_idx, d_gain, n, k, d_x, d_y=d_y)
+            consumed[i % copies][li].record(main_stream)
+            y_host[li].copy_(d_y, non_blocking=True)
+
+    def e2e_run(first: int, count: int) -> None:
+        e2e_copies(first)
+        for i in range(first, first + count):
+            if i + 1 < first + count:
+                e2e_copies(i + 1)
+            e2e_compute(i)
+            main_stream.synchronize()
+
+    e2e_run(0, 3)
     barrier()
     ev0.record()
-    for i in range(e2e_steps):
-        e2e_step(i)
+    e2e_run(3, e2e_steps)
     ev1.record()
     barrier()
     e2e_ms = max_over_ranks(ev0.elapsed_time(ev1) / e2e_steps, dist, "cuda")
