@@ -307,6 +307,18 @@ def extras(P, ctx) -> dict:
     token(0)
     torch.cuda.synchronize()
     sweep_us = _event_us(torch, token, 3)
+    # the same sweep on the sorted layout (every matrix rearranged once)
+    sorted_weights = [[P.llvq_sort_blocks(ctx, d_idx, n, k) for (n, k), (d_idx, _) in zip(shapes, layer)] for layer in sets]
+
+    def token_sorted(i):
+        for layer in range(32):
+            c = (i * 32 + layer) % 4
+            for (n, k), (_, d_gain), d_srt in zip(shapes, sets[c], sorted_weights[c]):
+                P.llvq_gemv_sorted(ctx, d_srt, d_gain, n, k, xs[k], d_y=ys[n])
+    token_sorted(0)
+    torch.cuda.synchronize()
+    sweep_sorted_us = _event_us(torch, token_sorted, 3)
+    del sorted_weights
     blocks = 32 * sum(n * ((k + 23) // 24) for n, k in shapes)
     by = blocks * (CODE_W // 8 + 2) + 32 * sum(2 * k + 2 * n for n, k in shapes)
     # --- the one shape the paper timed (App. C): (4096 x 4104) . (4104 x 1), single shell M = 3 (24-bit indices, 1 bit/weight)
@@ -359,7 +371,8 @@ def extras(P, ctx) -> dict:
     assert P.llvq_last_error(ctx) == (0, 0)
     del v_enc, p_enc, i_enc
     out["llama3_8b_linear_sweep"] = {"us_per_token": sweep_us, "tokens_per_s": 1e6 / sweep_us, "GBps": by / sweep_us / 1e3, "blocks_per_token": blocks,
-                                     "launches_per_token": 32 * len(shapes), "algorithmic_bytes": by}
+                                     "launches_per_token": 32 * len(shapes), "algorithmic_bytes": by,
+                                     "sorted_layout": {"us_per_token": sweep_sorted_us, "tokens_per_s": 1e6 / sweep_sorted_us, "GBps": by / sweep_sorted_us / 1e3}}
     return out
 
 

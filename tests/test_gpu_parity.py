@@ -483,3 +483,35 @@ def test_sorted_layout_unsupported_for_the_72_bit_code(lib, ctxs):
     buf = torch.zeros(4096, dtype=torch.uint8, device="cuda")
     assert ctx._lib.llvq_sort_blocks(ctx._h, buf.data_ptr(), 16, 96, buf.data_ptr(), None) == 3
     assert ctx._lib.llvq_gemv_sorted(ctx._h, buf.data_ptr(), buf.data_ptr(), 16, 96, buf.data_ptr(), buf.data_ptr(), 0, None) == 3
+
+
+def test_back_to_back_launches_see_the_previous_result(lib, ctxs, oracle_mod):
+    # the kernels start before their predecessor in the stream has finished (programmatic dependent launch) and must
+    # wait before reading its output: y1 = W1 x, y2 = W2 y1, y3 = W3 y2 queued without any synchronisation in between,
+    # repeated so that stale data from the previous round would show
+    o = _oracle(oracle_mod)((2, 13))
+    ctx = ctxs[(2, 13)]
+    n = 1536
+    layers = [gen.make_layer(o.N, o.W, n, n, 1, seed=40 + j)[:2] for j in range(3)]
+    dev = [(to_dev_u8(s), to_dev_f16(g)) for s, g in layers]
+    srt = [lib.llvq_sort_blocks(ctx, d[0], n, n) for d in dev]
+    ys = [torch.zeros(n, dtype=torch.bfloat16, device="cuda") for _ in range(3)]
+    for use_sorted in (False, True):
+        for rnd in range(3):
+            x = gen.normal_bf16(n, seed=50 + rnd)
+            d_x = to_dev_bf16(x)
+            cur = d_x
+            for j in range(3):
+                if use_sorted:
+                    lib.llvq_gemv_sorted(ctx, srt[j], dev[j][1], n, n, cur, d_y=ys[j])
+                else:
+                    lib.llvq_gemv(ctx, dev[j][0], dev[j][1], n, n, cur, d_y=ys[j])
+                cur = ys[j]
+            torch.cuda.synchronize()
+            ref_in = x
+            for j in range(3):
+                ref = o.gemv(layers[j][0], layers[j][1], n, n, ref_in, threads=4)
+                got = ys[j].float().cpu().numpy()
+                assert gemv_error(got, ref) <= TOL_BF16_OUT, (use_sorted, rnd, j)
+                ref_in = bf16_bits(ys[j])                    # the next layer's reference starts from what the device produced
+    assert lib.llvq_last_error(ctx) == (0, 0)
