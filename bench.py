@@ -271,7 +271,17 @@ def extras(P, ctx) -> dict:
         us = _event_us(torch, fn, 24)
         by = nb * (CODE_W // 8 + 2) + batch * k * 2 + batch * n * 2
         out[f"gemm_8192x8192_b{batch}"] = {"us": us, "GBps": by / us / 1e3, "TFLOPs": 2.0 * n * k * batch / us / 1e6, "algorithmic_bytes": by}
-    del bufs
+    # --- the same GEMM on its sorted layout (every matrix rearranged once)
+    srt = [P.llvq_sort_blocks_gemm(ctx, b[0], n, k) for b in bufs]
+    for batch in (16, 64):
+        x = dev(gen.normal_bf16((batch, k), seed=batch), np.int16).view(torch.bfloat16)
+        y = torch.empty((batch, n), dtype=torch.bfloat16, device="cuda")
+        fn = lambda i: P.llvq_gemm_small_batch_sorted(ctx, srt[i % 12], bufs[i % 12][1], n, k, x, d_y=y)
+        _event_us(torch, fn, 4)
+        us = _event_us(torch, fn, 24)
+        by = nb * (CODE_W // 8 + 2) + batch * k * 2 + batch * n * 2
+        out[f"gemm_8192x8192_b{batch}_sorted_layout"] = {"us": us, "GBps": by / us / 1e3, "TFLOPs": 2.0 * n * k * batch / us / 1e6, "algorithmic_bytes": by}
+    del bufs, srt
     # --- GEMM, 8192 x 8192 at ~3 bits/weight: 72-bit indices over shells 2..53
     ctx53 = P.Context(2, 53, device=torch.cuda.current_device())
     bufs = []

@@ -188,6 +188,21 @@ int llvq_gemm_small_batch(const llvq_ctx* ctx, const void* d_idx, const uint16_t
                           int batch, uint16_t* d_y_bf16, void* stream);
 
 /*
+ * Sorted layout for the small-batch product (same idea and same licence as llvq_sort_blocks): the blocks of every
+ * domain of 128 rows x 8 column blocks are stored ordered by decoder form, unranking steps and class, one 64-bit
+ * entry per block (stored index unchanged in the low 48 bits, position in the domain above).
+ * llvq_gemm_small_batch_sorted computes the same Y as llvq_gemm_small_batch from that stream and the unchanged
+ * ROWWISE gains; all of App. A steps 1-4 run in the kernel.  llvq_sorted_gemm_bytes() gives the stream length (8 bytes
+ * per block of the matrix padded to whole domains; 0 if unsupported: same codes as llvq_sort_blocks).
+ * d_sorted: device, 16-byte aligned.  Other arguments and limits as in llvq_gemm_small_batch.
+ */
+size_t llvq_sorted_gemm_bytes(const llvq_ctx* ctx, int64_t n_out, int64_t k_in);
+int llvq_sort_blocks_gemm(const llvq_ctx* ctx, const void* d_idx, int64_t n_out, int64_t k_in, void* d_sorted, void* stream);
+int llvq_gemm_small_batch_sorted(const llvq_ctx* ctx, const void* d_sorted, const uint16_t* d_gain_f16,
+                                 int64_t n_out, int64_t k_in, const uint16_t* d_x_bf16,
+                                 int batch, uint16_t* d_y_bf16, void* stream);
+
+/*
  * llvq_gemm_small_batch for callers that cannot allocate device memory.  (The paper has no
  * counterpart: this is a packaging variant of the call above, same arguments, same result.)
  *

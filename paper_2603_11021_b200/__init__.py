@@ -18,7 +18,7 @@ __all__ = [
     "Context", "llvq_decode_blocks", "llvq_dequant_matrix", "llvq_gemv", "llvq_gemm_small_batch", "llvq_gemm_small_batch_noalloc",
     "llvq_dequant_matrix_sg", "llvq_gemv_sg",
     "llvq_encode_blocks", "llvq_rank_blocks", "llvq_pack_fields", "LLVQ_EUCLIDEAN", "LLVQ_ANGULAR",
-    "llvq_sort_blocks", "llvq_gemv_sorted",
+    "llvq_sort_blocks", "llvq_gemv_sorted", "llvq_sort_blocks_gemm", "llvq_gemm_small_batch_sorted",
     "llvq_last_error", "LlvqError", "EXPORTS", "load_library",
     "LLVQ_LAYOUT_FLAT", "LLVQ_LAYOUT_ROWWISE", "LLVQ_F32", "LLVQ_BF16",
 ]
@@ -38,6 +38,7 @@ EXPORTS = [
     "llvq_field_bytes", "llvq_dequant_matrix_sg", "llvq_gemv_sg", "llvq_class_info", "llvq_golay_table",
     "llvq_encode_blocks", "llvq_rank_blocks", "llvq_pack_fields",
     "llvq_sorted_bytes", "llvq_sort_blocks", "llvq_gemv_sorted",
+    "llvq_sorted_gemm_bytes", "llvq_sort_blocks_gemm", "llvq_gemm_small_batch_sorted",
 ]
 
 
@@ -81,6 +82,10 @@ def load_library() -> ctypes.CDLL:
     lib.llvq_sorted_bytes.restype = ctypes.c_size_t
     lib.llvq_sort_blocks.argtypes = [vp, vp, i64, i64, vp, vp]
     lib.llvq_gemv_sorted.argtypes = [vp, vp, vp, i64, i64, vp, vp, ctypes.c_int, vp]
+    lib.llvq_sorted_gemm_bytes.argtypes = [vp, i64, i64]
+    lib.llvq_sorted_gemm_bytes.restype = ctypes.c_size_t
+    lib.llvq_sort_blocks_gemm.argtypes = [vp, vp, i64, i64, vp, vp]
+    lib.llvq_gemm_small_batch_sorted.argtypes = [vp, vp, vp, i64, i64, vp, ctypes.c_int, vp, vp]
     lib.llvq_encode_blocks.argtypes = [vp, vp, u64, ctypes.c_int, vp, vp, vp]
     lib.llvq_rank_blocks.argtypes = [vp, vp, u64, vp, vp]
     lib.llvq_pack_fields.argtypes = [vp, vp, vp, ctypes.c_int, u64, vp, vp]
@@ -293,6 +298,35 @@ def llvq_gemv_sorted(ctx: Context, d_sorted: torch.Tensor, d_gain: torch.Tensor,
     code = LLVQ_F32 if d_y.dtype == torch.float32 else LLVQ_BF16
     _check("llvq_gemv_sorted", ctx._lib.llvq_gemv_sorted(ctx._h, _dev(d_sorted, "d_sorted"), _dev(d_gain, "d_gain"), n_out, k_in,
                                                          _dev(d_x, "d_x"), _dev(d_y, "d_y"), code, _stream_ptr(stream)))
+    return d_y
+
+
+def llvq_sort_blocks_gemm(ctx: Context, d_idx: torch.Tensor, n_out: int, k_in: int, d_sorted: torch.Tensor | None = None, stream=None):
+    """Rewrite a ROWWISE index stream into the sorted layout of ``llvq_gemm_small_batch_sorted`` (done once per matrix)."""
+    nbytes = int(ctx._lib.llvq_sorted_gemm_bytes(ctx._h, n_out, k_in))
+    if nbytes == 0:
+        raise LlvqError("llvq_sorted_gemm_bytes", 3)
+    if d_sorted is None:
+        d_sorted = torch.empty(nbytes, dtype=torch.uint8, device=d_idx.device)
+    assert d_sorted.numel() * d_sorted.element_size() >= nbytes
+    assert d_idx.numel() * d_idx.element_size() >= ctx.index_bytes(n_out * ((k_in + 23) // 24))
+    _check("llvq_sort_blocks_gemm", ctx._lib.llvq_sort_blocks_gemm(ctx._h, _dev(d_idx, "d_idx"), n_out, k_in, _dev(d_sorted, "d_sorted"),
+                                                                   _stream_ptr(stream)))
+    return d_sorted
+
+
+def llvq_gemm_small_batch_sorted(ctx: Context, d_sorted: torch.Tensor, d_gain: torch.Tensor, n_out: int, k_in: int,
+                                 d_x: torch.Tensor, d_y: torch.Tensor | None = None, stream=None):
+    """Y[b, i] = sum_k X[b, k] W[i, k] from the sorted stream of ``llvq_sort_blocks_gemm``; same result as ``llvq_gemm_small_batch``."""
+    assert d_x.dtype == torch.bfloat16 and d_x.dim() == 2 and d_x.shape[1] == k_in and d_gain.dtype == torch.float16
+    batch = d_x.shape[0]
+    if d_y is None:
+        d_y = torch.empty((batch, n_out), dtype=torch.bfloat16, device=d_sorted.device)
+    assert d_y.dtype == torch.bfloat16 and d_y.numel() >= batch * n_out
+    assert d_gain.numel() >= n_out * ((k_in + 23) // 24)
+    assert d_sorted.numel() * d_sorted.element_size() >= int(ctx._lib.llvq_sorted_gemm_bytes(ctx._h, n_out, k_in))
+    _check("llvq_gemm_small_batch_sorted", ctx._lib.llvq_gemm_small_batch_sorted(
+        ctx._h, _dev(d_sorted, "d_sorted"), _dev(d_gain, "d_gain"), n_out, k_in, _dev(d_x, "d_x"), batch, _dev(d_y, "d_y"), _stream_ptr(stream)))
     return d_y
 
 

@@ -381,6 +381,34 @@ sort_blocks_kernel(FastArgs fa, const uint32_t* __restrict__ stream, const uint1
     });
 }
 
+// App. A steps 2-4 for one entry of a sorted layout: class lookup, then the unranker form the class needs.  The
+// lanes of a warp call this together; after sorting they almost always share the form (and the class).
+__device__ __forceinline__ void decode_sorted_entry(const FastArgs& fa, const FastSmem& T, uint64_t I, bool valid, Decoded& r)
+{
+    uint64_t local = 0;
+    const uint32_t cls = valid ? fast_find_class(T, I, local) : 0u;
+    const uint32_t h = T.desc[cls * kFastDescStride];
+    const uint32_t w8 = h & 0xffu;
+    const uint32_t kind = !valid ? kKindNull : ((h & (1u << 16)) ? kKindOdd : ((w8 == 8u || w8 == 12u || w8 == 16u) ? kKindEven : kKindOther));
+    Decoded d;
+    r.p0 = r.p1 = r.p2 = r.neg = r.vals_lo = r.vals_hi = 0u;
+    if (__any_sync(kFullMask, kind == kKindOdd)) {
+        const bool mine = kind == kKindOdd;
+        fast_decode_local<1>(T, mine ? cls : 0u, mine ? local : 0ull, mine, kFullMask, d);
+        if (mine) r = d;
+    }
+    if (__any_sync(kFullMask, kind == kKindEven)) {
+        const bool mine = kind == kKindEven;
+        fast_decode_local<0>(T, mine ? cls : 0u, mine ? local : 0ull, mine, kFullMask, d);
+        if (mine) r = d;
+    }
+    if (__any_sync(kFullMask, kind == kKindOther)) {
+        const bool mine = kind == kKindOther;
+        fast_decode_local<-1>(T, mine ? cls : 0u, mine ? local : 0ull, mine, kFullMask, d);
+        if (mine) r = d;
+    }
+}
+
 template <bool kOutBf16>
 __global__ void __launch_bounds__(kSortThreads, 1)
 gemv_sorted_kernel(FastArgs fa, const unsigned long long* __restrict__ sorted, const uint16_t* __restrict__ gain,
@@ -431,28 +459,8 @@ gemv_sorted_kernel(FastArgs fa, const unsigned long long* __restrict__ sorted, c
             const uint32_t rloc = (rg_off + q) * kGemvGroupRows + ((pos >> 2) & 7u);      // row inside the pass
             const uint32_t cb = kq * 4u + (pos & 3u);
             const float gn = valid ? gain_to_float(__ldg(gain + ((int64_t)rg0 * kGemvGroupRows + rloc) * bpr + cb)) : 0.f;
-            uint64_t local = 0;
-            const uint32_t cls = valid ? fast_find_class(T, I, local) : 0u;
-            const uint32_t h = T.desc[cls * kFastDescStride];
-            const uint32_t w8 = h & 0xffu;
-            const uint32_t kind = !valid ? kKindNull : ((h & (1u << 16)) ? kKindOdd : ((w8 == 8u || w8 == 12u || w8 == 16u) ? kKindEven : kKindOther));
-            Decoded d, r;
-            r.p0 = r.p1 = r.p2 = r.neg = r.vals_lo = r.vals_hi = 0u;
-            if (__any_sync(kFullMask, kind == kKindOdd)) {
-                const bool mine = kind == kKindOdd;
-                fast_decode_local<1>(T, mine ? cls : 0u, mine ? local : 0ull, mine, kFullMask, d);
-                if (mine) r = d;
-            }
-            if (__any_sync(kFullMask, kind == kKindEven)) {
-                const bool mine = kind == kKindEven;
-                fast_decode_local<0>(T, mine ? cls : 0u, mine ? local : 0ull, mine, kFullMask, d);
-                if (mine) r = d;
-            }
-            if (__any_sync(kFullMask, kind == kKindOther)) {
-                const bool mine = kind == kKindOther;
-                fast_decode_local<-1>(T, mine ? cls : 0u, mine ? local : 0ull, mine, kFullMask, d);
-                if (mine) r = d;
-            }
+            Decoded r;
+            decode_sorted_entry(fa, T, I, valid, r);
             uint32_t w[12];
             expand_bf16(r, gn, w);
             const uint4* xb = reinterpret_cast<const uint4*>(xs + cb * 12u);
@@ -655,6 +663,193 @@ gemm_kernel(FastArgs fa, const uint32_t* __restrict__ stream, const uint16_t* __
             tc_fence_before();
         }
         done[0] += has0; done[1] += has1;
+        if (ga.split > 1) {
+            __threadfence();
+            __syncthreads();
+            if (threadIdx.x == 0) *last_flag = (atomicAdd(ga.counters + rt, 1u) == (uint32_t)ga.split - 1u);
+            __syncthreads();
+            if (*last_flag) {
+                __threadfence();
+                for (int i = threadIdx.x; i < kGemmRows * ga.batch; i += kGemmThreads) {
+                    const int n = i / kGemmRows;
+                    const int64_t orow = rt * kGemmRows + (i % kGemmRows);
+                    if (orow < ga.n_out) {
+                        float* sp = ga.scratch + (int64_t)n * ga.scratch_ld + orow;
+                        reinterpret_cast<__nv_bfloat16*>(ga.y)[(int64_t)n * ga.n_out + orow] = __float2bfloat16_rn(__ldcg(sp));
+                        __stcg(sp, 0.f);
+                    }
+                }
+                if (threadIdx.x == 0) ga.counters[rt] = 0u;
+            }
+        }
+        __syncthreads();
+    }
+    if (timeout) atomicOr(fa.flags, 1u);
+    __syncthreads();
+    if (warp == 0) tmem_dealloc(tmem, kTmemCols);
+}
+
+// ===========================================================================
+// Sorted layout for the small-batch GEMM (llvq_sort_blocks_gemm / llvq_gemm_small_batch_sorted).
+// A domain is 128 rows x 8 column blocks (1024 blocks, two 96-column MMA stages); the stream holds the domains
+// row tile major, each domain's blocks ordered like the GEMV's sorted layout (decoder form, unranking steps,
+// class), one 64-bit entry per block: the stored index unchanged (48 bits) + position in the domain (row * 8 +
+// column block, 10 bits, stored in the high 16).  The kernel runs the whole CTA on one accumulator: per
+// iteration it unranks one domain (padded batch > 32) or two (warp w takes the w-th chunk of the first and the
+// (31-w)-th of the second: both are ordered from expensive to cheap, so the pairs balance), writing the bf16
+// weights straight to their place in the K-major A tiles, then one thread issues the tcgen05 MMAs of those stages.
+// ===========================================================================
+constexpr int kDomBlocks = 8;                          // column blocks per domain
+constexpr int kDomEntries = kGemmRows * kDomBlocks;    // 1024
+constexpr int kDomStages = 2;                          // 96-column MMA stages per domain
+
+__global__ void __launch_bounds__(kDomEntries, 1)
+sort_blocks_gemm_kernel(FastArgs fa, const uint32_t* __restrict__ stream, const uint16_t* __restrict__ sort_rank, int64_t n_out, int64_t bpr,
+                        int64_t ndomains, unsigned long long* __restrict__ out)
+{
+    FAST_PROLOGUE();
+    __shared__ uint32_t hist[1024], cursor[1024];
+    const int64_t nd = (bpr + kDomBlocks - 1) / kDomBlocks;
+    for (int64_t dom = blockIdx.x; dom < ndomains; dom += gridDim.x) {
+        hist[threadIdx.x] = 0; cursor[threadIdx.x] = 0;
+        __syncthreads();
+        const int64_t rt = dom / nd, d = dom - rt * nd;
+        const int i = threadIdx.x;
+        const int64_t row = rt * kGemmRows + (i >> 3), cb = d * kDomBlocks + (i & 7);
+        unsigned long long field = kSortIndexMask;
+        uint32_t key = 1023u;
+        if (row < n_out && cb < bpr) {
+            const uint64_t I = load_field(stream, (uint64_t)(row * bpr + cb), (int)fa.L.W);
+            if (I < fa.n_points) {
+                uint64_t local;
+                field = I;
+                key = __ldg(sort_rank + fast_find_class(T, I, local));
+            } else {
+                atomicAdd(fa.bad_index, 1ull);
+            }
+        }
+        atomicAdd(&hist[key], 1u);
+        __syncthreads();
+        if (threadIdx.x == 0) {
+            uint32_t run = 0;
+            for (int k = 0; k < 1024; ++k) { const uint32_t c = hist[k]; hist[k] = run; run += c; }
+        }
+        __syncthreads();
+        const uint32_t slot = hist[key] + atomicAdd(&cursor[key], 1u);
+        out[dom * kDomEntries + slot] = field | (unsigned long long)i << 48;
+        __syncthreads();
+    }
+}
+
+__global__ void __launch_bounds__(kGemmThreads, 1)
+gemm_sorted_kernel(FastArgs fa, const unsigned long long* __restrict__ sorted, const uint16_t* __restrict__ gain, GemmArgs ga, int dpi)
+{
+    extern __shared__ __align__(128) uint8_t smem[];
+    const uint32_t img_bytes = fa.L.total;
+    uint64_t* bar_img = reinterpret_cast<uint64_t*>(smem + img_bytes);
+    uint64_t* bar_free = bar_img + 1;                                     // the MMAs reading the A / B buffers are done
+    uint64_t* bar_done = bar_img + 2;                                     // the accumulator of this item is complete
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bar_img + 5);
+    uint32_t* last_flag = tmem_slot + 1;
+    const uint32_t a_off = (img_bytes + 64 + 1023) & ~1023u;
+    constexpr uint32_t kAStage = kGemmRows * kStageK * 2;                  // 24576
+    uint8_t* a_buf = smem + a_off;                                        // [dpi * 2 stages] x 24576
+    const uint32_t b_stage = (uint32_t)ga.npad * kStageK * 2;
+    uint8_t* b_buf = a_buf + (uint32_t)dpi * kDomStages * kAStage;         // [dpi * 2 stages] x npad * 192
+
+    pdl_launch_dependents();
+    if (!fast_load_image(smem, fa.image, fa.L.total, bar_img, fa.flags)) return;
+    pdl_wait();
+    const FastSmem T = fast_view(smem, fa.L);
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    if (threadIdx.x == 0) {
+        mbar_init(bar_free, 1); mbar_init(bar_done, 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 0) tmem_alloc(tmem_slot, kTmemCols);
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = *tmem_slot;
+    const uint32_t idesc = instr_desc_bf16_m128((uint32_t)ga.npad);
+    const int64_t row_tiles = (ga.n_out + kGemmRows - 1) / kGemmRows;
+    const int64_t nd = ga.nstages;                                         // domains per row tile
+    const int64_t items = row_tiles * ga.split;
+    uint32_t uses = 0, done = 0;
+    bool timeout = false;
+    for (int64_t item = blockIdx.x; item < items; item += gridDim.x) {
+        const int64_t rt = item / ga.split;
+        const int f = (int)(item % ga.split);
+        const int d_begin = (int)((int64_t)f * nd / ga.split), d_end = (int)((int64_t)(f + 1) * nd / ga.split);
+        for (int d0 = d_begin; d0 < d_end; d0 += dpi, ++uses) {
+            const int nd_now = min(dpi, d_end - d0);
+            if (uses > 0 && !mbar_wait(bar_free, (uses - 1u) & 1u)) timeout = true;   // the previous MMAs read these buffers
+            // ---- A: every warp unranks one chunk of 32 sorted entries per domain
+            for (int q = 0; q < nd_now; ++q) {
+                const int chunk = q == 0 ? warp : 31 - warp;
+                const unsigned long long e = __ldg(sorted + ((rt * nd + d0 + q) * kDomEntries + chunk * 32 + lane));
+                const uint64_t I = e & kSortIndexMask;
+                const uint32_t pos = (uint32_t)(e >> 48);
+                const bool valid = I < fa.n_points;
+                const uint32_t r = pos >> 3, c = pos & 7u;
+                const int64_t row = rt * kGemmRows + r, cb = (int64_t)(d0 + q) * kDomBlocks + c;
+                const float gn = valid ? gain_to_float(__ldg(gain + row * ga.bpr + cb)) : 0.f;
+                Decoded dec;
+                decode_sorted_entry(fa, T, I, valid, dec);
+                uint32_t w[12];
+                expand_bf16(dec, gn, w);
+                uint8_t* a_dst = a_buf + (uint32_t)(q * kDomStages + (c >> 2)) * kAStage + (r >> 3) * 128u + (r & 7u) * 16u + 3u * (c & 3u) * 2048u;
+#pragma unroll
+                for (int j = 0; j < 3; ++j)
+                    *reinterpret_cast<uint4*>(a_dst + j * 2048) = make_uint4(w[4 * j], w[4 * j + 1], w[4 * j + 2], w[4 * j + 3]);
+            }
+            // ---- B: the slice of X of these stages, 16-byte chunks (8 values along K)
+            const int kchunks = nd_now * kDomStages * (kStageK / 8);
+            for (int i = threadIdx.x; i < ga.npad * kchunks; i += kGemmThreads) {
+                const int kc = i / ga.npad, n = i % ga.npad;
+                const int64_t k = (int64_t)d0 * kDomBlocks * 24 + (int64_t)kc * 8;
+                uint4 v = make_uint4(0, 0, 0, 0);
+                if (n < ga.batch && k < ga.k_in) v = __ldg(reinterpret_cast<const uint4*>(ga.x + (int64_t)n * ga.k_in + k));
+                *reinterpret_cast<uint4*>(b_buf + (uint32_t)(kc / (kStageK / 8)) * b_stage + (uint32_t)(kc % (kStageK / 8)) * ga.npad * 16 + n * 16) = v;
+            }
+            fence_async_smem();
+            __syncthreads();
+            if (threadIdx.x == 0) {
+                tc_fence_after();
+                const uint32_t a_addr = smem_u32(a_buf), b_addr = smem_u32(b_buf);
+                for (int st = 0; st < nd_now * kDomStages; ++st)
+#pragma unroll
+                    for (int j = 0; j < kStageK / 16; ++j)
+                        umma_bf16(tmem, smem_desc(a_addr + st * kAStage + j * 4096, 2048, 128),
+                                  smem_desc(b_addr + st * b_stage + j * 2 * ga.npad * 16, ga.npad * 16, 128), idesc,
+                                  (d0 > d_begin || st > 0 || j > 0) ? 1u : 0u);
+                umma_commit(bar_free);
+                if (d0 + dpi >= d_end) umma_commit(bar_done);
+            }
+        }
+        // ---- epilogue: accumulator -> scratch (split-K) or Y
+        const bool has = d_end > d_begin;
+        if (warp < 4 && has) {
+            if (!mbar_wait(bar_done, done & 1u)) timeout = true;
+            tc_fence_after();
+            const int64_t orow = rt * kGemmRows + warp * 32 + lane;
+            for (int c0 = 0; c0 < ga.npad; c0 += 16) {
+                float v[16];
+                tmem_ld16(tmem + ((uint32_t)(warp * 32) << 16) + (uint32_t)c0, v);
+                if (orow < ga.n_out) {
+#pragma unroll
+                    for (int i = 0; i < 16; ++i) {
+                        const int n = c0 + i;
+                        if (n < ga.batch) {
+                            if (ga.split == 1) reinterpret_cast<__nv_bfloat16*>(ga.y)[(int64_t)n * ga.n_out + orow] = __float2bfloat16_rn(v[i]);
+                            else atomicAdd(ga.scratch + (int64_t)n * ga.scratch_ld + orow, v[i]);
+                        }
+                    }
+                }
+            }
+            tc_fence_before();
+        }
+        done += has;
         if (ga.split > 1) {
             __threadfence();
             __syncthreads();
@@ -1168,6 +1363,74 @@ int llvq_gemv_sorted(const llvq_ctx* ctx, const void* d_sorted, const uint16_t* 
         if (launch_pdl(gemv_sorted_kernel<false>, g, (unsigned)kSortThreads, smem, st, fast_args(ctx), sp, d_gain_f16, n_out, k_in, bpr, magic,
                        d_x_bf16, d_y, ctx->d_scratch, ctx->d_counters) != cudaSuccess) return LLVQ_ECUDA;
     }
+    return launch_status();
+}
+
+// Sorted layout of the small-batch GEMM (see the comment at sort_blocks_gemm_kernel).
+static bool gemm_sortable(const llvq_ctx* ctx)
+{
+    return ctx->fast && ctx->d_sort_rank && ctx->host.W <= 48 && ctx->host.N < (u128)kSortIndexMask;
+}
+
+size_t llvq_sorted_gemm_bytes(const llvq_ctx* ctx, int64_t n_out, int64_t k_in)
+{
+    if (!ctx || ctx->device < 0 || n_out <= 0 || k_in <= 0 || !gemm_sortable(ctx)) return 0;
+    const int64_t bpr = (k_in + 23) / 24;
+    return (size_t)(((n_out + kGemmRows - 1) / kGemmRows) * ((bpr + kDomBlocks - 1) / kDomBlocks)) * kDomEntries * 8;
+}
+
+int llvq_sort_blocks_gemm(const llvq_ctx* ctx, const void* d_idx, int64_t n_out, int64_t k_in, void* d_sorted, void* stream)
+{
+    if (int e = check_common(ctx, d_idx)) return e;
+    if (!d_sorted || n_out <= 0 || k_in <= 0) return LLVQ_EINVAL;
+    if (!aligned(d_sorted, 16)) return LLVQ_EALIGN;
+    if (!gemm_sortable(ctx)) return LLVQ_EUNSUPPORTED;
+    DeviceGuard guard(ctx->device);
+    if (!guard.ok) return LLVQ_ECUDA;
+    const int64_t bpr = (k_in + 23) / 24;
+    const int64_t ndomains = ((n_out + kGemmRows - 1) / kGemmRows) * ((bpr + kDomBlocks - 1) / kDomBlocks);
+    const size_t smem = ctx->fl.total + 16;
+    if (!set_smem(sort_blocks_gemm_kernel, smem)) return LLVQ_ECUDA;
+    const unsigned g = (unsigned)std::min<int64_t>(ndomains, 4ll * ctx->sm_count);
+    sort_blocks_gemm_kernel<<<g, kDomEntries, smem, (cudaStream_t)stream>>>(fast_args(ctx), static_cast<const uint32_t*>(d_idx), ctx->d_sort_rank,
+                                                                           n_out, bpr, ndomains, static_cast<unsigned long long*>(d_sorted));
+    return launch_status();
+}
+
+int llvq_gemm_small_batch_sorted(const llvq_ctx* ctx, const void* d_sorted, const uint16_t* d_gain_f16, int64_t n_out, int64_t k_in,
+                                 const uint16_t* d_x_bf16, int batch, uint16_t* d_y_bf16, void* stream)
+{
+    if (int e = check_gemm_args(ctx, d_sorted, d_gain_f16, n_out, k_in, d_x_bf16, batch, d_y_bf16)) return e;
+    if (n_out == 0) return LLVQ_OK;
+    if (!gemm_sortable(ctx) || n_out > kMaxScratchRows || k_in <= 0) return LLVQ_EUNSUPPORTED;
+    DeviceGuard guard(ctx->device);
+    if (!guard.ok) return LLVQ_ECUDA;
+    GemmArgs ga;
+    ga.n_out = n_out; ga.k_in = k_in; ga.bpr = (k_in + 23) / 24;
+    ga.batch = batch; ga.npad = (batch + 15) / 16 * 16;
+    ga.nstages = (int)((ga.bpr + kDomBlocks - 1) / kDomBlocks);              // domains per row tile
+    ga.x = d_x_bf16; ga.y = d_y_bf16; ga.scratch = ctx->d_scratch; ga.counters = ctx->d_counters;
+    const int dpi = ga.npad <= 32 ? 2 : 1;                                   // domains unranked per iteration (shared memory decides)
+    const int64_t row_tiles = (n_out + kGemmRows - 1) / kGemmRows;
+    ga.scratch_ld = row_tiles * kGemmRows;
+    // split K: minimise (waves of work items) x (iterations per item + the cost of an item's epilogue, about one
+    // iteration of a wide batch and half of one otherwise)
+    int best = 1; double best_cost = 1e30;
+    const double epilogue = ga.npad > 32 ? 1.0 : 0.5;
+    for (int f = 1; f <= 64 && f <= std::max(ga.nstages, 1); ++f) {
+        const int64_t waves = (row_tiles * f + ctx->sm_count - 1) / ctx->sm_count;
+        const int64_t iters = ((ga.nstages + f - 1) / f + dpi - 1) / dpi;
+        const double cost = (double)waves * ((double)iters + epilogue);
+        if (cost < best_cost - 1e-9) { best_cost = cost; best = f; }
+    }
+    ga.split = best;
+    const int64_t items = row_tiles * ga.split;
+    const unsigned grid = (unsigned)std::min<int64_t>(items, ctx->sm_count);
+    const size_t smem = ((ctx->fl.total + 64 + 1023) & ~size_t(1023)) + (size_t)dpi * kDomStages * (kGemmRows * kStageK * 2 + (size_t)ga.npad * kStageK * 2);
+    if (smem > 227 * 1024) return LLVQ_EUNSUPPORTED;
+    if (!set_smem(gemm_sorted_kernel, smem)) return LLVQ_ECUDA;
+    if (launch_pdl(gemm_sorted_kernel, grid, (unsigned)kGemmThreads, smem, (cudaStream_t)stream, fast_args(ctx),
+                   static_cast<const unsigned long long*>(d_sorted), d_gain_f16, ga, dpi) != cudaSuccess) return LLVQ_ECUDA;
     return launch_status();
 }
 

@@ -515,3 +515,88 @@ def test_back_to_back_launches_see_the_previous_result(lib, ctxs, oracle_mod):
                 assert gemv_error(got, ref) <= TOL_BF16_OUT, (use_sorted, rnd, j)
                 ref_in = bf16_bits(ys[j])                    # the next layer's reference starts from what the device produced
     assert lib.llvq_last_error(ctx) == (0, 0)
+
+
+# --------------------------------------------------------------------------
+# sorted layout of the small-batch product
+# --------------------------------------------------------------------------
+@pytest.mark.parametrize("code,n_out,k_in,batch", [((2, 13), 200, 480, 3), ((2, 13), 129, 1000, 16), ((2, 13), 1000, 2000, 33),
+                                                   ((2, 13), 64, 4096, 64), ((2, 13), 1, 24, 1), ((2, 2), 256, 768, 16),
+                                                   ((3, 3), 130, 4104, 20)])
+def test_gemm_sorted_small_shapes(lib, ctxs, oracle_mod, code, n_out, k_in, batch):
+    o = _oracle(oracle_mod)(code)
+    ctx = ctxs[code]
+    stream, gain, _ = gen.make_layer(o.N, o.W, n_out, k_in, 1, seed=24)
+    x = gen.normal_bf16((batch, k_in), seed=24)
+    want = o.gemm(stream, gain, n_out, k_in, x, threads=4)
+    srt = lib.llvq_sort_blocks_gemm(ctx, to_dev_u8(stream), n_out, k_in)
+    assert srt.numel() == 8192 * ((n_out + 127) // 128) * (((k_in + 23) // 24 + 7) // 8)
+    y = lib.llvq_gemm_small_batch_sorted(ctx, srt, to_dev_f16(gain), n_out, k_in, to_dev_bf16(x))
+    y_plain = lib.llvq_gemm_small_batch(ctx, to_dev_u8(stream), to_dev_f16(gain), n_out, k_in, to_dev_bf16(x))
+    torch.cuda.synchronize()
+    assert gemv_error(y.float().cpu().numpy(), want) <= TOL_BF16_OUT
+    assert gemv_error(y.float().cpu().numpy(), y_plain.float().cpu().numpy().astype(np.float64)) <= 2.0 ** -7
+    assert lib.llvq_last_error(ctx) == (0, 0)
+
+
+def test_sort_blocks_gemm_is_a_permutation_inside_every_domain(lib, ctxs, oracle_mod):
+    o = _oracle(oracle_mod)((2, 13))
+    ctx = ctxs[(2, 13)]
+    n_out, k_in = 300, 1000                                 # 3 row tiles (the last ragged), 42 blocks per row -> 6 domains (the last ragged)
+    bpr, nd = 42, 6
+    stream, _, nblocks = gen.make_layer(o.N, o.W, n_out, k_in, 1, seed=25)
+    idx = o.unpack(stream, nblocks)
+    e = lib.llvq_sort_blocks_gemm(ctx, to_dev_u8(stream), n_out, k_in).cpu().numpy().view(np.uint64).reshape(3 * nd, 1024)
+    offs = np.array([c["offset"] for c in o.classes()] + [o.N], dtype=np.uint64)
+    seen = set()
+    for dom in range(3 * nd):
+        rt, d = divmod(dom, nd)
+        last_parity_rank = -1
+        positions = set()
+        for ent in e[dom].tolist():
+            I, pos = ent & ((1 << 48) - 1), ent >> 48
+            row, cb = rt * 128 + pos // 8, d * 8 + pos % 8
+            assert pos < 1024 and pos not in positions
+            positions.add(pos)
+            if I == (1 << 48) - 1:
+                assert row >= n_out or cb >= bpr
+                last_parity_rank = 2
+                continue
+            b = row * bpr + cb
+            assert idx[b] == I and b not in seen
+            seen.add(b)
+            parity_rank = 0 if o.class_info(int(np.searchsorted(offs, np.uint64(I), side="right")) - 1)["parity"] else 1
+            assert parity_rank >= last_parity_rank          # odd classes first, then even, then the entries without a block
+            last_parity_rank = parity_rank
+    assert len(seen) == nblocks
+    assert lib.llvq_last_error(ctx) == (0, 0)
+
+
+@pytest.mark.parametrize("batch", [16, 64])
+def test_gemm_sorted_full_size_sampled_rows(lib, ctxs, oracle_mod, batch):
+    o = _oracle(oracle_mod)((2, 13))
+    ctx = ctxs[(2, 13)]
+    n_out, k_in = 8192, 8192
+    stream, gain, _ = gen.make_layer(o.N, o.W, n_out, k_in, 1, seed=0)
+    x = gen.normal_bf16((batch, k_in), seed=0)
+    srt = lib.llvq_sort_blocks_gemm(ctx, to_dev_u8(stream), n_out, k_in)
+    y = lib.llvq_gemm_small_batch_sorted(ctx, srt, to_dev_f16(gain), n_out, k_in, to_dev_bf16(x)).float().cpu().numpy()
+    rows = [0, 127, 128, 4095, 4096, 8191] + list(range(77, 8192, 1031))
+    ref = np.zeros((batch, len(rows)))
+    for j, r in enumerate(rows):
+        ref[:, j] = o.gemm(stream, gain, n_out, k_in, x, rows=(r, 1))[:, r]
+    assert gemv_error(y[:, rows], ref) <= TOL_BF16_OUT
+    assert lib.llvq_last_error(ctx) == (0, 0)
+
+
+def test_gemm_sorted_unsupported_and_arguments(lib, ctxs):
+    big = ctxs[(2, 53)]
+    buf = torch.zeros(8192, dtype=torch.uint8, device="cuda")
+    p = buf.data_ptr()
+    assert big._lib.llvq_sorted_gemm_bytes(big._h, 64, 96) == 0
+    assert big._lib.llvq_sort_blocks_gemm(big._h, p, 16, 96, p, None) == 3
+    assert big._lib.llvq_gemm_small_batch_sorted(big._h, p, p, 16, 96, p, 4, p, None) == 3
+    ctx = ctxs[(2, 13)]
+    assert ctx._lib.llvq_gemm_small_batch_sorted(ctx._h, p, p, 16, 96, p, 65, p, None) == 1       # batch out of range
+    assert ctx._lib.llvq_gemm_small_batch_sorted(ctx._h, p, p, 16, 100, p, 4, p, None) == 2      # k_in not a multiple of 8
+    assert ctx._lib.llvq_gemm_small_batch_sorted(ctx._h, None, None, 0, 96, None, 4, None, None) == 0
