@@ -923,6 +923,41 @@ int check_gemm_args(const llvq_ctx* ctx, const void* d_idx, const uint16_t* d_ga
     return LLVQ_OK;
 }
 
+// Enqueue gemm_sorted_kernel on a stream sorted by llvq_sort_blocks_gemm.
+int launch_gemm_domains(const llvq_ctx* ctx, const void* p, const uint16_t* d_gain_f16, int64_t n_out, int64_t k_in,
+                        const uint16_t* d_x_bf16, int batch, uint16_t* d_y_bf16, float* scratch, uint32_t* counters, void* stream)
+{
+    DeviceGuard guard(ctx->device);
+    if (!guard.ok) return LLVQ_ECUDA;
+    GemmArgs ga;
+    ga.n_out = n_out; ga.k_in = k_in; ga.bpr = (k_in + 23) / 24;
+    ga.batch = batch; ga.npad = (batch + 15) / 16 * 16;
+    ga.nstages = (int)((ga.bpr + kDomBlocks - 1) / kDomBlocks);              // domains per row tile
+    ga.x = d_x_bf16; ga.y = d_y_bf16; ga.scratch = scratch; ga.counters = counters;
+    const int dpi = ga.npad <= 32 ? 2 : 1;                                   // domains unranked per iteration (shared memory decides)
+    const int64_t row_tiles = (n_out + kGemmRows - 1) / kGemmRows;
+    ga.scratch_ld = row_tiles * kGemmRows;
+    // split K: minimise (waves of work items) x (iterations per item + the cost of an item's epilogue, about one
+    // iteration of a wide batch and half of one otherwise)
+    int best = 1; double best_cost = 1e30;
+    const double epilogue = ga.npad > 32 ? 1.0 : 0.5;
+    for (int f = 1; f <= 64 && f <= std::max(ga.nstages, 1); ++f) {
+        const int64_t waves = (row_tiles * f + ctx->sm_count - 1) / ctx->sm_count;
+        const int64_t iters = ((ga.nstages + f - 1) / f + dpi - 1) / dpi;
+        const double cost = (double)waves * ((double)iters + epilogue);
+        if (cost < best_cost - 1e-9) { best_cost = cost; best = f; }
+    }
+    ga.split = best;
+    const int64_t items = row_tiles * ga.split;
+    const unsigned grid = (unsigned)std::min<int64_t>(items, ctx->sm_count);
+    const size_t smem = ((ctx->fl.total + 64 + 1023) & ~size_t(1023)) + (size_t)dpi * kDomStages * (kGemmRows * kStageK * 2 + (size_t)ga.npad * kStageK * 2);
+    if (smem > 227 * 1024) return LLVQ_EUNSUPPORTED;
+    if (!set_smem(gemm_sorted_kernel, smem)) return LLVQ_ECUDA;
+    if (launch_pdl(gemm_sorted_kernel, grid, (unsigned)kGemmThreads, smem, (cudaStream_t)stream, fast_args(ctx),
+                   static_cast<const unsigned long long*>(p), d_gain_f16, ga, dpi) != cudaSuccess) return LLVQ_ECUDA;
+    return launch_status();
+}
+
 // Enqueue the small-batch GEMM with the given split-K scratch ([npad][row tiles * 128] floats) and counters
 // ([row tiles]); both must be zero when the kernel starts and are zero again when it ends.
 int launch_gemm(const llvq_ctx* ctx, const void* d_idx, const uint16_t* d_gain_f16, int64_t n_out, int64_t k_in,
@@ -1403,35 +1438,7 @@ int llvq_gemm_small_batch_sorted(const llvq_ctx* ctx, const void* d_sorted, cons
     if (int e = check_gemm_args(ctx, d_sorted, d_gain_f16, n_out, k_in, d_x_bf16, batch, d_y_bf16)) return e;
     if (n_out == 0) return LLVQ_OK;
     if (!gemm_sortable(ctx) || n_out > kMaxScratchRows || k_in <= 0) return LLVQ_EUNSUPPORTED;
-    DeviceGuard guard(ctx->device);
-    if (!guard.ok) return LLVQ_ECUDA;
-    GemmArgs ga;
-    ga.n_out = n_out; ga.k_in = k_in; ga.bpr = (k_in + 23) / 24;
-    ga.batch = batch; ga.npad = (batch + 15) / 16 * 16;
-    ga.nstages = (int)((ga.bpr + kDomBlocks - 1) / kDomBlocks);              // domains per row tile
-    ga.x = d_x_bf16; ga.y = d_y_bf16; ga.scratch = ctx->d_scratch; ga.counters = ctx->d_counters;
-    const int dpi = ga.npad <= 32 ? 2 : 1;                                   // domains unranked per iteration (shared memory decides)
-    const int64_t row_tiles = (n_out + kGemmRows - 1) / kGemmRows;
-    ga.scratch_ld = row_tiles * kGemmRows;
-    // split K: minimise (waves of work items) x (iterations per item + the cost of an item's epilogue, about one
-    // iteration of a wide batch and half of one otherwise)
-    int best = 1; double best_cost = 1e30;
-    const double epilogue = ga.npad > 32 ? 1.0 : 0.5;
-    for (int f = 1; f <= 64 && f <= std::max(ga.nstages, 1); ++f) {
-        const int64_t waves = (row_tiles * f + ctx->sm_count - 1) / ctx->sm_count;
-        const int64_t iters = ((ga.nstages + f - 1) / f + dpi - 1) / dpi;
-        const double cost = (double)waves * ((double)iters + epilogue);
-        if (cost < best_cost - 1e-9) { best_cost = cost; best = f; }
-    }
-    ga.split = best;
-    const int64_t items = row_tiles * ga.split;
-    const unsigned grid = (unsigned)std::min<int64_t>(items, ctx->sm_count);
-    const size_t smem = ((ctx->fl.total + 64 + 1023) & ~size_t(1023)) + (size_t)dpi * kDomStages * (kGemmRows * kStageK * 2 + (size_t)ga.npad * kStageK * 2);
-    if (smem > 227 * 1024) return LLVQ_EUNSUPPORTED;
-    if (!set_smem(gemm_sorted_kernel, smem)) return LLVQ_ECUDA;
-    if (launch_pdl(gemm_sorted_kernel, grid, (unsigned)kGemmThreads, smem, (cudaStream_t)stream, fast_args(ctx),
-                   static_cast<const unsigned long long*>(d_sorted), d_gain_f16, ga, dpi) != cudaSuccess) return LLVQ_ECUDA;
-    return launch_status();
+    return launch_gemm_domains(ctx, d_sorted, d_gain_f16, n_out, k_in, d_x_bf16, batch, d_y_bf16, ctx->d_scratch, ctx->d_counters, stream);
 }
 
 int llvq_gemm_small_batch(const llvq_ctx* ctx, const void* d_idx, const uint16_t* d_gain_f16, int64_t n_out, int64_t k_in,
