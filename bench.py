@@ -200,7 +200,7 @@ def profile_run(P, ctx, args) -> None:
     """A handful of launches of one kernel on buffers that do not fit L2 together, for profiler captures:
     gemv = the 11008x4096 layer, dequant = 4096x4096 FLAT, gemm = 8192x8192 at batch 16."""
     import torch
-    n, k = {"gemv": (11008, 4096), "gemv_sorted": (11008, 4096), "dequant": (4096, 4096), "gemm": (8192, 8192)}[args.profile]
+    n, k = {"gemv": (11008, 4096), "gemv_sorted": (11008, 4096), "dequant": (4096, 4096), "gemm": (8192, 8192), "gemm_sorted": (8192, 8192)}[args.profile]
     layout = 0 if args.profile == "dequant" else 1
     per_copy = algorithmic_bytes(n, k) + (n * k * 2 if args.profile == "dequant" else 0)
     copies = max(2, -(-2 * L2_BYTES // per_copy))
@@ -210,6 +210,8 @@ def profile_run(P, ctx, args) -> None:
         d_idx = torch.from_numpy(stream).cuda()
         if args.profile == "gemv_sorted":
             d_idx = P.llvq_sort_blocks(ctx, d_idx, n, k)
+        if args.profile == "gemm_sorted":
+            d_idx = P.llvq_sort_blocks_gemm(ctx, d_idx, n, k)
         bufs.append((d_idx, torch.from_numpy(gain.view(np.float16)).cuda()))
     x = torch.from_numpy(gen.normal_bf16((16, k), seed=0).view(np.int16)).cuda().view(torch.bfloat16)
     y = torch.empty(16 * n, dtype=torch.bfloat16, device="cuda")
@@ -220,6 +222,8 @@ def profile_run(P, ctx, args) -> None:
             P.llvq_gemv(ctx, d_idx, d_gain, n, k, x[0], d_y=y[:n])
         elif args.profile == "gemv_sorted":
             P.llvq_gemv_sorted(ctx, d_idx, d_gain, n, k, x[0], d_y=y[:n])
+        elif args.profile == "gemm_sorted":
+            P.llvq_gemm_small_batch_sorted(ctx, d_idx, d_gain, n, k, x, d_y=y.view(16, n))
         elif args.profile == "dequant":
             P.llvq_dequant_matrix(ctx, d_idx, d_gain, n, k, 0, d_w=w)
         else:
@@ -394,7 +398,7 @@ def main() -> None:
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-extras", action="store_true", help="skip the secondary configurations (dequant, GEMM, decoder sweep)")
-    ap.add_argument("--profile", default=None, choices=["gemv", "dequant", "gemm", "gemv_sorted"],
+    ap.add_argument("--profile", default=None, choices=["gemv", "dequant", "gemm", "gemv_sorted", "gemm_sorted"],
                     help="run only a few launches of one kernel over rotating buffers (for ncu captures); no timing line")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup

@@ -774,13 +774,15 @@ gemm_sorted_kernel(FastArgs fa, const unsigned long long* __restrict__ sorted, c
     const uint32_t idesc = instr_desc_bf16_m128((uint32_t)ga.npad);
     const int64_t row_tiles = (ga.n_out + kGemmRows - 1) / kGemmRows;
     const int64_t nd = ga.nstages;                                         // domains per row tile
-    const int64_t items = row_tiles * ga.split;
+    // every CTA takes an equal contiguous range of the row_tiles * nd domains (row tile major); the parts of a row
+    // tile that end up in different CTAs are summed through the scratch, as in the GEMV
+    const int64_t D = row_tiles * nd, G = gridDim.x;
+    const int64_t dom_begin = blockIdx.x * D / G, dom_end = (blockIdx.x + 1) * D / G;
     uint32_t uses = 0, done = 0;
     bool timeout = false;
-    for (int64_t item = blockIdx.x; item < items; item += gridDim.x) {
-        const int64_t rt = item / ga.split;
-        const int f = (int)(item % ga.split);
-        const int d_begin = (int)((int64_t)f * nd / ga.split), d_end = (int)((int64_t)(f + 1) * nd / ga.split);
+    for (int64_t rt = dom_begin / nd; rt * nd < dom_end; ++rt) {
+        const int d_begin = (int)(max(dom_begin, rt * nd) - rt * nd), d_end = (int)(min(dom_end, (rt + 1) * nd) - rt * nd);
+        const uint32_t parts = (uint32_t)(unit_owner((rt + 1) * nd - 1, D, G) - unit_owner(rt * nd, D, G) + 1);   // CTAs that share this row tile
         for (int d0 = d_begin; d0 < d_end; d0 += dpi, ++uses) {
             const int nd_now = min(dpi, d_end - d0);
             if (uses > 0 && !mbar_wait(bar_free, (uses - 1u) & 1u)) timeout = true;   // the previous MMAs read these buffers
@@ -841,7 +843,7 @@ gemm_sorted_kernel(FastArgs fa, const unsigned long long* __restrict__ sorted, c
                     for (int i = 0; i < 16; ++i) {
                         const int n = c0 + i;
                         if (n < ga.batch) {
-                            if (ga.split == 1) reinterpret_cast<__nv_bfloat16*>(ga.y)[(int64_t)n * ga.n_out + orow] = __float2bfloat16_rn(v[i]);
+                            if (parts == 1u) reinterpret_cast<__nv_bfloat16*>(ga.y)[(int64_t)n * ga.n_out + orow] = __float2bfloat16_rn(v[i]);
                             else atomicAdd(ga.scratch + (int64_t)n * ga.scratch_ld + orow, v[i]);
                         }
                     }
@@ -850,10 +852,10 @@ gemm_sorted_kernel(FastArgs fa, const unsigned long long* __restrict__ sorted, c
             tc_fence_before();
         }
         done += has;
-        if (ga.split > 1) {
+        if (parts > 1u) {
             __threadfence();
             __syncthreads();
-            if (threadIdx.x == 0) *last_flag = (atomicAdd(ga.counters + rt, 1u) == (uint32_t)ga.split - 1u);
+            if (threadIdx.x == 0) *last_flag = (atomicAdd(ga.counters + rt, 1u) == parts - 1u);
             __syncthreads();
             if (*last_flag) {
                 __threadfence();
@@ -937,19 +939,8 @@ int launch_gemm_domains(const llvq_ctx* ctx, const void* p, const uint16_t* d_ga
     const int dpi = ga.npad <= 32 ? 2 : 1;                                   // domains unranked per iteration (shared memory decides)
     const int64_t row_tiles = (n_out + kGemmRows - 1) / kGemmRows;
     ga.scratch_ld = row_tiles * kGemmRows;
-    // split K: minimise (waves of work items) x (iterations per item + the cost of an item's epilogue, about one
-    // iteration of a wide batch and half of one otherwise)
-    int best = 1; double best_cost = 1e30;
-    const double epilogue = ga.npad > 32 ? 1.0 : 0.5;
-    for (int f = 1; f <= 64 && f <= std::max(ga.nstages, 1); ++f) {
-        const int64_t waves = (row_tiles * f + ctx->sm_count - 1) / ctx->sm_count;
-        const int64_t iters = ((ga.nstages + f - 1) / f + dpi - 1) / dpi;
-        const double cost = (double)waves * ((double)iters + epilogue);
-        if (cost < best_cost - 1e-9) { best_cost = cost; best = f; }
-    }
-    ga.split = best;
-    const int64_t items = row_tiles * ga.split;
-    const unsigned grid = (unsigned)std::min<int64_t>(items, ctx->sm_count);
+    ga.split = 1;                                                             // unused: the kernel balances domains over the CTAs itself
+    const unsigned grid = (unsigned)std::min<int64_t>(row_tiles * ga.nstages, ctx->sm_count);
     const size_t smem = ((ctx->fl.total + 64 + 1023) & ~size_t(1023)) + (size_t)dpi * kDomStages * (kGemmRows * kStageK * 2 + (size_t)ga.npad * kStageK * 2);
     if (smem > 227 * 1024) return LLVQ_EUNSUPPORTED;
     if (!set_smem(gemm_sorted_kernel, smem)) return LLVQ_ECUDA;
