@@ -602,13 +602,14 @@ gemm_kernel(FastArgs fa, const uint32_t* __restrict__ stream, const uint16_t* __
         const int s_begin = (int)((int64_t)f * ga.nstages / ga.split), s_end = (int)((int64_t)(f + 1) * ga.nstages / ga.split);
         const int64_t row = rt * kGemmRows + gwarp * 8 + (lane & 7);
         for (int s = s_begin + group; s < s_end; s += 2, ++uses) {
-            if (uses > 0 && !mbar_wait(&bar_free[group], (uses - 1u) & 1u)) timeout = true;   // the MMAs of the previous stage read these buffers
             // ---- A: dequantize one block of 24 weights
             const int64_t cb = (int64_t)s * kStageBlocks + (lane >> 3);
             const bool in = row < ga.n_out && cb < ga.bpr;
             const uint64_t b = in ? (uint64_t)(row * ga.bpr + cb) : 0ull;
             uint32_t w[12];
             block_pairs<kBig>(fa, T, stream, gain, b, in, w);
+            // the MMAs of this group's previous stage read its buffers: wait for them only now, with the block already unranked
+            if (uses > 0 && !mbar_wait(&bar_free[group], (uses - 1u) & 1u)) timeout = true;
             uint8_t* a_dst = a_mine + gwarp * 128 + (lane & 7) * 16;
 #pragma unroll
             for (int j = 0; j < 3; ++j)
@@ -783,13 +784,21 @@ gemm_sorted_kernel(FastArgs fa, const unsigned long long* __restrict__ sorted, c
     for (int64_t rt = dom_begin / nd; rt * nd < dom_end; ++rt) {
         const int d_begin = (int)(max(dom_begin, rt * nd) - rt * nd), d_end = (int)(min(dom_end, (rt + 1) * nd) - rt * nd);
         const uint32_t parts = (uint32_t)(unit_owner((rt + 1) * nd - 1, D, G) - unit_owner(rt * nd, D, G) + 1);   // CTAs that share this row tile
+        // the entries of an iteration are requested one iteration ahead (they come from DRAM)
+        auto entry_at = [&](int d, int q) {
+            return d + q < d_end ? __ldg(sorted + ((rt * nd + d + q) * kDomEntries + (q == 0 ? warp : 31 - warp) * 32 + lane)) : kSortIndexMask;
+        };
+        unsigned long long e0 = entry_at(d_begin, 0), e1 = dpi > 1 ? entry_at(d_begin, 1) : kSortIndexMask;
         for (int d0 = d_begin; d0 < d_end; d0 += dpi, ++uses) {
             const int nd_now = min(dpi, d_end - d0);
-            if (uses > 0 && !mbar_wait(bar_free, (uses - 1u) & 1u)) timeout = true;   // the previous MMAs read these buffers
+            const unsigned long long cur0 = e0, cur1 = e1;
+            e0 = entry_at(d0 + dpi, 0);
+            if (dpi > 1) e1 = entry_at(d0 + dpi, 1);
             // ---- A: every warp unranks one chunk of 32 sorted entries per domain
-            for (int q = 0; q < nd_now; ++q) {
-                const int chunk = q == 0 ? warp : 31 - warp;
-                const unsigned long long e = __ldg(sorted + ((rt * nd + d0 + q) * kDomEntries + chunk * 32 + lane));
+#pragma unroll
+            for (int q = 0; q < 2; ++q) {
+                if (q >= nd_now) break;
+                const unsigned long long e = q == 0 ? cur0 : cur1;
                 const uint64_t I = e & kSortIndexMask;
                 const uint32_t pos = (uint32_t)(e >> 48);
                 const bool valid = I < fa.n_points;
@@ -800,6 +809,8 @@ gemm_sorted_kernel(FastArgs fa, const unsigned long long* __restrict__ sorted, c
                 decode_sorted_entry(fa, T, I, valid, dec);
                 uint32_t w[12];
                 expand_bf16(dec, gn, w);
+                // the previous MMAs read the buffers: wait for them only now, with the first chunk already unranked
+                if (q == 0 && uses > 0 && !mbar_wait(bar_free, (uses - 1u) & 1u)) timeout = true;
                 uint8_t* a_dst = a_buf + (uint32_t)(q * kDomStages + (c >> 2)) * kAStage + (r >> 3) * 128u + (r & 7u) * 16u + 3u * (c & 3u) * 2048u;
 #pragma unroll
                 for (int j = 0; j < 3; ++j)
