@@ -41,7 +41,7 @@ WORKLOAD = "configs[2]: fused dequant+GEMV batch 1 on W 4096x4096, 11008x4096, 4
 
 # dram__bytes_read.sum + dram__bytes_write.sum of one gemv_fast_kernel launch on the 11008x4096 layer, from the
 # ncu capture summarised under profiles/ (algorithmic bytes: 15 089 152)
-NCU_TRAFFIC_BYTES_11008x4096 = 15228928
+NCU_TRAFFIC_BYTES_11008x4096 = 15265024
 
 
 def layer_bytes(n_out: int, k_in: int) -> dict:
@@ -579,7 +579,7 @@ def main() -> None:
                               "ms_per_step": sorted_ms, "value": whole_job_value(world, step_bytes, sorted_ms), "unit": UNIT,
                               "speedup_over_stored_stream": ms_per_step / sorted_ms, "layers": sorted_layers},
             "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
-                         "traffic": NCU_TRAFFIC_BYTES_11008x4096, "kernel": "gemv_fast_kernel on 11008x4096",
+                         "traffic": NCU_TRAFFIC_BYTES_11008x4096, "kernel": "gemv_bin_kernel on 11008x4096",
                          "algorithmic_bytes_per_launch": dom_bytes, "peak_source": f"of {which}", "frac_of_nominal_8TBps": achieved / 8000.0},
             "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "ms_per_step": e2e_ms},
             "gpu_launches": timed_launches,

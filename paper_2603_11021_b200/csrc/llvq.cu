@@ -321,7 +321,7 @@ constexpr unsigned long long kSortIndexMask = (1ull << 48) - 1ull;
 // groups of the pass the segment belongs to (a pass covers at most kGemvGroupsPerPass row groups); first / last =
 // the segment opens / closes its pass.
 template <typename F>
-__device__ __forceinline__ void for_each_sorted_segment(int64_t U, int64_t G, int64_t nq, int64_t cta, F f)
+__device__ __forceinline__ void for_each_sorted_segment(int64_t U, int64_t G, int64_t nq, int64_t cta, F f, int seg_units = kSortSegUnits)
 {
     const int64_t u_begin = cta * U / G, u_end = (cta + 1) * U / G;
     if (u_begin >= u_end) return;
@@ -329,8 +329,8 @@ __device__ __forceinline__ void for_each_sorted_segment(int64_t U, int64_t G, in
     for (int64_t rg0 = rg_first; rg0 <= rg_last; rg0 += kGemvGroupsPerPass) {
         const int64_t rg1 = min(rg0 + kGemvGroupsPerPass - 1, rg_last);
         const int64_t p_begin = max(u_begin, rg0 * nq), p_end = min(u_end, (rg1 + 1) * nq);
-        for (int64_t tu0 = p_begin; tu0 < p_end; tu0 += kSortSegUnits)
-            f(tu0, min(tu0 + (int64_t)kSortSegUnits, p_end), rg0, rg1, tu0 == p_begin, tu0 + kSortSegUnits >= p_end);
+        for (int64_t tu0 = p_begin; tu0 < p_end; tu0 += seg_units)
+            f(tu0, min(tu0 + (int64_t)seg_units, p_end), rg0, rg1, tu0 == p_begin, tu0 + seg_units >= p_end);
     }
 }
 
@@ -383,10 +383,8 @@ sort_blocks_kernel(FastArgs fa, const uint32_t* __restrict__ stream, const uint1
 
 // App. A steps 2-4 for one entry of a sorted layout: class lookup, then the unranker form the class needs.  The
 // lanes of a warp call this together; after sorting they almost always share the form (and the class).
-__device__ __forceinline__ void decode_sorted_entry(const FastArgs& fa, const FastSmem& T, uint64_t I, bool valid, Decoded& r)
+__device__ __forceinline__ void decode_known_class(const FastSmem& T, uint32_t cls, uint64_t local, bool valid, Decoded& r)
 {
-    uint64_t local = 0;
-    const uint32_t cls = valid ? fast_find_class(T, I, local) : 0u;
     const uint32_t h = T.desc[cls * kFastDescStride];
     const uint32_t w8 = h & 0xffu;
     const uint32_t kind = !valid ? kKindNull : ((h & (1u << 16)) ? kKindOdd : ((w8 == 8u || w8 == 12u || w8 == 16u) ? kKindEven : kKindOther));
@@ -407,6 +405,13 @@ __device__ __forceinline__ void decode_sorted_entry(const FastArgs& fa, const Fa
         fast_decode_local<-1>(T, mine ? cls : 0u, mine ? local : 0ull, mine, kFullMask, d);
         if (mine) r = d;
     }
+}
+
+__device__ __forceinline__ void decode_sorted_entry(const FastArgs& fa, const FastSmem& T, uint64_t I, bool valid, Decoded& r)
+{
+    uint64_t local = 0;
+    const uint32_t cls = valid ? fast_find_class(T, I, local) : 0u;
+    decode_known_class(T, cls, local, valid, r);
 }
 
 template <bool kOutBf16>
@@ -518,6 +523,180 @@ gemv_sorted_kernel(FastArgs fa, const unsigned long long* __restrict__ sorted, c
         }
         __syncthreads();                                   // the sums are read above: the next pass may clear them only now
     });
+}
+
+// ===========================================================================
+// Fused GEMV on the stored stream with the blocks binned inside the kernel: the work split of gemv_fast_kernel, but a
+// CTA first looks up the class of every block of a segment of up to kBinSegUnits units (S1-S2), orders the
+// (class-local index, class, position) triples by the sorted layout's key with a counting sort in shared memory,
+// and then proceeds like gemv_sorted_kernel on those entries (S3-S8): a warp takes 32 consecutive entries, runs
+// the one unranker form they need and each lane forms its own dot product.
+// ===========================================================================
+constexpr int kBinSegUnits = 256;                    // 8192 blocks per segment
+constexpr int kBinPerThread = kBinSegUnits * 32 / kSortThreads;   // 8
+
+template <bool kOutBf16>
+__global__ void __launch_bounds__(kSortThreads, 1)
+gemv_bin_kernel(FastArgs fa, const uint32_t* __restrict__ stream, const uint16_t* __restrict__ sort_rank, const uint16_t* __restrict__ gain,
+                int64_t n_out, int64_t k_in, int64_t bpr, uint32_t nq_magic, const uint16_t* __restrict__ x, void* __restrict__ y,
+                float* __restrict__ scratch, uint32_t* __restrict__ counters)
+{
+    FAST_PROLOGUE();
+    const int64_t nq = (bpr + 3) / 4;
+    uint32_t* xs = reinterpret_cast<uint32_t*>(staging);            // [nq * 4][12] packed bf16 pairs of x
+    float* acc = reinterpret_cast<float*>(xs + nq * 48);            // [kSortAccCopies][kGemvGroupsPerPass][8]
+    uint32_t* last_flag = reinterpret_cast<uint32_t*>(acc + kSortAccCopies * kGemvGroupsPerPass * kGemvGroupRows);
+    uint32_t* next_chunk = last_flag + 1;
+    uint32_t* hist = last_flag + 4;                                  // [1024] bins in sort order; later their first slots
+    uint32_t* cursor = hist + 1024;                                  // [1024]
+    unsigned long long* ent = reinterpret_cast<unsigned long long*>(cursor + 1024);   // [kBinSegUnits * 32] class-local index | position << 48
+    uint16_t* ent_cls = reinterpret_cast<uint16_t*>(ent + kBinSegUnits * 32);         // [kBinSegUnits * 32] class, 0xffff = no block
+    for (int64_t i = threadIdx.x; i < nq * 48; i += blockDim.x) {
+        const int64_t e = 2 * i;
+        const uint32_t lo = e < k_in ? __ldg(x + e) : 0u, hi = e + 1 < k_in ? __ldg(x + e + 1) : 0u;
+        xs[i] = lo | hi << 16;
+    }
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const uint32_t kWarps = blockDim.x >> 5;
+    const int64_t groups = (n_out + kGemvGroupRows - 1) / kGemvGroupRows;
+    const int64_t U = groups * nq, G = gridDim.x;
+    const int64_t u_begin = blockIdx.x * U / G, u_end = (blockIdx.x + 1) * U / G;
+    const uint32_t nq32 = (uint32_t)nq;
+    for_each_sorted_segment(U, G, nq, blockIdx.x, [&](int64_t tu0, int64_t tu1, int64_t rg0, int64_t rg1, bool first, bool last) {
+        if (first)
+            for (int i = threadIdx.x; i < kSortAccCopies * kGemvGroupsPerPass * kGemvGroupRows; i += (int)blockDim.x) acc[i] = 0.f;
+        hist[threadIdx.x] = 0; cursor[threadIdx.x] = 0;
+        if (threadIdx.x == 0) *next_chunk = kWarps;
+        __syncthreads();
+        const int64_t rg_a = tu0 / nq;
+        const uint32_t kq_a = (uint32_t)(tu0 - rg_a * nq), rg_off = (uint32_t)(rg_a - rg0);
+        const int entries = (int)(tu1 - tu0) * 32;
+        // ---- S1-S2 for the whole segment and the histogram of the sort keys
+        unsigned long long mine_ent[kBinPerThread];
+        uint32_t mine_key[kBinPerThread];
+#pragma unroll
+        for (int q = 0; q < kBinPerThread; ++q) {
+            const int i = (int)threadIdx.x + q * kSortThreads;
+            mine_key[q] = 0xffffffffu; mine_ent[q] = 0ull;
+            if (i < entries) {
+                const uint32_t pos = (uint32_t)i;
+                const uint32_t v = kq_a + (pos >> 5);
+                uint32_t qd = __umulhi(v, nq_magic), kq = v - qd * nq32;
+                if (kq >= nq32) { kq -= nq32; ++qd; }
+                const int64_t row = (rg_a + qd) * kGemvGroupRows + ((pos >> 2) & 7u), cb = (int64_t)kq * 4 + (pos & 3u);
+                uint32_t key = 1023u, cls = 0xffffu;
+                uint64_t local = 0;
+                if (row < n_out && cb < bpr) {
+                    const uint64_t I = load_field(stream, (uint64_t)(row * bpr + cb), (int)fa.L.W);
+                    if (I < fa.n_points) { cls = fast_find_class(T, I, local); key = __ldg(sort_rank + cls); }
+                    else atomicAdd(fa.bad_index, 1ull);
+                }
+                mine_key[q] = key | cls << 16;
+                mine_ent[q] = local | (unsigned long long)pos << 48;
+                atomicAdd(&hist[key], 1u);
+            }
+        }
+        __syncthreads();
+        // exclusive prefix sum of the 1024 bins: one bin per thread
+        {
+            const uint32_t c = hist[threadIdx.x];
+            uint32_t incl = c;
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) { const uint32_t t = __shfl_up_sync(kFullMask, incl, o); if (lane >= o) incl += t; }
+            if (lane == 31) cursor[warp] = incl;                       // warp totals, parked in the cursor array for a moment
+            __syncthreads();
+            uint32_t before = 0;
+            for (int w2 = 0; w2 < warp; ++w2) before += cursor[w2];
+            __syncthreads();
+            hist[threadIdx.x] = before + incl - c;
+            cursor[threadIdx.x] = 0;
+        }
+        __syncthreads();
+#pragma unroll
+        for (int q = 0; q < kBinPerThread; ++q) {
+            if (mine_key[q] != 0xffffffffu) {
+                const uint32_t key = mine_key[q] & 0xffffu;
+                const uint32_t slot = hist[key] + atomicAdd(&cursor[key], 1u);
+                ent[slot] = mine_ent[q];
+                ent_cls[slot] = (uint16_t)(mine_key[q] >> 16);
+            }
+        }
+        __syncthreads();
+        // ---- S3-S8 on the ordered entries
+        const uint32_t nchunks = (uint32_t)(tu1 - tu0);
+        const uint16_t* gain_pass = gain + rg0 * kGemvGroupRows * bpr;
+        for (uint32_t ch = (uint32_t)warp; ch < nchunks;) {
+            uint32_t nxt = 0;
+            if (lane == 0) nxt = atomicAdd(next_chunk, 1u);
+            nxt = __shfl_sync(kFullMask, nxt, 0);
+            const unsigned long long e = ent[ch * 32 + lane];
+            const uint32_t cls16 = ent_cls[ch * 32 + lane];
+            const bool valid = cls16 != 0xffffu;
+            const uint32_t pos = (uint32_t)(e >> 48);
+            const uint32_t v = kq_a + (pos >> 5);
+            uint32_t q = __umulhi(v, nq_magic), kq = v - q * nq32;
+            if (kq >= nq32) { kq -= nq32; ++q; }
+            const uint32_t rloc = (rg_off + q) * kGemvGroupRows + ((pos >> 2) & 7u);
+            const uint32_t cb = kq * 4u + (pos & 3u);
+            const float gn = valid ? gain_to_float(__ldg(gain_pass + (int64_t)rloc * bpr + cb)) : 0.f;
+            Decoded r;
+            decode_known_class(T, valid ? cls16 : 0u, e & ((1ull << 48) - 1ull), valid, r);
+            uint32_t w[12];
+            expand_bf16(r, gn, w);
+            const uint4* xb = reinterpret_cast<const uint4*>(xs + cb * 12u);
+            const uint4 x0 = xb[0], x1 = xb[1], x2 = xb[2];
+            const uint32_t xv[12] = {x0.x, x0.y, x0.z, x0.w, x1.x, x1.y, x1.z, x1.w, x2.x, x2.y, x2.z, x2.w};
+            float s0 = 0.f, s1 = 0.f;
+#pragma unroll
+            for (int j = 0; j < 12; ++j) {
+                s0 = fmaf(__uint_as_float(w[j] << 16), __uint_as_float(xv[j] << 16), s0);
+                s1 = fmaf(__uint_as_float(w[j] & 0xffff0000u), __uint_as_float(xv[j] & 0xffff0000u), s1);
+            }
+            if (valid) atomicAdd(&acc[(warp & (kSortAccCopies - 1)) * (kGemvGroupsPerPass * kGemvGroupRows) + rloc], s0 + s1);
+            ch = nxt;
+        }
+        __syncthreads();
+        if (!last) return;
+        auto row_sum = [&](int64_t r) {
+            float v = 0.f;
+#pragma unroll
+            for (int c = 0; c < kSortAccCopies; ++c) v += acc[c * (kGemvGroupsPerPass * kGemvGroupRows) + r];
+            return v;
+        };
+        for (int64_t rg = rg0; rg <= rg1; ++rg) {
+            const bool whole = u_begin <= rg * nq && (rg + 1) * nq <= u_end;
+            const int64_t row = rg * kGemvGroupRows + threadIdx.x;
+            const bool mine = threadIdx.x < kGemvGroupRows && row < n_out;
+            if (whole) {
+                if (mine) {
+                    const float v = row_sum((rg - rg0) * kGemvGroupRows + threadIdx.x);
+                    if (kOutBf16) reinterpret_cast<__nv_bfloat16*>(y)[row] = __float2bfloat16_rn(v);
+                    else reinterpret_cast<float*>(y)[row] = v;
+                }
+                continue;
+            }
+            if (mine) atomicAdd(scratch + row, row_sum((rg - rg0) * kGemvGroupRows + threadIdx.x));
+            __threadfence();
+            __syncthreads();
+            if (threadIdx.x == 0) {
+                const uint32_t parts = (uint32_t)(unit_owner((rg + 1) * nq - 1, U, G) - unit_owner(rg * nq, U, G) + 1);
+                *last_flag = atomicAdd(counters + rg, 1u) == parts - 1u;
+            }
+            __syncthreads();
+            if (*last_flag) {
+                __threadfence();
+                if (mine) {
+                    const float v = __ldcg(scratch + row);
+                    if (kOutBf16) reinterpret_cast<__nv_bfloat16*>(y)[row] = __float2bfloat16_rn(v);
+                    else reinterpret_cast<float*>(y)[row] = v;
+                    __stcg(scratch + row, 0.f);
+                }
+                if (threadIdx.x == 0) counters[rg] = 0u;
+            }
+            __syncthreads();
+        }
+        __syncthreads();
+    }, kBinSegUnits);
 }
 
 // ===========================================================================
@@ -1267,6 +1446,23 @@ static int gemv_common(const llvq_ctx* ctx, const void* d_idx, const uint16_t* d
     const uint32_t* idx = static_cast<const uint32_t*>(d_idx);
     const FastArgs fa = fast_args(ctx);
     const SgArgs sga = sg ? *sg : SgArgs{};
+    // fast-path codes with many classes (mixed warps are what costs there): the kernel that bins the blocks of a segment by
+    // class before unranking them; codes with a handful of classes keep the direct kernel
+    const size_t smem_bin = ctx->fl.total + 16 + (size_t)nq * 48 * 4 + kSortAccCopies * kGemvGroupsPerPass * kGemvGroupRows * 4 + 16 +
+                            2 * 1024 * 4 + (size_t)kBinSegUnits * 32 * (8 + 2);
+    if (!sg && ctx->fast && ctx->d_sort_rank && ctx->host.desc.size() >= 64 && ctx->host.W <= 48 && smem_bin <= 227 * 1024 && nq < (1ll << 24)) {
+        const uint32_t magic = nq == 1 ? 0xffffffffu : (uint32_t)((1ull << 32) / (uint64_t)nq);
+        if (y_dtype == LLVQ_BF16) {
+            if (!set_smem(gemv_bin_kernel<true>, smem_bin)) return LLVQ_ECUDA;
+            if (launch_pdl(gemv_bin_kernel<true>, g, (unsigned)kSortThreads, smem_bin, st, fa, idx, ctx->d_sort_rank, d_gain_f16, n_out, k_in, bpr, magic,
+                           d_x_bf16, d_y, ctx->d_scratch, ctx->d_counters) != cudaSuccess) return LLVQ_ECUDA;
+        } else {
+            if (!set_smem(gemv_bin_kernel<false>, smem_bin)) return LLVQ_ECUDA;
+            if (launch_pdl(gemv_bin_kernel<false>, g, (unsigned)kSortThreads, smem_bin, st, fa, idx, ctx->d_sort_rank, d_gain_f16, n_out, k_in, bpr, magic,
+                           d_x_bf16, d_y, ctx->d_scratch, ctx->d_counters) != cudaSuccess) return LLVQ_ECUDA;
+        }
+        return launch_status();
+    }
 #define LLVQ_LAUNCH_GEMV(BIG, BF16, SG)                                                                            \
     do {                                                                                                           \
         if (!set_smem(gemv_fast_kernel<BIG, BF16, SG>, smem)) return LLVQ_ECUDA;                                   \
