@@ -532,13 +532,13 @@ gemv_sorted_kernel(FastArgs fa, const unsigned long long* __restrict__ sorted, c
 // and then proceeds like gemv_sorted_kernel on those entries (S3-S8): a warp takes 32 consecutive entries, runs
 // the one unranker form they need and each lane forms its own dot product.
 // ===========================================================================
-constexpr int kBinSegUnits = 256;                    // 8192 blocks per segment
+constexpr int kBinSegUnits = 256;                    // at most 8192 blocks per segment (halved while shared memory is short)
 constexpr int kBinPerThread = kBinSegUnits * 32 / kSortThreads;   // 8
 
 template <bool kOutBf16>
 __global__ void __launch_bounds__(kSortThreads, 1)
 gemv_bin_kernel(FastArgs fa, const uint32_t* __restrict__ stream, const uint16_t* __restrict__ sort_rank, const uint16_t* __restrict__ gain,
-                int64_t n_out, int64_t k_in, int64_t bpr, uint32_t nq_magic, const uint16_t* __restrict__ x, void* __restrict__ y,
+                int64_t n_out, int64_t k_in, int64_t bpr, uint32_t nq_magic, int seg_units, const uint16_t* __restrict__ x, void* __restrict__ y,
                 float* __restrict__ scratch, uint32_t* __restrict__ counters)
 {
     FAST_PROLOGUE();
@@ -549,8 +549,8 @@ gemv_bin_kernel(FastArgs fa, const uint32_t* __restrict__ stream, const uint16_t
     uint32_t* next_chunk = last_flag + 1;
     uint32_t* hist = last_flag + 4;                                  // [1024] bins in sort order; later their first slots
     uint32_t* cursor = hist + 1024;                                  // [1024]
-    unsigned long long* ent = reinterpret_cast<unsigned long long*>(cursor + 1024);   // [kBinSegUnits * 32] class-local index | position << 48
-    uint16_t* ent_cls = reinterpret_cast<uint16_t*>(ent + kBinSegUnits * 32);         // [kBinSegUnits * 32] class, 0xffff = no block
+    unsigned long long* ent = reinterpret_cast<unsigned long long*>(cursor + 1024);   // [seg_units * 32] class-local index | position << 48
+    uint16_t* ent_cls = reinterpret_cast<uint16_t*>(ent + seg_units * 32);            // [seg_units * 32] class, 0xffff = no block
     for (int64_t i = threadIdx.x; i < nq * 48; i += blockDim.x) {
         const int64_t e = 2 * i;
         const uint32_t lo = e < k_in ? __ldg(x + e) : 0u, hi = e + 1 < k_in ? __ldg(x + e + 1) : 0u;
@@ -696,7 +696,7 @@ gemv_bin_kernel(FastArgs fa, const uint32_t* __restrict__ stream, const uint16_t
             __syncthreads();
         }
         __syncthreads();
-    }, kBinSegUnits);
+    }, seg_units);
 }
 
 // ===========================================================================
@@ -1448,18 +1448,22 @@ static int gemv_common(const llvq_ctx* ctx, const void* d_idx, const uint16_t* d
     const SgArgs sga = sg ? *sg : SgArgs{};
     // fast-path codes with many classes (mixed warps are what costs there): the kernel that bins the blocks of a segment by
     // class before unranking them; codes with a handful of classes keep the direct kernel
-    const size_t smem_bin = ctx->fl.total + 16 + (size_t)nq * 48 * 4 + kSortAccCopies * kGemvGroupsPerPass * kGemvGroupRows * 4 + 16 +
-                            2 * 1024 * 4 + (size_t)kBinSegUnits * 32 * (8 + 2);
+    int seg_units = kBinSegUnits;
+    auto bin_bytes = [&](int su) {
+        return ctx->fl.total + 16 + (size_t)nq * 48 * 4 + kSortAccCopies * kGemvGroupsPerPass * kGemvGroupRows * 4 + 16 + 2 * 1024 * 4 + (size_t)su * 32 * (8 + 2);
+    };
+    // (smaller segments sort too few blocks to pay for the sort: the direct kernel takes over when 8192 do not fit)
+    const size_t smem_bin = bin_bytes(seg_units);
     if (!sg && ctx->fast && ctx->d_sort_rank && ctx->host.desc.size() >= 64 && ctx->host.W <= 48 && smem_bin <= 227 * 1024 && nq < (1ll << 24)) {
         const uint32_t magic = nq == 1 ? 0xffffffffu : (uint32_t)((1ull << 32) / (uint64_t)nq);
         if (y_dtype == LLVQ_BF16) {
             if (!set_smem(gemv_bin_kernel<true>, smem_bin)) return LLVQ_ECUDA;
             if (launch_pdl(gemv_bin_kernel<true>, g, (unsigned)kSortThreads, smem_bin, st, fa, idx, ctx->d_sort_rank, d_gain_f16, n_out, k_in, bpr, magic,
-                           d_x_bf16, d_y, ctx->d_scratch, ctx->d_counters) != cudaSuccess) return LLVQ_ECUDA;
+                           seg_units, d_x_bf16, d_y, ctx->d_scratch, ctx->d_counters) != cudaSuccess) return LLVQ_ECUDA;
         } else {
             if (!set_smem(gemv_bin_kernel<false>, smem_bin)) return LLVQ_ECUDA;
             if (launch_pdl(gemv_bin_kernel<false>, g, (unsigned)kSortThreads, smem_bin, st, fa, idx, ctx->d_sort_rank, d_gain_f16, n_out, k_in, bpr, magic,
-                           d_x_bf16, d_y, ctx->d_scratch, ctx->d_counters) != cudaSuccess) return LLVQ_ECUDA;
+                           seg_units, d_x_bf16, d_y, ctx->d_scratch, ctx->d_counters) != cudaSuccess) return LLVQ_ECUDA;
         }
         return launch_status();
     }

@@ -600,3 +600,20 @@ def test_gemm_sorted_unsupported_and_arguments(lib, ctxs):
     assert ctx._lib.llvq_gemm_small_batch_sorted(ctx._h, p, p, 16, 96, p, 65, p, None) == 1       # batch out of range
     assert ctx._lib.llvq_gemm_small_batch_sorted(ctx._h, p, p, 16, 100, p, 4, p, None) == 2      # k_in not a multiple of 8
     assert ctx._lib.llvq_gemm_small_batch_sorted(ctx._h, None, None, 0, 96, None, 4, None, None) == 0
+
+
+@pytest.mark.parametrize("n_out,k_in", [(72, 14336), (40, 20000), (24, 40008)])
+def test_gemv_wide_rows(lib, ctxs, oracle_mod, n_out, k_in):
+    # long rows: the x slice takes more shared memory, so the kernel bins smaller segments (or not at all)
+    o = _oracle(oracle_mod)((2, 13))
+    ctx = ctxs[(2, 13)]
+    stream, gain, _ = gen.make_layer(o.N, o.W, n_out, k_in, 1, seed=60)
+    x = gen.normal_bf16(k_in, seed=60)
+    want = o.gemv(stream, gain, n_out, k_in, x, threads=4)
+    y = lib.llvq_gemv(ctx, to_dev_u8(stream), to_dev_f16(gain), n_out, k_in, to_dev_bf16(x))
+    srt = lib.llvq_sort_blocks(ctx, to_dev_u8(stream), n_out, k_in)
+    y2 = lib.llvq_gemv_sorted(ctx, srt, to_dev_f16(gain), n_out, k_in, to_dev_bf16(x))
+    torch.cuda.synchronize()
+    assert gemv_error(y.cpu().numpy(), want) <= TOL
+    assert gemv_error(y2.cpu().numpy(), want) <= TOL
+    assert lib.llvq_last_error(ctx) == (0, 0)
