@@ -11,6 +11,11 @@
  *     never allocates, frees or retains them.  `stream` is a cudaStream_t
  *     passed as void* (NULL = default stream).  Work is enqueued on that
  *     stream and the call returns without synchronising, unless stated.
+ *   - The compute entry points only enqueue kernels (llvq_gemm_small_batch_noalloc also one memset) and
+ *     synchronise nothing, so a sequence of them can be captured into a CUDA graph once each kernel has been
+ *     launched at least once outside a capture.  The kernels use programmatic dependent launch: in a stream (or
+ *     graph) of them, a kernel's table load overlaps its predecessor's tail; it waits for the predecessor to
+ *     finish before it reads any argument buffer.
  *   - Every function returns a status code (LLVQ_OK = 0).  Bad arguments are
  *     rejected on the host before anything is launched.  Nothing throws,
  *     aborts or traps.

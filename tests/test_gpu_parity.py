@@ -617,3 +617,42 @@ def test_gemv_wide_rows(lib, ctxs, oracle_mod, n_out, k_in):
     assert gemv_error(y.cpu().numpy(), want) <= TOL
     assert gemv_error(y2.cpu().numpy(), want) <= TOL
     assert lib.llvq_last_error(ctx) == (0, 0)
+
+
+def test_chain_of_launches_replays_from_a_cuda_graph(lib, ctxs, oracle_mod):
+    # the entry points only enqueue kernels: a three-layer chain captured once into a CUDA graph gives, on every replay
+    # with new activations, what the directly launched chain gives
+    o = _oracle(oracle_mod)((2, 13))
+    ctx = ctxs[(2, 13)]
+    n = 1536
+    layers = [gen.make_layer(o.N, o.W, n, n, 1, seed=70 + j)[:2] for j in range(3)]
+    dev = [(to_dev_u8(s), to_dev_f16(g)) for s, g in layers]
+    x = torch.zeros(n, dtype=torch.bfloat16, device="cuda")
+    ys = [torch.zeros(n, dtype=torch.bfloat16, device="cuda") for _ in range(3)]
+
+    def chain():
+        cur = x
+        for j in range(3):
+            lib.llvq_gemv(ctx, dev[j][0], dev[j][1], n, n, cur, d_y=ys[j])
+            cur = ys[j]
+
+    side = torch.cuda.Stream()
+    with torch.cuda.stream(side):
+        chain()                                              # first use of the kernels outside the capture
+    side.synchronize()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph, stream=side):
+        chain()
+    for rnd in range(3):
+        xin = gen.normal_bf16(n, seed=80 + rnd)
+        x.copy_(to_dev_bf16(xin))
+        graph.replay()
+        torch.cuda.synchronize()
+        got = ys[2].float().cpu().numpy()
+        ref_in = xin
+        for j in range(3):
+            ref = o.gemv(layers[j][0], layers[j][1], n, n, ref_in, threads=4)
+            if j == 2:
+                assert gemv_error(got, ref) <= TOL_BF16_OUT, rnd
+            ref_in = bf16_bits(ys[j])
+    assert lib.llvq_last_error(ctx) == (0, 0)
