@@ -208,3 +208,24 @@ def test_gaussian_source_distortion_end_to_end(lib, ctxs):
         assert float((rec - beta * rec0).abs().max()) < 0.02          # the dequantizer reconstructs what was encoded (bf16 rounding)
     for c in ctxs.values():
         assert lib.llvq_last_error(c) == (0, 0)
+
+
+@pytest.mark.parametrize("code", [(2, 6), (2, 16), (2, 20), (2, 24)])
+def test_other_ball_cuts_decode_and_rank(lib, oracle_mod, code):
+    # cuts the benchmarks do not use: 36-, 52-, 56- and 59-bit indices; the last three keep their class tables in global memory
+    ctx = lib.Context(*code, device=0)
+    o = oracle_mod.Code(*code)
+    assert (ctx.index_bits, ctx.num_points, ctx.num_classes) == (o.W, o.N, o.num_classes)
+    n = 6000
+    lo, hi = gen.random_indices(o.N, o.W, n, seed=5)
+    cls = o.classes()
+    edges = [c["offset"] for c in cls[::17]] + [c["offset"] + c["card"] - 1 for c in cls[::17]]
+    lo = np.concatenate([lo, np.array(edges, dtype=np.uint64)])
+    hi = np.zeros_like(lo)
+    pts = lib.llvq_decode_blocks(ctx, to_dev_u8(gen.pack_indices(lo, hi, o.W)), len(lo))
+    assert np.array_equal(pts.cpu().numpy(), o.unrank_arrays(lo, hi))
+    assert np.array_equal(_idx_np(lib.llvq_rank_blocks(ctx, pts)), lo)
+    v = torch.randn((500, 24), device="cuda") * 2.5
+    p, i = lib.llvq_encode_blocks(ctx, v, lib.LLVQ_EUCLIDEAN)
+    assert torch.equal(lib.llvq_decode_blocks(ctx, lib.llvq_pack_fields(ctx, i), 500), p)
+    assert lib.llvq_last_error(ctx) == (0, 0)
