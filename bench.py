@@ -590,7 +590,10 @@ def main() -> None:
                               "speedup_over_stored_stream": ms_per_step / sorted_ms, "layers": sorted_layers},
             "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
                          "traffic": NCU_TRAFFIC_BYTES_11008x4096, "kernel": "gemv_bin_kernel on 11008x4096",
-                         "algorithmic_bytes_per_launch": dom_bytes, "peak_source": f"of {which}", "frac_of_nominal_8TBps": achieved / 8000.0},
+                         "algorithmic_bytes_per_launch": dom_bytes, "peak_source": f"of {which}", "frac_of_nominal_8TBps": achieved / 8000.0,
+                         # what binds the kernel instead of HBM: counters of the ncu capture summarised under profiles/
+                         "ncu": {"warp_instructions_per_block": 963, "issue_slots_used": 0.626, "alu_pipe_busy": 0.578,
+                                 "shared_memory_wavefronts_per_block": 210, "instructions_per_block_at_hbm_roofline": 46}},
             "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "ms_per_step": e2e_ms},
             "gpu_launches": timed_launches,
             "clocks": clocks.summary(),
