@@ -132,6 +132,14 @@ __device__ __forceinline__ void block_pairs_sg(const FastArgs& fa, const FastSme
 __device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 __device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 
+// Ask for the 128-byte lines of [p + first, p + last) in L2; the whole CTA calls this.
+__device__ __forceinline__ void prefetch_span_l2(const void* p, uint64_t first, uint64_t last)
+{
+    const uint8_t* base = static_cast<const uint8_t*>(p);
+    for (uint64_t o = (first & ~127ull) + (uint64_t)threadIdx.x * 128; o < last; o += (uint64_t)blockDim.x * 128)
+        asm volatile("prefetch.global.L2 [%0];" ::"l"(base + o));
+}
+
 #define FAST_PROLOGUE()                                                                         \
     extern __shared__ __align__(128) uint8_t smem[];                                            \
     uint64_t* bar = reinterpret_cast<uint64_t*>(smem + fa.L.total);                              \
@@ -437,6 +445,7 @@ gemv_sorted_kernel(FastArgs fa, const unsigned long long* __restrict__ sorted, c
     const int64_t U = groups * nq, G = gridDim.x;
     const int64_t u_begin = blockIdx.x * U / G, u_end = (blockIdx.x + 1) * U / G;
     const uint32_t nq32 = (uint32_t)nq;
+
     for_each_sorted_segment(U, G, nq, blockIdx.x, [&](int64_t tu0, int64_t tu1, int64_t rg0, int64_t rg1, bool first, bool last) {
         if (first)
             for (int i = threadIdx.x; i < kSortAccCopies * kGemvGroupsPerPass * kGemvGroupRows; i += (int)blockDim.x) acc[i] = 0.f;
@@ -562,6 +571,14 @@ gemv_bin_kernel(FastArgs fa, const uint32_t* __restrict__ stream, const uint16_t
     const int64_t U = groups * nq, G = gridDim.x;
     const int64_t u_begin = blockIdx.x * U / G, u_end = (blockIdx.x + 1) * U / G;
     const uint32_t nq32 = (uint32_t)nq;
+    if (u_begin < u_end) {
+        // the rows of the row groups this CTA touches are one contiguous span of the index stream and of the gains:
+        // request it from DRAM now, the binning phases then read it from L2
+        const uint64_t b_first = (uint64_t)(u_begin / nq) * kGemvGroupRows * (uint64_t)bpr;
+        const uint64_t b_last = (uint64_t)min(((u_end - 1) / nq + 1) * kGemvGroupRows, n_out) * (uint64_t)bpr;
+        prefetch_span_l2(stream, b_first * fa.L.W / 8, (b_last * fa.L.W + 7) / 8);
+        prefetch_span_l2(gain, b_first * 2, b_last * 2);
+    }
     for_each_sorted_segment(U, G, nq, blockIdx.x, [&](int64_t tu0, int64_t tu1, int64_t rg0, int64_t rg1, bool first, bool last) {
         if (first)
             for (int i = threadIdx.x; i < kSortAccCopies * kGemvGroupsPerPass * kGemvGroupRows; i += (int)blockDim.x) acc[i] = 0.f;
