@@ -377,8 +377,14 @@ def extras(P, ctx) -> dict:
     by12 = nb12 * 6 + 4 * n + 2 * k + 2 * n
     out["gemv_shape_gain_47p1_11008x4096"] = {"us": us12, "GBps": by12 / us12 / 1e3, "algorithmic_bytes": by12,
                                               "bits_per_weight": 48 * nb12 / (n * k)}
+    srt12 = [P.llvq_sort_blocks_sg(ctx12, b, 1, n, k) for b in bufs12]
+    fn = lambda i: P.llvq_gemv_sorted_sg(ctx12, srt12[i % 20], 1, d_cb, d_rs, n, k, x12, d_y=y12)
+    _event_us(torch, fn, 8)
+    us12s = _event_us(torch, fn, 60)
+    out["gemv_shape_gain_47p1_11008x4096"]["sorted_layout_us"] = us12s
+    out["gemv_shape_gain_47p1_11008x4096"]["sorted_layout_GBps"] = by12 / us12s / 1e3
     assert P.llvq_last_error(ctx12) == (0, 0)
-    del bufs12, ctx12
+    del bufs12, srt12, ctx12
     # --- encoder: nearest-point search + indexing of a 4096 x 4096 matrix worth of Gaussian blocks (offline step)
     nb_enc = 4096 * 4096 // 24
     torch.manual_seed(0)

@@ -180,6 +180,16 @@ int llvq_sort_blocks(const llvq_ctx* ctx, const void* d_idx, int64_t n_out, int6
 int llvq_gemv_sorted(const llvq_ctx* ctx, const void* d_sorted, const uint16_t* d_gain_f16,
                      int64_t n_out, int64_t k_in, const uint16_t* d_x_bf16,
                      void* d_y, int y_dtype, void* stream);
+/*
+ * The same for the shape-gain form: llvq_sort_blocks_sg sorts a stream of fields of llvq_index_bits(ctx) + gain_bits
+ * bits (at most 48 in all: the entry keeps the whole field, shape index and gain index), llvq_gemv_sorted_sg computes
+ * the y of llvq_gemv_sg from it.  Same size (llvq_sorted_bytes) and the same restrictions as above.
+ */
+int llvq_sort_blocks_sg(const llvq_ctx* ctx, const void* d_fields, int gain_bits, int64_t n_out, int64_t k_in,
+                        void* d_sorted, void* stream);
+int llvq_gemv_sorted_sg(const llvq_ctx* ctx, const void* d_sorted, int gain_bits, const float* d_codebook_f32,
+                        const float* d_row_scale_f32, int64_t n_out, int64_t k_in, const uint16_t* d_x_bf16,
+                        void* d_y, int y_dtype, void* stream);
 
 /*
  * The same product for a small batch, Y[b][i] = sum_k X[b][k] W[i][k]

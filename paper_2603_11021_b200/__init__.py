@@ -19,6 +19,7 @@ __all__ = [
     "llvq_dequant_matrix_sg", "llvq_gemv_sg",
     "llvq_encode_blocks", "llvq_rank_blocks", "llvq_pack_fields", "LLVQ_EUCLIDEAN", "LLVQ_ANGULAR",
     "llvq_sort_blocks", "llvq_gemv_sorted", "llvq_sort_blocks_gemm", "llvq_gemm_small_batch_sorted",
+    "llvq_sort_blocks_sg", "llvq_gemv_sorted_sg",
     "llvq_last_error", "LlvqError", "EXPORTS", "load_library",
     "LLVQ_LAYOUT_FLAT", "LLVQ_LAYOUT_ROWWISE", "LLVQ_F32", "LLVQ_BF16",
 ]
@@ -37,7 +38,7 @@ EXPORTS = [
     "llvq_selftest_wait_timeout", "llvq_last_error",
     "llvq_field_bytes", "llvq_dequant_matrix_sg", "llvq_gemv_sg", "llvq_class_info", "llvq_golay_table",
     "llvq_encode_blocks", "llvq_rank_blocks", "llvq_pack_fields",
-    "llvq_sorted_bytes", "llvq_sort_blocks", "llvq_gemv_sorted",
+    "llvq_sorted_bytes", "llvq_sort_blocks", "llvq_gemv_sorted", "llvq_sort_blocks_sg", "llvq_gemv_sorted_sg",
     "llvq_sorted_gemm_bytes", "llvq_sort_blocks_gemm", "llvq_gemm_small_batch_sorted",
 ]
 
@@ -82,6 +83,8 @@ def load_library() -> ctypes.CDLL:
     lib.llvq_sorted_bytes.restype = ctypes.c_size_t
     lib.llvq_sort_blocks.argtypes = [vp, vp, i64, i64, vp, vp]
     lib.llvq_gemv_sorted.argtypes = [vp, vp, vp, i64, i64, vp, vp, ctypes.c_int, vp]
+    lib.llvq_sort_blocks_sg.argtypes = [vp, vp, ctypes.c_int, i64, i64, vp, vp]
+    lib.llvq_gemv_sorted_sg.argtypes = [vp, vp, ctypes.c_int, vp, vp, i64, i64, vp, vp, ctypes.c_int, vp]
     lib.llvq_sorted_gemm_bytes.argtypes = [vp, i64, i64]
     lib.llvq_sorted_gemm_bytes.restype = ctypes.c_size_t
     lib.llvq_sort_blocks_gemm.argtypes = [vp, vp, i64, i64, vp, vp]
@@ -298,6 +301,39 @@ def llvq_gemv_sorted(ctx: Context, d_sorted: torch.Tensor, d_gain: torch.Tensor,
     code = LLVQ_F32 if d_y.dtype == torch.float32 else LLVQ_BF16
     _check("llvq_gemv_sorted", ctx._lib.llvq_gemv_sorted(ctx._h, _dev(d_sorted, "d_sorted"), _dev(d_gain, "d_gain"), n_out, k_in,
                                                          _dev(d_x, "d_x"), _dev(d_y, "d_y"), code, _stream_ptr(stream)))
+    return d_y
+
+
+def llvq_sort_blocks_sg(ctx: Context, d_fields: torch.Tensor, gain_bits: int, n_out: int, k_in: int,
+                        d_sorted: torch.Tensor | None = None, stream=None):
+    """``llvq_sort_blocks`` for a stream of shape-gain fields (index_bits + gain_bits <= 48 bits each)."""
+    nbytes = int(ctx._lib.llvq_sorted_bytes(ctx._h, n_out, k_in))
+    if nbytes == 0:
+        raise LlvqError("llvq_sorted_bytes", 3)
+    if d_sorted is None:
+        d_sorted = torch.empty(nbytes, dtype=torch.uint8, device=d_fields.device)
+    assert d_sorted.numel() * d_sorted.element_size() >= nbytes
+    assert d_fields.numel() * d_fields.element_size() >= int(ctx._lib.llvq_field_bytes(ctx._h, n_out * ((k_in + 23) // 24), gain_bits))
+    _check("llvq_sort_blocks_sg", ctx._lib.llvq_sort_blocks_sg(ctx._h, _dev(d_fields, "d_fields"), gain_bits, n_out, k_in,
+                                                               _dev(d_sorted, "d_sorted"), _stream_ptr(stream)))
+    return d_sorted
+
+
+def llvq_gemv_sorted_sg(ctx: Context, d_sorted: torch.Tensor, gain_bits: int, d_codebook: torch.Tensor,
+                        d_row_scale: torch.Tensor | None, n_out: int, k_in: int, d_x: torch.Tensor,
+                        d_y: torch.Tensor | None = None, y_dtype: torch.dtype = torch.float32, stream=None):
+    """y = W x with W in the shape-gain form, from the sorted stream of ``llvq_sort_blocks_sg``; same result as ``llvq_gemv_sg``."""
+    if d_y is None:
+        d_y = torch.empty(n_out, dtype=y_dtype, device=d_sorted.device)
+    assert d_x.dtype == torch.bfloat16 and d_x.numel() >= k_in
+    assert d_y.dtype in (torch.float32, torch.bfloat16) and d_y.numel() >= n_out
+    assert d_codebook.dtype == torch.float32 and d_codebook.numel() >= (1 << gain_bits)
+    assert d_row_scale is None or (d_row_scale.dtype == torch.float32 and d_row_scale.numel() >= n_out)
+    assert d_sorted.numel() * d_sorted.element_size() >= int(ctx._lib.llvq_sorted_bytes(ctx._h, n_out, k_in))
+    code = LLVQ_F32 if d_y.dtype == torch.float32 else LLVQ_BF16
+    _check("llvq_gemv_sorted_sg", ctx._lib.llvq_gemv_sorted_sg(
+        ctx._h, _dev(d_sorted, "d_sorted"), gain_bits, _dev(d_codebook, "d_codebook"),
+        None if d_row_scale is None else _dev(d_row_scale, "d_row_scale"), n_out, k_in, _dev(d_x, "d_x"), _dev(d_y, "d_y"), code, _stream_ptr(stream)))
     return d_y
 
 

@@ -343,8 +343,8 @@ __device__ __forceinline__ void for_each_sorted_segment(int64_t U, int64_t G, in
 }
 
 __global__ void __launch_bounds__(kSortThreads, 1)
-sort_blocks_kernel(FastArgs fa, const uint32_t* __restrict__ stream, const uint16_t* __restrict__ sort_rank, int64_t n_out, int64_t bpr,
-                   unsigned long long* __restrict__ out)
+sort_blocks_kernel(FastArgs fa, const uint32_t* __restrict__ stream, const uint16_t* __restrict__ sort_rank, int gain_bits, int64_t n_out,
+                   int64_t bpr, unsigned long long* __restrict__ out)
 {
     FAST_PROLOGUE();
     __shared__ uint32_t hist[1024], cursor[1024];                  // one bin per class, in sort order; bin 1023 = no block
@@ -363,10 +363,11 @@ sort_blocks_kernel(FastArgs fa, const uint32_t* __restrict__ stream, const uint1
             const int64_t row = rg * kGemvGroupRows + (lane >> 2), cb = kq * 4 + (lane & 3);
             field = kSortIndexMask;
             if (row >= n_out || cb >= bpr) return 1023u;
-            const uint64_t I = load_field(stream, (uint64_t)(row * bpr + cb), (int)fa.L.W);
+            const uint64_t f = load_field(stream, (uint64_t)(row * bpr + cb), (int)fa.L.W + gain_bits);   // shape index | gain index << W
+            const uint64_t I = f & ((1ull << fa.L.W) - 1ull);
             if (I >= fa.n_points) { if (count) atomicAdd(fa.bad_index, 1ull); return 1023u; }
             uint64_t local;
-            field = I;
+            field = f;
             return (uint32_t)__ldg(sort_rank + fast_find_class(T, I, local));
         };
         for (int i = threadIdx.x; i < entries; i += kSortThreads) {
@@ -415,16 +416,17 @@ __device__ __forceinline__ void decode_known_class(const FastSmem& T, uint32_t c
     }
 }
 
-__device__ __forceinline__ void decode_sorted_entry(const FastArgs& fa, const FastSmem& T, uint64_t I, bool valid, Decoded& r)
+__device__ __forceinline__ uint32_t decode_sorted_entry(const FastArgs& fa, const FastSmem& T, uint64_t I, bool valid, Decoded& r)
 {
     uint64_t local = 0;
     const uint32_t cls = valid ? fast_find_class(T, I, local) : 0u;
     decode_known_class(T, cls, local, valid, r);
+    return cls;
 }
 
-template <bool kOutBf16>
+template <bool kOutBf16, bool kSg = false>
 __global__ void __launch_bounds__(kSortThreads, 1)
-gemv_sorted_kernel(FastArgs fa, const unsigned long long* __restrict__ sorted, const uint16_t* __restrict__ gain,
+gemv_sorted_kernel(FastArgs fa, const unsigned long long* __restrict__ sorted, const uint16_t* __restrict__ gain, SgArgs sg,
                    int64_t n_out, int64_t k_in, int64_t bpr, uint32_t nq_magic, const uint16_t* __restrict__ x, void* __restrict__ y,
                    float* __restrict__ scratch, uint32_t* __restrict__ counters)
 {
@@ -463,18 +465,25 @@ gemv_sorted_kernel(FastArgs fa, const unsigned long long* __restrict__ sorted, c
             if (lane == 0) nxt = atomicAdd(next_chunk, 1u);
             nxt = __shfl_sync(kFullMask, nxt, 0);
             const unsigned long long e_next = nxt < nchunks ? __ldg(seg + (uint64_t)nxt * 32) : 0ull;
-            const uint64_t I = e & kSortIndexMask;
+            const uint64_t field = e & kSortIndexMask;
+            const uint64_t I = kSg ? field & ((1ull << fa.L.W) - 1ull) : field;     // shape-gain form: gain index above the shape index
             const uint32_t pos = (uint32_t)(e >> 48);
-            const bool valid = I < fa.n_points;
+            const bool valid = field != kSortIndexMask && I < fa.n_points;
             // where the block sits: unit = pos / 32 of the segment, (row, column block) = lane of the unit
             const uint32_t v = kq_a + (pos >> 5);
             uint32_t q = __umulhi(v, nq_magic), kq = v - q * nq32;
             if (kq >= nq32) { kq -= nq32; ++q; }
             const uint32_t rloc = (rg_off + q) * kGemvGroupRows + ((pos >> 2) & 7u);      // row inside the pass
             const uint32_t cb = kq * 4u + (pos & 3u);
-            const float gn = valid ? gain_to_float(__ldg(gain + ((int64_t)rg0 * kGemvGroupRows + rloc) * bpr + cb)) : 0.f;
+            float gn = 0.f;
+            if (!kSg && valid) gn = gain_to_float(__ldg(gain + ((int64_t)rg0 * kGemvGroupRows + rloc) * bpr + cb));
             Decoded r;
-            decode_sorted_entry(fa, T, I, valid, r);
+            const uint32_t cls = decode_sorted_entry(fa, T, I, valid, r);
+            if (kSg && valid) {
+                const float scale = sg.row_scale ? __ldg(sg.row_scale + (int64_t)rg0 * kGemvGroupRows + rloc) : 1.f;
+                gn = __fmul_rn(__fmul_rn(scale, __ldg(sg.codebook + (uint32_t)(field >> fa.L.W))),
+                               __uint_as_float(T.desc[cls * kFastDescStride + kFastDescRnorm]));
+            }
             uint32_t w[12];
             expand_bf16(r, gn, w);
             const uint4* xb = reinterpret_cast<const uint4*>(xs + cb * 12u);
@@ -1572,12 +1581,12 @@ size_t llvq_sorted_bytes(const llvq_ctx* ctx, int64_t n_out, int64_t k_in)
     return (size_t)(((n_out + kGemvGroupRows - 1) / kGemvGroupRows) * nq) * 32 * 8;
 }
 
-int llvq_sort_blocks(const llvq_ctx* ctx, const void* d_idx, int64_t n_out, int64_t k_in, void* d_sorted, void* stream)
+static int sort_blocks_common(const llvq_ctx* ctx, const void* d_fields, int gain_bits, int64_t n_out, int64_t k_in, void* d_sorted, void* stream)
 {
-    if (int e = check_common(ctx, d_idx)) return e;
-    if (!d_sorted || n_out <= 0 || k_in <= 0) return LLVQ_EINVAL;
+    if (int e = check_common(ctx, d_fields)) return e;
+    if (!d_sorted || n_out <= 0 || k_in <= 0 || gain_bits < 0 || gain_bits > 8) return LLVQ_EINVAL;
     if (!aligned(d_sorted, 16)) return LLVQ_EALIGN;
-    if (!sortable(ctx, k_in) || n_out > 64ll * kMaxScratchRows) return LLVQ_EUNSUPPORTED;
+    if (!sortable(ctx, k_in) || ctx->host.W + gain_bits > 48 || n_out > 64ll * kMaxScratchRows) return LLVQ_EUNSUPPORTED;
     DeviceGuard guard(ctx->device);
     if (!guard.ok) return LLVQ_ECUDA;
     const int64_t bpr = (k_in + 23) / 24, nq = (bpr + 3) / 4;
@@ -1585,19 +1594,28 @@ int llvq_sort_blocks(const llvq_ctx* ctx, const void* d_idx, int64_t n_out, int6
     const unsigned g = (unsigned)std::min<int64_t>(units, ctx->sm_count);
     const size_t smem = ctx->fl.total + 16;
     if (!set_smem(sort_blocks_kernel, smem)) return LLVQ_ECUDA;
-    sort_blocks_kernel<<<g, kSortThreads, smem, (cudaStream_t)stream>>>(fast_args(ctx), static_cast<const uint32_t*>(d_idx), ctx->d_sort_rank, n_out, bpr,
-                                                                       static_cast<unsigned long long*>(d_sorted));
+    sort_blocks_kernel<<<g, kSortThreads, smem, (cudaStream_t)stream>>>(fast_args(ctx), static_cast<const uint32_t*>(d_fields), ctx->d_sort_rank, gain_bits,
+                                                                       n_out, bpr, static_cast<unsigned long long*>(d_sorted));
     return launch_status();
 }
 
-int llvq_gemv_sorted(const llvq_ctx* ctx, const void* d_sorted, const uint16_t* d_gain_f16, int64_t n_out, int64_t k_in,
-                     const uint16_t* d_x_bf16, void* d_y, int y_dtype, void* stream)
+int llvq_sort_blocks(const llvq_ctx* ctx, const void* d_idx, int64_t n_out, int64_t k_in, void* d_sorted, void* stream)
 {
-    if (ctx && ctx->device >= 0 && n_out == 0) return LLVQ_OK;
-    if (int e = check_common(ctx, d_sorted)) return e;
-    if (!d_gain_f16 || !d_x_bf16 || !d_y || n_out < 0 || k_in <= 0) return LLVQ_EINVAL;
+    return sort_blocks_common(ctx, d_idx, 0, n_out, k_in, d_sorted, stream);
+}
+
+int llvq_sort_blocks_sg(const llvq_ctx* ctx, const void* d_fields, int gain_bits, int64_t n_out, int64_t k_in, void* d_sorted, void* stream)
+{
+    return sort_blocks_common(ctx, d_fields, gain_bits, n_out, k_in, d_sorted, stream);
+}
+
+// Exactly one of d_gain_f16 / sg is used.
+static int gemv_sorted_common(const llvq_ctx* ctx, const void* d_sorted, const uint16_t* d_gain_f16, const SgArgs* sg, int64_t n_out, int64_t k_in,
+                              const uint16_t* d_x_bf16, void* d_y, int y_dtype, void* stream)
+{
+    if (!d_x_bf16 || !d_y || n_out < 0 || k_in <= 0) return LLVQ_EINVAL;
     if (y_dtype != LLVQ_F32 && y_dtype != LLVQ_BF16) return LLVQ_EINVAL;
-    if (!aligned(d_gain_f16, 2) || !aligned(d_x_bf16, 2) || !aligned(d_y, y_dtype == LLVQ_F32 ? 4 : 2)) return LLVQ_EALIGN;
+    if (!aligned(d_x_bf16, 2) || !aligned(d_y, y_dtype == LLVQ_F32 ? 4 : 2)) return LLVQ_EALIGN;
     if (!sortable(ctx, k_in) || n_out > 64ll * kMaxScratchRows) return LLVQ_EUNSUPPORTED;
     DeviceGuard guard(ctx->device);
     if (!guard.ok) return LLVQ_ECUDA;
@@ -1608,16 +1626,37 @@ int llvq_gemv_sorted(const llvq_ctx* ctx, const void* d_sorted, const uint16_t* 
     const size_t smem = ctx->fl.total + 16 + (size_t)nq * 48 * 4 + kSortAccCopies * kGemvGroupsPerPass * kGemvGroupRows * 4 + 16;
     const uint32_t magic = nq == 1 ? 0xffffffffu : (uint32_t)((1ull << 32) / (uint64_t)nq);
     const unsigned long long* sp = static_cast<const unsigned long long*>(d_sorted);
-    if (y_dtype == LLVQ_BF16) {
-        if (!set_smem(gemv_sorted_kernel<true>, smem)) return LLVQ_ECUDA;
-        if (launch_pdl(gemv_sorted_kernel<true>, g, (unsigned)kSortThreads, smem, st, fast_args(ctx), sp, d_gain_f16, n_out, k_in, bpr, magic,
-                       d_x_bf16, d_y, ctx->d_scratch, ctx->d_counters) != cudaSuccess) return LLVQ_ECUDA;
-    } else {
-        if (!set_smem(gemv_sorted_kernel<false>, smem)) return LLVQ_ECUDA;
-        if (launch_pdl(gemv_sorted_kernel<false>, g, (unsigned)kSortThreads, smem, st, fast_args(ctx), sp, d_gain_f16, n_out, k_in, bpr, magic,
-                       d_x_bf16, d_y, ctx->d_scratch, ctx->d_counters) != cudaSuccess) return LLVQ_ECUDA;
-    }
+    const SgArgs sga = sg ? *sg : SgArgs{};
+#define LLVQ_LAUNCH_SORTED(BF16, SG)                                                                                    \
+    do {                                                                                                                \
+        if (!set_smem(gemv_sorted_kernel<BF16, SG>, smem)) return LLVQ_ECUDA;                                            \
+        if (launch_pdl(gemv_sorted_kernel<BF16, SG>, g, (unsigned)kSortThreads, smem, st, fast_args(ctx), sp, d_gain_f16, sga, n_out, k_in, bpr, \
+                       magic, d_x_bf16, d_y, ctx->d_scratch, ctx->d_counters) != cudaSuccess) return LLVQ_ECUDA;          \
+    } while (0)
+    if (sg) { if (y_dtype == LLVQ_BF16) LLVQ_LAUNCH_SORTED(true, true); else LLVQ_LAUNCH_SORTED(false, true); }
+    else    { if (y_dtype == LLVQ_BF16) LLVQ_LAUNCH_SORTED(true, false); else LLVQ_LAUNCH_SORTED(false, false); }
+#undef LLVQ_LAUNCH_SORTED
     return launch_status();
+}
+
+int llvq_gemv_sorted(const llvq_ctx* ctx, const void* d_sorted, const uint16_t* d_gain_f16, int64_t n_out, int64_t k_in,
+                     const uint16_t* d_x_bf16, void* d_y, int y_dtype, void* stream)
+{
+    if (ctx && ctx->device >= 0 && n_out == 0) return LLVQ_OK;
+    if (int e = check_common(ctx, d_sorted)) return e;
+    if (!d_gain_f16) return LLVQ_EINVAL;
+    if (!aligned(d_gain_f16, 2)) return LLVQ_EALIGN;
+    return gemv_sorted_common(ctx, d_sorted, d_gain_f16, nullptr, n_out, k_in, d_x_bf16, d_y, y_dtype, stream);
+}
+
+int llvq_gemv_sorted_sg(const llvq_ctx* ctx, const void* d_sorted, int gain_bits, const float* d_codebook_f32, const float* d_row_scale_f32,
+                        int64_t n_out, int64_t k_in, const uint16_t* d_x_bf16, void* d_y, int y_dtype, void* stream)
+{
+    if (ctx && ctx->device >= 0 && n_out == 0) return LLVQ_OK;
+    if (int e = check_sg(ctx, d_sorted, gain_bits, d_codebook_f32, d_row_scale_f32)) return e;
+    if (ctx->host.W + gain_bits > 48) return LLVQ_EUNSUPPORTED;
+    const SgArgs sg{d_codebook_f32, d_row_scale_f32, gain_bits};
+    return gemv_sorted_common(ctx, d_sorted, nullptr, &sg, n_out, k_in, d_x_bf16, d_y, y_dtype, stream);
 }
 
 // Sorted layout of the small-batch GEMM (see the comment at sort_blocks_gemm_kernel).

@@ -176,8 +176,10 @@ def test_gemv_small_shapes_both_output_types(lib, ctxs, oracle_mod, code, n_out,
     torch.cuda.synchronize()
     assert gemv_error(y32.cpu().numpy(), want) <= TOL
     assert gemv_error(y16.float().cpu().numpy(), want) <= TOL_BF16_OUT
-    # the bf16 output is the rounding of the fp32 one
-    assert torch.equal(y32.to(torch.bfloat16), y16)
+    # the bf16 output is the rounding of the fp32 one; the two launches may add their partial sums in a different
+    # order (shared-memory atomics), so a value next to a rounding boundary may land on either side of it
+    a, b = y32.to(torch.bfloat16).float(), y16.float()
+    assert float(((a - b).abs() / a.abs().clamp_min(1e-30)).max()) <= 2.0 ** -7
 
 
 def test_gemv_exact_integer_cases(lib, ctxs, oracle_mod):

@@ -154,3 +154,46 @@ def test_sg_argument_checks(lib, ctxs):
     big = lib.Context(2, 53, device=0)                                                       # class tables not in shared memory
     assert big._lib.llvq_dequant_matrix_sg(big._h, p, 0, c, None, 1, 24, o, 24, None) == 3
     assert lib.llvq_last_error(ctx) == (0, 0)
+
+
+@pytest.mark.parametrize("code,bits", [((2, 12), 1), ((2, 11), 2), ((2, 10), 4), ((2, 13), 0)])
+def test_gemv_sorted_sg(lib, ctxs, codes, code, bits):
+    o, ctx = codes[code], ctxs[code]
+    n_out, k_in = 333, 2000
+    stream, nblocks = gen.make_layer_sg(o.N, o.W, bits, n_out, k_in, seed=31)
+    cb = _codebook(bits)
+    rs = gen.row_scales_f32(n_out, seed=9)
+    x = gen.normal_bf16(k_in, seed=6)
+    ref = o.gemm_sg(stream, bits, cb, rs, n_out, k_in, x, threads=4)
+    d_cb, d_rs, d_x = _f32(cb), _f32(rs), to_dev_bf16(x)
+    srt = lib.llvq_sort_blocks_sg(ctx, to_dev_u8(stream), bits, n_out, k_in)
+    y = lib.llvq_gemv_sorted_sg(ctx, srt, bits, d_cb, d_rs, n_out, k_in, d_x)
+    yb = lib.llvq_gemv_sorted_sg(ctx, srt, bits, d_cb, None, n_out, k_in, d_x, y_dtype=torch.bfloat16)
+    torch.cuda.synchronize()
+    assert gemv_error(y.cpu().numpy(), ref) <= TOL
+    ref_noscale = o.gemm_sg(stream, bits, cb, None, n_out, k_in, x, threads=4)
+    assert gemv_error(yb.float().cpu().numpy(), ref_noscale) <= TOL_BF16_OUT
+    assert lib.llvq_last_error(ctx) == (0, 0)
+
+
+def test_gemv_sorted_sg_full_size_and_limits(lib, ctxs, codes):
+    code, bits = (2, 12), 1
+    o, ctx = codes[code], ctxs[code]
+    n_out, k_in = 4096, 4096
+    stream, nblocks = gen.make_layer_sg(o.N, o.W, bits, n_out, k_in, seed=2)
+    cb = _codebook(bits)
+    rs = gen.row_scales_f32(n_out, seed=2)
+    x = gen.normal_bf16(k_in, seed=2)
+    d_s = to_dev_u8(stream)
+    srt = lib.llvq_sort_blocks_sg(ctx, d_s, bits, n_out, k_in)
+    y = lib.llvq_gemv_sorted_sg(ctx, srt, bits, _f32(cb), _f32(rs), n_out, k_in, to_dev_bf16(x)).cpu().numpy()
+    y2 = lib.llvq_gemv_sg(ctx, d_s, bits, _f32(cb), _f32(rs), n_out, k_in, to_dev_bf16(x)).cpu().numpy()
+    assert gemv_error(y, y2.astype(np.float64)) <= 1e-4
+    rows = [0, 9, 2047, 4095] + list(range(123, 4096, 611))
+    ref = np.array([o.gemm_sg(stream, bits, cb, rs, n_out, k_in, x, rows=(r, 1))[r] for r in rows])
+    assert gemv_error(y[rows], ref) <= TOL
+    # 47 + 2 bits do not fit the 48-bit entry
+    buf = torch.zeros(4096, dtype=torch.uint8, device="cuda")
+    assert ctx._lib.llvq_sort_blocks_sg(ctx._h, buf.data_ptr(), 2, 8, 24, buf.data_ptr(), None) == 3
+    assert ctx._lib.llvq_gemv_sorted_sg(ctx._h, buf.data_ptr(), 2, buf.data_ptr(), None, 8, 24, buf.data_ptr(), buf.data_ptr(), 0, None) == 3
+    assert lib.llvq_last_error(ctx) == (0, 0)
