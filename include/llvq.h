@@ -125,6 +125,8 @@ int llvq_dequant_matrix(const llvq_ctx* ctx, const void* d_idx, const uint16_t* 
  * the bf16-rounded values llvq_dequant_matrix would produce; products are
  * accumulated in binary32.  d_x_bf16: device, [k_in] bf16 bits.
  * d_y: device, [n_out], float (y_dtype = LLVQ_F32) or bf16 bits (LLVQ_BF16).
+ * The order in which partial sums are added is not fixed (shared-memory and global atomics): two calls on the same
+ * inputs may differ in the last bits of y.  The same holds for every fused product of this library.
  */
 int llvq_gemv(const llvq_ctx* ctx, const void* d_idx, const uint16_t* d_gain_f16,
               int64_t n_out, int64_t k_in, const uint16_t* d_x_bf16,
