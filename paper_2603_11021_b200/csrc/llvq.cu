@@ -553,9 +553,9 @@ gemv_sorted_kernel(FastArgs fa, const unsigned long long* __restrict__ sorted, c
 constexpr int kBinSegUnits = 256;                    // at most 8192 blocks per segment (halved while shared memory is short)
 constexpr int kBinPerThread = kBinSegUnits * 32 / kSortThreads;   // 8
 
-template <bool kOutBf16>
+template <bool kOutBf16, bool kSg = false>
 __global__ void __launch_bounds__(kSortThreads, 1)
-gemv_bin_kernel(FastArgs fa, const uint32_t* __restrict__ stream, const uint16_t* __restrict__ sort_rank, const uint16_t* __restrict__ gain,
+gemv_bin_kernel(FastArgs fa, const uint32_t* __restrict__ stream, const uint16_t* __restrict__ sort_rank, const uint16_t* __restrict__ gain, SgArgs sg,
                 int64_t n_out, int64_t k_in, int64_t bpr, uint32_t nq_magic, int seg_units, const uint16_t* __restrict__ x, void* __restrict__ y,
                 float* __restrict__ scratch, uint32_t* __restrict__ counters)
 {
@@ -568,7 +568,7 @@ gemv_bin_kernel(FastArgs fa, const uint32_t* __restrict__ stream, const uint16_t
     uint32_t* hist = last_flag + 4;                                  // [1024] bins in sort order; later their first slots
     uint32_t* cursor = hist + 1024;                                  // [1024]
     unsigned long long* ent = reinterpret_cast<unsigned long long*>(cursor + 1024);   // [seg_units * 32] class-local index | position << 48
-    uint16_t* ent_cls = reinterpret_cast<uint16_t*>(ent + seg_units * 32);            // [seg_units * 32] class, 0xffff = no block
+    uint16_t* ent_cls = reinterpret_cast<uint16_t*>(ent + seg_units * 32);            // [seg_units * 32] class (| gain index << 10), 0xffff = no block
     for (int64_t i = threadIdx.x; i < nq * 48; i += blockDim.x) {
         const int64_t e = 2 * i;
         const uint32_t lo = e < k_in ? __ldg(x + e) : 0u, hi = e + 1 < k_in ? __ldg(x + e + 1) : 0u;
@@ -585,8 +585,9 @@ gemv_bin_kernel(FastArgs fa, const uint32_t* __restrict__ stream, const uint16_t
         // request it from DRAM now, the binning phases then read it from L2
         const uint64_t b_first = (uint64_t)(u_begin / nq) * kGemvGroupRows * (uint64_t)bpr;
         const uint64_t b_last = (uint64_t)min(((u_end - 1) / nq + 1) * kGemvGroupRows, n_out) * (uint64_t)bpr;
-        prefetch_span_l2(stream, b_first * fa.L.W / 8, (b_last * fa.L.W + 7) / 8);
-        prefetch_span_l2(gain, b_first * 2, b_last * 2);
+        const uint64_t wf = (uint64_t)fa.L.W + (kSg ? (uint64_t)sg.bits : 0ull);
+        prefetch_span_l2(stream, b_first * wf / 8, (b_last * wf + 7) / 8);
+        if (!kSg) prefetch_span_l2(gain, b_first * 2, b_last * 2);
     }
     for_each_sorted_segment(U, G, nq, blockIdx.x, [&](int64_t tu0, int64_t tu1, int64_t rg0, int64_t rg1, bool first, bool last) {
         if (first)
@@ -613,9 +614,13 @@ gemv_bin_kernel(FastArgs fa, const uint32_t* __restrict__ stream, const uint16_t
                 uint32_t key = 1023u, cls = 0xffffu;
                 uint64_t local = 0;
                 if (row < n_out && cb < bpr) {
-                    const uint64_t I = load_field(stream, (uint64_t)(row * bpr + cb), (int)fa.L.W);
-                    if (I < fa.n_points) { cls = fast_find_class(T, I, local); key = __ldg(sort_rank + cls); }
-                    else atomicAdd(fa.bad_index, 1ull);
+                    const uint64_t f = load_field(stream, (uint64_t)(row * bpr + cb), (int)fa.L.W + (kSg ? sg.bits : 0));
+                    const uint64_t I = kSg ? f & ((1ull << fa.L.W) - 1ull) : f;
+                    if (I < fa.n_points) {
+                        cls = fast_find_class(T, I, local);
+                        key = __ldg(sort_rank + cls);
+                        if (kSg) cls |= (uint32_t)(f >> fa.L.W) << 10;           // the gain index rides with the class
+                    } else atomicAdd(fa.bad_index, 1ull);
                 }
                 mine_key[q] = key | cls << 16;
                 mine_ent[q] = local | (unsigned long long)pos << 48;
@@ -664,9 +669,18 @@ gemv_bin_kernel(FastArgs fa, const uint32_t* __restrict__ stream, const uint16_t
             if (kq >= nq32) { kq -= nq32; ++q; }
             const uint32_t rloc = (rg_off + q) * kGemvGroupRows + ((pos >> 2) & 7u);
             const uint32_t cb = kq * 4u + (pos & 3u);
-            const float gn = valid ? gain_to_float(__ldg(gain_pass + (int64_t)rloc * bpr + cb)) : 0.f;
+            const uint32_t cls = valid ? (kSg ? cls16 & 1023u : cls16) : 0u;
+            float gn = 0.f;
+            if (valid) {
+                if (kSg) {
+                    const float scale = sg.row_scale ? __ldg(sg.row_scale + (int64_t)rg0 * kGemvGroupRows + rloc) : 1.f;
+                    gn = __fmul_rn(__fmul_rn(scale, __ldg(sg.codebook + (cls16 >> 10))), __uint_as_float(T.desc[cls * kFastDescStride + kFastDescRnorm]));
+                } else {
+                    gn = gain_to_float(__ldg(gain_pass + (int64_t)rloc * bpr + cb));
+                }
+            }
             Decoded r;
-            decode_known_class(T, valid ? cls16 : 0u, e & ((1ull << 48) - 1ull), valid, r);
+            decode_known_class(T, cls, e & ((1ull << 48) - 1ull), valid, r);
             uint32_t w[12];
             expand_bf16(r, gn, w);
             const uint4* xb = reinterpret_cast<const uint4*>(xs + cb * 12u);
@@ -1480,17 +1494,18 @@ static int gemv_common(const llvq_ctx* ctx, const void* d_idx, const uint16_t* d
     };
     // (smaller segments sort too few blocks to pay for the sort: the direct kernel takes over when 8192 do not fit)
     const size_t smem_bin = bin_bytes(seg_units);
-    if (!sg && ctx->fast && ctx->d_sort_rank && ctx->host.desc.size() >= 64 && ctx->host.W <= 48 && smem_bin <= 227 * 1024 && nq < (1ll << 24)) {
+    if ((!sg || sg->bits <= 5) && ctx->fast && ctx->d_sort_rank && ctx->host.desc.size() >= 64 && ctx->host.W <= 48 && smem_bin <= 227 * 1024 &&
+        nq < (1ll << 24)) {
         const uint32_t magic = nq == 1 ? 0xffffffffu : (uint32_t)((1ull << 32) / (uint64_t)nq);
-        if (y_dtype == LLVQ_BF16) {
-            if (!set_smem(gemv_bin_kernel<true>, smem_bin)) return LLVQ_ECUDA;
-            if (launch_pdl(gemv_bin_kernel<true>, g, (unsigned)kSortThreads, smem_bin, st, fa, idx, ctx->d_sort_rank, d_gain_f16, n_out, k_in, bpr, magic,
-                           seg_units, d_x_bf16, d_y, ctx->d_scratch, ctx->d_counters) != cudaSuccess) return LLVQ_ECUDA;
-        } else {
-            if (!set_smem(gemv_bin_kernel<false>, smem_bin)) return LLVQ_ECUDA;
-            if (launch_pdl(gemv_bin_kernel<false>, g, (unsigned)kSortThreads, smem_bin, st, fa, idx, ctx->d_sort_rank, d_gain_f16, n_out, k_in, bpr, magic,
-                           seg_units, d_x_bf16, d_y, ctx->d_scratch, ctx->d_counters) != cudaSuccess) return LLVQ_ECUDA;
-        }
+#define LLVQ_LAUNCH_BIN(BF16, SG)                                                                                          \
+    do {                                                                                                                   \
+        if (!set_smem(gemv_bin_kernel<BF16, SG>, smem_bin)) return LLVQ_ECUDA;                                              \
+        if (launch_pdl(gemv_bin_kernel<BF16, SG>, g, (unsigned)kSortThreads, smem_bin, st, fa, idx, ctx->d_sort_rank, d_gain_f16, sga, n_out, k_in, \
+                       bpr, magic, seg_units, d_x_bf16, d_y, ctx->d_scratch, ctx->d_counters) != cudaSuccess) return LLVQ_ECUDA; \
+    } while (0)
+        if (sg) { if (y_dtype == LLVQ_BF16) LLVQ_LAUNCH_BIN(true, true); else LLVQ_LAUNCH_BIN(false, true); }
+        else    { if (y_dtype == LLVQ_BF16) LLVQ_LAUNCH_BIN(true, false); else LLVQ_LAUNCH_BIN(false, false); }
+#undef LLVQ_LAUNCH_BIN
         return launch_status();
     }
 #define LLVQ_LAUNCH_GEMV(BIG, BF16, SG)                                                                            \
