@@ -286,6 +286,22 @@ def extras(P, ctx) -> dict:
         by = nb * (CODE_W // 8 + 2) + batch * k * 2 + batch * n * 2
         out[f"gemm_8192x8192_b{batch}_sorted_layout"] = {"us": us, "GBps": by / us / 1e3, "TFLOPs": 2.0 * n * k * batch / us / 1e6, "algorithmic_bytes": by}
     del bufs, srt
+    # --- the two rectangular shapes of the same configuration, batch 16 (4 rotating copies, 314 MB)
+    for (n2, k2) in ((28672, 8192), (8192, 28672)):
+        bufs2 = []
+        for c in range(4):
+            stream, gain, nb2 = gen.make_layer(CODE_N, CODE_W, n2, k2, 1, seed=220 + c)
+            d_i, d_g = dev(stream), dev(gain, np.float16)
+            bufs2.append((d_i, d_g, P.llvq_sort_blocks_gemm(ctx, d_i, n2, k2)))
+        x = dev(gen.normal_bf16((16, k2), seed=16), np.int16).view(torch.bfloat16)
+        y = torch.empty((16, n2), dtype=torch.bfloat16, device="cuda")
+        by = nb2 * (CODE_W // 8 + 2) + 16 * k2 * 2 + 16 * n2 * 2
+        for name, fn in (("", lambda i: P.llvq_gemm_small_batch(ctx, bufs2[i % 4][0], bufs2[i % 4][1], n2, k2, x, d_y=y)),
+                         ("_sorted_layout", lambda i: P.llvq_gemm_small_batch_sorted(ctx, bufs2[i % 4][2], bufs2[i % 4][1], n2, k2, x, d_y=y))):
+            _event_us(torch, fn, 2)
+            us = _event_us(torch, fn, 8)
+            out[f"gemm_{n2}x{k2}_b16{name}"] = {"us": us, "GBps": by / us / 1e3, "TFLOPs": 2.0 * n2 * k2 * 16 / us / 1e6, "algorithmic_bytes": by}
+        del bufs2
     # --- GEMM, 8192 x 8192 at ~3 bits/weight: 72-bit indices over shells 2..53
     ctx53 = P.Context(2, 53, device=torch.cuda.current_device())
     bufs = []
