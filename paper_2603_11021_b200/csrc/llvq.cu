@@ -380,7 +380,15 @@ sort_blocks_kernel(FastArgs fa, const uint32_t* __restrict__ stream, const uint1
             for (int k = 0; k < 1024; ++k) { const uint32_t c = hist[k]; hist[k] = run; run += c; }
         }
         __syncthreads();
-        for (int i = threadIdx.x; i < entries; i += kSortThreads) {
+        // the entries are visited column-block major (all row groups of a column unit, then the next unit): the blocks
+        // of a bin then come out roughly ordered by column block, and the 32 lanes of a GEMV warp read few different
+        // slices of x
+        const int64_t rg_a = tu0 / nq, nrg = (tu1 - 1) / nq - rg_a + 1;
+        for (int64_t e = threadIdx.x; e < nq * nrg * 32; e += kSortThreads) {
+            const int64_t kq = e / (nrg * 32), rem = e - kq * (nrg * 32);
+            const int64_t u = (rg_a + (rem >> 5)) * nq + kq;
+            if (u < tu0 || u >= tu1) continue;
+            const int i = (int)(u - tu0) * 32 + (int)(rem & 31);
             unsigned long long field;
             const uint32_t key = entry_of(i, false, field);
             const uint32_t slot = hist[key] + atomicAdd(&cursor[key], 1u);
