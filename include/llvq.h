@@ -160,6 +160,10 @@ int llvq_dequant_matrix_sg(const llvq_ctx* ctx, const void* d_fields, int gain_b
 int llvq_gemv_sg(const llvq_ctx* ctx, const void* d_fields, int gain_bits, const float* d_codebook_f32,
                  const float* d_row_scale_f32, int64_t n_out, int64_t k_in, const uint16_t* d_x_bf16,
                  void* d_y, int y_dtype, void* stream);
+/* The small-batch product (see llvq_gemm_small_batch for X, Y and batch) with W in the same shape-gain form. */
+int llvq_gemm_small_batch_sg(const llvq_ctx* ctx, const void* d_fields, int gain_bits, const float* d_codebook_f32,
+                             const float* d_row_scale_f32, int64_t n_out, int64_t k_in, const uint16_t* d_x_bf16,
+                             int batch, uint16_t* d_y_bf16, void* stream);
 
 /*
  * Sorted layout for the fused GEMV: a kernel-private arrangement of the same blocks, made once at load time (the

@@ -19,7 +19,7 @@ __all__ = [
     "llvq_dequant_matrix_sg", "llvq_gemv_sg",
     "llvq_encode_blocks", "llvq_rank_blocks", "llvq_pack_fields", "LLVQ_EUCLIDEAN", "LLVQ_ANGULAR",
     "llvq_sort_blocks", "llvq_gemv_sorted", "llvq_sort_blocks_gemm", "llvq_gemm_small_batch_sorted",
-    "llvq_sort_blocks_sg", "llvq_gemv_sorted_sg",
+    "llvq_sort_blocks_sg", "llvq_gemv_sorted_sg", "llvq_gemm_small_batch_sg",
     "llvq_last_error", "LlvqError", "EXPORTS", "load_library",
     "LLVQ_LAYOUT_FLAT", "LLVQ_LAYOUT_ROWWISE", "LLVQ_F32", "LLVQ_BF16",
 ]
@@ -39,7 +39,7 @@ EXPORTS = [
     "llvq_field_bytes", "llvq_dequant_matrix_sg", "llvq_gemv_sg", "llvq_class_info", "llvq_golay_table",
     "llvq_encode_blocks", "llvq_rank_blocks", "llvq_pack_fields",
     "llvq_sorted_bytes", "llvq_sort_blocks", "llvq_gemv_sorted", "llvq_sort_blocks_sg", "llvq_gemv_sorted_sg",
-    "llvq_sorted_gemm_bytes", "llvq_sort_blocks_gemm", "llvq_gemm_small_batch_sorted",
+    "llvq_sorted_gemm_bytes", "llvq_sort_blocks_gemm", "llvq_gemm_small_batch_sorted", "llvq_gemm_small_batch_sg",
 ]
 
 
@@ -83,6 +83,7 @@ def load_library() -> ctypes.CDLL:
     lib.llvq_sorted_bytes.restype = ctypes.c_size_t
     lib.llvq_sort_blocks.argtypes = [vp, vp, i64, i64, vp, vp]
     lib.llvq_gemv_sorted.argtypes = [vp, vp, vp, i64, i64, vp, vp, ctypes.c_int, vp]
+    lib.llvq_gemm_small_batch_sg.argtypes = [vp, vp, ctypes.c_int, vp, vp, i64, i64, vp, ctypes.c_int, vp, vp]
     lib.llvq_sort_blocks_sg.argtypes = [vp, vp, ctypes.c_int, i64, i64, vp, vp]
     lib.llvq_gemv_sorted_sg.argtypes = [vp, vp, ctypes.c_int, vp, vp, i64, i64, vp, vp, ctypes.c_int, vp]
     lib.llvq_sorted_gemm_bytes.argtypes = [vp, i64, i64]
@@ -244,6 +245,21 @@ def llvq_gemv_sg(ctx: Context, d_fields: torch.Tensor, gain_bits: int, d_codeboo
     code = LLVQ_F32 if d_y.dtype == torch.float32 else LLVQ_BF16
     _check("llvq_gemv_sg", ctx._lib.llvq_gemv_sg(ctx._h, _dev(d_fields, "d_fields"), gain_bits, cb, rs, n_out, k_in,
                                                  _dev(d_x, "d_x"), _dev(d_y, "d_y"), code, _stream_ptr(stream)))
+    return d_y
+
+
+def llvq_gemm_small_batch_sg(ctx: Context, d_fields: torch.Tensor, gain_bits: int, d_codebook: torch.Tensor,
+                             d_row_scale: torch.Tensor | None, n_out: int, k_in: int, d_x: torch.Tensor,
+                             d_y: torch.Tensor | None = None, stream=None):
+    """Y[b, i] = sum_k X[b, k] W[i, k] with W in the shape-gain form of ``llvq_dequant_matrix_sg``; batch <= 64."""
+    assert d_x.dtype == torch.bfloat16 and d_x.dim() == 2 and d_x.shape[1] == k_in
+    batch = d_x.shape[0]
+    if d_y is None:
+        d_y = torch.empty((batch, n_out), dtype=torch.bfloat16, device=d_fields.device)
+    assert d_y.dtype == torch.bfloat16 and d_y.numel() >= batch * n_out
+    cb, rs = _sg_args(ctx, d_fields, gain_bits, d_codebook, d_row_scale, n_out, n_out * ((k_in + 23) // 24))
+    _check("llvq_gemm_small_batch_sg", ctx._lib.llvq_gemm_small_batch_sg(
+        ctx._h, _dev(d_fields, "d_fields"), gain_bits, cb, rs, n_out, k_in, _dev(d_x, "d_x"), batch, _dev(d_y, "d_y"), _stream_ptr(stream)))
     return d_y
 
 

@@ -781,9 +781,9 @@ __device__ __forceinline__ void group_barrier(int group)
     asm volatile("bar.sync %0, %1;" ::"r"(1 + group), "n"(kGemmGroupThreads) : "memory");
 }
 
-template <bool kBig>
+template <bool kBig, bool kSg = false>
 __global__ void __launch_bounds__(kGemmThreads, 1)
-gemm_kernel(FastArgs fa, const uint32_t* __restrict__ stream, const uint16_t* __restrict__ gain, GemmArgs ga)
+gemm_kernel(FastArgs fa, const uint32_t* __restrict__ stream, const uint16_t* __restrict__ gain, SgArgs sg, GemmArgs ga)
 {
     extern __shared__ __align__(128) uint8_t smem[];
     const uint32_t img_bytes = fa.L.total;
@@ -834,7 +834,8 @@ gemm_kernel(FastArgs fa, const uint32_t* __restrict__ stream, const uint16_t* __
             const bool in = row < ga.n_out && cb < ga.bpr;
             const uint64_t b = in ? (uint64_t)(row * ga.bpr + cb) : 0ull;
             uint32_t w[12];
-            block_pairs<kBig>(fa, T, stream, gain, b, in, w);
+            if (kSg) block_pairs_sg(fa, T, stream, sg, b, row, in, w);
+            else block_pairs<kBig>(fa, T, stream, gain, b, in, w);
             // the MMAs of this group's previous stage read its buffers: wait for them only now, with the block already unranked
             if (uses > 0 && !mbar_wait(&bar_free[group], (uses - 1u) & 1u)) timeout = true;
             uint8_t* a_dst = a_mine + gwarp * 128 + (lane & 7) * 16;
@@ -1190,7 +1191,8 @@ int launch_gemm_domains(const llvq_ctx* ctx, const void* p, const uint16_t* d_ga
 // Enqueue the small-batch GEMM with the given split-K scratch ([npad][row tiles * 128] floats) and counters
 // ([row tiles]); both must be zero when the kernel starts and are zero again when it ends.
 int launch_gemm(const llvq_ctx* ctx, const void* d_idx, const uint16_t* d_gain_f16, int64_t n_out, int64_t k_in,
-                const uint16_t* d_x_bf16, int batch, uint16_t* d_y_bf16, float* scratch, uint32_t* counters, void* stream)
+                const uint16_t* d_x_bf16, int batch, uint16_t* d_y_bf16, float* scratch, uint32_t* counters, void* stream,
+                const SgArgs* sg = nullptr)
 {
     if (n_out == 0) return LLVQ_OK;
     DeviceGuard guard(ctx->device);
@@ -1218,12 +1220,15 @@ int launch_gemm(const llvq_ctx* ctx, const void* d_idx, const uint16_t* d_gain_f
     const size_t smem = ((img + 64 + 1023) & ~size_t(1023)) + 2 * kGemmRows * kStageK * 2 + 2 * (size_t)ga.npad * kStageK * 2;
     if (smem > 227 * 1024) return LLVQ_EUNSUPPORTED;
     const uint32_t* idx = static_cast<const uint32_t*>(d_idx);
-    if (ctx->fast) {
-        if (!set_smem(gemm_kernel<false>, smem)) return LLVQ_ECUDA;
-        if (launch_pdl(gemm_kernel<false>, grid, (unsigned)kGemmThreads, smem, st, fast_args(ctx), idx, d_gain_f16, ga) != cudaSuccess) return LLVQ_ECUDA;
+    if (sg) {
+        if (!set_smem(gemm_kernel<false, true>, smem)) return LLVQ_ECUDA;
+        if (launch_pdl(gemm_kernel<false, true>, grid, (unsigned)kGemmThreads, smem, st, fast_args(ctx), idx, d_gain_f16, *sg, ga) != cudaSuccess) return LLVQ_ECUDA;
+    } else if (ctx->fast) {
+        if (!set_smem(gemm_kernel<false, false>, smem)) return LLVQ_ECUDA;
+        if (launch_pdl(gemm_kernel<false, false>, grid, (unsigned)kGemmThreads, smem, st, fast_args(ctx), idx, d_gain_f16, SgArgs{}, ga) != cudaSuccess) return LLVQ_ECUDA;
     } else {
-        if (!set_smem(gemm_kernel<true>, smem)) return LLVQ_ECUDA;
-        if (launch_pdl(gemm_kernel<true>, grid, (unsigned)kGemmThreads, smem, st, fast_args(ctx), idx, d_gain_f16, ga) != cudaSuccess) return LLVQ_ECUDA;
+        if (!set_smem(gemm_kernel<true, false>, smem)) return LLVQ_ECUDA;
+        if (launch_pdl(gemm_kernel<true, false>, grid, (unsigned)kGemmThreads, smem, st, fast_args(ctx), idx, d_gain_f16, SgArgs{}, ga) != cudaSuccess) return LLVQ_ECUDA;
     }
     return launch_status();
 }
@@ -1720,6 +1725,18 @@ int llvq_gemm_small_batch_sorted(const llvq_ctx* ctx, const void* d_sorted, cons
     if (n_out == 0) return LLVQ_OK;
     if (!gemm_sortable(ctx) || n_out > kMaxScratchRows || k_in <= 0) return LLVQ_EUNSUPPORTED;
     return launch_gemm_domains(ctx, d_sorted, d_gain_f16, n_out, k_in, d_x_bf16, batch, d_y_bf16, ctx->d_scratch, ctx->d_counters, stream);
+}
+
+int llvq_gemm_small_batch_sg(const llvq_ctx* ctx, const void* d_fields, int gain_bits, const float* d_codebook_f32, const float* d_row_scale_f32,
+                             int64_t n_out, int64_t k_in, const uint16_t* d_x_bf16, int batch, uint16_t* d_y_bf16, void* stream)
+{
+    if (ctx && ctx->device >= 0 && n_out == 0 && batch >= 1 && batch <= 64) return LLVQ_OK;   // nothing to do: pointers may be null
+    if (int e = check_sg(ctx, d_fields, gain_bits, d_codebook_f32, d_row_scale_f32)) return e;
+    if (!d_x_bf16 || !d_y_bf16 || n_out < 0 || k_in < 0 || batch < 1 || batch > 64) return LLVQ_EINVAL;
+    if (!aligned(d_x_bf16, 16) || !aligned(d_y_bf16, 2) || (k_in & 7)) return LLVQ_EALIGN;
+    if (n_out > kMaxScratchRows) return LLVQ_EUNSUPPORTED;
+    const SgArgs sg{d_codebook_f32, d_row_scale_f32, gain_bits};
+    return launch_gemm(ctx, d_fields, nullptr, n_out, k_in, d_x_bf16, batch, d_y_bf16, ctx->d_scratch, ctx->d_counters, stream, &sg);
 }
 
 int llvq_gemm_small_batch(const llvq_ctx* ctx, const void* d_idx, const uint16_t* d_gain_f16, int64_t n_out, int64_t k_in,

@@ -197,3 +197,22 @@ def test_gemv_sorted_sg_full_size_and_limits(lib, ctxs, codes):
     assert ctx._lib.llvq_sort_blocks_sg(ctx._h, buf.data_ptr(), 2, 8, 24, buf.data_ptr(), None) == 3
     assert ctx._lib.llvq_gemv_sorted_sg(ctx._h, buf.data_ptr(), 2, buf.data_ptr(), None, 8, 24, buf.data_ptr(), buf.data_ptr(), 0, None) == 3
     assert lib.llvq_last_error(ctx) == (0, 0)
+
+
+@pytest.mark.parametrize("code,bits,n_out,k_in,batch", [((2, 12), 1, 200, 480, 5), ((2, 10), 4, 129, 1000, 16), ((2, 13), 0, 300, 2000, 40),
+                                                        ((3, 3), 0, 64, 4104, 64)])
+def test_gemm_small_batch_sg(lib, ctxs, codes, code, bits, n_out, k_in, batch):
+    o, ctx = codes[code], ctxs[code]
+    stream, nblocks = gen.make_layer_sg(o.N, o.W, bits, n_out, k_in, seed=41)
+    cb = _codebook(bits)
+    rs = gen.row_scales_f32(n_out, seed=10)
+    x = gen.normal_bf16((batch, k_in), seed=7)
+    ref = o.gemm_sg(stream, bits, cb, rs, n_out, k_in, x, threads=4)
+    y = lib.llvq_gemm_small_batch_sg(ctx, to_dev_u8(stream), bits, _f32(cb), _f32(rs), n_out, k_in, to_dev_bf16(x))
+    torch.cuda.synchronize()
+    assert gemv_error(y.float().cpu().numpy(), ref) <= TOL_BF16_OUT
+    # batch 1 agrees with the fused matrix-vector product
+    y1 = lib.llvq_gemm_small_batch_sg(ctx, to_dev_u8(stream), bits, _f32(cb), _f32(rs), n_out, k_in, to_dev_bf16(x[:1]))
+    yv = lib.llvq_gemv_sg(ctx, to_dev_u8(stream), bits, _f32(cb), _f32(rs), n_out, k_in, to_dev_bf16(x[0]), y_dtype=torch.bfloat16)
+    assert gemv_error(y1[0].float().cpu().numpy(), yv.float().cpu().numpy().astype(np.float64)) <= 2.0 ** -7
+    assert lib.llvq_last_error(ctx) == (0, 0)
