@@ -401,6 +401,34 @@ def extras(P, ctx) -> dict:
     out["gemv_shape_gain_47p1_11008x4096"]["sorted_layout_GBps"] = by12 / us12s / 1e3
     assert P.llvq_last_error(ctx12) == (0, 0)
     del bufs12, srt12, ctx12
+    # --- one rank's step of the row-sharded GEMV at world size 8 on the 11008 x 4096 layer (band of 1376 rows, sorted layout):
+    # band GEMV writing into 8 copies of y, flag stores, bounded wait.  One GPU: all 8 copies and all flag words live
+    # on this device, so the NVLink latency of the remote stores is not in the number.
+    n, k, world = 11008, 4096, 8
+    n_band = n // world
+    bands = []
+    for c in range(112):                                  # 112 x 2.8 MB > 2 x L2
+        stream, gain, nbb = gen.make_layer(CODE_N, CODE_W, n_band, k, 1, seed=700 + c)
+        bands.append((P.llvq_sort_blocks(ctx, dev(stream), n_band, k), dev(gain, np.float16)))
+    xb = dev(gen.normal_bf16(k, seed=70), np.int16).view(torch.bfloat16)
+    copies = [torch.empty(n, dtype=torch.bfloat16, device="cuda") for _ in range(world)]
+    flags = torch.zeros(world, dtype=torch.int32, device="cuda")
+    words = [flags.data_ptr() + 4 * p for p in range(1, world)]
+    epoch = [0]
+
+    def shard_step(i):
+        epoch[0] += 1
+        P.llvq_gemv_sorted_rowshard(ctx, bands[i % 112][0], bands[i % 112][1], n_band, k, xb, copies, 0, 0, torch.bfloat16)
+        P.llvq_signal_ranks(ctx, words, epoch[0])
+        P.llvq_wait_ranks(ctx, flags, world, 0, epoch[0])
+    _event_us(torch, shard_step, 16)
+    us_sh = _event_us(torch, shard_step, 224)
+    band_only = _event_us(torch, lambda i: P.llvq_gemv_sorted(ctx, bands[i % 112][0], bands[i % 112][1], n_band, k, xb, d_y=copies[0]), 224)
+    out["rowshard_world8_rank_step_11008x4096_sorted_layout"] = {
+        "us": us_sh, "band_gemv_alone_us": band_only, "rows_per_rank": n_band, "launches_per_step": 3,
+        "note": "emulated on one GPU: peer copies of y and flag words are local memory"}
+    assert P.llvq_last_error(ctx) == (0, 0)
+    del bands, copies
     # --- encoder: nearest-point search + indexing of a 4096 x 4096 matrix worth of Gaussian blocks (offline step)
     nb_enc = 4096 * 4096 // 24
     torch.manual_seed(0)

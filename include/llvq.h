@@ -280,6 +280,57 @@ int llvq_pack_fields(const llvq_ctx* ctx, const uint64_t* d_index, const uint8_t
                      uint64_t nblocks, void* d_fields, void* stream);
 
 /*
+ * Row-sharded GEMV over several GPUs, one process per GPU (App. A step 5: blocks are independent, so W splits by
+ * output rows with no change to the arithmetic; x is the same on every rank).  A rank owns the band of rows
+ * [row0, row0 + n_rows) of W: d_idx / d_gain_f16 (or d_sorted from llvq_sort_blocks, called with n_out = n_rows)
+ * describe that band alone, ROWWISE, exactly as llvq_gemv / llvq_gemv_sorted take them.  The kernel writes the band's
+ * results into EVERY rank's copy of the full vector: d_y_all is a HOST array of n_dest (1..8) DEVICE pointers, each
+ * the start of a full-length y (element type y_dtype) that the calling process can store to - own_slot names this
+ * rank's own copy, the others are the peers' exchange buffers opened with llvq_exchange_open (the stores cross
+ * NVLink as plain remote writes; nothing is read from a peer).  Row row0 + i of every copy receives what llvq_gemv
+ * would have put in y[i].  Copies may be the same pointer only if n_dest = 1.  Everything else (sizes, alignment,
+ * errors, summation order) as llvq_gemv / llvq_gemv_sorted.  The call only enqueues the kernel; the ranks learn of
+ * each other's completion through llvq_signal_ranks / llvq_wait_ranks below.
+ */
+int llvq_gemv_rowshard(const llvq_ctx* ctx, const void* d_idx, const uint16_t* d_gain_f16, int64_t n_rows, int64_t k_in,
+                       const uint16_t* d_x_bf16, void* const* d_y_all, int n_dest, int own_slot, int64_t row0,
+                       int y_dtype, void* stream);
+int llvq_gemv_sorted_rowshard(const llvq_ctx* ctx, const void* d_sorted, const uint16_t* d_gain_f16, int64_t n_rows,
+                              int64_t k_in, const uint16_t* d_x_bf16, void* const* d_y_all, int n_dest, int own_slot,
+                              int64_t row0, int y_dtype, void* stream);
+
+/*
+ * Exchange buffers for the above (no counterpart in the paper: plumbing between processes).
+ * llvq_exchange_create allocates `bytes` of zeroed device memory on the context's device as an allocation of its
+ * own (so that it can be exported whole), returns it in *d_buf and writes its inter-process handle
+ * (LLVQ_EXCHANGE_HANDLE_BYTES bytes, host) to handle64; the caller carries the handle to the other processes by any
+ * host channel.  llvq_exchange_open maps another PROCESS's buffer (same machine, peer access possible) and returns
+ * the pointer usable on this context's device; llvq_exchange_close unmaps it; llvq_exchange_destroy frees an own
+ * buffer (after every peer has closed it).  These four calls synchronise the device.  LLVQ_ECUDA when the runtime
+ * refuses (for instance a handle opened in the process that made it).
+ */
+#define LLVQ_EXCHANGE_HANDLE_BYTES 64
+int llvq_exchange_create(const llvq_ctx* ctx, size_t bytes, void** d_buf, unsigned char* handle64);
+int llvq_exchange_destroy(const llvq_ctx* ctx, void* d_buf);
+int llvq_exchange_open(const llvq_ctx* ctx, const unsigned char* handle64, void** d_peer_buf);
+int llvq_exchange_close(const llvq_ctx* ctx, void* d_peer_buf);
+
+/*
+ * llvq_signal_ranks: enqueue, after the kernels already on `stream`, a release store of `epoch` to each of the n
+ * (0..8) DEVICE words listed in the HOST array d_flag_words (one word in each peer's exchange buffer, reserved for
+ * this rank as the only writer).  Every store those kernels made, remote ones included, is visible to whoever then
+ * reads the word with acquire semantics and finds the epoch.
+ * llvq_wait_ranks: enqueue a one-warp kernel that waits until the words d_flags[p], p = 0..world-1 except p = skip
+ * (pass -1 to wait on all), own DEVICE memory, 4-byte aligned, have reached `epoch` (modular comparison, so epochs may
+ * wrap).  The wait is bounded: after max_spins polls (0 = the library's limit of about a second; larger values are
+ * clamped to it) the kernel sets LLVQ_FLAG_WAIT_TIMEOUT, which llvq_last_error reports, and returns normally; what
+ * follows on the stream then still runs, on incomplete data, so check the flag before trusting a step.
+ */
+int llvq_signal_ranks(const llvq_ctx* ctx, uint32_t* const* d_flag_words, int n, uint32_t epoch, void* stream);
+int llvq_wait_ranks(const llvq_ctx* ctx, const uint32_t* d_flags, int world, int skip, uint32_t epoch,
+                    uint32_t max_spins, void* stream);
+
+/*
  * Self-test of the error path every kernel of this library uses for its device-side waits (table copy,
  * tensor-core completion): launches a one-warp kernel that waits, with a small iteration limit, on a barrier
  * nothing arrives at, sees the limit run out, sets LLVQ_FLAG_WAIT_TIMEOUT and returns normally.  Nothing

@@ -20,6 +20,8 @@ __all__ = [
     "llvq_encode_blocks", "llvq_rank_blocks", "llvq_pack_fields", "LLVQ_EUCLIDEAN", "LLVQ_ANGULAR",
     "llvq_sort_blocks", "llvq_gemv_sorted", "llvq_sort_blocks_gemm", "llvq_gemm_small_batch_sorted",
     "llvq_sort_blocks_sg", "llvq_gemv_sorted_sg", "llvq_gemm_small_batch_sg",
+    "llvq_gemv_rowshard", "llvq_gemv_sorted_rowshard", "llvq_exchange_create", "llvq_exchange_destroy", "llvq_exchange_open",
+    "llvq_exchange_close", "llvq_signal_ranks", "llvq_wait_ranks", "LLVQ_EXCHANGE_HANDLE_BYTES",
     "llvq_last_error", "LlvqError", "EXPORTS", "load_library",
     "LLVQ_LAYOUT_FLAT", "LLVQ_LAYOUT_ROWWISE", "LLVQ_F32", "LLVQ_BF16",
 ]
@@ -28,6 +30,7 @@ LLVQ_LAYOUT_FLAT, LLVQ_LAYOUT_ROWWISE = 0, 1
 LLVQ_F32, LLVQ_BF16 = 0, 1
 LLVQ_EUCLIDEAN, LLVQ_ANGULAR = 0, 1
 LLVQ_FLAG_WAIT_TIMEOUT, LLVQ_FLAG_SEARCH_GAVE_UP = 1, 4
+LLVQ_EXCHANGE_HANDLE_BYTES = 64
 _STATUS = {0: "LLVQ_OK", 1: "LLVQ_EINVAL", 2: "LLVQ_EALIGN", 3: "LLVQ_EUNSUPPORTED", 4: "LLVQ_ECUDA",
            5: "LLVQ_EINDEX", 6: "LLVQ_ETIMEOUT"}
 
@@ -40,6 +43,8 @@ EXPORTS = [
     "llvq_encode_blocks", "llvq_rank_blocks", "llvq_pack_fields",
     "llvq_sorted_bytes", "llvq_sort_blocks", "llvq_gemv_sorted", "llvq_sort_blocks_sg", "llvq_gemv_sorted_sg",
     "llvq_sorted_gemm_bytes", "llvq_sort_blocks_gemm", "llvq_gemm_small_batch_sorted", "llvq_gemm_small_batch_sg",
+    "llvq_gemv_rowshard", "llvq_gemv_sorted_rowshard", "llvq_exchange_create", "llvq_exchange_destroy", "llvq_exchange_open",
+    "llvq_exchange_close", "llvq_signal_ranks", "llvq_wait_ranks",
 ]
 
 
@@ -96,6 +101,15 @@ def load_library() -> ctypes.CDLL:
     lib.llvq_last_error.argtypes = [vp, vp, ctypes.POINTER(u64), ctypes.POINTER(ctypes.c_uint32)]
     lib.llvq_class_info.argtypes = [vp, ctypes.c_int, vp, vp, vp, vp, vp, vp]
     lib.llvq_golay_table.argtypes = [vp, vp]
+    shard = [vp, vp, vp, i64, i64, vp, ctypes.POINTER(vp), ctypes.c_int, ctypes.c_int, i64, ctypes.c_int, vp]
+    lib.llvq_gemv_rowshard.argtypes = shard
+    lib.llvq_gemv_sorted_rowshard.argtypes = shard
+    lib.llvq_exchange_create.argtypes = [vp, ctypes.c_size_t, ctypes.POINTER(vp), ctypes.c_char_p]
+    lib.llvq_exchange_destroy.argtypes = [vp, vp]
+    lib.llvq_exchange_open.argtypes = [vp, ctypes.c_char_p, ctypes.POINTER(vp)]
+    lib.llvq_exchange_close.argtypes = [vp, vp]
+    lib.llvq_signal_ranks.argtypes = [vp, ctypes.POINTER(vp), ctypes.c_int, ctypes.c_uint32, vp]
+    lib.llvq_wait_ranks.argtypes = [vp, vp, ctypes.c_int, ctypes.c_int, ctypes.c_uint32, ctypes.c_uint32, vp]
     _lib = lib
     return lib
 
@@ -423,6 +437,72 @@ def llvq_pack_fields(ctx: Context, d_index: torch.Tensor, d_gain_index: torch.Te
         ctx._h, _dev(d_index, "d_index"), None if d_gain_index is None or gain_bits == 0 else _dev(d_gain_index, "d_gain_index"),
         gain_bits, n, _dev(d_fields, "d_fields"), _stream_ptr(stream)))
     return d_fields
+
+
+def _ptr(p, name: str) -> int:
+    """A device address given as an int or as a CUDA tensor."""
+    return _dev(p, name) if isinstance(p, torch.Tensor) else int(p)
+
+
+def _gemv_rowshard(call: str, ctx: Context, d_stream, d_gain, n_rows, k_in, d_x, y_all, own_slot, row0, y_dtype, stream):
+    assert d_x.dtype == torch.bfloat16 and d_x.numel() >= k_in and d_gain.dtype == torch.float16
+    assert y_dtype in (torch.float32, torch.bfloat16) and 1 <= len(y_all) <= 8
+    assert d_gain.numel() >= n_rows * ((k_in + 23) // 24)
+    ptrs = (ctypes.c_void_p * len(y_all))(*[_ptr(y, "y_all") for y in y_all])
+    code = LLVQ_F32 if y_dtype == torch.float32 else LLVQ_BF16
+    _check(call, getattr(ctx._lib, call)(ctx._h, _dev(d_stream, "d_stream"), _dev(d_gain, "d_gain"), n_rows, k_in, _dev(d_x, "d_x"),
+                                         ptrs, len(y_all), own_slot, row0, code, _stream_ptr(stream)))
+
+
+def llvq_gemv_rowshard(ctx: Context, d_idx: torch.Tensor, d_gain: torch.Tensor, n_rows: int, k_in: int, d_x: torch.Tensor,
+                       y_all, own_slot: int, row0: int, y_dtype: torch.dtype = torch.float32, stream=None) -> None:
+    """``llvq_gemv`` of one rank's band of rows, written at row ``row0`` of every full-length y in ``y_all``
+    (tensors or device addresses; ``y_all[own_slot]`` is this rank's own copy)."""
+    assert d_idx.numel() * d_idx.element_size() >= ctx.index_bytes(n_rows * ((k_in + 23) // 24))
+    _gemv_rowshard("llvq_gemv_rowshard", ctx, d_idx, d_gain, n_rows, k_in, d_x, y_all, own_slot, row0, y_dtype, stream)
+
+
+def llvq_gemv_sorted_rowshard(ctx: Context, d_sorted: torch.Tensor, d_gain: torch.Tensor, n_rows: int, k_in: int, d_x: torch.Tensor,
+                              y_all, own_slot: int, row0: int, y_dtype: torch.dtype = torch.float32, stream=None) -> None:
+    """``llvq_gemv_rowshard`` from the band's sorted stream (``llvq_sort_blocks`` with n_out = n_rows)."""
+    assert d_sorted.numel() * d_sorted.element_size() >= int(ctx._lib.llvq_sorted_bytes(ctx._h, n_rows, k_in))
+    _gemv_rowshard("llvq_gemv_sorted_rowshard", ctx, d_sorted, d_gain, n_rows, k_in, d_x, y_all, own_slot, row0, y_dtype, stream)
+
+
+def llvq_exchange_create(ctx: Context, nbytes: int) -> tuple[int, bytes]:
+    """(device address of a new zeroed exchange buffer, its 64-byte inter-process handle)."""
+    buf = ctypes.c_void_p()
+    handle = ctypes.create_string_buffer(LLVQ_EXCHANGE_HANDLE_BYTES)
+    _check("llvq_exchange_create", ctx._lib.llvq_exchange_create(ctx._h, nbytes, ctypes.byref(buf), handle))
+    return int(buf.value), handle.raw
+
+
+def llvq_exchange_destroy(ctx: Context, d_buf: int) -> None:
+    _check("llvq_exchange_destroy", ctx._lib.llvq_exchange_destroy(ctx._h, d_buf))
+
+
+def llvq_exchange_open(ctx: Context, handle: bytes) -> int:
+    """Device address, in this process, of another process's exchange buffer."""
+    assert len(handle) == LLVQ_EXCHANGE_HANDLE_BYTES
+    buf = ctypes.c_void_p()
+    _check("llvq_exchange_open", ctx._lib.llvq_exchange_open(ctx._h, handle, ctypes.byref(buf)))
+    return int(buf.value)
+
+
+def llvq_exchange_close(ctx: Context, d_peer_buf: int) -> None:
+    _check("llvq_exchange_close", ctx._lib.llvq_exchange_close(ctx._h, d_peer_buf))
+
+
+def llvq_signal_ranks(ctx: Context, flag_words, epoch: int, stream=None) -> None:
+    """After the work already on the stream, store ``epoch`` to each device word in ``flag_words`` (addresses)."""
+    ptrs = (ctypes.c_void_p * max(len(flag_words), 1))(*[_ptr(w, "flag_words") for w in flag_words])
+    _check("llvq_signal_ranks", ctx._lib.llvq_signal_ranks(ctx._h, ptrs, len(flag_words), epoch & 0xffffffff, _stream_ptr(stream)))
+
+
+def llvq_wait_ranks(ctx: Context, d_flags, world: int, skip: int, epoch: int, max_spins: int = 0, stream=None) -> None:
+    """Bounded device-side wait until the words d_flags[p], p != skip, reach ``epoch``; expiry sets LLVQ_FLAG_WAIT_TIMEOUT."""
+    _check("llvq_wait_ranks", ctx._lib.llvq_wait_ranks(ctx._h, _ptr(d_flags, "d_flags"), world, skip, epoch & 0xffffffff, max_spins,
+                                                       _stream_ptr(stream)))
 
 
 def llvq_selftest_wait_timeout(ctx: Context, stream=None) -> None:

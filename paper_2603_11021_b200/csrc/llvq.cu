@@ -221,22 +221,117 @@ __device__ __forceinline__ void mma_bf16_16816(float c[4], uint32_t a0, uint32_t
 // CTA that owns unit u when G CTAs split U units into ranges [c*U/G, (c+1)*U/G).
 __device__ __forceinline__ int64_t unit_owner(int64_t u, int64_t U, int64_t G) { return ((u + 1) * G - 1) / U; }
 
+// Where a GEMV kernel puts y.  Row-sharded over several GPUs (each rank owns a band of output rows, x is the same
+// everywhere), a rank writes its band straight into every rank's copy of the full vector: `y` is this rank's copy
+// and `peer` the other ranks' copies mapped into this process, every pointer already advanced to the band's first
+// row.  The stores to a peer travel over NVLink as plain remote writes.  n_peer = 0 is the single-GPU case.
+constexpr int kMaxShardPeers = 7;
+struct YOut {
+    void* y;
+    void* peer[kMaxShardPeers];
+    int n_peer;
+};
+
+template <bool kOutBf16>
+__device__ __forceinline__ void store_y(const YOut& yo, int64_t row, float v)
+{
+    if (kOutBf16) {
+        const __nv_bfloat16 h = __float2bfloat16_rn(v);
+        reinterpret_cast<__nv_bfloat16*>(yo.y)[row] = h;
+#pragma unroll
+        for (int p = 0; p < kMaxShardPeers; ++p)          // static indices: the struct stays in the parameter bank
+            if (p < yo.n_peer) reinterpret_cast<__nv_bfloat16*>(yo.peer[p])[row] = h;
+    } else {
+        reinterpret_cast<float*>(yo.y)[row] = v;
+#pragma unroll
+        for (int p = 0; p < kMaxShardPeers; ++p)
+            if (p < yo.n_peer) reinterpret_cast<float*>(yo.peer[p])[row] = v;
+    }
+}
+
+// Stages x for a GEMV CTA: xs[cb * 12 + j] = the bf16 pair (x[24 cb + 2j], x[24 cb + 2j + 1]), zero beyond k_in; `words`
+// = 12 x the number of column blocks staged.  16-byte loads where x allows them.
+__device__ __forceinline__ void stage_x(uint32_t* xs, const uint16_t* __restrict__ x, int64_t k_in, int64_t words)
+{
+    if ((reinterpret_cast<uintptr_t>(x) & 15) == 0) {
+        const int64_t full = k_in / 8;                                       // whole groups of 8 elements
+        for (int64_t v = threadIdx.x; v < words / 4; v += blockDim.x) {
+            uint4 q = make_uint4(0u, 0u, 0u, 0u);
+            if (v < full) q = __ldg(reinterpret_cast<const uint4*>(x) + v);
+            else {
+                uint32_t t[4];
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    const int64_t e = 8 * v + 2 * j;
+                    const uint32_t lo = e < k_in ? __ldg(x + e) : 0u, hi = e + 1 < k_in ? __ldg(x + e + 1) : 0u;
+                    t[j] = lo | hi << 16;
+                }
+                q = make_uint4(t[0], t[1], t[2], t[3]);
+            }
+            reinterpret_cast<uint4*>(xs)[v] = q;
+        }
+        return;
+    }
+    for (int64_t i = threadIdx.x; i < words; i += blockDim.x) {
+        const int64_t e = 2 * i;
+        const uint32_t lo = e < k_in ? __ldg(x + e) : 0u, hi = e + 1 < k_in ? __ldg(x + e + 1) : 0u;
+        xs[i] = lo | hi << 16;
+    }
+}
+
+// End of a pass of a GEMV CTA over row groups rg0..rg1 (8 rows each; the CTA owns units [u_begin, u_end) of U, nq
+// units per row group, G CTAs): row_sum(i) is the CTA's sum for row i of the pass.  One warp per row group, lanes
+// 0..7 its rows, no CTA-wide barrier inside.  A group the CTA covers completely is final.  A group it shares with
+// neighbouring CTAs goes through the scratch row in global memory: add, make the add visible, count the arrival;
+// whoever arrives last reads the total, writes y and leaves scratch and counter zero for the next launch.
+// The caller puts a __syncthreads() before (sums complete) and after (sums may be cleared) the call.
+template <bool kOutBf16, typename RowSum>
+__device__ __forceinline__ void finish_pass(const YOut& yo, int64_t rg0, int64_t rg1, int64_t nq, int64_t u_begin, int64_t u_end,
+                                            int64_t U, int64_t G, int64_t n_out, float* __restrict__ scratch,
+                                            uint32_t* __restrict__ counters, RowSum row_sum)
+{
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, nwarps = (int)(blockDim.x >> 5);
+    for (int64_t rg = rg0 + warp; rg <= rg1; rg += nwarps) {
+        const bool whole = u_begin <= rg * nq && (rg + 1) * nq <= u_end;
+        const int64_t row = rg * kGemvGroupRows + lane;
+        const bool mine = lane < kGemvGroupRows && row < n_out;
+        const float part = lane < kGemvGroupRows ? row_sum((rg - rg0) * kGemvGroupRows + lane) : 0.f;
+        if (whole) {
+            if (mine) store_y<kOutBf16>(yo, row, part);
+            continue;
+        }
+        if (mine) atomicAdd(scratch + row, part);
+        __threadfence();                               // every lane's add is performed before ...
+        __syncwarp();
+        uint32_t is_last = 0u;
+        if (lane == 0) {
+            __threadfence();                           // ... lane 0 counts the arrival
+            const uint32_t parts = (uint32_t)(unit_owner((rg + 1) * nq - 1, U, G) - unit_owner(rg * nq, U, G) + 1);
+            is_last = atomicAdd(counters + rg, 1u) == parts - 1u;
+        }
+        is_last = __shfl_sync(kFullMask, is_last, 0);
+        if (is_last) {
+            __threadfence();
+            if (mine) {
+                store_y<kOutBf16>(yo, row, __ldcg(scratch + row));
+                __stcg(scratch + row, 0.f);
+            }
+            if (lane == 0) counters[rg] = 0u;
+        }
+    }
+}
+
 template <bool kBig, bool kOutBf16, bool kSg = false>
 __global__ void __launch_bounds__(kGemvThreads, 1)
 gemv_fast_kernel(FastArgs fa, const uint32_t* __restrict__ stream, const uint16_t* __restrict__ gain, SgArgs sg,
-                 int64_t n_out, int64_t k_in, int64_t bpr, const uint16_t* __restrict__ x, void* __restrict__ y,
+                 int64_t n_out, int64_t k_in, int64_t bpr, const uint16_t* __restrict__ x, YOut yo,
                  float* __restrict__ scratch, uint32_t* __restrict__ counters)
 {
     FAST_PROLOGUE();
     const int64_t nq = (bpr + 3) / 4;                               // units along K
     uint32_t* xs = reinterpret_cast<uint32_t*>(staging);            // [nq * 4][12] packed bf16 pairs of x
     float* acc = reinterpret_cast<float*>(xs + nq * 48);            // [kGemvGroupsPerPass][8]
-    uint32_t* last_flag = reinterpret_cast<uint32_t*>(acc + kGemvGroupsPerPass * kGemvGroupRows);
-    for (int64_t i = threadIdx.x; i < nq * 48; i += blockDim.x) {
-        const int64_t e = 2 * i;
-        const uint32_t lo = e < k_in ? __ldg(x + e) : 0u, hi = e + 1 < k_in ? __ldg(x + e + 1) : 0u;
-        xs[i] = lo | hi << 16;
-    }
+    stage_x(xs, x, k_in, nq * 48);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, g = lane >> 2, t = lane & 3;
     const int kWarps = (int)(blockDim.x >> 5);
     const int64_t groups = (n_out + kGemvGroupRows - 1) / kGemvGroupRows;
@@ -270,38 +365,7 @@ gemv_fast_kernel(FastArgs fa, const uint32_t* __restrict__ stream, const uint16_
         }
         __syncthreads();
         // row groups this CTA covers completely are final; the (at most two) split ones go through the scratch
-        for (int64_t rg = rg0; rg <= rg1; ++rg) {
-            const bool whole = u_begin <= rg * nq && (rg + 1) * nq <= u_end;
-            const int64_t row = rg * kGemvGroupRows + threadIdx.x;
-            const bool mine = threadIdx.x < kGemvGroupRows && row < n_out;
-            if (whole) {
-                if (mine) {
-                    const float v = acc[(rg - rg0) * kGemvGroupRows + threadIdx.x];
-                    if (kOutBf16) reinterpret_cast<__nv_bfloat16*>(y)[row] = __float2bfloat16_rn(v);
-                    else reinterpret_cast<float*>(y)[row] = v;
-                }
-                continue;
-            }
-            if (mine) atomicAdd(scratch + row, acc[(rg - rg0) * kGemvGroupRows + threadIdx.x]);
-            __threadfence();
-            __syncthreads();
-            if (threadIdx.x == 0) {
-                const uint32_t parts = (uint32_t)(unit_owner((rg + 1) * nq - 1, U, G) - unit_owner(rg * nq, U, G) + 1);
-                *last_flag = atomicAdd(counters + rg, 1u) == parts - 1u;
-            }
-            __syncthreads();
-            if (*last_flag) {
-                __threadfence();
-                if (mine) {
-                    const float v = __ldcg(scratch + row);
-                    if (kOutBf16) reinterpret_cast<__nv_bfloat16*>(y)[row] = __float2bfloat16_rn(v);
-                    else reinterpret_cast<float*>(y)[row] = v;
-                    __stcg(scratch + row, 0.f);
-                }
-                if (threadIdx.x == 0) counters[rg] = 0u;
-            }
-            __syncthreads();
-        }
+        finish_pass<kOutBf16>(yo, rg0, rg1, nq, u_begin, u_end, U, G, n_out, scratch, counters, [&](int64_t r) { return acc[r]; });
         __syncthreads();                                   // the sums are read above: the next pass may clear them only now
     }
 }
@@ -435,7 +499,7 @@ __device__ __forceinline__ uint32_t decode_sorted_entry(const FastArgs& fa, cons
 template <bool kOutBf16, bool kSg = false>
 __global__ void __launch_bounds__(kSortThreads, 1)
 gemv_sorted_kernel(FastArgs fa, const unsigned long long* __restrict__ sorted, const uint16_t* __restrict__ gain, SgArgs sg,
-                   int64_t n_out, int64_t k_in, int64_t bpr, uint32_t nq_magic, const uint16_t* __restrict__ x, void* __restrict__ y,
+                   int64_t n_out, int64_t k_in, int64_t bpr, uint32_t nq_magic, const uint16_t* __restrict__ x, YOut yo,
                    float* __restrict__ scratch, uint32_t* __restrict__ counters)
 {
     FAST_PROLOGUE();
@@ -444,11 +508,7 @@ gemv_sorted_kernel(FastArgs fa, const unsigned long long* __restrict__ sorted, c
     float* acc = reinterpret_cast<float*>(xs + nq * 48);            // [kSortAccCopies][kGemvGroupsPerPass][8]: warps spread their adds over the copies
     uint32_t* last_flag = reinterpret_cast<uint32_t*>(acc + kSortAccCopies * kGemvGroupsPerPass * kGemvGroupRows);
     uint32_t* next_chunk = last_flag + 1;
-    for (int64_t i = threadIdx.x; i < nq * 48; i += blockDim.x) {
-        const int64_t e = 2 * i;
-        const uint32_t lo = e < k_in ? __ldg(x + e) : 0u, hi = e + 1 < k_in ? __ldg(x + e + 1) : 0u;
-        xs[i] = lo | hi << 16;
-    }
+    stage_x(xs, x, k_in, nq * 48);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const uint32_t kWarps = blockDim.x >> 5;
     const int64_t groups = (n_out + kGemvGroupRows - 1) / kGemvGroupRows;
@@ -515,38 +575,7 @@ gemv_sorted_kernel(FastArgs fa, const unsigned long long* __restrict__ sorted, c
             for (int c = 0; c < kSortAccCopies; ++c) v += acc[c * (kGemvGroupsPerPass * kGemvGroupRows) + r];
             return v;
         };
-        for (int64_t rg = rg0; rg <= rg1; ++rg) {
-            const bool whole = u_begin <= rg * nq && (rg + 1) * nq <= u_end;
-            const int64_t row = rg * kGemvGroupRows + threadIdx.x;
-            const bool mine = threadIdx.x < kGemvGroupRows && row < n_out;
-            if (whole) {
-                if (mine) {
-                    const float v = row_sum((rg - rg0) * kGemvGroupRows + threadIdx.x);
-                    if (kOutBf16) reinterpret_cast<__nv_bfloat16*>(y)[row] = __float2bfloat16_rn(v);
-                    else reinterpret_cast<float*>(y)[row] = v;
-                }
-                continue;
-            }
-            if (mine) atomicAdd(scratch + row, row_sum((rg - rg0) * kGemvGroupRows + threadIdx.x));
-            __threadfence();
-            __syncthreads();
-            if (threadIdx.x == 0) {
-                const uint32_t parts = (uint32_t)(unit_owner((rg + 1) * nq - 1, U, G) - unit_owner(rg * nq, U, G) + 1);
-                *last_flag = atomicAdd(counters + rg, 1u) == parts - 1u;
-            }
-            __syncthreads();
-            if (*last_flag) {
-                __threadfence();
-                if (mine) {
-                    const float v = __ldcg(scratch + row);
-                    if (kOutBf16) reinterpret_cast<__nv_bfloat16*>(y)[row] = __float2bfloat16_rn(v);
-                    else reinterpret_cast<float*>(y)[row] = v;
-                    __stcg(scratch + row, 0.f);
-                }
-                if (threadIdx.x == 0) counters[rg] = 0u;
-            }
-            __syncthreads();
-        }
+        finish_pass<kOutBf16>(yo, rg0, rg1, nq, u_begin, u_end, U, G, n_out, scratch, counters, row_sum);
         __syncthreads();                                   // the sums are read above: the next pass may clear them only now
     });
 }
@@ -564,7 +593,7 @@ constexpr int kBinPerThread = kBinSegUnits * 32 / kSortThreads;   // 8
 template <bool kOutBf16, bool kSg = false>
 __global__ void __launch_bounds__(kSortThreads, 1)
 gemv_bin_kernel(FastArgs fa, const uint32_t* __restrict__ stream, const uint16_t* __restrict__ sort_rank, const uint16_t* __restrict__ gain, SgArgs sg,
-                int64_t n_out, int64_t k_in, int64_t bpr, uint32_t nq_magic, int seg_units, const uint16_t* __restrict__ x, void* __restrict__ y,
+                int64_t n_out, int64_t k_in, int64_t bpr, uint32_t nq_magic, int seg_units, const uint16_t* __restrict__ x, YOut yo,
                 float* __restrict__ scratch, uint32_t* __restrict__ counters)
 {
     FAST_PROLOGUE();
@@ -577,11 +606,7 @@ gemv_bin_kernel(FastArgs fa, const uint32_t* __restrict__ stream, const uint16_t
     uint32_t* cursor = hist + 1024;                                  // [1024]
     unsigned long long* ent = reinterpret_cast<unsigned long long*>(cursor + 1024);   // [seg_units * 32] class-local index | position << 48
     uint16_t* ent_cls = reinterpret_cast<uint16_t*>(ent + seg_units * 32);            // [seg_units * 32] class (| gain index << 10), 0xffff = no block
-    for (int64_t i = threadIdx.x; i < nq * 48; i += blockDim.x) {
-        const int64_t e = 2 * i;
-        const uint32_t lo = e < k_in ? __ldg(x + e) : 0u, hi = e + 1 < k_in ? __ldg(x + e + 1) : 0u;
-        xs[i] = lo | hi << 16;
-    }
+    stage_x(xs, x, k_in, nq * 48);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const uint32_t kWarps = blockDim.x >> 5;
     const int64_t groups = (n_out + kGemvGroupRows - 1) / kGemvGroupRows;
@@ -711,38 +736,7 @@ gemv_bin_kernel(FastArgs fa, const uint32_t* __restrict__ stream, const uint16_t
             for (int c = 0; c < kSortAccCopies; ++c) v += acc[c * (kGemvGroupsPerPass * kGemvGroupRows) + r];
             return v;
         };
-        for (int64_t rg = rg0; rg <= rg1; ++rg) {
-            const bool whole = u_begin <= rg * nq && (rg + 1) * nq <= u_end;
-            const int64_t row = rg * kGemvGroupRows + threadIdx.x;
-            const bool mine = threadIdx.x < kGemvGroupRows && row < n_out;
-            if (whole) {
-                if (mine) {
-                    const float v = row_sum((rg - rg0) * kGemvGroupRows + threadIdx.x);
-                    if (kOutBf16) reinterpret_cast<__nv_bfloat16*>(y)[row] = __float2bfloat16_rn(v);
-                    else reinterpret_cast<float*>(y)[row] = v;
-                }
-                continue;
-            }
-            if (mine) atomicAdd(scratch + row, row_sum((rg - rg0) * kGemvGroupRows + threadIdx.x));
-            __threadfence();
-            __syncthreads();
-            if (threadIdx.x == 0) {
-                const uint32_t parts = (uint32_t)(unit_owner((rg + 1) * nq - 1, U, G) - unit_owner(rg * nq, U, G) + 1);
-                *last_flag = atomicAdd(counters + rg, 1u) == parts - 1u;
-            }
-            __syncthreads();
-            if (*last_flag) {
-                __threadfence();
-                if (mine) {
-                    const float v = __ldcg(scratch + row);
-                    if (kOutBf16) reinterpret_cast<__nv_bfloat16*>(y)[row] = __float2bfloat16_rn(v);
-                    else reinterpret_cast<float*>(y)[row] = v;
-                    __stcg(scratch + row, 0.f);
-                }
-                if (threadIdx.x == 0) counters[rg] = 0u;
-            }
-            __syncthreads();
-        }
+        finish_pass<kOutBf16>(yo, rg0, rg1, nq, u_begin, u_end, U, G, n_out, scratch, counters, row_sum);
         __syncthreads();
     }, seg_units);
 }
@@ -1468,19 +1462,44 @@ int llvq_dequant_matrix(const llvq_ctx* ctx, const void* d_idx, const uint16_t* 
     return launch_status();
 }
 
-// Shared by llvq_gemv and llvq_gemv_sg: exactly one of d_gain_f16 / sg is used.
-static int gemv_common(const llvq_ctx* ctx, const void* d_idx, const uint16_t* d_gain_f16, const SgArgs* sg, int64_t n_out, int64_t k_in,
-                       const uint16_t* d_x_bf16, void* d_y, int y_dtype, void* stream)
+// Checks the destinations of a GEMV: every pointer present and aligned for the output type.
+static int check_yout(const YOut& yo, int y_dtype)
 {
-    if (!d_x_bf16 || !d_y || n_out < 0 || k_in < 0) return LLVQ_EINVAL;
     if (y_dtype != LLVQ_F32 && y_dtype != LLVQ_BF16) return LLVQ_EINVAL;
-    if (!aligned(d_x_bf16, 2) || !aligned(d_y, y_dtype == LLVQ_F32 ? 4 : 2)) return LLVQ_EALIGN;
+    if (!yo.y || yo.n_peer < 0 || yo.n_peer > kMaxShardPeers) return LLVQ_EINVAL;
+    const size_t a = y_dtype == LLVQ_F32 ? 4 : 2;
+    if (!aligned(yo.y, a)) return LLVQ_EALIGN;
+    for (int p = 0; p < yo.n_peer; ++p) {
+        if (!yo.peer[p]) return LLVQ_EINVAL;
+        if (!aligned(yo.peer[p], a)) return LLVQ_EALIGN;
+    }
+    return LLVQ_OK;
+}
+
+static YOut single_y(void* d_y)
+{
+    YOut yo{};
+    yo.y = d_y;
+    return yo;
+}
+
+// Shared by llvq_gemv, llvq_gemv_sg and llvq_gemv_rowshard: exactly one of d_gain_f16 / sg is used.
+static int gemv_common(const llvq_ctx* ctx, const void* d_idx, const uint16_t* d_gain_f16, const SgArgs* sg, int64_t n_out, int64_t k_in,
+                       const uint16_t* d_x_bf16, const YOut& yo, int y_dtype, void* stream)
+{
+    if (!d_x_bf16 || n_out < 0 || k_in < 0) return LLVQ_EINVAL;
+    if (int e = check_yout(yo, y_dtype)) return e;
+    if (!aligned(d_x_bf16, 2)) return LLVQ_EALIGN;
     if (n_out == 0) return LLVQ_OK;
     DeviceGuard guard(ctx->device);
     if (!guard.ok) return LLVQ_ECUDA;
     cudaStream_t st = (cudaStream_t)stream;
     if (k_in == 0) {
-        return cudaMemsetAsync(d_y, 0, (size_t)n_out * (y_dtype == LLVQ_F32 ? 4 : 2), st) == cudaSuccess ? LLVQ_OK : LLVQ_ECUDA;
+        const size_t bytes = (size_t)n_out * (y_dtype == LLVQ_F32 ? 4 : 2);
+        if (cudaMemsetAsync(yo.y, 0, bytes, st) != cudaSuccess) return LLVQ_ECUDA;
+        for (int p = 0; p < yo.n_peer; ++p)
+            if (cudaMemsetAsync(yo.peer[p], 0, bytes, st) != cudaSuccess) return LLVQ_ECUDA;
+        return LLVQ_OK;
     }
     const int64_t bpr = (k_in + 23) / 24;
     const int64_t nq = (bpr + 3) / 4;
@@ -1514,7 +1533,7 @@ static int gemv_common(const llvq_ctx* ctx, const void* d_idx, const uint16_t* d
     do {                                                                                                                   \
         if (!set_smem(gemv_bin_kernel<BF16, SG>, smem_bin)) return LLVQ_ECUDA;                                              \
         if (launch_pdl(gemv_bin_kernel<BF16, SG>, g, (unsigned)kSortThreads, smem_bin, st, fa, idx, ctx->d_sort_rank, d_gain_f16, sga, n_out, k_in, \
-                       bpr, magic, seg_units, d_x_bf16, d_y, ctx->d_scratch, ctx->d_counters) != cudaSuccess) return LLVQ_ECUDA; \
+                       bpr, magic, seg_units, d_x_bf16, yo, ctx->d_scratch, ctx->d_counters) != cudaSuccess) return LLVQ_ECUDA; \
     } while (0)
         if (sg) { if (y_dtype == LLVQ_BF16) LLVQ_LAUNCH_BIN(true, true); else LLVQ_LAUNCH_BIN(false, true); }
         else    { if (y_dtype == LLVQ_BF16) LLVQ_LAUNCH_BIN(true, false); else LLVQ_LAUNCH_BIN(false, false); }
@@ -1524,7 +1543,7 @@ static int gemv_common(const llvq_ctx* ctx, const void* d_idx, const uint16_t* d
 #define LLVQ_LAUNCH_GEMV(BIG, BF16, SG)                                                                            \
     do {                                                                                                           \
         if (!set_smem(gemv_fast_kernel<BIG, BF16, SG>, smem)) return LLVQ_ECUDA;                                   \
-        if (launch_pdl(gemv_fast_kernel<BIG, BF16, SG>, g, threads, smem, st, fa, idx, d_gain_f16, sga, n_out, k_in, bpr, d_x_bf16, d_y, \
+        if (launch_pdl(gemv_fast_kernel<BIG, BF16, SG>, g, threads, smem, st, fa, idx, d_gain_f16, sga, n_out, k_in, bpr, d_x_bf16, yo, \
                        ctx->d_scratch, ctx->d_counters) != cudaSuccess) return LLVQ_ECUDA;                         \
     } while (0)
     if (sg)             { if (y_dtype == LLVQ_BF16) LLVQ_LAUNCH_GEMV(false, true, true);  else LLVQ_LAUNCH_GEMV(false, false, true); }
@@ -1541,7 +1560,7 @@ int llvq_gemv(const llvq_ctx* ctx, const void* d_idx, const uint16_t* d_gain_f16
     if (int e = check_common(ctx, d_idx)) return e;
     if (!d_gain_f16) return LLVQ_EINVAL;
     if (!aligned(d_gain_f16, 2)) return LLVQ_EALIGN;
-    return gemv_common(ctx, d_idx, d_gain_f16, nullptr, n_out, k_in, d_x_bf16, d_y, y_dtype, stream);
+    return gemv_common(ctx, d_idx, d_gain_f16, nullptr, n_out, k_in, d_x_bf16, single_y(d_y), y_dtype, stream);
 }
 
 // Argument checks of the shape-gain entry points.
@@ -1589,7 +1608,7 @@ int llvq_gemv_sg(const llvq_ctx* ctx, const void* d_fields, int gain_bits, const
     if (ctx && ctx->device >= 0 && n_out == 0) return LLVQ_OK;                     // nothing to do: pointers may be null
     if (int e = check_sg(ctx, d_fields, gain_bits, d_codebook_f32, d_row_scale_f32)) return e;
     const SgArgs sg{d_codebook_f32, d_row_scale_f32, gain_bits};
-    return gemv_common(ctx, d_fields, nullptr, &sg, n_out, k_in, d_x_bf16, d_y, y_dtype, stream);
+    return gemv_common(ctx, d_fields, nullptr, &sg, n_out, k_in, d_x_bf16, single_y(d_y), y_dtype, stream);
 }
 
 // Sorted layout (see the comment at sort_blocks_kernel).  Available for fast-path codes whose indices fit 48 bits
@@ -1639,11 +1658,11 @@ int llvq_sort_blocks_sg(const llvq_ctx* ctx, const void* d_fields, int gain_bits
 
 // Exactly one of d_gain_f16 / sg is used.
 static int gemv_sorted_common(const llvq_ctx* ctx, const void* d_sorted, const uint16_t* d_gain_f16, const SgArgs* sg, int64_t n_out, int64_t k_in,
-                              const uint16_t* d_x_bf16, void* d_y, int y_dtype, void* stream)
+                              const uint16_t* d_x_bf16, const YOut& yo, int y_dtype, void* stream)
 {
-    if (!d_x_bf16 || !d_y || n_out < 0 || k_in <= 0) return LLVQ_EINVAL;
-    if (y_dtype != LLVQ_F32 && y_dtype != LLVQ_BF16) return LLVQ_EINVAL;
-    if (!aligned(d_x_bf16, 2) || !aligned(d_y, y_dtype == LLVQ_F32 ? 4 : 2)) return LLVQ_EALIGN;
+    if (!d_x_bf16 || n_out < 0 || k_in <= 0) return LLVQ_EINVAL;
+    if (int e = check_yout(yo, y_dtype)) return e;
+    if (!aligned(d_x_bf16, 2)) return LLVQ_EALIGN;
     if (!sortable(ctx, k_in) || n_out > 64ll * kMaxScratchRows) return LLVQ_EUNSUPPORTED;
     DeviceGuard guard(ctx->device);
     if (!guard.ok) return LLVQ_ECUDA;
@@ -1659,7 +1678,7 @@ static int gemv_sorted_common(const llvq_ctx* ctx, const void* d_sorted, const u
     do {                                                                                                                \
         if (!set_smem(gemv_sorted_kernel<BF16, SG>, smem)) return LLVQ_ECUDA;                                            \
         if (launch_pdl(gemv_sorted_kernel<BF16, SG>, g, (unsigned)kSortThreads, smem, st, fast_args(ctx), sp, d_gain_f16, sga, n_out, k_in, bpr, \
-                       magic, d_x_bf16, d_y, ctx->d_scratch, ctx->d_counters) != cudaSuccess) return LLVQ_ECUDA;          \
+                       magic, d_x_bf16, yo, ctx->d_scratch, ctx->d_counters) != cudaSuccess) return LLVQ_ECUDA;          \
     } while (0)
     if (sg) { if (y_dtype == LLVQ_BF16) LLVQ_LAUNCH_SORTED(true, true); else LLVQ_LAUNCH_SORTED(false, true); }
     else    { if (y_dtype == LLVQ_BF16) LLVQ_LAUNCH_SORTED(true, false); else LLVQ_LAUNCH_SORTED(false, false); }
@@ -1674,7 +1693,7 @@ int llvq_gemv_sorted(const llvq_ctx* ctx, const void* d_sorted, const uint16_t* 
     if (int e = check_common(ctx, d_sorted)) return e;
     if (!d_gain_f16) return LLVQ_EINVAL;
     if (!aligned(d_gain_f16, 2)) return LLVQ_EALIGN;
-    return gemv_sorted_common(ctx, d_sorted, d_gain_f16, nullptr, n_out, k_in, d_x_bf16, d_y, y_dtype, stream);
+    return gemv_sorted_common(ctx, d_sorted, d_gain_f16, nullptr, n_out, k_in, d_x_bf16, single_y(d_y), y_dtype, stream);
 }
 
 int llvq_gemv_sorted_sg(const llvq_ctx* ctx, const void* d_sorted, int gain_bits, const float* d_codebook_f32, const float* d_row_scale_f32,
@@ -1684,7 +1703,49 @@ int llvq_gemv_sorted_sg(const llvq_ctx* ctx, const void* d_sorted, int gain_bits
     if (int e = check_sg(ctx, d_sorted, gain_bits, d_codebook_f32, d_row_scale_f32)) return e;
     if (ctx->host.W + gain_bits > 48) return LLVQ_EUNSUPPORTED;
     const SgArgs sg{d_codebook_f32, d_row_scale_f32, gain_bits};
-    return gemv_sorted_common(ctx, d_sorted, nullptr, &sg, n_out, k_in, d_x_bf16, d_y, y_dtype, stream);
+    return gemv_sorted_common(ctx, d_sorted, nullptr, &sg, n_out, k_in, d_x_bf16, single_y(d_y), y_dtype, stream);
+}
+
+// Row-sharded GEMV: the destinations of one rank's band.  d_y_all[0..n_dest) are the ranks' full-length copies of y
+// (own_slot = this rank's own copy), the band starts at row row0.
+static int shard_yout(void* const* d_y_all, int n_dest, int own_slot, int64_t row0, int y_dtype, YOut* yo)
+{
+    if (!d_y_all || n_dest < 1 || n_dest > kMaxShardPeers + 1 || own_slot < 0 || own_slot >= n_dest || row0 < 0) return LLVQ_EINVAL;
+    if (y_dtype != LLVQ_F32 && y_dtype != LLVQ_BF16) return LLVQ_EINVAL;
+    const size_t es = y_dtype == LLVQ_F32 ? 4 : 2;
+    *yo = YOut{};
+    for (int d = 0; d < n_dest; ++d) {
+        if (!d_y_all[d]) return LLVQ_EINVAL;
+        void* at = static_cast<unsigned char*>(d_y_all[d]) + (size_t)row0 * es;
+        if (d == own_slot) yo->y = at;
+        else yo->peer[yo->n_peer++] = at;
+    }
+    return LLVQ_OK;
+}
+
+int llvq_gemv_rowshard(const llvq_ctx* ctx, const void* d_idx, const uint16_t* d_gain_f16, int64_t n_rows, int64_t k_in,
+                       const uint16_t* d_x_bf16, void* const* d_y_all, int n_dest, int own_slot, int64_t row0, int y_dtype, void* stream)
+{
+    YOut yo;
+    if (int e = shard_yout(d_y_all, n_dest, own_slot, row0, y_dtype, &yo)) return e;
+    if (ctx && ctx->device >= 0 && n_rows == 0) return LLVQ_OK;
+    if (int e = check_common(ctx, d_idx)) return e;
+    if (!d_gain_f16) return LLVQ_EINVAL;
+    if (!aligned(d_gain_f16, 2)) return LLVQ_EALIGN;
+    return gemv_common(ctx, d_idx, d_gain_f16, nullptr, n_rows, k_in, d_x_bf16, yo, y_dtype, stream);
+}
+
+int llvq_gemv_sorted_rowshard(const llvq_ctx* ctx, const void* d_sorted, const uint16_t* d_gain_f16, int64_t n_rows, int64_t k_in,
+                              const uint16_t* d_x_bf16, void* const* d_y_all, int n_dest, int own_slot, int64_t row0, int y_dtype,
+                              void* stream)
+{
+    YOut yo;
+    if (int e = shard_yout(d_y_all, n_dest, own_slot, row0, y_dtype, &yo)) return e;
+    if (ctx && ctx->device >= 0 && n_rows == 0) return LLVQ_OK;
+    if (int e = check_common(ctx, d_sorted)) return e;
+    if (!d_gain_f16) return LLVQ_EINVAL;
+    if (!aligned(d_gain_f16, 2)) return LLVQ_EALIGN;
+    return gemv_sorted_common(ctx, d_sorted, d_gain_f16, nullptr, n_rows, k_in, d_x_bf16, yo, y_dtype, stream);
 }
 
 // Sorted layout of the small-batch GEMM (see the comment at sort_blocks_gemm_kernel).
