@@ -402,7 +402,7 @@ def extras(P, ctx) -> dict:
     assert P.llvq_last_error(ctx12) == (0, 0)
     del bufs12, srt12, ctx12
     # --- one rank's step of the row-sharded GEMV at world size 8 on the 11008 x 4096 layer (band of 1376 rows, sorted layout):
-    # band GEMV writing into 8 copies of y, flag stores, bounded wait.  One GPU: all 8 copies and all flag words live
+    # band GEMV writing into 8 copies of y and raising the flags, then the bounded wait.  One GPU: all 8 copies and all flag words live
     # on this device, so the NVLink latency of the remote stores is not in the number.
     n, k, world = 11008, 4096, 8
     n_band = n // world
@@ -413,19 +413,19 @@ def extras(P, ctx) -> dict:
     xb = dev(gen.normal_bf16(k, seed=70), np.int16).view(torch.bfloat16)
     copies = [torch.empty(n, dtype=torch.bfloat16, device="cuda") for _ in range(world)]
     flags = torch.zeros(world, dtype=torch.int32, device="cuda")
-    words = [flags.data_ptr() + 4 * p for p in range(1, world)]
+    words = [flags.data_ptr() + 4 * p for p in range(world)]          # stand-ins for this rank's word at every peer
     epoch = [0]
 
     def shard_step(i):
         epoch[0] += 1
-        P.llvq_gemv_sorted_rowshard(ctx, bands[i % 112][0], bands[i % 112][1], n_band, k, xb, copies, 0, 0, torch.bfloat16)
-        P.llvq_signal_ranks(ctx, words, epoch[0])
+        P.llvq_gemv_sorted_rowshard(ctx, bands[i % 112][0], bands[i % 112][1], n_band, k, xb, copies, 0, 0, torch.bfloat16,
+                                    flag_words=words, epoch=epoch[0])
         P.llvq_wait_ranks(ctx, flags, world, 0, epoch[0])
     _event_us(torch, shard_step, 16)
     us_sh = _event_us(torch, shard_step, 224)
     band_only = _event_us(torch, lambda i: P.llvq_gemv_sorted(ctx, bands[i % 112][0], bands[i % 112][1], n_band, k, xb, d_y=copies[0]), 224)
     out["rowshard_world8_rank_step_11008x4096_sorted_layout"] = {
-        "us": us_sh, "band_gemv_alone_us": band_only, "rows_per_rank": n_band, "launches_per_step": 3,
+        "us": us_sh, "band_gemv_alone_us": band_only, "rows_per_rank": n_band, "launches_per_step": 2,
         "note": "emulated on one GPU: peer copies of y and flag words are local memory"}
     assert P.llvq_last_error(ctx) == (0, 0)
     del bands, copies

@@ -289,15 +289,19 @@ int llvq_pack_fields(const llvq_ctx* ctx, const uint64_t* d_index, const uint8_t
  * rank's own copy, the others are the peers' exchange buffers opened with llvq_exchange_open (the stores cross
  * NVLink as plain remote writes; nothing is read from a peer).  Row row0 + i of every copy receives what llvq_gemv
  * would have put in y[i].  Copies may be the same pointer only if n_dest = 1.  Everything else (sizes, alignment,
- * errors, summation order) as llvq_gemv / llvq_gemv_sorted.  The call only enqueues the kernel; the ranks learn of
- * each other's completion through llvq_signal_ranks / llvq_wait_ranks below.
+ * errors, summation order) as llvq_gemv / llvq_gemv_sorted.
+ * d_flag_words: NULL, or a HOST array of n_dest DEVICE addresses of 32-bit words (4-byte aligned; the entry at own_slot
+ * is not read), one in each peer's exchange buffer with this rank as its only writer.  The kernel itself then stores
+ * `epoch` there, with release semantics at system scope, once every row of the band is in place in every copy (the
+ * last CTA to finish does it; with n_rows = 0 or k_in = 0 a one-warp kernel does) - what llvq_signal_ranks would do
+ * in a launch of its own.  The peers see it through llvq_wait_ranks.  One such call at a time per context.
  */
 int llvq_gemv_rowshard(const llvq_ctx* ctx, const void* d_idx, const uint16_t* d_gain_f16, int64_t n_rows, int64_t k_in,
                        const uint16_t* d_x_bf16, void* const* d_y_all, int n_dest, int own_slot, int64_t row0,
-                       int y_dtype, void* stream);
+                       int y_dtype, uint32_t* const* d_flag_words, uint32_t epoch, void* stream);
 int llvq_gemv_sorted_rowshard(const llvq_ctx* ctx, const void* d_sorted, const uint16_t* d_gain_f16, int64_t n_rows,
                               int64_t k_in, const uint16_t* d_x_bf16, void* const* d_y_all, int n_dest, int own_slot,
-                              int64_t row0, int y_dtype, void* stream);
+                              int64_t row0, int y_dtype, uint32_t* const* d_flag_words, uint32_t epoch, void* stream);
 
 /*
  * Exchange buffers for the above (no counterpart in the paper: plumbing between processes).

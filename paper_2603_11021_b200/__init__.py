@@ -101,7 +101,8 @@ def load_library() -> ctypes.CDLL:
     lib.llvq_last_error.argtypes = [vp, vp, ctypes.POINTER(u64), ctypes.POINTER(ctypes.c_uint32)]
     lib.llvq_class_info.argtypes = [vp, ctypes.c_int, vp, vp, vp, vp, vp, vp]
     lib.llvq_golay_table.argtypes = [vp, vp]
-    shard = [vp, vp, vp, i64, i64, vp, ctypes.POINTER(vp), ctypes.c_int, ctypes.c_int, i64, ctypes.c_int, vp]
+    shard = [vp, vp, vp, i64, i64, vp, ctypes.POINTER(vp), ctypes.c_int, ctypes.c_int, i64, ctypes.c_int, ctypes.POINTER(vp),
+             ctypes.c_uint32, vp]
     lib.llvq_gemv_rowshard.argtypes = shard
     lib.llvq_gemv_sorted_rowshard.argtypes = shard
     lib.llvq_exchange_create.argtypes = [vp, ctypes.c_size_t, ctypes.POINTER(vp), ctypes.c_char_p]
@@ -444,29 +445,37 @@ def _ptr(p, name: str) -> int:
     return _dev(p, name) if isinstance(p, torch.Tensor) else int(p)
 
 
-def _gemv_rowshard(call: str, ctx: Context, d_stream, d_gain, n_rows, k_in, d_x, y_all, own_slot, row0, y_dtype, stream):
+def _gemv_rowshard(call: str, ctx: Context, d_stream, d_gain, n_rows, k_in, d_x, y_all, own_slot, row0, y_dtype, flag_words, epoch, stream):
     assert d_x.dtype == torch.bfloat16 and d_x.numel() >= k_in and d_gain.dtype == torch.float16
     assert y_dtype in (torch.float32, torch.bfloat16) and 1 <= len(y_all) <= 8
     assert d_gain.numel() >= n_rows * ((k_in + 23) // 24)
     ptrs = (ctypes.c_void_p * len(y_all))(*[_ptr(y, "y_all") for y in y_all])
     code = LLVQ_F32 if y_dtype == torch.float32 else LLVQ_BF16
+    flags = None
+    if flag_words is not None:
+        assert len(flag_words) == len(y_all)
+        flags = (ctypes.c_void_p * len(y_all))(*[_ptr(w, "flag_words") for w in flag_words])
     _check(call, getattr(ctx._lib, call)(ctx._h, _dev(d_stream, "d_stream"), _dev(d_gain, "d_gain"), n_rows, k_in, _dev(d_x, "d_x"),
-                                         ptrs, len(y_all), own_slot, row0, code, _stream_ptr(stream)))
+                                         ptrs, len(y_all), own_slot, row0, code, flags, epoch & 0xffffffff, _stream_ptr(stream)))
 
 
 def llvq_gemv_rowshard(ctx: Context, d_idx: torch.Tensor, d_gain: torch.Tensor, n_rows: int, k_in: int, d_x: torch.Tensor,
-                       y_all, own_slot: int, row0: int, y_dtype: torch.dtype = torch.float32, stream=None) -> None:
+                       y_all, own_slot: int, row0: int, y_dtype: torch.dtype = torch.float32, flag_words=None, epoch: int = 0,
+                       stream=None) -> None:
     """``llvq_gemv`` of one rank's band of rows, written at row ``row0`` of every full-length y in ``y_all``
-    (tensors or device addresses; ``y_all[own_slot]`` is this rank's own copy)."""
+    (tensors or device addresses; ``y_all[own_slot]`` is this rank's own copy).  With ``flag_words`` (one device
+    address per destination) the kernel also stores ``epoch`` to every peer's word when the band is in place."""
     assert d_idx.numel() * d_idx.element_size() >= ctx.index_bytes(n_rows * ((k_in + 23) // 24))
-    _gemv_rowshard("llvq_gemv_rowshard", ctx, d_idx, d_gain, n_rows, k_in, d_x, y_all, own_slot, row0, y_dtype, stream)
+    _gemv_rowshard("llvq_gemv_rowshard", ctx, d_idx, d_gain, n_rows, k_in, d_x, y_all, own_slot, row0, y_dtype, flag_words, epoch, stream)
 
 
 def llvq_gemv_sorted_rowshard(ctx: Context, d_sorted: torch.Tensor, d_gain: torch.Tensor, n_rows: int, k_in: int, d_x: torch.Tensor,
-                              y_all, own_slot: int, row0: int, y_dtype: torch.dtype = torch.float32, stream=None) -> None:
+                              y_all, own_slot: int, row0: int, y_dtype: torch.dtype = torch.float32, flag_words=None,
+                              epoch: int = 0, stream=None) -> None:
     """``llvq_gemv_rowshard`` from the band's sorted stream (``llvq_sort_blocks`` with n_out = n_rows)."""
     assert d_sorted.numel() * d_sorted.element_size() >= int(ctx._lib.llvq_sorted_bytes(ctx._h, n_rows, k_in))
-    _gemv_rowshard("llvq_gemv_sorted_rowshard", ctx, d_sorted, d_gain, n_rows, k_in, d_x, y_all, own_slot, row0, y_dtype, stream)
+    _gemv_rowshard("llvq_gemv_sorted_rowshard", ctx, d_sorted, d_gain, n_rows, k_in, d_x, y_all, own_slot, row0, y_dtype, flag_words,
+                   epoch, stream)
 
 
 def llvq_exchange_create(ctx: Context, nbytes: int) -> tuple[int, bytes]:

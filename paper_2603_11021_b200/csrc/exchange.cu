@@ -36,18 +36,24 @@ __global__ void signal_ranks_kernel(PeerFlags pf, int n, uint32_t epoch)
 }
 
 // Thread p waits until writer p has raised its word to `epoch` (or beyond: the comparison is modular).
+// Launched as a programmatic dependent: it may start while the kernel before it on the stream is still running
+// (the polling then overlaps that kernel's tail), lets the kernel after it start its own prologue, and returns
+// only after the kernel before it has completed, so that stream order means what it always means.
 __global__ void wait_ranks_kernel(const uint32_t* flags, int world, int skip, uint32_t epoch, uint32_t spins, uint32_t* err_flags)
 {
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     const int p = threadIdx.x;
-    if (p >= world || p == skip) return;
-    bool seen = false;
-    for (uint32_t it = 0; it < spins && !seen; ++it) {
-        uint32_t v;
-        asm volatile("ld.acquire.sys.global.u32 %0, [%1];" : "=r"(v) : "l"(flags + p) : "memory");
-        seen = (int32_t)(v - epoch) >= 0;
-        if (!seen) __nanosleep(64);
+    if (p < world && p != skip) {
+        bool seen = false;
+        for (uint32_t it = 0; it < spins && !seen; ++it) {
+            uint32_t v;
+            asm volatile("ld.acquire.sys.global.u32 %0, [%1];" : "=r"(v) : "l"(flags + p) : "memory");
+            seen = (int32_t)(v - epoch) >= 0;
+            if (!seen) __nanosleep(64);
+        }
+        if (!seen) atomicOr(err_flags, (uint32_t)LLVQ_FLAG_WAIT_TIMEOUT);
     }
-    if (!seen) atomicOr(err_flags, (uint32_t)LLVQ_FLAG_WAIT_TIMEOUT);
+    asm volatile("griddepcontrol.wait;" ::: "memory");
 }
 
 int status()
@@ -135,7 +141,16 @@ int llvq_wait_ranks(const llvq_ctx* ctx, const uint32_t* d_flags, int world, int
     DeviceGuard guard(ctx->device);
     if (!guard.ok) return LLVQ_ECUDA;
     const uint32_t spins = max_spins == 0 ? kWaitSpins : (max_spins < kWaitSpins ? max_spins : kWaitSpins);
-    wait_ranks_kernel<<<1, 32, 0, (cudaStream_t)stream>>>(d_flags, world, skip, epoch, spins, ctx->dev.flags);
+    cudaLaunchConfig_t cfg{};
+    cfg.gridDim = dim3(1);
+    cfg.blockDim = dim3(32);
+    cfg.stream = (cudaStream_t)stream;
+    cudaLaunchAttribute attr{};
+    attr.id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr.val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = &attr;
+    cfg.numAttrs = 1;
+    if (cudaLaunchKernelEx(&cfg, wait_ranks_kernel, d_flags, world, skip, epoch, spins, ctx->dev.flags) != cudaSuccess) return LLVQ_ECUDA;
     return status();
 }
 

@@ -230,6 +230,12 @@ struct YOut {
     void* y;
     void* peer[kMaxShardPeers];
     int n_peer;
+    // optional: one word per peer that receives `epoch` once the whole grid has stored its rows (done = the
+    // context's arrival counter, zero between launches)
+    uint32_t* flag[kMaxShardPeers];
+    uint32_t* done;
+    uint32_t epoch;
+    int n_flag;
 };
 
 template <bool kOutBf16>
@@ -297,7 +303,10 @@ __device__ __forceinline__ void finish_pass(const YOut& yo, int64_t rg0, int64_t
         const bool mine = lane < kGemvGroupRows && row < n_out;
         const float part = lane < kGemvGroupRows ? row_sum((rg - rg0) * kGemvGroupRows + lane) : 0.f;
         if (whole) {
-            if (mine) store_y<kOutBf16>(yo, row, part);
+            if (mine) {
+                store_y<kOutBf16>(yo, row, part);
+                if (yo.n_peer) __threadfence_system();
+            }
             continue;
         }
         if (mine) atomicAdd(scratch + row, part);
@@ -315,10 +324,28 @@ __device__ __forceinline__ void finish_pass(const YOut& yo, int64_t rg0, int64_t
             if (mine) {
                 store_y<kOutBf16>(yo, row, __ldcg(scratch + row));
                 __stcg(scratch + row, 0.f);
+                if (yo.n_peer) __threadfence_system();
             }
             if (lane == 0) counters[rg] = 0u;
         }
     }
+}
+
+// Last step of a row-sharded GEMV CTA (all threads call it, after their last store to y): counts the CTA in; the CTA
+// that completes the grid raises the epoch in every peer's flag word.  The remote stores of y are fenced at system
+// scope by the threads that made them (finish_pass) and once more, cumulatively, by the thread that counts.
+__device__ __forceinline__ void shard_arrive(const YOut& yo)
+{
+    if (yo.n_flag == 0) return;
+    __syncthreads();
+    if (threadIdx.x != 0) return;
+    __threadfence_system();
+    if (atomicAdd(yo.done, 1u) != gridDim.x - 1u) return;
+    atomicExch(yo.done, 0u);
+    __threadfence_system();
+#pragma unroll
+    for (int p = 0; p < kMaxShardPeers; ++p)
+        if (p < yo.n_flag) asm volatile("st.release.sys.global.u32 [%0], %1;" ::"l"(yo.flag[p]), "r"(yo.epoch) : "memory");
 }
 
 template <bool kBig, bool kOutBf16, bool kSg = false>
@@ -337,8 +364,7 @@ gemv_fast_kernel(FastArgs fa, const uint32_t* __restrict__ stream, const uint16_
     const int64_t groups = (n_out + kGemvGroupRows - 1) / kGemvGroupRows;
     const int64_t U = groups * nq, G = gridDim.x;
     const int64_t u_begin = blockIdx.x * U / G, u_end = (blockIdx.x + 1) * U / G;
-    if (u_begin >= u_end) return;
-    const int64_t rg_first = u_begin / nq, rg_last = (u_end - 1) / nq;
+    const int64_t rg_first = u_begin / nq, rg_last = u_begin < u_end ? (u_end - 1) / nq : rg_first - 1;   // no units: no pass
     for (int64_t rg0 = rg_first; rg0 <= rg_last; rg0 += kGemvGroupsPerPass) {
         const int64_t rg1 = min(rg0 + kGemvGroupsPerPass - 1, rg_last);
         for (int i = threadIdx.x; i < kGemvGroupsPerPass * kGemvGroupRows; i += (int)blockDim.x) acc[i] = 0.f;
@@ -368,6 +394,7 @@ gemv_fast_kernel(FastArgs fa, const uint32_t* __restrict__ stream, const uint16_
         finish_pass<kOutBf16>(yo, rg0, rg1, nq, u_begin, u_end, U, G, n_out, scratch, counters, [&](int64_t r) { return acc[r]; });
         __syncthreads();                                   // the sums are read above: the next pass may clear them only now
     }
+    shard_arrive(yo);
 }
 
 constexpr uint32_t kKindEven = 0u, kKindOdd = 1u, kKindOther = 2u, kKindNull = 3u;   // decoder form a class needs
@@ -578,6 +605,7 @@ gemv_sorted_kernel(FastArgs fa, const unsigned long long* __restrict__ sorted, c
         finish_pass<kOutBf16>(yo, rg0, rg1, nq, u_begin, u_end, U, G, n_out, scratch, counters, row_sum);
         __syncthreads();                                   // the sums are read above: the next pass may clear them only now
     });
+    shard_arrive(yo);
 }
 
 // ===========================================================================
@@ -739,6 +767,7 @@ gemv_bin_kernel(FastArgs fa, const uint32_t* __restrict__ stream, const uint16_t
         finish_pass<kOutBf16>(yo, rg0, rg1, nq, u_begin, u_end, U, G, n_out, scratch, counters, row_sum);
         __syncthreads();
     }, seg_units);
+    shard_arrive(yo);
 }
 
 // ===========================================================================
@@ -757,6 +786,7 @@ constexpr int kGemmRows = 128;
 constexpr int kStageBlocks = 4;                       // column blocks per stage
 constexpr int kStageK = kStageBlocks * 24;            // 96
 constexpr int kMaxScratchRows = 65536;
+constexpr int kCounterWords = 64 * kMaxScratchRows / 8;      // the word after them counts the CTAs of a row-sharded GEMV that have finished
 constexpr uint32_t kTmemCols = 128;
 
 struct GemmArgs {
@@ -1306,7 +1336,7 @@ int llvq_create(llvq_ctx** out, int m_lo, int m_hi, int device)
         for (uint32_t r = 0; r < ncls; ++r) sort_rank[order[r]] = (uint16_t)r;
     }
     size_t o_cnt = up(o_srk + sort_rank.size() * 2);
-    size_t o_scr = up(o_cnt + (size_t)(64 * kMaxScratchRows / 8) * 4);    // one counter per group of 8 rows (GEMV) / per 128-row tile (GEMM)
+    size_t o_scr = up(o_cnt + (size_t)(kCounterWords + 16) * 4);   // one counter per group of 8 rows (GEMV) / per 128-row tile (GEMM), then the grid arrival counter
     size_t total = o_scr + (size_t)64 * kMaxScratchRows * 4;
     std::vector<uint8_t> blob(o_cnt, 0);
     std::memcpy(blob.data() + o_offhi, off_hi.data(), (ncls + 1) * 4);
@@ -1707,9 +1737,12 @@ int llvq_gemv_sorted_sg(const llvq_ctx* ctx, const void* d_sorted, int gain_bits
 }
 
 // Row-sharded GEMV: the destinations of one rank's band.  d_y_all[0..n_dest) are the ranks' full-length copies of y
-// (own_slot = this rank's own copy), the band starts at row row0.
-static int shard_yout(void* const* d_y_all, int n_dest, int own_slot, int64_t row0, int y_dtype, YOut* yo)
+// (own_slot = this rank's own copy), the band starts at row row0; d_flag_words (optional) = for every destination
+// the word that receives `epoch` when the band is in place (the own slot's entry is not used).
+static int shard_yout(const llvq_ctx* ctx, void* const* d_y_all, int n_dest, int own_slot, int64_t row0, int y_dtype,
+                      uint32_t* const* d_flag_words, uint32_t epoch, YOut* yo)
 {
+    if (!ctx || ctx->device < 0) return LLVQ_EINVAL;
     if (!d_y_all || n_dest < 1 || n_dest > kMaxShardPeers + 1 || own_slot < 0 || own_slot >= n_dest || row0 < 0) return LLVQ_EINVAL;
     if (y_dtype != LLVQ_F32 && y_dtype != LLVQ_BF16) return LLVQ_EINVAL;
     const size_t es = y_dtype == LLVQ_F32 ? 4 : 2;
@@ -1717,31 +1750,50 @@ static int shard_yout(void* const* d_y_all, int n_dest, int own_slot, int64_t ro
     for (int d = 0; d < n_dest; ++d) {
         if (!d_y_all[d]) return LLVQ_EINVAL;
         void* at = static_cast<unsigned char*>(d_y_all[d]) + (size_t)row0 * es;
-        if (d == own_slot) yo->y = at;
-        else yo->peer[yo->n_peer++] = at;
+        if (d == own_slot) { yo->y = at; continue; }
+        yo->peer[yo->n_peer++] = at;
+        if (d_flag_words) {
+            if (!d_flag_words[d]) return LLVQ_EINVAL;
+            if (!aligned(d_flag_words[d], 4)) return LLVQ_EALIGN;
+            yo->flag[yo->n_flag++] = d_flag_words[d];
+        }
     }
+    yo->done = ctx->d_counters + kCounterWords;
+    yo->epoch = epoch;
     return LLVQ_OK;
 }
 
+// A band without rows still has to tell the peers that it is done with the step.
+static int signal_only(const llvq_ctx* ctx, const YOut& yo, void* stream)
+{
+    if (yo.n_flag == 0) return LLVQ_OK;
+    return llvq_signal_ranks(ctx, yo.flag, yo.n_flag, yo.epoch, stream);
+}
+
 int llvq_gemv_rowshard(const llvq_ctx* ctx, const void* d_idx, const uint16_t* d_gain_f16, int64_t n_rows, int64_t k_in,
-                       const uint16_t* d_x_bf16, void* const* d_y_all, int n_dest, int own_slot, int64_t row0, int y_dtype, void* stream)
+                       const uint16_t* d_x_bf16, void* const* d_y_all, int n_dest, int own_slot, int64_t row0, int y_dtype,
+                       uint32_t* const* d_flag_words, uint32_t epoch, void* stream)
 {
     YOut yo;
-    if (int e = shard_yout(d_y_all, n_dest, own_slot, row0, y_dtype, &yo)) return e;
-    if (ctx && ctx->device >= 0 && n_rows == 0) return LLVQ_OK;
+    if (int e = shard_yout(ctx, d_y_all, n_dest, own_slot, row0, y_dtype, d_flag_words, epoch, &yo)) return e;
+    if (n_rows == 0) return signal_only(ctx, yo, stream);
     if (int e = check_common(ctx, d_idx)) return e;
     if (!d_gain_f16) return LLVQ_EINVAL;
     if (!aligned(d_gain_f16, 2)) return LLVQ_EALIGN;
+    if (k_in == 0) {                                   // y = 0 by copies, no kernel to raise the flags
+        if (int e = gemv_common(ctx, d_idx, d_gain_f16, nullptr, n_rows, k_in, d_x_bf16, yo, y_dtype, stream)) return e;
+        return signal_only(ctx, yo, stream);
+    }
     return gemv_common(ctx, d_idx, d_gain_f16, nullptr, n_rows, k_in, d_x_bf16, yo, y_dtype, stream);
 }
 
 int llvq_gemv_sorted_rowshard(const llvq_ctx* ctx, const void* d_sorted, const uint16_t* d_gain_f16, int64_t n_rows, int64_t k_in,
                               const uint16_t* d_x_bf16, void* const* d_y_all, int n_dest, int own_slot, int64_t row0, int y_dtype,
-                              void* stream)
+                              uint32_t* const* d_flag_words, uint32_t epoch, void* stream)
 {
     YOut yo;
-    if (int e = shard_yout(d_y_all, n_dest, own_slot, row0, y_dtype, &yo)) return e;
-    if (ctx && ctx->device >= 0 && n_rows == 0) return LLVQ_OK;
+    if (int e = shard_yout(ctx, d_y_all, n_dest, own_slot, row0, y_dtype, d_flag_words, epoch, &yo)) return e;
+    if (n_rows == 0) return signal_only(ctx, yo, stream);
     if (int e = check_common(ctx, d_sorted)) return e;
     if (!d_gain_f16) return LLVQ_EINVAL;
     if (!aligned(d_gain_f16, 2)) return LLVQ_EALIGN;

@@ -81,7 +81,7 @@ class RowShardedGemv:
     """y = W x with the rows of W spread over the ranks of a process group; every rank ends up with all of y.
 
     Each rank passes its own band (``row_bands(n_out, world)[rank]``) as device tensors.  One step is
-    ``launch(x)`` (the band's fused GEMV, writing into every rank's y, then the epoch flag to every peer) followed by
+    ``launch(x)`` (one kernel: the band's fused GEMV, writing into every rank's y and then the epoch flag of every peer) followed by
     ``wait()`` (bounded device-side wait for the other ranks' flags) — ``__call__`` does both and returns this
     rank's y.  Two y buffers alternate between steps: a rank that is one step ahead writes the other buffer, and it
     cannot be two steps ahead because each step waits for every rank's previous flag.
@@ -121,11 +121,12 @@ class RowShardedGemv:
         """Enqueue this rank's part of the next step."""
         self.epoch += 1
         call = llvq_gemv_sorted_rowshard if self.sorted_layout else llvq_gemv_rowshard
+        words = [b + 4 * self.rank for b in self._bufs]                  # this rank's word in every buffer
         if self.n_rows:
             call(self.ctx, self.d_stream, self.d_gain, self.n_rows, self.k_in, d_x, self._y_all(self.epoch & 1), self.rank, self.row0,
-                 self.y_dtype, stream)
-        words = [self._bufs[r] + 4 * self.rank for r in range(self.world) if r != self.rank]
-        llvq_signal_ranks(self.ctx, words, self.epoch, stream)
+                 self.y_dtype, words, self.epoch, stream)
+        else:
+            llvq_signal_ranks(self.ctx, [w for r, w in enumerate(words) if r != self.rank], self.epoch, stream)
 
     def wait(self, stream=None, max_spins: int = 0) -> torch.Tensor:
         """Enqueue the wait for the other ranks' parts of the step launched last; returns this rank's y (valid in

@@ -62,9 +62,13 @@ def test_every_copy_of_y_holds_the_product(lib, ctx, code, n_out, k_in, world, d
     flags = [torch.zeros(world, dtype=torch.int32, device="cuda") for _ in range(world)]
     call = lib.llvq_gemv_sorted_rowshard if sorted_layout else lib.llvq_gemv_rowshard
     for r, (row0, n, ds, dg) in enumerate(_bands_on_device(lib, ctx, o, stream, gain, n_out, k_in, world, sorted_layout)):
-        if n:
-            call(ctx, ds, dg, n, k_in, dx, copies, r, row0, dtype)
-        lib.llvq_signal_ranks(ctx, [flags[p].data_ptr() + 4 * r for p in range(world) if p != r], 1)
+        words = [flags[p].data_ptr() + 4 * r for p in range(world)]      # rank r's word at every rank
+        if r % 2:                                                         # the kernel raises the flags itself ...
+            call(ctx, ds, dg, n, k_in, dx, copies, r, row0, dtype, flag_words=words, epoch=1)
+        else:                                                             # ... or a launch of its own does
+            if n:
+                call(ctx, ds, dg, n, k_in, dx, copies, r, row0, dtype)
+            lib.llvq_signal_ranks(ctx, [w for p, w in enumerate(words) if p != r], 1)
     for r in range(world):                         # every flag is up already: the waits return at their first look
         lib.llvq_wait_ranks(ctx, flags[r], world, r, 1)
     torch.cuda.synchronize()
