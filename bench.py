@@ -316,8 +316,17 @@ def extras(P, ctx) -> dict:
         us = _event_us(torch, fn, 16)
         by = nb * (72 // 8 + 2) + batch * k * 2 + batch * n * 2
         out[f"gemm_8192x8192_b{batch}_72bit"] = {"us": us, "GBps": by / us / 1e3, "TFLOPs": 2.0 * n * k * batch / us / 1e6, "algorithmic_bytes": by}
+    srt = [P.llvq_sort_blocks_gemm(ctx53, b[0], n, k) for b in bufs]      # 128-bit entries: index, class, position
+    for batch in (16, 64):
+        x = dev(gen.normal_bf16((batch, k), seed=batch), np.int16).view(torch.bfloat16)
+        y = torch.empty((batch, n), dtype=torch.bfloat16, device="cuda")
+        fn = lambda i: P.llvq_gemm_small_batch_sorted(ctx53, srt[i % 8], bufs[i % 8][1], n, k, x, d_y=y)
+        _event_us(torch, fn, 4)
+        us = _event_us(torch, fn, 16)
+        by = nb * (72 // 8 + 2) + batch * k * 2 + batch * n * 2
+        out[f"gemm_8192x8192_b{batch}_72bit_sorted_layout"] = {"us": us, "GBps": by / us / 1e3, "TFLOPs": 2.0 * n * k * batch / us / 1e6, "algorithmic_bytes": by}
     assert P.llvq_last_error(ctx53) == (0, 0)
-    del bufs, ctx53
+    del bufs, srt, ctx53
     # --- decoder sweep: q, k, v, o, gate, up, down of one layer; 32 layers; 4 distinct layer sets (> 2 x L2)
     shapes = [(4096, 4096), (1024, 4096), (1024, 4096), (4096, 4096), (14336, 4096), (14336, 4096), (4096, 14336)]
     sets = []

@@ -214,7 +214,11 @@ int llvq_gemm_small_batch(const llvq_ctx* ctx, const void* d_idx, const uint16_t
  * entry per block (stored index unchanged in the low 48 bits, position in the domain above).
  * llvq_gemm_small_batch_sorted computes the same Y as llvq_gemm_small_batch from that stream and the unchanged
  * ROWWISE gains; all of App. A steps 1-4 run in the kernel.  llvq_sorted_gemm_bytes() gives the stream length (8 bytes
- * per block of the matrix padded to whole domains; 0 if unsupported: same codes as llvq_sort_blocks).
+ * per block of the matrix padded to whole domains; 0 if unsupported: same codes as llvq_sort_blocks, plus the one below).
+ * Codes whose class tables live in global memory (the 72-bit code, shells 2..53) take 128-bit entries, 16 bytes per
+ * block: the stored index unchanged (72 bits), the number of its class (24 bits: App. A step 2 is then a table look-up
+ * in the kernel instead of a search; steps 1, 3, 4 run there as before) and the position in the domain; the order is
+ * by unranking steps, then class.  Out-of-range indices are counted by llvq_sort_blocks_gemm and stored as "no block".
  * d_sorted: device, 16-byte aligned.  Other arguments and limits as in llvq_gemm_small_batch.
  */
 size_t llvq_sorted_gemm_bytes(const llvq_ctx* ctx, int64_t n_out, int64_t k_in);

@@ -994,6 +994,59 @@ sort_blocks_gemm_kernel(FastArgs fa, const uint32_t* __restrict__ stream, const 
     }
 }
 
+// The same layout for codes whose class tables live in global memory (72-bit indices): 128-bit entries, x = the low 64
+// bits of the stored index, y = its bits 64.. (8 bits) | class << 8 (24 bits) | position in the domain << 32 (10 bits);
+// bit 63 of y marks "no block" (ragged edge or index out of range).  The class rides along so that the GEMM kernel does
+// not search for it again; the blocks of a domain are ordered by unranking steps (most first), then by class, so that
+// the lanes of a warp run the same trip counts and read neighbouring class descriptors.
+constexpr unsigned long long kBigNoBlock = 1ull << 63;
+
+__global__ void __launch_bounds__(kDomEntries, 1)
+sort_blocks_gemm_big_kernel(FastArgs fa, const uint32_t* __restrict__ stream, int64_t n_out, int64_t bpr, int64_t ndomains,
+                            ulonglong2* __restrict__ out)
+{
+    __shared__ uint32_t keys[kDomEntries];
+    __shared__ unsigned long long ex[kDomEntries], ey[kDomEntries];
+    const int64_t nd = (bpr + kDomBlocks - 1) / kDomBlocks;
+    const int i = threadIdx.x;
+    for (int64_t dom = blockIdx.x; dom < ndomains; dom += gridDim.x) {
+        const int64_t rt = dom / nd, d = dom - rt * nd;
+        const int64_t row = rt * kGemmRows + (i >> 3), cb = d * kDomBlocks + (i & 7);
+        unsigned long long x = 0ull, y = kBigNoBlock | (unsigned long long)i << 32;
+        uint32_t key = 0x7ffffc00u | (uint32_t)i;                   // no block: after everything else
+        if (row < n_out && cb < bpr) {
+            uint64_t lo, hi;
+            load_index(stream, (uint64_t)(row * bpr + cb), fa.dc.W, lo, hi);
+            if (hi < fa.dc.n_hi || (hi == fa.dc.n_hi && lo < fa.dc.n_lo)) {
+                uint64_t local;
+                const uint32_t cls = (uint32_t)big_find_class(fa.dc, lo, hi, local);
+                const uint32_t h0y = __ldg(reinterpret_cast<const uint32_t*>(fa.dc.cls + cls) + 1);
+                const uint32_t nlev = (h0y & 0xff) + ((h0y >> 8) & 0xff);
+                x = lo;
+                y = (hi & 0xffull) | (unsigned long long)cls << 8 | (unsigned long long)i << 32;
+                key = (15u - min(nlev, 15u)) << 27 | cls << 10 | (uint32_t)i;
+            } else {
+                atomicAdd(fa.bad_index, 1ull);
+            }
+        }
+        keys[i] = key; ex[i] = x; ey[i] = y;
+        __syncthreads();
+        for (int k = 2; k <= kDomEntries; k <<= 1)                   // bitonic sort of the 1024 keys
+            for (int j = k >> 1; j > 0; j >>= 1) {
+                const int o = i ^ j;
+                if (o > i) {
+                    const uint32_t a = keys[i], b = keys[o];
+                    if ((a > b) == ((i & k) == 0)) { keys[i] = b; keys[o] = a; }
+                }
+                __syncthreads();
+            }
+        const uint32_t src = keys[i] & 1023u;
+        out[dom * kDomEntries + i] = make_ulonglong2(ex[src], ey[src]);
+        __syncthreads();
+    }
+}
+
+template <bool kBig>
 __global__ void __launch_bounds__(kGemmThreads, 1)
 gemm_sorted_kernel(FastArgs fa, const unsigned long long* __restrict__ sorted, const uint16_t* __restrict__ gain, GemmArgs ga, int dpi)
 {
@@ -1037,30 +1090,46 @@ gemm_sorted_kernel(FastArgs fa, const unsigned long long* __restrict__ sorted, c
         const int d_begin = (int)(max(dom_begin, rt * nd) - rt * nd), d_end = (int)(min(dom_end, (rt + 1) * nd) - rt * nd);
         const uint32_t parts = (uint32_t)(unit_owner((rt + 1) * nd - 1, D, G) - unit_owner(rt * nd, D, G) + 1);   // CTAs that share this row tile
         // the entries of an iteration are requested one iteration ahead (they come from DRAM)
+        const ulonglong2 no_entry = make_ulonglong2(kSortIndexMask, kBigNoBlock);
         auto entry_at = [&](int d, int q) {
-            return d + q < d_end ? __ldg(sorted + ((rt * nd + d + q) * kDomEntries + (q == 0 ? warp : 31 - warp) * 32 + lane)) : kSortIndexMask;
+            if (d + q >= d_end) return no_entry;
+            const int64_t at = (rt * nd + d + q) * kDomEntries + (q == 0 ? warp : 31 - warp) * 32 + lane;
+            if (kBig) return __ldg(reinterpret_cast<const ulonglong2*>(sorted) + at);
+            return make_ulonglong2(__ldg(sorted + at), 0ull);
         };
-        unsigned long long e0 = entry_at(d_begin, 0), e1 = dpi > 1 ? entry_at(d_begin, 1) : kSortIndexMask;
+        ulonglong2 e0 = entry_at(d_begin, 0), e1 = dpi > 1 ? entry_at(d_begin, 1) : no_entry;
         for (int d0 = d_begin; d0 < d_end; d0 += dpi, ++uses) {
             const int nd_now = min(dpi, d_end - d0);
-            const unsigned long long cur0 = e0, cur1 = e1;
+            const ulonglong2 cur0 = e0, cur1 = e1;
             e0 = entry_at(d0 + dpi, 0);
             if (dpi > 1) e1 = entry_at(d0 + dpi, 1);
             // ---- A: every warp unranks one chunk of 32 sorted entries per domain
 #pragma unroll
             for (int q = 0; q < 2; ++q) {
                 if (q >= nd_now) break;
-                const unsigned long long e = q == 0 ? cur0 : cur1;
-                const uint64_t I = e & kSortIndexMask;
-                const uint32_t pos = (uint32_t)(e >> 48);
-                const bool valid = I < fa.n_points;
+                const ulonglong2 e = q == 0 ? cur0 : cur1;
+                const uint64_t I = e.x & kSortIndexMask;
+                const uint32_t pos = kBig ? (uint32_t)(e.y >> 32) & 1023u : (uint32_t)(e.x >> 48);
+                const bool valid = kBig ? !(e.y >> 63) : I < fa.n_points;
                 const uint32_t r = pos >> 3, c = pos & 7u;
                 const int64_t row = rt * kGemmRows + r, cb = (int64_t)(d0 + q) * kDomBlocks + c;
                 const float gn = valid ? gain_to_float(__ldg(gain + row * ga.bpr + cb)) : 0.f;
-                Decoded dec;
-                decode_sorted_entry(fa, T, I, valid, dec);
                 uint32_t w[12];
-                expand_bf16(dec, gn, w);
+                if (kBig) {
+                    const int cls = valid ? (int)((uint32_t)(e.y >> 8) & 0xffffffu) : 0;
+                    const uint64_t local = valid ? e.x - __ldg(fa.dc.off_lo + cls) : 0ull;     // class sizes fit 63 bits: exact mod 2^64
+                    Point pt;
+                    big_decode_local(T, fa.dc, cls, local, valid, pt);
+#pragma unroll
+                    for (int j = 0; j < 12; ++j) {
+                        __nv_bfloat162 h = __halves2bfloat162(dequant(gn, pt, 2 * j), dequant(gn, pt, 2 * j + 1));
+                        w[j] = *reinterpret_cast<uint32_t*>(&h);
+                    }
+                } else {
+                    Decoded dec;
+                    decode_sorted_entry(fa, T, I, valid, dec);
+                    expand_bf16(dec, gn, w);
+                }
                 // the previous MMAs read the buffers: wait for them only now, with the first chunk already unranked
                 if (q == 0 && uses > 0 && !mbar_wait(bar_free, (uses - 1u) & 1u)) timeout = true;
                 uint8_t* a_dst = a_buf + (uint32_t)(q * kDomStages + (c >> 2)) * kAStage + (r >> 3) * 128u + (r & 7u) * 16u + 3u * (c & 3u) * 2048u;
@@ -1206,9 +1275,15 @@ int launch_gemm_domains(const llvq_ctx* ctx, const void* p, const uint16_t* d_ga
     const unsigned grid = (unsigned)std::min<int64_t>(row_tiles * ga.nstages, ctx->sm_count);
     const size_t smem = ((ctx->fl.total + 64 + 1023) & ~size_t(1023)) + (size_t)dpi * kDomStages * (kGemmRows * kStageK * 2 + (size_t)ga.npad * kStageK * 2);
     if (smem > 227 * 1024) return LLVQ_EUNSUPPORTED;
-    if (!set_smem(gemm_sorted_kernel, smem)) return LLVQ_ECUDA;
-    if (launch_pdl(gemm_sorted_kernel, grid, (unsigned)kGemmThreads, smem, (cudaStream_t)stream, fast_args(ctx),
-                   static_cast<const unsigned long long*>(p), d_gain_f16, ga, dpi) != cudaSuccess) return LLVQ_ECUDA;
+    if (ctx->fast) {
+        if (!set_smem(gemm_sorted_kernel<false>, smem)) return LLVQ_ECUDA;
+        if (launch_pdl(gemm_sorted_kernel<false>, grid, (unsigned)kGemmThreads, smem, (cudaStream_t)stream, fast_args(ctx),
+                       static_cast<const unsigned long long*>(p), d_gain_f16, ga, dpi) != cudaSuccess) return LLVQ_ECUDA;
+    } else {
+        if (!set_smem(gemm_sorted_kernel<true>, smem)) return LLVQ_ECUDA;
+        if (launch_pdl(gemm_sorted_kernel<true>, grid, (unsigned)kGemmThreads, smem, (cudaStream_t)stream, fast_args(ctx),
+                       static_cast<const unsigned long long*>(p), d_gain_f16, ga, dpi) != cudaSuccess) return LLVQ_ECUDA;
+    }
     return launch_status();
 }
 
@@ -1803,14 +1878,15 @@ int llvq_gemv_sorted_rowshard(const llvq_ctx* ctx, const void* d_sorted, const u
 // Sorted layout of the small-batch GEMM (see the comment at sort_blocks_gemm_kernel).
 static bool gemm_sortable(const llvq_ctx* ctx)
 {
-    return ctx->fast && ctx->d_sort_rank && ctx->host.W <= 48 && ctx->host.N < (u128)kSortIndexMask;
+    if (!ctx->fast) return ctx->host.W <= 72 && ctx->dev.nclasses < (1 << 17);     // 128-bit entries: 72-bit index + class + position
+    return ctx->d_sort_rank && ctx->host.W <= 48 && ctx->host.N < (u128)kSortIndexMask;
 }
 
 size_t llvq_sorted_gemm_bytes(const llvq_ctx* ctx, int64_t n_out, int64_t k_in)
 {
     if (!ctx || ctx->device < 0 || n_out <= 0 || k_in <= 0 || !gemm_sortable(ctx)) return 0;
     const int64_t bpr = (k_in + 23) / 24;
-    return (size_t)(((n_out + kGemmRows - 1) / kGemmRows) * ((bpr + kDomBlocks - 1) / kDomBlocks)) * kDomEntries * 8;
+    return (size_t)(((n_out + kGemmRows - 1) / kGemmRows) * ((bpr + kDomBlocks - 1) / kDomBlocks)) * kDomEntries * (ctx->fast ? 8 : 16);
 }
 
 int llvq_sort_blocks_gemm(const llvq_ctx* ctx, const void* d_idx, int64_t n_out, int64_t k_in, void* d_sorted, void* stream)
@@ -1823,9 +1899,14 @@ int llvq_sort_blocks_gemm(const llvq_ctx* ctx, const void* d_idx, int64_t n_out,
     if (!guard.ok) return LLVQ_ECUDA;
     const int64_t bpr = (k_in + 23) / 24;
     const int64_t ndomains = ((n_out + kGemmRows - 1) / kGemmRows) * ((bpr + kDomBlocks - 1) / kDomBlocks);
+    const unsigned g = (unsigned)std::min<int64_t>(ndomains, 4ll * ctx->sm_count);
+    if (!ctx->fast) {
+        sort_blocks_gemm_big_kernel<<<g, kDomEntries, 0, (cudaStream_t)stream>>>(fast_args(ctx), static_cast<const uint32_t*>(d_idx), n_out, bpr,
+                                                                                 ndomains, static_cast<ulonglong2*>(d_sorted));
+        return launch_status();
+    }
     const size_t smem = ctx->fl.total + 16;
     if (!set_smem(sort_blocks_gemm_kernel, smem)) return LLVQ_ECUDA;
-    const unsigned g = (unsigned)std::min<int64_t>(ndomains, 4ll * ctx->sm_count);
     sort_blocks_gemm_kernel<<<g, kDomEntries, smem, (cudaStream_t)stream>>>(fast_args(ctx), static_cast<const uint32_t*>(d_idx), ctx->d_sort_rank,
                                                                            n_out, bpr, ndomains, static_cast<unsigned long long*>(d_sorted));
     return launch_status();

@@ -524,7 +524,8 @@ def test_back_to_back_launches_see_the_previous_result(lib, ctxs, oracle_mod):
 # --------------------------------------------------------------------------
 @pytest.mark.parametrize("code,n_out,k_in,batch", [((2, 13), 200, 480, 3), ((2, 13), 129, 1000, 16), ((2, 13), 1000, 2000, 33),
                                                    ((2, 13), 64, 4096, 64), ((2, 13), 1, 24, 1), ((2, 2), 256, 768, 16),
-                                                   ((3, 3), 130, 4104, 20)])
+                                                   ((3, 3), 130, 4104, 20), ((2, 53), 200, 480, 3), ((2, 53), 300, 2000, 33),
+                                                   ((2, 53), 129, 1000, 64)])
 def test_gemm_sorted_small_shapes(lib, ctxs, oracle_mod, code, n_out, k_in, batch):
     o = _oracle(oracle_mod)(code)
     ctx = ctxs[code]
@@ -532,7 +533,8 @@ def test_gemm_sorted_small_shapes(lib, ctxs, oracle_mod, code, n_out, k_in, batc
     x = gen.normal_bf16((batch, k_in), seed=24)
     want = o.gemm(stream, gain, n_out, k_in, x, threads=4)
     srt = lib.llvq_sort_blocks_gemm(ctx, to_dev_u8(stream), n_out, k_in)
-    assert srt.numel() == 8192 * ((n_out + 127) // 128) * (((k_in + 23) // 24 + 7) // 8)
+    entry_bytes = 16 if o.W > 48 else 8                      # the 72-bit code keeps index, class and position in 128 bits
+    assert srt.numel() == 1024 * entry_bytes * ((n_out + 127) // 128) * (((k_in + 23) // 24 + 7) // 8)
     y = lib.llvq_gemm_small_batch_sorted(ctx, srt, to_dev_f16(gain), n_out, k_in, to_dev_bf16(x))
     y_plain = lib.llvq_gemm_small_batch(ctx, to_dev_u8(stream), to_dev_f16(gain), n_out, k_in, to_dev_bf16(x))
     torch.cuda.synchronize()
@@ -591,14 +593,73 @@ def test_gemm_sorted_full_size_sampled_rows(lib, ctxs, oracle_mod, batch):
     assert lib.llvq_last_error(ctx) == (0, 0)
 
 
+def test_sort_blocks_gemm_72bit_entries(lib, ctxs, oracle_mod):
+    # 128-bit entries: the stored index unchanged, its class, its position; inside a domain every class forms one
+    # run (the order is by unranking steps, then class, then position); entries without a block last
+    o = _oracle(oracle_mod)((2, 53))
+    ctx = ctxs[(2, 53)]
+    n_out, k_in = 200, 1000                                 # 2 row tiles, 42 blocks per row -> 6 domains per tile, ragged both ways
+    bpr, nd = 42, 6
+    stream, _, nblocks = gen.make_layer(o.N, o.W, n_out, k_in, 1, seed=26)
+    idx = o.unpack(stream, nblocks)
+    e = lib.llvq_sort_blocks_gemm(ctx, to_dev_u8(stream), n_out, k_in).cpu().numpy().view(np.uint64).reshape(2 * nd, 1024, 2)
+    offs = [c["offset"] for c in o.classes()] + [o.N]
+    import bisect
+    seen = set()
+    for dom in range(2 * nd):
+        rt, d = divmod(dom, nd)
+        positions, last_key, closed = set(), (-1, -1), set()
+        for x, y in e[dom].tolist():
+            pos = (y >> 32) & 1023
+            row, cb = rt * 128 + pos // 8, d * 8 + pos % 8
+            assert pos not in positions
+            positions.add(pos)
+            if y >> 63:
+                assert row >= n_out or cb >= bpr
+                closed.add(last_key[0])
+                last_key = (-2, 0)                          # nothing with a block may follow
+                continue
+            assert last_key[0] != -2
+            I, cls = x | (y & 0xff) << 64, (y >> 8) & 0xffffff
+            b = row * bpr + cb
+            assert idx[b] == I and b not in seen
+            seen.add(b)
+            assert cls == bisect.bisect_right(offs, I) - 1
+            # the key is a function of the class (then the position): a class forms one run, positions ascending inside
+            if cls == last_key[0]:
+                assert pos > last_key[1]
+            else:
+                assert cls not in closed
+                closed.add(last_key[0])
+            last_key = (cls, pos)
+    assert len(seen) == nblocks
+    assert lib.llvq_last_error(ctx) == (0, 0)
+
+
+@pytest.mark.parametrize("batch", [16, 64])
+def test_gemm_sorted_72bit_full_size_sampled_rows(lib, ctxs, oracle_mod, batch):
+    o = _oracle(oracle_mod)((2, 53))
+    ctx = ctxs[(2, 53)]
+    n_out, k_in = 8192, 8192
+    stream, gain, _ = gen.make_layer(o.N, o.W, n_out, k_in, 1, seed=0)
+    x = gen.normal_bf16((batch, k_in), seed=0)
+    srt = lib.llvq_sort_blocks_gemm(ctx, to_dev_u8(stream), n_out, k_in)
+    y = lib.llvq_gemm_small_batch_sorted(ctx, srt, to_dev_f16(gain), n_out, k_in, to_dev_bf16(x)).float().cpu().numpy()
+    rows = [0, 127, 128, 4096, 8191] + list(range(77, 8192, 2063))
+    ref = np.zeros((batch, len(rows)))
+    for j, r in enumerate(rows):
+        ref[:, j] = o.gemm(stream, gain, n_out, k_in, x, rows=(r, 1))[:, r]
+    assert gemv_error(y[:, rows], ref) <= TOL_BF16_OUT
+    assert lib.llvq_last_error(ctx) == (0, 0)
+
+
 def test_gemm_sorted_unsupported_and_arguments(lib, ctxs):
-    big = ctxs[(2, 53)]
     buf = torch.zeros(8192, dtype=torch.uint8, device="cuda")
     p = buf.data_ptr()
-    assert big._lib.llvq_sorted_gemm_bytes(big._h, 64, 96) == 0
-    assert big._lib.llvq_sort_blocks_gemm(big._h, p, 16, 96, p, None) == 3
-    assert big._lib.llvq_gemm_small_batch_sorted(big._h, p, p, 16, 96, p, 4, p, None) == 3
+    big = ctxs[(2, 53)]
+    assert big._lib.llvq_sorted_gemm_bytes(big._h, 64, 96) == 1024 * 16
     ctx = ctxs[(2, 13)]
+    assert ctx._lib.llvq_sorted_gemm_bytes(ctx._h, 64, 96) == 1024 * 8
     assert ctx._lib.llvq_gemm_small_batch_sorted(ctx._h, p, p, 16, 96, p, 65, p, None) == 1       # batch out of range
     assert ctx._lib.llvq_gemm_small_batch_sorted(ctx._h, p, p, 16, 100, p, 4, p, None) == 2      # k_in not a multiple of 8
     assert ctx._lib.llvq_gemm_small_batch_sorted(ctx._h, None, None, 0, 96, None, 4, None, None) == 0
