@@ -41,7 +41,7 @@ WORKLOAD = "configs[2]: fused dequant+GEMV batch 1 on W 4096x4096, 11008x4096, 4
 
 # dram__bytes_read.sum + dram__bytes_write.sum of one gemv_fast_kernel launch on the 11008x4096 layer, from the
 # ncu capture summarised under profiles/ (algorithmic bytes: 15 089 152)
-NCU_TRAFFIC_BYTES_11008x4096 = 15265024
+NCU_TRAFFIC_BYTES_11008x4096 = 15272960
 
 
 def layer_bytes(n_out: int, k_in: int) -> dict:
@@ -200,17 +200,22 @@ def profile_run(P, ctx, args) -> None:
     """A handful of launches of one kernel on buffers that do not fit L2 together, for profiler captures:
     gemv = the 11008x4096 layer, dequant = 4096x4096 FLAT, gemm = 8192x8192 at batch 16."""
     import torch
-    n, k = {"gemv": (11008, 4096), "gemv_sorted": (11008, 4096), "dequant": (4096, 4096), "gemm": (8192, 8192), "gemm_sorted": (8192, 8192)}[args.profile]
+    n, k = {"gemv": (11008, 4096), "gemv_sorted": (11008, 4096), "dequant": (4096, 4096), "gemm": (8192, 8192), "gemm_sorted": (8192, 8192),
+            "gemm_72bit": (8192, 8192), "gemm_sorted_72bit": (8192, 8192)}[args.profile]
+    code_n, code_w = CODE_N, CODE_W
+    if args.profile.endswith("72bit"):                       # ~3 bits/weight: shells 2..53
+        ctx = P.Context(2, 53, device=torch.cuda.current_device())
+        code_n, code_w = ctx.num_points, ctx.index_bits
     layout = 0 if args.profile == "dequant" else 1
     per_copy = algorithmic_bytes(n, k) + (n * k * 2 if args.profile == "dequant" else 0)
     copies = max(2, -(-2 * L2_BYTES // per_copy))
     bufs = []
     for c in range(copies):
-        stream, gain, _ = gen.make_layer(CODE_N, CODE_W, n, k, layout, seed=c)
+        stream, gain, _ = gen.make_layer(code_n, code_w, n, k, layout, seed=c)
         d_idx = torch.from_numpy(stream).cuda()
         if args.profile == "gemv_sorted":
             d_idx = P.llvq_sort_blocks(ctx, d_idx, n, k)
-        if args.profile == "gemm_sorted":
+        if args.profile.startswith("gemm_sorted"):
             d_idx = P.llvq_sort_blocks_gemm(ctx, d_idx, n, k)
         bufs.append((d_idx, torch.from_numpy(gain.view(np.float16)).cuda()))
     x = torch.from_numpy(gen.normal_bf16((16, k), seed=0).view(np.int16)).cuda().view(torch.bfloat16)
@@ -222,7 +227,7 @@ def profile_run(P, ctx, args) -> None:
             P.llvq_gemv(ctx, d_idx, d_gain, n, k, x[0], d_y=y[:n])
         elif args.profile == "gemv_sorted":
             P.llvq_gemv_sorted(ctx, d_idx, d_gain, n, k, x[0], d_y=y[:n])
-        elif args.profile == "gemm_sorted":
+        elif args.profile.startswith("gemm_sorted"):
             P.llvq_gemm_small_batch_sorted(ctx, d_idx, d_gain, n, k, x, d_y=y.view(16, n))
         elif args.profile == "dequant":
             P.llvq_dequant_matrix(ctx, d_idx, d_gain, n, k, 0, d_w=w)
@@ -366,6 +371,27 @@ def extras(P, ctx) -> dict:
     torch.cuda.synchronize()
     sweep_graph_us = _event_us(torch, lambda i: graph.replay(), 3)
     del graph, sorted_weights
+    # ... and with the matrices that share an input stored as one (q|k|v: 6144 x 4096, gate|up: 28672 x 4096): the same
+    # blocks in 4 launches per layer instead of 7
+    fused_shapes = [(6144, 4096), (4096, 4096), (28672, 4096), (4096, 14336)]
+    assert sum(n * ((k + 23) // 24) for n, k in fused_shapes) == sum(n * ((k + 23) // 24) for n, k in shapes)
+    fused = []
+    for c in range(4):
+        layer = []
+        for li, (n, k) in enumerate(fused_shapes):
+            stream, gain, nb = gen.make_layer(CODE_N, CODE_W, n, k, 1, seed=350 + 10 * c + li)
+            layer.append((P.llvq_sort_blocks(ctx, dev(stream), n, k), dev(gain, np.float16)))
+        fused.append(layer)
+    ysf = {n: torch.empty(n, dtype=torch.bfloat16, device="cuda") for n in (6144, 4096, 28672)}
+
+    def token_fused(i):
+        for layer in range(32):
+            for (n, k), (d_srt, d_gain) in zip(fused_shapes, fused[(i * 32 + layer) % 4]):
+                P.llvq_gemv_sorted(ctx, d_srt, d_gain, n, k, xs[k], d_y=ysf[n])
+    token_fused(0)
+    torch.cuda.synchronize()
+    sweep_fused_us = _event_us(torch, token_fused, 3)
+    del fused
     blocks = 32 * sum(n * ((k + 23) // 24) for n, k in shapes)
     by = blocks * (CODE_W // 8 + 2) + 32 * sum(2 * k + 2 * n for n, k in shapes)
     # --- the one shape the paper timed (App. C): (4096 x 4104) . (4104 x 1), single shell M = 3 (24-bit indices, 1 bit/weight)
@@ -454,6 +480,8 @@ def extras(P, ctx) -> dict:
     out["llama3_8b_linear_sweep"] = {"us_per_token": sweep_us, "tokens_per_s": 1e6 / sweep_us, "GBps": by / sweep_us / 1e3, "blocks_per_token": blocks,
                                      "launches_per_token": 32 * len(shapes), "algorithmic_bytes": by,
                                      "sorted_layout": {"us_per_token": sweep_sorted_us, "tokens_per_s": 1e6 / sweep_sorted_us, "GBps": by / sweep_sorted_us / 1e3},
+                                     "sorted_layout_fused_qkv_gateup": {"us_per_token": sweep_fused_us, "tokens_per_s": 1e6 / sweep_fused_us,
+                                                                        "launches_per_token": 32 * len(fused_shapes)},
                                      "sorted_layout_cuda_graph": {"us_per_token": sweep_graph_us, "tokens_per_s": 1e6 / sweep_graph_us,
                                                                   "note": "one layer set (73 MB sorted + 18 MB gains) replayed: partly L2-resident"}}
     return out
@@ -467,7 +495,7 @@ def main() -> None:
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-extras", action="store_true", help="skip the secondary configurations (dequant, GEMM, decoder sweep)")
-    ap.add_argument("--profile", default=None, choices=["gemv", "dequant", "gemm", "gemv_sorted", "gemm_sorted"],
+    ap.add_argument("--profile", default=None, choices=["gemv", "dequant", "gemm", "gemv_sorted", "gemm_sorted", "gemm_72bit", "gemm_sorted_72bit"],
                     help="run only a few launches of one kernel over rotating buffers (for ncu captures); no timing line")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
@@ -651,8 +679,8 @@ def main() -> None:
                          "traffic": NCU_TRAFFIC_BYTES_11008x4096, "kernel": "gemv_bin_kernel on 11008x4096",
                          "algorithmic_bytes_per_launch": dom_bytes, "peak_source": f"of {which}", "frac_of_nominal_8TBps": achieved / 8000.0,
                          # what binds the kernel instead of HBM: counters of the ncu capture summarised under profiles/
-                         "ncu": {"warp_instructions_per_block": 963, "issue_slots_used": 0.626, "alu_pipe_busy": 0.578,
-                                 "shared_memory_wavefronts_per_block": 210, "instructions_per_block_at_hbm_roofline": 46}},
+                         "ncu": {"warp_instructions_per_block": 946, "issue_slots_used": 0.655, "alu_pipe_busy": 0.599,
+                                 "shared_memory_wavefronts_per_block": 208, "instructions_per_block_at_hbm_roofline": 46}},
             "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "ms_per_step": e2e_ms},
             "gpu_launches": timed_launches,
             "clocks": clocks.summary(),

@@ -85,6 +85,26 @@ def test_every_copy_of_y_holds_the_product(lib, ctx, code, n_out, k_in, world, d
         assert torch.equal(copies[r][:n_out], copies[0][:n_out])
 
 
+def test_degenerate_bands_still_raise_their_flags(lib, ctx, code):
+    o = code
+    stream, gain, _ = gen.make_layer(o.N, o.W, 8, 48, 1, seed=2)
+    ds, dg, dx = to_dev_u8(stream), to_dev_f16(gain), to_dev_bf16(gen.normal_bf16(48, seed=2))
+    copies = [torch.full((16,), 5.0, device="cuda") for _ in range(2)]
+    flags = [torch.zeros(2, dtype=torch.int32, device="cuda") for _ in range(2)]
+    words = lambda r: [flags[p].data_ptr() + 4 * r for p in range(2)]
+    # rank 0 has no rows at all: nothing is written, the peer still hears from it
+    lib.llvq_gemv_rowshard(ctx, ds, dg, 0, 48, dx, copies, 0, 0, torch.float32, flag_words=words(0), epoch=3)
+    # rank 1 has rows but no columns: its rows are zero everywhere
+    lib.llvq_gemv_rowshard(ctx, ds, dg, 8, 0, dx, copies, 1, 8, torch.float32, flag_words=words(1), epoch=3)
+    for r in range(2):
+        lib.llvq_wait_ranks(ctx, flags[r], 2, r, 3)
+    torch.cuda.synchronize()
+    assert lib.llvq_last_error(ctx) == (0, 0)
+    assert flags[0].tolist() == [0, 3] and flags[1].tolist() == [3, 0]
+    for c in copies:
+        assert c[:8].tolist() == [5.0] * 8 and c[8:].tolist() == [0.0] * 8
+
+
 def test_wait_runs_out_on_a_flag_nobody_raises(lib, ctx):
     flags = torch.zeros(4, dtype=torch.int32, device="cuda")
     flags[1] = 7
