@@ -42,6 +42,8 @@ WORKLOAD = "configs[2]: fused dequant+GEMV batch 1 on W 4096x4096, 11008x4096, 4
 # dram__bytes_read.sum + dram__bytes_write.sum of one gemv_fast_kernel launch on the 11008x4096 layer, from the
 # ncu capture summarised under profiles/ (algorithmic bytes: 15 089 152)
 NCU_TRAFFIC_BYTES_11008x4096 = 15272960
+NCU_WARP_INSTRUCTIONS_11008x4096 = 55678667          # smsp__inst_executed.sum of the same capture
+ISSUE_PEAK_WARP_INST_PER_S = 148 * 4 * 1.965e9       # SMs x schedulers x max SM clock: one warp instruction per scheduler and cycle
 
 
 def layer_bytes(n_out: int, k_in: int) -> dict:
@@ -681,6 +683,11 @@ def main() -> None:
                          # what binds the kernel instead of HBM: counters of the ncu capture summarised under profiles/
                          "ncu": {"warp_instructions_per_block": 946, "issue_slots_used": 0.655, "alu_pipe_busy": 0.599,
                                  "shared_memory_wavefronts_per_block": 208, "instructions_per_block_at_hbm_roofline": 46}},
+            # the same launch against what actually binds it: instruction issue (instructions per launch from the ncu
+            # capture, duration measured live)
+            "roofline_issue": {"bound": "alu", "achieved": NCU_WARP_INSTRUCTIONS_11008x4096 / (dom["us"] * 1e-6), "peak": ISSUE_PEAK_WARP_INST_PER_S,
+                               "unit": "warp-instructions/s", "frac": NCU_WARP_INSTRUCTIONS_11008x4096 / (dom["us"] * 1e-6) / ISSUE_PEAK_WARP_INST_PER_S,
+                               "kernel": "gemv_bin_kernel on 11008x4096", "peak_source": "148 SMs x 4 schedulers x 1.965 GHz"},
             "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "ms_per_step": e2e_ms},
             "gpu_launches": timed_launches,
             "clocks": clocks.summary(),
