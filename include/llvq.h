@@ -308,6 +308,21 @@ int llvq_gemv_sorted_rowshard(const llvq_ctx* ctx, const void* d_sorted, const u
                               int64_t row0, int y_dtype, uint32_t* const* d_flag_words, uint32_t epoch, void* stream);
 
 /*
+ * The same for the small-batch product: the band's rows are the columns [row0, row0 + n_rows) of every rank's
+ * Y [batch][n_out_total] (bf16).  d_y_all lists the starts of those full matrices.  Stream, gains, X, batch and limits
+ * as in llvq_gemm_small_batch / llvq_gemm_small_batch_sorted (called with n_out = n_rows), flags as above.
+ */
+int llvq_gemm_small_batch_rowshard(const llvq_ctx* ctx, const void* d_idx, const uint16_t* d_gain_f16, int64_t n_rows,
+                                   int64_t k_in, const uint16_t* d_x_bf16, int batch, void* const* d_y_all, int n_dest,
+                                   int own_slot, int64_t row0, int64_t n_out_total, uint32_t* const* d_flag_words,
+                                   uint32_t epoch, void* stream);
+int llvq_gemm_small_batch_sorted_rowshard(const llvq_ctx* ctx, const void* d_sorted, const uint16_t* d_gain_f16,
+                                          int64_t n_rows, int64_t k_in, const uint16_t* d_x_bf16, int batch,
+                                          void* const* d_y_all, int n_dest, int own_slot, int64_t row0,
+                                          int64_t n_out_total, uint32_t* const* d_flag_words, uint32_t epoch,
+                                          void* stream);
+
+/*
  * Exchange buffers for the above (no counterpart in the paper: plumbing between processes).
  * llvq_exchange_create allocates `bytes` of zeroed device memory on the context's device as an allocation of its
  * own (so that it can be exported whole), returns it in *d_buf and writes its inter-process handle

@@ -22,6 +22,7 @@ __all__ = [
     "llvq_sort_blocks_sg", "llvq_gemv_sorted_sg", "llvq_gemm_small_batch_sg",
     "llvq_gemv_rowshard", "llvq_gemv_sorted_rowshard", "llvq_exchange_create", "llvq_exchange_destroy", "llvq_exchange_open",
     "llvq_exchange_close", "llvq_signal_ranks", "llvq_wait_ranks", "LLVQ_EXCHANGE_HANDLE_BYTES",
+    "llvq_gemm_small_batch_rowshard", "llvq_gemm_small_batch_sorted_rowshard",
     "llvq_last_error", "LlvqError", "EXPORTS", "load_library",
     "LLVQ_LAYOUT_FLAT", "LLVQ_LAYOUT_ROWWISE", "LLVQ_F32", "LLVQ_BF16",
 ]
@@ -45,6 +46,7 @@ EXPORTS = [
     "llvq_sorted_gemm_bytes", "llvq_sort_blocks_gemm", "llvq_gemm_small_batch_sorted", "llvq_gemm_small_batch_sg",
     "llvq_gemv_rowshard", "llvq_gemv_sorted_rowshard", "llvq_exchange_create", "llvq_exchange_destroy", "llvq_exchange_open",
     "llvq_exchange_close", "llvq_signal_ranks", "llvq_wait_ranks",
+    "llvq_gemm_small_batch_rowshard", "llvq_gemm_small_batch_sorted_rowshard",
 ]
 
 
@@ -105,6 +107,10 @@ def load_library() -> ctypes.CDLL:
              ctypes.c_uint32, vp]
     lib.llvq_gemv_rowshard.argtypes = shard
     lib.llvq_gemv_sorted_rowshard.argtypes = shard
+    gshard = [vp, vp, vp, i64, i64, vp, ctypes.c_int, ctypes.POINTER(vp), ctypes.c_int, ctypes.c_int, i64, i64, ctypes.POINTER(vp),
+              ctypes.c_uint32, vp]
+    lib.llvq_gemm_small_batch_rowshard.argtypes = gshard
+    lib.llvq_gemm_small_batch_sorted_rowshard.argtypes = gshard
     lib.llvq_exchange_create.argtypes = [vp, ctypes.c_size_t, ctypes.POINTER(vp), ctypes.c_char_p]
     lib.llvq_exchange_destroy.argtypes = [vp, vp]
     lib.llvq_exchange_open.argtypes = [vp, ctypes.c_char_p, ctypes.POINTER(vp)]
@@ -476,6 +482,31 @@ def llvq_gemv_sorted_rowshard(ctx: Context, d_sorted: torch.Tensor, d_gain: torc
     assert d_sorted.numel() * d_sorted.element_size() >= int(ctx._lib.llvq_sorted_bytes(ctx._h, n_rows, k_in))
     _gemv_rowshard("llvq_gemv_sorted_rowshard", ctx, d_sorted, d_gain, n_rows, k_in, d_x, y_all, own_slot, row0, y_dtype, flag_words,
                    epoch, stream)
+
+
+def llvq_gemm_small_batch_rowshard(ctx: Context, d_stream: torch.Tensor, d_gain: torch.Tensor, n_rows: int, k_in: int, d_x: torch.Tensor,
+                                   y_all, own_slot: int, row0: int, n_out_total: int, flag_words=None, epoch: int = 0,
+                                   sorted_layout: bool = False, stream=None) -> None:
+    """Small-batch product of one rank's band of rows, written into columns ``row0..`` of every Y [batch][n_out_total]
+    (bf16) in ``y_all``; ``sorted_layout`` = the stream comes from ``llvq_sort_blocks_gemm`` (called with n_out = n_rows)."""
+    assert d_x.dtype == torch.bfloat16 and d_x.dim() == 2 and d_x.shape[1] == k_in and d_gain.dtype == torch.float16
+    assert 1 <= len(y_all) <= 8 and d_gain.numel() >= n_rows * ((k_in + 23) // 24)
+    ptrs = (ctypes.c_void_p * len(y_all))(*[_ptr(y, "y_all") for y in y_all])
+    flags = None
+    if flag_words is not None:
+        assert len(flag_words) == len(y_all)
+        flags = (ctypes.c_void_p * len(y_all))(*[_ptr(w, "flag_words") for w in flag_words])
+    call = "llvq_gemm_small_batch_sorted_rowshard" if sorted_layout else "llvq_gemm_small_batch_rowshard"
+    _check(call, getattr(ctx._lib, call)(ctx._h, _dev(d_stream, "d_stream"), _dev(d_gain, "d_gain"), n_rows, k_in, _dev(d_x, "d_x"),
+                                         d_x.shape[0], ptrs, len(y_all), own_slot, row0, n_out_total, flags, epoch & 0xffffffff,
+                                         _stream_ptr(stream)))
+
+
+def llvq_gemm_small_batch_sorted_rowshard(ctx: Context, d_sorted, d_gain, n_rows, k_in, d_x, y_all, own_slot, row0, n_out_total,
+                                          flag_words=None, epoch: int = 0, stream=None) -> None:
+    """``llvq_gemm_small_batch_rowshard`` from the band's sorted stream."""
+    llvq_gemm_small_batch_rowshard(ctx, d_sorted, d_gain, n_rows, k_in, d_x, y_all, own_slot, row0, n_out_total, flag_words, epoch,
+                                   sorted_layout=True, stream=stream)
 
 
 def llvq_exchange_create(ctx: Context, nbytes: int) -> tuple[int, bytes]:

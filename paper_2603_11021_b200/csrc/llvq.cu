@@ -794,7 +794,8 @@ struct GemmArgs {
     int batch, npad;
     int nstages, split;
     const uint16_t* x;
-    uint16_t* y;
+    YOut yo;                   // Y [batch][y_ld] bf16: this rank's copy (and, row-sharded, the peers'), at the first row of the band
+    int64_t y_ld;
     float* scratch;            // [npad][scratch_ld] binary32, all zero on entry and on exit
     int64_t scratch_ld;        // row tiles * 128
     uint32_t* counters;        // [row tiles], zero on entry and on exit
@@ -907,7 +908,7 @@ gemm_kernel(FastArgs fa, const uint32_t* __restrict__ stream, const uint16_t* __
                     for (int i = 0; i < 16; ++i) {
                         const int n = c0 + i;
                         if (n < ga.batch) {
-                            if (ga.split == 1) reinterpret_cast<__nv_bfloat16*>(ga.y)[(int64_t)n * ga.n_out + orow] = __float2bfloat16_rn(v[i]);
+                            if (ga.split == 1) store_y<true>(ga.yo, (int64_t)n * ga.y_ld + orow, v[i]);
                             else atomicAdd(ga.scratch + (int64_t)n * ga.scratch_ld + orow, v[i]);
                         }
                     }
@@ -928,7 +929,7 @@ gemm_kernel(FastArgs fa, const uint32_t* __restrict__ stream, const uint16_t* __
                     const int64_t orow = rt * kGemmRows + (i % kGemmRows);
                     if (orow < ga.n_out) {
                         float* sp = ga.scratch + (int64_t)n * ga.scratch_ld + orow;
-                        reinterpret_cast<__nv_bfloat16*>(ga.y)[(int64_t)n * ga.n_out + orow] = __float2bfloat16_rn(__ldcg(sp));
+                        store_y<true>(ga.yo, (int64_t)n * ga.y_ld + orow, __ldcg(sp));
                         __stcg(sp, 0.f);
                     }
                 }
@@ -938,6 +939,8 @@ gemm_kernel(FastArgs fa, const uint32_t* __restrict__ stream, const uint16_t* __
         __syncthreads();
     }
     if (timeout) atomicOr(fa.flags, 1u);
+    if (ga.yo.n_peer) __threadfence_system();             // this thread's stores to the peers' copies, before the CTA counts itself in
+    shard_arrive(ga.yo);
     __syncthreads();
     if (warp == 0) tmem_dealloc(tmem, kTmemCols);
 }
@@ -1175,7 +1178,7 @@ gemm_sorted_kernel(FastArgs fa, const unsigned long long* __restrict__ sorted, c
                     for (int i = 0; i < 16; ++i) {
                         const int n = c0 + i;
                         if (n < ga.batch) {
-                            if (parts == 1u) reinterpret_cast<__nv_bfloat16*>(ga.y)[(int64_t)n * ga.n_out + orow] = __float2bfloat16_rn(v[i]);
+                            if (parts == 1u) store_y<true>(ga.yo, (int64_t)n * ga.y_ld + orow, v[i]);
                             else atomicAdd(ga.scratch + (int64_t)n * ga.scratch_ld + orow, v[i]);
                         }
                     }
@@ -1196,7 +1199,7 @@ gemm_sorted_kernel(FastArgs fa, const unsigned long long* __restrict__ sorted, c
                     const int64_t orow = rt * kGemmRows + (i % kGemmRows);
                     if (orow < ga.n_out) {
                         float* sp = ga.scratch + (int64_t)n * ga.scratch_ld + orow;
-                        reinterpret_cast<__nv_bfloat16*>(ga.y)[(int64_t)n * ga.n_out + orow] = __float2bfloat16_rn(__ldcg(sp));
+                        store_y<true>(ga.yo, (int64_t)n * ga.y_ld + orow, __ldcg(sp));
                         __stcg(sp, 0.f);
                     }
                 }
@@ -1206,6 +1209,8 @@ gemm_sorted_kernel(FastArgs fa, const unsigned long long* __restrict__ sorted, c
         __syncthreads();
     }
     if (timeout) atomicOr(fa.flags, 1u);
+    if (ga.yo.n_peer) __threadfence_system();             // this thread's stores to the peers' copies, before the CTA counts itself in
+    shard_arrive(ga.yo);
     __syncthreads();
     if (warp == 0) tmem_dealloc(tmem, kTmemCols);
 }
@@ -1259,15 +1264,18 @@ int check_gemm_args(const llvq_ctx* ctx, const void* d_idx, const uint16_t* d_ga
 
 // Enqueue gemm_sorted_kernel on a stream sorted by llvq_sort_blocks_gemm.
 int launch_gemm_domains(const llvq_ctx* ctx, const void* p, const uint16_t* d_gain_f16, int64_t n_out, int64_t k_in,
-                        const uint16_t* d_x_bf16, int batch, uint16_t* d_y_bf16, float* scratch, uint32_t* counters, void* stream)
+                        const uint16_t* d_x_bf16, int batch, uint16_t* d_y_bf16, float* scratch, uint32_t* counters, void* stream,
+                        const YOut* yo = nullptr, int64_t y_ld = 0)
 {
     DeviceGuard guard(ctx->device);
     if (!guard.ok) return LLVQ_ECUDA;
     GemmArgs ga;
+    ga.yo = YOut{}; ga.yo.y = d_y_bf16; ga.y_ld = n_out;
+    if (yo) { ga.yo = *yo; ga.y_ld = y_ld; }
     ga.n_out = n_out; ga.k_in = k_in; ga.bpr = (k_in + 23) / 24;
     ga.batch = batch; ga.npad = (batch + 15) / 16 * 16;
     ga.nstages = (int)((ga.bpr + kDomBlocks - 1) / kDomBlocks);              // domains per row tile
-    ga.x = d_x_bf16; ga.y = d_y_bf16; ga.scratch = scratch; ga.counters = counters;
+    ga.x = d_x_bf16; ga.scratch = scratch; ga.counters = counters;
     const int dpi = ga.npad <= 32 ? 2 : 1;                                   // domains unranked per iteration (shared memory decides)
     const int64_t row_tiles = (n_out + kGemmRows - 1) / kGemmRows;
     ga.scratch_ld = row_tiles * kGemmRows;
@@ -1291,7 +1299,7 @@ int launch_gemm_domains(const llvq_ctx* ctx, const void* p, const uint16_t* d_ga
 // ([row tiles]); both must be zero when the kernel starts and are zero again when it ends.
 int launch_gemm(const llvq_ctx* ctx, const void* d_idx, const uint16_t* d_gain_f16, int64_t n_out, int64_t k_in,
                 const uint16_t* d_x_bf16, int batch, uint16_t* d_y_bf16, float* scratch, uint32_t* counters, void* stream,
-                const SgArgs* sg = nullptr)
+                const SgArgs* sg = nullptr, const YOut* yo = nullptr, int64_t y_ld = 0)
 {
     if (n_out == 0) return LLVQ_OK;
     DeviceGuard guard(ctx->device);
@@ -1299,10 +1307,12 @@ int launch_gemm(const llvq_ctx* ctx, const void* d_idx, const uint16_t* d_gain_f
     cudaStream_t st = (cudaStream_t)stream;
     if (k_in == 0) return cudaMemsetAsync(d_y_bf16, 0, (size_t)n_out * batch * 2, st) == cudaSuccess ? LLVQ_OK : LLVQ_ECUDA;
     GemmArgs ga;
+    ga.yo = YOut{}; ga.yo.y = d_y_bf16; ga.y_ld = n_out;
+    if (yo) { ga.yo = *yo; ga.y_ld = y_ld; }
     ga.n_out = n_out; ga.k_in = k_in; ga.bpr = (k_in + 23) / 24;
     ga.batch = batch; ga.npad = (batch + 15) / 16 * 16;
     ga.nstages = (int)((ga.bpr + kStageBlocks - 1) / kStageBlocks);
-    ga.x = d_x_bf16; ga.y = d_y_bf16; ga.scratch = scratch; ga.counters = counters;
+    ga.x = d_x_bf16; ga.scratch = scratch; ga.counters = counters;
     // split K so that the work items fill the SMs evenly, keeping at least four stages per item
     const int64_t row_tiles = (n_out + kGemmRows - 1) / kGemmRows;
     ga.scratch_ld = row_tiles * kGemmRows;
@@ -1824,6 +1834,7 @@ static int shard_yout(const llvq_ctx* ctx, void* const* d_y_all, int n_dest, int
     *yo = YOut{};
     for (int d = 0; d < n_dest; ++d) {
         if (!d_y_all[d]) return LLVQ_EINVAL;
+        if (!aligned(d_y_all[d], es)) return LLVQ_EALIGN;
         void* at = static_cast<unsigned char*>(d_y_all[d]) + (size_t)row0 * es;
         if (d == own_slot) { yo->y = at; continue; }
         yo->peer[yo->n_peer++] = at;
@@ -1939,6 +1950,50 @@ int llvq_gemm_small_batch(const llvq_ctx* ctx, const void* d_idx, const uint16_t
     if (int e = check_gemm_args(ctx, d_idx, d_gain_f16, n_out, k_in, d_x_bf16, batch, d_y_bf16)) return e;
     if (n_out > kMaxScratchRows) return LLVQ_EUNSUPPORTED;
     return launch_gemm(ctx, d_idx, d_gain_f16, n_out, k_in, d_x_bf16, batch, d_y_bf16, ctx->d_scratch, ctx->d_counters, stream);
+}
+
+// Row-sharded small-batch GEMM: the band's columns [row0, row0 + n_rows) of every rank's Y [batch][n_out_total].
+static int gemm_rowshard(const llvq_ctx* ctx, const void* d_stream, bool sorted, const uint16_t* d_gain_f16, int64_t n_rows, int64_t k_in,
+                         const uint16_t* d_x_bf16, int batch, void* const* d_y_all, int n_dest, int own_slot, int64_t row0,
+                         int64_t n_out_total, uint32_t* const* d_flag_words, uint32_t epoch, void* stream)
+{
+    YOut yo;
+    if (int e = shard_yout(ctx, d_y_all, n_dest, own_slot, row0, LLVQ_BF16, d_flag_words, epoch, &yo)) return e;
+    if (n_rows < 0 || n_out_total < row0 + n_rows) return LLVQ_EINVAL;
+    if (n_rows == 0) return signal_only(ctx, yo, stream);
+    if (int e = check_gemm_args(ctx, d_stream, d_gain_f16, n_rows, k_in, d_x_bf16, batch, static_cast<const uint16_t*>(yo.y))) return e;
+    if (n_rows > kMaxScratchRows) return LLVQ_EUNSUPPORTED;
+    if (k_in == 0) {                                   // Y = 0 by copies, no kernel to raise the flags
+        DeviceGuard guard(ctx->device);
+        if (!guard.ok) return LLVQ_ECUDA;
+        for (int p = -1; p < yo.n_peer; ++p)
+            if (cudaMemset2DAsync(p < 0 ? yo.y : yo.peer[p], (size_t)n_out_total * 2, 0, (size_t)n_rows * 2, (size_t)batch,
+                                  (cudaStream_t)stream) != cudaSuccess) return LLVQ_ECUDA;
+        return signal_only(ctx, yo, stream);
+    }
+    if (sorted) {
+        if (!gemm_sortable(ctx)) return LLVQ_EUNSUPPORTED;
+        return launch_gemm_domains(ctx, d_stream, d_gain_f16, n_rows, k_in, d_x_bf16, batch, nullptr, ctx->d_scratch, ctx->d_counters, stream,
+                                   &yo, n_out_total);
+    }
+    return launch_gemm(ctx, d_stream, d_gain_f16, n_rows, k_in, d_x_bf16, batch, nullptr, ctx->d_scratch, ctx->d_counters, stream, nullptr,
+                       &yo, n_out_total);
+}
+
+int llvq_gemm_small_batch_rowshard(const llvq_ctx* ctx, const void* d_idx, const uint16_t* d_gain_f16, int64_t n_rows, int64_t k_in,
+                                   const uint16_t* d_x_bf16, int batch, void* const* d_y_all, int n_dest, int own_slot, int64_t row0,
+                                   int64_t n_out_total, uint32_t* const* d_flag_words, uint32_t epoch, void* stream)
+{
+    return gemm_rowshard(ctx, d_idx, false, d_gain_f16, n_rows, k_in, d_x_bf16, batch, d_y_all, n_dest, own_slot, row0, n_out_total,
+                         d_flag_words, epoch, stream);
+}
+
+int llvq_gemm_small_batch_sorted_rowshard(const llvq_ctx* ctx, const void* d_sorted, const uint16_t* d_gain_f16, int64_t n_rows, int64_t k_in,
+                                          const uint16_t* d_x_bf16, int batch, void* const* d_y_all, int n_dest, int own_slot, int64_t row0,
+                                          int64_t n_out_total, uint32_t* const* d_flag_words, uint32_t epoch, void* stream)
+{
+    return gemm_rowshard(ctx, d_sorted, true, d_gain_f16, n_rows, k_in, d_x_bf16, batch, d_y_all, n_dest, own_slot, row0, n_out_total,
+                         d_flag_words, epoch, stream);
 }
 
 

@@ -85,6 +85,38 @@ def test_every_copy_of_y_holds_the_product(lib, ctx, code, n_out, k_in, world, d
         assert torch.equal(copies[r][:n_out], copies[0][:n_out])
 
 
+@pytest.mark.parametrize("sorted_layout", [False, True])
+@pytest.mark.parametrize("n_out,k_in,world,batch", [(1000, 2000, 2, 16), (520, 1536, 4, 5), (300, 4096, 3, 64)])
+def test_every_copy_of_the_batched_product(lib, ctx, code, n_out, k_in, world, batch, sorted_layout):
+    from paper_2603_11021_b200.rowshard import band_of_stream, row_bands
+    o = code
+    stream, gain, _ = gen.make_layer(o.N, o.W, n_out, k_in, 1, seed=33)
+    x = gen.normal_bf16((batch, k_in), seed=33)
+    want = o.gemm(stream, gain, n_out, k_in, x, threads=4)
+    dx = to_dev_bf16(x)
+    copies = [torch.full((batch + 1, n_out), float("nan"), dtype=torch.bfloat16, device="cuda") for _ in range(world)]
+    flags = [torch.zeros(world, dtype=torch.int32, device="cuda") for _ in range(world)]
+    for r, (row0, n) in enumerate(row_bands(n_out, world, align=128 if sorted_layout else 8)):
+        s, g = band_of_stream(stream, gain, k_in, o.W, row0, n)
+        ds, dg = to_dev_u8(s), to_dev_f16(g)
+        if sorted_layout and n:
+            ds = lib.llvq_sort_blocks_gemm(ctx, ds, n, k_in)
+        words = [flags[p].data_ptr() + 4 * r for p in range(world)]
+        lib.llvq_gemm_small_batch_rowshard(ctx, ds, dg, n, k_in, dx, copies, r, row0, n_out, flag_words=words, epoch=2,
+                                           sorted_layout=sorted_layout)
+    for r in range(world):
+        lib.llvq_wait_ranks(ctx, flags[r], world, r, 2)
+    torch.cuda.synchronize()
+    assert lib.llvq_last_error(ctx) == (0, 0)
+    for r in range(world):
+        f = flags[r].cpu().numpy()
+        assert all(f[p] == (0 if p == r else 2) for p in range(world))
+        y = copies[r].float().cpu().numpy()
+        assert np.isnan(y[batch]).all()            # nothing written past the matrix
+        assert gemv_error(y[:batch], want) <= TOL_BF16_OUT
+        assert torch.equal(copies[r][:batch], copies[0][:batch])
+
+
 def test_degenerate_bands_still_raise_their_flags(lib, ctx, code):
     o = code
     stream, gain, _ = gen.make_layer(o.N, o.W, 8, 48, 1, seed=2)
