@@ -50,6 +50,8 @@ def band_of_stream(stream: np.ndarray, gains: np.ndarray, k_in: int, index_bits:
     back padded to a multiple of 16, as the device calls expect.
     """
     bpr = (k_in + 23) // 24
+    if n_rows == 0:                                # an empty band (more ranks than row groups) may sit anywhere
+        return np.zeros(0, dtype=np.uint8), np.asarray(gains)[:0].copy()
     b0, b1 = row0 * bpr * index_bits, (row0 + n_rows) * bpr * index_bits
     if b0 % 8:
         raise ValueError("band_of_stream: the band does not start on a byte boundary")

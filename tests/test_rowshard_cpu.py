@@ -37,7 +37,8 @@ def test_row_bands_rejects_nonsense():
             row_bands(*args)
 
 
-@pytest.mark.parametrize("code,n_out,k_in,world", [((2, 13), 67, 500, 3), ((2, 2), 40, 768, 2), ((3, 3), 24, 100, 4)])
+@pytest.mark.parametrize("code,n_out,k_in,world", [((2, 13), 67, 500, 3), ((2, 2), 40, 768, 2), ((3, 3), 24, 100, 4),
+                                                   ((2, 2), 5, 24, 3)])          # the last one: empty bands that start at row 5
 def test_bands_of_a_stream_give_the_bands_of_y(oracle_mod, code, n_out, k_in, world):
     o = oracle_mod.Code(*code)
     stream, gain, _ = gen.make_layer(o.N, o.W, n_out, k_in, 1, seed=12)
