@@ -226,6 +226,12 @@ int llvq_sort_blocks_gemm(const llvq_ctx* ctx, const void* d_idx, int64_t n_out,
 int llvq_gemm_small_batch_sorted(const llvq_ctx* ctx, const void* d_sorted, const uint16_t* d_gain_f16,
                                  int64_t n_out, int64_t k_in, const uint16_t* d_x_bf16,
                                  int batch, uint16_t* d_y_bf16, void* stream);
+/* The same for the shape-gain form (fields of llvq_index_bits(ctx) + gain_bits <= 48 bits; see llvq_sort_blocks_sg). */
+int llvq_sort_blocks_gemm_sg(const llvq_ctx* ctx, const void* d_fields, int gain_bits, int64_t n_out, int64_t k_in,
+                             void* d_sorted, void* stream);
+int llvq_gemm_small_batch_sorted_sg(const llvq_ctx* ctx, const void* d_sorted, int gain_bits, const float* d_codebook_f32,
+                                    const float* d_row_scale_f32, int64_t n_out, int64_t k_in, const uint16_t* d_x_bf16,
+                                    int batch, uint16_t* d_y_bf16, void* stream);
 
 /*
  * llvq_gemm_small_batch for callers that cannot allocate device memory.  (The paper has no

@@ -23,6 +23,7 @@ __all__ = [
     "llvq_gemv_rowshard", "llvq_gemv_sorted_rowshard", "llvq_exchange_create", "llvq_exchange_destroy", "llvq_exchange_open",
     "llvq_exchange_close", "llvq_signal_ranks", "llvq_wait_ranks", "LLVQ_EXCHANGE_HANDLE_BYTES",
     "llvq_gemm_small_batch_rowshard", "llvq_gemm_small_batch_sorted_rowshard",
+    "llvq_sort_blocks_gemm_sg", "llvq_gemm_small_batch_sorted_sg",
     "llvq_last_error", "LlvqError", "EXPORTS", "load_library",
     "LLVQ_LAYOUT_FLAT", "LLVQ_LAYOUT_ROWWISE", "LLVQ_F32", "LLVQ_BF16",
 ]
@@ -47,6 +48,7 @@ EXPORTS = [
     "llvq_gemv_rowshard", "llvq_gemv_sorted_rowshard", "llvq_exchange_create", "llvq_exchange_destroy", "llvq_exchange_open",
     "llvq_exchange_close", "llvq_signal_ranks", "llvq_wait_ranks",
     "llvq_gemm_small_batch_rowshard", "llvq_gemm_small_batch_sorted_rowshard",
+    "llvq_sort_blocks_gemm_sg", "llvq_gemm_small_batch_sorted_sg",
 ]
 
 
@@ -91,6 +93,8 @@ def load_library() -> ctypes.CDLL:
     lib.llvq_sort_blocks.argtypes = [vp, vp, i64, i64, vp, vp]
     lib.llvq_gemv_sorted.argtypes = [vp, vp, vp, i64, i64, vp, vp, ctypes.c_int, vp]
     lib.llvq_gemm_small_batch_sg.argtypes = [vp, vp, ctypes.c_int, vp, vp, i64, i64, vp, ctypes.c_int, vp, vp]
+    lib.llvq_sort_blocks_gemm_sg.argtypes = [vp, vp, ctypes.c_int, i64, i64, vp, vp]
+    lib.llvq_gemm_small_batch_sorted_sg.argtypes = [vp, vp, ctypes.c_int, vp, vp, i64, i64, vp, ctypes.c_int, vp, vp]
     lib.llvq_sort_blocks_sg.argtypes = [vp, vp, ctypes.c_int, i64, i64, vp, vp]
     lib.llvq_gemv_sorted_sg.argtypes = [vp, vp, ctypes.c_int, vp, vp, i64, i64, vp, vp, ctypes.c_int, vp]
     lib.llvq_sorted_gemm_bytes.argtypes = [vp, i64, i64]
@@ -400,6 +404,39 @@ def llvq_gemm_small_batch_sorted(ctx: Context, d_sorted: torch.Tensor, d_gain: t
     assert d_sorted.numel() * d_sorted.element_size() >= int(ctx._lib.llvq_sorted_gemm_bytes(ctx._h, n_out, k_in))
     _check("llvq_gemm_small_batch_sorted", ctx._lib.llvq_gemm_small_batch_sorted(
         ctx._h, _dev(d_sorted, "d_sorted"), _dev(d_gain, "d_gain"), n_out, k_in, _dev(d_x, "d_x"), batch, _dev(d_y, "d_y"), _stream_ptr(stream)))
+    return d_y
+
+
+def llvq_sort_blocks_gemm_sg(ctx: Context, d_fields: torch.Tensor, gain_bits: int, n_out: int, k_in: int,
+                             d_sorted: torch.Tensor | None = None, stream=None):
+    """``llvq_sort_blocks_gemm`` for a stream of shape-gain fields (index_bits + gain_bits <= 48 bits each)."""
+    nbytes = int(ctx._lib.llvq_sorted_gemm_bytes(ctx._h, n_out, k_in))
+    if nbytes == 0:
+        raise LlvqError("llvq_sorted_gemm_bytes", 3)
+    if d_sorted is None:
+        d_sorted = torch.empty(nbytes, dtype=torch.uint8, device=d_fields.device)
+    assert d_sorted.numel() * d_sorted.element_size() >= nbytes
+    _check("llvq_sort_blocks_gemm_sg", ctx._lib.llvq_sort_blocks_gemm_sg(ctx._h, _dev(d_fields, "d_fields"), gain_bits, n_out, k_in,
+                                                                         _dev(d_sorted, "d_sorted"), _stream_ptr(stream)))
+    return d_sorted
+
+
+def llvq_gemm_small_batch_sorted_sg(ctx: Context, d_sorted: torch.Tensor, gain_bits: int, d_codebook: torch.Tensor,
+                                    d_row_scale: torch.Tensor | None, n_out: int, k_in: int, d_x: torch.Tensor,
+                                    d_y: torch.Tensor | None = None, stream=None):
+    """``llvq_gemm_small_batch_sg`` from the sorted stream of ``llvq_sort_blocks_gemm_sg``."""
+    assert d_x.dtype == torch.bfloat16 and d_x.dim() == 2 and d_x.shape[1] == k_in
+    batch = d_x.shape[0]
+    if d_y is None:
+        d_y = torch.empty((batch, n_out), dtype=torch.bfloat16, device=d_sorted.device)
+    assert d_y.dtype == torch.bfloat16 and d_y.numel() >= batch * n_out
+    assert d_sorted.numel() * d_sorted.element_size() >= int(ctx._lib.llvq_sorted_gemm_bytes(ctx._h, n_out, k_in))
+    assert d_codebook.dtype == torch.float32 and d_codebook.numel() >= (1 << gain_bits)
+    assert d_row_scale is None or (d_row_scale.dtype == torch.float32 and d_row_scale.numel() >= n_out)
+    _check("llvq_gemm_small_batch_sorted_sg", ctx._lib.llvq_gemm_small_batch_sorted_sg(
+        ctx._h, _dev(d_sorted, "d_sorted"), gain_bits, _dev(d_codebook, "d_codebook"),
+        None if d_row_scale is None else _dev(d_row_scale, "d_row_scale"), n_out, k_in, _dev(d_x, "d_x"), batch, _dev(d_y, "d_y"),
+        _stream_ptr(stream)))
     return d_y
 
 

@@ -25,6 +25,7 @@ struct llvq_ctx {
     int sm_count = 0;
     float* d_scratch = nullptr;      // split-K accumulation buffer of the small-batch GEMM, kept all-zero between calls
     uint32_t* d_counters = nullptr;  // per row tile arrival counters, kept zero between calls
+    void* d_shard = nullptr;         // device copy of the destinations (peers' Y and flags) of the row-sharded GEMM in flight
     bool fast = false;               // class tables fit the shared-memory image; otherwise they are read from global memory
     llvq::FastLayout fl{};
     const uint8_t* d_image = nullptr;

@@ -238,17 +238,19 @@ struct YOut {
     int n_flag;
 };
 
-template <bool kOutBf16>
+template <bool kOutBf16, bool kShard>
 __device__ __forceinline__ void store_y(const YOut& yo, int64_t row, float v)
 {
     if (kOutBf16) {
         const __nv_bfloat16 h = __float2bfloat16_rn(v);
         reinterpret_cast<__nv_bfloat16*>(yo.y)[row] = h;
+        if (!kShard) return;                              // the single-GPU instantiations carry none of what follows
 #pragma unroll
         for (int p = 0; p < kMaxShardPeers; ++p)          // static indices: the struct stays in the parameter bank
             if (p < yo.n_peer) reinterpret_cast<__nv_bfloat16*>(yo.peer[p])[row] = h;
     } else {
         reinterpret_cast<float*>(yo.y)[row] = v;
+        if (!kShard) return;
 #pragma unroll
         for (int p = 0; p < kMaxShardPeers; ++p)
             if (p < yo.n_peer) reinterpret_cast<float*>(yo.peer[p])[row] = v;
@@ -291,7 +293,7 @@ __device__ __forceinline__ void stage_x(uint32_t* xs, const uint16_t* __restrict
 // neighbouring CTAs goes through the scratch row in global memory: add, make the add visible, count the arrival;
 // whoever arrives last reads the total, writes y and leaves scratch and counter zero for the next launch.
 // The caller puts a __syncthreads() before (sums complete) and after (sums may be cleared) the call.
-template <bool kOutBf16, typename RowSum>
+template <bool kOutBf16, bool kShard, typename RowSum>
 __device__ __forceinline__ void finish_pass(const YOut& yo, int64_t rg0, int64_t rg1, int64_t nq, int64_t u_begin, int64_t u_end,
                                             int64_t U, int64_t G, int64_t n_out, float* __restrict__ scratch,
                                             uint32_t* __restrict__ counters, RowSum row_sum)
@@ -304,8 +306,8 @@ __device__ __forceinline__ void finish_pass(const YOut& yo, int64_t rg0, int64_t
         const float part = lane < kGemvGroupRows ? row_sum((rg - rg0) * kGemvGroupRows + lane) : 0.f;
         if (whole) {
             if (mine) {
-                store_y<kOutBf16>(yo, row, part);
-                if (yo.n_peer) __threadfence_system();
+                store_y<kOutBf16, kShard>(yo, row, part);
+                if (kShard) __threadfence_system();
             }
             continue;
         }
@@ -322,9 +324,9 @@ __device__ __forceinline__ void finish_pass(const YOut& yo, int64_t rg0, int64_t
         if (is_last) {
             __threadfence();
             if (mine) {
-                store_y<kOutBf16>(yo, row, __ldcg(scratch + row));
+                store_y<kOutBf16, kShard>(yo, row, __ldcg(scratch + row));
                 __stcg(scratch + row, 0.f);
-                if (yo.n_peer) __threadfence_system();
+                if (kShard) __threadfence_system();
             }
             if (lane == 0) counters[rg] = 0u;
         }
@@ -348,7 +350,7 @@ __device__ __forceinline__ void shard_arrive(const YOut& yo)
         if (p < yo.n_flag) asm volatile("st.release.sys.global.u32 [%0], %1;" ::"l"(yo.flag[p]), "r"(yo.epoch) : "memory");
 }
 
-template <bool kBig, bool kOutBf16, bool kSg = false>
+template <bool kBig, bool kOutBf16, bool kSg = false, bool kShard = false>
 __global__ void __launch_bounds__(kGemvThreads, 1)
 gemv_fast_kernel(FastArgs fa, const uint32_t* __restrict__ stream, const uint16_t* __restrict__ gain, SgArgs sg,
                  int64_t n_out, int64_t k_in, int64_t bpr, const uint16_t* __restrict__ x, YOut yo,
@@ -391,10 +393,10 @@ gemv_fast_kernel(FastArgs fa, const uint32_t* __restrict__ stream, const uint16_
         }
         __syncthreads();
         // row groups this CTA covers completely are final; the (at most two) split ones go through the scratch
-        finish_pass<kOutBf16>(yo, rg0, rg1, nq, u_begin, u_end, U, G, n_out, scratch, counters, [&](int64_t r) { return acc[r]; });
+        finish_pass<kOutBf16, kShard>(yo, rg0, rg1, nq, u_begin, u_end, U, G, n_out, scratch, counters, [&](int64_t r) { return acc[r]; });
         __syncthreads();                                   // the sums are read above: the next pass may clear them only now
     }
-    shard_arrive(yo);
+    if (kShard) shard_arrive(yo);
 }
 
 constexpr uint32_t kKindEven = 0u, kKindOdd = 1u, kKindOther = 2u, kKindNull = 3u;   // decoder form a class needs
@@ -523,7 +525,7 @@ __device__ __forceinline__ uint32_t decode_sorted_entry(const FastArgs& fa, cons
     return cls;
 }
 
-template <bool kOutBf16, bool kSg = false>
+template <bool kOutBf16, bool kSg = false, bool kShard = false>
 __global__ void __launch_bounds__(kSortThreads, 1)
 gemv_sorted_kernel(FastArgs fa, const unsigned long long* __restrict__ sorted, const uint16_t* __restrict__ gain, SgArgs sg,
                    int64_t n_out, int64_t k_in, int64_t bpr, uint32_t nq_magic, const uint16_t* __restrict__ x, YOut yo,
@@ -540,7 +542,6 @@ gemv_sorted_kernel(FastArgs fa, const unsigned long long* __restrict__ sorted, c
     const uint32_t kWarps = blockDim.x >> 5;
     const int64_t groups = (n_out + kGemvGroupRows - 1) / kGemvGroupRows;
     const int64_t U = groups * nq, G = gridDim.x;
-    const int64_t u_begin = blockIdx.x * U / G, u_end = (blockIdx.x + 1) * U / G;
     const uint32_t nq32 = (uint32_t)nq;
 
     for_each_sorted_segment(U, G, nq, blockIdx.x, [&](int64_t tu0, int64_t tu1, int64_t rg0, int64_t rg1, bool first, bool last) {
@@ -602,10 +603,11 @@ gemv_sorted_kernel(FastArgs fa, const unsigned long long* __restrict__ sorted, c
             for (int c = 0; c < kSortAccCopies; ++c) v += acc[c * (kGemvGroupsPerPass * kGemvGroupRows) + r];
             return v;
         };
-        finish_pass<kOutBf16>(yo, rg0, rg1, nq, u_begin, u_end, U, G, n_out, scratch, counters, row_sum);
+        const int64_t ub = blockIdx.x * U / G, ue = (blockIdx.x + 1) * U / G;     // recomputed here: nothing 64-bit lives across the main loop
+        finish_pass<kOutBf16, kShard>(yo, rg0, rg1, nq, ub, ue, U, G, n_out, scratch, counters, row_sum);
         __syncthreads();                                   // the sums are read above: the next pass may clear them only now
     });
-    shard_arrive(yo);
+    if (kShard) shard_arrive(yo);
 }
 
 // ===========================================================================
@@ -618,7 +620,7 @@ gemv_sorted_kernel(FastArgs fa, const unsigned long long* __restrict__ sorted, c
 constexpr int kBinSegUnits = 256;                    // at most 8192 blocks per segment (halved while shared memory is short)
 constexpr int kBinPerThread = kBinSegUnits * 32 / kSortThreads;   // 8
 
-template <bool kOutBf16, bool kSg = false>
+template <bool kOutBf16, bool kSg = false, bool kShard = false>
 __global__ void __launch_bounds__(kSortThreads, 1)
 gemv_bin_kernel(FastArgs fa, const uint32_t* __restrict__ stream, const uint16_t* __restrict__ sort_rank, const uint16_t* __restrict__ gain, SgArgs sg,
                 int64_t n_out, int64_t k_in, int64_t bpr, uint32_t nq_magic, int seg_units, const uint16_t* __restrict__ x, YOut yo,
@@ -764,10 +766,11 @@ gemv_bin_kernel(FastArgs fa, const uint32_t* __restrict__ stream, const uint16_t
             for (int c = 0; c < kSortAccCopies; ++c) v += acc[c * (kGemvGroupsPerPass * kGemvGroupRows) + r];
             return v;
         };
-        finish_pass<kOutBf16>(yo, rg0, rg1, nq, u_begin, u_end, U, G, n_out, scratch, counters, row_sum);
+        const int64_t ub = blockIdx.x * U / G, ue = (blockIdx.x + 1) * U / G;     // recomputed here: nothing 64-bit lives across the main loop
+        finish_pass<kOutBf16, kShard>(yo, rg0, rg1, nq, ub, ue, U, G, n_out, scratch, counters, row_sum);
         __syncthreads();
     }, seg_units);
-    shard_arrive(yo);
+    if (kShard) shard_arrive(yo);
 }
 
 // ===========================================================================
@@ -794,19 +797,34 @@ struct GemmArgs {
     int batch, npad;
     int nstages, split;
     const uint16_t* x;
-    YOut yo;                   // Y [batch][y_ld] bf16: this rank's copy (and, row-sharded, the peers'), at the first row of the band
+    uint16_t* y;               // Y [batch][y_ld] bf16, at the first row of this launch's rows
     int64_t y_ld;
+    const YOut* shard;         // row-sharded launch: the peers' copies and flags (device memory), else null
     float* scratch;            // [npad][scratch_ld] binary32, all zero on entry and on exit
     int64_t scratch_ld;        // row tiles * 128
     uint32_t* counters;        // [row tiles], zero on entry and on exit
 };
+
+// One element of Y; a row-sharded launch also writes it into the peers' copies (their description sits in device
+// memory so that the ordinary launch's parameters stay as small as they were).
+template <bool kShard>
+__device__ __forceinline__ void gemm_store(const GemmArgs& ga, int n, int64_t orow, float v)
+{
+    const __nv_bfloat16 h = __float2bfloat16_rn(v);
+    const int64_t at = (int64_t)n * ga.y_ld + orow;
+    reinterpret_cast<__nv_bfloat16*>(ga.y)[at] = h;
+    if (kShard) {
+        const int np = ga.shard->n_peer;
+        for (int p = 0; p < np; ++p) reinterpret_cast<__nv_bfloat16*>(ga.shard->peer[p])[at] = h;
+    }
+}
 
 __device__ __forceinline__ void group_barrier(int group)
 {
     asm volatile("bar.sync %0, %1;" ::"r"(1 + group), "n"(kGemmGroupThreads) : "memory");
 }
 
-template <bool kBig, bool kSg = false>
+template <bool kBig, bool kSg = false, bool kShard = false>
 __global__ void __launch_bounds__(kGemmThreads, 1)
 gemm_kernel(FastArgs fa, const uint32_t* __restrict__ stream, const uint16_t* __restrict__ gain, SgArgs sg, GemmArgs ga)
 {
@@ -908,7 +926,7 @@ gemm_kernel(FastArgs fa, const uint32_t* __restrict__ stream, const uint16_t* __
                     for (int i = 0; i < 16; ++i) {
                         const int n = c0 + i;
                         if (n < ga.batch) {
-                            if (ga.split == 1) store_y<true>(ga.yo, (int64_t)n * ga.y_ld + orow, v[i]);
+                            if (ga.split == 1) gemm_store<kShard>(ga, n, orow, v[i]);
                             else atomicAdd(ga.scratch + (int64_t)n * ga.scratch_ld + orow, v[i]);
                         }
                     }
@@ -929,7 +947,7 @@ gemm_kernel(FastArgs fa, const uint32_t* __restrict__ stream, const uint16_t* __
                     const int64_t orow = rt * kGemmRows + (i % kGemmRows);
                     if (orow < ga.n_out) {
                         float* sp = ga.scratch + (int64_t)n * ga.scratch_ld + orow;
-                        store_y<true>(ga.yo, (int64_t)n * ga.y_ld + orow, __ldcg(sp));
+                        gemm_store<kShard>(ga, n, orow, __ldcg(sp));
                         __stcg(sp, 0.f);
                     }
                 }
@@ -939,8 +957,10 @@ gemm_kernel(FastArgs fa, const uint32_t* __restrict__ stream, const uint16_t* __
         __syncthreads();
     }
     if (timeout) atomicOr(fa.flags, 1u);
-    if (ga.yo.n_peer) __threadfence_system();             // this thread's stores to the peers' copies, before the CTA counts itself in
-    shard_arrive(ga.yo);
+    if (kShard) {
+        __threadfence_system();                           // this thread's stores to the peers' copies, before the CTA counts itself in
+        shard_arrive(*ga.shard);
+    }
     __syncthreads();
     if (warp == 0) tmem_dealloc(tmem, kTmemCols);
 }
@@ -960,8 +980,8 @@ constexpr int kDomEntries = kGemmRows * kDomBlocks;    // 1024
 constexpr int kDomStages = 2;                          // 96-column MMA stages per domain
 
 __global__ void __launch_bounds__(kDomEntries, 1)
-sort_blocks_gemm_kernel(FastArgs fa, const uint32_t* __restrict__ stream, const uint16_t* __restrict__ sort_rank, int64_t n_out, int64_t bpr,
-                        int64_t ndomains, unsigned long long* __restrict__ out)
+sort_blocks_gemm_kernel(FastArgs fa, const uint32_t* __restrict__ stream, const uint16_t* __restrict__ sort_rank, int gain_bits, int64_t n_out,
+                        int64_t bpr, int64_t ndomains, unsigned long long* __restrict__ out)
 {
     FAST_PROLOGUE();
     __shared__ uint32_t hist[1024], cursor[1024];
@@ -975,10 +995,11 @@ sort_blocks_gemm_kernel(FastArgs fa, const uint32_t* __restrict__ stream, const 
         unsigned long long field = kSortIndexMask;
         uint32_t key = 1023u;
         if (row < n_out && cb < bpr) {
-            const uint64_t I = load_field(stream, (uint64_t)(row * bpr + cb), (int)fa.L.W);
+            const uint64_t f = load_field(stream, (uint64_t)(row * bpr + cb), (int)fa.L.W + gain_bits);   // shape index | gain index << W
+            const uint64_t I = f & ((1ull << fa.L.W) - 1ull);
             if (I < fa.n_points) {
                 uint64_t local;
-                field = I;
+                field = f;
                 key = __ldg(sort_rank + fast_find_class(T, I, local));
             } else {
                 atomicAdd(fa.bad_index, 1ull);
@@ -1049,9 +1070,9 @@ sort_blocks_gemm_big_kernel(FastArgs fa, const uint32_t* __restrict__ stream, in
     }
 }
 
-template <bool kBig>
+template <bool kBig, bool kSg = false, bool kShard = false>
 __global__ void __launch_bounds__(kGemmThreads, 1)
-gemm_sorted_kernel(FastArgs fa, const unsigned long long* __restrict__ sorted, const uint16_t* __restrict__ gain, GemmArgs ga, int dpi)
+gemm_sorted_kernel(FastArgs fa, const unsigned long long* __restrict__ sorted, const uint16_t* __restrict__ gain, SgArgs sg, GemmArgs ga, int dpi)
 {
     extern __shared__ __align__(128) uint8_t smem[];
     const uint32_t img_bytes = fa.L.total;
@@ -1111,12 +1132,13 @@ gemm_sorted_kernel(FastArgs fa, const unsigned long long* __restrict__ sorted, c
             for (int q = 0; q < 2; ++q) {
                 if (q >= nd_now) break;
                 const ulonglong2 e = q == 0 ? cur0 : cur1;
-                const uint64_t I = e.x & kSortIndexMask;
+                const uint64_t field = e.x & kSortIndexMask;
+                const uint64_t I = kSg ? field & ((1ull << fa.L.W) - 1ull) : field;     // shape-gain form: gain index above the shape index
                 const uint32_t pos = kBig ? (uint32_t)(e.y >> 32) & 1023u : (uint32_t)(e.x >> 48);
-                const bool valid = kBig ? !(e.y >> 63) : I < fa.n_points;
+                const bool valid = kBig ? !(e.y >> 63) : (field != kSortIndexMask && I < fa.n_points);
                 const uint32_t r = pos >> 3, c = pos & 7u;
                 const int64_t row = rt * kGemmRows + r, cb = (int64_t)(d0 + q) * kDomBlocks + c;
-                const float gn = valid ? gain_to_float(__ldg(gain + row * ga.bpr + cb)) : 0.f;
+                float gn = (!kSg && valid) ? gain_to_float(__ldg(gain + row * ga.bpr + cb)) : 0.f;
                 uint32_t w[12];
                 if (kBig) {
                     const int cls = valid ? (int)((uint32_t)(e.y >> 8) & 0xffffffu) : 0;
@@ -1130,7 +1152,12 @@ gemm_sorted_kernel(FastArgs fa, const unsigned long long* __restrict__ sorted, c
                     }
                 } else {
                     Decoded dec;
-                    decode_sorted_entry(fa, T, I, valid, dec);
+                    const uint32_t cls = decode_sorted_entry(fa, T, I, valid, dec);
+                    if (kSg && valid) {
+                        const float scale = sg.row_scale ? __ldg(sg.row_scale + row) : 1.f;
+                        gn = __fmul_rn(__fmul_rn(scale, __ldg(sg.codebook + (uint32_t)(field >> fa.L.W))),
+                                       __uint_as_float(T.desc[cls * kFastDescStride + kFastDescRnorm]));
+                    }
                     expand_bf16(dec, gn, w);
                 }
                 // the previous MMAs read the buffers: wait for them only now, with the first chunk already unranked
@@ -1178,7 +1205,7 @@ gemm_sorted_kernel(FastArgs fa, const unsigned long long* __restrict__ sorted, c
                     for (int i = 0; i < 16; ++i) {
                         const int n = c0 + i;
                         if (n < ga.batch) {
-                            if (parts == 1u) store_y<true>(ga.yo, (int64_t)n * ga.y_ld + orow, v[i]);
+                            if (parts == 1u) gemm_store<kShard>(ga, n, orow, v[i]);
                             else atomicAdd(ga.scratch + (int64_t)n * ga.scratch_ld + orow, v[i]);
                         }
                     }
@@ -1199,7 +1226,7 @@ gemm_sorted_kernel(FastArgs fa, const unsigned long long* __restrict__ sorted, c
                     const int64_t orow = rt * kGemmRows + (i % kGemmRows);
                     if (orow < ga.n_out) {
                         float* sp = ga.scratch + (int64_t)n * ga.scratch_ld + orow;
-                        store_y<true>(ga.yo, (int64_t)n * ga.y_ld + orow, __ldcg(sp));
+                        gemm_store<kShard>(ga, n, orow, __ldcg(sp));
                         __stcg(sp, 0.f);
                     }
                 }
@@ -1209,8 +1236,10 @@ gemm_sorted_kernel(FastArgs fa, const unsigned long long* __restrict__ sorted, c
         __syncthreads();
     }
     if (timeout) atomicOr(fa.flags, 1u);
-    if (ga.yo.n_peer) __threadfence_system();             // this thread's stores to the peers' copies, before the CTA counts itself in
-    shard_arrive(ga.yo);
+    if (kShard) {
+        __threadfence_system();                           // this thread's stores to the peers' copies, before the CTA counts itself in
+        shard_arrive(*ga.shard);
+    }
     __syncthreads();
     if (warp == 0) tmem_dealloc(tmem, kTmemCols);
 }
@@ -1265,13 +1294,16 @@ int check_gemm_args(const llvq_ctx* ctx, const void* d_idx, const uint16_t* d_ga
 // Enqueue gemm_sorted_kernel on a stream sorted by llvq_sort_blocks_gemm.
 int launch_gemm_domains(const llvq_ctx* ctx, const void* p, const uint16_t* d_gain_f16, int64_t n_out, int64_t k_in,
                         const uint16_t* d_x_bf16, int batch, uint16_t* d_y_bf16, float* scratch, uint32_t* counters, void* stream,
-                        const YOut* yo = nullptr, int64_t y_ld = 0)
+                        const YOut* yo = nullptr, int64_t y_ld = 0, const SgArgs* sg = nullptr)
 {
     DeviceGuard guard(ctx->device);
     if (!guard.ok) return LLVQ_ECUDA;
     GemmArgs ga;
-    ga.yo = YOut{}; ga.yo.y = d_y_bf16; ga.y_ld = n_out;
-    if (yo) { ga.yo = *yo; ga.y_ld = y_ld; }
+    ga.y = d_y_bf16; ga.y_ld = n_out; ga.shard = nullptr;
+    if (yo) {                                             // the description travels ahead of the kernel on the same stream
+        ga.y = static_cast<uint16_t*>(yo->y); ga.y_ld = y_ld; ga.shard = static_cast<const YOut*>(ctx->d_shard);
+        if (cudaMemcpyAsync(ctx->d_shard, yo, sizeof(YOut), cudaMemcpyHostToDevice, (cudaStream_t)stream) != cudaSuccess) return LLVQ_ECUDA;
+    }
     ga.n_out = n_out; ga.k_in = k_in; ga.bpr = (k_in + 23) / 24;
     ga.batch = batch; ga.npad = (batch + 15) / 16 * 16;
     ga.nstages = (int)((ga.bpr + kDomBlocks - 1) / kDomBlocks);              // domains per row tile
@@ -1283,14 +1315,29 @@ int launch_gemm_domains(const llvq_ctx* ctx, const void* p, const uint16_t* d_ga
     const unsigned grid = (unsigned)std::min<int64_t>(row_tiles * ga.nstages, ctx->sm_count);
     const size_t smem = ((ctx->fl.total + 64 + 1023) & ~size_t(1023)) + (size_t)dpi * kDomStages * (kGemmRows * kStageK * 2 + (size_t)ga.npad * kStageK * 2);
     if (smem > 227 * 1024) return LLVQ_EUNSUPPORTED;
-    if (ctx->fast) {
-        if (!set_smem(gemm_sorted_kernel<false>, smem)) return LLVQ_ECUDA;
-        if (launch_pdl(gemm_sorted_kernel<false>, grid, (unsigned)kGemmThreads, smem, (cudaStream_t)stream, fast_args(ctx),
-                       static_cast<const unsigned long long*>(p), d_gain_f16, ga, dpi) != cudaSuccess) return LLVQ_ECUDA;
+    if (yo) {                                            // row-sharded: stored-gain form only
+        if (sg) return LLVQ_EUNSUPPORTED;
+        if (ctx->fast) {
+            if (!set_smem(gemm_sorted_kernel<false, false, true>, smem)) return LLVQ_ECUDA;
+            if (launch_pdl(gemm_sorted_kernel<false, false, true>, grid, (unsigned)kGemmThreads, smem, (cudaStream_t)stream, fast_args(ctx),
+                           static_cast<const unsigned long long*>(p), d_gain_f16, SgArgs{}, ga, dpi) != cudaSuccess) return LLVQ_ECUDA;
+        } else {
+            if (!set_smem(gemm_sorted_kernel<true, false, true>, smem)) return LLVQ_ECUDA;
+            if (launch_pdl(gemm_sorted_kernel<true, false, true>, grid, (unsigned)kGemmThreads, smem, (cudaStream_t)stream, fast_args(ctx),
+                           static_cast<const unsigned long long*>(p), d_gain_f16, SgArgs{}, ga, dpi) != cudaSuccess) return LLVQ_ECUDA;
+        }
+    } else if (sg) {
+        if (!set_smem(gemm_sorted_kernel<false, true>, smem)) return LLVQ_ECUDA;
+        if (launch_pdl(gemm_sorted_kernel<false, true>, grid, (unsigned)kGemmThreads, smem, (cudaStream_t)stream, fast_args(ctx),
+                       static_cast<const unsigned long long*>(p), d_gain_f16, *sg, ga, dpi) != cudaSuccess) return LLVQ_ECUDA;
+    } else if (ctx->fast) {
+        if (!set_smem(gemm_sorted_kernel<false, false>, smem)) return LLVQ_ECUDA;
+        if (launch_pdl(gemm_sorted_kernel<false, false>, grid, (unsigned)kGemmThreads, smem, (cudaStream_t)stream, fast_args(ctx),
+                       static_cast<const unsigned long long*>(p), d_gain_f16, SgArgs{}, ga, dpi) != cudaSuccess) return LLVQ_ECUDA;
     } else {
-        if (!set_smem(gemm_sorted_kernel<true>, smem)) return LLVQ_ECUDA;
-        if (launch_pdl(gemm_sorted_kernel<true>, grid, (unsigned)kGemmThreads, smem, (cudaStream_t)stream, fast_args(ctx),
-                       static_cast<const unsigned long long*>(p), d_gain_f16, ga, dpi) != cudaSuccess) return LLVQ_ECUDA;
+        if (!set_smem(gemm_sorted_kernel<true, false>, smem)) return LLVQ_ECUDA;
+        if (launch_pdl(gemm_sorted_kernel<true, false>, grid, (unsigned)kGemmThreads, smem, (cudaStream_t)stream, fast_args(ctx),
+                       static_cast<const unsigned long long*>(p), d_gain_f16, SgArgs{}, ga, dpi) != cudaSuccess) return LLVQ_ECUDA;
     }
     return launch_status();
 }
@@ -1307,8 +1354,11 @@ int launch_gemm(const llvq_ctx* ctx, const void* d_idx, const uint16_t* d_gain_f
     cudaStream_t st = (cudaStream_t)stream;
     if (k_in == 0) return cudaMemsetAsync(d_y_bf16, 0, (size_t)n_out * batch * 2, st) == cudaSuccess ? LLVQ_OK : LLVQ_ECUDA;
     GemmArgs ga;
-    ga.yo = YOut{}; ga.yo.y = d_y_bf16; ga.y_ld = n_out;
-    if (yo) { ga.yo = *yo; ga.y_ld = y_ld; }
+    ga.y = d_y_bf16; ga.y_ld = n_out; ga.shard = nullptr;
+    if (yo) {                                             // the description travels ahead of the kernel on the same stream
+        ga.y = static_cast<uint16_t*>(yo->y); ga.y_ld = y_ld; ga.shard = static_cast<const YOut*>(ctx->d_shard);
+        if (cudaMemcpyAsync(ctx->d_shard, yo, sizeof(YOut), cudaMemcpyHostToDevice, (cudaStream_t)stream) != cudaSuccess) return LLVQ_ECUDA;
+    }
     ga.n_out = n_out; ga.k_in = k_in; ga.bpr = (k_in + 23) / 24;
     ga.batch = batch; ga.npad = (batch + 15) / 16 * 16;
     ga.nstages = (int)((ga.bpr + kStageBlocks - 1) / kStageBlocks);
@@ -1329,7 +1379,16 @@ int launch_gemm(const llvq_ctx* ctx, const void* d_idx, const uint16_t* d_gain_f
     const size_t smem = ((img + 64 + 1023) & ~size_t(1023)) + 2 * kGemmRows * kStageK * 2 + 2 * (size_t)ga.npad * kStageK * 2;
     if (smem > 227 * 1024) return LLVQ_EUNSUPPORTED;
     const uint32_t* idx = static_cast<const uint32_t*>(d_idx);
-    if (sg) {
+    if (yo) {                                            // row-sharded: stored-gain form only
+        if (sg) return LLVQ_EUNSUPPORTED;
+        if (ctx->fast) {
+            if (!set_smem(gemm_kernel<false, false, true>, smem)) return LLVQ_ECUDA;
+            if (launch_pdl(gemm_kernel<false, false, true>, grid, (unsigned)kGemmThreads, smem, st, fast_args(ctx), idx, d_gain_f16, SgArgs{}, ga) != cudaSuccess) return LLVQ_ECUDA;
+        } else {
+            if (!set_smem(gemm_kernel<true, false, true>, smem)) return LLVQ_ECUDA;
+            if (launch_pdl(gemm_kernel<true, false, true>, grid, (unsigned)kGemmThreads, smem, st, fast_args(ctx), idx, d_gain_f16, SgArgs{}, ga) != cudaSuccess) return LLVQ_ECUDA;
+        }
+    } else if (sg) {
         if (!set_smem(gemm_kernel<false, true>, smem)) return LLVQ_ECUDA;
         if (launch_pdl(gemm_kernel<false, true>, grid, (unsigned)kGemmThreads, smem, st, fast_args(ctx), idx, d_gain_f16, *sg, ga) != cudaSuccess) return LLVQ_ECUDA;
     } else if (ctx->fast) {
@@ -1421,7 +1480,7 @@ int llvq_create(llvq_ctx** out, int m_lo, int m_hi, int device)
         for (uint32_t r = 0; r < ncls; ++r) sort_rank[order[r]] = (uint16_t)r;
     }
     size_t o_cnt = up(o_srk + sort_rank.size() * 2);
-    size_t o_scr = up(o_cnt + (size_t)(kCounterWords + 16) * 4);   // one counter per group of 8 rows (GEMV) / per 128-row tile (GEMM), then the grid arrival counter
+    size_t o_scr = up(o_cnt + (size_t)(kCounterWords + 16) * 4 + 256);   // ... and the peers' description of a row-sharded GEMM   // one counter per group of 8 rows (GEMV) / per 128-row tile (GEMM), then the grid arrival counter
     size_t total = o_scr + (size_t)64 * kMaxScratchRows * 4;
     std::vector<uint8_t> blob(o_cnt, 0);
     std::memcpy(blob.data() + o_offhi, off_hi.data(), (ncls + 1) * 4);
@@ -1463,6 +1522,8 @@ int llvq_create(llvq_ctx** out, int m_lo, int m_hi, int device)
     ctx->enc.hash_mask = hkeys.empty() ? 0u : (uint32_t)(hkeys.size() - 1);
     ctx->d_counters = reinterpret_cast<uint32_t*>(d + o_cnt);
     ctx->d_scratch = reinterpret_cast<float*>(d + o_scr);
+    ctx->d_shard = d + o_cnt + (size_t)(kCounterWords + 16) * 4;
+    static_assert(sizeof(YOut) <= 256, "the space reserved behind the counters");
     *out = ctx;
     return LLVQ_OK;
 }
@@ -1633,6 +1694,8 @@ static int gemv_common(const llvq_ctx* ctx, const void* d_idx, const uint16_t* d
     const uint32_t* idx = static_cast<const uint32_t*>(d_idx);
     const FastArgs fa = fast_args(ctx);
     const SgArgs sga = sg ? *sg : SgArgs{};
+    const bool shard = yo.n_peer > 0 || yo.n_flag > 0;                  // row-sharded launch: stored-gain form only
+    if (shard && sg) return LLVQ_EUNSUPPORTED;
     // fast-path codes with many classes (mixed warps are what costs there): the kernel that bins the blocks of a segment by
     // class before unranking them; codes with a handful of classes keep the direct kernel
     int seg_units = kBinSegUnits;
@@ -1644,26 +1707,29 @@ static int gemv_common(const llvq_ctx* ctx, const void* d_idx, const uint16_t* d
     if ((!sg || sg->bits <= 5) && ctx->fast && ctx->d_sort_rank && ctx->host.desc.size() >= 64 && ctx->host.W <= 48 && smem_bin <= 227 * 1024 &&
         nq < (1ll << 24)) {
         const uint32_t magic = nq == 1 ? 0xffffffffu : (uint32_t)((1ull << 32) / (uint64_t)nq);
-#define LLVQ_LAUNCH_BIN(BF16, SG)                                                                                          \
+#define LLVQ_LAUNCH_BIN(BF16, SG, SH)                                                                                      \
     do {                                                                                                                   \
-        if (!set_smem(gemv_bin_kernel<BF16, SG>, smem_bin)) return LLVQ_ECUDA;                                              \
-        if (launch_pdl(gemv_bin_kernel<BF16, SG>, g, (unsigned)kSortThreads, smem_bin, st, fa, idx, ctx->d_sort_rank, d_gain_f16, sga, n_out, k_in, \
+        if (!set_smem(gemv_bin_kernel<BF16, SG, SH>, smem_bin)) return LLVQ_ECUDA;                                          \
+        if (launch_pdl(gemv_bin_kernel<BF16, SG, SH>, g, (unsigned)kSortThreads, smem_bin, st, fa, idx, ctx->d_sort_rank, d_gain_f16, sga, n_out, k_in, \
                        bpr, magic, seg_units, d_x_bf16, yo, ctx->d_scratch, ctx->d_counters) != cudaSuccess) return LLVQ_ECUDA; \
     } while (0)
-        if (sg) { if (y_dtype == LLVQ_BF16) LLVQ_LAUNCH_BIN(true, true); else LLVQ_LAUNCH_BIN(false, true); }
-        else    { if (y_dtype == LLVQ_BF16) LLVQ_LAUNCH_BIN(true, false); else LLVQ_LAUNCH_BIN(false, false); }
+        if (shard)   { if (y_dtype == LLVQ_BF16) LLVQ_LAUNCH_BIN(true, false, true); else LLVQ_LAUNCH_BIN(false, false, true); }
+        else if (sg) { if (y_dtype == LLVQ_BF16) LLVQ_LAUNCH_BIN(true, true, false); else LLVQ_LAUNCH_BIN(false, true, false); }
+        else         { if (y_dtype == LLVQ_BF16) LLVQ_LAUNCH_BIN(true, false, false); else LLVQ_LAUNCH_BIN(false, false, false); }
 #undef LLVQ_LAUNCH_BIN
         return launch_status();
     }
-#define LLVQ_LAUNCH_GEMV(BIG, BF16, SG)                                                                            \
+#define LLVQ_LAUNCH_GEMV(BIG, BF16, SG, SH)                                                                        \
     do {                                                                                                           \
-        if (!set_smem(gemv_fast_kernel<BIG, BF16, SG>, smem)) return LLVQ_ECUDA;                                   \
-        if (launch_pdl(gemv_fast_kernel<BIG, BF16, SG>, g, threads, smem, st, fa, idx, d_gain_f16, sga, n_out, k_in, bpr, d_x_bf16, yo, \
+        if (!set_smem(gemv_fast_kernel<BIG, BF16, SG, SH>, smem)) return LLVQ_ECUDA;                               \
+        if (launch_pdl(gemv_fast_kernel<BIG, BF16, SG, SH>, g, threads, smem, st, fa, idx, d_gain_f16, sga, n_out, k_in, bpr, d_x_bf16, yo, \
                        ctx->d_scratch, ctx->d_counters) != cudaSuccess) return LLVQ_ECUDA;                         \
     } while (0)
-    if (sg)             { if (y_dtype == LLVQ_BF16) LLVQ_LAUNCH_GEMV(false, true, true);  else LLVQ_LAUNCH_GEMV(false, false, true); }
-    else if (ctx->fast) { if (y_dtype == LLVQ_BF16) LLVQ_LAUNCH_GEMV(false, true, false); else LLVQ_LAUNCH_GEMV(false, false, false); }
-    else                { if (y_dtype == LLVQ_BF16) LLVQ_LAUNCH_GEMV(true, true, false);  else LLVQ_LAUNCH_GEMV(true, false, false); }
+    if (shard && ctx->fast) { if (y_dtype == LLVQ_BF16) LLVQ_LAUNCH_GEMV(false, true, false, true); else LLVQ_LAUNCH_GEMV(false, false, false, true); }
+    else if (shard)         { if (y_dtype == LLVQ_BF16) LLVQ_LAUNCH_GEMV(true, true, false, true);  else LLVQ_LAUNCH_GEMV(true, false, false, true); }
+    else if (sg)            { if (y_dtype == LLVQ_BF16) LLVQ_LAUNCH_GEMV(false, true, true, false);  else LLVQ_LAUNCH_GEMV(false, false, true, false); }
+    else if (ctx->fast)     { if (y_dtype == LLVQ_BF16) LLVQ_LAUNCH_GEMV(false, true, false, false); else LLVQ_LAUNCH_GEMV(false, false, false, false); }
+    else                    { if (y_dtype == LLVQ_BF16) LLVQ_LAUNCH_GEMV(true, true, false, false);  else LLVQ_LAUNCH_GEMV(true, false, false, false); }
 #undef LLVQ_LAUNCH_GEMV
     return launch_status();
 }
@@ -1789,14 +1855,17 @@ static int gemv_sorted_common(const llvq_ctx* ctx, const void* d_sorted, const u
     const uint32_t magic = nq == 1 ? 0xffffffffu : (uint32_t)((1ull << 32) / (uint64_t)nq);
     const unsigned long long* sp = static_cast<const unsigned long long*>(d_sorted);
     const SgArgs sga = sg ? *sg : SgArgs{};
-#define LLVQ_LAUNCH_SORTED(BF16, SG)                                                                                    \
+#define LLVQ_LAUNCH_SORTED(BF16, SG, SH)                                                                                \
     do {                                                                                                                \
-        if (!set_smem(gemv_sorted_kernel<BF16, SG>, smem)) return LLVQ_ECUDA;                                            \
-        if (launch_pdl(gemv_sorted_kernel<BF16, SG>, g, (unsigned)kSortThreads, smem, st, fast_args(ctx), sp, d_gain_f16, sga, n_out, k_in, bpr, \
+        if (!set_smem(gemv_sorted_kernel<BF16, SG, SH>, smem)) return LLVQ_ECUDA;                                        \
+        if (launch_pdl(gemv_sorted_kernel<BF16, SG, SH>, g, (unsigned)kSortThreads, smem, st, fast_args(ctx), sp, d_gain_f16, sga, n_out, k_in, bpr, \
                        magic, d_x_bf16, yo, ctx->d_scratch, ctx->d_counters) != cudaSuccess) return LLVQ_ECUDA;          \
     } while (0)
-    if (sg) { if (y_dtype == LLVQ_BF16) LLVQ_LAUNCH_SORTED(true, true); else LLVQ_LAUNCH_SORTED(false, true); }
-    else    { if (y_dtype == LLVQ_BF16) LLVQ_LAUNCH_SORTED(true, false); else LLVQ_LAUNCH_SORTED(false, false); }
+    const bool shard = yo.n_peer > 0 || yo.n_flag > 0;                  // row-sharded launch: stored-gain form only
+    if (shard && sg) return LLVQ_EUNSUPPORTED;
+    if (shard)   { if (y_dtype == LLVQ_BF16) LLVQ_LAUNCH_SORTED(true, false, true); else LLVQ_LAUNCH_SORTED(false, false, true); }
+    else if (sg) { if (y_dtype == LLVQ_BF16) LLVQ_LAUNCH_SORTED(true, true, false); else LLVQ_LAUNCH_SORTED(false, true, false); }
+    else         { if (y_dtype == LLVQ_BF16) LLVQ_LAUNCH_SORTED(true, false, false); else LLVQ_LAUNCH_SORTED(false, false, false); }
 #undef LLVQ_LAUNCH_SORTED
     return launch_status();
 }
@@ -1900,12 +1969,12 @@ size_t llvq_sorted_gemm_bytes(const llvq_ctx* ctx, int64_t n_out, int64_t k_in)
     return (size_t)(((n_out + kGemmRows - 1) / kGemmRows) * ((bpr + kDomBlocks - 1) / kDomBlocks)) * kDomEntries * (ctx->fast ? 8 : 16);
 }
 
-int llvq_sort_blocks_gemm(const llvq_ctx* ctx, const void* d_idx, int64_t n_out, int64_t k_in, void* d_sorted, void* stream)
+static int sort_blocks_gemm_common(const llvq_ctx* ctx, const void* d_idx, int gain_bits, int64_t n_out, int64_t k_in, void* d_sorted, void* stream)
 {
     if (int e = check_common(ctx, d_idx)) return e;
-    if (!d_sorted || n_out <= 0 || k_in <= 0) return LLVQ_EINVAL;
+    if (!d_sorted || n_out <= 0 || k_in <= 0 || gain_bits < 0 || gain_bits > 8) return LLVQ_EINVAL;
     if (!aligned(d_sorted, 16)) return LLVQ_EALIGN;
-    if (!gemm_sortable(ctx)) return LLVQ_EUNSUPPORTED;
+    if (!gemm_sortable(ctx) || (gain_bits > 0 && !ctx->fast) || (ctx->fast && ctx->host.W + gain_bits > 48)) return LLVQ_EUNSUPPORTED;
     DeviceGuard guard(ctx->device);
     if (!guard.ok) return LLVQ_ECUDA;
     const int64_t bpr = (k_in + 23) / 24;
@@ -1919,8 +1988,32 @@ int llvq_sort_blocks_gemm(const llvq_ctx* ctx, const void* d_idx, int64_t n_out,
     const size_t smem = ctx->fl.total + 16;
     if (!set_smem(sort_blocks_gemm_kernel, smem)) return LLVQ_ECUDA;
     sort_blocks_gemm_kernel<<<g, kDomEntries, smem, (cudaStream_t)stream>>>(fast_args(ctx), static_cast<const uint32_t*>(d_idx), ctx->d_sort_rank,
-                                                                           n_out, bpr, ndomains, static_cast<unsigned long long*>(d_sorted));
+                                                                           gain_bits, n_out, bpr, ndomains, static_cast<unsigned long long*>(d_sorted));
     return launch_status();
+}
+
+int llvq_sort_blocks_gemm(const llvq_ctx* ctx, const void* d_idx, int64_t n_out, int64_t k_in, void* d_sorted, void* stream)
+{
+    return sort_blocks_gemm_common(ctx, d_idx, 0, n_out, k_in, d_sorted, stream);
+}
+
+int llvq_sort_blocks_gemm_sg(const llvq_ctx* ctx, const void* d_fields, int gain_bits, int64_t n_out, int64_t k_in, void* d_sorted, void* stream)
+{
+    return sort_blocks_gemm_common(ctx, d_fields, gain_bits, n_out, k_in, d_sorted, stream);
+}
+
+int llvq_gemm_small_batch_sorted_sg(const llvq_ctx* ctx, const void* d_sorted, int gain_bits, const float* d_codebook_f32,
+                                    const float* d_row_scale_f32, int64_t n_out, int64_t k_in, const uint16_t* d_x_bf16, int batch,
+                                    uint16_t* d_y_bf16, void* stream)
+{
+    if (ctx && ctx->device >= 0 && n_out == 0) return LLVQ_OK;
+    if (int e = check_sg(ctx, d_sorted, gain_bits, d_codebook_f32, d_row_scale_f32)) return e;
+    if (!d_x_bf16 || !d_y_bf16 || n_out < 0 || k_in < 0 || batch < 1 || batch > 64) return LLVQ_EINVAL;
+    if (!aligned(d_x_bf16, 16) || !aligned(d_y_bf16, 2) || (k_in & 7)) return LLVQ_EALIGN;
+    if (!gemm_sortable(ctx) || ctx->host.W + gain_bits > 48 || n_out > kMaxScratchRows || k_in <= 0) return LLVQ_EUNSUPPORTED;
+    const SgArgs sg{d_codebook_f32, d_row_scale_f32, gain_bits};
+    return launch_gemm_domains(ctx, d_sorted, nullptr, n_out, k_in, d_x_bf16, batch, d_y_bf16, ctx->d_scratch, ctx->d_counters, stream,
+                               nullptr, 0, &sg);
 }
 
 int llvq_gemm_small_batch_sorted(const llvq_ctx* ctx, const void* d_sorted, const uint16_t* d_gain_f16, int64_t n_out, int64_t k_in,

@@ -211,6 +211,11 @@ def test_gemm_small_batch_sg(lib, ctxs, codes, code, bits, n_out, k_in, batch):
     y = lib.llvq_gemm_small_batch_sg(ctx, to_dev_u8(stream), bits, _f32(cb), _f32(rs), n_out, k_in, to_dev_bf16(x))
     torch.cuda.synchronize()
     assert gemv_error(y.float().cpu().numpy(), ref) <= TOL_BF16_OUT
+    # the same product from the sorted layout
+    srt = lib.llvq_sort_blocks_gemm_sg(ctx, to_dev_u8(stream), bits, n_out, k_in)
+    ys = lib.llvq_gemm_small_batch_sorted_sg(ctx, srt, bits, _f32(cb), _f32(rs), n_out, k_in, to_dev_bf16(x))
+    torch.cuda.synchronize()
+    assert gemv_error(ys.float().cpu().numpy(), ref) <= TOL_BF16_OUT
     # batch 1 agrees with the fused matrix-vector product
     y1 = lib.llvq_gemm_small_batch_sg(ctx, to_dev_u8(stream), bits, _f32(cb), _f32(rs), n_out, k_in, to_dev_bf16(x[:1]))
     yv = lib.llvq_gemv_sg(ctx, to_dev_u8(stream), bits, _f32(cb), _f32(rs), n_out, k_in, to_dev_bf16(x[0]), y_dtype=torch.bfloat16)
