@@ -304,7 +304,8 @@ int llvq_pack_fields(const llvq_ctx* ctx, const uint64_t* d_index, const uint8_t
  * is not read), one in each peer's exchange buffer with this rank as its only writer.  The kernel itself then stores
  * `epoch` there, with release semantics at system scope, once every row of the band is in place in every copy (the
  * last CTA to finish does it; with n_rows = 0 or k_in = 0 a one-warp kernel does) - what llvq_signal_ranks would do
- * in a launch of its own.  The peers see it through llvq_wait_ranks.  One such call at a time per context.
+ * in a launch of its own.  The peers see it through llvq_wait_ranks.  One such call at a time per context.  The epoch
+ * is an argument of the launch: a captured CUDA graph would replay the same epoch, so these calls are made live.
  */
 int llvq_gemv_rowshard(const llvq_ctx* ctx, const void* d_idx, const uint16_t* d_gain_f16, int64_t n_rows, int64_t k_in,
                        const uint16_t* d_x_bf16, void* const* d_y_all, int n_dest, int own_slot, int64_t row0,

@@ -805,6 +805,11 @@ struct GemmArgs {
     uint32_t* counters;        // [row tiles], zero on entry and on exit
 };
 
+__global__ void put_shard_kernel(YOut yo, YOut* dst)
+{
+    if (threadIdx.x == 0) *dst = yo;
+}
+
 // One element of Y; a row-sharded launch also writes it into the peers' copies (their description sits in device
 // memory so that the ordinary launch's parameters stay as small as they were).
 template <bool kShard>
@@ -1302,7 +1307,7 @@ int launch_gemm_domains(const llvq_ctx* ctx, const void* p, const uint16_t* d_ga
     ga.y = d_y_bf16; ga.y_ld = n_out; ga.shard = nullptr;
     if (yo) {                                             // the description travels ahead of the kernel on the same stream
         ga.y = static_cast<uint16_t*>(yo->y); ga.y_ld = y_ld; ga.shard = static_cast<const YOut*>(ctx->d_shard);
-        if (cudaMemcpyAsync(ctx->d_shard, yo, sizeof(YOut), cudaMemcpyHostToDevice, (cudaStream_t)stream) != cudaSuccess) return LLVQ_ECUDA;
+        put_shard_kernel<<<1, 32, 0, (cudaStream_t)stream>>>(*yo, static_cast<YOut*>(ctx->d_shard));   // by value: safe under stream capture
     }
     ga.n_out = n_out; ga.k_in = k_in; ga.bpr = (k_in + 23) / 24;
     ga.batch = batch; ga.npad = (batch + 15) / 16 * 16;
@@ -1357,7 +1362,7 @@ int launch_gemm(const llvq_ctx* ctx, const void* d_idx, const uint16_t* d_gain_f
     ga.y = d_y_bf16; ga.y_ld = n_out; ga.shard = nullptr;
     if (yo) {                                             // the description travels ahead of the kernel on the same stream
         ga.y = static_cast<uint16_t*>(yo->y); ga.y_ld = y_ld; ga.shard = static_cast<const YOut*>(ctx->d_shard);
-        if (cudaMemcpyAsync(ctx->d_shard, yo, sizeof(YOut), cudaMemcpyHostToDevice, (cudaStream_t)stream) != cudaSuccess) return LLVQ_ECUDA;
+        put_shard_kernel<<<1, 32, 0, (cudaStream_t)stream>>>(*yo, static_cast<YOut*>(ctx->d_shard));   // by value: safe under stream capture
     }
     ga.n_out = n_out; ga.k_in = k_in; ga.bpr = (k_in + 23) / 24;
     ga.batch = batch; ga.npad = (batch + 15) / 16 * 16;
