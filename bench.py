@@ -409,9 +409,13 @@ def extras(P, ctx) -> dict:
     _event_us(torch, fn, 16)
     us3 = _event_us(torch, fn, 128)
     by3 = nb3 * (24 // 8 + 2) + 2 * k + 2 * n
+    srt3 = [P.llvq_sort_blocks(ctx3, b[0], n, k) for b in bufs3]
+    fn = lambda i: P.llvq_gemv_sorted(ctx3, srt3[i % 64], bufs3[i % 64][1], n, k, x3, d_y=y3)
+    _event_us(torch, fn, 16)
+    us3s = _event_us(torch, fn, 128)
     out["paper_shape_shell3_4096x4104_gemv"] = {"us": us3, "GBps": by3 / us3 / 1e3, "weights_per_s": n * k / (us3 * 1e-6),
-                                                "paper_us_fp16_unnamed_gpu": 11.94, "algorithmic_bytes": by3}
-    del bufs3
+                                                "sorted_layout_us": us3s, "paper_us_fp16_unnamed_gpu": 11.94, "algorithmic_bytes": by3}
+    del bufs3, srt3
     # --- shape-gain form at the same 48 bits per block: shells 2..12 (47-bit shape index) + 1 gain bit, row scales
     ctx12 = P.Context(2, 12, device=torch.cuda.current_device())
     from_codebook = np.array([4.3157, 5.4413], dtype=np.float32)       # Lloyd-Max levels of chi(24) at one bit
