@@ -225,6 +225,7 @@ __device__ __forceinline__ int64_t unit_owner(int64_t u, int64_t U, int64_t G) {
 // everywhere), a rank writes its band straight into every rank's copy of the full vector: `y` is this rank's copy
 // and `peer` the other ranks' copies mapped into this process, every pointer already advanced to the band's first
 // row.  The stores to a peer travel over NVLink as plain remote writes.  n_peer = 0 is the single-GPU case.
+constexpr int64_t kPairSlotOffset = 64ll * 65536;      // floats: the 64-bit slots of finish_pass lie behind the binary32 scratch rows
 constexpr int kMaxShardPeers = 7;
 struct YOut {
     void* y;
@@ -291,7 +292,8 @@ __device__ __forceinline__ void stage_x(uint32_t* xs, const uint16_t* __restrict
 // units per row group, G CTAs): row_sum(i) is the CTA's sum for row i of the pass.  One warp per row group, lanes
 // 0..7 its rows, no CTA-wide barrier inside.  A group the CTA covers completely is final.  A group it shares with
 // neighbouring CTAs goes through the scratch row in global memory: add, make the add visible, count the arrival;
-// whoever arrives last reads the total, writes y and leaves scratch and counter zero for the next launch.
+// whoever arrives last reads the total, writes y and leaves scratch and counter zero for the next launch (groups shared
+// by exactly two CTAs take a shorter way, below).
 // The caller puts a __syncthreads() before (sums complete) and after (sums may be cleared) the call.
 template <bool kOutBf16, bool kShard, typename RowSum>
 __device__ __forceinline__ void finish_pass(const YOut& yo, int64_t rg0, int64_t rg1, int64_t nq, int64_t u_begin, int64_t u_end,
@@ -311,13 +313,28 @@ __device__ __forceinline__ void finish_pass(const YOut& yo, int64_t rg0, int64_t
             }
             continue;
         }
+        const uint32_t parts = (uint32_t)(unit_owner((rg + 1) * nq - 1, U, G) - unit_owner(rg * nq, U, G) + 1);
+        if (parts == 2u) {
+            // two CTAs share the group (the usual case): one compare-and-swap on a 64-bit slot carries both the sum
+            // and the arrival.  Whoever finds the slot empty leaves (its sum, 1) there; the other gets that back from
+            // its failed swap, adds its own sum, stores y and empties the slot.  One round trip each, no fence.
+            if (mine) {
+                unsigned long long* slot = reinterpret_cast<unsigned long long*>(scratch + kPairSlotOffset) + row;
+                const unsigned long long seen = atomicCAS(slot, 0ull, (unsigned long long)__float_as_uint(part) | 1ull << 32);
+                if (seen != 0ull) {
+                    store_y<kOutBf16, kShard>(yo, row, __fadd_rn(__uint_as_float((uint32_t)seen), part));
+                    __stcg(slot, 0ull);
+                    if (kShard) __threadfence_system();
+                }
+            }
+            continue;
+        }
         if (mine) atomicAdd(scratch + row, part);
         __threadfence();                               // every lane's add is performed before ...
         __syncwarp();
         uint32_t is_last = 0u;
         if (lane == 0) {
             __threadfence();                           // ... lane 0 counts the arrival
-            const uint32_t parts = (uint32_t)(unit_owner((rg + 1) * nq - 1, U, G) - unit_owner(rg * nq, U, G) + 1);
             is_last = atomicAdd(counters + rg, 1u) == parts - 1u;
         }
         is_last = __shfl_sync(kFullMask, is_last, 0);
@@ -1486,7 +1503,8 @@ int llvq_create(llvq_ctx** out, int m_lo, int m_hi, int device)
     }
     size_t o_cnt = up(o_srk + sort_rank.size() * 2);
     size_t o_scr = up(o_cnt + (size_t)(kCounterWords + 16) * 4 + 256);   // ... and the peers' description of a row-sharded GEMM   // one counter per group of 8 rows (GEMV) / per 128-row tile (GEMM), then the grid arrival counter
-    size_t total = o_scr + (size_t)64 * kMaxScratchRows * 4;
+    static_assert(kPairSlotOffset == 64ll * kMaxScratchRows, "the pair slots start where the scratch rows end");
+    size_t total = o_scr + (size_t)64 * kMaxScratchRows * (4 + 8);       // binary32 scratch rows, then one 64-bit pair slot per GEMV row
     std::vector<uint8_t> blob(o_cnt, 0);
     std::memcpy(blob.data() + o_offhi, off_hi.data(), (ncls + 1) * 4);
     std::memcpy(blob.data() + o_offlo, off_lo.data(), (ncls + 1) * 8);
