@@ -73,6 +73,10 @@ enum { LLVQ_EUCLIDEAN = 0, LLVQ_ANGULAR = 1 };   /* scoring of the encoder's sea
  * Allocates the library's own host and device tables; *out is freed by
  * llvq_destroy.  Synchronous.  device < 0 builds a host-only context: the
  * query functions work, every function that would launch returns LLVQ_EINVAL.
+ * A context also owns the device scratch (partial sums of rows or row tiles that
+ * several thread blocks share, arrival counters) that the fused products keep
+ * zero between launches: launches that use the same context must be ordered, on
+ * one stream or by events; launches that may overlap need a context each.
  */
 int llvq_create(llvq_ctx** out, int m_lo, int m_hi, int device);
 void llvq_destroy(llvq_ctx* ctx);
