@@ -479,6 +479,27 @@ def test_gemv_sorted_many_row_groups_per_thread_block(lib, ctxs, oracle_mod):
     assert lib.llvq_last_error(ctx) == (0, 0)
 
 
+def test_gemv_at_the_largest_row_count(lib, ctxs, oracle_mod):
+    # 64 * 65536 rows is the most the scratch rows, arrival counters and pair slots of a context are sized for
+    o = _oracle(oracle_mod)((2, 2))
+    ctx = ctxs[(2, 2)]
+    n_out, k_in = 64 * 65536, 24
+    stream, gain, _ = gen.make_layer(o.N, o.W, n_out, k_in, 1, seed=9)
+    x = gen.normal_bf16(k_in, seed=9)
+    ds, dg, dx = to_dev_u8(stream), to_dev_f16(gain), to_dev_bf16(x)
+    y = lib.llvq_gemv(ctx, ds, dg, n_out, k_in, dx)
+    ys = lib.llvq_gemv_sorted(ctx, lib.llvq_sort_blocks(ctx, ds, n_out, k_in), dg, n_out, k_in, dx)
+    torch.cuda.synchronize()
+    assert torch.equal(y, ys)                                  # one block per row: no summation order to differ in
+    rows = [0, 7, 8, n_out // 2 + 3, n_out - 9, n_out - 1] + list(range(11, n_out, n_out // 17))
+    ref = np.array([o.gemv(stream, gain, n_out, k_in, x, rows=(r, 1))[r] for r in rows])
+    got = y.cpu().numpy()[rows]
+    assert (np.abs(got - ref) / np.maximum(np.abs(ref), 1e-3 * np.abs(ref).max())).max() <= TOL
+    assert lib.llvq_last_error(ctx) == (0, 0)
+    # one row group more is refused, not truncated (nothing is launched, so the short buffers do not matter)
+    assert ctx._lib.llvq_gemv(ctx._h, ds.data_ptr(), dg.data_ptr(), n_out + 8, k_in, dx.data_ptr(), y.data_ptr(), 0, None) == 3
+
+
 def test_sorted_layout_unsupported_for_the_72_bit_code(lib, ctxs):
     ctx = ctxs[(2, 53)]
     assert ctx._lib.llvq_sorted_bytes(ctx._h, 64, 96) == 0
