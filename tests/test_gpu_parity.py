@@ -479,6 +479,27 @@ def test_gemv_sorted_many_row_groups_per_thread_block(lib, ctxs, oracle_mod):
     assert lib.llvq_last_error(ctx) == (0, 0)
 
 
+@pytest.mark.parametrize("n_out,k_in", [(14336, 4096), (1024, 4096), (4096, 14336), (28672, 4096)])
+def test_gemv_decoder_sweep_shapes_sampled_rows(lib, ctxs, oracle_mod, n_out, k_in):
+    # the layer shapes of the 8B-decoder sweep the benchmark times (gate/up, k/v, down, and gate|up stored as one),
+    # stored stream and sorted layout; the oracle recomputes a sample of rows
+    o = _oracle(oracle_mod)((2, 13))
+    ctx = ctxs[(2, 13)]
+    stream, gain, _ = gen.make_layer(o.N, o.W, n_out, k_in, 1, seed=50)
+    x = gen.normal_bf16(k_in, seed=50)
+    ds, dg, dx = to_dev_u8(stream), to_dev_f16(gain), to_dev_bf16(x)
+    y = lib.llvq_gemv(ctx, ds, dg, n_out, k_in, dx, y_dtype=torch.bfloat16).float().cpu().numpy()
+    ys = lib.llvq_gemv_sorted(ctx, lib.llvq_sort_blocks(ctx, ds, n_out, k_in), dg, n_out, k_in, dx,
+                              y_dtype=torch.bfloat16).float().cpu().numpy()
+    rows = sorted(set([0, 7, 8, n_out // 2, n_out - 9, n_out - 1] + list(range(3, n_out, n_out // 19))))
+    ref = np.array([o.gemv(stream, gain, n_out, k_in, x, rows=(r, 1))[r] for r in rows])
+    floor = 1e-3 * float(np.abs(ref).max())
+    for got in (y, ys):
+        assert (np.abs(got[rows] - ref) / np.maximum(np.abs(ref), floor)).max() <= TOL_BF16_OUT
+    assert gemv_error(ys, y.astype(np.float64)) <= 2.0 ** -7          # all rows, one kernel against the other
+    assert lib.llvq_last_error(ctx) == (0, 0)
+
+
 def test_gemv_at_the_largest_row_count(lib, ctxs, oracle_mod):
     # 64 * 65536 rows is the most the scratch rows, arrival counters and pair slots of a context are sized for
     o = _oracle(oracle_mod)((2, 2))
