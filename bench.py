@@ -108,7 +108,7 @@ class ClockSampler:
                         self.reasons.add(k)
             except Exception:
                 pass
-            time.sleep(0.002)
+            time.sleep(0.0005)
 
     def __enter__(self):
         if self._nv is not None:
@@ -575,6 +575,10 @@ def main() -> None:
     value = whole_job_value(world, step_bytes, ms_per_step)
     timed_launches = launches
 
+    # a second sampler covers every other timed pass of this run (per layer, sorted layout, end to end)
+    clocks_rest = ClockSampler(local_rank)
+    clocks_rest.__enter__()
+
     # per-layer device time of the kernel: events around a run of back-to-back launches of that layer, same rotation
     per_layer = []
     for li, (n, k) in enumerate(LAYERS):
@@ -658,6 +662,7 @@ def main() -> None:
     barrier()
     e2e_ms = max_over_ranks(ev0.elapsed_time(ev1) / e2e_steps, dist, "cuda")
     e2e_value = whole_job_value(world, step_bytes, e2e_ms)
+    clocks_rest.__exit__(None, None, None)
 
     bad, flags = P.llvq_last_error(ctx)
     if bad or flags:
@@ -695,6 +700,7 @@ def main() -> None:
             "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "ms_per_step": e2e_ms},
             "gpu_launches": timed_launches,
             "clocks": clocks.summary(),
+            "clocks_other_timed_passes": clocks_rest.summary(),
         }
         if world == 1 and not args.no_extras:
             del sets, host_sets
