@@ -107,14 +107,15 @@ class RowShardedGemv:
         self._own, handle = llvq_exchange_create(ctx, _FLAG_BYTES + 2 * self._y_bytes)
         handles = exchange_handles(handle, group)
         self._bufs = [self._own if r == self.rank else llvq_exchange_open(ctx, handles[r]) for r in range(self.world)]
-        typestr = "<f4" if y_dtype == torch.float32 else "<i2"
-        self._views = []
-        for parity in range(2):
-            raw = torch.as_tensor(_RawDeviceArray(self._own + _FLAG_BYTES + parity * self._y_bytes, n_out, typestr),
-                                  device=torch.device("cuda", ctx.device))
-            self._views.append(raw if y_dtype == torch.float32 else raw.view(torch.bfloat16))
+        self._views = [self._wrap(self._own + _FLAG_BYTES + parity * self._y_bytes) for parity in range(2)]
         self.epoch = 0
         dist.barrier(group)                         # every buffer is mapped everywhere before anybody writes
+
+    def _wrap(self, ptr: int) -> torch.Tensor:
+        """A tensor over one of the own y buffers (device memory that the library allocated)."""
+        typestr = "<f4" if self.y_dtype == torch.float32 else "<i2"
+        raw = torch.as_tensor(_RawDeviceArray(ptr, self.n_out, typestr), device=torch.device("cuda", self.ctx.device))
+        return raw if self.y_dtype == torch.float32 else raw.view(torch.bfloat16)
 
     def _y_all(self, parity: int) -> list[int]:
         return [b + _FLAG_BYTES + parity * self._y_bytes for b in self._bufs]
@@ -140,12 +141,15 @@ class RowShardedGemv:
         self.launch(d_x, stream)
         return self.wait(stream)
 
+    def _synchronize(self) -> None:
+        torch.cuda.synchronize(self.ctx.device)
+
     def close(self) -> None:
         """Collective: unmap the peers' buffers, then free the own one."""
         import torch.distributed as dist
         if self._bufs is None:
             return
-        torch.cuda.synchronize(self.ctx.device)
+        self._synchronize()
         for r, b in enumerate(self._bufs):
             if r != self.rank:
                 llvq_exchange_close(self.ctx, b)

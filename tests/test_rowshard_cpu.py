@@ -98,3 +98,73 @@ def test_two_ranks_assemble_the_unsharded_product():
         assert handles == [bytes([0]) * 64, bytes([1]) * 64]    # every rank holds every handle, in rank order
         assert same
     assert res[0][2] == (0, 48) and res[1][2] == (48, 35)
+
+
+def _protocol_rank(rank, world, port, out):
+    """The order and the arguments of the device calls of RowShardedGemv, with the library calls replaced by recorders."""
+    sys.path.insert(0, ROOT)
+    from types import SimpleNamespace
+    import torch
+    import torch.distributed as dist
+    import paper_2603_11021_b200.rowshard as rs
+    os.environ.update(MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port), RANK=str(rank), WORLD_SIZE=str(world))
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    log = []
+    own = 0x10000000 * (rank + 1)
+    mapped = lambda r: 0x10000000 * (r + 1) + 0x5000000              # where this process "maps" rank r's buffer
+    rs.llvq_exchange_create = lambda ctx, nbytes: (log.append(("create", nbytes)), (own, bytes([rank]) * 64))[1]
+    rs.llvq_exchange_open = lambda ctx, handle: mapped(handle[0])
+    rs.llvq_exchange_close = lambda ctx, p: log.append(("close", p))
+    rs.llvq_exchange_destroy = lambda ctx, p: log.append(("destroy", p))
+    rs.llvq_gemv_rowshard = lambda ctx, s, g, n, k, x, y_all, slot, row0, dt, words, epoch, stream: \
+        log.append(("gemv", n, k, x, tuple(y_all), slot, row0, tuple(words), epoch))
+    rs.llvq_signal_ranks = lambda ctx, words, epoch, stream=None: log.append(("signal", tuple(words), epoch))
+    rs.llvq_wait_ranks = lambda ctx, flags, w, skip, epoch, spins=0, stream=None: log.append(("wait", flags, w, skip, epoch))
+
+    class Recorded(rs.RowShardedGemv):
+        def _wrap(self, ptr):
+            return ptr
+
+        def _synchronize(self):
+            pass
+
+    n_out, k_in = 12, 600                                             # two row groups: ranks 0 and 1 get 8 and 4 rows, rank 2 none
+    op = Recorded(SimpleNamespace(device=0), n_out, k_in, "stream", "gain", torch.float32)
+    y1 = op(d_x="x1")
+    y2 = op(d_x="x2")
+    op.close()
+    out[rank] = (log, y1, y2, own, [mapped(r) for r in range(world)])
+    dist.barrier()
+    dist.destroy_process_group()
+
+
+def test_three_ranks_step_protocol():
+    world = 3
+    ctx = mp.get_context("spawn")
+    with ctx.Manager() as m:
+        out = m.dict()
+        procs = [ctx.Process(target=_protocol_rank, args=(r, world, 29553, out)) for r in range(world)]
+        for p in procs:
+            p.start()
+        for p in procs:
+            p.join(180)
+            assert p.exitcode == 0
+        res = dict(out)
+    y_bytes = 256                                                     # 12 floats, padded to 256 bytes
+    bands = [(0, 8), (8, 4), (12, 0)]
+    for r in range(world):
+        log, y1, y2, own, mapped = res[r]
+        bufs = [own if q == r else mapped[q] for q in range(world)]
+        words = tuple(b + 4 * r for b in bufs)                        # this rank's flag word in every buffer
+        y_at = lambda parity: tuple(b + 256 + parity * y_bytes for b in bufs)
+        assert log[0] == ("create", 256 + 2 * y_bytes)
+        row0, n = bands[r]
+        if n:
+            step1 = ("gemv", n, 600, "x1", y_at(1), r, row0, words, 1)
+            step2 = ("gemv", n, 600, "x2", y_at(0), r, row0, words, 2)
+        else:                                                         # no rows: the flags still go out
+            peers = tuple(w for q, w in enumerate(words) if q != r)
+            step1, step2 = ("signal", peers, 1), ("signal", peers, 2)
+        assert log[1:5] == [step1, ("wait", own, world, r, 1), step2, ("wait", own, world, r, 2)]
+        assert (y1, y2) == (own + 256 + y_bytes, own + 256)           # the two y buffers alternate with the epoch
+        assert log[5:] == [("close", mapped[q]) for q in range(world) if q != r] + [("destroy", own)]
