@@ -1139,7 +1139,10 @@ gemm_sorted_kernel(FastArgs fa, const unsigned long long* __restrict__ sorted, c
         const ulonglong2 no_entry = make_ulonglong2(kSortIndexMask, kBigNoBlock);
         auto entry_at = [&](int d, int q) {
             if (d + q >= d_end) return no_entry;
-            const int64_t at = (rt * nd + d + q) * kDomEntries + (q == 0 ? warp : 31 - warp) * 32 + lane;
+            // warp 0 also issues the MMAs of every iteration: it takes the cheapest chunk of each domain (the last), the other
+            // warps pair chunk w - 1 of the first domain with chunk 31 - w of the second
+            const int chunk = warp == 0 ? 31 : (q == 0 ? warp - 1 : 31 - warp);
+            const int64_t at = (rt * nd + d + q) * kDomEntries + chunk * 32 + lane;
             if (kBig) return __ldg(reinterpret_cast<const ulonglong2*>(sorted) + at);
             return make_ulonglong2(__ldg(sorted + at), 0ull);
         };
@@ -1266,6 +1269,220 @@ gemm_sorted_kernel(FastArgs fa, const unsigned long long* __restrict__ sorted, c
     if (warp == 0) tmem_dealloc(tmem, kTmemCols);
 }
 
+// The same product for padded batch <= 32, where two domains' tiles fit: the two buffer sets alternate between
+// consecutive domains and nobody waits for the whole CTA.  Warps 1..31 unrank: the chunks of 32 sorted entries of a
+// row tile are handed out by a ticket counter (ticket t = chunk t % 32 of the tile's domain t / 32, so from expensive
+// to cheap inside a domain), a warp always holding its next ticket with that chunk's entries already requested.
+// It unranks the chunk, waits (rarely) until the MMAs that read this buffer two domains ago are done, writes its
+// part of A and arrives on the buffer's "full" barrier.  Warp 0 stages the X slice of the next domain, arrives too,
+// and its first thread issues the MMAs of a domain as soon as that barrier completes.
+template <bool kBig, bool kSg = false, bool kShard = false>
+__global__ void __launch_bounds__(kGemmThreads, 1)
+gemm_pipe_kernel(FastArgs fa, const unsigned long long* __restrict__ sorted, const uint16_t* __restrict__ gain, SgArgs sg, GemmArgs ga,
+                 int b_double)
+{
+    extern __shared__ __align__(128) uint8_t smem[];
+    const uint32_t img_bytes = fa.L.total;
+    uint64_t* bar_img = reinterpret_cast<uint64_t*>(smem + img_bytes);
+    uint64_t* bar_full = bar_img + 1;                                     // [2] 32 chunks of A and the X slice are in the buffer
+    uint64_t* bar_free = bar_img + 3;                                     // [2] the MMAs reading the buffer are done
+    uint64_t* bar_done = bar_img + 5;                                     // the accumulator of this row tile is complete
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bar_img + 6);
+    uint32_t* last_flag = tmem_slot + 1;
+    uint32_t* ticket = tmem_slot + 2;                                     // next chunk ticket of the row tile in progress
+    const uint32_t a_off = (img_bytes + 64 + 1023) & ~1023u;
+    constexpr uint32_t kAStage = kGemmRows * kStageK * 2;                  // 24576
+    uint8_t* a_buf = smem + a_off;                                        // [2 buffers][2 stages] x 24576
+    const uint32_t b_stage = (uint32_t)ga.npad * kStageK * 2;
+    uint8_t* b_buf = a_buf + 2u * kDomStages * kAStage;                    // [2 buffers, or 1][2 stages] x npad * 192
+    constexpr uint32_t kWorkers = kGemmThreads / 32 - 1;                   // 31 unranking warps
+
+    pdl_launch_dependents();
+    if (!fast_load_image(smem, fa.image, fa.L.total, bar_img, fa.flags)) return;
+    pdl_wait();
+    const FastSmem T = fast_view(smem, fa.L);
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    if (threadIdx.x == 0) {
+        mbar_init(bar_full, 33); mbar_init(bar_full + 1, 33);             // 32 chunks + the X slice
+        mbar_init(bar_free, 1); mbar_init(bar_free + 1, 1); mbar_init(bar_done, 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 0) tmem_alloc(tmem_slot, kTmemCols);
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = *tmem_slot;
+    const uint32_t idesc = instr_desc_bf16_m128((uint32_t)ga.npad);
+    const int64_t row_tiles = (ga.n_out + kGemmRows - 1) / kGemmRows;
+    const int64_t nd = ga.nstages;                                         // domains per row tile
+    const int64_t D = row_tiles * nd, G = gridDim.x;
+    const int64_t dom_begin = blockIdx.x * D / G, dom_end = (blockIdx.x + 1) * D / G;
+    uint32_t g_base = 0, done = 0;                                         // domains this CTA has finished (domain g uses buffer g & 1 for the (g >> 1)-th time)
+    bool timeout = false;
+    const ulonglong2 no_entry = make_ulonglong2(kSortIndexMask, kBigNoBlock);
+    auto arrive_full = [&](uint32_t b) {
+        fence_async_smem();
+        __syncwarp();
+        if (lane == 0) asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar_full + b)) : "memory");
+    };
+
+    for (int64_t rt = dom_begin / nd; rt * nd < dom_end; ++rt) {
+        const int d_begin = (int)(max(dom_begin, rt * nd) - rt * nd), d_end = (int)(min(dom_end, (rt + 1) * nd) - rt * nd);
+        const uint32_t parts = (uint32_t)(unit_owner((rt + 1) * nd - 1, D, G) - unit_owner(rt * nd, D, G) + 1);   // CTAs that share this row tile
+        const uint32_t n_dom = (uint32_t)(d_end - d_begin), n_tickets = n_dom * 32u;
+        if (threadIdx.x == 0) *ticket = kWorkers;                          // the first tickets are the workers' own numbers
+        __syncthreads();
+        if (warp == 0) {
+            // ---- X slices and MMAs
+            // the slice of domain j of this tile, 16-byte chunks (8 values along K).  With two X buffers it may be written once
+            // the MMAs of two domains ago are done; with one (wide batches: no room for two), only after the previous domain's
+            auto stage_b = [&](uint32_t j) {
+                const uint32_t gd = g_base + j, b = gd & 1u, bx = b_double ? b : 0u;
+                if (b_double) { if (gd >= 2u && !mbar_wait(bar_free + b, ((gd >> 1) - 1u) & 1u)) timeout = true; }
+                else if (gd >= 1u && !mbar_wait(bar_free + ((gd - 1u) & 1u), ((gd - 1u) >> 1) & 1u)) timeout = true;
+                const int64_t k0 = (int64_t)(d_begin + (int)j) * kDomBlocks * 24;
+                for (int n = lane; n < ga.npad; n += 32) {
+                    const uint16_t* xr = ga.x + (int64_t)n * ga.k_in + k0;
+                    uint8_t* dst = b_buf + bx * kDomStages * b_stage + n * 16;
+#pragma unroll 4
+                    for (int kc = 0; kc < kDomStages * (kStageK / 8); ++kc) {        // 24 asynchronous 16-byte copies per row, zero-filled outside X
+                        const bool in = n < ga.batch && k0 + kc * 8 < ga.k_in;
+                        const uint32_t to = smem_u32(dst + (uint32_t)(kc / (kStageK / 8)) * b_stage + (uint32_t)(kc % (kStageK / 8)) * ga.npad * 16);
+                        asm volatile("cp.async.ca.shared.global [%0], [%1], 16, %2;" ::"r"(to), "l"(in ? xr + kc * 8 : ga.x), "r"(in ? 16u : 0u) : "memory");
+                    }
+                }
+                asm volatile("cp.async.wait_all;" ::: "memory");
+                arrive_full(b);
+            };
+            if (n_dom > 0) stage_b(0);
+            for (uint32_t j = 0; j < n_dom; ++j) {
+                if (b_double && j + 1 < n_dom) stage_b(j + 1);
+                const uint32_t gd = g_base + j, b = gd & 1u, bx = b_double ? b : 0u;
+                if (lane == 0) {
+                    if (!mbar_wait(bar_full + b, (gd >> 1) & 1u)) timeout = true;
+                    tc_fence_after();
+                    const uint32_t a_addr = smem_u32(a_buf) + b * kDomStages * kAStage, b_addr = smem_u32(b_buf) + bx * kDomStages * b_stage;
+                    for (int st = 0; st < kDomStages; ++st)
+#pragma unroll
+                        for (int jj = 0; jj < kStageK / 16; ++jj)
+                            umma_bf16(tmem, smem_desc(a_addr + st * kAStage + jj * 4096, 2048, 128),
+                                      smem_desc(b_addr + st * b_stage + jj * 2 * ga.npad * 16, ga.npad * 16, 128), idesc,
+                                      (j > 0 || st > 0 || jj > 0) ? 1u : 0u);
+                    umma_commit(bar_free + b);
+                    if (j + 1 == n_dom) umma_commit(bar_done);
+                }
+                __syncwarp();
+                if (!b_double && j + 1 < n_dom) stage_b(j + 1);
+            }
+        } else {
+            // ---- A: unrank chunks until the tile's tickets are gone
+            auto entry_of = [&](uint32_t t) {
+                if (t >= n_tickets) return no_entry;
+                const int64_t at = (rt * nd + d_begin + (int)(t >> 5)) * kDomEntries + (t & 31u) * 32u + lane;
+                if (kBig) return __ldg(reinterpret_cast<const ulonglong2*>(sorted) + at);
+                return make_ulonglong2(__ldg(sorted + at), 0ull);
+            };
+            uint32_t tk = (uint32_t)warp - 1u;
+            ulonglong2 e = entry_of(tk);
+            while (tk < n_tickets) {
+                uint32_t tk_next = 0;
+                if (lane == 0) tk_next = atomicAdd(ticket, 1u);
+                tk_next = __shfl_sync(kFullMask, tk_next, 0);
+                const ulonglong2 e_next = entry_of(tk_next);                // requested a chunk ahead (it comes from DRAM)
+                const uint32_t j = tk >> 5, gd = g_base + j, b = gd & 1u;
+                const int d = d_begin + (int)j;
+                const uint64_t field = e.x & kSortIndexMask;
+                const uint64_t I = kSg ? field & ((1ull << fa.L.W) - 1ull) : field;     // shape-gain form: gain index above the shape index
+                const uint32_t pos = kBig ? (uint32_t)(e.y >> 32) & 1023u : (uint32_t)(e.x >> 48);
+                const bool valid = kBig ? !(e.y >> 63) : (field != kSortIndexMask && I < fa.n_points);
+                const uint32_t r = pos >> 3, c = pos & 7u;
+                const int64_t row = rt * kGemmRows + r, cb = (int64_t)d * kDomBlocks + c;
+                float gn = (!kSg && valid) ? gain_to_float(__ldg(gain + row * ga.bpr + cb)) : 0.f;
+                uint32_t w[12];
+                if (kBig) {
+                    const int cls = valid ? (int)((uint32_t)(e.y >> 8) & 0xffffffu) : 0;
+                    const uint64_t local = valid ? e.x - __ldg(fa.dc.off_lo + cls) : 0ull;     // class sizes fit 63 bits: exact mod 2^64
+                    Point pt;
+                    big_decode_local(T, fa.dc, cls, local, valid, pt);
+#pragma unroll
+                    for (int jj = 0; jj < 12; ++jj) {
+                        __nv_bfloat162 h = __halves2bfloat162(dequant(gn, pt, 2 * jj), dequant(gn, pt, 2 * jj + 1));
+                        w[jj] = *reinterpret_cast<uint32_t*>(&h);
+                    }
+                } else {
+                    Decoded dec;
+                    const uint32_t cls = decode_sorted_entry(fa, T, I, valid, dec);
+                    if (kSg && valid) {
+                        const float scale = sg.row_scale ? __ldg(sg.row_scale + row) : 1.f;
+                        gn = __fmul_rn(__fmul_rn(scale, __ldg(sg.codebook + (uint32_t)(field >> fa.L.W))),
+                                       __uint_as_float(T.desc[cls * kFastDescStride + kFastDescRnorm]));
+                    }
+                    expand_bf16(dec, gn, w);
+                }
+                // the MMAs of two domains ago read this buffer: wait for them only now, with the chunk already unranked
+                if (gd >= 2u && !mbar_wait(bar_free + b, ((gd >> 1) - 1u) & 1u)) timeout = true;
+                uint8_t* a_dst = a_buf + (b * kDomStages + (c >> 2)) * kAStage + (r >> 3) * 128u + (r & 7u) * 16u + 3u * (c & 3u) * 2048u;
+#pragma unroll
+                for (int jj = 0; jj < 3; ++jj)
+                    *reinterpret_cast<uint4*>(a_dst + jj * 2048) = make_uint4(w[4 * jj], w[4 * jj + 1], w[4 * jj + 2], w[4 * jj + 3]);
+                arrive_full(b);
+                tk = tk_next; e = e_next;
+            }
+        }
+        g_base += n_dom;
+        const bool has = d_end > d_begin;
+        // ---- epilogue: accumulator -> scratch (split-K) or Y
+        if (warp < 4 && has) {
+            if (!mbar_wait(bar_done, done & 1u)) timeout = true;
+            tc_fence_after();
+            const int64_t orow = rt * kGemmRows + warp * 32 + lane;
+            for (int c0 = 0; c0 < ga.npad; c0 += 16) {
+                float v[16];
+                tmem_ld16(tmem + ((uint32_t)(warp * 32) << 16) + (uint32_t)c0, v);
+                if (orow < ga.n_out) {
+#pragma unroll
+                    for (int i = 0; i < 16; ++i) {
+                        const int n = c0 + i;
+                        if (n < ga.batch) {
+                            if (parts == 1u) gemm_store<kShard>(ga, n, orow, v[i]);
+                            else atomicAdd(ga.scratch + (int64_t)n * ga.scratch_ld + orow, v[i]);
+                        }
+                    }
+                }
+            }
+            tc_fence_before();
+        }
+        done += has;
+        if (parts > 1u) {
+            __threadfence();
+            __syncthreads();
+            if (threadIdx.x == 0) *last_flag = (atomicAdd(ga.counters + rt, 1u) == parts - 1u);
+            __syncthreads();
+            if (*last_flag) {
+                __threadfence();
+                for (int i = threadIdx.x; i < kGemmRows * ga.batch; i += kGemmThreads) {
+                    const int n = i / kGemmRows;
+                    const int64_t orow = rt * kGemmRows + (i % kGemmRows);
+                    if (orow < ga.n_out) {
+                        float* sp = ga.scratch + (int64_t)n * ga.scratch_ld + orow;
+                        gemm_store<kShard>(ga, n, orow, __ldcg(sp));
+                        __stcg(sp, 0.f);
+                    }
+                }
+                if (threadIdx.x == 0) ga.counters[rt] = 0u;
+            }
+        }
+        __syncthreads();
+    }
+    if (timeout) atomicOr(fa.flags, 1u);
+    if (kShard) {
+        __threadfence_system();                           // this thread's stores to the peers' copies, before the CTA counts itself in
+        shard_arrive(*ga.shard);
+    }
+    __syncthreads();
+    if (warp == 0) tmem_dealloc(tmem, kTmemCols);
+}
+
 FastArgs fast_args(const llvq_ctx* ctx)
 {
     FastArgs fa;
@@ -1330,37 +1547,44 @@ int launch_gemm_domains(const llvq_ctx* ctx, const void* p, const uint16_t* d_ga
     ga.batch = batch; ga.npad = (batch + 15) / 16 * 16;
     ga.nstages = (int)((ga.bpr + kDomBlocks - 1) / kDomBlocks);              // domains per row tile
     ga.x = d_x_bf16; ga.scratch = scratch; ga.counters = counters;
-    const int dpi = ga.npad <= 32 ? 2 : 1;                                   // domains unranked per iteration (shared memory decides)
+    int dpi = ga.npad <= 32 ? 2 : 1;                                         // gemm_sorted_kernel: domains unranked per iteration (shared memory decides)
     const int64_t row_tiles = (n_out + kGemmRows - 1) / kGemmRows;
     ga.scratch_ld = row_tiles * kGemmRows;
     ga.split = 1;                                                             // unused: the kernel balances domains over the CTAs itself
     const unsigned grid = (unsigned)std::min<int64_t>(row_tiles * ga.nstages, ctx->sm_count);
-    const size_t smem = ((ctx->fl.total + 64 + 1023) & ~size_t(1023)) + (size_t)dpi * kDomStages * (kGemmRows * kStageK * 2 + (size_t)ga.npad * kStageK * 2);
+    // gemm_pipe_kernel: two A buffer sets and two X buffer sets, or one X set when two do not fit; else the kernel with the block barrier
+    const size_t head = (ctx->fl.total + 64 + 1023) & ~size_t(1023), a_set = (size_t)kDomStages * kGemmRows * kStageK * 2,
+                 x_set = (size_t)kDomStages * ga.npad * kStageK * 2;
+    int pipe = 0, b_double = 0;
+    size_t smem = head + (size_t)dpi * (a_set + x_set);
+    if (!ctx->fast) {}                                   // the 72-bit code gains nothing from the pipeline (measured): it keeps the kernel below
+    else if (head + 2 * a_set + 2 * x_set <= 227 * 1024) { pipe = 1; b_double = 1; smem = head + 2 * a_set + 2 * x_set; }
+    else if (head + 2 * a_set + x_set <= 227 * 1024) { pipe = 1; smem = head + 2 * a_set + x_set; }
     if (smem > 227 * 1024) return LLVQ_EUNSUPPORTED;
+#define LLVQ_LAUNCH_DOMAINS(BIG, SG, SH)                                                                                      \
+    do {                                                                                                                     \
+        if (pipe) {                                                                                                          \
+            if (!set_smem(gemm_pipe_kernel<BIG, SG, SH>, smem)) return LLVQ_ECUDA;                                            \
+            if (launch_pdl(gemm_pipe_kernel<BIG, SG, SH>, grid, (unsigned)kGemmThreads, smem, (cudaStream_t)stream, fast_args(ctx), \
+                           static_cast<const unsigned long long*>(p), d_gain_f16, sga, ga, b_double) != cudaSuccess) return LLVQ_ECUDA; \
+        } else {                                                                                                             \
+            if (!set_smem(gemm_sorted_kernel<BIG, SG, SH>, smem)) return LLVQ_ECUDA;                                          \
+            if (launch_pdl(gemm_sorted_kernel<BIG, SG, SH>, grid, (unsigned)kGemmThreads, smem, (cudaStream_t)stream, fast_args(ctx), \
+                           static_cast<const unsigned long long*>(p), d_gain_f16, sga, ga, dpi) != cudaSuccess) return LLVQ_ECUDA; \
+        }                                                                                                                    \
+    } while (0)
+    const SgArgs sga = sg ? *sg : SgArgs{};
     if (yo) {                                            // row-sharded: stored-gain form only
         if (sg) return LLVQ_EUNSUPPORTED;
-        if (ctx->fast) {
-            if (!set_smem(gemm_sorted_kernel<false, false, true>, smem)) return LLVQ_ECUDA;
-            if (launch_pdl(gemm_sorted_kernel<false, false, true>, grid, (unsigned)kGemmThreads, smem, (cudaStream_t)stream, fast_args(ctx),
-                           static_cast<const unsigned long long*>(p), d_gain_f16, SgArgs{}, ga, dpi) != cudaSuccess) return LLVQ_ECUDA;
-        } else {
-            if (!set_smem(gemm_sorted_kernel<true, false, true>, smem)) return LLVQ_ECUDA;
-            if (launch_pdl(gemm_sorted_kernel<true, false, true>, grid, (unsigned)kGemmThreads, smem, (cudaStream_t)stream, fast_args(ctx),
-                           static_cast<const unsigned long long*>(p), d_gain_f16, SgArgs{}, ga, dpi) != cudaSuccess) return LLVQ_ECUDA;
-        }
+        if (ctx->fast) LLVQ_LAUNCH_DOMAINS(false, false, true); else LLVQ_LAUNCH_DOMAINS(true, false, true);
     } else if (sg) {
-        if (!set_smem(gemm_sorted_kernel<false, true>, smem)) return LLVQ_ECUDA;
-        if (launch_pdl(gemm_sorted_kernel<false, true>, grid, (unsigned)kGemmThreads, smem, (cudaStream_t)stream, fast_args(ctx),
-                       static_cast<const unsigned long long*>(p), d_gain_f16, *sg, ga, dpi) != cudaSuccess) return LLVQ_ECUDA;
+        LLVQ_LAUNCH_DOMAINS(false, true, false);
     } else if (ctx->fast) {
-        if (!set_smem(gemm_sorted_kernel<false, false>, smem)) return LLVQ_ECUDA;
-        if (launch_pdl(gemm_sorted_kernel<false, false>, grid, (unsigned)kGemmThreads, smem, (cudaStream_t)stream, fast_args(ctx),
-                       static_cast<const unsigned long long*>(p), d_gain_f16, SgArgs{}, ga, dpi) != cudaSuccess) return LLVQ_ECUDA;
+        LLVQ_LAUNCH_DOMAINS(false, false, false);
     } else {
-        if (!set_smem(gemm_sorted_kernel<true, false>, smem)) return LLVQ_ECUDA;
-        if (launch_pdl(gemm_sorted_kernel<true, false>, grid, (unsigned)kGemmThreads, smem, (cudaStream_t)stream, fast_args(ctx),
-                       static_cast<const unsigned long long*>(p), d_gain_f16, SgArgs{}, ga, dpi) != cudaSuccess) return LLVQ_ECUDA;
+        LLVQ_LAUNCH_DOMAINS(true, false, false);
     }
+#undef LLVQ_LAUNCH_DOMAINS
     return launch_status();
 }
 
