@@ -1276,11 +1276,14 @@ gemm_sorted_kernel(FastArgs fa, const unsigned long long* __restrict__ sorted, c
 // It unranks the chunk, waits (rarely) until the MMAs that read this buffer two domains ago are done, writes its
 // part of A and arrives on the buffer's "full" barrier.  Warp 0 stages the X slice of the next domain, arrives too,
 // and its first thread issues the MMAs of a domain as soon as that barrier completes.
-template <bool kBig, bool kSg = false, bool kShard = false>
+// kStored: the same structure on the stored stream (`sorted` then points at it): a chunk is 32 consecutive blocks of the
+// domain in natural order (4 rows x 8 column blocks), unranked by the any-class decoder.
+template <bool kBig, bool kSg = false, bool kShard = false, bool kStored = false>
 __global__ void __launch_bounds__(kGemmThreads, 1)
 gemm_pipe_kernel(FastArgs fa, const unsigned long long* __restrict__ sorted, const uint16_t* __restrict__ gain, SgArgs sg, GemmArgs ga,
                  int b_double)
 {
+    static_assert(!(kStored && kBig), "the stored-stream form exists for the codes with tables in shared memory");
     extern __shared__ __align__(128) uint8_t smem[];
     const uint32_t img_bytes = fa.L.total;
     uint64_t* bar_img = reinterpret_cast<uint64_t*>(smem + img_bytes);
@@ -1378,6 +1381,14 @@ gemm_pipe_kernel(FastArgs fa, const unsigned long long* __restrict__ sorted, con
             // ---- A: unrank chunks until the tile's tickets are gone
             auto entry_of = [&](uint32_t t) {
                 if (t >= n_tickets) return no_entry;
+                if (kStored) {                                               // the field itself, its position in the high 16 bits
+                    const uint32_t pos = (t & 31u) * 32u + lane;
+                    const int64_t row = rt * kGemmRows + (pos >> 3), cb = (int64_t)(d_begin + (int)(t >> 5)) * kDomBlocks + (pos & 7u);
+                    unsigned long long f = kSortIndexMask;
+                    if (row < ga.n_out && cb < ga.bpr)
+                        f = load_field(reinterpret_cast<const uint32_t*>(sorted), (uint64_t)(row * ga.bpr + cb), (int)fa.L.W + (kSg ? sg.bits : 0));
+                    return make_ulonglong2(f | (unsigned long long)pos << 48, 0ull);
+                }
                 const int64_t at = (rt * nd + d_begin + (int)(t >> 5)) * kDomEntries + (t & 31u) * 32u + lane;
                 if (kBig) return __ldg(reinterpret_cast<const ulonglong2*>(sorted) + at);
                 return make_ulonglong2(__ldg(sorted + at), 0ull);
@@ -1411,7 +1422,15 @@ gemm_pipe_kernel(FastArgs fa, const unsigned long long* __restrict__ sorted, con
                     }
                 } else {
                     Decoded dec;
-                    const uint32_t cls = decode_sorted_entry(fa, T, I, valid, dec);
+                    uint32_t cls;
+                    if (kStored) {
+                        if (field != kSortIndexMask && !valid) atomicAdd(fa.bad_index, 1ull);
+                        uint64_t local = 0;
+                        cls = valid ? fast_find_class(T, I, local) : 0u;
+                        fast_decode_local<-1>(T, cls, local, valid, kFullMask, dec);
+                    } else {
+                        cls = decode_sorted_entry(fa, T, I, valid, dec);
+                    }
                     if (kSg && valid) {
                         const float scale = sg.row_scale ? __ldg(sg.row_scale + row) : 1.f;
                         gn = __fmul_rn(__fmul_rn(scale, __ldg(sg.codebook + (uint32_t)(field >> fa.L.W))),
@@ -1625,8 +1644,32 @@ int launch_gemm(const llvq_ctx* ctx, const void* d_idx, const uint16_t* d_gain_f
     const size_t smem = ((img + 64 + 1023) & ~size_t(1023)) + 2 * kGemmRows * kStageK * 2 + 2 * (size_t)ga.npad * kStageK * 2;
     if (smem > 227 * 1024) return LLVQ_EUNSUPPORTED;
     const uint32_t* idx = static_cast<const uint32_t*>(d_idx);
-    if (yo) {                                            // row-sharded: stored-gain form only
-        if (sg) return LLVQ_EUNSUPPORTED;
+    if (yo && sg) return LLVQ_EUNSUPPORTED;              // row-sharded: stored-gain form only
+    if (ctx->fast) {
+        // codes with their tables in shared memory: the kernel without a block barrier (see gemm_pipe_kernel), if its buffers fit
+        const size_t head = (img + 64 + 1023) & ~size_t(1023), a_set = (size_t)kDomStages * kGemmRows * kStageK * 2,
+                     x_set = (size_t)kDomStages * ga.npad * kStageK * 2;
+        const int b_double = head + 2 * a_set + 2 * x_set <= 227 * 1024;
+        const size_t smem_pipe = head + 2 * a_set + (b_double ? 2 : 1) * x_set;
+        if (smem_pipe <= 227 * 1024) {
+            GemmArgs gp = ga;
+            gp.nstages = (int)((ga.bpr + kDomBlocks - 1) / kDomBlocks);        // domains per row tile
+            gp.split = 1;
+            const unsigned grid_pipe = (unsigned)std::min<int64_t>(row_tiles * gp.nstages, ctx->sm_count);
+            const unsigned long long* words = static_cast<const unsigned long long*>(d_idx);
+            const SgArgs sga = sg ? *sg : SgArgs{};
+#define LLVQ_LAUNCH_PIPE_STORED(SG, SH)                                                                                         \
+    do {                                                                                                                        \
+        if (!set_smem(gemm_pipe_kernel<false, SG, SH, true>, smem_pipe)) return LLVQ_ECUDA;                                      \
+        if (launch_pdl(gemm_pipe_kernel<false, SG, SH, true>, grid_pipe, (unsigned)kGemmThreads, smem_pipe, st, fast_args(ctx), words, \
+                       d_gain_f16, sga, gp, b_double) != cudaSuccess) return LLVQ_ECUDA;                                        \
+    } while (0)
+            if (yo) LLVQ_LAUNCH_PIPE_STORED(false, true); else if (sg) LLVQ_LAUNCH_PIPE_STORED(true, false); else LLVQ_LAUNCH_PIPE_STORED(false, false);
+#undef LLVQ_LAUNCH_PIPE_STORED
+            return launch_status();
+        }
+    }
+    if (yo) {
         if (ctx->fast) {
             if (!set_smem(gemm_kernel<false, false, true>, smem)) return LLVQ_ECUDA;
             if (launch_pdl(gemm_kernel<false, false, true>, grid, (unsigned)kGemmThreads, smem, st, fast_args(ctx), idx, d_gain_f16, SgArgs{}, ga) != cudaSuccess) return LLVQ_ECUDA;
