@@ -1283,7 +1283,7 @@ __global__ void __launch_bounds__(kGemmThreads, 1)
 gemm_pipe_kernel(FastArgs fa, const unsigned long long* __restrict__ sorted, const uint16_t* __restrict__ gain, SgArgs sg, GemmArgs ga,
                  int b_double)
 {
-    static_assert(!(kStored && kBig), "the stored-stream form exists for the codes with tables in shared memory");
+    static_assert(!(kStored && kBig && kSg), "no shape-gain form for the codes with tables in global memory");
     extern __shared__ __align__(128) uint8_t smem[];
     const uint32_t img_bytes = fa.L.total;
     uint64_t* bar_img = reinterpret_cast<uint64_t*>(smem + img_bytes);
@@ -1381,6 +1381,13 @@ gemm_pipe_kernel(FastArgs fa, const unsigned long long* __restrict__ sorted, con
             // ---- A: unrank chunks until the tile's tickets are gone
             auto entry_of = [&](uint32_t t) {
                 if (t >= n_tickets) return no_entry;
+                if (kStored && kBig) {                                       // the index itself, in the form of the sorted layout's entries
+                    const uint32_t pos = (t & 31u) * 32u + lane;
+                    const int64_t row = rt * kGemmRows + (pos >> 3), cb = (int64_t)(d_begin + (int)(t >> 5)) * kDomBlocks + (pos & 7u);
+                    uint64_t lo = 0, hi = kBigNoBlock;
+                    if (row < ga.n_out && cb < ga.bpr) load_index(reinterpret_cast<const uint32_t*>(sorted), (uint64_t)(row * ga.bpr + cb), fa.dc.W, lo, hi);
+                    return make_ulonglong2(lo, hi | (unsigned long long)pos << 32);
+                }
                 if (kStored) {                                               // the field itself, its position in the high 16 bits
                     const uint32_t pos = (t & 31u) * 32u + lane;
                     const int64_t row = rt * kGemmRows + (pos >> 3), cb = (int64_t)(d_begin + (int)(t >> 5)) * kDomBlocks + (pos & 7u);
@@ -1405,14 +1412,24 @@ gemm_pipe_kernel(FastArgs fa, const unsigned long long* __restrict__ sorted, con
                 const uint64_t field = e.x & kSortIndexMask;
                 const uint64_t I = kSg ? field & ((1ull << fa.L.W) - 1ull) : field;     // shape-gain form: gain index above the shape index
                 const uint32_t pos = kBig ? (uint32_t)(e.y >> 32) & 1023u : (uint32_t)(e.x >> 48);
-                const bool valid = kBig ? !(e.y >> 63) : (field != kSortIndexMask && I < fa.n_points);
+                bool valid = kBig ? !(e.y >> 63) : (field != kSortIndexMask && I < fa.n_points);
+                if (kStored && kBig && valid) {                               // the stored index may be out of range: count it, treat it as no block
+                    const uint64_t hi = e.y & 0xffull;
+                    valid = hi < fa.dc.n_hi || (hi == fa.dc.n_hi && e.x < fa.dc.n_lo);
+                    if (!valid) atomicAdd(fa.bad_index, 1ull);
+                }
                 const uint32_t r = pos >> 3, c = pos & 7u;
                 const int64_t row = rt * kGemmRows + r, cb = (int64_t)d * kDomBlocks + c;
                 float gn = (!kSg && valid) ? gain_to_float(__ldg(gain + row * ga.bpr + cb)) : 0.f;
                 uint32_t w[12];
                 if (kBig) {
-                    const int cls = valid ? (int)((uint32_t)(e.y >> 8) & 0xffffffu) : 0;
-                    const uint64_t local = valid ? e.x - __ldg(fa.dc.off_lo + cls) : 0ull;     // class sizes fit 63 bits: exact mod 2^64
+                    int cls = 0;
+                    uint64_t local = 0;
+                    if (kStored) { if (valid) cls = big_find_class(fa.dc, e.x, e.y & 0xffull, local); }
+                    else if (valid) {
+                        cls = (int)((uint32_t)(e.y >> 8) & 0xffffffu);
+                        local = e.x - __ldg(fa.dc.off_lo + cls);                 // class sizes fit 63 bits: exact mod 2^64
+                    }
                     Point pt;
                     big_decode_local(T, fa.dc, cls, local, valid, pt);
 #pragma unroll
@@ -1645,26 +1662,29 @@ int launch_gemm(const llvq_ctx* ctx, const void* d_idx, const uint16_t* d_gain_f
     if (smem > 227 * 1024) return LLVQ_EUNSUPPORTED;
     const uint32_t* idx = static_cast<const uint32_t*>(d_idx);
     if (yo && sg) return LLVQ_EUNSUPPORTED;              // row-sharded: stored-gain form only
-    if (ctx->fast) {
-        // codes with their tables in shared memory: the kernel without a block barrier (see gemm_pipe_kernel), if its buffers fit
+    {
+        // the kernel without a block barrier (see gemm_pipe_kernel), if its buffers fit
         const size_t head = (img + 64 + 1023) & ~size_t(1023), a_set = (size_t)kDomStages * kGemmRows * kStageK * 2,
                      x_set = (size_t)kDomStages * ga.npad * kStageK * 2;
         const int b_double = head + 2 * a_set + 2 * x_set <= 227 * 1024;
         const size_t smem_pipe = head + 2 * a_set + (b_double ? 2 : 1) * x_set;
-        if (smem_pipe <= 227 * 1024) {
+        if (smem_pipe <= 227 * 1024 && (ctx->fast || ga.npad <= 32)) {    // 72-bit code at wide batches: slower than gemm_kernel (measured)
             GemmArgs gp = ga;
             gp.nstages = (int)((ga.bpr + kDomBlocks - 1) / kDomBlocks);        // domains per row tile
             gp.split = 1;
             const unsigned grid_pipe = (unsigned)std::min<int64_t>(row_tiles * gp.nstages, ctx->sm_count);
             const unsigned long long* words = static_cast<const unsigned long long*>(d_idx);
             const SgArgs sga = sg ? *sg : SgArgs{};
-#define LLVQ_LAUNCH_PIPE_STORED(SG, SH)                                                                                         \
+#define LLVQ_LAUNCH_PIPE_STORED(BIG, SG, SH)                                                                                    \
     do {                                                                                                                        \
-        if (!set_smem(gemm_pipe_kernel<false, SG, SH, true>, smem_pipe)) return LLVQ_ECUDA;                                      \
-        if (launch_pdl(gemm_pipe_kernel<false, SG, SH, true>, grid_pipe, (unsigned)kGemmThreads, smem_pipe, st, fast_args(ctx), words, \
+        if (!set_smem(gemm_pipe_kernel<BIG, SG, SH, true>, smem_pipe)) return LLVQ_ECUDA;                                        \
+        if (launch_pdl(gemm_pipe_kernel<BIG, SG, SH, true>, grid_pipe, (unsigned)kGemmThreads, smem_pipe, st, fast_args(ctx), words, \
                        d_gain_f16, sga, gp, b_double) != cudaSuccess) return LLVQ_ECUDA;                                        \
     } while (0)
-            if (yo) LLVQ_LAUNCH_PIPE_STORED(false, true); else if (sg) LLVQ_LAUNCH_PIPE_STORED(true, false); else LLVQ_LAUNCH_PIPE_STORED(false, false);
+            if (!ctx->fast) { if (yo) LLVQ_LAUNCH_PIPE_STORED(true, false, true); else LLVQ_LAUNCH_PIPE_STORED(true, false, false); }
+            else if (yo) LLVQ_LAUNCH_PIPE_STORED(false, false, true);
+            else if (sg) LLVQ_LAUNCH_PIPE_STORED(false, true, false);
+            else LLVQ_LAUNCH_PIPE_STORED(false, false, false);
 #undef LLVQ_LAUNCH_PIPE_STORED
             return launch_status();
         }
