@@ -264,6 +264,14 @@ def test_gemm_small_batch_other_codes(lib, ctxs, oracle_mod, code, n_out, k_in, 
     _gemm_check(lib, ctxs[code], _oracle(oracle_mod)(code), n_out, k_in, batch, seed=8)
 
 
+@pytest.mark.parametrize("batch", [16, 64])
+def test_gemm_code_whose_tables_leave_no_room_for_two_buffer_sets(lib, oracle_mod, batch):
+    # shells 2..16: 788 classes, tables still in shared memory but too large for the kernel without a block barrier,
+    # so the product runs through the kernel with the two alternating thread groups
+    ctx = lib.Context(2, 16, device=0)
+    _gemm_check(lib, ctx, _oracle(oracle_mod)((2, 16)), 300, 1000, batch, seed=9)
+
+
 def test_gemm_exact_integer_case(lib, ctxs, oracle_mod):
     # gains = 1, X = 0/1 patterns: every partial sum is a small integer, exact in binary32 and in bf16
     o = _oracle(oracle_mod)((2, 13))
