@@ -203,1321 +203,8 @@ dequant_fast_kernel(FastArgs fa, const uint32_t* __restrict__ stream, const uint
     }
 }
 
-// Fused dequant + GEMV.  The work is cut into units of 8 rows x 4 column blocks, numbered row group major, and
-// every CTA takes an equal contiguous range of units.  In a unit lane (g, t) = (lane / 4, lane % 4) decodes the
-// block (row g, column block 4q + t); its 12 packed bf16 pairs are the A fragments (rows 0..7; rows 8..15 are
-// zero) of six m16n8k16 tensor-core MMAs whose B fragment carries the matching 4 x 24 activations (the same in
-// all 8 columns), accumulating in binary32.  Row sums are collected in shared memory; a row group that is
-// split between CTAs is finished through a zero-kept global scratch and an arrival counter.
-constexpr int kGemvGroupRows = 8;        // rows per unit
-constexpr int kGemvGroupsPerPass = 128;  // row groups whose sums a CTA keeps in shared memory at a time
-
-__device__ __forceinline__ void mma_bf16_16816(float c[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0, uint32_t b1)
-{
-    asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
-                 : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3]) : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
-}
-
-// CTA that owns unit u when G CTAs split U units into ranges [c*U/G, (c+1)*U/G).
-__device__ __forceinline__ int64_t unit_owner(int64_t u, int64_t U, int64_t G) { return ((u + 1) * G - 1) / U; }
-
-// Where a GEMV kernel puts y.  Row-sharded over several GPUs (each rank owns a band of output rows, x is the same
-// everywhere), a rank writes its band straight into every rank's copy of the full vector: `y` is this rank's copy
-// and `peer` the other ranks' copies mapped into this process, every pointer already advanced to the band's first
-// row.  The stores to a peer travel over NVLink as plain remote writes.  n_peer = 0 is the single-GPU case.
-constexpr int64_t kPairSlotOffset = 64ll * 65536;      // floats: the 64-bit slots of finish_pass lie behind the binary32 scratch rows
-constexpr int kMaxShardPeers = 7;
-struct YOut {
-    void* y;
-    void* peer[kMaxShardPeers];
-    int n_peer;
-    // optional: one word per peer that receives `epoch` once the whole grid has stored its rows (done = the
-    // context's arrival counter, zero between launches)
-    uint32_t* flag[kMaxShardPeers];
-    uint32_t* done;
-    uint32_t epoch;
-    int n_flag;
-};
-
-template <bool kOutBf16, bool kShard>
-__device__ __forceinline__ void store_y(const YOut& yo, int64_t row, float v)
-{
-    if (kOutBf16) {
-        const __nv_bfloat16 h = __float2bfloat16_rn(v);
-        reinterpret_cast<__nv_bfloat16*>(yo.y)[row] = h;
-        if (!kShard) return;                              // the single-GPU instantiations carry none of what follows
-#pragma unroll
-        for (int p = 0; p < kMaxShardPeers; ++p)          // static indices: the struct stays in the parameter bank
-            if (p < yo.n_peer) reinterpret_cast<__nv_bfloat16*>(yo.peer[p])[row] = h;
-    } else {
-        reinterpret_cast<float*>(yo.y)[row] = v;
-        if (!kShard) return;
-#pragma unroll
-        for (int p = 0; p < kMaxShardPeers; ++p)
-            if (p < yo.n_peer) reinterpret_cast<float*>(yo.peer[p])[row] = v;
-    }
-}
-
-// Stages x for a GEMV CTA: xs[cb * 12 + j] = the bf16 pair (x[24 cb + 2j], x[24 cb + 2j + 1]), zero beyond k_in; `words`
-// = 12 x the number of column blocks staged.  16-byte loads where x allows them.
-__device__ __forceinline__ void stage_x(uint32_t* xs, const uint16_t* __restrict__ x, int64_t k_in, int64_t words)
-{
-    if ((reinterpret_cast<uintptr_t>(x) & 15) == 0) {
-        const int64_t full = k_in / 8;                                       // whole groups of 8 elements
-        for (int64_t v = threadIdx.x; v < words / 4; v += blockDim.x) {
-            uint4 q = make_uint4(0u, 0u, 0u, 0u);
-            if (v < full) q = __ldg(reinterpret_cast<const uint4*>(x) + v);
-            else {
-                uint32_t t[4];
-#pragma unroll
-                for (int j = 0; j < 4; ++j) {
-                    const int64_t e = 8 * v + 2 * j;
-                    const uint32_t lo = e < k_in ? __ldg(x + e) : 0u, hi = e + 1 < k_in ? __ldg(x + e + 1) : 0u;
-                    t[j] = lo | hi << 16;
-                }
-                q = make_uint4(t[0], t[1], t[2], t[3]);
-            }
-            reinterpret_cast<uint4*>(xs)[v] = q;
-        }
-        return;
-    }
-    for (int64_t i = threadIdx.x; i < words; i += blockDim.x) {
-        const int64_t e = 2 * i;
-        const uint32_t lo = e < k_in ? __ldg(x + e) : 0u, hi = e + 1 < k_in ? __ldg(x + e + 1) : 0u;
-        xs[i] = lo | hi << 16;
-    }
-}
-
-// End of a pass of a GEMV CTA over row groups rg0..rg1 (8 rows each; the CTA owns units [u_begin, u_end) of U, nq
-// units per row group, G CTAs): row_sum(i) is the CTA's sum for row i of the pass.  One warp per row group, lanes
-// 0..7 its rows, no CTA-wide barrier inside.  A group the CTA covers completely is final.  A group it shares with
-// neighbouring CTAs goes through the scratch row in global memory: add, make the add visible, count the arrival;
-// whoever arrives last reads the total, writes y and leaves scratch and counter zero for the next launch (groups shared
-// by exactly two CTAs take a shorter way, below).
-// The caller puts a __syncthreads() before (sums complete) and after (sums may be cleared) the call.
-template <bool kOutBf16, bool kShard, typename RowSum>
-__device__ __forceinline__ void finish_pass(const YOut& yo, int64_t rg0, int64_t rg1, int64_t nq, int64_t u_begin, int64_t u_end,
-                                            int64_t U, int64_t G, int64_t n_out, float* __restrict__ scratch,
-                                            uint32_t* __restrict__ counters, RowSum row_sum)
-{
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, nwarps = (int)(blockDim.x >> 5);
-    for (int64_t rg = rg0 + warp; rg <= rg1; rg += nwarps) {
-        const bool whole = u_begin <= rg * nq && (rg + 1) * nq <= u_end;
-        const int64_t row = rg * kGemvGroupRows + lane;
-        const bool mine = lane < kGemvGroupRows && row < n_out;
-        const float part = lane < kGemvGroupRows ? row_sum((rg - rg0) * kGemvGroupRows + lane) : 0.f;
-        if (whole) {
-            if (mine) {
-                store_y<kOutBf16, kShard>(yo, row, part);
-                if (kShard) __threadfence_system();
-            }
-            continue;
-        }
-        const uint32_t parts = (uint32_t)(unit_owner((rg + 1) * nq - 1, U, G) - unit_owner(rg * nq, U, G) + 1);
-        if (parts == 2u) {
-            // two CTAs share the group (the usual case): one compare-and-swap on a 64-bit slot carries both the sum
-            // and the arrival.  Whoever finds the slot empty leaves (its sum, 1) there; the other gets that back from
-            // its failed swap, adds its own sum, stores y and empties the slot.  One round trip each, no fence.
-            if (mine) {
-                unsigned long long* slot = reinterpret_cast<unsigned long long*>(scratch + kPairSlotOffset) + row;
-                const unsigned long long seen = atomicCAS(slot, 0ull, (unsigned long long)__float_as_uint(part) | 1ull << 32);
-                if (seen != 0ull) {
-                    store_y<kOutBf16, kShard>(yo, row, __fadd_rn(__uint_as_float((uint32_t)seen), part));
-                    __stcg(slot, 0ull);
-                    if (kShard) __threadfence_system();
-                }
-            }
-            continue;
-        }
-        if (mine) atomicAdd(scratch + row, part);
-        __threadfence();                               // every lane's add is performed before ...
-        __syncwarp();
-        uint32_t is_last = 0u;
-        if (lane == 0) {
-            __threadfence();                           // ... lane 0 counts the arrival
-            is_last = atomicAdd(counters + rg, 1u) == parts - 1u;
-        }
-        is_last = __shfl_sync(kFullMask, is_last, 0);
-        if (is_last) {
-            __threadfence();
-            if (mine) {
-                store_y<kOutBf16, kShard>(yo, row, __ldcg(scratch + row));
-                __stcg(scratch + row, 0.f);
-                if (kShard) __threadfence_system();
-            }
-            if (lane == 0) counters[rg] = 0u;
-        }
-    }
-}
-
-// Last step of a row-sharded GEMV CTA (all threads call it, after their last store to y): counts the CTA in; the CTA
-// that completes the grid raises the epoch in every peer's flag word.  The remote stores of y are fenced at system
-// scope by the threads that made them (finish_pass) and once more, cumulatively, by the thread that counts.
-__device__ __forceinline__ void shard_arrive(const YOut& yo)
-{
-    if (yo.n_flag == 0) return;
-    __syncthreads();
-    if (threadIdx.x != 0) return;
-    __threadfence_system();
-    if (atomicAdd(yo.done, 1u) != gridDim.x - 1u) return;
-    atomicExch(yo.done, 0u);
-    __threadfence_system();
-#pragma unroll
-    for (int p = 0; p < kMaxShardPeers; ++p)
-        if (p < yo.n_flag) asm volatile("st.release.sys.global.u32 [%0], %1;" ::"l"(yo.flag[p]), "r"(yo.epoch) : "memory");
-}
-
-template <bool kBig, bool kOutBf16, bool kSg = false, bool kShard = false>
-__global__ void __launch_bounds__(kGemvThreads, 1)
-gemv_fast_kernel(FastArgs fa, const uint32_t* __restrict__ stream, const uint16_t* __restrict__ gain, SgArgs sg,
-                 int64_t n_out, int64_t k_in, int64_t bpr, const uint16_t* __restrict__ x, YOut yo,
-                 float* __restrict__ scratch, uint32_t* __restrict__ counters)
-{
-    FAST_PROLOGUE();
-    const int64_t nq = (bpr + 3) / 4;                               // units along K
-    uint32_t* xs = reinterpret_cast<uint32_t*>(staging);            // [nq * 4][12] packed bf16 pairs of x
-    float* acc = reinterpret_cast<float*>(xs + nq * 48);            // [kGemvGroupsPerPass][8]
-    stage_x(xs, x, k_in, nq * 48);
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, g = lane >> 2, t = lane & 3;
-    const int kWarps = (int)(blockDim.x >> 5);
-    const int64_t groups = (n_out + kGemvGroupRows - 1) / kGemvGroupRows;
-    const int64_t U = groups * nq, G = gridDim.x;
-    const int64_t u_begin = blockIdx.x * U / G, u_end = (blockIdx.x + 1) * U / G;
-    const int64_t rg_first = u_begin / nq, rg_last = u_begin < u_end ? (u_end - 1) / nq : rg_first - 1;   // no units: no pass
-    for (int64_t rg0 = rg_first; rg0 <= rg_last; rg0 += kGemvGroupsPerPass) {
-        const int64_t rg1 = min(rg0 + kGemvGroupsPerPass - 1, rg_last);
-        for (int i = threadIdx.x; i < kGemvGroupsPerPass * kGemvGroupRows; i += (int)blockDim.x) acc[i] = 0.f;
-        __syncthreads();
-        const int64_t p_begin = max(u_begin, rg0 * nq), p_end = min(u_end, (rg1 + 1) * nq);
-        int64_t rg = (p_begin + warp) / nq, kq = (p_begin + warp) - rg * nq;      // walked along with u: no division per unit
-        for (int64_t u = p_begin + warp; u < p_end; u += kWarps, kq += kWarps) {
-            while (kq >= nq) { kq -= nq; ++rg; }
-            const int64_t cb = kq * 4 + t;
-            const int64_t row = rg * kGemvGroupRows + g;
-            const bool in = row < n_out && cb < bpr;
-            const uint64_t b = (uint64_t)(row * bpr + cb);
-            uint32_t w[12];
-            if (kSg) block_pairs_sg(fa, T, stream, sg, b, row, in, w);
-            else block_pairs<kBig>(fa, T, stream, gain, b, in, w);
-            const uint4* xb = reinterpret_cast<const uint4*>(xs + cb * 12);
-            const uint4 x0 = xb[0], x1 = xb[1], x2 = xb[2];
-            const uint32_t xv[12] = {x0.x, x0.y, x0.z, x0.w, x1.x, x1.y, x1.z, x1.w, x2.x, x2.y, x2.z, x2.w};
-            float c[4] = {0.f, 0.f, 0.f, 0.f};
-#pragma unroll
-            for (int q = 0; q < 6; ++q)
-                mma_bf16_16816(c, w[2 * q], 0u, w[2 * q + 1], 0u, xv[2 * q], xv[2 * q + 1]);
-            if (t == 0) atomicAdd(&acc[(rg - rg0) * kGemvGroupRows + g], c[0]);
-        }
-        __syncthreads();
-        // row groups this CTA covers completely are final; the (at most two) split ones go through the scratch
-        finish_pass<kOutBf16, kShard>(yo, rg0, rg1, nq, u_begin, u_end, U, G, n_out, scratch, counters, [&](int64_t r) { return acc[r]; });
-        __syncthreads();                                   // the sums are read above: the next pass may clear them only now
-    }
-    if (kShard) shard_arrive(yo);
-}
-
-constexpr uint32_t kKindEven = 0u, kKindOdd = 1u, kKindOther = 2u, kKindNull = 3u;   // decoder form a class needs
-
-// ===========================================================================
-// Sorted layout for the fused GEMV (llvq_sort_blocks / llvq_gemv_sorted).
-// The work is cut exactly as in gemv_fast_kernel: units of 8 rows x 4 column blocks, row group major, an equal
-// contiguous range of units per CTA (for the CTA count of this device).  Inside a CTA's range the units are taken
-// in segments of up to kSortSegUnits units, and the blocks of a segment are stored sorted by the decoder form
-// their class needs (odd / even with Golay weight 8, 12, 16 / other) and its number of unranking steps (most
-// expensive first), so that the 32 lanes of a warp run the same form with the same trip count.  Each block is a
-// 64-bit entry: the stored index I unchanged in the low 48 bits, its position in the segment (unit * 32 + lane)
-// in the high 16 bits; entries that do not exist (ragged edges) or are out of range carry I = 2^48 - 1.
-// All of App. A runs in the GEMV kernel.  A warp takes 32 consecutive entries, each lane unranks its block and
-// multiplies it with its own slice of x (binary32 FMAs), and adds the partial row sum to the CTA's row sums.
-// ===========================================================================
-constexpr int kSortSegUnits = 2048;                  // 65536 blocks
-constexpr int kSortThreads = 1024;
-constexpr int kSortAccCopies = 4;                    // copies of the row sums in shared memory (a power of two)
-constexpr unsigned long long kSortIndexMask = (1ull << 48) - 1ull;
-
-// Calls f(tu0, tu1, rg0, rg1, first, last) for every segment [tu0, tu1) of CTA `cta` (of G) in order; rg0..rg1 = row
-// groups of the pass the segment belongs to (a pass covers at most kGemvGroupsPerPass row groups); first / last =
-// the segment opens / closes its pass.
-template <typename F>
-__device__ __forceinline__ void for_each_sorted_segment(int64_t U, int64_t G, int64_t nq, int64_t cta, F f, int seg_units = kSortSegUnits)
-{
-    const int64_t u_begin = cta * U / G, u_end = (cta + 1) * U / G;
-    if (u_begin >= u_end) return;
-    const int64_t rg_first = u_begin / nq, rg_last = (u_end - 1) / nq;
-    for (int64_t rg0 = rg_first; rg0 <= rg_last; rg0 += kGemvGroupsPerPass) {
-        const int64_t rg1 = min(rg0 + kGemvGroupsPerPass - 1, rg_last);
-        const int64_t p_begin = max(u_begin, rg0 * nq), p_end = min(u_end, (rg1 + 1) * nq);
-        for (int64_t tu0 = p_begin; tu0 < p_end; tu0 += seg_units)
-            f(tu0, min(tu0 + (int64_t)seg_units, p_end), rg0, rg1, tu0 == p_begin, tu0 + seg_units >= p_end);
-    }
-}
-
-__global__ void __launch_bounds__(kSortThreads, 1)
-sort_blocks_kernel(FastArgs fa, const uint32_t* __restrict__ stream, const uint16_t* __restrict__ sort_rank, int gain_bits, int64_t n_out,
-                   int64_t bpr, unsigned long long* __restrict__ out)
-{
-    FAST_PROLOGUE();
-    __shared__ uint32_t hist[1024], cursor[1024];                  // one bin per class, in sort order; bin 1023 = no block
-    const int64_t nq = (bpr + 3) / 4;
-    const int64_t groups = (n_out + kGemvGroupRows - 1) / kGemvGroupRows;
-    const int64_t U = groups * nq, G = gridDim.x;
-    for_each_sorted_segment(U, G, nq, blockIdx.x, [&](int64_t tu0, int64_t tu1, int64_t, int64_t, bool, bool) {
-        const int entries = (int)(tu1 - tu0) * 32;
-        hist[threadIdx.x] = 0; cursor[threadIdx.x] = 0;
-        __syncthreads();
-        // key and field of entry i of the segment; count = the first pass (out-of-range fields are counted once)
-        auto entry_of = [&](int i, bool count, unsigned long long& field) {
-            const int64_t u = tu0 + (i >> 5);
-            const int lane = i & 31;
-            const int64_t rg = u / nq, kq = u - rg * nq;
-            const int64_t row = rg * kGemvGroupRows + (lane >> 2), cb = kq * 4 + (lane & 3);
-            field = kSortIndexMask;
-            if (row >= n_out || cb >= bpr) return 1023u;
-            const uint64_t f = load_field(stream, (uint64_t)(row * bpr + cb), (int)fa.L.W + gain_bits);   // shape index | gain index << W
-            const uint64_t I = f & ((1ull << fa.L.W) - 1ull);
-            if (I >= fa.n_points) { if (count) atomicAdd(fa.bad_index, 1ull); return 1023u; }
-            uint64_t local;
-            field = f;
-            return (uint32_t)__ldg(sort_rank + fast_find_class(T, I, local));
-        };
-        for (int i = threadIdx.x; i < entries; i += kSortThreads) {
-            unsigned long long field;
-            atomicAdd(&hist[entry_of(i, true, field)], 1u);
-        }
-        __syncthreads();
-        if (threadIdx.x == 0) {
-            uint32_t run = 0;
-            for (int k = 0; k < 1024; ++k) { const uint32_t c = hist[k]; hist[k] = run; run += c; }
-        }
-        __syncthreads();
-        // the entries are visited column-block major (all row groups of a column unit, then the next unit): the blocks
-        // of a bin then come out roughly ordered by column block, and the 32 lanes of a GEMV warp read few different
-        // slices of x
-        const int64_t rg_a = tu0 / nq, nrg = (tu1 - 1) / nq - rg_a + 1;
-        for (int64_t e = threadIdx.x; e < nq * nrg * 32; e += kSortThreads) {
-            const int64_t kq = e / (nrg * 32), rem = e - kq * (nrg * 32);
-            const int64_t u = (rg_a + (rem >> 5)) * nq + kq;
-            if (u < tu0 || u >= tu1) continue;
-            const int i = (int)(u - tu0) * 32 + (int)(rem & 31);
-            unsigned long long field;
-            const uint32_t key = entry_of(i, false, field);
-            const uint32_t slot = hist[key] + atomicAdd(&cursor[key], 1u);
-            out[tu0 * 32 + slot] = field | (unsigned long long)i << 48;
-        }
-        __syncthreads();
-    });
-}
-
-// App. A steps 2-4 for one entry of a sorted layout: class lookup, then the unranker form the class needs.  The
-// lanes of a warp call this together; after sorting they almost always share the form (and the class).
-__device__ __forceinline__ void decode_known_class(const FastSmem& T, uint32_t cls, uint64_t local, bool valid, Decoded& r)
-{
-    const uint32_t h = T.desc[cls * kFastDescStride];
-    const uint32_t w8 = h & 0xffu;
-    const uint32_t kind = !valid ? kKindNull : ((h & (1u << 16)) ? kKindOdd : ((w8 == 8u || w8 == 12u || w8 == 16u) ? kKindEven : kKindOther));
-    Decoded d;
-    r.p0 = r.p1 = r.p2 = r.neg = r.vals_lo = r.vals_hi = 0u;
-    if (__any_sync(kFullMask, kind == kKindOdd)) {
-        const bool mine = kind == kKindOdd;
-        fast_decode_local<1>(T, mine ? cls : 0u, mine ? local : 0ull, mine, kFullMask, d);
-        if (mine) r = d;
-    }
-    if (__any_sync(kFullMask, kind == kKindEven)) {
-        const bool mine = kind == kKindEven;
-        fast_decode_local<0>(T, mine ? cls : 0u, mine ? local : 0ull, mine, kFullMask, d);
-        if (mine) r = d;
-    }
-    if (__any_sync(kFullMask, kind == kKindOther)) {
-        const bool mine = kind == kKindOther;
-        fast_decode_local<-1>(T, mine ? cls : 0u, mine ? local : 0ull, mine, kFullMask, d);
-        if (mine) r = d;
-    }
-}
-
-__device__ __forceinline__ uint32_t decode_sorted_entry(const FastArgs& fa, const FastSmem& T, uint64_t I, bool valid, Decoded& r)
-{
-    uint64_t local = 0;
-    const uint32_t cls = valid ? fast_find_class(T, I, local) : 0u;
-    decode_known_class(T, cls, local, valid, r);
-    return cls;
-}
-
-template <bool kOutBf16, bool kSg = false, bool kShard = false>
-__global__ void __launch_bounds__(kSortThreads, 1)
-gemv_sorted_kernel(FastArgs fa, const unsigned long long* __restrict__ sorted, const uint16_t* __restrict__ gain, SgArgs sg,
-                   int64_t n_out, int64_t k_in, int64_t bpr, uint32_t nq_magic, const uint16_t* __restrict__ x, YOut yo,
-                   float* __restrict__ scratch, uint32_t* __restrict__ counters)
-{
-    FAST_PROLOGUE();
-    const int64_t nq = (bpr + 3) / 4;
-    uint32_t* xs = reinterpret_cast<uint32_t*>(staging);            // [nq * 4][12] packed bf16 pairs of x
-    float* acc = reinterpret_cast<float*>(xs + nq * 48);            // [kSortAccCopies][kGemvGroupsPerPass][8]: warps spread their adds over the copies
-    uint32_t* last_flag = reinterpret_cast<uint32_t*>(acc + kSortAccCopies * kGemvGroupsPerPass * kGemvGroupRows);
-    uint32_t* next_chunk = last_flag + 1;
-    stage_x(xs, x, k_in, nq * 48);
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const uint32_t kWarps = blockDim.x >> 5;
-    const int64_t groups = (n_out + kGemvGroupRows - 1) / kGemvGroupRows;
-    const int64_t U = groups * nq, G = gridDim.x;
-    const uint32_t nq32 = (uint32_t)nq;
-
-    for_each_sorted_segment(U, G, nq, blockIdx.x, [&](int64_t tu0, int64_t tu1, int64_t rg0, int64_t rg1, bool first, bool last) {
-        if (first)
-            for (int i = threadIdx.x; i < kSortAccCopies * kGemvGroupsPerPass * kGemvGroupRows; i += (int)blockDim.x) acc[i] = 0.f;
-        if (threadIdx.x == 0) *next_chunk = kWarps;
-        __syncthreads();
-        const int64_t rg_a = tu0 / nq;
-        const uint32_t kq_a = (uint32_t)(tu0 - rg_a * nq), rg_off = (uint32_t)(rg_a - rg0);
-        const uint32_t nchunks = (uint32_t)(tu1 - tu0);
-        const unsigned long long* seg = sorted + tu0 * 32 + lane;
-        uint32_t ch = (uint32_t)warp;
-        unsigned long long e = ch < nchunks ? __ldg(seg + (uint64_t)ch * 32) : 0ull;
-        while (ch < nchunks) {
-            // chunks are handed out dynamically (their cost depends on the form); the next entry is fetched ahead
-            uint32_t nxt = 0;
-            if (lane == 0) nxt = atomicAdd(next_chunk, 1u);
-            nxt = __shfl_sync(kFullMask, nxt, 0);
-            const unsigned long long e_next = nxt < nchunks ? __ldg(seg + (uint64_t)nxt * 32) : 0ull;
-            const uint64_t field = e & kSortIndexMask;
-            const uint64_t I = kSg ? field & ((1ull << fa.L.W) - 1ull) : field;     // shape-gain form: gain index above the shape index
-            const uint32_t pos = (uint32_t)(e >> 48);
-            const bool valid = field != kSortIndexMask && I < fa.n_points;
-            // where the block sits: unit = pos / 32 of the segment, (row, column block) = lane of the unit
-            const uint32_t v = kq_a + (pos >> 5);
-            uint32_t q = __umulhi(v, nq_magic), kq = v - q * nq32;
-            if (kq >= nq32) { kq -= nq32; ++q; }
-            const uint32_t rloc = (rg_off + q) * kGemvGroupRows + ((pos >> 2) & 7u);      // row inside the pass
-            const uint32_t cb = kq * 4u + (pos & 3u);
-            float gn = 0.f;
-            if (!kSg && valid) gn = gain_to_float(__ldg(gain + ((int64_t)rg0 * kGemvGroupRows + rloc) * bpr + cb));
-            Decoded r;
-            const uint32_t cls = decode_sorted_entry(fa, T, I, valid, r);
-            if (kSg && valid) {
-                const float scale = sg.row_scale ? __ldg(sg.row_scale + (int64_t)rg0 * kGemvGroupRows + rloc) : 1.f;
-                gn = __fmul_rn(__fmul_rn(scale, __ldg(sg.codebook + (uint32_t)(field >> fa.L.W))),
-                               __uint_as_float(T.desc[cls * kFastDescStride + kFastDescRnorm]));
-            }
-            uint32_t w[12];
-            expand_bf16(r, gn, w);
-            const uint4* xb = reinterpret_cast<const uint4*>(xs + cb * 12u);
-            const uint4 x0 = xb[0], x1 = xb[1], x2 = xb[2];
-            const uint32_t xv[12] = {x0.x, x0.y, x0.z, x0.w, x1.x, x1.y, x1.z, x1.w, x2.x, x2.y, x2.z, x2.w};
-            float s0 = 0.f, s1 = 0.f;
-#pragma unroll
-            for (int j = 0; j < 12; ++j) {                        // bf16 x bf16 products are exact in binary32
-                s0 = fmaf(__uint_as_float(w[j] << 16), __uint_as_float(xv[j] << 16), s0);
-                s1 = fmaf(__uint_as_float(w[j] & 0xffff0000u), __uint_as_float(xv[j] & 0xffff0000u), s1);
-            }
-            if (valid) atomicAdd(&acc[(warp & (kSortAccCopies - 1)) * (kGemvGroupsPerPass * kGemvGroupRows) + rloc], s0 + s1);
-            ch = nxt; e = e_next;
-        }
-        __syncthreads();
-        if (!last) return;
-        // end of the pass: row groups this CTA covers completely are final; the split ones go through the scratch
-        auto row_sum = [&](int64_t r) {
-            float v = 0.f;
-#pragma unroll
-            for (int c = 0; c < kSortAccCopies; ++c) v += acc[c * (kGemvGroupsPerPass * kGemvGroupRows) + r];
-            return v;
-        };
-        const int64_t ub = blockIdx.x * U / G, ue = (blockIdx.x + 1) * U / G;     // recomputed here: nothing 64-bit lives across the main loop
-        finish_pass<kOutBf16, kShard>(yo, rg0, rg1, nq, ub, ue, U, G, n_out, scratch, counters, row_sum);
-        __syncthreads();                                   // the sums are read above: the next pass may clear them only now
-    });
-    if (kShard) shard_arrive(yo);
-}
-
-// ===========================================================================
-// Fused GEMV on the stored stream with the blocks binned inside the kernel: the work split of gemv_fast_kernel, but a
-// CTA first looks up the class of every block of a segment of up to kBinSegUnits units (S1-S2), orders the
-// (class-local index, class, position) triples by the sorted layout's key with a counting sort in shared memory,
-// and then proceeds like gemv_sorted_kernel on those entries (S3-S8): a warp takes 32 consecutive entries, runs
-// the one unranker form they need and each lane forms its own dot product.
-// ===========================================================================
-constexpr int kBinSegUnits = 256;                    // at most 8192 blocks per segment (halved while shared memory is short)
-constexpr int kBinPerThread = kBinSegUnits * 32 / kSortThreads;   // 8
-
-template <bool kOutBf16, bool kSg = false, bool kShard = false>
-__global__ void __launch_bounds__(kSortThreads, 1)
-gemv_bin_kernel(FastArgs fa, const uint32_t* __restrict__ stream, const uint16_t* __restrict__ sort_rank, const uint16_t* __restrict__ gain, SgArgs sg,
-                int64_t n_out, int64_t k_in, int64_t bpr, uint32_t nq_magic, int seg_units, const uint16_t* __restrict__ x, YOut yo,
-                float* __restrict__ scratch, uint32_t* __restrict__ counters)
-{
-    FAST_PROLOGUE();
-    const int64_t nq = (bpr + 3) / 4;
-    uint32_t* xs = reinterpret_cast<uint32_t*>(staging);            // [nq * 4][12] packed bf16 pairs of x
-    float* acc = reinterpret_cast<float*>(xs + nq * 48);            // [kSortAccCopies][kGemvGroupsPerPass][8]
-    uint32_t* last_flag = reinterpret_cast<uint32_t*>(acc + kSortAccCopies * kGemvGroupsPerPass * kGemvGroupRows);
-    uint32_t* next_chunk = last_flag + 1;
-    uint32_t* hist = last_flag + 4;                                  // [1024] bins in sort order; later their first slots
-    uint32_t* cursor = hist + 1024;                                  // [1024]
-    unsigned long long* ent = reinterpret_cast<unsigned long long*>(cursor + 1024);   // [seg_units * 32] class-local index | position << 48
-    uint16_t* ent_cls = reinterpret_cast<uint16_t*>(ent + seg_units * 32);            // [seg_units * 32] class (| gain index << 10), 0xffff = no block
-    stage_x(xs, x, k_in, nq * 48);
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const uint32_t kWarps = blockDim.x >> 5;
-    const int64_t groups = (n_out + kGemvGroupRows - 1) / kGemvGroupRows;
-    const int64_t U = groups * nq, G = gridDim.x;
-    const int64_t u_begin = blockIdx.x * U / G, u_end = (blockIdx.x + 1) * U / G;
-    const uint32_t nq32 = (uint32_t)nq;
-    if (u_begin < u_end) {
-        // the rows of the row groups this CTA touches are one contiguous span of the index stream and of the gains:
-        // request it from DRAM now, the binning phases then read it from L2
-        const uint64_t b_first = (uint64_t)(u_begin / nq) * kGemvGroupRows * (uint64_t)bpr;
-        const uint64_t b_last = (uint64_t)min(((u_end - 1) / nq + 1) * kGemvGroupRows, n_out) * (uint64_t)bpr;
-        const uint64_t wf = (uint64_t)fa.L.W + (kSg ? (uint64_t)sg.bits : 0ull);
-        prefetch_span_l2(stream, b_first * wf / 8, (b_last * wf + 7) / 8);
-        if (!kSg) prefetch_span_l2(gain, b_first * 2, b_last * 2);
-    }
-    for_each_sorted_segment(U, G, nq, blockIdx.x, [&](int64_t tu0, int64_t tu1, int64_t rg0, int64_t rg1, bool first, bool last) {
-        if (first)
-            for (int i = threadIdx.x; i < kSortAccCopies * kGemvGroupsPerPass * kGemvGroupRows; i += (int)blockDim.x) acc[i] = 0.f;
-        hist[threadIdx.x] = 0; cursor[threadIdx.x] = 0;
-        if (threadIdx.x == 0) *next_chunk = kWarps;
-        __syncthreads();
-        const int64_t rg_a = tu0 / nq;
-        const uint32_t kq_a = (uint32_t)(tu0 - rg_a * nq), rg_off = (uint32_t)(rg_a - rg0);
-        const int entries = (int)(tu1 - tu0) * 32;
-        // ---- S1-S2 for the whole segment and the histogram of the sort keys
-        unsigned long long mine_ent[kBinPerThread];
-        uint32_t mine_key[kBinPerThread];
-#pragma unroll
-        for (int q = 0; q < kBinPerThread; ++q) {
-            const int i = (int)threadIdx.x + q * kSortThreads;
-            mine_key[q] = 0xffffffffu; mine_ent[q] = 0ull;
-            if (i < entries) {
-                const uint32_t pos = (uint32_t)i;
-                const uint32_t v = kq_a + (pos >> 5);
-                uint32_t qd = __umulhi(v, nq_magic), kq = v - qd * nq32;
-                if (kq >= nq32) { kq -= nq32; ++qd; }
-                const int64_t row = (rg_a + qd) * kGemvGroupRows + ((pos >> 2) & 7u), cb = (int64_t)kq * 4 + (pos & 3u);
-                uint32_t key = 1023u, cls = 0xffffu;
-                uint64_t local = 0;
-                if (row < n_out && cb < bpr) {
-                    const uint64_t f = load_field(stream, (uint64_t)(row * bpr + cb), (int)fa.L.W + (kSg ? sg.bits : 0));
-                    const uint64_t I = kSg ? f & ((1ull << fa.L.W) - 1ull) : f;
-                    if (I < fa.n_points) {
-                        cls = fast_find_class(T, I, local);
-                        key = __ldg(sort_rank + cls);
-                        if (kSg) cls |= (uint32_t)(f >> fa.L.W) << 10;           // the gain index rides with the class
-                    } else atomicAdd(fa.bad_index, 1ull);
-                }
-                mine_key[q] = key | cls << 16;
-                mine_ent[q] = local | (unsigned long long)pos << 48;
-                atomicAdd(&hist[key], 1u);
-            }
-        }
-        __syncthreads();
-        // exclusive prefix sum of the 1024 bins: one bin per thread
-        {
-            const uint32_t c = hist[threadIdx.x];
-            uint32_t incl = c;
-#pragma unroll
-            for (int o = 1; o < 32; o <<= 1) { const uint32_t t = __shfl_up_sync(kFullMask, incl, o); if (lane >= o) incl += t; }
-            if (lane == 31) cursor[warp] = incl;                       // warp totals, parked in the cursor array for a moment
-            __syncthreads();
-            uint32_t before = 0;
-            for (int w2 = 0; w2 < warp; ++w2) before += cursor[w2];
-            __syncthreads();
-            hist[threadIdx.x] = before + incl - c;
-            cursor[threadIdx.x] = 0;
-        }
-        __syncthreads();
-#pragma unroll
-        for (int q = 0; q < kBinPerThread; ++q) {
-            if (mine_key[q] != 0xffffffffu) {
-                const uint32_t key = mine_key[q] & 0xffffu;
-                const uint32_t slot = hist[key] + atomicAdd(&cursor[key], 1u);
-                ent[slot] = mine_ent[q];
-                ent_cls[slot] = (uint16_t)(mine_key[q] >> 16);
-            }
-        }
-        __syncthreads();
-        // ---- S3-S8 on the ordered entries
-        const uint32_t nchunks = (uint32_t)(tu1 - tu0);
-        const uint16_t* gain_pass = gain + rg0 * kGemvGroupRows * bpr;
-        for (uint32_t ch = (uint32_t)warp; ch < nchunks;) {
-            uint32_t nxt = 0;
-            if (lane == 0) nxt = atomicAdd(next_chunk, 1u);
-            nxt = __shfl_sync(kFullMask, nxt, 0);
-            const unsigned long long e = ent[ch * 32 + lane];
-            const uint32_t cls16 = ent_cls[ch * 32 + lane];
-            const bool valid = cls16 != 0xffffu;
-            const uint32_t pos = (uint32_t)(e >> 48);
-            const uint32_t v = kq_a + (pos >> 5);
-            uint32_t q = __umulhi(v, nq_magic), kq = v - q * nq32;
-            if (kq >= nq32) { kq -= nq32; ++q; }
-            const uint32_t rloc = (rg_off + q) * kGemvGroupRows + ((pos >> 2) & 7u);
-            const uint32_t cb = kq * 4u + (pos & 3u);
-            const uint32_t cls = valid ? (kSg ? cls16 & 1023u : cls16) : 0u;
-            float gn = 0.f;
-            if (valid) {
-                if (kSg) {
-                    const float scale = sg.row_scale ? __ldg(sg.row_scale + (int64_t)rg0 * kGemvGroupRows + rloc) : 1.f;
-                    gn = __fmul_rn(__fmul_rn(scale, __ldg(sg.codebook + (cls16 >> 10))), __uint_as_float(T.desc[cls * kFastDescStride + kFastDescRnorm]));
-                } else {
-                    gn = gain_to_float(__ldg(gain_pass + (int64_t)rloc * bpr + cb));
-                }
-            }
-            Decoded r;
-            decode_known_class(T, cls, e & ((1ull << 48) - 1ull), valid, r);
-            uint32_t w[12];
-            expand_bf16(r, gn, w);
-            const uint4* xb = reinterpret_cast<const uint4*>(xs + cb * 12u);
-            const uint4 x0 = xb[0], x1 = xb[1], x2 = xb[2];
-            const uint32_t xv[12] = {x0.x, x0.y, x0.z, x0.w, x1.x, x1.y, x1.z, x1.w, x2.x, x2.y, x2.z, x2.w};
-            float s0 = 0.f, s1 = 0.f;
-#pragma unroll
-            for (int j = 0; j < 12; ++j) {
-                s0 = fmaf(__uint_as_float(w[j] << 16), __uint_as_float(xv[j] << 16), s0);
-                s1 = fmaf(__uint_as_float(w[j] & 0xffff0000u), __uint_as_float(xv[j] & 0xffff0000u), s1);
-            }
-            if (valid) atomicAdd(&acc[(warp & (kSortAccCopies - 1)) * (kGemvGroupsPerPass * kGemvGroupRows) + rloc], s0 + s1);
-            ch = nxt;
-        }
-        __syncthreads();
-        if (!last) return;
-        auto row_sum = [&](int64_t r) {
-            float v = 0.f;
-#pragma unroll
-            for (int c = 0; c < kSortAccCopies; ++c) v += acc[c * (kGemvGroupsPerPass * kGemvGroupRows) + r];
-            return v;
-        };
-        const int64_t ub = blockIdx.x * U / G, ue = (blockIdx.x + 1) * U / G;     // recomputed here: nothing 64-bit lives across the main loop
-        finish_pass<kOutBf16, kShard>(yo, rg0, rg1, nq, ub, ue, U, G, n_out, scratch, counters, row_sum);
-        __syncthreads();
-    }, seg_units);
-    if (kShard) shard_arrive(yo);
-}
-
-// ===========================================================================
-// llvq_gemm_small_batch: Y[b][i] = sum_k X[b][k] W[i][k] on the tensor cores.
-// A work item is a tile of 128 output rows x a range of K stages (96 columns = 4 blocks of 24 per row).
-// Per stage every thread of a 512-thread group dequantizes one block into the group's shared-memory A tile
-// (bf16, K-major core-matrix layout), the matching slice of X goes into its B tile, and one thread issues
-// six tcgen05 MMAs (M = 128, N = padded batch, K = 16) into the group's accumulator in tensor memory.
-// The two groups of a CTA take alternate stages, so two stages are in flight.
-// Split-K partial sums are added into a zero-initialised binary32 scratch [npad][n_out]; the last item
-// of a row tile converts it to bf16 and clears it again.
-// ===========================================================================
-constexpr int kGemmThreads = 1024;
-constexpr int kGemmGroupThreads = 512;
-constexpr int kGemmRows = 128;
-constexpr int kStageBlocks = 4;                       // column blocks per stage
-constexpr int kStageK = kStageBlocks * 24;            // 96
-constexpr int kMaxScratchRows = 65536;
-constexpr int kCounterWords = 64 * kMaxScratchRows / 8;      // the word after them counts the CTAs of a row-sharded GEMV that have finished
-constexpr uint32_t kTmemCols = 128;
-
-struct GemmArgs {
-    int64_t n_out, k_in, bpr;
-    int batch, npad;
-    int nstages, split;
-    const uint16_t* x;
-    uint16_t* y;               // Y [batch][y_ld] bf16, at the first row of this launch's rows
-    int64_t y_ld;
-    const YOut* shard;         // row-sharded launch: the peers' copies and flags (device memory), else null
-    float* scratch;            // [npad][scratch_ld] binary32, all zero on entry and on exit
-    int64_t scratch_ld;        // row tiles * 128
-    uint32_t* counters;        // [row tiles], zero on entry and on exit
-};
-
-__global__ void put_shard_kernel(YOut yo, YOut* dst)
-{
-    if (threadIdx.x == 0) *dst = yo;
-}
-
-// One element of Y; a row-sharded launch also writes it into the peers' copies (their description sits in device
-// memory so that the ordinary launch's parameters stay as small as they were).
-template <bool kShard>
-__device__ __forceinline__ void gemm_store(const GemmArgs& ga, int n, int64_t orow, float v)
-{
-    const __nv_bfloat16 h = __float2bfloat16_rn(v);
-    const int64_t at = (int64_t)n * ga.y_ld + orow;
-    reinterpret_cast<__nv_bfloat16*>(ga.y)[at] = h;
-    if (kShard) {
-        const int np = ga.shard->n_peer;
-        for (int p = 0; p < np; ++p) reinterpret_cast<__nv_bfloat16*>(ga.shard->peer[p])[at] = h;
-    }
-}
-
-__device__ __forceinline__ void group_barrier(int group)
-{
-    asm volatile("bar.sync %0, %1;" ::"r"(1 + group), "n"(kGemmGroupThreads) : "memory");
-}
-
-template <bool kBig, bool kSg = false, bool kShard = false>
-__global__ void __launch_bounds__(kGemmThreads, 1)
-gemm_kernel(FastArgs fa, const uint32_t* __restrict__ stream, const uint16_t* __restrict__ gain, SgArgs sg, GemmArgs ga)
-{
-    extern __shared__ __align__(128) uint8_t smem[];
-    const uint32_t img_bytes = fa.L.total;
-    uint64_t* bar_img = reinterpret_cast<uint64_t*>(smem + img_bytes);
-    uint64_t* bar_free = bar_img + 1;                                     // [2]: the MMAs reading group h's buffers are done
-    uint64_t* bar_done = bar_img + 3;                                     // [2]: group h's accumulator of this item is complete
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bar_img + 5);
-    uint32_t* last_flag = tmem_slot + 1;
-    const uint32_t a_off = (img_bytes + 64 + 1023) & ~1023u;
-    uint8_t* a_buf = smem + a_off;                                        // [2 groups] x 24576
-    uint8_t* b_buf = a_buf + 2 * kGemmRows * kStageK * 2;                  // [2 groups] x npad * 192
-    const uint32_t b_stage = (uint32_t)ga.npad * kStageK * 2;
-
-    pdl_launch_dependents();
-    if (!fast_load_image(smem, fa.image, fa.L.total, bar_img, fa.flags)) return;
-    pdl_wait();
-    const FastSmem T = fast_view(smem, fa.L);
-    // Two groups of 512 threads fill alternate stages, each into its own buffers and its own accumulator
-    // (TMEM columns [64 h, 64 h + npad)); the epilogue adds the two accumulators.
-    const int group = threadIdx.x / kGemmGroupThreads, gtid = threadIdx.x % kGemmGroupThreads;
-    const int gwarp = gtid >> 5, lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    if (threadIdx.x == 0) {
-        mbar_init(&bar_free[0], 1); mbar_init(&bar_free[1], 1); mbar_init(&bar_done[0], 1); mbar_init(&bar_done[1], 1);
-        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-    }
-    if (warp == 0) tmem_alloc(tmem_slot, kTmemCols);
-    tc_fence_before();
-    __syncthreads();
-    tc_fence_after();
-    const uint32_t tmem = *tmem_slot;
-    const uint32_t idesc = instr_desc_bf16_m128((uint32_t)ga.npad);
-    uint8_t* const a_mine = a_buf + group * (kGemmRows * kStageK * 2);
-    uint8_t* const b_mine = b_buf + group * b_stage;
-
-    const int64_t row_tiles = (ga.n_out + kGemmRows - 1) / kGemmRows;
-    const int64_t items = row_tiles * ga.split;
-    uint32_t uses = 0;                                  // stages this group has filled so far
-    uint32_t done[2] = {0, 0};                          // completed accumulations per group
-    bool timeout = false;
-    for (int64_t item = blockIdx.x; item < items; item += gridDim.x) {
-        const int64_t rt = item / ga.split;
-        const int f = (int)(item % ga.split);
-        const int s_begin = (int)((int64_t)f * ga.nstages / ga.split), s_end = (int)((int64_t)(f + 1) * ga.nstages / ga.split);
-        const int64_t row = rt * kGemmRows + gwarp * 8 + (lane & 7);
-        for (int s = s_begin + group; s < s_end; s += 2, ++uses) {
-            // ---- A: dequantize one block of 24 weights
-            const int64_t cb = (int64_t)s * kStageBlocks + (lane >> 3);
-            const bool in = row < ga.n_out && cb < ga.bpr;
-            const uint64_t b = in ? (uint64_t)(row * ga.bpr + cb) : 0ull;
-            uint32_t w[12];
-            if (kSg) block_pairs_sg(fa, T, stream, sg, b, row, in, w);
-            else block_pairs<kBig>(fa, T, stream, gain, b, in, w);
-            // the MMAs of this group's previous stage read its buffers: wait for them only now, with the block already unranked
-            if (uses > 0 && !mbar_wait(&bar_free[group], (uses - 1u) & 1u)) timeout = true;
-            uint8_t* a_dst = a_mine + gwarp * 128 + (lane & 7) * 16;
-#pragma unroll
-            for (int j = 0; j < 3; ++j)
-                *reinterpret_cast<uint4*>(a_dst + (3 * (lane >> 3) + j) * 2048) = make_uint4(w[4 * j], w[4 * j + 1], w[4 * j + 2], w[4 * j + 3]);
-            // ---- B: the slice of X, 16-byte chunks (8 values along K)
-            for (int i = gtid; i < ga.npad * (kStageK / 8); i += kGemmGroupThreads) {
-                const int kc = i / ga.npad, n = i % ga.npad;
-                const int64_t k = (int64_t)s * kStageK + kc * 8;
-                uint4 v = make_uint4(0, 0, 0, 0);
-                if (n < ga.batch && k < ga.k_in) v = __ldg(reinterpret_cast<const uint4*>(ga.x + (int64_t)n * ga.k_in + k));
-                *reinterpret_cast<uint4*>(b_mine + (uint32_t)kc * ga.npad * 16 + n * 16) = v;
-            }
-            fence_async_smem();
-            group_barrier(group);
-            if (gtid == 0) {
-                tc_fence_after();
-                const uint32_t a_addr = smem_u32(a_mine), b_addr = smem_u32(b_mine);
-#pragma unroll
-                for (int j = 0; j < kStageK / 16; ++j)
-                    umma_bf16(tmem + 64u * group, smem_desc(a_addr + j * 4096, 2048, 128),
-                              smem_desc(b_addr + j * 2 * ga.npad * 16, ga.npad * 16, 128), idesc, (s > s_begin + group || j > 0) ? 1u : 0u);
-                umma_commit(&bar_free[group]);
-                if (s + 2 >= s_end) umma_commit(&bar_done[group]);
-            }
-        }
-        // ---- epilogue: accumulators -> scratch (split-K) or Y
-        const bool has0 = s_end > s_begin, has1 = s_end > s_begin + 1;
-        if (warp < 4) {
-            if (has0 && !mbar_wait(&bar_done[0], done[0] & 1u)) timeout = true;
-            if (has1 && !mbar_wait(&bar_done[1], done[1] & 1u)) timeout = true;
-            tc_fence_after();
-            const int64_t orow = rt * kGemmRows + warp * 32 + lane;
-            for (int c0 = 0; c0 < ga.npad && has0; c0 += 16) {
-                float v[16], v1[16];
-                tmem_ld16(tmem + ((uint32_t)(warp * 32) << 16) + (uint32_t)c0, v);
-                if (has1) {
-                    tmem_ld16(tmem + ((uint32_t)(warp * 32) << 16) + 64u + (uint32_t)c0, v1);
-#pragma unroll
-                    for (int i = 0; i < 16; ++i) v[i] += v1[i];
-                }
-                if (orow < ga.n_out) {
-#pragma unroll
-                    for (int i = 0; i < 16; ++i) {
-                        const int n = c0 + i;
-                        if (n < ga.batch) {
-                            if (ga.split == 1) gemm_store<kShard>(ga, n, orow, v[i]);
-                            else atomicAdd(ga.scratch + (int64_t)n * ga.scratch_ld + orow, v[i]);
-                        }
-                    }
-                }
-            }
-            tc_fence_before();
-        }
-        done[0] += has0; done[1] += has1;
-        if (ga.split > 1) {
-            __threadfence();
-            __syncthreads();
-            if (threadIdx.x == 0) *last_flag = (atomicAdd(ga.counters + rt, 1u) == (uint32_t)ga.split - 1u);
-            __syncthreads();
-            if (*last_flag) {
-                __threadfence();
-                for (int i = threadIdx.x; i < kGemmRows * ga.batch; i += kGemmThreads) {
-                    const int n = i / kGemmRows;
-                    const int64_t orow = rt * kGemmRows + (i % kGemmRows);
-                    if (orow < ga.n_out) {
-                        float* sp = ga.scratch + (int64_t)n * ga.scratch_ld + orow;
-                        gemm_store<kShard>(ga, n, orow, __ldcg(sp));
-                        __stcg(sp, 0.f);
-                    }
-                }
-                if (threadIdx.x == 0) ga.counters[rt] = 0u;
-            }
-        }
-        __syncthreads();
-    }
-    if (timeout) atomicOr(fa.flags, 1u);
-    if (kShard) {
-        __threadfence_system();                           // this thread's stores to the peers' copies, before the CTA counts itself in
-        shard_arrive(*ga.shard);
-    }
-    __syncthreads();
-    if (warp == 0) tmem_dealloc(tmem, kTmemCols);
-}
-
-// ===========================================================================
-// Sorted layout for the small-batch GEMM (llvq_sort_blocks_gemm / llvq_gemm_small_batch_sorted).
-// A domain is 128 rows x 8 column blocks (1024 blocks, two 96-column MMA stages); the stream holds the domains
-// row tile major, each domain's blocks ordered like the GEMV's sorted layout (decoder form, unranking steps,
-// class), one 64-bit entry per block: the stored index unchanged (48 bits) + position in the domain (row * 8 +
-// column block, 10 bits, stored in the high 16).  The kernel runs the whole CTA on one accumulator: per
-// iteration it unranks one domain (padded batch > 32) or two (warp w takes the w-th chunk of the first and the
-// (31-w)-th of the second: both are ordered from expensive to cheap, so the pairs balance), writing the bf16
-// weights straight to their place in the K-major A tiles, then one thread issues the tcgen05 MMAs of those stages.
-// ===========================================================================
-constexpr int kDomBlocks = 8;                          // column blocks per domain
-constexpr int kDomEntries = kGemmRows * kDomBlocks;    // 1024
-constexpr int kDomStages = 2;                          // 96-column MMA stages per domain
-
-__global__ void __launch_bounds__(kDomEntries, 1)
-sort_blocks_gemm_kernel(FastArgs fa, const uint32_t* __restrict__ stream, const uint16_t* __restrict__ sort_rank, int gain_bits, int64_t n_out,
-                        int64_t bpr, int64_t ndomains, unsigned long long* __restrict__ out)
-{
-    FAST_PROLOGUE();
-    __shared__ uint32_t hist[1024], cursor[1024];
-    const int64_t nd = (bpr + kDomBlocks - 1) / kDomBlocks;
-    for (int64_t dom = blockIdx.x; dom < ndomains; dom += gridDim.x) {
-        hist[threadIdx.x] = 0; cursor[threadIdx.x] = 0;
-        __syncthreads();
-        const int64_t rt = dom / nd, d = dom - rt * nd;
-        const int i = threadIdx.x;
-        const int64_t row = rt * kGemmRows + (i >> 3), cb = d * kDomBlocks + (i & 7);
-        unsigned long long field = kSortIndexMask;
-        uint32_t key = 1023u;
-        if (row < n_out && cb < bpr) {
-            const uint64_t f = load_field(stream, (uint64_t)(row * bpr + cb), (int)fa.L.W + gain_bits);   // shape index | gain index << W
-            const uint64_t I = f & ((1ull << fa.L.W) - 1ull);
-            if (I < fa.n_points) {
-                uint64_t local;
-                field = f;
-                key = __ldg(sort_rank + fast_find_class(T, I, local));
-            } else {
-                atomicAdd(fa.bad_index, 1ull);
-            }
-        }
-        atomicAdd(&hist[key], 1u);
-        __syncthreads();
-        if (threadIdx.x == 0) {
-            uint32_t run = 0;
-            for (int k = 0; k < 1024; ++k) { const uint32_t c = hist[k]; hist[k] = run; run += c; }
-        }
-        __syncthreads();
-        const uint32_t slot = hist[key] + atomicAdd(&cursor[key], 1u);
-        out[dom * kDomEntries + slot] = field | (unsigned long long)i << 48;
-        __syncthreads();
-    }
-}
-
-// The same layout for codes whose class tables live in global memory (72-bit indices): 128-bit entries, x = the low 64
-// bits of the stored index, y = its bits 64.. (8 bits) | class << 8 (24 bits) | position in the domain << 32 (10 bits);
-// bit 63 of y marks "no block" (ragged edge or index out of range).  The class rides along so that the GEMM kernel does
-// not search for it again; the blocks of a domain are ordered by unranking steps (most first), then by class, so that
-// the lanes of a warp run the same trip counts and read neighbouring class descriptors.
-constexpr unsigned long long kBigNoBlock = 1ull << 63;
-
-__global__ void __launch_bounds__(kDomEntries, 1)
-sort_blocks_gemm_big_kernel(FastArgs fa, const uint32_t* __restrict__ stream, int64_t n_out, int64_t bpr, int64_t ndomains,
-                            ulonglong2* __restrict__ out)
-{
-    __shared__ uint32_t keys[kDomEntries];
-    __shared__ unsigned long long ex[kDomEntries], ey[kDomEntries];
-    const int64_t nd = (bpr + kDomBlocks - 1) / kDomBlocks;
-    const int i = threadIdx.x;
-    for (int64_t dom = blockIdx.x; dom < ndomains; dom += gridDim.x) {
-        const int64_t rt = dom / nd, d = dom - rt * nd;
-        const int64_t row = rt * kGemmRows + (i >> 3), cb = d * kDomBlocks + (i & 7);
-        unsigned long long x = 0ull, y = kBigNoBlock | (unsigned long long)i << 32;
-        uint32_t key = 0x7ffffc00u | (uint32_t)i;                   // no block: after everything else
-        if (row < n_out && cb < bpr) {
-            uint64_t lo, hi;
-            load_index(stream, (uint64_t)(row * bpr + cb), fa.dc.W, lo, hi);
-            if (hi < fa.dc.n_hi || (hi == fa.dc.n_hi && lo < fa.dc.n_lo)) {
-                uint64_t local;
-                const uint32_t cls = (uint32_t)big_find_class(fa.dc, lo, hi, local);
-                const uint32_t h0y = __ldg(reinterpret_cast<const uint32_t*>(fa.dc.cls + cls) + 1);
-                const uint32_t nlev = (h0y & 0xff) + ((h0y >> 8) & 0xff);
-                x = lo;
-                y = (hi & 0xffull) | (unsigned long long)cls << 8 | (unsigned long long)i << 32;
-                key = (15u - min(nlev, 15u)) << 27 | cls << 10 | (uint32_t)i;
-            } else {
-                atomicAdd(fa.bad_index, 1ull);
-            }
-        }
-        keys[i] = key; ex[i] = x; ey[i] = y;
-        __syncthreads();
-        for (int k = 2; k <= kDomEntries; k <<= 1)                   // bitonic sort of the 1024 keys
-            for (int j = k >> 1; j > 0; j >>= 1) {
-                const int o = i ^ j;
-                if (o > i) {
-                    const uint32_t a = keys[i], b = keys[o];
-                    if ((a > b) == ((i & k) == 0)) { keys[i] = b; keys[o] = a; }
-                }
-                __syncthreads();
-            }
-        const uint32_t src = keys[i] & 1023u;
-        out[dom * kDomEntries + i] = make_ulonglong2(ex[src], ey[src]);
-        __syncthreads();
-    }
-}
-
-template <bool kBig, bool kSg = false, bool kShard = false>
-__global__ void __launch_bounds__(kGemmThreads, 1)
-gemm_sorted_kernel(FastArgs fa, const unsigned long long* __restrict__ sorted, const uint16_t* __restrict__ gain, SgArgs sg, GemmArgs ga, int dpi)
-{
-    extern __shared__ __align__(128) uint8_t smem[];
-    const uint32_t img_bytes = fa.L.total;
-    uint64_t* bar_img = reinterpret_cast<uint64_t*>(smem + img_bytes);
-    uint64_t* bar_free = bar_img + 1;                                     // the MMAs reading the A / B buffers are done
-    uint64_t* bar_done = bar_img + 2;                                     // the accumulator of this item is complete
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bar_img + 5);
-    uint32_t* last_flag = tmem_slot + 1;
-    const uint32_t a_off = (img_bytes + 64 + 1023) & ~1023u;
-    constexpr uint32_t kAStage = kGemmRows * kStageK * 2;                  // 24576
-    uint8_t* a_buf = smem + a_off;                                        // [dpi * 2 stages] x 24576
-    const uint32_t b_stage = (uint32_t)ga.npad * kStageK * 2;
-    uint8_t* b_buf = a_buf + (uint32_t)dpi * kDomStages * kAStage;         // [dpi * 2 stages] x npad * 192
-
-    pdl_launch_dependents();
-    if (!fast_load_image(smem, fa.image, fa.L.total, bar_img, fa.flags)) return;
-    pdl_wait();
-    const FastSmem T = fast_view(smem, fa.L);
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    if (threadIdx.x == 0) {
-        mbar_init(bar_free, 1); mbar_init(bar_done, 1);
-        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-    }
-    if (warp == 0) tmem_alloc(tmem_slot, kTmemCols);
-    tc_fence_before();
-    __syncthreads();
-    tc_fence_after();
-    const uint32_t tmem = *tmem_slot;
-    const uint32_t idesc = instr_desc_bf16_m128((uint32_t)ga.npad);
-    const int64_t row_tiles = (ga.n_out + kGemmRows - 1) / kGemmRows;
-    const int64_t nd = ga.nstages;                                         // domains per row tile
-    // every CTA takes an equal contiguous range of the row_tiles * nd domains (row tile major); the parts of a row
-    // tile that end up in different CTAs are summed through the scratch, as in the GEMV
-    const int64_t D = row_tiles * nd, G = gridDim.x;
-    const int64_t dom_begin = blockIdx.x * D / G, dom_end = (blockIdx.x + 1) * D / G;
-    uint32_t uses = 0, done = 0;
-    bool timeout = false;
-    for (int64_t rt = dom_begin / nd; rt * nd < dom_end; ++rt) {
-        const int d_begin = (int)(max(dom_begin, rt * nd) - rt * nd), d_end = (int)(min(dom_end, (rt + 1) * nd) - rt * nd);
-        const uint32_t parts = (uint32_t)(unit_owner((rt + 1) * nd - 1, D, G) - unit_owner(rt * nd, D, G) + 1);   // CTAs that share this row tile
-        // the entries of an iteration are requested one iteration ahead (they come from DRAM)
-        const ulonglong2 no_entry = make_ulonglong2(kSortIndexMask, kBigNoBlock);
-        auto entry_at = [&](int d, int q) {
-            if (d + q >= d_end) return no_entry;
-            // warp 0 also issues the MMAs of every iteration: it takes the cheapest chunk of each domain (the last), the other
-            // warps pair chunk w - 1 of the first domain with chunk 31 - w of the second
-            const int chunk = warp == 0 ? 31 : (q == 0 ? warp - 1 : 31 - warp);
-            const int64_t at = (rt * nd + d + q) * kDomEntries + chunk * 32 + lane;
-            if (kBig) return __ldg(reinterpret_cast<const ulonglong2*>(sorted) + at);
-            return make_ulonglong2(__ldg(sorted + at), 0ull);
-        };
-        ulonglong2 e0 = entry_at(d_begin, 0), e1 = dpi > 1 ? entry_at(d_begin, 1) : no_entry;
-        for (int d0 = d_begin; d0 < d_end; d0 += dpi, ++uses) {
-            const int nd_now = min(dpi, d_end - d0);
-            const ulonglong2 cur0 = e0, cur1 = e1;
-            e0 = entry_at(d0 + dpi, 0);
-            if (dpi > 1) e1 = entry_at(d0 + dpi, 1);
-            // ---- A: every warp unranks one chunk of 32 sorted entries per domain
-#pragma unroll
-            for (int q = 0; q < 2; ++q) {
-                if (q >= nd_now) break;
-                const ulonglong2 e = q == 0 ? cur0 : cur1;
-                const uint64_t field = e.x & kSortIndexMask;
-                const uint64_t I = kSg ? field & ((1ull << fa.L.W) - 1ull) : field;     // shape-gain form: gain index above the shape index
-                const uint32_t pos = kBig ? (uint32_t)(e.y >> 32) & 1023u : (uint32_t)(e.x >> 48);
-                const bool valid = kBig ? !(e.y >> 63) : (field != kSortIndexMask && I < fa.n_points);
-                const uint32_t r = pos >> 3, c = pos & 7u;
-                const int64_t row = rt * kGemmRows + r, cb = (int64_t)(d0 + q) * kDomBlocks + c;
-                float gn = (!kSg && valid) ? gain_to_float(__ldg(gain + row * ga.bpr + cb)) : 0.f;
-                uint32_t w[12];
-                if (kBig) {
-                    const int cls = valid ? (int)((uint32_t)(e.y >> 8) & 0xffffffu) : 0;
-                    const uint64_t local = valid ? e.x - __ldg(fa.dc.off_lo + cls) : 0ull;     // class sizes fit 63 bits: exact mod 2^64
-                    Point pt;
-                    big_decode_local(T, fa.dc, cls, local, valid, pt);
-#pragma unroll
-                    for (int j = 0; j < 12; ++j) {
-                        __nv_bfloat162 h = __halves2bfloat162(dequant(gn, pt, 2 * j), dequant(gn, pt, 2 * j + 1));
-                        w[j] = *reinterpret_cast<uint32_t*>(&h);
-                    }
-                } else {
-                    Decoded dec;
-                    const uint32_t cls = decode_sorted_entry(fa, T, I, valid, dec);
-                    if (kSg && valid) {
-                        const float scale = sg.row_scale ? __ldg(sg.row_scale + row) : 1.f;
-                        gn = __fmul_rn(__fmul_rn(scale, __ldg(sg.codebook + (uint32_t)(field >> fa.L.W))),
-                                       __uint_as_float(T.desc[cls * kFastDescStride + kFastDescRnorm]));
-                    }
-                    expand_bf16(dec, gn, w);
-                }
-                // the previous MMAs read the buffers: wait for them only now, with the first chunk already unranked
-                if (q == 0 && uses > 0 && !mbar_wait(bar_free, (uses - 1u) & 1u)) timeout = true;
-                uint8_t* a_dst = a_buf + (uint32_t)(q * kDomStages + (c >> 2)) * kAStage + (r >> 3) * 128u + (r & 7u) * 16u + 3u * (c & 3u) * 2048u;
-#pragma unroll
-                for (int j = 0; j < 3; ++j)
-                    *reinterpret_cast<uint4*>(a_dst + j * 2048) = make_uint4(w[4 * j], w[4 * j + 1], w[4 * j + 2], w[4 * j + 3]);
-            }
-            // ---- B: the slice of X of these stages, 16-byte chunks (8 values along K)
-            const int kchunks = nd_now * kDomStages * (kStageK / 8);
-            for (int i = threadIdx.x; i < ga.npad * kchunks; i += kGemmThreads) {
-                const int kc = i / ga.npad, n = i % ga.npad;
-                const int64_t k = (int64_t)d0 * kDomBlocks * 24 + (int64_t)kc * 8;
-                uint4 v = make_uint4(0, 0, 0, 0);
-                if (n < ga.batch && k < ga.k_in) v = __ldg(reinterpret_cast<const uint4*>(ga.x + (int64_t)n * ga.k_in + k));
-                *reinterpret_cast<uint4*>(b_buf + (uint32_t)(kc / (kStageK / 8)) * b_stage + (uint32_t)(kc % (kStageK / 8)) * ga.npad * 16 + n * 16) = v;
-            }
-            fence_async_smem();
-            __syncthreads();
-            if (threadIdx.x == 0) {
-                tc_fence_after();
-                const uint32_t a_addr = smem_u32(a_buf), b_addr = smem_u32(b_buf);
-                for (int st = 0; st < nd_now * kDomStages; ++st)
-#pragma unroll
-                    for (int j = 0; j < kStageK / 16; ++j)
-                        umma_bf16(tmem, smem_desc(a_addr + st * kAStage + j * 4096, 2048, 128),
-                                  smem_desc(b_addr + st * b_stage + j * 2 * ga.npad * 16, ga.npad * 16, 128), idesc,
-                                  (d0 > d_begin || st > 0 || j > 0) ? 1u : 0u);
-                umma_commit(bar_free);
-                if (d0 + dpi >= d_end) umma_commit(bar_done);
-            }
-        }
-        // ---- epilogue: accumulator -> scratch (split-K) or Y
-        const bool has = d_end > d_begin;
-        if (warp < 4 && has) {
-            if (!mbar_wait(bar_done, done & 1u)) timeout = true;
-            tc_fence_after();
-            const int64_t orow = rt * kGemmRows + warp * 32 + lane;
-            for (int c0 = 0; c0 < ga.npad; c0 += 16) {
-                float v[16];
-                tmem_ld16(tmem + ((uint32_t)(warp * 32) << 16) + (uint32_t)c0, v);
-                if (orow < ga.n_out) {
-#pragma unroll
-                    for (int i = 0; i < 16; ++i) {
-                        const int n = c0 + i;
-                        if (n < ga.batch) {
-                            if (parts == 1u) gemm_store<kShard>(ga, n, orow, v[i]);
-                            else atomicAdd(ga.scratch + (int64_t)n * ga.scratch_ld + orow, v[i]);
-                        }
-                    }
-                }
-            }
-            tc_fence_before();
-        }
-        done += has;
-        if (parts > 1u) {
-            __threadfence();
-            __syncthreads();
-            if (threadIdx.x == 0) *last_flag = (atomicAdd(ga.counters + rt, 1u) == parts - 1u);
-            __syncthreads();
-            if (*last_flag) {
-                __threadfence();
-                for (int i = threadIdx.x; i < kGemmRows * ga.batch; i += kGemmThreads) {
-                    const int n = i / kGemmRows;
-                    const int64_t orow = rt * kGemmRows + (i % kGemmRows);
-                    if (orow < ga.n_out) {
-                        float* sp = ga.scratch + (int64_t)n * ga.scratch_ld + orow;
-                        gemm_store<kShard>(ga, n, orow, __ldcg(sp));
-                        __stcg(sp, 0.f);
-                    }
-                }
-                if (threadIdx.x == 0) ga.counters[rt] = 0u;
-            }
-        }
-        __syncthreads();
-    }
-    if (timeout) atomicOr(fa.flags, 1u);
-    if (kShard) {
-        __threadfence_system();                           // this thread's stores to the peers' copies, before the CTA counts itself in
-        shard_arrive(*ga.shard);
-    }
-    __syncthreads();
-    if (warp == 0) tmem_dealloc(tmem, kTmemCols);
-}
-
-// The same product for padded batch <= 32, where two domains' tiles fit: the two buffer sets alternate between
-// consecutive domains and nobody waits for the whole CTA.  Warps 1..31 unrank: the chunks of 32 sorted entries of a
-// row tile are handed out by a ticket counter (ticket t = chunk t % 32 of the tile's domain t / 32, so from expensive
-// to cheap inside a domain), a warp always holding its next ticket with that chunk's entries already requested.
-// It unranks the chunk, waits (rarely) until the MMAs that read this buffer two domains ago are done, writes its
-// part of A and arrives on the buffer's "full" barrier.  Warp 0 stages the X slice of the next domain, arrives too,
-// and its first thread issues the MMAs of a domain as soon as that barrier completes.
-// kStored: the same structure on the stored stream (`sorted` then points at it): a chunk is 32 consecutive blocks of the
-// domain in natural order (4 rows x 8 column blocks), unranked by the any-class decoder.
-template <bool kBig, bool kSg = false, bool kShard = false, bool kStored = false>
-__global__ void __launch_bounds__(kGemmThreads, 1)
-gemm_pipe_kernel(FastArgs fa, const unsigned long long* __restrict__ sorted, const uint16_t* __restrict__ gain, SgArgs sg, GemmArgs ga,
-                 int b_double)
-{
-    static_assert(!(kStored && kBig && kSg), "no shape-gain form for the codes with tables in global memory");
-    extern __shared__ __align__(128) uint8_t smem[];
-    const uint32_t img_bytes = fa.L.total;
-    uint64_t* bar_img = reinterpret_cast<uint64_t*>(smem + img_bytes);
-    uint64_t* bar_full = bar_img + 1;                                     // [2] 32 chunks of A and the X slice are in the buffer
-    uint64_t* bar_free = bar_img + 3;                                     // [2] the MMAs reading the buffer are done
-    uint64_t* bar_done = bar_img + 5;                                     // the accumulator of this row tile is complete
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bar_img + 6);
-    uint32_t* last_flag = tmem_slot + 1;
-    uint32_t* ticket = tmem_slot + 2;                                     // next chunk ticket of the row tile in progress
-    const uint32_t a_off = (img_bytes + 64 + 1023) & ~1023u;
-    constexpr uint32_t kAStage = kGemmRows * kStageK * 2;                  // 24576
-    uint8_t* a_buf = smem + a_off;                                        // [2 buffers][2 stages] x 24576
-    const uint32_t b_stage = (uint32_t)ga.npad * kStageK * 2;
-    uint8_t* b_buf = a_buf + 2u * kDomStages * kAStage;                    // [2 buffers, or 1][2 stages] x npad * 192
-    constexpr uint32_t kWorkers = kGemmThreads / 32 - 1;                   // 31 unranking warps
-
-    pdl_launch_dependents();
-    if (!fast_load_image(smem, fa.image, fa.L.total, bar_img, fa.flags)) return;
-    pdl_wait();
-    const FastSmem T = fast_view(smem, fa.L);
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    if (threadIdx.x == 0) {
-        mbar_init(bar_full, 33); mbar_init(bar_full + 1, 33);             // 32 chunks + the X slice
-        mbar_init(bar_free, 1); mbar_init(bar_free + 1, 1); mbar_init(bar_done, 1);
-        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-    }
-    if (warp == 0) tmem_alloc(tmem_slot, kTmemCols);
-    tc_fence_before();
-    __syncthreads();
-    tc_fence_after();
-    const uint32_t tmem = *tmem_slot;
-    const uint32_t idesc = instr_desc_bf16_m128((uint32_t)ga.npad);
-    const int64_t row_tiles = (ga.n_out + kGemmRows - 1) / kGemmRows;
-    const int64_t nd = ga.nstages;                                         // domains per row tile
-    const int64_t D = row_tiles * nd, G = gridDim.x;
-    const int64_t dom_begin = blockIdx.x * D / G, dom_end = (blockIdx.x + 1) * D / G;
-    uint32_t g_base = 0, done = 0;                                         // domains this CTA has finished (domain g uses buffer g & 1 for the (g >> 1)-th time)
-    bool timeout = false;
-    const ulonglong2 no_entry = make_ulonglong2(kSortIndexMask, kBigNoBlock);
-    auto arrive_full = [&](uint32_t b) {
-        fence_async_smem();
-        __syncwarp();
-        if (lane == 0) asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar_full + b)) : "memory");
-    };
-
-    for (int64_t rt = dom_begin / nd; rt * nd < dom_end; ++rt) {
-        const int d_begin = (int)(max(dom_begin, rt * nd) - rt * nd), d_end = (int)(min(dom_end, (rt + 1) * nd) - rt * nd);
-        const uint32_t parts = (uint32_t)(unit_owner((rt + 1) * nd - 1, D, G) - unit_owner(rt * nd, D, G) + 1);   // CTAs that share this row tile
-        const uint32_t n_dom = (uint32_t)(d_end - d_begin), n_tickets = n_dom * 32u;
-        if (threadIdx.x == 0) *ticket = kWorkers;                          // the first tickets are the workers' own numbers
-        __syncthreads();
-        if (warp == 0) {
-            // ---- X slices and MMAs
-            // the slice of domain j of this tile, 16-byte chunks (8 values along K).  With two X buffers it may be written once
-            // the MMAs of two domains ago are done; with one (wide batches: no room for two), only after the previous domain's
-            auto stage_b = [&](uint32_t j) {
-                const uint32_t gd = g_base + j, b = gd & 1u, bx = b_double ? b : 0u;
-                if (b_double) { if (gd >= 2u && !mbar_wait(bar_free + b, ((gd >> 1) - 1u) & 1u)) timeout = true; }
-                else if (gd >= 1u && !mbar_wait(bar_free + ((gd - 1u) & 1u), ((gd - 1u) >> 1) & 1u)) timeout = true;
-                const int64_t k0 = (int64_t)(d_begin + (int)j) * kDomBlocks * 24;
-                for (int n = lane; n < ga.npad; n += 32) {
-                    const uint16_t* xr = ga.x + (int64_t)n * ga.k_in + k0;
-                    uint8_t* dst = b_buf + bx * kDomStages * b_stage + n * 16;
-#pragma unroll 4
-                    for (int kc = 0; kc < kDomStages * (kStageK / 8); ++kc) {        // 24 asynchronous 16-byte copies per row, zero-filled outside X
-                        const bool in = n < ga.batch && k0 + kc * 8 < ga.k_in;
-                        const uint32_t to = smem_u32(dst + (uint32_t)(kc / (kStageK / 8)) * b_stage + (uint32_t)(kc % (kStageK / 8)) * ga.npad * 16);
-                        asm volatile("cp.async.ca.shared.global [%0], [%1], 16, %2;" ::"r"(to), "l"(in ? xr + kc * 8 : ga.x), "r"(in ? 16u : 0u) : "memory");
-                    }
-                }
-                asm volatile("cp.async.wait_all;" ::: "memory");
-                arrive_full(b);
-            };
-            if (n_dom > 0) stage_b(0);
-            for (uint32_t j = 0; j < n_dom; ++j) {
-                if (b_double && j + 1 < n_dom) stage_b(j + 1);
-                const uint32_t gd = g_base + j, b = gd & 1u, bx = b_double ? b : 0u;
-                if (lane == 0) {
-                    if (!mbar_wait(bar_full + b, (gd >> 1) & 1u)) timeout = true;
-                    tc_fence_after();
-                    const uint32_t a_addr = smem_u32(a_buf) + b * kDomStages * kAStage, b_addr = smem_u32(b_buf) + bx * kDomStages * b_stage;
-                    for (int st = 0; st < kDomStages; ++st)
-#pragma unroll
-                        for (int jj = 0; jj < kStageK / 16; ++jj)
-                            umma_bf16(tmem, smem_desc(a_addr + st * kAStage + jj * 4096, 2048, 128),
-                                      smem_desc(b_addr + st * b_stage + jj * 2 * ga.npad * 16, ga.npad * 16, 128), idesc,
-                                      (j > 0 || st > 0 || jj > 0) ? 1u : 0u);
-                    umma_commit(bar_free + b);
-                    if (j + 1 == n_dom) umma_commit(bar_done);
-                }
-                __syncwarp();
-                if (!b_double && j + 1 < n_dom) stage_b(j + 1);
-            }
-        } else {
-            // ---- A: unrank chunks until the tile's tickets are gone
-            auto entry_of = [&](uint32_t t) {
-                if (t >= n_tickets) return no_entry;
-                if (kStored && kBig) {                                       // the index itself, in the form of the sorted layout's entries
-                    const uint32_t pos = (t & 31u) * 32u + lane;
-                    const int64_t row = rt * kGemmRows + (pos >> 3), cb = (int64_t)(d_begin + (int)(t >> 5)) * kDomBlocks + (pos & 7u);
-                    uint64_t lo = 0, hi = kBigNoBlock;
-                    if (row < ga.n_out && cb < ga.bpr) load_index(reinterpret_cast<const uint32_t*>(sorted), (uint64_t)(row * ga.bpr + cb), fa.dc.W, lo, hi);
-                    return make_ulonglong2(lo, hi | (unsigned long long)pos << 32);
-                }
-                if (kStored) {                                               // the field itself, its position in the high 16 bits
-                    const uint32_t pos = (t & 31u) * 32u + lane;
-                    const int64_t row = rt * kGemmRows + (pos >> 3), cb = (int64_t)(d_begin + (int)(t >> 5)) * kDomBlocks + (pos & 7u);
-                    unsigned long long f = kSortIndexMask;
-                    if (row < ga.n_out && cb < ga.bpr)
-                        f = load_field(reinterpret_cast<const uint32_t*>(sorted), (uint64_t)(row * ga.bpr + cb), (int)fa.L.W + (kSg ? sg.bits : 0));
-                    return make_ulonglong2(f | (unsigned long long)pos << 48, 0ull);
-                }
-                const int64_t at = (rt * nd + d_begin + (int)(t >> 5)) * kDomEntries + (t & 31u) * 32u + lane;
-                if (kBig) return __ldg(reinterpret_cast<const ulonglong2*>(sorted) + at);
-                return make_ulonglong2(__ldg(sorted + at), 0ull);
-            };
-            uint32_t tk = (uint32_t)warp - 1u;
-            ulonglong2 e = entry_of(tk);
-            while (tk < n_tickets) {
-                uint32_t tk_next = 0;
-                if (lane == 0) tk_next = atomicAdd(ticket, 1u);
-                tk_next = __shfl_sync(kFullMask, tk_next, 0);
-                const ulonglong2 e_next = entry_of(tk_next);                // requested a chunk ahead (it comes from DRAM)
-                const uint32_t j = tk >> 5, gd = g_base + j, b = gd & 1u;
-                const int d = d_begin + (int)j;
-                const uint64_t field = e.x & kSortIndexMask;
-                const uint64_t I = kSg ? field & ((1ull << fa.L.W) - 1ull) : field;     // shape-gain form: gain index above the shape index
-                const uint32_t pos = kBig ? (uint32_t)(e.y >> 32) & 1023u : (uint32_t)(e.x >> 48);
-                bool valid = kBig ? !(e.y >> 63) : (field != kSortIndexMask && I < fa.n_points);
-                if (kStored && kBig && valid) {                               // the stored index may be out of range: count it, treat it as no block
-                    const uint64_t hi = e.y & 0xffull;
-                    valid = hi < fa.dc.n_hi || (hi == fa.dc.n_hi && e.x < fa.dc.n_lo);
-                    if (!valid) atomicAdd(fa.bad_index, 1ull);
-                }
-                const uint32_t r = pos >> 3, c = pos & 7u;
-                const int64_t row = rt * kGemmRows + r, cb = (int64_t)d * kDomBlocks + c;
-                float gn = (!kSg && valid) ? gain_to_float(__ldg(gain + row * ga.bpr + cb)) : 0.f;
-                uint32_t w[12];
-                if (kBig) {
-                    int cls = 0;
-                    uint64_t local = 0;
-                    if (kStored) { if (valid) cls = big_find_class(fa.dc, e.x, e.y & 0xffull, local); }
-                    else if (valid) {
-                        cls = (int)((uint32_t)(e.y >> 8) & 0xffffffu);
-                        local = e.x - __ldg(fa.dc.off_lo + cls);                 // class sizes fit 63 bits: exact mod 2^64
-                    }
-                    Point pt;
-                    big_decode_local(T, fa.dc, cls, local, valid, pt);
-#pragma unroll
-                    for (int jj = 0; jj < 12; ++jj) {
-                        __nv_bfloat162 h = __halves2bfloat162(dequant(gn, pt, 2 * jj), dequant(gn, pt, 2 * jj + 1));
-                        w[jj] = *reinterpret_cast<uint32_t*>(&h);
-                    }
-                } else {
-                    Decoded dec;
-                    uint32_t cls;
-                    if (kStored) {
-                        if (field != kSortIndexMask && !valid) atomicAdd(fa.bad_index, 1ull);
-                        uint64_t local = 0;
-                        cls = valid ? fast_find_class(T, I, local) : 0u;
-                        fast_decode_local<-1>(T, cls, local, valid, kFullMask, dec);
-                    } else {
-                        cls = decode_sorted_entry(fa, T, I, valid, dec);
-                    }
-                    if (kSg && valid) {
-                        const float scale = sg.row_scale ? __ldg(sg.row_scale + row) : 1.f;
-                        gn = __fmul_rn(__fmul_rn(scale, __ldg(sg.codebook + (uint32_t)(field >> fa.L.W))),
-                                       __uint_as_float(T.desc[cls * kFastDescStride + kFastDescRnorm]));
-                    }
-                    expand_bf16(dec, gn, w);
-                }
-                // the MMAs of two domains ago read this buffer: wait for them only now, with the chunk already unranked
-                if (gd >= 2u && !mbar_wait(bar_free + b, ((gd >> 1) - 1u) & 1u)) timeout = true;
-                uint8_t* a_dst = a_buf + (b * kDomStages + (c >> 2)) * kAStage + (r >> 3) * 128u + (r & 7u) * 16u + 3u * (c & 3u) * 2048u;
-#pragma unroll
-                for (int jj = 0; jj < 3; ++jj)
-                    *reinterpret_cast<uint4*>(a_dst + jj * 2048) = make_uint4(w[4 * jj], w[4 * jj + 1], w[4 * jj + 2], w[4 * jj + 3]);
-                arrive_full(b);
-                tk = tk_next; e = e_next;
-            }
-        }
-        g_base += n_dom;
-        const bool has = d_end > d_begin;
-        // ---- epilogue: accumulator -> scratch (split-K) or Y
-        if (warp < 4 && has) {
-            if (!mbar_wait(bar_done, done & 1u)) timeout = true;
-            tc_fence_after();
-            const int64_t orow = rt * kGemmRows + warp * 32 + lane;
-            for (int c0 = 0; c0 < ga.npad; c0 += 16) {
-                float v[16];
-                tmem_ld16(tmem + ((uint32_t)(warp * 32) << 16) + (uint32_t)c0, v);
-                if (orow < ga.n_out) {
-#pragma unroll
-                    for (int i = 0; i < 16; ++i) {
-                        const int n = c0 + i;
-                        if (n < ga.batch) {
-                            if (parts == 1u) gemm_store<kShard>(ga, n, orow, v[i]);
-                            else atomicAdd(ga.scratch + (int64_t)n * ga.scratch_ld + orow, v[i]);
-                        }
-                    }
-                }
-            }
-            tc_fence_before();
-        }
-        done += has;
-        if (parts > 1u) {
-            __threadfence();
-            __syncthreads();
-            if (threadIdx.x == 0) *last_flag = (atomicAdd(ga.counters + rt, 1u) == parts - 1u);
-            __syncthreads();
-            if (*last_flag) {
-                __threadfence();
-                for (int i = threadIdx.x; i < kGemmRows * ga.batch; i += kGemmThreads) {
-                    const int n = i / kGemmRows;
-                    const int64_t orow = rt * kGemmRows + (i % kGemmRows);
-                    if (orow < ga.n_out) {
-                        float* sp = ga.scratch + (int64_t)n * ga.scratch_ld + orow;
-                        gemm_store<kShard>(ga, n, orow, __ldcg(sp));
-                        __stcg(sp, 0.f);
-                    }
-                }
-                if (threadIdx.x == 0) ga.counters[rt] = 0u;
-            }
-        }
-        __syncthreads();
-    }
-    if (timeout) atomicOr(fa.flags, 1u);
-    if (kShard) {
-        __threadfence_system();                           // this thread's stores to the peers' copies, before the CTA counts itself in
-        shard_arrive(*ga.shard);
-    }
-    __syncthreads();
-    if (warp == 0) tmem_dealloc(tmem, kTmemCols);
-}
+#include "gemv_kernels.cuh"
+#include "gemm_kernels.cuh"
 
 FastArgs fast_args(const llvq_ctx* ctx)
 {
