@@ -45,16 +45,18 @@ __device__ __forceinline__ void store_y(const YOut& yo, int64_t row, float v)
     if (kOutBf16) {
         const __nv_bfloat16 h = __float2bfloat16_rn(v);
         reinterpret_cast<__nv_bfloat16*>(yo.y)[row] = h;
-        if (!kShard) return;                              // the single-GPU instantiations carry none of what follows
+        if (kShard) {                                     // the single-GPU instantiations carry none of this
 #pragma unroll
-        for (int p = 0; p < kMaxShardPeers; ++p)          // static indices: the struct stays in the parameter bank
-            if (p < yo.n_peer) reinterpret_cast<__nv_bfloat16*>(yo.peer[p])[row] = h;
+            for (int p = 0; p < kMaxShardPeers; ++p)      // static indices: the struct stays in the parameter bank
+                if (p < yo.n_peer) reinterpret_cast<__nv_bfloat16*>(yo.peer[p])[row] = h;
+        }
     } else {
         reinterpret_cast<float*>(yo.y)[row] = v;
-        if (!kShard) return;
+        if (kShard) {
 #pragma unroll
-        for (int p = 0; p < kMaxShardPeers; ++p)
-            if (p < yo.n_peer) reinterpret_cast<float*>(yo.peer[p])[row] = v;
+            for (int p = 0; p < kMaxShardPeers; ++p)
+                if (p < yo.n_peer) reinterpret_cast<float*>(yo.peer[p])[row] = v;
+        }
     }
 }
 

@@ -143,8 +143,7 @@ __device__ __forceinline__ void prefetch_span_l2(const void* p, uint64_t first, 
 #define FAST_PROLOGUE()                                                                         \
     extern __shared__ __align__(128) uint8_t smem[];                                            \
     uint64_t* bar = reinterpret_cast<uint64_t*>(smem + fa.L.total);                              \
-    uint8_t* staging = smem + fa.L.total + 16;                                                  \
-    (void)staging;                                                                              \
+    [[maybe_unused]] uint8_t* staging = smem + fa.L.total + 16;                                 \
     pdl_launch_dependents();                                                                    \
     if (!fast_load_image(smem, fa.image, fa.L.total, bar, fa.flags)) return;                    \
     pdl_wait();                                                                                 \
