@@ -350,6 +350,12 @@ gemv_sorted_kernel(FastArgs fa, const unsigned long long* __restrict__ sorted, c
                    int64_t n_out, int64_t k_in, int64_t bpr, uint32_t nq_magic, const uint16_t* __restrict__ x, YOut yo,
                    float* __restrict__ scratch, uint32_t* __restrict__ counters)
 {
+    {   // ask for the warps' first chunks in L2 while the table image is on its way (one request per 128-byte line)
+        const int64_t nq0 = (bpr + 3) / 4, U0 = ((n_out + kGemvGroupRows - 1) / kGemvGroupRows) * nq0;
+        const int64_t ub = blockIdx.x * U0 / gridDim.x, ue = (blockIdx.x + 1) * U0 / gridDim.x;
+        if ((threadIdx.x & 15u) == 0u && ub + (int64_t)(threadIdx.x >> 5) < ue)
+            asm volatile("prefetch.global.L2 [%0];" ::"l"(sorted + ub * 32 + threadIdx.x));
+    }
     FAST_PROLOGUE();
     const int64_t nq = (bpr + 3) / 4;
     uint32_t* xs = reinterpret_cast<uint32_t*>(staging);            // [nq * 4][12] packed bf16 pairs of x
@@ -445,6 +451,19 @@ gemv_bin_kernel(FastArgs fa, const uint32_t* __restrict__ stream, const uint16_t
                 int64_t n_out, int64_t k_in, int64_t bpr, uint32_t nq_magic, int seg_units, const uint16_t* __restrict__ x, YOut yo,
                 float* __restrict__ scratch, uint32_t* __restrict__ counters)
 {
+    {
+        // the rows of the row groups this CTA touches are one contiguous span of the index stream and of the gains:
+        // request it from DRAM now, while the table image is on its way; the binning phases then read it from L2
+        const int64_t nq0 = (bpr + 3) / 4, U0 = ((n_out + kGemvGroupRows - 1) / kGemvGroupRows) * nq0;
+        const int64_t ub = blockIdx.x * U0 / gridDim.x, ue = (blockIdx.x + 1) * U0 / gridDim.x;
+        if (ub < ue) {
+            const uint64_t b_first = (uint64_t)(ub / nq0) * kGemvGroupRows * (uint64_t)bpr;
+            const uint64_t b_last = (uint64_t)min(((ue - 1) / nq0 + 1) * kGemvGroupRows, n_out) * (uint64_t)bpr;
+            const uint64_t wf = (uint64_t)fa.L.W + (kSg ? (uint64_t)sg.bits : 0ull);
+            prefetch_span_l2(stream, b_first * wf / 8, (b_last * wf + 7) / 8);
+            if (!kSg) prefetch_span_l2(gain, b_first * 2, b_last * 2);
+        }
+    }
     FAST_PROLOGUE();
     const int64_t nq = (bpr + 3) / 4;
     uint32_t* xs = reinterpret_cast<uint32_t*>(staging);            // [nq * 4][12] packed bf16 pairs of x
@@ -460,17 +479,7 @@ gemv_bin_kernel(FastArgs fa, const uint32_t* __restrict__ stream, const uint16_t
     const uint32_t kWarps = blockDim.x >> 5;
     const int64_t groups = (n_out + kGemvGroupRows - 1) / kGemvGroupRows;
     const int64_t U = groups * nq, G = gridDim.x;
-    const int64_t u_begin = blockIdx.x * U / G, u_end = (blockIdx.x + 1) * U / G;
     const uint32_t nq32 = (uint32_t)nq;
-    if (u_begin < u_end) {
-        // the rows of the row groups this CTA touches are one contiguous span of the index stream and of the gains:
-        // request it from DRAM now, the binning phases then read it from L2
-        const uint64_t b_first = (uint64_t)(u_begin / nq) * kGemvGroupRows * (uint64_t)bpr;
-        const uint64_t b_last = (uint64_t)min(((u_end - 1) / nq + 1) * kGemvGroupRows, n_out) * (uint64_t)bpr;
-        const uint64_t wf = (uint64_t)fa.L.W + (kSg ? (uint64_t)sg.bits : 0ull);
-        prefetch_span_l2(stream, b_first * wf / 8, (b_last * wf + 7) / 8);
-        if (!kSg) prefetch_span_l2(gain, b_first * 2, b_last * 2);
-    }
     for_each_sorted_segment(U, G, nq, blockIdx.x, [&](int64_t tu0, int64_t tu1, int64_t rg0, int64_t rg1, bool first, bool last) {
         if (first)
             for (int i = threadIdx.x; i < kSortAccCopies * kGemvGroupsPerPass * kGemvGroupRows; i += (int)blockDim.x) acc[i] = 0.f;
