@@ -41,8 +41,8 @@ WORKLOAD = "configs[2]: fused dequant+GEMV batch 1 on W 4096x4096, 11008x4096, 4
 
 # dram__bytes_read.sum + dram__bytes_write.sum of one gemv_fast_kernel launch on the 11008x4096 layer, from the
 # ncu capture summarised under profiles/ (algorithmic bytes: 15 089 152)
-NCU_TRAFFIC_BYTES_11008x4096 = 15261952
-NCU_WARP_INSTRUCTIONS_11008x4096 = 55404893          # smsp__inst_executed.sum of the same capture
+NCU_TRAFFIC_BYTES_11008x4096 = 15262208
+NCU_WARP_INSTRUCTIONS_11008x4096 = 55592066          # smsp__inst_executed.sum of the same capture
 ISSUE_PEAK_WARP_INST_PER_S = 148 * 4 * 1.965e9       # SMs x schedulers x max SM clock: one warp instruction per scheduler and cycle
 
 
@@ -690,7 +690,7 @@ def main() -> None:
                          "traffic": NCU_TRAFFIC_BYTES_11008x4096, "kernel": "gemv_bin_kernel on 11008x4096",
                          "algorithmic_bytes_per_launch": dom_bytes, "peak_source": f"of {which}", "frac_of_nominal_8TBps": achieved / 8000.0,
                          # what binds the kernel instead of HBM: counters of the ncu capture summarised under profiles/
-                         "ncu": {"warp_instructions_per_block": 941, "issue_slots_used": 0.668, "alu_pipe_busy": 0.614,
+                         "ncu": {"warp_instructions_per_block": 945, "issue_slots_used": 0.653, "alu_pipe_busy": 0.599,
                                  "shared_memory_wavefronts_per_block": 208, "instructions_per_block_at_hbm_roofline": 46}},
             # the same launch against what actually binds it: instruction issue (instructions per launch from the ncu
             # capture, duration measured live)
