@@ -67,7 +67,22 @@ __device__ __forceinline__ void big_decode_local(const FastSmem& T, const DevCod
         const uint4 L = active ? __ldg(cd + 2 + l) : zero4;
         const uint32_t k = L.y & 0xff, val = (L.y >> 8) & 0xff, n = (L.y >> 16) & 0xff;
         uint32_t rho = 0;
-        if (active) { uint64_t pq; divmod_magic(p, L.x, ((uint64_t)L.w << 32) | L.z, pq, rho); p = pq; }
+        if (active) {
+            if ((p >> 32) == 0ull) {
+                // the rank has shrunk to 32 bits (it only ever gets smaller): the high word of the 64-bit magic,
+                // floor(2^32 / d) or one less, gives an estimate at most two too small
+                const uint32_t p32 = (uint32_t)p;
+                uint32_t q32 = __umulhi(p32, L.w);
+                uint32_t r32 = p32 - q32 * L.x;
+                if (r32 >= L.x) { r32 -= L.x; ++q32; }
+                if (r32 >= L.x) { r32 -= L.x; ++q32; }
+                rho = r32; p = q32;
+            } else {
+                uint64_t pq;
+                divmod_magic(p, L.x, ((uint64_t)L.w << 32) | L.z, pq, rho);
+                p = pq;
+            }
+        }
         const int top = __reduce_max_sync(kFullMask, n);
         const uint32_t rel = nth_subset(T, k, rho, top);
         const uint32_t a = deposit24(T.pd6, rel, freem);
