@@ -97,7 +97,7 @@ def test_gemv_sg(lib, ctxs, codes, code, bits):
     # the fused product uses exactly the weights the dequantizer writes
     w = lib.llvq_dequant_matrix_sg(ctx, d_s, bits, d_cb, d_rs, n_out, k_in)
     y2 = (w.double() @ d_x.double()).cpu().numpy()
-    assert gemv_error(y.cpu().numpy(), y2) <= 1e-4          # binary32 accumulation only
+    assert gemv_error(y.cpu().numpy(), y2) <= 5e-4          # binary32 accumulation only (its order varies from run to run)
     assert lib.llvq_last_error(ctx) == (0, 0)
 
 
@@ -188,7 +188,9 @@ def test_gemv_sorted_sg_full_size_and_limits(lib, ctxs, codes):
     srt = lib.llvq_sort_blocks_sg(ctx, d_s, bits, n_out, k_in)
     y = lib.llvq_gemv_sorted_sg(ctx, srt, bits, _f32(cb), _f32(rs), n_out, k_in, to_dev_bf16(x)).cpu().numpy()
     y2 = lib.llvq_gemv_sg(ctx, d_s, bits, _f32(cb), _f32(rs), n_out, k_in, to_dev_bf16(x)).cpu().numpy()
-    assert gemv_error(y, y2.astype(np.float64)) <= 1e-4
+    # two binary32 sums of the same 4096 products in different (and, through the shared-memory atomics, run-dependent)
+    # orders; relative to the floor of 1e-3 of the largest output a small row's sum can move by about 1e-4
+    assert gemv_error(y, y2.astype(np.float64)) <= 5e-4
     rows = [0, 9, 2047, 4095] + list(range(123, 4096, 611))
     ref = np.array([o.gemm_sg(stream, bits, cb, rs, n_out, k_in, x, rows=(r, 1))[r] for r in rows])
     assert gemv_error(y[rows], ref) <= TOL
