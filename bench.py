@@ -268,72 +268,41 @@ def extras(P, ctx) -> dict:
     by = nb * (CODE_W // 8 + 2) + rows * cols * 2
     out["dequant_4096x4096_flat"] = {"us": us, "GBps": by / us / 1e3, "weights_per_s": rows * cols / (us * 1e-6), "algorithmic_bytes": by}
     del bufs
-    # --- GEMM, 8192 x 8192
-    n, k = 8192, 8192
-    bufs = []
-    for c in range(12):
-        stream, gain, nb = gen.make_layer(CODE_N, CODE_W, n, k, 1, seed=200 + c)
-        bufs.append((dev(stream), dev(gain, np.float16)))
-    for batch in (16, 64):
-        x = dev(gen.normal_bf16((batch, k), seed=batch), np.int16).view(torch.bfloat16)
-        y = torch.empty((batch, n), dtype=torch.bfloat16, device="cuda")
-        fn = lambda i: P.llvq_gemm_small_batch(ctx, bufs[i % 12][0], bufs[i % 12][1], n, k, x, d_y=y)
-        _event_us(torch, fn, 4)
-        us = _event_us(torch, fn, 24)
-        by = nb * (CODE_W // 8 + 2) + batch * k * 2 + batch * n * 2
-        out[f"gemm_8192x8192_b{batch}"] = {"us": us, "GBps": by / us / 1e3, "TFLOPs": 2.0 * n * k * batch / us / 1e6, "algorithmic_bytes": by}
-    # --- the same GEMM on its sorted layout (every matrix rearranged once)
-    srt = [P.llvq_sort_blocks_gemm(ctx, b[0], n, k) for b in bufs]
-    for batch in (16, 64):
-        x = dev(gen.normal_bf16((batch, k), seed=batch), np.int16).view(torch.bfloat16)
-        y = torch.empty((batch, n), dtype=torch.bfloat16, device="cuda")
-        fn = lambda i: P.llvq_gemm_small_batch_sorted(ctx, srt[i % 12], bufs[i % 12][1], n, k, x, d_y=y)
-        _event_us(torch, fn, 4)
-        us = _event_us(torch, fn, 24)
-        by = nb * (CODE_W // 8 + 2) + batch * k * 2 + batch * n * 2
-        out[f"gemm_8192x8192_b{batch}_sorted_layout"] = {"us": us, "GBps": by / us / 1e3, "TFLOPs": 2.0 * n * k * batch / us / 1e6, "algorithmic_bytes": by}
-    del bufs, srt
-    # --- the two rectangular shapes of the same configuration, batch 16 (4 rotating copies, 314 MB)
-    for (n2, k2) in ((28672, 8192), (8192, 28672)):
-        bufs2 = []
-        for c in range(4):
-            stream, gain, nb2 = gen.make_layer(CODE_N, CODE_W, n2, k2, 1, seed=220 + c)
-            d_i, d_g = dev(stream), dev(gain, np.float16)
-            bufs2.append((d_i, d_g, P.llvq_sort_blocks_gemm(ctx, d_i, n2, k2)))
-        x = dev(gen.normal_bf16((16, k2), seed=16), np.int16).view(torch.bfloat16)
-        y = torch.empty((16, n2), dtype=torch.bfloat16, device="cuda")
-        by = nb2 * (CODE_W // 8 + 2) + 16 * k2 * 2 + 16 * n2 * 2
-        for name, fn in (("", lambda i: P.llvq_gemm_small_batch(ctx, bufs2[i % 4][0], bufs2[i % 4][1], n2, k2, x, d_y=y)),
-                         ("_sorted_layout", lambda i: P.llvq_gemm_small_batch_sorted(ctx, bufs2[i % 4][2], bufs2[i % 4][1], n2, k2, x, d_y=y))):
-            _event_us(torch, fn, 2)
-            us = _event_us(torch, fn, 8)
-            out[f"gemm_{n2}x{k2}_b16{name}"] = {"us": us, "GBps": by / us / 1e3, "TFLOPs": 2.0 * n2 * k2 * 16 / us / 1e6, "algorithmic_bytes": by}
-        del bufs2
-    # --- GEMM, 8192 x 8192 at ~3 bits/weight: 72-bit indices over shells 2..53
+    # --- small-batch GEMM, every cell of the 70B-shaped configuration: three shapes x batch 16 / 64 x the ~2 bits/weight
+    # (48-bit, shells 2..13) and ~3 bits/weight (72-bit, shells 2..53) codes, stored stream and sorted layout.  One
+    # layer per cell is generated on the host; the rotating copies (more than L2 together) are the same rows in a
+    # different order, rolled on the device: valid streams with the same class mix.
     ctx53 = P.Context(2, 53, device=torch.cuda.current_device())
-    bufs = []
-    for c in range(8):
-        stream, gain, nb = gen.make_layer(ctx53.num_points, ctx53.index_bits, n, k, 1, seed=250 + c)
-        bufs.append((dev(stream), dev(gain, np.float16)))
-    for batch in (16, 64):
-        x = dev(gen.normal_bf16((batch, k), seed=batch), np.int16).view(torch.bfloat16)
-        y = torch.empty((batch, n), dtype=torch.bfloat16, device="cuda")
-        fn = lambda i: P.llvq_gemm_small_batch(ctx53, bufs[i % 8][0], bufs[i % 8][1], n, k, x, d_y=y)
-        _event_us(torch, fn, 4)
-        us = _event_us(torch, fn, 16)
-        by = nb * (72 // 8 + 2) + batch * k * 2 + batch * n * 2
-        out[f"gemm_8192x8192_b{batch}_72bit"] = {"us": us, "GBps": by / us / 1e3, "TFLOPs": 2.0 * n * k * batch / us / 1e6, "algorithmic_bytes": by}
-    srt = [P.llvq_sort_blocks_gemm(ctx53, b[0], n, k) for b in bufs]      # 128-bit entries: index, class, position
-    for batch in (16, 64):
-        x = dev(gen.normal_bf16((batch, k), seed=batch), np.int16).view(torch.bfloat16)
-        y = torch.empty((batch, n), dtype=torch.bfloat16, device="cuda")
-        fn = lambda i: P.llvq_gemm_small_batch_sorted(ctx53, srt[i % 8], bufs[i % 8][1], n, k, x, d_y=y)
-        _event_us(torch, fn, 4)
-        us = _event_us(torch, fn, 16)
-        by = nb * (72 // 8 + 2) + batch * k * 2 + batch * n * 2
-        out[f"gemm_8192x8192_b{batch}_72bit_sorted_layout"] = {"us": us, "GBps": by / us / 1e3, "TFLOPs": 2.0 * n * k * batch / us / 1e6, "algorithmic_bytes": by}
+    for bits, cctx in ((48, ctx), (72, ctx53)):
+        for (n, k) in ((8192, 8192), (28672, 8192), (8192, 28672)):
+            stream, gain, nb = gen.make_layer(cctx.num_points, cctx.index_bits, n, k, 1, seed=200 + bits)
+            row_bytes = ((k + 23) // 24) * bits // 8
+            d_i0 = dev(stream)[: n * row_bytes].view(n, row_bytes)
+            d_g0 = dev(gain, np.float16).view(n, -1)
+            copies = max(2, -(-(3 * L2_BYTES // 2) // (nb * (bits // 8 + 2))))
+            bufs = []
+            for c in range(copies):
+                shift = 128 * (c * (n // 128) // copies)                      # whole row tiles
+                d_i = torch.zeros(cctx.index_bytes(nb), dtype=torch.uint8, device="cuda")
+                d_i[: n * row_bytes] = torch.roll(d_i0, shift, 0).reshape(-1)
+                d_g = torch.roll(d_g0, shift, 0).reshape(-1).contiguous()
+                bufs.append((d_i, d_g, P.llvq_sort_blocks_gemm(cctx, d_i, n, k)))
+            del d_i0, d_g0
+            for batch in (16, 64):
+                x = dev(gen.normal_bf16((batch, k), seed=batch), np.int16).view(torch.bfloat16)
+                y = torch.empty((batch, n), dtype=torch.bfloat16, device="cuda")
+                by = nb * (bits // 8 + 2) + batch * k * 2 + batch * n * 2
+                reps = 24 if n * k <= 8192 * 8192 else 8
+                for name, fn in (("", lambda i: P.llvq_gemm_small_batch(cctx, bufs[i % copies][0], bufs[i % copies][1], n, k, x, d_y=y)),
+                                 ("_sorted_layout", lambda i: P.llvq_gemm_small_batch_sorted(cctx, bufs[i % copies][2], bufs[i % copies][1], n, k, x, d_y=y))):
+                    _event_us(torch, fn, 3)
+                    us = _event_us(torch, fn, reps)
+                    out[f"gemm_{n}x{k}_b{batch}_{bits}bit{name}"] = {
+                        "us": us, "GBps": by / us / 1e3, "frac_of_hbm_peak": by / us / 1e3 / measured_peaks()[0],
+                        "TFLOPs": 2.0 * n * k * batch / us / 1e6, "algorithmic_bytes": by, "rotating_copies": copies}
+            del bufs
     assert P.llvq_last_error(ctx53) == (0, 0)
-    del bufs, srt, ctx53
+    del ctx53
     # --- decoder sweep: q, k, v, o, gate, up, down of one layer; 32 layers; 4 distinct layer sets (> 2 x L2)
     shapes = [(4096, 4096), (1024, 4096), (1024, 4096), (4096, 4096), (14336, 4096), (14336, 4096), (4096, 14336)]
     sets = []
@@ -345,6 +314,26 @@ def extras(P, ctx) -> dict:
         sets.append(layer)
     xs = {k: dev(gen.normal_bf16(k, seed=k), np.int16).view(torch.bfloat16) for k in (4096, 14336)}
     ys = {n: torch.empty(n, dtype=torch.bfloat16, device="cuda") for n in (4096, 1024, 14336)}
+
+    # whole-model bulk dequantization: the 7 matrices of each of the 32 layers through llvq_dequant_matrix (ROWWISE), the
+    # four layer sets and four sets of bf16 outputs (4 x 436 MB) visited in turn
+    w_out = [[torch.empty((n, k), dtype=torch.bfloat16, device="cuda") for (n, k) in shapes] for _ in range(4)]
+
+    def bulk(i):
+        for layer in range(32):
+            c = (i * 32 + layer) % 4
+            for (n, k), (d_idx, d_gain), d_w in zip(shapes, sets[c], w_out[c]):
+                P.llvq_dequant_matrix(ctx, d_idx, d_gain, n, k, 1, d_w=d_w)
+    bulk(0)
+    torch.cuda.synchronize()
+    bulk_us = _event_us(torch, bulk, 2)
+    del w_out
+    bulk_weights = 32 * sum(n * k for n, k in shapes)
+    bulk_bytes = 32 * sum(n * ((k + 23) // 24) for n, k in shapes) * (CODE_W // 8 + 2) + 2 * bulk_weights
+    out["llama3_8b_bulk_dequant"] = {"ms_per_model": bulk_us / 1e3, "weights_per_s": bulk_weights / (bulk_us * 1e-6),
+                                     "GBps": bulk_bytes / bulk_us / 1e3, "frac_of_hbm_peak": bulk_bytes / bulk_us / 1e3 / measured_peaks()[0],
+                                     "algorithmic_bytes": bulk_bytes, "launches": 32 * len(shapes),
+                                     "note": "index + gain bytes in, 2 bytes per weight out; the written matrices are 14 GB per pass"}
 
     def token(i):
         for layer in range(32):

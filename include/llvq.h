@@ -171,7 +171,7 @@ int llvq_gemm_small_batch_sg(const llvq_ctx* ctx, const void* d_fields, int gain
 
 /*
  * Sorted layout for the fused GEMV: a kernel-private arrangement of the same blocks, made once at load time (the
- * paper describes no storage layout beyond "a compact integer index" per block, Sec. 1, and App. A step 5 notes
+ * paper fixes no storage layout, only that every block is stored as one integer, Sec. 1; App. A step 5 notes
  * that blocks are independent, which is what makes reordering them legitimate).  llvq_sort_blocks rewrites a
  * ROWWISE index stream for the GPU of this context: the blocks each thread block of the GEMV will own are stored,
  * in segments of up to 65536 blocks, ordered by the form of App. A steps 3-4 their class needs (odd / even with

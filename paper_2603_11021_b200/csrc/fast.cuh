@@ -70,7 +70,15 @@ __device__ __forceinline__ bool fast_load_image(uint8_t* dst, const uint8_t* __r
         asm volatile("{\n .reg .pred p;\n mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n selp.u32 %0, 1, 0, p;\n}"
                      : "=r"(done) : "r"(bar_a), "r"(0u) : "memory");
     }
-    if (!done) atomicOr(err_flags, 1u);
+    if (!done) {
+        atomicOr(err_flags, 1u);
+        // the copy may still be writing this CTA's shared memory: give it the same limit once more before the caller returns
+        for (uint32_t it = 0; it < (1u << 20) && !done; ++it) {
+            asm volatile("{\n .reg .pred p;\n mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n selp.u32 %0, 1, 0, p;\n}"
+                         : "=r"(done) : "r"(bar_a), "r"(0u) : "memory");
+        }
+        done = 0;
+    }
     return __syncthreads_and((int)done) != 0;
 }
 

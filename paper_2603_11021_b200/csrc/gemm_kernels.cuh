@@ -77,8 +77,12 @@ gemm_kernel(FastArgs fa, const uint32_t* __restrict__ stream, const uint16_t* __
     const uint32_t b_stage = (uint32_t)ga.npad * kStageK * 2;
 
     pdl_launch_dependents();
-    if (!fast_load_image(smem, fa.image, fa.L.total, bar_img, fa.flags)) return;
-    pdl_wait();
+    const bool image_ok = fast_load_image(smem, fa.image, fa.L.total, bar_img, fa.flags);
+    pdl_wait();                                        // also when the image did not arrive: the dependents of this launch rely on it
+    if (!image_ok) {
+        if (kShard) shard_arrive(*ga.shard);           // the peers must not wait for this rank
+        return;
+    }
     const FastSmem T = fast_view(smem, fa.L);
     // Two groups of 512 threads fill alternate stages, each into its own buffers and its own accumulator
     // (TMEM columns [64 h, 64 h + npad)); the epilogue adds the two accumulators.
@@ -324,8 +328,12 @@ gemm_sorted_kernel(FastArgs fa, const unsigned long long* __restrict__ sorted, c
     uint8_t* b_buf = a_buf + (uint32_t)dpi * kDomStages * kAStage;         // [dpi * 2 stages] x npad * 192
 
     pdl_launch_dependents();
-    if (!fast_load_image(smem, fa.image, fa.L.total, bar_img, fa.flags)) return;
-    pdl_wait();
+    const bool image_ok = fast_load_image(smem, fa.image, fa.L.total, bar_img, fa.flags);
+    pdl_wait();                                        // also when the image did not arrive: the dependents of this launch rely on it
+    if (!image_ok) {
+        if (kShard) shard_arrive(*ga.shard);           // the peers must not wait for this rank
+        return;
+    }
     const FastSmem T = fast_view(smem, fa.L);
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     if (threadIdx.x == 0) {
@@ -515,8 +523,12 @@ gemm_pipe_kernel(FastArgs fa, const unsigned long long* __restrict__ sorted, con
     constexpr uint32_t kWorkers = kGemmThreads / 32 - 1;                   // 31 unranking warps
 
     pdl_launch_dependents();
-    if (!fast_load_image(smem, fa.image, fa.L.total, bar_img, fa.flags)) return;
-    pdl_wait();
+    const bool image_ok = fast_load_image(smem, fa.image, fa.L.total, bar_img, fa.flags);
+    pdl_wait();                                        // also when the image did not arrive: the dependents of this launch rely on it
+    if (!image_ok) {
+        if (kShard) shard_arrive(*ga.shard);           // the peers must not wait for this rank
+        return;
+    }
     const FastSmem T = fast_view(smem, fa.L);
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     if (threadIdx.x == 0) {

@@ -175,7 +175,7 @@ gemv_fast_kernel(FastArgs fa, const uint32_t* __restrict__ stream, const uint16_
                  int64_t n_out, int64_t k_in, int64_t bpr, const uint16_t* __restrict__ x, YOut yo,
                  float* __restrict__ scratch, uint32_t* __restrict__ counters)
 {
-    FAST_PROLOGUE();
+    FAST_PROLOGUE(if (kShard) shard_arrive(yo));
     const int64_t nq = (bpr + 3) / 4;                               // units along K
     uint32_t* xs = reinterpret_cast<uint32_t*>(staging);            // [nq * 4][12] packed bf16 pairs of x
     float* acc = reinterpret_cast<float*>(xs + nq * 48);            // [kGemvGroupsPerPass][8]
@@ -356,7 +356,7 @@ gemv_sorted_kernel(FastArgs fa, const unsigned long long* __restrict__ sorted, c
         if ((threadIdx.x & 15u) == 0u && ub + (int64_t)(threadIdx.x >> 5) < ue)
             asm volatile("prefetch.global.L2 [%0];" ::"l"(sorted + ub * 32 + threadIdx.x));
     }
-    FAST_PROLOGUE();
+    FAST_PROLOGUE(if (kShard) shard_arrive(yo));
     const int64_t nq = (bpr + 3) / 4;
     uint32_t* xs = reinterpret_cast<uint32_t*>(staging);            // [nq * 4][12] packed bf16 pairs of x
     float* acc = reinterpret_cast<float*>(xs + nq * 48);            // [kSortAccCopies][kGemvGroupsPerPass][8]: warps spread their adds over the copies
@@ -464,7 +464,7 @@ gemv_bin_kernel(FastArgs fa, const uint32_t* __restrict__ stream, const uint16_t
             if (!kSg) prefetch_span_l2(gain, b_first * 2, b_last * 2);
         }
     }
-    FAST_PROLOGUE();
+    FAST_PROLOGUE(if (kShard) shard_arrive(yo));
     const int64_t nq = (bpr + 3) / 4;
     uint32_t* xs = reinterpret_cast<uint32_t*>(staging);            // [nq * 4][12] packed bf16 pairs of x
     float* acc = reinterpret_cast<float*>(xs + nq * 48);            // [kSortAccCopies][kGemvGroupsPerPass][8]

@@ -140,13 +140,17 @@ __device__ __forceinline__ void prefetch_span_l2(const void* p, uint64_t first, 
         asm volatile("prefetch.global.L2 [%0];" ::"l"(base + o));
 }
 
-#define FAST_PROLOGUE()                                                                         \
+// The optional argument is what a kernel still owes its peers when the table image did not arrive (the row-sharded
+// kernels count themselves in so that the other ranks do not wait for them).  Also on that path the kernel waits for
+// its predecessor before it retires, so that its own programmatic dependent never passes its wait too early.
+#define FAST_PROLOGUE(...)                                                                      \
     extern __shared__ __align__(128) uint8_t smem[];                                            \
     uint64_t* bar = reinterpret_cast<uint64_t*>(smem + fa.L.total);                              \
     [[maybe_unused]] uint8_t* staging = smem + fa.L.total + 16;                                 \
     pdl_launch_dependents();                                                                    \
-    if (!fast_load_image(smem, fa.image, fa.L.total, bar, fa.flags)) return;                    \
+    const bool image_ok = fast_load_image(smem, fa.image, fa.L.total, bar, fa.flags);           \
     pdl_wait();                                                                                 \
+    if (!image_ok) { __VA_ARGS__; return; }                                                     \
     const FastSmem T = fast_view(smem, fa.L);
 
 template <bool kBig>

@@ -125,13 +125,9 @@ def test_gemv_sg_full_size_sampled_rows(lib, ctxs, codes):
     rs = gen.row_scales_f32(n_out, seed=1)
     x = gen.normal_bf16(k_in, seed=1)
     y = lib.llvq_gemv_sg(ctx, to_dev_u8(stream), bits, _f32(cb), _f32(rs), n_out, k_in, to_dev_bf16(x)).cpu().numpy()
-    rows = [0, 1, 7, 8, 2047, 2048, 4094, 4095] + list(range(100, 4096, 397))
-    ref = np.zeros(n_out)
-    for r in rows:
-        ref[r] = o.gemm_sg(stream, bits, cb, rs, n_out, k_in, x, rows=(r, 1))[r]
-    floor = 1e-3 * np.abs(ref[rows]).max()
-    err = np.max(np.abs(y[rows] - ref[rows]) / np.maximum(np.abs(ref[rows]), floor))
-    assert err <= TOL
+    import os
+    ref = o.gemm_sg(stream, bits, cb, rs, n_out, k_in, x, threads=os.cpu_count() or 1)     # every output row
+    assert gemv_error(y, ref) <= TOL
     assert lib.llvq_last_error(ctx) == (0, 0)
 
 
@@ -191,9 +187,10 @@ def test_gemv_sorted_sg_full_size_and_limits(lib, ctxs, codes):
     # two binary32 sums of the same 4096 products in different (and, through the shared-memory atomics, run-dependent)
     # orders; relative to the floor of 1e-3 of the largest output a small row's sum can move by about 1e-4
     assert gemv_error(y, y2.astype(np.float64)) <= 5e-4
-    rows = [0, 9, 2047, 4095] + list(range(123, 4096, 611))
-    ref = np.array([o.gemm_sg(stream, bits, cb, rs, n_out, k_in, x, rows=(r, 1))[r] for r in rows])
-    assert gemv_error(y[rows], ref) <= TOL
+    import os
+    ref = o.gemm_sg(stream, bits, cb, rs, n_out, k_in, x, threads=os.cpu_count() or 1)     # every output row, both kernels
+    assert gemv_error(y, ref) <= TOL
+    assert gemv_error(y2, ref) <= TOL
     # 47 + 2 bits do not fit the 48-bit entry
     buf = torch.zeros(4096, dtype=torch.uint8, device="cuda")
     assert ctx._lib.llvq_sort_blocks_sg(ctx._h, buf.data_ptr(), 2, 8, 24, buf.data_ptr(), None) == 3

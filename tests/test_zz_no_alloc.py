@@ -3,9 +3,12 @@
 Some callers of this library may only launch work: all device memory already belongs to their own pool,
 or they sit in a decode loop that cannot afford the device-wide synchronisation an allocation implies.
 For them `llvq_gemm_small_batch_noalloc` keeps its split-K scratch in an array built into the library.
-This file checks, through the C ABI, that it returns what `llvq_gemm_small_batch` returns, twice in a row
-(the built-in array is shared by all calls and keeps old contents, so the second call proves it is cleared),
-and that it refuses sizes the array cannot hold.  It is named to be collected last.
+This file checks, through the C ABI, that it returns what `llvq_gemm_small_batch` returns and what the CPU
+oracle computes, twice in a row with different activations (the built-in array is shared by all calls, so the
+second call runs on whatever the first one left there), and that it refuses sizes the array cannot hold.
+The kernels themselves hand every scratch word they touch back as zero, so the clearing the entry point does
+before each launch only matters after a call that was cut short; no test provokes that.  The file is named to be
+collected last.
 """
 import numpy as np
 import pytest
@@ -20,6 +23,8 @@ pytestmark = pytest.mark.gpu
 # moves a bf16 output by at most one rounding step: 2^-7 of its value when it sits just above a power of two (both
 # sides are bf16 here, so the step is the full spacing, not the half spacing of a comparison with an exact value)
 TOL = 2.0 ** -7
+# against the binary64 oracle: binary32 accumulation (1e-3) plus the rounding of the bf16 output
+TOL_ORACLE = 1e-3 + 2.0 ** -8
 
 
 def _rel_err(a, ref):
@@ -28,7 +33,7 @@ def _rel_err(a, ref):
 
 
 @pytest.mark.parametrize("n_out,k_in,batch", [(640, 2048, 16), (300, 1000, 64)])
-def test_noalloc_gemm_matches_regular_entry_point_twice(n_out, k_in, batch):
+def test_noalloc_gemm_matches_regular_entry_point_and_oracle_twice(n_out, k_in, batch, code_2_13):
     import paper_2603_11021_b200 as P
     assert torch.cuda.is_available(), "needs a CUDA device; there is no CPU path"
     ctx = P.Context(2, 13, device=0)
@@ -45,6 +50,8 @@ def test_noalloc_gemm_matches_regular_entry_point_twice(n_out, k_in, batch):
         got = y_new.float().cpu().numpy()
         assert np.isfinite(got).all()
         assert _rel_err(got, want) <= TOL, f"call {call}"
+        ref = code_2_13.gemm(stream, gain, n_out, k_in, X, threads=4)
+        assert _rel_err(got, ref) <= TOL_ORACLE, f"call {call} against the oracle"
     assert P.llvq_last_error(ctx) == (0, 0)
 
 
