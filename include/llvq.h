@@ -190,6 +190,29 @@ int llvq_sort_blocks(const llvq_ctx* ctx, const void* d_idx, int64_t n_out, int6
 int llvq_gemv_sorted(const llvq_ctx* ctx, const void* d_sorted, const uint16_t* d_gain_f16,
                      int64_t n_out, int64_t k_in, const uint16_t* d_x_bf16,
                      void* d_y, int y_dtype, void* stream);
+
+/*
+ * Several independent products y_i = W_i x_i in one launch (App. C's fused product, applied to the matrices of a
+ * decoder layer that read the same or unrelated inputs: q, k and v; gate and up).  Blocks, and therefore matrices,
+ * are independent (App. A step 5), so the thread blocks take their share of each matrix in turn and the fixed cost
+ * of a launch (table staging, first loads, drain) is paid once.  No output may be an input of another matrix of the
+ * same call.  descs: HOST array of n_mats (1..8) descriptions; every pointer inside is a device pointer owned by the
+ * caller with the alignment llvq_gemv / llvq_gemv_sorted ask for; d_weights is the stored index stream
+ * (llvq_gemv_multi) or the stream made by llvq_sort_blocks (llvq_gemv_sorted_multi).  All outputs have type
+ * y_dtype.  The descriptions are copied into the launch, nothing is kept.  Results are those of the single calls (the
+ * same kernels' code runs per matrix).  LLVQ_EUNSUPPORTED: more than 8 matrices, a code or a k_in the single call does
+ * not take in this form either, a matrix with fewer 8-row x 4-block units than the device has SMs, or more than
+ * 64 * 65536 output rows in total.
+ */
+typedef struct {
+    const void* d_weights;
+    const uint16_t* d_gain_f16;     /* [n_out * ceil(k_in / 24)] ROWWISE */
+    int64_t n_out, k_in;
+    const uint16_t* d_x_bf16;       /* [k_in] */
+    void* d_y;                      /* [n_out] */
+} llvq_gemv_desc;
+int llvq_gemv_multi(const llvq_ctx* ctx, const llvq_gemv_desc* descs, int n_mats, int y_dtype, void* stream);
+int llvq_gemv_sorted_multi(const llvq_ctx* ctx, const llvq_gemv_desc* descs, int n_mats, int y_dtype, void* stream);
 /*
  * The same for the shape-gain form: llvq_sort_blocks_sg sorts a stream of fields of llvq_index_bits(ctx) + gain_bits
  * bits (at most 48 in all: the entry keeps the whole field, shape index and gain index), llvq_gemv_sorted_sg computes

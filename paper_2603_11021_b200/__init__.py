@@ -61,6 +61,12 @@ class LlvqError(RuntimeError):
 _lib = None
 
 
+class GemvDesc(ctypes.Structure):
+    """llvq_gemv_desc of include/llvq.h: one matrix of a multi-matrix GEMV call."""
+    _fields_ = [("d_weights", ctypes.c_void_p), ("d_gain_f16", ctypes.c_void_p), ("n_out", ctypes.c_int64), ("k_in", ctypes.c_int64),
+                ("d_x_bf16", ctypes.c_void_p), ("d_y", ctypes.c_void_p)]
+
+
 def load_library() -> ctypes.CDLL:
     """Load libllvq.so (built in-tree by ``paper_2603_11021_b200.build``); raises if it is missing."""
     global _lib
@@ -92,6 +98,8 @@ def load_library() -> ctypes.CDLL:
     lib.llvq_sorted_bytes.restype = ctypes.c_size_t
     lib.llvq_sort_blocks.argtypes = [vp, vp, i64, i64, vp, vp]
     lib.llvq_gemv_sorted.argtypes = [vp, vp, vp, i64, i64, vp, vp, ctypes.c_int, vp]
+    lib.llvq_gemv_multi.argtypes = [vp, ctypes.POINTER(GemvDesc), ctypes.c_int, ctypes.c_int, vp]
+    lib.llvq_gemv_sorted_multi.argtypes = [vp, ctypes.POINTER(GemvDesc), ctypes.c_int, ctypes.c_int, vp]
     lib.llvq_gemm_small_batch_sg.argtypes = [vp, vp, ctypes.c_int, vp, vp, i64, i64, vp, ctypes.c_int, vp, vp]
     lib.llvq_sort_blocks_gemm_sg.argtypes = [vp, vp, ctypes.c_int, i64, i64, vp, vp]
     lib.llvq_gemm_small_batch_sorted_sg.argtypes = [vp, vp, ctypes.c_int, vp, vp, i64, i64, vp, ctypes.c_int, vp, vp]
@@ -343,6 +351,27 @@ def llvq_gemv_sorted(ctx: Context, d_sorted: torch.Tensor, d_gain: torch.Tensor,
     _check("llvq_gemv_sorted", ctx._lib.llvq_gemv_sorted(ctx._h, _dev(d_sorted, "d_sorted"), _dev(d_gain, "d_gain"), n_out, k_in,
                                                          _dev(d_x, "d_x"), _dev(d_y, "d_y"), code, _stream_ptr(stream)))
     return d_y
+
+
+def _gemv_multi(call: str, ctx: Context, mats, y_dtype, stream):
+    descs = (GemvDesc * len(mats))()
+    for d, (d_w, d_gain, n_out, k_in, d_x, d_y) in zip(descs, mats):
+        assert d_x.dtype == torch.bfloat16 and d_x.numel() >= k_in and d_gain.dtype == torch.float16
+        assert d_y.dtype == y_dtype and d_y.numel() >= n_out and d_gain.numel() >= n_out * ((k_in + 23) // 24)
+        d.d_weights, d.d_gain_f16, d.n_out, d.k_in = _dev(d_w, "d_weights"), _dev(d_gain, "d_gain"), n_out, k_in
+        d.d_x_bf16, d.d_y = _dev(d_x, "d_x"), _dev(d_y, "d_y")
+    _check(call, getattr(ctx._lib, call)(ctx._h, descs, len(mats), LLVQ_F32 if y_dtype == torch.float32 else LLVQ_BF16, _stream_ptr(stream)))
+
+
+def llvq_gemv_multi(ctx: Context, mats, y_dtype: torch.dtype = torch.float32, stream=None) -> None:
+    """Up to 8 independent products in one launch.  mats: (d_idx, d_gain, n_out, k_in, d_x, d_y) per matrix, all device tensors
+    owned by the caller (outputs included); no d_y may be a d_x of the same call."""
+    _gemv_multi("llvq_gemv_multi", ctx, mats, y_dtype, stream)
+
+
+def llvq_gemv_sorted_multi(ctx: Context, mats, y_dtype: torch.dtype = torch.float32, stream=None) -> None:
+    """The same on streams made by ``llvq_sort_blocks``: (d_sorted, d_gain, n_out, k_in, d_x, d_y) per matrix."""
+    _gemv_multi("llvq_gemv_sorted_multi", ctx, mats, y_dtype, stream)
 
 
 def llvq_sort_blocks_sg(ctx: Context, d_fields: torch.Tensor, gain_bits: int, n_out: int, k_in: int,

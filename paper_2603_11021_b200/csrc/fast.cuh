@@ -23,10 +23,14 @@ struct FastSmem {
     const uint8_t* pd6;
     const uint64_t* off;
     const uint32_t* desc;
+    uint32_t sub3;            // shared-window byte address of the table of small subsets, 0 when the kernel did not load it
     uint32_t lut_shift;
 };
 
-__device__ __forceinline__ FastSmem fast_view(const uint8_t* smem, const FastLayout& L)
+__device__ __forceinline__ uint32_t smem_addr(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+// with_small_subsets: the kernel loaded L.total_ext bytes of the image, not only L.total
+__device__ __forceinline__ FastSmem fast_view(const uint8_t* smem, const FastLayout& L, bool with_small_subsets = false)
 {
     FastSmem T;
     T.golay = reinterpret_cast<const uint32_t*>(smem + L.golay);
@@ -37,11 +41,10 @@ __device__ __forceinline__ FastSmem fast_view(const uint8_t* smem, const FastLay
     T.pd6 = smem + L.pd6;
     T.off = reinterpret_cast<const uint64_t*>(smem + L.off);
     T.desc = reinterpret_cast<const uint32_t*>(smem + L.desc);
+    T.sub3 = with_small_subsets ? smem_addr(smem + L.sub3) : 0u;
     T.lut_shift = L.lut_shift;
     return T;
 }
-
-__device__ __forceinline__ uint32_t smem_addr(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 
 // Copy the table image into shared memory with bulk asynchronous copies (TMA,
 // no multicast) tracked by one mbarrier.  Every thread of the CTA must call this.
@@ -126,6 +129,29 @@ __device__ __forceinline__ uint32_t nth_subset(const FastSmem& T, uint32_t k, ui
     return m | (uint32_t)T.r14[first + rho];
 }
 
+// The rho-th k-subset of up to 24 slots for k <= 3: one lookup behind a four-word directory (T.sub3 != 0).
+__device__ __forceinline__ uint32_t small_subset(const FastSmem& T, uint32_t k, uint32_t rho)
+{
+    uint32_t first, m;
+    asm volatile("ld.shared.u32 %0, [%1];" : "=r"(first) : "r"(T.sub3 + k * 4u));
+    asm volatile("ld.shared.u32 %0, [%1];" : "=r"(m) : "r"(T.sub3 + (first + rho) * 4u));
+    return m;
+}
+
+// Deposit into a mask that is 24 ones with at most two holes: open a gap at each hole, lowest first.
+__device__ __forceinline__ uint32_t deposit_two_holes(uint32_t src, uint32_t mask)
+{
+    uint32_t holes = ~mask & 0xffffffu;
+#pragma unroll
+    for (int i = 0; i < 2; ++i) {
+        const uint32_t b = holes & (0u - holes);          // lowest hole, or 0: then nothing moves
+        const uint32_t low = b - 1u;
+        src = (src & low) | ((src & ~low) << 1);
+        holes ^= b;
+    }
+    return src;
+}
+
 // Result of the index -> point map in a form the consumers expand cheaply:
 // three bit planes giving each position a value id (0..7), the table of
 // absolute values per id, and the mask of negative positions.
@@ -147,6 +173,7 @@ __device__ __forceinline__ uint32_t fast_find_class(const FastSmem& T, uint64_t 
 // S3-S6.  `mask` = the lanes of the warp that call this together.  kPar = -1: any class.  kPar = 1: all calling lanes
 // hold odd classes.  kPar = 0: all calling lanes hold even classes of Golay weight 8, 12 or 16 (both slot groups have
 // at most 16 slots).  The specialised forms drop the work the other parity needs (slot decisions above 16, sign deposits).
+// Writes d only where `valid`: the caller presets it (zeros for "no block").
 template <int kPar>
 __device__ __forceinline__ void fast_decode_local(const FastSmem& T, uint32_t cls, uint64_t local, bool valid, uint32_t mask, Decoded& d)
 {
@@ -156,6 +183,8 @@ __device__ __forceinline__ void fast_decode_local(const FastSmem& T, uint32_t cl
     const uint32_t nlev1 = kPar == 1 ? 0u : (h.x >> 24) & 0xf, nlev = valid ? h.x >> 28 : 0u;
     const uint32_t goff = h.y & 0xffff, A = h.y >> 16;
     const bool odd = kPar == 1 || (kPar == -1 && (flags & 1u));
+    // the arrangement rank of every calling lane fits 32 bits (all but the largest class of the 48-bit code): no 64-bit division
+    const bool rank32 = kPar != -1 && __all_sync(mask, !valid || (flags & kFastFlagRank32));
 
     // S3: r fastest, then the sign word s, then the arrangement rank p
     uint64_t q;
@@ -179,7 +208,7 @@ __device__ __forceinline__ void fast_decode_local(const FastSmem& T, uint32_t cl
     uint32_t freem = kPar == 1 ? 0xffffffu : F1;
     bool in_group0 = kPar == 1;
     uint32_t p0 = 0, p1 = 0, p2 = 0, bit1 = 0, nz0 = 0;
-    uint32_t p32 = 0;
+    uint32_t p32 = (uint32_t)p;
     const uint32_t lwords[4] = {lw.x, lw.y, lw.z, lw.w};
     const uint32_t magics[4] = {0u, mg.x, mg.y, mg.z};
     const int maxlev = __reduce_max_sync(mask, nlev);
@@ -195,25 +224,34 @@ __device__ __forceinline__ void fast_decode_local(const FastSmem& T, uint32_t cl
             const uint32_t word = lwords[l];
             const uint32_t radix = word & 0x3fffffu;
             const uint32_t k = active ? (word >> 22) & 31u : 0u;
+            const uint32_t nfree = (mg.w >> (8 * l)) & 0xffu;            // slots free before this step
             uint32_t rho;
-            if (l == 0) {
+            if (l == 0 && !rank32) {
                 uint64_t qq = __umul64hi(p, ((uint64_t)v.w << 32) | v.z);
                 uint64_t rem = p - qq * radix;
                 if (rem >= radix) { rem -= radix; ++qq; }
                 p32 = (uint32_t)qq; rho = (uint32_t)rem;
             } else {
-                uint32_t qq = __umulhi(p32, magics[l]);
+                uint32_t qq = __umulhi(p32, l == 0 ? T.desc[cls * kFastDescStride + kFastDescMagic0] : magics[l]);
                 uint32_t rem = p32 - qq * radix;
                 if (rem >= radix) { rem -= radix; ++qq; }
                 p32 = qq; rho = rem;
             }
             if (!active) rho = 0u;
-            int top;
-            if (kPar == 0) top = 16;
-            else if (kPar == 1 && l == 0) top = 24;
-            else top = __reduce_max_sync(mask, active ? (mg.w >> (8 * l)) & 0xffu : 0u);
-            const uint32_t rel = nth_subset(T, k, rho, top);
-            const uint32_t a = (kPar == 1 && l == 0) ? rel : deposit24(T.pd6, rel, freem);   // odd, first step: every position is free
+            uint32_t rel;
+            if (T.sub3 != 0u && __all_sync(mask, k <= (uint32_t)kSmallSubsetMaxK)) {
+                rel = small_subset(T, k, rho);                          // few elements: one lookup whatever the number of slots
+            } else {
+                int top;
+                if (kPar == 0) top = 16;
+                else if (kPar == 1 && l == 0) top = 24;
+                else top = __reduce_max_sync(mask, active ? nfree : 0u);
+                rel = nth_subset(T, k, rho, top);
+            }
+            uint32_t a;
+            if (kPar == 1 && l == 0) a = rel;                           // odd, first step: every position is free
+            else if (kPar == 1 && l == 1 && __all_sync(mask, !active || nfree >= 22u)) a = deposit_two_holes(rel, freem);
+            else a = deposit24(T.pd6, rel, freem);
             freem ^= a;
             if (word & (1u << 27)) p0 |= a;
             if (word & (1u << 28)) p1 |= a;
@@ -241,13 +279,15 @@ __device__ __forceinline__ void fast_decode_local(const FastSmem& T, uint32_t cl
         const uint32_t neg_even = deposit24(T.pd6, src1, F1) | deposit24(T.pd6, s >> nf1, odd ? 0u : nz0);
         neg = odd ? (c ^ bit1) : neg_even;
     }
-    if (!valid) { p0 = p1 = p2 = 0; neg = 0; }
-    d.p0 = p0; d.p1 = p1; d.p2 = p2; d.neg = neg;
-    d.vals_lo = valid ? v.x : 0u; d.vals_hi = valid ? v.y : 0u;
+    if (valid) {
+        d.p0 = p0; d.p1 = p1; d.p2 = p2; d.neg = neg;
+        d.vals_lo = v.x; d.vals_hi = v.y;
+    }
 }
 
 __device__ __forceinline__ void fast_decode(const FastSmem& T, uint64_t I, bool valid, Decoded& d)
 {
+    d.p0 = d.p1 = d.p2 = d.neg = d.vals_lo = d.vals_hi = 0u;
     uint64_t local = 0;
     const uint32_t cls = valid ? fast_find_class(T, I, local) : 0u;
     fast_decode_local<-1>(T, cls, local, valid, kFullMask, d);

@@ -1,7 +1,7 @@
 // The fused dequant + small-batch GEMM kernels (tcgen05, accumulator in tensor memory): the kernel with two thread
 // groups on alternating stages, the sorted layouts (sort kernels and the consumer with a block barrier), and the
-// kernel without a block barrier that both entry points run for the 48-bit codes.  Included by llvq.cu inside its
-// unnamed namespace, after gemv_kernels.cuh (YOut, unit_owner, shard_arrive); no other file includes it.
+// kernel without a block barrier that both entry points run for the 48-bit codes.  Included by gemm.cu inside its
+// unnamed namespace, after kernels_common.cuh and gemv_kernels.cuh (unit_owner, shard_arrive).
 #pragma once
 
 // ===========================================================================
@@ -16,11 +16,8 @@
 // ===========================================================================
 constexpr int kGemmThreads = 1024;
 constexpr int kGemmGroupThreads = 512;
-constexpr int kGemmRows = 128;
 constexpr int kStageBlocks = 4;                       // column blocks per stage
 constexpr int kStageK = kStageBlocks * 24;            // 96
-constexpr int kMaxScratchRows = 65536;
-constexpr int kCounterWords = 64 * kMaxScratchRows / 8;      // the word after them counts the CTAs of a row-sharded GEMV that have finished
 constexpr uint32_t kTmemCols = 128;
 
 struct GemmArgs {
@@ -65,7 +62,7 @@ __global__ void __launch_bounds__(kGemmThreads, 1)
 gemm_kernel(FastArgs fa, const uint32_t* __restrict__ stream, const uint16_t* __restrict__ gain, SgArgs sg, GemmArgs ga)
 {
     extern __shared__ __align__(128) uint8_t smem[];
-    const uint32_t img_bytes = fa.L.total;
+    const uint32_t img_bytes = fa.image_bytes;
     uint64_t* bar_img = reinterpret_cast<uint64_t*>(smem + img_bytes);
     uint64_t* bar_free = bar_img + 1;                                     // [2]: the MMAs reading group h's buffers are done
     uint64_t* bar_done = bar_img + 3;                                     // [2]: group h's accumulator of this item is complete
@@ -77,7 +74,7 @@ gemm_kernel(FastArgs fa, const uint32_t* __restrict__ stream, const uint16_t* __
     const uint32_t b_stage = (uint32_t)ga.npad * kStageK * 2;
 
     pdl_launch_dependents();
-    const bool image_ok = fast_load_image(smem, fa.image, fa.L.total, bar_img, fa.flags);
+    const bool image_ok = fast_load_image(smem, fa.image, fa.image_bytes, bar_img, fa.flags);
     pdl_wait();                                        // also when the image did not arrive: the dependents of this launch rely on it
     if (!image_ok) {
         if (kShard) shard_arrive(*ga.shard);           // the peers must not wait for this rank
@@ -315,7 +312,7 @@ __global__ void __launch_bounds__(kGemmThreads, 1)
 gemm_sorted_kernel(FastArgs fa, const unsigned long long* __restrict__ sorted, const uint16_t* __restrict__ gain, SgArgs sg, GemmArgs ga, int dpi)
 {
     extern __shared__ __align__(128) uint8_t smem[];
-    const uint32_t img_bytes = fa.L.total;
+    const uint32_t img_bytes = fa.image_bytes;
     uint64_t* bar_img = reinterpret_cast<uint64_t*>(smem + img_bytes);
     uint64_t* bar_free = bar_img + 1;                                     // the MMAs reading the A / B buffers are done
     uint64_t* bar_done = bar_img + 2;                                     // the accumulator of this item is complete
@@ -328,7 +325,7 @@ gemm_sorted_kernel(FastArgs fa, const unsigned long long* __restrict__ sorted, c
     uint8_t* b_buf = a_buf + (uint32_t)dpi * kDomStages * kAStage;         // [dpi * 2 stages] x npad * 192
 
     pdl_launch_dependents();
-    const bool image_ok = fast_load_image(smem, fa.image, fa.L.total, bar_img, fa.flags);
+    const bool image_ok = fast_load_image(smem, fa.image, fa.image_bytes, bar_img, fa.flags);
     pdl_wait();                                        // also when the image did not arrive: the dependents of this launch rely on it
     if (!image_ok) {
         if (kShard) shard_arrive(*ga.shard);           // the peers must not wait for this rank
@@ -398,7 +395,7 @@ gemm_sorted_kernel(FastArgs fa, const unsigned long long* __restrict__ sorted, c
                         w[j] = *reinterpret_cast<uint32_t*>(&h);
                     }
                 } else {
-                    Decoded dec;
+                    Decoded dec{};
                     const uint32_t cls = decode_sorted_entry(fa, T, I, valid, dec);
                     if (kSg && valid) {
                         const float scale = sg.row_scale ? __ldg(sg.row_scale + row) : 1.f;
@@ -507,7 +504,7 @@ gemm_pipe_kernel(FastArgs fa, const unsigned long long* __restrict__ sorted, con
 {
     static_assert(!(kStored && kBig && kSg), "no shape-gain form for the codes with tables in global memory");
     extern __shared__ __align__(128) uint8_t smem[];
-    const uint32_t img_bytes = fa.L.total;
+    const uint32_t img_bytes = fa.image_bytes;
     uint64_t* bar_img = reinterpret_cast<uint64_t*>(smem + img_bytes);
     uint64_t* bar_full = bar_img + 1;                                     // [2] 32 chunks of A and the X slice are in the buffer
     uint64_t* bar_free = bar_img + 3;                                     // [2] the MMAs reading the buffer are done
@@ -523,7 +520,7 @@ gemm_pipe_kernel(FastArgs fa, const unsigned long long* __restrict__ sorted, con
     constexpr uint32_t kWorkers = kGemmThreads / 32 - 1;                   // 31 unranking warps
 
     pdl_launch_dependents();
-    const bool image_ok = fast_load_image(smem, fa.image, fa.L.total, bar_img, fa.flags);
+    const bool image_ok = fast_load_image(smem, fa.image, fa.image_bytes, bar_img, fa.flags);
     pdl_wait();                                        // also when the image did not arrive: the dependents of this launch rely on it
     if (!image_ok) {
         if (kShard) shard_arrive(*ga.shard);           // the peers must not wait for this rank
@@ -664,7 +661,7 @@ gemm_pipe_kernel(FastArgs fa, const unsigned long long* __restrict__ sorted, con
                         w[jj] = *reinterpret_cast<uint32_t*>(&h);
                     }
                 } else {
-                    Decoded dec;
+                    Decoded dec{};
                     uint32_t cls;
                     if (kStored) {
                         if (field != kSortIndexMask && !valid) atomicAdd(fa.bad_index, 1ull);

@@ -1,6 +1,6 @@
 // The fused dequant + GEMV kernels: the direct kernel (tensor-core reduction), the sorted layout (sort kernel and
-// consumer) and the kernel that bins a segment's blocks by class itself.  Included by llvq.cu inside its unnamed
-// namespace, after FastArgs, block_pairs and FAST_PROLOGUE; no other file includes it.
+// consumer) and the kernel that bins a segment's blocks by class itself.  Included by gemv.cu and gemm.cu inside their
+// unnamed namespaces, after kernels_common.cuh.
 #pragma once
 
 // Fused dequant + GEMV.  The work is cut into units of 8 rows x 4 column blocks, numbered row group major, and
@@ -9,8 +9,6 @@
 // zero) of six m16n8k16 tensor-core MMAs whose B fragment carries the matching 4 x 24 activations (the same in
 // all 8 columns), accumulating in binary32.  Row sums are collected in shared memory; a row group that is
 // split between CTAs is finished through a zero-kept global scratch and an arrival counter.
-constexpr int kGemvGroupRows = 8;        // rows per unit
-constexpr int kGemvGroupsPerPass = 128;  // row groups whose sums a CTA keeps in shared memory at a time
 
 __device__ __forceinline__ void mma_bf16_16816(float c[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0, uint32_t b1)
 {
@@ -20,24 +18,6 @@ __device__ __forceinline__ void mma_bf16_16816(float c[4], uint32_t a0, uint32_t
 
 // CTA that owns unit u when G CTAs split U units into ranges [c*U/G, (c+1)*U/G).
 __device__ __forceinline__ int64_t unit_owner(int64_t u, int64_t U, int64_t G) { return ((u + 1) * G - 1) / U; }
-
-// Where a GEMV kernel puts y.  Row-sharded over several GPUs (each rank owns a band of output rows, x is the same
-// everywhere), a rank writes its band straight into every rank's copy of the full vector: `y` is this rank's copy
-// and `peer` the other ranks' copies mapped into this process, every pointer already advanced to the band's first
-// row.  The stores to a peer travel over NVLink as plain remote writes.  n_peer = 0 is the single-GPU case.
-constexpr int64_t kPairSlotOffset = 64ll * 65536;      // floats: the 64-bit slots of finish_pass lie behind the binary32 scratch rows
-constexpr int kMaxShardPeers = 7;
-struct YOut {
-    void* y;
-    void* peer[kMaxShardPeers];
-    int n_peer;
-    // optional: one word per peer that receives `epoch` once the whole grid has stored its rows (done = the
-    // context's arrival counter, zero between launches)
-    uint32_t* flag[kMaxShardPeers];
-    uint32_t* done;
-    uint32_t epoch;
-    int n_flag;
-};
 
 template <bool kOutBf16, bool kShard>
 __device__ __forceinline__ void store_y(const YOut& yo, int64_t row, float v)
@@ -97,10 +77,11 @@ __device__ __forceinline__ void stage_x(uint32_t* xs, const uint16_t* __restrict
 // whoever arrives last reads the total, writes y and leaves scratch and counter zero for the next launch (groups shared
 // by exactly two CTAs take a shorter way, below).
 // The caller puts a __syncthreads() before (sums complete) and after (sums may be cleared) the call.
+// slot0 (a multiple of 8) = first scratch row / pair slot of this matrix when one launch works on several matrices.
 template <bool kOutBf16, bool kShard, typename RowSum>
 __device__ __forceinline__ void finish_pass(const YOut& yo, int64_t rg0, int64_t rg1, int64_t nq, int64_t u_begin, int64_t u_end,
                                             int64_t U, int64_t G, int64_t n_out, float* __restrict__ scratch,
-                                            uint32_t* __restrict__ counters, RowSum row_sum)
+                                            uint32_t* __restrict__ counters, RowSum row_sum, int64_t slot0 = 0)
 {
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, nwarps = (int)(blockDim.x >> 5);
     for (int64_t rg = rg0 + warp; rg <= rg1; rg += nwarps) {
@@ -121,7 +102,7 @@ __device__ __forceinline__ void finish_pass(const YOut& yo, int64_t rg0, int64_t
             // and the arrival.  Whoever finds the slot empty leaves (its sum, 1) there; the other gets that back from
             // its failed swap, adds its own sum, stores y and empties the slot.  One round trip each, no fence.
             if (mine) {
-                unsigned long long* slot = reinterpret_cast<unsigned long long*>(scratch + kPairSlotOffset) + row;
+                unsigned long long* slot = reinterpret_cast<unsigned long long*>(scratch + kPairSlotOffset) + slot0 + row;
                 const unsigned long long seen = atomicCAS(slot, 0ull, (unsigned long long)__float_as_uint(part) | 1ull << 32);
                 if (seen != 0ull) {
                     store_y<kOutBf16, kShard>(yo, row, __fadd_rn(__uint_as_float((uint32_t)seen), part));
@@ -131,23 +112,23 @@ __device__ __forceinline__ void finish_pass(const YOut& yo, int64_t rg0, int64_t
             }
             continue;
         }
-        if (mine) atomicAdd(scratch + row, part);
+        if (mine) atomicAdd(scratch + slot0 + row, part);
         __threadfence();                               // every lane's add is performed before ...
         __syncwarp();
         uint32_t is_last = 0u;
         if (lane == 0) {
             __threadfence();                           // ... lane 0 counts the arrival
-            is_last = atomicAdd(counters + rg, 1u) == parts - 1u;
+            is_last = atomicAdd(counters + slot0 / kGemvGroupRows + rg, 1u) == parts - 1u;
         }
         is_last = __shfl_sync(kFullMask, is_last, 0);
         if (is_last) {
             __threadfence();
             if (mine) {
-                store_y<kOutBf16, kShard>(yo, row, __ldcg(scratch + row));
-                __stcg(scratch + row, 0.f);
+                store_y<kOutBf16, kShard>(yo, row, __ldcg(scratch + slot0 + row));
+                __stcg(scratch + slot0 + row, 0.f);
                 if (kShard) __threadfence_system();
             }
-            if (lane == 0) counters[rg] = 0u;
+            if (lane == 0) counters[slot0 / kGemvGroupRows + rg] = 0u;
         }
     }
 }
@@ -167,6 +148,20 @@ __device__ __forceinline__ void shard_arrive(const YOut& yo)
 #pragma unroll
     for (int p = 0; p < kMaxShardPeers; ++p)
         if (p < yo.n_flag) asm volatile("st.release.sys.global.u32 [%0], %1;" ::"l"(yo.flag[p]), "r"(yo.epoch) : "memory");
+}
+
+// sum_j w_j x_j over 12 packed bf16 pairs with binary32 accumulation: fma.rn.f32.bf16 takes the bf16 halves as they are
+// (products of two bf16 values are exact in binary32, so this is the chain of 24 binary32 FMAs without the unpacking).
+__device__ __forceinline__ float dot24_bf16(const uint32_t w[12], const uint32_t x[12])
+{
+    float s0 = 0.f, s1 = 0.f;
+#pragma unroll
+    for (int j = 0; j < 12; ++j) {
+        asm("{\n .reg .b16 wl, wh, xl, xh;\n mov.b32 {wl, wh}, %2;\n mov.b32 {xl, xh}, %3;\n"
+            " fma.rn.f32.bf16 %0, wl, xl, %0;\n fma.rn.f32.bf16 %1, wh, xh, %1;\n}"
+            : "+f"(s0), "+f"(s1) : "r"(w[j]), "r"(x[j]));
+    }
+    return s0 + s1;
 }
 
 template <bool kBig, bool kOutBf16, bool kSg = false, bool kShard = false>
@@ -317,22 +312,19 @@ __device__ __forceinline__ void decode_known_class(const FastSmem& T, uint32_t c
     const uint32_t h = T.desc[cls * kFastDescStride];
     const uint32_t w8 = h & 0xffu;
     const uint32_t kind = !valid ? kKindNull : ((h & (1u << 16)) ? kKindOdd : ((w8 == 8u || w8 == 12u || w8 == 16u) ? kKindEven : kKindOther));
-    Decoded d;
     r.p0 = r.p1 = r.p2 = r.neg = r.vals_lo = r.vals_hi = 0u;
+    // every form writes r only for its own lanes
     if (__any_sync(kFullMask, kind == kKindOdd)) {
         const bool mine = kind == kKindOdd;
-        fast_decode_local<1>(T, mine ? cls : 0u, mine ? local : 0ull, mine, kFullMask, d);
-        if (mine) r = d;
+        fast_decode_local<1>(T, mine ? cls : 0u, mine ? local : 0ull, mine, kFullMask, r);
     }
     if (__any_sync(kFullMask, kind == kKindEven)) {
         const bool mine = kind == kKindEven;
-        fast_decode_local<0>(T, mine ? cls : 0u, mine ? local : 0ull, mine, kFullMask, d);
-        if (mine) r = d;
+        fast_decode_local<0>(T, mine ? cls : 0u, mine ? local : 0ull, mine, kFullMask, r);
     }
     if (__any_sync(kFullMask, kind == kKindOther)) {
         const bool mine = kind == kKindOther;
-        fast_decode_local<-1>(T, mine ? cls : 0u, mine ? local : 0ull, mine, kFullMask, d);
-        if (mine) r = d;
+        fast_decode_local<-1>(T, mine ? cls : 0u, mine ? local : 0ull, mine, kFullMask, r);
     }
 }
 
@@ -344,19 +336,41 @@ __device__ __forceinline__ uint32_t decode_sorted_entry(const FastArgs& fa, cons
     return cls;
 }
 
-template <bool kOutBf16, bool kSg = false, bool kShard = false>
-__global__ void __launch_bounds__(kSortThreads, 1)
-gemv_sorted_kernel(FastArgs fa, const unsigned long long* __restrict__ sorted, const uint16_t* __restrict__ gain, SgArgs sg,
-                   int64_t n_out, int64_t k_in, int64_t bpr, uint32_t nq_magic, const uint16_t* __restrict__ x, YOut yo,
-                   float* __restrict__ scratch, uint32_t* __restrict__ counters)
+// One matrix of a launch that works through several matrices one after another (llvq_gemv_multi, llvq_gemv_sorted_multi):
+// every CTA takes its share of each matrix in turn, so the table image, the launch and the ramp-up are paid once.
+constexpr int kMaxMultiMats = 8;
+struct GemvMat {
+    const void* weights;        // stored stream or sorted entries
+    const uint16_t* gain;
+    const uint16_t* x;
+    void* y;
+    int64_t n_out, k_in;
+    int64_t slot0;              // first scratch row / pair slot of this matrix (a multiple of 8)
+    uint32_t nq_magic;          // floor(2^32 / units per row group)
+    int32_t seg_units;          // stored stream only: units per binned segment
+};
+struct GemvMulti {
+    GemvMat m[kMaxMultiMats];
+    int n;
+};
+
+// Ask for the first chunk of every warp of this CTA in L2 (one request per 128-byte line).
+__device__ __forceinline__ void prefetch_first_chunks(const unsigned long long* sorted, int64_t n_out, int64_t bpr)
 {
-    {   // ask for the warps' first chunks in L2 while the table image is on its way (one request per 128-byte line)
-        const int64_t nq0 = (bpr + 3) / 4, U0 = ((n_out + kGemvGroupRows - 1) / kGemvGroupRows) * nq0;
-        const int64_t ub = blockIdx.x * U0 / gridDim.x, ue = (blockIdx.x + 1) * U0 / gridDim.x;
-        if ((threadIdx.x & 15u) == 0u && ub + (int64_t)(threadIdx.x >> 5) < ue)
-            asm volatile("prefetch.global.L2 [%0];" ::"l"(sorted + ub * 32 + threadIdx.x));
-    }
-    FAST_PROLOGUE(if (kShard) shard_arrive(yo));
+    const int64_t nq0 = (bpr + 3) / 4, U0 = ((n_out + kGemvGroupRows - 1) / kGemvGroupRows) * nq0;
+    const int64_t ub = blockIdx.x * U0 / gridDim.x, ue = (blockIdx.x + 1) * U0 / gridDim.x;
+    if ((threadIdx.x & 15u) == 0u && ub + (int64_t)(threadIdx.x >> 5) < ue)
+        asm volatile("prefetch.global.L2 [%0];" ::"l"(sorted + ub * 32 + threadIdx.x));
+}
+
+// The sorted-layout GEMV of one matrix by this CTA (all threads call it; shared memory behind `staging` is reused by the
+// next call, which the caller separates with a block barrier).
+template <bool kOutBf16, bool kSg, bool kShard>
+__device__ __forceinline__ void gemv_sorted_body(const FastArgs& fa, const FastSmem& T, uint8_t* staging,
+                                                 const unsigned long long* __restrict__ sorted, const uint16_t* __restrict__ gain, const SgArgs& sg,
+                                                 int64_t n_out, int64_t k_in, int64_t bpr, uint32_t nq_magic, const uint16_t* __restrict__ x,
+                                                 const YOut& yo, float* __restrict__ scratch, uint32_t* __restrict__ counters, int64_t slot0)
+{
     const int64_t nq = (bpr + 3) / 4;
     uint32_t* xs = reinterpret_cast<uint32_t*>(staging);            // [nq * 4][12] packed bf16 pairs of x
     float* acc = reinterpret_cast<float*>(xs + nq * 48);            // [kSortAccCopies][kGemvGroupsPerPass][8]: warps spread their adds over the copies
@@ -410,13 +424,8 @@ gemv_sorted_kernel(FastArgs fa, const unsigned long long* __restrict__ sorted, c
             const uint4* xb = reinterpret_cast<const uint4*>(xs + cb * 12u);
             const uint4 x0 = xb[0], x1 = xb[1], x2 = xb[2];
             const uint32_t xv[12] = {x0.x, x0.y, x0.z, x0.w, x1.x, x1.y, x1.z, x1.w, x2.x, x2.y, x2.z, x2.w};
-            float s0 = 0.f, s1 = 0.f;
-#pragma unroll
-            for (int j = 0; j < 12; ++j) {                        // bf16 x bf16 products are exact in binary32
-                s0 = fmaf(__uint_as_float(w[j] << 16), __uint_as_float(xv[j] << 16), s0);
-                s1 = fmaf(__uint_as_float(w[j] & 0xffff0000u), __uint_as_float(xv[j] & 0xffff0000u), s1);
-            }
-            if (valid) atomicAdd(&acc[(warp & (kSortAccCopies - 1)) * (kGemvGroupsPerPass * kGemvGroupRows) + rloc], s0 + s1);
+            const float dot = dot24_bf16(w, xv);
+            if (valid) atomicAdd(&acc[(warp & (kSortAccCopies - 1)) * (kGemvGroupsPerPass * kGemvGroupRows) + rloc], dot);
             ch = nxt; e = e_next;
         }
         __syncthreads();
@@ -429,10 +438,40 @@ gemv_sorted_kernel(FastArgs fa, const unsigned long long* __restrict__ sorted, c
             return v;
         };
         const int64_t ub = blockIdx.x * U / G, ue = (blockIdx.x + 1) * U / G;     // recomputed here: nothing 64-bit lives across the main loop
-        finish_pass<kOutBf16, kShard>(yo, rg0, rg1, nq, ub, ue, U, G, n_out, scratch, counters, row_sum);
+        finish_pass<kOutBf16, kShard>(yo, rg0, rg1, nq, ub, ue, U, G, n_out, scratch, counters, row_sum, slot0);
         __syncthreads();                                   // the sums are read above: the next pass may clear them only now
     });
+}
+
+template <bool kOutBf16, bool kSg = false, bool kShard = false>
+__global__ void __launch_bounds__(kSortThreads, 1)
+gemv_sorted_kernel(FastArgs fa, const unsigned long long* __restrict__ sorted, const uint16_t* __restrict__ gain, SgArgs sg,
+                   int64_t n_out, int64_t k_in, int64_t bpr, uint32_t nq_magic, const uint16_t* __restrict__ x, YOut yo,
+                   float* __restrict__ scratch, uint32_t* __restrict__ counters)
+{
+    prefetch_first_chunks(sorted, n_out, bpr);          // while the table image is on its way
+    FAST_PROLOGUE(if (kShard) shard_arrive(yo));
+    gemv_sorted_body<kOutBf16, kSg, kShard>(fa, T, staging, sorted, gain, sg, n_out, k_in, bpr, nq_magic, x, yo, scratch, counters, 0);
     if (kShard) shard_arrive(yo);
+}
+
+// Several independent matrices in one launch (no output of one may be an input of another).
+template <bool kOutBf16>
+__global__ void __launch_bounds__(kSortThreads, 1)
+gemv_sorted_multi_kernel(FastArgs fa, const __grid_constant__ GemvMulti mm, float* __restrict__ scratch, uint32_t* __restrict__ counters)
+{
+    prefetch_first_chunks(static_cast<const unsigned long long*>(mm.m[0].weights), mm.m[0].n_out, (mm.m[0].k_in + 23) / 24);
+    FAST_PROLOGUE();
+    for (int i = 0; i < mm.n; ++i) {
+        const GemvMat& M = mm.m[i];
+        if (i + 1 < mm.n)
+            prefetch_first_chunks(static_cast<const unsigned long long*>(mm.m[i + 1].weights), mm.m[i + 1].n_out, (mm.m[i + 1].k_in + 23) / 24);
+        YOut yo{};
+        yo.y = M.y;
+        gemv_sorted_body<kOutBf16, false, false>(fa, T, staging, static_cast<const unsigned long long*>(M.weights), M.gain, SgArgs{}, M.n_out, M.k_in,
+                                                 (M.k_in + 23) / 24, M.nq_magic, M.x, yo, scratch, counters, M.slot0);
+        __syncthreads();                                   // the next matrix restages x and clears the row sums
+    }
 }
 
 // ===========================================================================
@@ -445,26 +484,30 @@ gemv_sorted_kernel(FastArgs fa, const unsigned long long* __restrict__ sorted, c
 constexpr int kBinSegUnits = 256;                    // at most 8192 blocks per segment (halved while shared memory is short)
 constexpr int kBinPerThread = kBinSegUnits * 32 / kSortThreads;   // 8
 
-template <bool kOutBf16, bool kSg = false, bool kShard = false>
-__global__ void __launch_bounds__(kSortThreads, 1)
-gemv_bin_kernel(FastArgs fa, const uint32_t* __restrict__ stream, const uint16_t* __restrict__ sort_rank, const uint16_t* __restrict__ gain, SgArgs sg,
-                int64_t n_out, int64_t k_in, int64_t bpr, uint32_t nq_magic, int seg_units, const uint16_t* __restrict__ x, YOut yo,
-                float* __restrict__ scratch, uint32_t* __restrict__ counters)
+// The span of the index stream and of the gains that this CTA's row groups cover is contiguous: request it from DRAM ahead
+// of time; the binning phases then read it from L2.
+template <bool kSg>
+__device__ __forceinline__ void prefetch_bin_span(const FastArgs& fa, const uint32_t* stream, const uint16_t* gain, const SgArgs& sg,
+                                                  int64_t n_out, int64_t bpr)
 {
-    {
-        // the rows of the row groups this CTA touches are one contiguous span of the index stream and of the gains:
-        // request it from DRAM now, while the table image is on its way; the binning phases then read it from L2
-        const int64_t nq0 = (bpr + 3) / 4, U0 = ((n_out + kGemvGroupRows - 1) / kGemvGroupRows) * nq0;
-        const int64_t ub = blockIdx.x * U0 / gridDim.x, ue = (blockIdx.x + 1) * U0 / gridDim.x;
-        if (ub < ue) {
-            const uint64_t b_first = (uint64_t)(ub / nq0) * kGemvGroupRows * (uint64_t)bpr;
-            const uint64_t b_last = (uint64_t)min(((ue - 1) / nq0 + 1) * kGemvGroupRows, n_out) * (uint64_t)bpr;
-            const uint64_t wf = (uint64_t)fa.L.W + (kSg ? (uint64_t)sg.bits : 0ull);
-            prefetch_span_l2(stream, b_first * wf / 8, (b_last * wf + 7) / 8);
-            if (!kSg) prefetch_span_l2(gain, b_first * 2, b_last * 2);
-        }
+    const int64_t nq0 = (bpr + 3) / 4, U0 = ((n_out + kGemvGroupRows - 1) / kGemvGroupRows) * nq0;
+    const int64_t ub = blockIdx.x * U0 / gridDim.x, ue = (blockIdx.x + 1) * U0 / gridDim.x;
+    if (ub < ue) {
+        const uint64_t b_first = (uint64_t)(ub / nq0) * kGemvGroupRows * (uint64_t)bpr;
+        const uint64_t b_last = (uint64_t)min(((ue - 1) / nq0 + 1) * kGemvGroupRows, n_out) * (uint64_t)bpr;
+        const uint64_t wf = (uint64_t)fa.L.W + (kSg ? (uint64_t)sg.bits : 0ull);
+        prefetch_span_l2(stream, b_first * wf / 8, (b_last * wf + 7) / 8);
+        if (!kSg) prefetch_span_l2(gain, b_first * 2, b_last * 2);
     }
-    FAST_PROLOGUE(if (kShard) shard_arrive(yo));
+}
+
+template <bool kOutBf16, bool kSg, bool kShard>
+__device__ __forceinline__ void gemv_bin_body(const FastArgs& fa, const FastSmem& T, uint8_t* staging, const uint32_t* __restrict__ stream,
+                                              const uint16_t* __restrict__ sort_rank, const uint16_t* __restrict__ gain, const SgArgs& sg,
+                                              int64_t n_out, int64_t k_in, int64_t bpr, uint32_t nq_magic, int seg_units,
+                                              const uint16_t* __restrict__ x, const YOut& yo, float* __restrict__ scratch,
+                                              uint32_t* __restrict__ counters, int64_t slot0)
+{
     const int64_t nq = (bpr + 3) / 4;
     uint32_t* xs = reinterpret_cast<uint32_t*>(staging);            // [nq * 4][12] packed bf16 pairs of x
     float* acc = reinterpret_cast<float*>(xs + nq * 48);            // [kSortAccCopies][kGemvGroupsPerPass][8]
@@ -577,13 +620,8 @@ gemv_bin_kernel(FastArgs fa, const uint32_t* __restrict__ stream, const uint16_t
             const uint4* xb = reinterpret_cast<const uint4*>(xs + cb * 12u);
             const uint4 x0 = xb[0], x1 = xb[1], x2 = xb[2];
             const uint32_t xv[12] = {x0.x, x0.y, x0.z, x0.w, x1.x, x1.y, x1.z, x1.w, x2.x, x2.y, x2.z, x2.w};
-            float s0 = 0.f, s1 = 0.f;
-#pragma unroll
-            for (int j = 0; j < 12; ++j) {
-                s0 = fmaf(__uint_as_float(w[j] << 16), __uint_as_float(xv[j] << 16), s0);
-                s1 = fmaf(__uint_as_float(w[j] & 0xffff0000u), __uint_as_float(xv[j] & 0xffff0000u), s1);
-            }
-            if (valid) atomicAdd(&acc[(warp & (kSortAccCopies - 1)) * (kGemvGroupsPerPass * kGemvGroupRows) + rloc], s0 + s1);
+            const float dot = dot24_bf16(w, xv);
+            if (valid) atomicAdd(&acc[(warp & (kSortAccCopies - 1)) * (kGemvGroupsPerPass * kGemvGroupRows) + rloc], dot);
             ch = nxt;
         }
         __syncthreads();
@@ -595,8 +633,40 @@ gemv_bin_kernel(FastArgs fa, const uint32_t* __restrict__ stream, const uint16_t
             return v;
         };
         const int64_t ub = blockIdx.x * U / G, ue = (blockIdx.x + 1) * U / G;     // recomputed here: nothing 64-bit lives across the main loop
-        finish_pass<kOutBf16, kShard>(yo, rg0, rg1, nq, ub, ue, U, G, n_out, scratch, counters, row_sum);
+        finish_pass<kOutBf16, kShard>(yo, rg0, rg1, nq, ub, ue, U, G, n_out, scratch, counters, row_sum, slot0);
         __syncthreads();
     }, seg_units);
+}
+
+template <bool kOutBf16, bool kSg = false, bool kShard = false>
+__global__ void __launch_bounds__(kSortThreads, 1)
+gemv_bin_kernel(FastArgs fa, const uint32_t* __restrict__ stream, const uint16_t* __restrict__ sort_rank, const uint16_t* __restrict__ gain, SgArgs sg,
+                int64_t n_out, int64_t k_in, int64_t bpr, uint32_t nq_magic, int seg_units, const uint16_t* __restrict__ x, YOut yo,
+                float* __restrict__ scratch, uint32_t* __restrict__ counters)
+{
+    prefetch_bin_span<kSg>(fa, stream, gain, sg, n_out, bpr);       // while the table image is on its way
+    FAST_PROLOGUE(if (kShard) shard_arrive(yo));
+    gemv_bin_body<kOutBf16, kSg, kShard>(fa, T, staging, stream, sort_rank, gain, sg, n_out, k_in, bpr, nq_magic, seg_units, x, yo, scratch, counters, 0);
     if (kShard) shard_arrive(yo);
+}
+
+// Several independent matrices on their stored streams in one launch.
+template <bool kOutBf16>
+__global__ void __launch_bounds__(kSortThreads, 1)
+gemv_bin_multi_kernel(FastArgs fa, const uint16_t* __restrict__ sort_rank, const __grid_constant__ GemvMulti mm, float* __restrict__ scratch,
+                      uint32_t* __restrict__ counters)
+{
+    prefetch_bin_span<false>(fa, static_cast<const uint32_t*>(mm.m[0].weights), mm.m[0].gain, SgArgs{}, mm.m[0].n_out, (mm.m[0].k_in + 23) / 24);
+    FAST_PROLOGUE();
+    for (int i = 0; i < mm.n; ++i) {
+        const GemvMat& M = mm.m[i];
+        if (i + 1 < mm.n)
+            prefetch_bin_span<false>(fa, static_cast<const uint32_t*>(mm.m[i + 1].weights), mm.m[i + 1].gain, SgArgs{}, mm.m[i + 1].n_out,
+                                     (mm.m[i + 1].k_in + 23) / 24);
+        YOut yo{};
+        yo.y = M.y;
+        gemv_bin_body<kOutBf16, false, false>(fa, T, staging, static_cast<const uint32_t*>(M.weights), sort_rank, M.gain, SgArgs{}, M.n_out, M.k_in,
+                                              (M.k_in + 23) / 24, M.nq_magic, M.seg_units, M.x, yo, scratch, counters, M.slot0);
+        __syncthreads();
+    }
 }

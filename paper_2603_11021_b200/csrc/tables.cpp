@@ -233,10 +233,24 @@ bool build_fast_image(const HostTables& t, FastLayout& L, std::vector<uint8_t>& 
     L.off = up16(L.pd6 + 4096);
     L.desc = up16(L.off + (with_classes ? (ncls + 1) * 8 : 0));
     L.total = up16(L.desc + ncls * kFastDescStride * 4);
+    L.sub3 = L.total;
+    L.total_ext = up16(L.sub3 + kSmallSubsetWords * 4);
     L.lut_shift = (uint32_t)(t.W >= 12 ? t.W - 12 : 0);
     L.ncls = (uint32_t)ncls;
     L.W = (uint32_t)t.W;
-    img.assign(L.total, 0);
+    img.assign(L.total_ext, 0);
+    {
+        // all k-subsets of 24 slots for k <= 3, each group in numeric order (= the order of their combinatorial-number-system
+        // ranks, whatever the number of slots in use), behind a four-word directory
+        uint32_t* sub = reinterpret_cast<uint32_t*>(img.data() + L.sub3);
+        uint32_t at = 4;
+        for (int k = 0; k <= kSmallSubsetMaxK; ++k) {
+            sub[k] = at;
+            for (uint32_t m = 0; m < (1u << kDim); ++m)
+                if (__builtin_popcount(m) == k) sub[at++] = m;
+        }
+        if (at != (uint32_t)kSmallSubsetWords) return false;
+    }
     std::memcpy(img.data() + L.golay, t.golay.data(), 4096 * 4);
     std::memcpy(img.data() + L.pascal, t.pascal, 625 * 4);
     for (int n = 0; n < 25; ++n)                           // column 0 is a sentinel in the image: "no element left to place"
@@ -270,6 +284,7 @@ bool build_fast_image(const HostTables& t, FastLayout& L, std::vector<uint8_t>& 
         if (nlev > kFastMaxLevels || nlev + 2 > 8) return false;
         uint32_t flags = (d.parity ? 1u : 0u) | (d.signpar ? 2u : 0u) | (d.fill0 ? 4u : 0u) |
                          ((d.fill1 & 2) ? 8u : 0u) | ((d.fill0 & 2) ? 16u : 0u);
+        if (!((t.info[j].card / ((u128)d.A << d.B)) >> 32)) flags |= kFastFlagRank32;
         w[0] = d.w | (uint32_t)d.B << 8 | flags << 16 | (uint32_t)d.nlev1 << 24 | (uint32_t)nlev << 28;
         w[1] = d.goff | (uint32_t)d.A << 16;
         w[2] = (uint32_t)d.magicA; w[3] = (uint32_t)(d.magicA >> 32);
@@ -282,7 +297,10 @@ bool build_fast_image(const HostTables& t, FastLayout& L, std::vector<uint8_t>& 
             vals[2 + l] = lv.val;
             w[8 + l] = lv.radix | (uint32_t)lv.k << 22 | (uint32_t)(2 + l) << 27 | ((lv.val & 2) ? 1u << 30 : 0u) | (lv.val ? 1u << 31 : 0u);
             nbytes |= (uint32_t)lv.n << (8 * l);
-            if (l == 0) { w[6] = (uint32_t)lv.magic; w[7] = (uint32_t)(lv.magic >> 32); p_after = (p_after + lv.radix - 1) / lv.radix; }
+            if (l == 0) {
+                w[6] = (uint32_t)lv.magic; w[7] = (uint32_t)(lv.magic >> 32); p_after = (p_after + lv.radix - 1) / lv.radix;
+                w[kFastDescMagic0] = lv.radix > 1 ? (uint32_t)((1ull << 32) / lv.radix) : 0xffffffffu;
+            }
             else {
                 if (p_after >> 32) return false;                     // 32-bit quotient chain after the first step
                 w[11 + l] = (uint32_t)((1ull << 32) / lv.radix);

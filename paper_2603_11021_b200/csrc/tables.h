@@ -77,8 +77,12 @@ bool build_tables(int m_lo, int m_hi, HostTables& out);
 namespace llvq {
 
 constexpr int kFastMaxLevels = 4;      // unranking steps per class on the fast path
-constexpr int kFastDescWords = 17;     // words of a class descriptor that carry data
+constexpr int kFastDescWords = 18;     // words of a class descriptor that carry data
 constexpr int kFastDescRnorm = 16;     // word holding 1 / sqrt(16 m) as binary32
+constexpr int kFastDescMagic0 = 17;    // word holding floor(2^32 / radix) of level 0 (used when the arrangement rank fits 32 bits)
+constexpr uint32_t kFastFlagRank32 = 32u;   // descriptor flag: the class has fewer than 2^32 arrangements
+constexpr int kSmallSubsetMaxK = 3;    // the table of all k-subsets of 24 slots covers k = 0..3
+constexpr int kSmallSubsetWords = 4 + 1 + 24 + 276 + 2024;   // [first entry of k = 0..3][the subsets, by k, each group in numeric order]
 constexpr int kFastDescStride = 20;    // words between descriptors: 80 bytes spread consecutive classes over all bank groups
 constexpr int kLowBits = 14;           // slots resolved by one table lookup in the subset unranking
 
@@ -93,7 +97,9 @@ struct FastLayout {
     uint32_t pd6;         // u8[4096]: [f << 6 | s] = low bits of s deposited into the set bits of f
     uint32_t off;         // u64[ncls + 1]
     uint32_t desc;        // u32[ncls][kFastDescStride]
-    uint32_t total;       // bytes, multiple of 16
+    uint32_t total;       // bytes of the image proper, multiple of 16
+    uint32_t sub3;        // u32[kSmallSubsetWords], behind the image proper: kernels with room for it load total_ext bytes
+    uint32_t total_ext;   // bytes including sub3, multiple of 16
     uint32_t lut_shift;
     uint32_t ncls;
     uint32_t W;
@@ -101,7 +107,8 @@ struct FastLayout {
 
 // Word layout of a fast descriptor:
 //  0: w | B << 8 | flags << 16 | nlev1 << 24 | nlev << 28
-//       flags: bit0 parity, bit1 signpar, bit2 fill0 is nonzero, bit3 fill1 has value bit 1, bit4 fill0 has value bit 1
+//       flags: bit0 parity, bit1 signpar, bit2 fill0 is nonzero, bit3 fill1 has value bit 1, bit4 fill0 has value bit 1,
+//              bit5 the arrangement rank of the class fits 32 bits
 //  1: goff | A << 16
 //  2,3: magicA = floor((2^64-1)/A)
 //  4,5: absolute value of id 0..7 (one byte each): id 0 = fill0, id 1 = fill1, ids 2.. = levels in order
@@ -110,6 +117,7 @@ struct FastLayout {
 //  12..14: floor(2^32 / radix) of levels 1..3
 //  15: n (free slots before the step) of levels 0..3, one byte each
 //  16: binary32 bits of 1 / |x| = 1 / sqrt(16 m) (formed in binary64, rounded once), for the shape-gain form
+//  17: floor(2^32 / radix) of level 0
 // with_classes = false builds only the class-independent tables (Golay, Pascal, subsets, deposit): codes whose class
 // tables do not fit shared memory keep those in global memory.
 bool build_fast_image(const HostTables& t, FastLayout& layout, std::vector<uint8_t>& image, bool with_classes = true);
