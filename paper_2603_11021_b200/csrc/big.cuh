@@ -1,7 +1,8 @@
 // Dequantizer for codes whose class tables do not fit shared memory (the 72-bit code: 114 976 classes, up to
-// seven unranking steps and nine distinct values per class).  The class-independent tables (Golay, Pascal,
-// 14-slot subsets, deposit) are served from shared memory as on the fast path; class offsets and descriptors
-// are read from global memory (they stay in L2).  Produces the point as 24 signed bytes.
+// seven unranking steps and nine distinct values per class).  The class-independent tables (Golay, Pascal and the
+// reciprocals of its entries, 14-slot subsets, small subsets, deposit) are served from shared memory as on the fast
+// path; class offsets and the 32-byte class records are read from global memory (they stay in L2).  Produces the point
+// as bit planes of value ids, like the fast path.
 #pragma once
 #include "decode.cuh"
 #include "fast.cuh"
@@ -25,22 +26,56 @@ __device__ __forceinline__ int big_find_class(const DevCode& dc, uint64_t lo, ui
     return a;
 }
 
-// S3-S6 for any class of any supported code.  All 32 lanes of the warp call this together.
-__device__ __forceinline__ void big_decode_local(const FastSmem& T, const DevCode& dc, int cls, uint64_t local, bool valid, Point& pt)
+// Result of the table-driven decoder below: the planes of the fast path plus a fourth one, set where the value id is 8
+// (classes with nine distinct values or odd classes with eight; rare), and that value.
+struct DecodedBig {
+    Decoded d;
+    uint32_t p3;
+    uint32_t val8;
+};
+
+__device__ __forceinline__ uint32_t lds_u32(uint32_t addr)
 {
-    const uint4* cd = reinterpret_cast<const uint4*>(dc.cls + (valid ? cls : 0));
+    uint32_t v;
+    asm volatile("ld.shared.u32 %0, [%1];" : "=r"(v) : "r"(addr));
+    return v;
+}
+
+__device__ __forceinline__ uint64_t lds_u64(uint32_t addr)
+{
+    uint64_t v;
+    asm volatile("ld.shared.u64 %0, [%1];" : "=l"(v) : "r"(addr));
+    return v;
+}
+
+// S3-S6 for any class of a code whose class tables live in global memory, in the manner of fast_decode_local: the class
+// record is 32 bytes (BigDesc), the radix of a step is C(free slots, k) from the Pascal triangle in shared memory, its
+// reciprocal comes from the tables beside it (64-bit while the arrangement rank needs it, 32-bit afterwards), steps that
+// take at most three slots are one lookup in the table of small subsets, and the point comes out as bit planes of value
+// ids.  All lanes of `mask` call this together; writes `out` only where `valid` (the caller presets it).
+__device__ __forceinline__ void big_decode_planes(const FastSmem& T, const DevCode& dc, int cls, uint64_t local, bool valid, uint32_t mask,
+                                                  DecodedBig& out)
+{
+    const uint4* cd = reinterpret_cast<const uint4*>(dc.big + (valid ? cls : 0));
     const uint4 zero4 = make_uint4(0u, 0u, 0u, 0u);
     const uint4 h0 = valid ? __ldg(cd) : zero4, h1 = valid ? __ldg(cd + 1) : zero4;
-    const uint32_t parity = h0.x & 0xff, w = (h0.x >> 8) & 0xff, B = (h0.x >> 16) & 0xff, signpar = h0.x >> 24;
-    const uint32_t nlev1 = h0.y & 0xff, nlev0 = (h0.y >> 8) & 0xff, fill1 = (h0.y >> 16) & 0xff, fill0 = h0.y >> 24;
-    const uint32_t goff = h0.z & 0xffff, A = h0.z >> 16;
-    const uint32_t nlev = nlev1 + nlev0;
+    const uint32_t w = h0.x & 0xff, B = (h0.x >> 8) & 0xff, flags = (h0.x >> 16) & 0xff;
+    const uint32_t nlev1 = (h0.x >> 24) & 0xf, nlev = h0.x >> 28;
+    const uint32_t goff = h0.y & 0xffff, A = h0.y >> 16;
+    const uint32_t lvl_bit1 = (h1.z >> 8) & 0xff, lvl_nz = (h1.z >> 16) & 0xff;
+    const bool odd = (flags & 1u) != 0u;
 
     // S3: r fastest, then the sign word s, then the arrangement rank p
     uint64_t q = local;
     uint32_t r = 0;
     if (A == 4096u) { r = (uint32_t)local & 4095u; q = local >> 12; }
-    else if (A > 1u) divmod_magic(local, A, ((uint64_t)h1.y << 32) | h1.x, q, r);
+    else if (A > 1u) {                                   // 759 or 2576 codewords of weight 8 / 16 or 12
+        const uint64_t magic = A == 759u ? 0xffffffffffffffffull / 759u : 0xffffffffffffffffull / 2576u;
+        q = __umul64hi(local, magic);
+        uint64_t rem = local - q * A;
+        if (rem >= A) { rem -= A; ++q; }
+        r = (uint32_t)rem;
+    }
     const uint32_t s = (uint32_t)q & ((1u << B) - 1u);
     uint64_t p = q >> B;
 
@@ -48,64 +83,101 @@ __device__ __forceinline__ void big_decode_local(const FastSmem& T, const DevCod
     const uint32_t c = T.golay[goff + r];
 
     // S5: arrangement.  Group 1 on F1(c), then group 0 on F0(c) (odd classes: one group 0 on all positions).
-    const bool odd = parity != 0u;
     const uint32_t F1 = odd ? 0u : c;
     const uint32_t F0 = ~F1 & 0xffffffu;
-    uint32_t freem = F1;
+    uint32_t freem = F1, nfree = odd ? 0u : w;
     bool in_group0 = false;
-    uint32_t bit1 = 0, nz0 = 0;
+    uint32_t p0 = 0, p1 = 0, p2 = 0, p3 = 0, bit1 = 0, nz0 = 0;
+    const uint32_t pascal_a = smem_addr(T.pascal), r64_a = smem_addr(T.recip64), r32_a = smem_addr(T.recip32);
+    const int maxlev = __reduce_max_sync(mask, nlev);
 #pragma unroll
-    for (int i = 0; i < 6; ++i) pt.w[i] = 0u;
-    const int maxlev = __reduce_max_sync(kFullMask, nlev);
-    for (int l = 0; l < maxlev; ++l) {
-        if (!in_group0 && (uint32_t)l >= nlev1) {               // group 1 done: its last value fills what is left of F1
-            place_value(pt, freem, fill1);
-            if (fill1 & 2u) bit1 |= freem;
-            freem = F0; in_group0 = true;
-        }
-        const bool active = (uint32_t)l < nlev;
-        const uint4 L = active ? __ldg(cd + 2 + l) : zero4;
-        const uint32_t k = L.y & 0xff, val = (L.y >> 8) & 0xff, n = (L.y >> 16) & 0xff;
-        uint32_t rho = 0;
-        if (active) {
-            if ((p >> 32) == 0ull) {
-                // the rank has shrunk to 32 bits (it only ever gets smaller): the high word of the 64-bit magic,
-                // floor(2^32 / d) or one less, gives an estimate at most two too small
-                const uint32_t p32 = (uint32_t)p;
-                uint32_t q32 = __umulhi(p32, L.w);
-                uint32_t r32 = p32 - q32 * L.x;
-                if (r32 >= L.x) { r32 -= L.x; ++q32; }
-                if (r32 >= L.x) { r32 -= L.x; ++q32; }
-                rho = r32; p = q32;
-            } else {
-                uint64_t pq;
-                divmod_magic(p, L.x, ((uint64_t)L.w << 32) | L.z, pq, rho);
-                p = pq;
+    for (int l = 0; l < kMaxLevels - 1; ++l) {
+        if (l < maxlev) {
+            if (!in_group0 && (uint32_t)l >= nlev1) {               // group 1 done: its filler gets id 1
+                p0 |= freem;
+                if (flags & 8u) bit1 |= freem;
+                freem = F0; nfree = 24u - (odd ? 0u : w); in_group0 = true;
             }
+            const bool active = (uint32_t)l < nlev;
+            const uint32_t k = active ? ((l < 4 ? h1.x : h1.y) >> (8 * (l & 3))) & 0xffu : 0u;
+            const uint32_t cell = nfree * 25u + k;                  // C(nfree, k) and its reciprocals
+            const uint32_t radix = lds_u32(pascal_a + cell * 4u);
+            uint32_t rho = 0u;
+            if (__any_sync(mask, (uint32_t)(p >> 32) != 0u)) {
+                const uint64_t qq0 = __umul64hi(p, lds_u64(r64_a + cell * 8u));
+                uint64_t qq = qq0, rem = p - qq * radix;
+                if (rem >= radix) { rem -= radix; ++qq; }
+                if (active) { p = qq; rho = (uint32_t)rem; }
+            } else {
+                const uint32_t p32 = (uint32_t)p;
+                uint32_t qq = __umulhi(p32, lds_u32(r32_a + cell * 4u));
+                uint32_t rem = p32 - qq * radix;
+                if (rem >= radix) { rem -= radix; ++qq; }
+                if (active) { p = qq; rho = rem; }
+            }
+            uint32_t rel;
+            if (T.sub3 != 0u && __all_sync(mask, k <= (uint32_t)kSmallSubsetMaxK)) rel = small_subset(T, k, rho);
+            else rel = nth_subset(T, k, rho, (int)__reduce_max_sync(mask, active ? nfree : 0u));
+            const uint32_t a = deposit24(T.pd6, rel, freem);
+            freem ^= a; nfree -= k;
+            if ((l + 2) & 1) p0 |= a;                               // id of level l is l + 2
+            if ((l + 2) & 2) p1 |= a;
+            if ((l + 2) & 4) p2 |= a;
+            if ((l + 2) & 8) p3 |= a;
+            if ((lvl_bit1 >> l) & 1u) bit1 |= a;
+            if (in_group0 && ((lvl_nz >> l) & 1u)) nz0 |= a;
         }
-        const int top = __reduce_max_sync(kFullMask, n);
-        const uint32_t rel = nth_subset(T, k, rho, top);
-        const uint32_t a = deposit24(T.pd6, rel, freem);
-        freem ^= a;
-        place_value(pt, a, val);
-        if (val & 2u) bit1 |= a;
-        if (in_group0 && val) nz0 |= a;
     }
     if (!in_group0) {
-        place_value(pt, freem, fill1);
-        if (fill1 & 2u) bit1 |= freem;
+        p0 |= freem;
+        if (flags & 8u) bit1 |= freem;
         freem = F0;
     }
-    place_value(pt, freem, fill0);
-    if (fill0 & 2u) bit1 |= freem;
-    if (fill0) nz0 |= freem;
+    if (flags & 16u) bit1 |= freem;                                 // filler of group 0 keeps id 0
+    if (flags & 4u) nz0 |= freem;
 
     // S6: signs
-    const uint32_t nf1 = w ? w - 1u : 0u;                       // free sign bits on F1
+    const uint32_t nf1 = w ? w - 1u : 0u;                           // free sign bits on F1
     const uint32_t s1 = s & ((1u << nf1) - 1u);
-    const uint32_t src1 = s1 | (((__popc(s1) + signpar) & 1u) << nf1);     // last F1 position: sum = 0 mod 8
-    const uint32_t neg_even = deposit24(T.pd6, src1, F1) | deposit24(T.pd6, s >> nf1, odd ? 0u : nz0);
-    negate_at(pt, valid ? (odd ? (c ^ bit1) : neg_even) : 0u);
+    const uint32_t src1 = s1 | (((__popc(s1) + (flags >> 1)) & 1u) << nf1);     // last F1 position: sum = 0 mod 8
+    uint32_t neg;
+    if (__all_sync(mask, odd)) neg = c ^ bit1;                      // 1 mod 4 on F0, 3 mod 4 on F1
+    else {
+        const uint32_t neg_even = deposit24(T.pd6, src1, F1) | deposit24(T.pd6, s >> nf1, odd ? 0u : nz0);
+        neg = odd ? (c ^ bit1) : neg_even;
+    }
+    if (valid) {
+        out.d.p0 = p0; out.d.p1 = p1; out.d.p2 = p2; out.d.neg = neg;
+        out.d.vals_lo = h0.z; out.d.vals_hi = h0.w;
+        out.p3 = p3; out.val8 = h1.z & 0xffu;
+    }
+}
+
+// Where the fourth plane is set the value id is 8: put bf16(gain * val8), signed, over what the three-plane expansion
+// left there.  All lanes of the warp call this together.
+__device__ __forceinline__ void patch_id8_bf16(const DecodedBig& b, float gain, uint32_t w[12])
+{
+    if (!__any_sync(kFullMask, b.p3 != 0u)) return;
+    const uint32_t v = (uint32_t)__bfloat16_as_ushort(__float2bfloat16_rn(gain * (float)b.val8));
+#pragma unroll
+    for (int j = 0; j < 12; ++j) {
+        const uint32_t lo = (b.p3 >> (2 * j)) & 1u, hi = (b.p3 >> (2 * j + 1)) & 1u;
+        const uint32_t m = (lo ? 0xffffu : 0u) | (hi ? 0xffff0000u : 0u);
+        const uint32_t sg = (((b.d.neg >> (2 * j)) & 1u) << 15) | (((b.d.neg >> (2 * j + 1)) & 1u) << 31);
+        w[j] = (w[j] & ~m) | (((v | v << 16) ^ sg) & m);
+    }
+}
+
+__device__ __forceinline__ void patch_id8_bytes(const DecodedBig& b, uint32_t out[6])
+{
+    if (!__any_sync(kFullMask, b.p3 != 0u)) return;
+#pragma unroll
+    for (int i = 0; i < 24; ++i) {
+        if ((b.p3 >> i) & 1u) {
+            const uint32_t byte = ((b.d.neg >> i) & 1u) ? (0u - b.val8) & 0xffu : b.val8;
+            out[i >> 2] = (out[i >> 2] & ~(0xffu << (8 * (i & 3)))) | byte << (8 * (i & 3));
+        }
+    }
 }
 
 }  // namespace llvq

@@ -12,7 +12,8 @@ namespace llvq {
 // Device view of one code's class tables in global memory (pointers owned by the context).  Codes whose class
 // tables fit shared memory use the copies inside the table image instead.
 struct DevCode {
-    const ClassDesc* cls;           // [nclasses]
+    const ClassDesc* cls;           // [nclasses] (codes whose tables fit shared memory: read by the encoder's indexing kernel)
+    const BigDesc* big;             // [nclasses] compact records (codes whose class tables stay in global memory)
     const uint64_t* off_lo;         // [nclasses + 1] low 64 bits of the class offsets
     const uint32_t* off_hi;         // [nclasses + 1] bits 64.. of the class offsets
     const uint32_t* lut16;          // [65537] class of the first index of bucket (I >> (W - 16)), then the last class

@@ -23,6 +23,8 @@ struct FastSmem {
     const uint8_t* pd6;
     const uint64_t* off;
     const uint32_t* desc;
+    const uint64_t* recip64;  // images without class tables: reciprocals of the Pascal entries
+    const uint32_t* recip32;
     uint32_t sub3;            // shared-window byte address of the table of small subsets, 0 when the kernel did not load it
     uint32_t lut_shift;
 };
@@ -41,6 +43,8 @@ __device__ __forceinline__ FastSmem fast_view(const uint8_t* smem, const FastLay
     T.pd6 = smem + L.pd6;
     T.off = reinterpret_cast<const uint64_t*>(smem + L.off);
     T.desc = reinterpret_cast<const uint32_t*>(smem + L.desc);
+    T.recip64 = reinterpret_cast<const uint64_t*>(smem + L.recip64);
+    T.recip32 = reinterpret_cast<const uint32_t*>(smem + L.recip32);
     T.sub3 = with_small_subsets ? smem_addr(smem + L.sub3) : 0u;
     T.lut_shift = L.lut_shift;
     return T;

@@ -8,6 +8,9 @@ namespace {
 #include "gemv_kernels.cuh"
 #include "gemm_kernels.cuh"
 
+// The codes whose class tables stay in global memory have room for the table of small subsets beside the GEMM's buffers.
+size_t gemm_image_bytes(const llvq_ctx* ctx) { return ctx->fast ? ctx->fl.total : ctx->fl.total_ext; }
+
 int check_gemm_args(const llvq_ctx* ctx, const void* d_idx, const uint16_t* d_gain_f16, int64_t n_out, int64_t k_in,
                     const uint16_t* d_x_bf16, int batch, const uint16_t* d_y_bf16)
 {
@@ -21,12 +24,12 @@ int check_gemm_args(const llvq_ctx* ctx, const void* d_idx, const uint16_t* d_ga
 // Enqueue gemm_sorted_kernel on a stream sorted by llvq_sort_blocks_gemm.
 int launch_gemm_domains(const llvq_ctx* ctx, const void* p, const uint16_t* d_gain_f16, int64_t n_out, int64_t k_in,
                         const uint16_t* d_x_bf16, int batch, uint16_t* d_y_bf16, float* scratch, uint32_t* counters, void* stream,
-                        const YOut* yo = nullptr, int64_t y_ld = 0, const SgArgs* sg = nullptr)
+                        const YOut* yo = nullptr, int64_t y_ld = 0, const SgArgs* sg = nullptr, int y_f32 = 0)
 {
     DeviceGuard guard(ctx->device);
     if (!guard.ok) return LLVQ_ECUDA;
     GemmArgs ga;
-    ga.y = d_y_bf16; ga.y_ld = n_out; ga.shard = nullptr;
+    ga.y = d_y_bf16; ga.y_ld = n_out; ga.shard = nullptr; ga.y_f32 = y_f32;
     if (yo) {                                             // the description travels ahead of the kernel on the same stream
         ga.y = static_cast<uint16_t*>(yo->y); ga.y_ld = y_ld; ga.shard = static_cast<const YOut*>(ctx->d_shard);
         put_shard_kernel<<<1, 32, 0, (cudaStream_t)stream>>>(*yo, static_cast<YOut*>(ctx->d_shard));   // by value: safe under stream capture
@@ -41,23 +44,22 @@ int launch_gemm_domains(const llvq_ctx* ctx, const void* p, const uint16_t* d_ga
     ga.split = 1;                                                             // unused: the kernel balances domains over the CTAs itself
     const unsigned grid = (unsigned)std::min<int64_t>(row_tiles * ga.nstages, ctx->sm_count);
     // gemm_pipe_kernel: two A buffer sets and two X buffer sets, or one X set when two do not fit; else the kernel with the block barrier
-    const size_t head = (ctx->fl.total + 64 + 1023) & ~size_t(1023), a_set = (size_t)kDomStages * kGemmRows * kStageK * 2,
+    const size_t head = (gemm_image_bytes(ctx) + 64 + 1023) & ~size_t(1023), a_set = (size_t)kDomStages * kGemmRows * kStageK * 2,
                  x_set = (size_t)kDomStages * ga.npad * kStageK * 2;
     int pipe = 0, b_double = 0;
     size_t smem = head + (size_t)dpi * (a_set + x_set);
-    if (!ctx->fast) {}                                   // the 72-bit code gains nothing from the pipeline (measured): it keeps the kernel below
-    else if (head + 2 * a_set + 2 * x_set <= 227 * 1024) { pipe = 1; b_double = 1; smem = head + 2 * a_set + 2 * x_set; }
+    if (head + 2 * a_set + 2 * x_set <= 227 * 1024) { pipe = 1; b_double = 1; smem = head + 2 * a_set + 2 * x_set; }
     else if (head + 2 * a_set + x_set <= 227 * 1024) { pipe = 1; smem = head + 2 * a_set + x_set; }
     if (smem > 227 * 1024) return LLVQ_EUNSUPPORTED;
 #define LLVQ_LAUNCH_DOMAINS(BIG, SG, SH)                                                                                      \
     do {                                                                                                                     \
         if (pipe) {                                                                                                          \
             if (!set_smem(gemm_pipe_kernel<BIG, SG, SH>, smem)) return LLVQ_ECUDA;                                            \
-            if (launch_pdl(gemm_pipe_kernel<BIG, SG, SH>, grid, (unsigned)kGemmThreads, smem, (cudaStream_t)stream, fast_args(ctx), \
+            if (launch_pdl(gemm_pipe_kernel<BIG, SG, SH>, grid, (unsigned)kGemmThreads, smem, (cudaStream_t)stream, fast_args(ctx, !ctx->fast), \
                            static_cast<const unsigned long long*>(p), d_gain_f16, sga, ga, b_double) != cudaSuccess) return LLVQ_ECUDA; \
         } else {                                                                                                             \
             if (!set_smem(gemm_sorted_kernel<BIG, SG, SH>, smem)) return LLVQ_ECUDA;                                          \
-            if (launch_pdl(gemm_sorted_kernel<BIG, SG, SH>, grid, (unsigned)kGemmThreads, smem, (cudaStream_t)stream, fast_args(ctx), \
+            if (launch_pdl(gemm_sorted_kernel<BIG, SG, SH>, grid, (unsigned)kGemmThreads, smem, (cudaStream_t)stream, fast_args(ctx, !ctx->fast), \
                            static_cast<const unsigned long long*>(p), d_gain_f16, sga, ga, dpi) != cudaSuccess) return LLVQ_ECUDA; \
         }                                                                                                                    \
     } while (0)
@@ -88,7 +90,7 @@ int launch_gemm(const llvq_ctx* ctx, const void* d_idx, const uint16_t* d_gain_f
     cudaStream_t st = (cudaStream_t)stream;
     if (k_in == 0) return cudaMemsetAsync(d_y_bf16, 0, (size_t)n_out * batch * 2, st) == cudaSuccess ? LLVQ_OK : LLVQ_ECUDA;
     GemmArgs ga;
-    ga.y = d_y_bf16; ga.y_ld = n_out; ga.shard = nullptr;
+    ga.y = d_y_bf16; ga.y_ld = n_out; ga.shard = nullptr; ga.y_f32 = 0;
     if (yo) {                                             // the description travels ahead of the kernel on the same stream
         ga.y = static_cast<uint16_t*>(yo->y); ga.y_ld = y_ld; ga.shard = static_cast<const YOut*>(ctx->d_shard);
         put_shard_kernel<<<1, 32, 0, (cudaStream_t)stream>>>(*yo, static_cast<YOut*>(ctx->d_shard));   // by value: safe under stream capture
@@ -109,7 +111,7 @@ int launch_gemm(const llvq_ctx* ctx, const void* d_idx, const uint16_t* d_gain_f
     ga.split = best;
     const int64_t items = row_tiles * ga.split;
     const unsigned grid = (unsigned)std::min<int64_t>(items, ctx->sm_count);
-    const size_t img = ctx->fl.total;
+    const size_t img = gemm_image_bytes(ctx);
     const size_t smem = ((img + 64 + 1023) & ~size_t(1023)) + 2 * kGemmRows * kStageK * 2 + 2 * (size_t)ga.npad * kStageK * 2;
     if (smem > 227 * 1024) return LLVQ_EUNSUPPORTED;
     const uint32_t* idx = static_cast<const uint32_t*>(d_idx);
@@ -130,7 +132,7 @@ int launch_gemm(const llvq_ctx* ctx, const void* d_idx, const uint16_t* d_gain_f
 #define LLVQ_LAUNCH_PIPE_STORED(BIG, SG, SH)                                                                                    \
     do {                                                                                                                        \
         if (!set_smem(gemm_pipe_kernel<BIG, SG, SH, true>, smem_pipe)) return LLVQ_ECUDA;                                        \
-        if (launch_pdl(gemm_pipe_kernel<BIG, SG, SH, true>, grid_pipe, (unsigned)kGemmThreads, smem_pipe, st, fast_args(ctx), words, \
+        if (launch_pdl(gemm_pipe_kernel<BIG, SG, SH, true>, grid_pipe, (unsigned)kGemmThreads, smem_pipe, st, fast_args(ctx, !ctx->fast), words, \
                        d_gain_f16, sga, gp, b_double) != cudaSuccess) return LLVQ_ECUDA;                                        \
     } while (0)
             if (!ctx->fast) { if (yo) LLVQ_LAUNCH_PIPE_STORED(true, false, true); else LLVQ_LAUNCH_PIPE_STORED(true, false, false); }
@@ -144,20 +146,20 @@ int launch_gemm(const llvq_ctx* ctx, const void* d_idx, const uint16_t* d_gain_f
     if (yo) {
         if (ctx->fast) {
             if (!set_smem(gemm_kernel<false, false, true>, smem)) return LLVQ_ECUDA;
-            if (launch_pdl(gemm_kernel<false, false, true>, grid, (unsigned)kGemmThreads, smem, st, fast_args(ctx), idx, d_gain_f16, SgArgs{}, ga) != cudaSuccess) return LLVQ_ECUDA;
+            if (launch_pdl(gemm_kernel<false, false, true>, grid, (unsigned)kGemmThreads, smem, st, fast_args(ctx, !ctx->fast), idx, d_gain_f16, SgArgs{}, ga) != cudaSuccess) return LLVQ_ECUDA;
         } else {
             if (!set_smem(gemm_kernel<true, false, true>, smem)) return LLVQ_ECUDA;
-            if (launch_pdl(gemm_kernel<true, false, true>, grid, (unsigned)kGemmThreads, smem, st, fast_args(ctx), idx, d_gain_f16, SgArgs{}, ga) != cudaSuccess) return LLVQ_ECUDA;
+            if (launch_pdl(gemm_kernel<true, false, true>, grid, (unsigned)kGemmThreads, smem, st, fast_args(ctx, !ctx->fast), idx, d_gain_f16, SgArgs{}, ga) != cudaSuccess) return LLVQ_ECUDA;
         }
     } else if (sg) {
         if (!set_smem(gemm_kernel<false, true>, smem)) return LLVQ_ECUDA;
-        if (launch_pdl(gemm_kernel<false, true>, grid, (unsigned)kGemmThreads, smem, st, fast_args(ctx), idx, d_gain_f16, *sg, ga) != cudaSuccess) return LLVQ_ECUDA;
+        if (launch_pdl(gemm_kernel<false, true>, grid, (unsigned)kGemmThreads, smem, st, fast_args(ctx, !ctx->fast), idx, d_gain_f16, *sg, ga) != cudaSuccess) return LLVQ_ECUDA;
     } else if (ctx->fast) {
         if (!set_smem(gemm_kernel<false, false>, smem)) return LLVQ_ECUDA;
-        if (launch_pdl(gemm_kernel<false, false>, grid, (unsigned)kGemmThreads, smem, st, fast_args(ctx), idx, d_gain_f16, SgArgs{}, ga) != cudaSuccess) return LLVQ_ECUDA;
+        if (launch_pdl(gemm_kernel<false, false>, grid, (unsigned)kGemmThreads, smem, st, fast_args(ctx, !ctx->fast), idx, d_gain_f16, SgArgs{}, ga) != cudaSuccess) return LLVQ_ECUDA;
     } else {
         if (!set_smem(gemm_kernel<true, false>, smem)) return LLVQ_ECUDA;
-        if (launch_pdl(gemm_kernel<true, false>, grid, (unsigned)kGemmThreads, smem, st, fast_args(ctx), idx, d_gain_f16, SgArgs{}, ga) != cudaSuccess) return LLVQ_ECUDA;
+        if (launch_pdl(gemm_kernel<true, false>, grid, (unsigned)kGemmThreads, smem, st, fast_args(ctx, !ctx->fast), idx, d_gain_f16, SgArgs{}, ga) != cudaSuccess) return LLVQ_ECUDA;
     }
     return launch_status();
 }
@@ -169,7 +171,7 @@ extern "C" {
 // Sorted layout of the small-batch GEMM (see the comment at sort_blocks_gemm_kernel).
 static bool gemm_sortable(const llvq_ctx* ctx)
 {
-    if (!ctx->fast) return ctx->host.W <= 72 && ctx->dev.nclasses < (1 << 17);     // 128-bit entries: 72-bit index + class + position
+    if (!ctx->fast) return ctx->host.W <= 72 && ctx->bucket_classes_max <= (int)kBigDeltaMask;   // 96-bit entries: 72-bit index + class within its bucket + position
     return ctx->d_sort_rank && ctx->host.W <= 48 && ctx->host.N < (u128)kSortIndexMask;
 }
 
@@ -177,7 +179,7 @@ size_t llvq_sorted_gemm_bytes(const llvq_ctx* ctx, int64_t n_out, int64_t k_in)
 {
     if (!ctx || ctx->device < 0 || n_out <= 0 || k_in <= 0 || !gemm_sortable(ctx)) return 0;
     const int64_t bpr = (k_in + 23) / 24;
-    return (size_t)(((n_out + kGemmRows - 1) / kGemmRows) * ((bpr + kDomBlocks - 1) / kDomBlocks)) * kDomEntries * (ctx->fast ? 8 : 16);
+    return (size_t)(((n_out + kGemmRows - 1) / kGemmRows) * ((bpr + kDomBlocks - 1) / kDomBlocks)) * kDomEntries * (ctx->fast ? 8 : 4 * kBigEntryWords);
 }
 
 static int sort_blocks_gemm_common(const llvq_ctx* ctx, const void* d_idx, int gain_bits, int64_t n_out, int64_t k_in, void* d_sorted, void* stream)
@@ -192,13 +194,13 @@ static int sort_blocks_gemm_common(const llvq_ctx* ctx, const void* d_idx, int g
     const int64_t ndomains = ((n_out + kGemmRows - 1) / kGemmRows) * ((bpr + kDomBlocks - 1) / kDomBlocks);
     const unsigned g = (unsigned)std::min<int64_t>(ndomains, 4ll * ctx->sm_count);
     if (!ctx->fast) {
-        sort_blocks_gemm_big_kernel<<<g, kDomEntries, 0, (cudaStream_t)stream>>>(fast_args(ctx), static_cast<const uint32_t*>(d_idx), n_out, bpr,
-                                                                                 ndomains, static_cast<ulonglong2*>(d_sorted));
+        sort_blocks_gemm_big_kernel<<<g, kDomEntries, 0, (cudaStream_t)stream>>>(fast_args(ctx, !ctx->fast), static_cast<const uint32_t*>(d_idx), n_out, bpr,
+                                                                                 ndomains, static_cast<uint32_t*>(d_sorted));
         return launch_status();
     }
     const size_t smem = ctx->fl.total + 16;
     if (!set_smem(sort_blocks_gemm_kernel, smem)) return LLVQ_ECUDA;
-    sort_blocks_gemm_kernel<<<g, kDomEntries, smem, (cudaStream_t)stream>>>(fast_args(ctx), static_cast<const uint32_t*>(d_idx), ctx->d_sort_rank,
+    sort_blocks_gemm_kernel<<<g, kDomEntries, smem, (cudaStream_t)stream>>>(fast_args(ctx, !ctx->fast), static_cast<const uint32_t*>(d_idx), ctx->d_sort_rank,
                                                                            gain_bits, n_out, bpr, ndomains, static_cast<unsigned long long*>(d_sorted));
     return launch_status();
 }
@@ -344,3 +346,15 @@ int llvq_gemm_small_batch_noalloc(const llvq_ctx* ctx, const void* d_idx, const 
 }
 
 }  // extern "C"
+
+// llvq_gemv_sorted of the codes whose class tables stay in global memory: the batch-1 case of the sorted small-batch
+// product (same layout, same kernel), with the output type of the GEMV.  Called from gemv.cu.
+__attribute__((visibility("hidden")))
+int llvq_internal_gemv_domains(const llvq_ctx* ctx, const void* d_sorted, const uint16_t* d_gain_f16, int64_t n_out, int64_t k_in,
+                               const uint16_t* d_x_bf16, void* d_y, int y_dtype, void* stream)
+{
+    if (!gemm_sortable(ctx) || n_out > kMaxScratchRows || k_in <= 0) return LLVQ_EUNSUPPORTED;
+    if (!aligned(d_x_bf16, 16) || (k_in & 7)) return LLVQ_EALIGN;          // the tensor-core kernel stages x in 16-byte pieces
+    return launch_gemm_domains(ctx, d_sorted, d_gain_f16, n_out, k_in, d_x_bf16, 1, static_cast<uint16_t*>(d_y), ctx->d_scratch, ctx->d_counters,
+                               stream, nullptr, 0, nullptr, y_dtype == LLVQ_F32 ? 1 : 0);
+}

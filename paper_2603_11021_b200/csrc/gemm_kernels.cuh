@@ -31,6 +31,7 @@ struct GemmArgs {
     float* scratch;            // [npad][scratch_ld] binary32, all zero on entry and on exit
     int64_t scratch_ld;        // row tiles * 128
     uint32_t* counters;        // [row tiles], zero on entry and on exit
+    int y_f32;                 // Y holds binary32 instead of bf16 (the batch-1 product behind llvq_gemv_sorted of the 72-bit code)
 };
 
 __global__ void put_shard_kernel(YOut yo, YOut* dst)
@@ -45,6 +46,7 @@ __device__ __forceinline__ void gemm_store(const GemmArgs& ga, int n, int64_t or
 {
     const __nv_bfloat16 h = __float2bfloat16_rn(v);
     const int64_t at = (int64_t)n * ga.y_ld + orow;
+    if (!kShard && ga.y_f32) { reinterpret_cast<float*>(ga.y)[at] = v; return; }
     reinterpret_cast<__nv_bfloat16*>(ga.y)[at] = h;
     if (kShard) {
         const int np = ga.shard->n_peer;
@@ -255,16 +257,41 @@ sort_blocks_gemm_kernel(FastArgs fa, const uint32_t* __restrict__ stream, const 
     }
 }
 
-// The same layout for codes whose class tables live in global memory (72-bit indices): 128-bit entries, x = the low 64
-// bits of the stored index, y = its bits 64.. (8 bits) | class << 8 (24 bits) | position in the domain << 32 (10 bits);
-// bit 63 of y marks "no block" (ragged edge or index out of range).  The class rides along so that the GEMM kernel does
-// not search for it again; the blocks of a domain are ordered by unranking steps (most first), then by class, so that
-// the lanes of a warp run the same trip counts and read neighbouring class descriptors.
+// The same layout for codes whose class tables live in global memory (72-bit indices): 96-bit entries (three 32-bit
+// words): the stored index unchanged (bits 0..71), then 14 bits that name its class relative to the first class of
+// the index's bucket in the table on the top 16 index bits (so the kernel finds the class with one table read instead
+// of a bisection over 128-bit offsets), then the position in the domain (10 bits).  An index byte 64..71 of 0xff marks
+// "no block" (ragged edge or index out of range).  The blocks of a domain are ordered by the shape of their unranking:
+// parity (odd first), number of steps (most first), which of the steps take at most three slots, steps of the first
+// group; the lanes of a warp then run the same trip counts over similar slot counts and mostly agree on the cheap form
+// of a step.
+// Inside the kernels an entry travels as two 64-bit words: x = index bits 0..63, y = bits 64..71 | class << 8 |
+// position << 32, bit 63 = no block.
 constexpr unsigned long long kBigNoBlock = 1ull << 63;
+constexpr int kBigEntryWords = 3;
+constexpr uint32_t kBigDeltaMask = 0x3fffu;
+
+// Top 16 bits of a W-bit index (hi:lo): the bucket of the class table.
+__device__ __forceinline__ uint32_t big_bucket(const DevCode& dc, uint64_t lo, uint64_t hi)
+{
+    const int sh = dc.W > 16 ? dc.W - 16 : 0;
+    return (uint32_t)(sh >= 64 ? hi >> (sh - 64) : (sh ? (lo >> sh) | (hi << (64 - sh)) : lo)) & 0xffffu;
+}
+
+// Entry `at` of a sorted stream of 96-bit entries, in the two-word form the kernels use (one read of the bucket table).
+__device__ __forceinline__ ulonglong2 load_big_entry(const DevCode& dc, const void* sorted, int64_t at)
+{
+    const uint32_t* p = static_cast<const uint32_t*>(sorted) + at * kBigEntryWords;
+    const uint32_t w0 = __ldg(p), w1 = __ldg(p + 1), w2 = __ldg(p + 2);
+    const unsigned long long lo = (unsigned long long)w1 << 32 | w0, hi = w2 & 0xffu, pos = w2 >> 22;
+    if (hi == 0xffull) return make_ulonglong2(0ull, kBigNoBlock | pos << 32);
+    const uint32_t cls = __ldg(dc.lut16 + big_bucket(dc, lo, hi)) + ((w2 >> 8) & kBigDeltaMask);
+    return make_ulonglong2(lo, hi | (unsigned long long)cls << 8 | pos << 32);
+}
 
 __global__ void __launch_bounds__(kDomEntries, 1)
 sort_blocks_gemm_big_kernel(FastArgs fa, const uint32_t* __restrict__ stream, int64_t n_out, int64_t bpr, int64_t ndomains,
-                            ulonglong2* __restrict__ out)
+                            uint32_t* __restrict__ out)
 {
     __shared__ uint32_t keys[kDomEntries];
     __shared__ unsigned long long ex[kDomEntries], ey[kDomEntries];
@@ -273,7 +300,7 @@ sort_blocks_gemm_big_kernel(FastArgs fa, const uint32_t* __restrict__ stream, in
     for (int64_t dom = blockIdx.x; dom < ndomains; dom += gridDim.x) {
         const int64_t rt = dom / nd, d = dom - rt * nd;
         const int64_t row = rt * kGemmRows + (i >> 3), cb = d * kDomBlocks + (i & 7);
-        unsigned long long x = 0ull, y = kBigNoBlock | (unsigned long long)i << 32;
+        unsigned long long x = 0ull, y = 0xffull | (unsigned long long)i << 22;   // word 2 of an entry: index byte 0xff = no block
         uint32_t key = 0x7ffffc00u | (uint32_t)i;                   // no block: after everything else
         if (row < n_out && cb < bpr) {
             uint64_t lo, hi;
@@ -281,11 +308,14 @@ sort_blocks_gemm_big_kernel(FastArgs fa, const uint32_t* __restrict__ stream, in
             if (hi < fa.dc.n_hi || (hi == fa.dc.n_hi && lo < fa.dc.n_lo)) {
                 uint64_t local;
                 const uint32_t cls = (uint32_t)big_find_class(fa.dc, lo, hi, local);
-                const uint32_t h0y = __ldg(reinterpret_cast<const uint32_t*>(fa.dc.cls + cls) + 1);
-                const uint32_t nlev = (h0y & 0xff) + ((h0y >> 8) & 0xff);
+                const uint32_t* rec = reinterpret_cast<const uint32_t*>(fa.dc.big + cls);
+                const uint32_t h = __ldg(rec), small_k = __ldg(rec + 6) >> 24;
+                const uint32_t nlev = h >> 28, nlev1 = (h >> 24) & 7u, parity = (h >> 16) & 1u;
+                const uint32_t delta = cls - __ldg(fa.dc.lut16 + big_bucket(fa.dc, lo, hi));      // < 2^14: checked when the context was made
                 x = lo;
-                y = (hi & 0xffull) | (unsigned long long)cls << 8 | (unsigned long long)i << 32;
-                key = (15u - min(nlev, 15u)) << 27 | cls << 10 | (uint32_t)i;
+                y = (hi & 0xffull) | (unsigned long long)delta << 8 | (unsigned long long)i << 22;
+                // odd classes first (their steps choose among up to 24 slots, the even classes' among at most 16), then by steps
+                key = (1u - parity) << 24 | (7u - min(nlev, 7u)) << 21 | (small_k & 0x7fu) << 14 | nlev1 << 11 | (uint32_t)i;
             } else {
                 atomicAdd(fa.bad_index, 1ull);
             }
@@ -302,7 +332,8 @@ sort_blocks_gemm_big_kernel(FastArgs fa, const uint32_t* __restrict__ stream, in
                 __syncthreads();
             }
         const uint32_t src = keys[i] & 1023u;
-        out[dom * kDomEntries + i] = make_ulonglong2(ex[src], ey[src]);
+        uint32_t* o = out + (dom * kDomEntries + i) * kBigEntryWords;
+        o[0] = (uint32_t)ex[src]; o[1] = (uint32_t)(ex[src] >> 32); o[2] = (uint32_t)ey[src];
         __syncthreads();
     }
 }
@@ -362,7 +393,7 @@ gemm_sorted_kernel(FastArgs fa, const unsigned long long* __restrict__ sorted, c
             // warps pair chunk w - 1 of the first domain with chunk 31 - w of the second
             const int chunk = warp == 0 ? 31 : (q == 0 ? warp - 1 : 31 - warp);
             const int64_t at = (rt * nd + d + q) * kDomEntries + chunk * 32 + lane;
-            if (kBig) return __ldg(reinterpret_cast<const ulonglong2*>(sorted) + at);
+            if (kBig) return load_big_entry(fa.dc, sorted, at);
             return make_ulonglong2(__ldg(sorted + at), 0ull);
         };
         ulonglong2 e0 = entry_at(d_begin, 0), e1 = dpi > 1 ? entry_at(d_begin, 1) : no_entry;
@@ -387,13 +418,10 @@ gemm_sorted_kernel(FastArgs fa, const unsigned long long* __restrict__ sorted, c
                 if (kBig) {
                     const int cls = valid ? (int)((uint32_t)(e.y >> 8) & 0xffffffu) : 0;
                     const uint64_t local = valid ? e.x - __ldg(fa.dc.off_lo + cls) : 0ull;     // class sizes fit 63 bits: exact mod 2^64
-                    Point pt;
-                    big_decode_local(T, fa.dc, cls, local, valid, pt);
-#pragma unroll
-                    for (int j = 0; j < 12; ++j) {
-                        __nv_bfloat162 h = __halves2bfloat162(dequant(gn, pt, 2 * j), dequant(gn, pt, 2 * j + 1));
-                        w[j] = *reinterpret_cast<uint32_t*>(&h);
-                    }
+                    DecodedBig dec{};
+                    big_decode_planes(T, fa.dc, cls, local, valid, kFullMask, dec);
+                    expand_bf16(dec.d, gn, w);
+                    patch_id8_bf16(dec, gn, w);
                 } else {
                     Decoded dec{};
                     const uint32_t cls = decode_sorted_entry(fa, T, I, valid, dec);
@@ -620,7 +648,7 @@ gemm_pipe_kernel(FastArgs fa, const unsigned long long* __restrict__ sorted, con
                     return make_ulonglong2(f | (unsigned long long)pos << 48, 0ull);
                 }
                 const int64_t at = (rt * nd + d_begin + (int)(t >> 5)) * kDomEntries + (t & 31u) * 32u + lane;
-                if (kBig) return __ldg(reinterpret_cast<const ulonglong2*>(sorted) + at);
+                if (kBig) return load_big_entry(fa.dc, sorted, at);
                 return make_ulonglong2(__ldg(sorted + at), 0ull);
             };
             uint32_t tk = (uint32_t)warp - 1u;
@@ -653,13 +681,10 @@ gemm_pipe_kernel(FastArgs fa, const unsigned long long* __restrict__ sorted, con
                         cls = (int)((uint32_t)(e.y >> 8) & 0xffffffu);
                         local = e.x - __ldg(fa.dc.off_lo + cls);                 // class sizes fit 63 bits: exact mod 2^64
                     }
-                    Point pt;
-                    big_decode_local(T, fa.dc, cls, local, valid, pt);
-#pragma unroll
-                    for (int jj = 0; jj < 12; ++jj) {
-                        __nv_bfloat162 h = __halves2bfloat162(dequant(gn, pt, 2 * jj), dequant(gn, pt, 2 * jj + 1));
-                        w[jj] = *reinterpret_cast<uint32_t*>(&h);
-                    }
+                    DecodedBig dec{};
+                    big_decode_planes(T, fa.dc, cls, local, valid, kFullMask, dec);
+                    expand_bf16(dec.d, gn, w);
+                    patch_id8_bf16(dec, gn, w);
                 } else {
                     Decoded dec{};
                     uint32_t cls;

@@ -2,6 +2,9 @@
 // form and the row-sharded variants, with the kernels they launch (gemv_kernels.cuh).
 #include "kernels_common.cuh"
 
+int llvq_internal_gemv_domains(const llvq_ctx* ctx, const void* d_sorted, const uint16_t* d_gain_f16, int64_t n_out, int64_t k_in,
+                               const uint16_t* d_x_bf16, void* d_y, int y_dtype, void* stream);      // gemm.cu
+
 namespace {
 
 #include "gemv_kernels.cuh"
@@ -54,7 +57,7 @@ int gemv_common(const llvq_ctx* ctx, const void* d_idx, const uint16_t* d_gain_f
     const int64_t nq = (bpr + 3) / 4;
     const size_t kSmemMax = 227 * 1024;
     const size_t rest = 16 + (size_t)nq * 48 * 4 + kGemvGroupsPerPass * kGemvGroupRows * 4 + 16;
-    const bool ext_direct = ctx->fast && ctx->fl.total_ext + rest <= kSmemMax;      // room for the table of small subsets
+    const bool ext_direct = ctx->fl.total_ext + rest <= kSmemMax;      // room for the table of small subsets
     const size_t smem = (ext_direct ? ctx->fl.total_ext : ctx->fl.total) + rest;
     if (smem > kSmemMax || n_out > 64ll * kMaxScratchRows) return LLVQ_EUNSUPPORTED;
     const int64_t units = ((n_out + kGemvGroupRows - 1) / kGemvGroupRows) * nq;
@@ -144,6 +147,7 @@ int llvq_gemv_sg(const llvq_ctx* ctx, const void* d_fields, int gain_bits, const
 
 size_t llvq_sorted_bytes(const llvq_ctx* ctx, int64_t n_out, int64_t k_in)
 {
+    if (ctx && !ctx->fast) return llvq_sorted_gemm_bytes(ctx, n_out, k_in);      // one sorted layout serves both products of these codes
     if (!ctx || ctx->device < 0 || n_out <= 0 || k_in <= 0 || !sortable(ctx, k_in)) return 0;
     const int64_t nq = ((k_in + 23) / 24 + 3) / 4;
     return (size_t)(((n_out + kGemvGroupRows - 1) / kGemvGroupRows) * nq) * 32 * 8;
@@ -169,6 +173,7 @@ static int sort_blocks_common(const llvq_ctx* ctx, const void* d_fields, int gai
 
 int llvq_sort_blocks(const llvq_ctx* ctx, const void* d_idx, int64_t n_out, int64_t k_in, void* d_sorted, void* stream)
 {
+    if (ctx && !ctx->fast) return llvq_sort_blocks_gemm(ctx, d_idx, n_out, k_in, d_sorted, stream);
     return sort_blocks_common(ctx, d_idx, 0, n_out, k_in, d_sorted, stream);
 }
 
@@ -219,6 +224,11 @@ int llvq_gemv_sorted(const llvq_ctx* ctx, const void* d_sorted, const uint16_t* 
     if (int e = check_common(ctx, d_sorted)) return e;
     if (!d_gain_f16) return LLVQ_EINVAL;
     if (!aligned(d_gain_f16, 2)) return LLVQ_EALIGN;
+    if (!ctx->fast) {
+        if (!d_x_bf16 || n_out < 0 || k_in <= 0) return LLVQ_EINVAL;
+        if (int e = check_yout(single_y(d_y), y_dtype)) return e;
+        return llvq_internal_gemv_domains(ctx, d_sorted, d_gain_f16, n_out, k_in, d_x_bf16, d_y, y_dtype, stream);
+    }
     return gemv_sorted_common(ctx, d_sorted, d_gain_f16, nullptr, n_out, k_in, d_x_bf16, single_y(d_y), y_dtype, stream);
 }
 

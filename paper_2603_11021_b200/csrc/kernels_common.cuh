@@ -8,6 +8,7 @@
 
 #include <algorithm>
 #include <cstdio>
+#include <cstdlib>
 #include <cstring>
 #include <mutex>
 #include <new>
@@ -70,9 +71,9 @@ struct FastArgs {
 // One block of 24 weights, end to end, in the two forms the consumers use.  kBig selects the decoder for codes
 // whose class tables live in global memory; otherwise everything is served from the shared-memory image.
 // All 32 lanes of a warp call these together; `in` = the block exists.
-template <bool kBig>
-__device__ __forceinline__ void block_point(const FastArgs& fa, const FastSmem& T, const uint32_t* __restrict__ stream,
-                                            uint64_t b, bool in, Point& pt)
+// The table-driven decoder of the codes whose class tables stay in global memory, from the stored stream.
+__device__ __forceinline__ void block_planes_big(const FastArgs& fa, const FastSmem& T, const uint32_t* __restrict__ stream,
+                                                 uint64_t b, bool in, DecodedBig& d)
 {
     uint64_t lo = 0, hi = 0;
     if (in) load_index(stream, b, fa.dc.W, lo, hi);
@@ -80,7 +81,7 @@ __device__ __forceinline__ void block_point(const FastArgs& fa, const FastSmem& 
     if (in && !valid) atomicAdd(fa.bad_index, 1ull);
     uint64_t local = 0;
     const int cls = valid ? big_find_class(fa.dc, lo, hi, local) : 0;
-    big_decode_local(T, fa.dc, cls, local, valid, pt);
+    big_decode_planes(T, fa.dc, cls, local, valid, kFullMask, d);
 }
 
 template <bool kBig>
@@ -88,10 +89,12 @@ __device__ __forceinline__ void block_bytes(const FastArgs& fa, const FastSmem& 
                                             uint64_t b, bool in, uint32_t w[6])
 {
     if (kBig) {
-        Point pt;
-        block_point<kBig>(fa, T, stream, b, in, pt);
-#pragma unroll
-        for (int i = 0; i < 6; ++i) w[i] = pt.w[i];
+        DecodedBig d{};
+        block_planes_big(fa, T, stream, b, in, d);
+        Decoded three = d.d;
+        three.neg &= ~d.p3;                               // those positions are written by the patch (a negated zero filler would carry)
+        expand_bytes(three, w);
+        patch_id8_bytes(d, w);
     } else {
         const uint64_t I = in ? load_field(stream, b, (int)fa.L.W) : 0ull;
         const bool valid = in && I < fa.n_points;
@@ -108,13 +111,10 @@ __device__ __forceinline__ void block_pairs(const FastArgs& fa, const FastSmem& 
 {
     const float g = in ? gain_to_float(__ldg(gain + b)) : 0.f;
     if (kBig) {
-        Point pt;
-        block_point<kBig>(fa, T, stream, b, in, pt);
-#pragma unroll
-        for (int j = 0; j < 12; ++j) {
-            __nv_bfloat162 h = __halves2bfloat162(dequant(g, pt, 2 * j), dequant(g, pt, 2 * j + 1));
-            w[j] = *reinterpret_cast<uint32_t*>(&h);
-        }
+        DecodedBig d{};
+        block_planes_big(fa, T, stream, b, in, d);
+        expand_bf16(d.d, g, w);
+        patch_id8_bf16(d, g, w);
     } else {
         const uint64_t I = in ? load_field(stream, b, (int)fa.L.W) : 0ull;
         const bool valid = in && I < fa.n_points;

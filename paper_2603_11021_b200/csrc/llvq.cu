@@ -86,6 +86,17 @@ int llvq_create(llvq_ctx** out, int m_lo, int m_hi, int device)
     if (!ctx->fast && !build_fast_image(h, ctx->fl, image, false)) { delete ctx; return LLVQ_EUNSUPPORTED; }
     std::vector<uint32_t> lut16;
     build_bucket_table(h, lut16);
+    for (size_t b = 0; b + 1 < lut16.size(); ++b) ctx->bucket_classes_max = std::max(ctx->bucket_classes_max, (int)(lut16[b + 1] - lut16[b]));
+    // class records in global memory: the full descriptors where the encoder's indexing kernel reads them (codes with their
+    // tables in shared memory), the compact 32-byte records for the codes whose decoders read them from global memory
+    std::vector<BigDesc> big;
+    if (!ctx->fast) {
+        if (h.max_levels > kMaxLevels - 1) { delete ctx; return LLVQ_EUNSUPPORTED; }
+        build_big_descs(h, big);
+    }
+    const bool full_descs = ctx->fast || h.W <= 64;      // the encoder's indexing kernel reads them
+    const size_t cls_bytes = (full_descs ? ncls * sizeof(ClassDesc) : 0) + 256 + big.size() * sizeof(BigDesc);
+    const size_t big_at = ((full_descs ? ncls * sizeof(ClassDesc) : 0) + 255) & ~size_t(255);
 
     // encoder tables (point -> index), for codes the encoder supports
     std::vector<uint64_t> hkeys; std::vector<uint32_t> hcls;
@@ -107,7 +118,7 @@ int llvq_create(llvq_ctx** out, int m_lo, int m_hi, int device)
     size_t o_offhi = 0;
     size_t o_offlo = up(o_offhi + (ncls + 1) * 4);
     size_t o_cls = up(o_offlo + (ncls + 1) * 8);
-    size_t o_lut = up(o_cls + ncls * sizeof(ClassDesc));
+    size_t o_lut = up(o_cls + cls_bytes);
     size_t o_err = up(o_lut + lut16.size() * 4);
     size_t o_img = up(o_err + 256);
     size_t o_gol = up(o_img + image.size());
@@ -137,7 +148,8 @@ int llvq_create(llvq_ctx** out, int m_lo, int m_hi, int device)
     std::vector<uint8_t> blob(o_cnt, 0);
     std::memcpy(blob.data() + o_offhi, off_hi.data(), (ncls + 1) * 4);
     std::memcpy(blob.data() + o_offlo, off_lo.data(), (ncls + 1) * 8);
-    std::memcpy(blob.data() + o_cls, h.desc.data(), ncls * sizeof(ClassDesc));
+    if (full_descs) std::memcpy(blob.data() + o_cls, h.desc.data(), ncls * sizeof(ClassDesc));
+    if (!big.empty()) std::memcpy(blob.data() + o_cls + big_at, big.data(), big.size() * sizeof(BigDesc));
     std::memcpy(blob.data() + o_lut, lut16.data(), lut16.size() * 4);
     std::memcpy(blob.data() + o_img, image.data(), image.size());
     std::memcpy(blob.data() + o_gol, h.golay.data(), 4096 * 4);
@@ -156,7 +168,8 @@ int llvq_create(llvq_ctx** out, int m_lo, int m_hi, int device)
     uint8_t* d = static_cast<uint8_t*>(ctx->d_blob);
     ctx->dev.off_hi = reinterpret_cast<const uint32_t*>(d + o_offhi);
     ctx->dev.off_lo = reinterpret_cast<const uint64_t*>(d + o_offlo);
-    ctx->dev.cls = reinterpret_cast<const ClassDesc*>(d + o_cls);
+    ctx->dev.cls = full_descs ? reinterpret_cast<const ClassDesc*>(d + o_cls) : nullptr;
+    ctx->dev.big = big.empty() ? nullptr : reinterpret_cast<const BigDesc*>(d + o_cls + big_at);
     ctx->dev.lut16 = reinterpret_cast<const uint32_t*>(d + o_lut);
     ctx->d_err = reinterpret_cast<unsigned long long*>(d + o_err);
     ctx->dev.bad_index = ctx->d_err;

@@ -232,7 +232,14 @@ bool build_fast_image(const HostTables& t, FastLayout& L, std::vector<uint8_t>& 
     L.pd6 = up16(L.r14 + r14.size() * 2);
     L.off = up16(L.pd6 + 4096);
     L.desc = up16(L.off + (with_classes ? (ncls + 1) * 8 : 0));
-    L.total = up16(L.desc + ncls * kFastDescStride * 4);
+    L.recip64 = L.recip32 = 0;
+    size_t end = L.desc + ncls * kFastDescStride * 4;
+    if (!with_classes) {                                   // the class-independent reciprocals the compact class records rely on
+        L.recip64 = up16(end);
+        L.recip32 = up16(L.recip64 + 625 * 8);
+        end = L.recip32 + 625 * 4;
+    }
+    L.total = up16(end);
     L.sub3 = L.total;
     L.total_ext = up16(L.sub3 + kSmallSubsetWords * 4);
     L.lut_shift = (uint32_t)(t.W >= 12 ? t.W - 12 : 0);
@@ -265,7 +272,16 @@ bool build_fast_image(const HostTables& t, FastLayout& L, std::vector<uint8_t>& 
                 if ((f >> b) & 1u) { if (src & 1u) out |= 1u << b; src >>= 1; }
             img[L.pd6 + (f << 6 | s)] = (uint8_t)out;
         }
-    if (!with_classes) return true;                        // small tables only: the class tables stay in global memory
+    if (!with_classes) {                                   // small tables only: the class tables stay in global memory
+        uint64_t* r64 = reinterpret_cast<uint64_t*>(img.data() + L.recip64);
+        uint32_t* r32 = reinterpret_cast<uint32_t*>(img.data() + L.recip32);
+        for (int i = 0; i < 625; ++i) {
+            const uint32_t c = t.pascal[i];
+            r64[i] = c ? ~0ull / c : 0ull;
+            r32[i] = c > 1 ? (uint32_t)((1ull << 32) / c) : 0xffffffffu;
+        }
+        return true;
+    }
     // class lookup by the top 12 bits of the index
     uint16_t* lut = reinterpret_cast<uint16_t*>(img.data() + L.lut);
     size_t c = 0;
@@ -312,6 +328,29 @@ bool build_fast_image(const HostTables& t, FastLayout& L, std::vector<uint8_t>& 
         std::memcpy(&w[kFastDescRnorm], &rnorm, 4);
     }
     return true;
+}
+
+void build_big_descs(const HostTables& t, std::vector<BigDesc>& out)
+{
+    out.assign(t.desc.size(), BigDesc{});
+    for (size_t j = 0; j < t.desc.size(); ++j) {
+        const ClassDesc& d = t.desc[j];
+        BigDesc& b = out[j];
+        const int nlev = d.nlev1 + d.nlev0;
+        b.w = d.w; b.B = d.B;
+        b.flags = (uint8_t)((d.parity ? 1u : 0u) | (d.signpar ? 2u : 0u) | (d.fill0 ? 4u : 0u) | ((d.fill1 & 2) ? 8u : 0u) | ((d.fill0 & 2) ? 16u : 0u));
+        b.nlev = (uint8_t)(d.nlev1 | nlev << 4);
+        b.goff = d.goff; b.A = d.A;
+        b.val[0] = d.fill0; b.val[1] = d.fill1;
+        for (int l = 0; l < nlev && l < kMaxLevels - 1; ++l) {
+            const LevelDesc& lv = d.lev[l];
+            if (l < 6) b.val[2 + l] = lv.val; else b.val8 = lv.val;
+            b.k[l] = lv.k;
+            if (lv.val & 2) b.lvl_bit1 |= (uint8_t)(1u << l);
+            if (lv.val) b.lvl_nz |= (uint8_t)(1u << l);
+            if (lv.k <= kSmallSubsetMaxK) b.small_k |= (uint8_t)(1u << l);
+        }
+    }
 }
 
 // Class of the first index of every bucket (I >> (W - 16)), plus a final entry = last class: the class of an

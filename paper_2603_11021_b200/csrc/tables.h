@@ -46,6 +46,25 @@ struct ClassDesc {
 };
 static_assert(sizeof(ClassDesc) == 32 + 16 * kMaxLevels, "ClassDesc layout");
 
+// Compact form of ClassDesc for the codes whose class tables stay in global memory (32 bytes, two 16-byte loads): the
+// radix of a step is C(free slots, k) from the Pascal triangle in shared memory and its reciprocals come from two tables
+// beside it, so only the multiplicities and the values are stored per class.  Value ids: 0 = filler of group 0,
+// 1 = filler of group 1, 2 + l = level l.
+struct BigDesc {
+    uint8_t w, B;
+    uint8_t flags;         // bit0 parity, bit1 signpar, bit2 fill0 is nonzero, bit3 fill1 has value bit 1, bit4 fill0 has value bit 1
+    uint8_t nlev;          // nlev1 | (nlev1 + nlev0) << 4
+    uint16_t goff, A;
+    uint8_t val[8];        // absolute value of ids 0..7
+    uint8_t k[8];          // slots taken by level 0..7 (bytes 7 unused: at most 7 levels)
+    uint8_t val8;          // absolute value of id 8 (classes with 9 distinct values)
+    uint8_t lvl_bit1;      // bit l: the value of level l has value bit 1 (= 2 or 3 mod 4)
+    uint8_t lvl_nz;        // bit l: the value of level l is nonzero
+    uint8_t small_k;       // bit l: level l takes at most kSmallSubsetMaxK slots (part of the sorted layouts' key)
+    uint32_t pad;
+};
+static_assert(sizeof(BigDesc) == 32, "BigDesc layout");
+
 struct ClassInfo {           // host-only description, for queries and tests
     int m, parity, w, B;
     uint64_t A;
@@ -98,6 +117,8 @@ struct FastLayout {
     uint32_t off;         // u64[ncls + 1]
     uint32_t desc;        // u32[ncls][kFastDescStride]
     uint32_t total;       // bytes of the image proper, multiple of 16
+    uint32_t recip64;     // u64[25*25] floor((2^64 - 1) / C(n, k)) and
+    uint32_t recip32;     // u32[25*25] floor(2^32 / C(n, k)) (0xffffffff for C = 1): images without class tables only, else 0
     uint32_t sub3;        // u32[kSmallSubsetWords], behind the image proper: kernels with room for it load total_ext bytes
     uint32_t total_ext;   // bytes including sub3, multiple of 16
     uint32_t lut_shift;
@@ -121,6 +142,7 @@ struct FastLayout {
 // with_classes = false builds only the class-independent tables (Golay, Pascal, subsets, deposit): codes whose class
 // tables do not fit shared memory keep those in global memory.
 bool build_fast_image(const HostTables& t, FastLayout& layout, std::vector<uint8_t>& image, bool with_classes = true);
+void build_big_descs(const HostTables& t, std::vector<BigDesc>& out);
 void build_bucket_table(const HostTables& t, std::vector<uint32_t>& lut);   // u32[65537], see tables.cpp
 
 // Encoder side (point -> class).  Signature of a class: sum over its 24 absolute values of a fixed pseudo-random

@@ -546,12 +546,26 @@ def test_gemv_at_the_largest_row_count(lib, ctxs, oracle_mod):
     assert ctx._lib.llvq_gemv(ctx._h, ds.data_ptr(), dg.data_ptr(), n_out + 8, k_in, dx.data_ptr(), y.data_ptr(), 0, None) == 3
 
 
-def test_sorted_layout_unsupported_for_the_72_bit_code(lib, ctxs):
+@pytest.mark.parametrize("n_out,k_in", [(4096, 4096), (200, 1000), (129, 24)])
+def test_gemv_72bit_stored_and_sorted_all_rows(lib, ctxs, oracle_mod, n_out, k_in):
+    # the ~3 bits/weight code: the fused product on the stored stream and on the sorted layout (for this code the layout
+    # of the small-batch product serves both), both output types, every row against the oracle
+    o = _oracle(oracle_mod)((2, 53))
     ctx = ctxs[(2, 53)]
-    assert ctx._lib.llvq_sorted_bytes(ctx._h, 64, 96) == 0
-    buf = torch.zeros(4096, dtype=torch.uint8, device="cuda")
-    assert ctx._lib.llvq_sort_blocks(ctx._h, buf.data_ptr(), 16, 96, buf.data_ptr(), None) == 3
-    assert ctx._lib.llvq_gemv_sorted(ctx._h, buf.data_ptr(), buf.data_ptr(), 16, 96, buf.data_ptr(), buf.data_ptr(), 0, None) == 3
+    stream, gain, _ = gen.make_layer(o.N, o.W, n_out, k_in, 1, seed=31)
+    x = gen.normal_bf16(k_in, seed=31)
+    ds, dg, dx = to_dev_u8(stream), to_dev_f16(gain), to_dev_bf16(x)
+    ref = o.gemv(stream, gain, n_out, k_in, x, threads=_threads())
+    assert ctx._lib.llvq_sorted_bytes(ctx._h, n_out, k_in) == ctx._lib.llvq_sorted_gemm_bytes(ctx._h, n_out, k_in) > 0
+    srt = lib.llvq_sort_blocks(ctx, ds, n_out, k_in)
+    assert torch.equal(srt, lib.llvq_sort_blocks_gemm(ctx, ds, n_out, k_in))
+    for dt, tol in ((torch.float32, TOL), (torch.bfloat16, TOL_BF16_OUT)):
+        y = lib.llvq_gemv(ctx, ds, dg, n_out, k_in, dx, y_dtype=dt)
+        ys = lib.llvq_gemv_sorted(ctx, srt, dg, n_out, k_in, dx, y_dtype=dt)
+        torch.cuda.synchronize()
+        assert gemv_error(y.float().cpu().numpy(), ref) <= tol
+        assert gemv_error(ys.float().cpu().numpy(), ref) <= tol
+    assert lib.llvq_last_error(ctx) == (0, 0)
 
 
 def test_back_to_back_launches_see_the_previous_result(lib, ctxs, oracle_mod):
@@ -600,7 +614,7 @@ def test_gemm_sorted_small_shapes(lib, ctxs, oracle_mod, code, n_out, k_in, batc
     x = gen.normal_bf16((batch, k_in), seed=24)
     want = o.gemm(stream, gain, n_out, k_in, x, threads=4)
     srt = lib.llvq_sort_blocks_gemm(ctx, to_dev_u8(stream), n_out, k_in)
-    entry_bytes = 16 if o.W > 48 else 8                      # the 72-bit code keeps index, class and position in 128 bits
+    entry_bytes = 12 if o.W > 48 else 8                      # the 72-bit code keeps index, class within its bucket and position in 96 bits
     assert srt.numel() == 1024 * entry_bytes * ((n_out + 127) // 128) * (((k_in + 23) // 24 + 7) // 8)
     y = lib.llvq_gemm_small_batch_sorted(ctx, srt, to_dev_f16(gain), n_out, k_in, to_dev_bf16(x))
     y_plain = lib.llvq_gemm_small_batch(ctx, to_dev_u8(stream), to_dev_f16(gain), n_out, k_in, to_dev_bf16(x))
@@ -644,44 +658,50 @@ def test_sort_blocks_gemm_is_a_permutation_inside_every_domain(lib, ctxs, oracle
 
 
 def test_sort_blocks_gemm_72bit_entries(lib, ctxs, oracle_mod):
-    # 128-bit entries: the stored index unchanged, its class, its position; inside a domain every class forms one
-    # run (the order is by unranking steps, then class, then position); entries without a block last
+    # 96-bit entries: the stored index unchanged, its class relative to the first class of its bucket (top 16 index bits),
+    # its position; a domain is ordered by the shape of the unranking (odd classes first, then by number of steps, most
+    # first); entries without a block come last
     o = _oracle(oracle_mod)((2, 53))
     ctx = ctxs[(2, 53)]
     n_out, k_in = 200, 1000                                 # 2 row tiles, 42 blocks per row -> 6 domains per tile, ragged both ways
     bpr, nd = 42, 6
     stream, _, nblocks = gen.make_layer(o.N, o.W, n_out, k_in, 1, seed=26)
     idx = o.unpack(stream, nblocks)
-    e = lib.llvq_sort_blocks_gemm(ctx, to_dev_u8(stream), n_out, k_in).cpu().numpy().view(np.uint64).reshape(2 * nd, 1024, 2)
-    offs = [c["offset"] for c in o.classes()] + [o.N]
+    e = lib.llvq_sort_blocks_gemm(ctx, to_dev_u8(stream), n_out, k_in).cpu().numpy().view(np.uint32).reshape(2 * nd, 1024, 3)
+    classes = o.classes()
+    offs = [c["offset"] for c in classes] + [o.N]
     import bisect
+
+    def steps(c):
+        if c["parity"]:
+            return len(c["values"]) - 1
+        g1 = sum(1 for v in c["values"] if v % 4 == 2)
+        g0 = len(c["values"]) - g1
+        return max(g1 - 1, 0) + max(g0 - 1, 0)
     seen = set()
     for dom in range(2 * nd):
         rt, d = divmod(dom, nd)
-        positions, last_key, closed = set(), (-1, -1), set()
-        for x, y in e[dom].tolist():
-            pos = (y >> 32) & 1023
+        positions, last_key, ended = set(), (-1, -99), False
+        for w0, w1, w2 in e[dom].tolist():
+            pos = w2 >> 22
             row, cb = rt * 128 + pos // 8, d * 8 + pos % 8
             assert pos not in positions
             positions.add(pos)
-            if y >> 63:
+            if (w2 & 0xff) == 0xff:
                 assert row >= n_out or cb >= bpr
-                closed.add(last_key[0])
-                last_key = (-2, 0)                          # nothing with a block may follow
+                ended = True                                # nothing with a block may follow
                 continue
-            assert last_key[0] != -2
-            I, cls = x | (y & 0xff) << 64, (y >> 8) & 0xffffff
+            assert not ended
+            I = w0 | w1 << 32 | (w2 & 0xff) << 64
             b = row * bpr + cb
             assert idx[b] == I and b not in seen
             seen.add(b)
-            assert cls == bisect.bisect_right(offs, I) - 1
-            # the key is a function of the class (then the position): a class forms one run, positions ascending inside
-            if cls == last_key[0]:
-                assert pos > last_key[1]
-            else:
-                assert cls not in closed
-                closed.add(last_key[0])
-            last_key = (cls, pos)
+            cls = bisect.bisect_right(offs, I) - 1
+            first_of_bucket = bisect.bisect_right(offs, (I >> 56) << 56) - 1
+            assert (w2 >> 8) & 0x3fff == cls - first_of_bucket
+            key = (1 - classes[cls]["parity"], -steps(classes[cls]))
+            assert key >= last_key
+            last_key = key
     assert len(seen) == nblocks
     assert lib.llvq_last_error(ctx) == (0, 0)
 
@@ -690,7 +710,7 @@ def test_gemm_sorted_unsupported_and_arguments(lib, ctxs):
     buf = torch.zeros(8192, dtype=torch.uint8, device="cuda")
     p = buf.data_ptr()
     big = ctxs[(2, 53)]
-    assert big._lib.llvq_sorted_gemm_bytes(big._h, 64, 96) == 1024 * 16
+    assert big._lib.llvq_sorted_gemm_bytes(big._h, 64, 96) == 1024 * 12
     ctx = ctxs[(2, 13)]
     assert ctx._lib.llvq_sorted_gemm_bytes(ctx._h, 64, 96) == 1024 * 8
     assert ctx._lib.llvq_gemm_small_batch_sorted(ctx._h, p, p, 16, 96, p, 65, p, None) == 1       # batch out of range
