@@ -4,10 +4,12 @@
 A "step" is one pass of the fused dequant+GEMV (batch 1) over the three
 7B-shaped layers of the headline workload -- 4096x4096, 11008x4096 and
 4096x11008 at ~2 bits/weight (48-bit indices over the union of shells 2..13,
-fp16 gain per block of 24), bf16 activations, fp32 accumulation, bf16 output.
-Inputs are seeded and synthetic (uniform indices, |N(0,1)|*0.02 gains, N(0,1)
-activations).  The metric is algorithmic GB/s: compressed index + gain +
-activation + output bytes per second, the numerator of the HBM roofline.
+fp16 gain per block of 24), bf16 activations, fp32 accumulation, bf16 output:
+one llvq_gemv_sorted_multi launch on the layers' load-time sorted layout (the
+same step on the stored streams is timed beside it).  Inputs are seeded and
+synthetic (uniform indices, |N(0,1)|*0.02 gains, N(0,1) activations).  The
+metric is algorithmic GB/s: compressed index + gain + activation + output
+bytes per second, the numerator of the HBM roofline.
 
 Timing: CUDA events on the launching stream; the step rotates over several
 distinct copies of the layers whose total size exceeds L2, so no timed
@@ -39,11 +41,11 @@ METRIC = "fused dequant+GEMV algorithmic GB/s (index+gain+activation+output byte
 UNIT = "GB/s"
 WORKLOAD = "configs[2]: fused dequant+GEMV batch 1 on W 4096x4096, 11008x4096, 4096x11008, 48-bit indices (shells 2..13), fp16 gain per 24 weights"
 
-# dram__bytes_read.sum + dram__bytes_write.sum of one gemv_fast_kernel launch on the 11008x4096 layer, from the
-# ncu capture summarised under profiles/ (algorithmic bytes: 15 089 152)
-NCU_TRAFFIC_BYTES_11008x4096 = 15262208
-NCU_WARP_INSTRUCTIONS_11008x4096 = 55592066          # smsp__inst_executed.sum of the same capture
+# Counters of the committed ncu capture of the headline kernel (written by paper_2603_11021_b200.ncu_counters next to the
+# capture's summary); quoted only while the kernel sources still hash to what the capture ran.
+COUNTER_FILE = os.path.join(ROOT, "profiles", "gemv_sorted_multi_kernel_7B_step_counters.json")
 ISSUE_PEAK_WARP_INST_PER_S = 148 * 4 * 1.965e9       # SMs x schedulers x max SM clock: one warp instruction per scheduler and cycle
+ALU_PEAK_WARP_INST_PER_S = 148 * 4 * 1.965e9 / 2     # the integer / logic pipe takes a warp instruction every other cycle per scheduler
 
 
 def layer_bytes(n_out: int, k_in: int) -> dict:
@@ -200,8 +202,29 @@ def cpu_baseline() -> dict:
 
 def profile_run(P, ctx, args) -> None:
     """A handful of launches of one kernel on buffers that do not fit L2 together, for profiler captures:
-    gemv = the 11008x4096 layer, dequant = 4096x4096 FLAT, gemm = 8192x8192 at batch 16."""
+    gemv* = the 11008x4096 layer, step_* = the three-layer step in one launch, dequant = 4096x4096 FLAT, gemm* = 8192x8192 at batch 16."""
     import torch
+    if args.profile in ("step_sorted_multi", "step_multi"):
+        srt = args.profile == "step_sorted_multi"
+        step_bytes = sum(algorithmic_bytes(n, k) for n, k in LAYERS)
+        copies = max(2, -(-2 * L2_BYTES // step_bytes))
+        sets = []
+        for c in range(copies):
+            mats = []
+            for li, (n, k) in enumerate(LAYERS):
+                stream, gain, x, _ = host_layer(n, k, seed=rank_seed(0, c, li))
+                d_w = torch.from_numpy(stream).cuda()
+                if srt:
+                    d_w = P.llvq_sort_blocks(ctx, d_w, n, k)
+                mats.append((d_w, torch.from_numpy(gain.view(np.float16)).cuda(), n, k,
+                             torch.from_numpy(x.view(np.int16)).cuda().view(torch.bfloat16), torch.empty(n, dtype=torch.bfloat16, device="cuda")))
+            sets.append(mats)
+        call = P.llvq_gemv_sorted_multi if srt else P.llvq_gemv_multi
+        for i in range(args.warmup + args.steps):
+            call(ctx, sets[i % copies], y_dtype=torch.bfloat16)
+        torch.cuda.synchronize()
+        print(json.dumps({"profile": args.profile, "launches": args.warmup + args.steps, "copies": copies, "errors": P.llvq_last_error(ctx)}))
+        return
     n, k = {"gemv": (11008, 4096), "gemv_sorted": (11008, 4096), "dequant": (4096, 4096), "gemm": (8192, 8192), "gemm_sorted": (8192, 8192),
             "gemm_72bit": (8192, 8192), "gemm_sorted_72bit": (8192, 8192)}[args.profile]
     code_n, code_w = CODE_N, CODE_W
@@ -226,9 +249,9 @@ def profile_run(P, ctx, args) -> None:
     for i in range(args.warmup + args.steps):
         d_idx, d_gain = bufs[i % copies]
         if args.profile == "gemv":
-            P.llvq_gemv(ctx, d_idx, d_gain, n, k, x[0], d_y=y[:n])
+            P.llvq_gemv(ctx, d_idx, d_gain, n, k, x[0], d_y=y[:n], y_dtype=torch.bfloat16)
         elif args.profile == "gemv_sorted":
-            P.llvq_gemv_sorted(ctx, d_idx, d_gain, n, k, x[0], d_y=y[:n])
+            P.llvq_gemv_sorted(ctx, d_idx, d_gain, n, k, x[0], d_y=y[:n], y_dtype=torch.bfloat16)
         elif args.profile.startswith("gemm_sorted"):
             P.llvq_gemm_small_batch_sorted(ctx, d_idx, d_gain, n, k, x, d_y=y.view(16, n))
         elif args.profile == "dequant":
@@ -362,6 +385,30 @@ def extras(P, ctx) -> dict:
     torch.cuda.synchronize()
     sweep_graph_us = _event_us(torch, lambda i: graph.replay(), 3)
     del graph, sorted_weights
+    # ... and with the independent matrices of a layer in one launch each (llvq_gemv_sorted_multi): {q, k, v}, {o}, {gate, up}, {down} --
+    # 4 launches per layer, no change to the stored matrices -- and, as the bound of what launch merging can give, all 7 in one
+    sorted_sets2 = [[P.llvq_sort_blocks(ctx, d_idx, n, k) for (n, k), (d_idx, _) in zip(shapes, layer)] for layer in sets]
+    groups = [(0, 1, 2), (3,), (4, 5), (6,)]
+
+    def mats(c, idxs):
+        return [(sorted_sets2[c][j], sets[c][j][1], shapes[j][0], shapes[j][1], xs[shapes[j][1]], ys_each[j]) for j in idxs]
+    ys_each = [torch.empty(n, dtype=torch.bfloat16, device="cuda") for n, _ in shapes]
+    grouped = [[mats(c, g) for g in groups] for c in range(4)]
+    all7 = [mats(c, range(7)) for c in range(4)]
+
+    def token_multi(i):
+        for layer in range(32):
+            for m in grouped[(i * 32 + layer) % 4]:
+                P.llvq_gemv_sorted_multi(ctx, m, y_dtype=torch.bfloat16)
+
+    def token_multi7(i):
+        for layer in range(32):
+            P.llvq_gemv_sorted_multi(ctx, all7[(i * 32 + layer) % 4], y_dtype=torch.bfloat16)
+    token_multi(0); token_multi7(0)
+    torch.cuda.synchronize()
+    sweep_multi_us = _event_us(torch, token_multi, 3)
+    sweep_multi7_us = _event_us(torch, token_multi7, 3)
+    del sorted_sets2, grouped, all7
     # ... and with the matrices that share an input stored as one (q|k|v: 6144 x 4096, gate|up: 28672 x 4096): the same
     # blocks in 4 launches per layer instead of 7
     fused_shapes = [(6144, 4096), (4096, 4096), (28672, 4096), (4096, 14336)]
@@ -477,6 +524,12 @@ def extras(P, ctx) -> dict:
                                      "sorted_layout": {"us_per_token": sweep_sorted_us, "tokens_per_s": 1e6 / sweep_sorted_us, "GBps": by / sweep_sorted_us / 1e3},
                                      "sorted_layout_fused_qkv_gateup": {"us_per_token": sweep_fused_us, "tokens_per_s": 1e6 / sweep_fused_us,
                                                                         "launches_per_token": 32 * len(fused_shapes)},
+                                     "sorted_layout_multi_launch": {"us_per_token": sweep_multi_us, "tokens_per_s": 1e6 / sweep_multi_us,
+                                                                    "launches_per_token": 32 * 4, "groups": "{q,k,v} {o} {gate,up} {down}"},
+                                     "sorted_layout_multi_launch_all7": {"us_per_token": sweep_multi7_us, "tokens_per_s": 1e6 / sweep_multi7_us,
+                                                                         "launches_per_token": 32,
+                                                                         "note": "upper bound of launch merging: the 7 matrices of a layer are not independent in a real decoder"},
+                                     "tokens_per_s_at_hbm_roofline": measured_peaks()[0] * 1e9 / by,
                                      "sorted_layout_cuda_graph": {"us_per_token": sweep_graph_us, "tokens_per_s": 1e6 / sweep_graph_us,
                                                                   "note": "one layer set (73 MB sorted + 18 MB gains) replayed: partly L2-resident"}}
     return out
@@ -490,7 +543,8 @@ def main() -> None:
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-extras", action="store_true", help="skip the secondary configurations (dequant, GEMM, decoder sweep)")
-    ap.add_argument("--profile", default=None, choices=["gemv", "dequant", "gemm", "gemv_sorted", "gemm_sorted", "gemm_72bit", "gemm_sorted_72bit"],
+    ap.add_argument("--profile", default=None, choices=["gemv", "dequant", "gemm", "gemv_sorted", "gemm_sorted", "gemm_72bit", "gemm_sorted_72bit",
+                                                       "step_sorted_multi", "step_multi"],
                     help="run only a few launches of one kernel over rotating buffers (for ncu captures); no timing line")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
@@ -501,6 +555,7 @@ def main() -> None:
 
     import torch
     import paper_2603_11021_b200 as P
+    from paper_2603_11021_b200 import ncu_counters
 
     rank = int(os.environ.get("RANK", "0"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
@@ -533,75 +588,83 @@ def main() -> None:
             dev.append(tuple(t.cuda() for t in h) + (torch.empty(n, dtype=torch.bfloat16, device="cuda"),))
         sets.append(dev)
         host_sets.append(host)
+    # the load-time step: every layer rearranged once into the sorted layout (outside every timed region)
+    sorted_sets = [[P.llvq_sort_blocks(ctx, d_idx, n, k) for (n, k), (d_idx, _, _, _) in zip(LAYERS, dev)] for dev in sets]
     torch.cuda.synchronize()
+
+    def mats_of(c: int, srt: bool):
+        return [(sorted_sets[c][li] if srt else sets[c][li][0], sets[c][li][1], n, k, sets[c][li][2], sets[c][li][3]) for li, (n, k) in enumerate(LAYERS)]
+    multi_sorted = [mats_of(c, True) for c in range(copies)]
+    multi_stored = [mats_of(c, False) for c in range(copies)]
 
     launches = 0
 
-    def step(i: int) -> None:
+    def step(i: int) -> None:                      # the headline step: one launch for the three layers, sorted layout
         nonlocal launches
-        for (n, k), (d_idx, d_gain, d_x, d_y) in zip(LAYERS, sets[i % copies]):
-            P.llvq_gemv(ctx, d_idx, d_gain, n, k, d_x, d_y=d_y)
-            launches += 1
+        P.llvq_gemv_sorted_multi(ctx, multi_sorted[i % copies], y_dtype=torch.bfloat16)
+        launches += 1
 
     def barrier():
         if dist is not None:
             dist.barrier()
         torch.cuda.synchronize()
 
-    for i in range(args.warmup):
-        step(i)
-    barrier()
-    launches = 0
-    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    with ClockSampler(local_rank) as clocks:
-        ev0.record()
-        for i in range(args.steps):
-            step(i)
-        ev1.record()
+    def timed(fn, steps: int, warmup: int) -> float:
+        """ms per step of fn over `steps` steps after `warmup` untimed ones: CUDA events on the launching stream, max over ranks."""
+        for i in range(warmup):
+            fn(i)
         barrier()
-    ms_total = max_over_ranks(ev0.elapsed_time(ev1), dist, "cuda")
-    ms_per_step = ms_total / args.steps
-    value = whole_job_value(world, step_bytes, ms_per_step)
-    timed_launches = launches
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for i in range(steps):
+            fn(i)
+        e1.record()
+        barrier()
+        return max_over_ranks(e0.elapsed_time(e1), dist, "cuda") / steps
 
-    # a second sampler covers every other timed pass of this run (per layer, sorted layout, end to end)
+    with ClockSampler(local_rank) as clocks:
+        ms_per_step = timed(step, args.steps, args.warmup)
+        timed_launches = launches
+        # the same step for at least a quarter of a second, so that the clock samples cover a region of the headline kernel
+        # that is long enough to mean something (the region above lasts a few milliseconds at small --steps)
+        sustained_steps = max(args.steps, int(0.25 / (ms_per_step * 1e-3)))
+        sustained_ms = timed(step, sustained_steps, 0)
+    value = whole_job_value(world, step_bytes, ms_per_step)
+
+    # a second sampler covers every other timed pass of this run (per layer, stored streams, end to end)
     clocks_rest = ClockSampler(local_rank)
     clocks_rest.__enter__()
+    reps = max(10, min(args.steps, 100))
 
-    # per-layer device time of the kernel: events around a run of back-to-back launches of that layer, same rotation
+    # the same step as three launches, and on the stored streams (one launch / three launches)
+    def step_sorted_single(i):
+        for (d_w, d_gain, n, k, d_x, d_y) in multi_sorted[i % copies]:
+            P.llvq_gemv_sorted(ctx, d_w, d_gain, n, k, d_x, d_y=d_y, y_dtype=torch.bfloat16)
+
+    def step_stored_single(i):
+        for (d_w, d_gain, n, k, d_x, d_y) in multi_stored[i % copies]:
+            P.llvq_gemv(ctx, d_w, d_gain, n, k, d_x, d_y=d_y, y_dtype=torch.bfloat16)
+    sorted_single_ms = timed(step_sorted_single, reps, 3)
+    stored_multi_ms = timed(lambda i: P.llvq_gemv_multi(ctx, multi_stored[i % copies], y_dtype=torch.bfloat16), reps, 3)
+    stored_single_ms = timed(step_stored_single, reps, 3)
+
+    # per-layer device time of the kernels: events around a run of back-to-back launches of that layer, same rotation
     per_layer = []
     for li, (n, k) in enumerate(LAYERS):
-        fn = lambda i: P.llvq_gemv(ctx, sets[i % copies][li][0], sets[i % copies][li][1], n, k, sets[i % copies][li][2], d_y=sets[i % copies][li][3])
-        _event_us(torch, fn, 5)
-        us = _event_us(torch, fn, max(10, min(args.steps, 100)))
+        f_sorted = lambda i: P.llvq_gemv_sorted(ctx, sorted_sets[i % copies][li], sets[i % copies][li][1], n, k, sets[i % copies][li][2],
+                                                d_y=sets[i % copies][li][3], y_dtype=torch.bfloat16)
+        f_stored = lambda i: P.llvq_gemv(ctx, sets[i % copies][li][0], sets[i % copies][li][1], n, k, sets[i % copies][li][2],
+                                         d_y=sets[i % copies][li][3], y_dtype=torch.bfloat16)
+        _event_us(torch, f_sorted, 5)
+        us = _event_us(torch, f_sorted, reps)
+        _event_us(torch, f_stored, 5)
+        us_stored = _event_us(torch, f_stored, reps)
         by = algorithmic_bytes(n, k)
-        per_layer.append({"n_out": n, "k_in": k, "us": us, "GBps": by / us / 1e3,
-                          "weights_per_s": n * k / (us * 1e-6)})
+        per_layer.append({"n_out": n, "k_in": k, "us": us, "GBps": by / us / 1e3, "weights_per_s": n * k / (us * 1e-6),
+                          "stored_stream_us": us_stored, "stored_stream_GBps": by / us_stored / 1e3})
 
-    # the same step on the sorted layout: every layer rearranged once (load-time step, outside the timed region)
-    sorted_sets = [[P.llvq_sort_blocks(ctx, d_idx, n, k) for (n, k), (d_idx, _, _, _) in zip(LAYERS, dev)] for dev in sets]
-
-    def sorted_step(i: int) -> None:
-        for (n, k), (_, d_gain, d_x, d_y), d_srt in zip(LAYERS, sets[i % copies], sorted_sets[i % copies]):
-            P.llvq_gemv_sorted(ctx, d_srt, d_gain, n, k, d_x, d_y=d_y)
-
-    for i in range(args.warmup):
-        sorted_step(i)
-    barrier()
-    ev0.record()
-    for i in range(args.steps):
-        sorted_step(i)
-    ev1.record()
-    barrier()
-    sorted_ms = max_over_ranks(ev0.elapsed_time(ev1), dist, "cuda") / args.steps
-    sorted_layers = []
-    for li, (n, k) in enumerate(LAYERS):
-        fn = lambda i: P.llvq_gemv_sorted(ctx, sorted_sets[i % copies][li], sets[i % copies][li][1], n, k, sets[i % copies][li][2], d_y=sets[i % copies][li][3])
-        us = _event_us(torch, fn, max(10, min(args.steps, 100)))
-        sorted_layers.append({"n_out": n, "k_in": k, "us_back_to_back": us, "GBps": algorithmic_bytes(n, k) / us / 1e3})
-    del sorted_sets
-
-    # end to end: inputs start in pinned host memory, the result is read back to the host, every step
+    # end to end: the stored streams, gains and activations start in pinned host memory, the result is read back to the host,
+    # every step (the stored form is what a caller holds on the host: the sorted layout is made on the device at load time)
     h2d = sum(layer_bytes(n, k)["idx"] + layer_bytes(n, k)["gain"] + layer_bytes(n, k)["x"] for n, k in LAYERS)
     d2h = sum(layer_bytes(n, k)["y"] for n, k in LAYERS)
     y_host = [torch.empty(n, dtype=torch.bfloat16).pin_memory() for n, _ in LAYERS]
@@ -610,30 +673,30 @@ def main() -> None:
     # copies run on their own stream, one step ahead of the kernels (the device buffers rotate, so the copy of
     # step i + 1 never touches what step i reads); every step ends with the host holding that step's result
     main_stream, copy_stream = torch.cuda.current_stream(), torch.cuda.Stream()
-    copied = [[torch.cuda.Event() for _ in LAYERS] for _ in range(copies)]
-    consumed = [[torch.cuda.Event() for _ in LAYERS] for _ in range(copies)]
-    for c in range(copies):
-        for e in consumed[c]:
-            e.record(main_stream)
+    copied = [torch.cuda.Event() for _ in range(copies)]
+    consumed = [torch.cuda.Event() for _ in range(copies)]
+    for e in consumed:
+        e.record(main_stream)
 
     def e2e_copies(i: int) -> None:
+        c = i % copies
         with torch.cuda.stream(copy_stream):
+            copy_stream.wait_event(consumed[c])
             for li in range(len(LAYERS)):
-                h_idx, h_gain, h_x = host_sets[i % copies][li]
-                d_idx, d_gain, d_x, _ = sets[i % copies][li]
-                copy_stream.wait_event(consumed[i % copies][li])
+                h_idx, h_gain, h_x = host_sets[c][li]
+                d_idx, d_gain, d_x, _ = sets[c][li]
                 d_idx.copy_(h_idx, non_blocking=True)
                 d_gain.copy_(h_gain, non_blocking=True)
                 d_x.copy_(h_x, non_blocking=True)
-                copied[i % copies][li].record(copy_stream)
+            copied[c].record(copy_stream)
 
     def e2e_compute(i: int) -> None:
-        for li, (n, k) in enumerate(LAYERS):
-            d_idx, d_gain, d_x, d_y = sets[i % copies][li]
-            main_stream.wait_event(copied[i % copies][li])
-            P.llvq_gemv(ctx, d_idx, d_gain, n, k, d_x, d_y=d_y)
-            consumed[i % copies][li].record(main_stream)
-            y_host[li].copy_(d_y, non_blocking=True)
+        c = i % copies
+        main_stream.wait_event(copied[c])
+        P.llvq_gemv_multi(ctx, multi_stored[c], y_dtype=torch.bfloat16)
+        consumed[c].record(main_stream)
+        for li in range(len(LAYERS)):
+            y_host[li].copy_(sets[c][li][3], non_blocking=True)
 
     def e2e_run(first: int, count: int) -> None:
         e2e_copies(first)
@@ -645,6 +708,7 @@ def main() -> None:
 
     e2e_run(0, 3)
     barrier()
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     ev0.record()
     e2e_run(3, e2e_steps)
     ev1.record()
@@ -659,40 +723,54 @@ def main() -> None:
 
     if rank == 0:
         peak, which = measured_peaks()
-        dom = per_layer[1]                                   # the 11008x4096 launch: largest share of the step
-        dom_bytes = algorithmic_bytes(*LAYERS[1])
-        achieved = dom_bytes / dom["us"] / 1e3
+        blocks_per_step = sum(layer_bytes(n, k)["nblocks"] for n, k in LAYERS)
+        achieved = step_bytes / ms_per_step / 1e6                # one launch = one step
+        counters = ncu_counters.load(COUNTER_FILE)               # None when the kernel sources changed after the capture
+        roofline = {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
+                    "traffic": counters["dram_traffic_bytes"] if counters else None,
+                    "kernel": "gemv_sorted_multi_kernel on the three layers of a step (one launch)",
+                    "algorithmic_bytes_per_launch": step_bytes, "peak_source": f"of {which}", "frac_of_nominal_8TBps": achieved / 8000.0,
+                    "note": "the sorted layout stores 10 bytes per block (48-bit index, 16-bit position, fp16 gain) against the 8 algorithmic ones; "
+                            "what binds the kernel is the integer pipe, see roofline_issue"}
+        roofline_issue = None
+        if counters:
+            roofline["ncu"] = {"source_hash": counters["source_hash"], "git_commit": counters.get("git_commit"),
+                               "thread_instructions_per_block": counters["thread_instructions_per_block"],
+                               "issue_slots_used": counters.get("issue_active_pct", 0.0) / 100.0, "alu_pipe_busy": counters.get("pipe_alu_pct", 0.0) / 100.0,
+                               "instructions_per_block_at_hbm_roofline": 46}
+            wi = counters["warp_instructions"] * blocks_per_step / counters["blocks_per_launch"]
+            roofline_issue = {"bound": "alu", "achieved": wi / (ms_per_step * 1e-3), "peak": ISSUE_PEAK_WARP_INST_PER_S, "unit": "warp-instructions/s",
+                              "frac": wi / (ms_per_step * 1e-3) / ISSUE_PEAK_WARP_INST_PER_S, "kernel": roofline["kernel"],
+                              "peak_source": "148 SMs x 4 schedulers x 1.965 GHz; instructions per launch from the committed ncu capture, duration measured live"}
+        else:
+            roofline["ncu"] = None
+            roofline["ncu_note"] = "no counters quoted: the kernel sources differ from those of the committed capture (or it is missing)"
         out = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
             "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
             "dtype": "bf16 weights x bf16 activations, f32 accumulate", "data": "synthetic",
             "config": {"workload": WORKLOAD, "l2": f"rotation over {copies} distinct copies of the layers ({copies * step_bytes / 1e6:.0f} MB > 2 x L2)",
-                       "bytes_per_step": step_bytes, "blocks_per_step": sum(layer_bytes(n, k)["nblocks"] for n, k in LAYERS)},
+                       "bytes_per_step": step_bytes, "blocks_per_step": blocks_per_step,
+                       "layout": "load-time sorted layout (llvq_sort_blocks), one llvq_gemv_sorted_multi launch per step; end to end: stored streams from the "
+                                 "host, one llvq_gemv_multi launch per step"},
             "weights_per_s": world * sum(n * k for n, k in LAYERS) / (ms_per_step * 1e-3),
             "frac_of_hbm_peak": value / world / peak,
+            "sustained": {"steps": sustained_steps, "ms_per_step": sustained_ms, "value": whole_job_value(world, step_bytes, sustained_ms),
+                          "ms_x_sm_mhz": sustained_ms * (clocks.summary()["sm_mhz"] or 0)},
             "layers": per_layer,
-            "sorted_layout": {"note": "same step through llvq_gemv_sorted on streams rearranged once by llvq_sort_blocks (64-bit entries: 48-bit index + "
-                                      "16-bit position; all decode steps still run in the kernel); GB/s counted on the same algorithmic bytes",
-                              "ms_per_step": sorted_ms, "value": whole_job_value(world, step_bytes, sorted_ms), "unit": UNIT,
-                              "speedup_over_stored_stream": ms_per_step / sorted_ms, "layers": sorted_layers},
-            "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
-                         "traffic": NCU_TRAFFIC_BYTES_11008x4096, "kernel": "gemv_bin_kernel on 11008x4096",
-                         "algorithmic_bytes_per_launch": dom_bytes, "peak_source": f"of {which}", "frac_of_nominal_8TBps": achieved / 8000.0,
-                         # what binds the kernel instead of HBM: counters of the ncu capture summarised under profiles/
-                         "ncu": {"warp_instructions_per_block": 945, "issue_slots_used": 0.653, "alu_pipe_busy": 0.599,
-                                 "shared_memory_wavefronts_per_block": 208, "instructions_per_block_at_hbm_roofline": 46}},
-            # the same launch against what actually binds it: instruction issue (instructions per launch from the ncu
-            # capture, duration measured live)
-            "roofline_issue": {"bound": "alu", "achieved": NCU_WARP_INSTRUCTIONS_11008x4096 / (dom["us"] * 1e-6), "peak": ISSUE_PEAK_WARP_INST_PER_S,
-                               "unit": "warp-instructions/s", "frac": NCU_WARP_INSTRUCTIONS_11008x4096 / (dom["us"] * 1e-6) / ISSUE_PEAK_WARP_INST_PER_S,
-                               "kernel": "gemv_bin_kernel on 11008x4096", "peak_source": "148 SMs x 4 schedulers x 1.965 GHz"},
+            "same_step_other_paths": {"sorted_layout_three_launches_ms": sorted_single_ms, "stored_stream_one_launch_ms": stored_multi_ms,
+                                      "stored_stream_three_launches_ms": stored_single_ms,
+                                      "stored_stream_value": whole_job_value(world, step_bytes, stored_multi_ms), "unit": UNIT},
+            "roofline": roofline,
             "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "ms_per_step": e2e_ms},
             "gpu_launches": timed_launches,
             "clocks": clocks.summary(),
             "clocks_other_timed_passes": clocks_rest.summary(),
         }
+        if roofline_issue:
+            out["roofline_issue"] = roofline_issue
         if world == 1 and not args.no_extras:
-            del sets, host_sets
+            del sets, host_sets, sorted_sets, multi_sorted, multi_stored
             torch.cuda.empty_cache()
             out["extras"] = extras(P, ctx)
         if world == 1 and not args.no_cpu_baseline:
