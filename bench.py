@@ -200,6 +200,86 @@ def cpu_baseline() -> dict:
             "sample": f"{reps} x the 4096x4096 layer ({nblocks} blocks each), fp64 GEMV", "blocks_per_s": nblocks * reps / dt}
 
 
+ROWSHARD_SHAPES = [(11008, 4096), (6144, 4096), (4096, 4096), (28672, 4096), (4096, 14336)]   # the dominant layer, then q|k|v, o, gate|up, down
+
+
+def rowshard_plan(n_out: int, k_in: int, world: int, rank: int) -> dict:
+    """What one rank holds of a matrix whose rows are spread over `world` ranks: its band and the bytes it reads per step."""
+    from paper_2603_11021_b200.rowshard import row_bands
+    row0, rows = row_bands(n_out, world, 8)[rank]
+    bpr = (k_in + 23) // 24
+    return {"row0": row0, "rows": rows, "blocks": rows * bpr, "band_bytes": rows * bpr * (CODE_W // 8 + 2) + 2 * k_in + 2 * rows}
+
+
+def ranks_agree(y, dist) -> bool:
+    """True on every rank iff all ranks hold bit-identical copies of y (rank 0's copy is the one compared against)."""
+    import torch
+    ref = y.clone()
+    dist.broadcast(ref, src=0)
+    ok = torch.tensor([1 if torch.equal(ref.view(torch.int16) if ref.dtype == torch.bfloat16 else ref, y.view(torch.int16) if y.dtype == torch.bfloat16 else y) else 0],
+                      dtype=torch.int32, device=y.device)
+    dist.all_reduce(ok, op=dist.ReduceOp.MIN)
+    return bool(ok.item())
+
+
+def rowshard_leg(P, ctx, dist, rank: int, world: int, shapes=None, reps: int = 50) -> dict:
+    """Strong scaling of one matrix over the ranks: every rank owns a band of rows (sorted layout), its fused GEMV writes the
+    band into every rank's copy of y over NVLink and raises a flag per peer, a bounded device-side wait completes the step.
+    Per shape: device time of a step (launch + wait, max over ranks), of the band's GEMV alone, and whether all ranks ended
+    up with the same y, which is also compared with the unsharded product.  The band's weights rotate over copies that
+    exceed L2 together (the same rows in a different order)."""
+    import torch
+    from paper_2603_11021_b200.rowshard import RowShardedGemv, band_of_stream
+    out = {"world": world, "shapes": {}}
+    dev = lambda a, view=None: torch.from_numpy(a if view is None else a.view(view)).cuda()
+    for (n, k) in (shapes or ROWSHARD_SHAPES):
+        plan = rowshard_plan(n, k, world, rank)
+        stream, gain, x, _ = host_layer(n, k, seed=900 + (n + k) % 97)              # the same matrix on every rank
+        s, g = band_of_stream(stream, gain, k, CODE_W, plan["row0"], plan["rows"])
+        d_x = dev(x, np.int16).view(torch.bfloat16)
+        op = RowShardedGemv(ctx, n, k, dev(s), dev(g, np.float16), torch.bfloat16, sorted_layout=True)
+        y = op(d_x).clone()
+        torch.cuda.synchronize()
+        agree = ranks_agree(y, dist)
+        full = P.llvq_gemv_sorted(ctx, P.llvq_sort_blocks(ctx, dev(stream), n, k), dev(gain, np.float16), n, k, d_x, y_dtype=torch.bfloat16)
+        a, b = y.float(), full.float()
+        err = float(((a - b).abs() / b.abs().clamp_min(1e-3 * float(b.abs().max()))).max())        # another split of the sums: one bf16 step at most
+        # rotating copies of the band: the same rows rolled by whole row groups
+        rows, bpr = plan["rows"], (k + 23) // 24
+        copies = 1 if rows == 0 else max(2, min(64, -(-2 * L2_BYTES // max(plan["band_bytes"], 1))))
+        bands = [(op.d_stream, op.d_gain)]
+        if rows:
+            raw = dev(s)[: rows * bpr * 6].view(rows, bpr * 6)
+            gr = dev(g, np.float16).view(rows, bpr)
+            for c in range(1, copies):
+                sh = 8 * (c * (rows // 8) // copies)
+                d_i = torch.zeros(ctx.index_bytes(rows * bpr), dtype=torch.uint8, device="cuda")
+                d_i[: rows * bpr * 6] = torch.roll(raw, sh, 0).reshape(-1)
+                bands.append((P.llvq_sort_blocks(ctx, d_i, rows, k), torch.roll(gr, sh, 0).reshape(-1).contiguous()))
+
+        def step(i):
+            op.d_stream, op.d_gain = bands[i % len(bands)]
+            op(d_x)
+
+        def band_only(i):
+            if rows:
+                P.llvq_gemv_sorted(ctx, bands[i % len(bands)][0], bands[i % len(bands)][1], rows, k, d_x, d_y=y[:rows], y_dtype=torch.bfloat16)
+        for fn in (step, band_only):
+            _event_us(torch, fn, 5)
+        dist.barrier()
+        torch.cuda.synchronize()
+        us_step = max_over_ranks(_event_us(torch, step, reps), dist, "cuda")
+        us_band = max_over_ranks(_event_us(torch, band_only, reps), dist, "cuda")
+        out["shapes"][f"{n}x{k}"] = {"us_per_step": us_step, "us_band_gemv": us_band, "us_wait": max(us_step - us_band, 0.0),
+                                     "rows_per_rank": rows, "rotating_copies": len(bands), "all_ranks_same_y": agree,
+                                     "max_rel_diff_to_unsharded": err}
+        op.close()
+        if not agree or err > 2.0 ** -7:
+            raise SystemExit(f"row-sharded GEMV {n}x{k}: ranks agree = {agree}, difference to the unsharded product {err}")
+    out["errors"] = P.llvq_last_error(ctx)
+    return out
+
+
 def profile_run(P, ctx, args) -> None:
     """A handful of launches of one kernel on buffers that do not fit L2 together, for profiler captures:
     gemv* = the 11008x4096 layer, step_* = the three-layer step in one launch, dequant = 4096x4096 FLAT, gemm* = 8192x8192 at batch 16."""
@@ -543,6 +623,8 @@ def main() -> None:
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-extras", action="store_true", help="skip the secondary configurations (dequant, GEMM, decoder sweep)")
+    ap.add_argument("--rowshard-leg", action="store_true",
+                    help="also run the strong-scaling leg (one matrix spread over the ranks) when there is a single rank; with several ranks it always runs")
     ap.add_argument("--profile", default=None, choices=["gemv", "dequant", "gemm", "gemv_sorted", "gemm_sorted", "gemm_72bit", "gemm_sorted_72bit",
                                                        "step_sorted_multi", "step_multi"],
                     help="run only a few launches of one kernel over rotating buffers (for ncu captures); no timing line")
@@ -721,6 +803,19 @@ def main() -> None:
     if bad or flags:
         raise SystemExit(f"device error state: {bad} invalid fields, flags {flags}")
 
+    # strong scaling: one matrix spread over the ranks (the headline above is weak scaling: every rank its own layers)
+    rowshard = None
+    if world > 1 or args.rowshard_leg:
+        if dist is None:                                   # a single rank still needs a process group for the handle exchange
+            import torch.distributed as dist1
+            os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+            os.environ.setdefault("MASTER_PORT", "29577")
+            dist1.init_process_group("gloo", rank=0, world_size=1)
+            rowshard = rowshard_leg(P, ctx, dist1, 0, 1)
+            dist1.destroy_process_group()
+        else:
+            rowshard = rowshard_leg(P, ctx, dist, rank, world)
+
     if rank == 0:
         peak, which = measured_peaks()
         blocks_per_step = sum(layer_bytes(n, k)["nblocks"] for n, k in LAYERS)
@@ -769,6 +864,8 @@ def main() -> None:
         }
         if roofline_issue:
             out["roofline_issue"] = roofline_issue
+        if rowshard:
+            out["rowshard"] = rowshard
         if world == 1 and not args.no_extras:
             del sets, host_sets, sorted_sets, multi_sorted, multi_stored
             torch.cuda.empty_cache()

@@ -39,6 +39,43 @@ def test_max_over_ranks_and_weak_scaling_value():
     assert res[0][2] != res[1][2]                                      # ranks draw different layers
 
 
+def _agree_worker(rank, world, port, out):
+    import torch
+    import torch.distributed as dist
+    sys.path.insert(0, ROOT)
+    import bench
+    os.environ.update(MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port), RANK=str(rank), WORLD_SIZE=str(world))
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    same = torch.arange(64, dtype=torch.float32).to(torch.bfloat16)
+    differs = same.clone()
+    if rank == 1:
+        differs[17] = -1.0                                             # one rank ends up with another value in one row
+    plans = [bench.rowshard_plan(11008, 4096, world, r) for r in range(world)]
+    out[rank] = (bench.ranks_agree(same, dist), bench.ranks_agree(differs, dist), plans)
+    dist.destroy_process_group()
+
+
+def test_strong_scaling_leg_host_logic():
+    # the band plan of the row-sharded leg covers the matrix, and the agreement check fails on every rank as soon as one
+    # rank's copy of y differs
+    ctx = mp.get_context("spawn")
+    with ctx.Manager() as m:
+        out = m.dict()
+        procs = [ctx.Process(target=_agree_worker, args=(r, 2, 29537, out)) for r in range(2)]
+        for p in procs:
+            p.start()
+        for p in procs:
+            p.join(120)
+            assert p.exitcode == 0
+        res = dict(out)
+    for r in range(2):
+        agree_same, agree_differs, plans = res[r]
+        assert agree_same is True and agree_differs is False
+        assert [p["row0"] for p in plans] == [0, 5504] and sum(p["rows"] for p in plans) == 11008
+        assert all(p["rows"] % 8 == 0 for p in plans)
+        assert plans[0]["band_bytes"] == 5504 * 171 * 8 + 2 * 4096 + 2 * 5504
+
+
 def test_single_process_path_has_no_collective():
     sys.path.insert(0, ROOT)
     import bench

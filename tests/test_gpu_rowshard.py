@@ -224,3 +224,21 @@ def test_two_processes_exchange_through_ipc_buffers():
             p.join(300)
             assert p.exitcode == 0
         assert dict(out) == {0: True, 1: True}
+
+
+def test_bench_strong_scaling_leg_runs_on_one_rank():
+    # the benchmark's strong-scaling leg (one matrix spread over the ranks, rotating band copies, agreement of all ranks' y,
+    # comparison with the unsharded product), driven with a single rank: every code path but the peer stores
+    import json
+    import subprocess
+    env = dict(os.environ, MASTER_PORT="29591")
+    r = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--steps", "3", "--warmup", "3", "--no-extras", "--no-cpu-baseline",
+                        "--rowshard-leg"], capture_output=True, text=True, env=env, timeout=900)
+    assert r.returncode == 0, r.stderr[-2000:]
+    line = json.loads(r.stdout.strip().splitlines()[-1])
+    leg = line["rowshard"]
+    assert leg["world"] == 1 and leg["errors"] == [0, 0]
+    assert set(leg["shapes"]) == {"11008x4096", "6144x4096", "4096x4096", "28672x4096", "4096x14336"}
+    for shape in leg["shapes"].values():
+        assert shape["all_ranks_same_y"] and shape["max_rel_diff_to_unsharded"] <= 2.0 ** -7
+        assert shape["us_per_step"] >= shape["us_band_gemv"] > 0
