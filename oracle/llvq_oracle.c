@@ -832,18 +832,21 @@ int64_t oc_gemm_rows_sg(const oc_code* code, const uint8_t* stream, int gain_bit
 /* codeword position in T; inside a coset the first coordinate with the        */
 /* largest error.  Inputs are in integer-coordinate units (|x|^2 = 16 m).      */
 /*                                                                           */
-/* Restriction to the shells m_lo..m_hi of the code (m_lo must be 2, m_hi >= 6):*/
-/* EUCLIDEAN (metric 0): the input is projected into the ball of radius        */
-/*   sqrt(16 m_hi) (App. E "Spherical shaping"); while the nearest lattice      */
-/*   point of the working vector lies beyond the last shell the working vector  */
-/*   is shrunk by 2 %; if the nearest point is the origin the input is scaled   */
-/*   to the radius of the first shell and decoded once more.                   */
+/* Restriction to the shells m_lo..m_hi of the code (m_lo must be 2, m_hi >= 3).  */
+/* Inputs are binary32 values widened exactly; every operation below is one     */
+/* binary64 operation (no contraction), sums run over the coordinates in order. */
+/* EUCLIDEAN (metric 0): if the nearest lattice point of the input lies in the   */
+/*   code it is the answer (it is then the nearest point of the cut as well).   */
+/*   Otherwise -- the input lies outside the ball of App. E "Spherical shaping", */
+/*   or so close to the origin that the origin is nearest -- the input direction */
+/*   is decoded at every shell radius sqrt(16 m), and of the candidates that lie  */
+/*   in the code the one nearest to the input wins (first radius on ties).       */
 /* ANGULAR (metric 1): for every shell radius sqrt(16 m) the input direction    */
 /*   scaled to that radius is decoded; of the candidates that lie in the code   */
 /*   the one with the largest cosine wins (first radius on ties).              */
-/* A zero input encodes to index 0.  This is a practical search, exact for the */
-/* unbounded lattice and near-optimal on the cut; what is pinned is the exact  */
-/* part (brute force over small shells) and the distortion it reaches.        */
+/* A zero input encodes to index 0.  The search is exact for the unbounded      */
+/* lattice, hence on the cut whenever the unconstrained answer lies in it; for  */
+/* the other inputs it is a candidate search, pinned by what it reaches.        */
 /* ------------------------------------------------------------------------- */
 static double nearest_in_lattice(const double v[OC_DIM], int best_x[OC_DIM])
 {
@@ -887,29 +890,34 @@ static int encode_point(const oc_code* code, const double v[OC_DIM], int metric,
     double n2 = 0;
     for (int i = 0; i < OC_DIM; ++i) n2 += v[i] * v[i];
     int ok = 0;
-    if (code->m_lo != 2 || code->m_hi < 6) { unrank_point(code, 0, out); return 1; }
+    if (code->m_lo != 2 || code->m_hi < 3) { unrank_point(code, 0, out); return 1; }
     if (n2 == 0) { unrank_point(code, 0, out); return 0; }
+    int direct = 0;
     if (metric == 0) {
-        double R2 = 16.0 * code->m_hi, u[OC_DIM], f = n2 > R2 ? sqrt(R2 / n2) : 1.0;
-        for (int i = 0; i < OC_DIM; ++i) u[i] = v[i] * f;
-        for (int it = 0; it < 64 && !ok; ++it) {
-            nearest_in_lattice(u, x);
-            int m = shell_of(x);
-            if (m > code->m_hi) { for (int i = 0; i < OC_DIM; ++i) u[i] *= 0.98; }
-            else if (m < 2) { double g = sqrt(32.0 / n2); for (int i = 0; i < OC_DIM; ++i) u[i] = v[i] * g; }
-            else { ok = 1; memcpy(bestx, x, sizeof x); }
-        }
-    } else {
+        nearest_in_lattice(v, x);
+        int m = shell_of(x);
+        if (m >= code->m_lo && m <= code->m_hi) { ok = direct = 1; memcpy(bestx, x, sizeof x); }
+    }
+    if (!direct) {
+        /* the input direction at every shell radius; metric 0 keeps the candidate nearest to the input, metric 1 the one
+           with the largest cosine */
         double best = -INFINITY, rn = 1.0 / sqrt(n2);
         for (int m = code->m_lo; m <= code->m_hi; ++m) {
             double u[OC_DIM], rad = sqrt(16.0 * m);
-            for (int i = 0; i < OC_DIM; ++i) u[i] = v[i] * rn * rad;
+            for (int i = 0; i < OC_DIM; ++i) u[i] = (v[i] * rn) * rad;
             nearest_in_lattice(u, x);
             int mx = shell_of(x);
             if (mx < code->m_lo || mx > code->m_hi) continue;
-            double dot = 0, xx = 0;
-            for (int i = 0; i < OC_DIM; ++i) { dot += v[i] * rn * x[i]; xx += (double)x[i] * x[i]; }
-            double score = dot / sqrt(xx);
+            double score;
+            if (metric == 0) {
+                double d2 = 0;
+                for (int i = 0; i < OC_DIM; ++i) { double d = v[i] - x[i]; d2 += d * d; }
+                score = -d2;
+            } else {
+                double dot = 0, xx = 0;
+                for (int i = 0; i < OC_DIM; ++i) { dot += (v[i] * rn) * x[i]; xx += (double)x[i] * x[i]; }
+                score = dot / sqrt(xx);
+            }
             if (score > best) { best = score; ok = 1; memcpy(bestx, x, sizeof x); }
         }
     }
