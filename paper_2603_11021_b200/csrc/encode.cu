@@ -20,6 +20,8 @@ constexpr uint32_t kFull = 0xffffffffu;
 constexpr int kEncWarps = 8;               // vectors in flight per CTA, one warp each
 constexpr uint32_t kFlagSearchGaveUp = 4u; // LLVQ_FLAG_SEARCH_GAVE_UP
 
+constexpr int kMaxCand = 64;               // cosets re-scored in binary64 per search; more (massive ties) means all 8192 are
+
 // Per-warp scratch of the lattice search.
 struct WarpTables {
     float2 grp[2][4][64];   // [parity][group of 6 coordinates][bit pattern]: {sum of squared errors, smallest cost of
@@ -27,28 +29,48 @@ struct WarpTables {
     float e[24][4];         // squared rounding error of coordinate i for offset b = parity + 2 * codeword bit
     float d[24][4];         // cost of moving it to the other neighbour: 1 - 2 |error|
     uint8_t zp[24][4];      // z & 1
+    uint32_t cand[kMaxCand];
+    uint32_t ncand;
 };
 
-__device__ __forceinline__ float warp_sum(float v)
+// sum of the values of lanes 0..23, added in lane order, one binary64 rounding per addition (every lane gets the sum)
+__device__ __forceinline__ double seq_sum24(double v)
 {
+    double acc = 0.0;
 #pragma unroll
-    for (int o = 16; o; o >>= 1) v += __shfl_xor_sync(kFull, v, o);
-    return v;
+    for (int i = 0; i < 24; ++i) acc = __dadd_rn(acc, __shfl_sync(kFull, v, i));
+    return acc;
+}
+
+// Cost of coset (pi, codeword j) from the group tables, in units of 16 (binary32).
+__device__ __forceinline__ float coset_cost(const WarpTables& W, uint32_t c, uint32_t pi)
+{
+    const float2 a0 = W.grp[pi][0][c & 63u], a1 = W.grp[pi][1][(c >> 6) & 63u], a2 = W.grp[pi][2][(c >> 12) & 63u], a3 = W.grp[pi][3][c >> 18];
+    float cost = (a0.x + a1.x) + (a2.x + a3.x);
+    const uint32_t par = (__float_as_uint(a0.y) ^ __float_as_uint(a1.y) ^ __float_as_uint(a2.y) ^ __float_as_uint(a3.y)) >> 31;
+    if (par != pi) cost += fminf(fminf(fabsf(a0.y), fabsf(a1.y)), fminf(fabsf(a2.y), fabsf(a3.y)));
+    return cost;
 }
 
 // Nearest point of the unbounded lattice to u (one coordinate per lane, lanes 0..23; all in units of the integer
 // coordinates).  Every lattice point is b + 4 z with b_i = parity + 2 c_i, c a Golay codeword, and sum z = parity
 // (mod 2) (the sum rules of Sec. 2.4: all Golay weights are multiples of 4).  For each of the 2 x 4096 cosets the
 // best z is the rounded one, with the coordinate of largest rounding error moved to its other neighbour when the
-// sum rule fails.  Costs are in units of 16 (squared distance / 16).  Ties: lowest parity, then lowest codeword
-// position; inside a coset the first coordinate with the largest error.  Returns the coordinate of this lane
-// (0 for lanes >= 24) and the squared norm of the point.
-__device__ int lattice_nearest(WarpTables& W, const uint32_t* __restrict__ golay_s, float u, int lane, int& norm2)
+// sum rule fails.
+// Two stages.  A binary32 scan of all cosets through tables per group of 6 coordinates (4 reads and about 20
+// instructions per coset) finds the smallest cost; every coset whose binary32 cost is within 2^-12 (+ 2^-13 of the
+// cost) of it -- far more than the binary32 scan can err, costs are at most 1 -- is then evaluated again in binary64,
+// coordinate by coordinate in lane order, one rounding per operation: its point, and the squared distance as the sum
+// over the coordinates in order.  The smallest distance wins, the lowest (parity, codeword position) among equal ones;
+// inside a coset the first coordinate with the largest error moves.  The result does not depend on the first stage's
+// rounding.  Returns the coordinate of this lane (0 for lanes >= 24) and the squared norm of the point.
+__device__ int lattice_nearest(WarpTables& W, const uint32_t* __restrict__ golay_s, double u, int lane, int& norm2)
 {
+    const float uf = (float)u;
     if (lane < 24) {
 #pragma unroll
         for (int b = 0; b < 4; ++b) {
-            const float t = (u - (float)b) * 0.25f;
+            const float t = (uf - (float)b) * 0.25f;
             const float z = rintf(t);
             const float err = t - z;
             W.e[lane][b] = err * err;
@@ -56,6 +78,7 @@ __device__ int lattice_nearest(WarpTables& W, const uint32_t* __restrict__ golay
             W.zp[lane][b] = (uint8_t)((int)z & 1);
         }
     }
+    if (lane == 0) W.ncand = 0u;
     __syncwarp();
     for (int q = 0; q < 16; ++q) {
         const int id = q * 32 + lane, pi = id >> 8, g = (id >> 6) & 3, pat = id & 63;
@@ -72,54 +95,68 @@ __device__ int lattice_nearest(WarpTables& W, const uint32_t* __restrict__ golay
     }
     __syncwarp();
     float best = 3.0e38f;
-    uint32_t best_id = 0xffffffffu;
+    for (int s = 0; s < 128; ++s) {
+        const uint32_t c = golay_s[s * 32 + lane];
+        best = fminf(best, fminf(coset_cost(W, c, 0u), coset_cost(W, c, 1u)));
+    }
+#pragma unroll
+    for (int o = 16; o; o >>= 1) best = fminf(best, __shfl_xor_sync(kFull, best, o));
+    const float thr = best + (1.f / 4096.f + best * (1.f / 8192.f));
     for (int s = 0; s < 128; ++s) {
         const uint32_t j = (uint32_t)(s * 32 + lane), c = golay_s[j];
-        const uint32_t p0 = c & 63u, p1 = (c >> 6) & 63u, p2 = (c >> 12) & 63u, p3 = c >> 18;
 #pragma unroll
         for (uint32_t pi = 0; pi < 2; ++pi) {
-            const float2 a0 = W.grp[pi][0][p0], a1 = W.grp[pi][1][p1], a2 = W.grp[pi][2][p2], a3 = W.grp[pi][3][p3];
-            float cost = (a0.x + a1.x) + (a2.x + a3.x);
-            const uint32_t par = (__float_as_uint(a0.y) ^ __float_as_uint(a1.y) ^ __float_as_uint(a2.y) ^ __float_as_uint(a3.y)) >> 31;
-            if (par != pi) cost += fminf(fminf(fabsf(a0.y), fabsf(a1.y)), fminf(fabsf(a2.y), fabsf(a3.y)));
-            const uint32_t id = pi << 12 | j;
-            if (cost < best || (cost == best && id < best_id)) { best = cost; best_id = id; }
+            if (coset_cost(W, c, pi) <= thr) {
+                const uint32_t slot = atomicAdd(&W.ncand, 1u);
+                if (slot < (uint32_t)kMaxCand) W.cand[slot] = pi << 12 | j;
+            }
         }
     }
-#pragma unroll
-    for (int o = 16; o; o >>= 1) {
-        const float oc = __shfl_xor_sync(kFull, best, o);
-        const uint32_t oid = __shfl_xor_sync(kFull, best_id, o);
-        if (oc < best || (oc == best && oid < best_id)) { best = oc; best_id = oid; }
-    }
-    // rebuild the point of the winning coset
-    const int pi = (int)(best_id >> 12);
-    const uint32_t c = golay_s[best_id & 4095u];
-    const int b = pi + 2 * (int)((c >> (lane & 31)) & 1u);
-    const float t = (u - (float)b) * 0.25f;
-    const float z = rintf(t);
-    const float err = t - z;
-    int zi = (int)z;
-    const bool mine = lane < 24;
-    const int parity = __popc(__ballot_sync(kFull, mine && (zi & 1))) & 1;
-    if (parity != pi) {
-        const uint32_t mag = mine ? __float_as_uint(fabsf(err)) : 0u;
-        const uint32_t top = __reduce_max_sync(kFull, mag);
-        const uint32_t who = __ballot_sync(kFull, mine && mag == top);
-        if (lane == __ffs(who) - 1) zi += err < 0.f ? -1 : 1;
-    }
-    const int x = mine ? b + 4 * zi : 0;
-    norm2 = __reduce_add_sync(kFull, x * x);
     __syncwarp();
-    return x;
+    const uint32_t listed = W.ncand;
+    const uint32_t n = listed > (uint32_t)kMaxCand ? 8192u : listed;          // too many near-ties to list: every coset
+    const bool mine = lane < 24;
+    double best_d2 = 1.0e300;
+    uint32_t best_id = 0xffffffffu;
+    int best_x = 0;
+    for (uint32_t t = 0; t < n; ++t) {
+        const uint32_t id = listed > (uint32_t)kMaxCand ? t : W.cand[t];
+        const int pi = (int)(id >> 12);
+        const uint32_t c = golay_s[id & 4095u];
+        const int b = pi + 2 * (int)((c >> (lane & 31)) & 1u);
+        const double tt = __dmul_rn(__dsub_rn(u, (double)b), 0.25);
+        const double z = rint(tt);
+        const double err = __dsub_rn(tt, z);
+        int x = mine ? b + 4 * (int)z : 0;
+        const int sum = __reduce_add_sync(kFull, x);
+        if ((((sum % 8) + 8) % 8) != (pi ? 4 : 0)) {
+            // the first coordinate with the largest |error| moves by 4 (binary64 magnitudes compare like their bit patterns)
+            unsigned long long key = mine ? (unsigned long long)__double_as_longlong(fabs(err)) : 0ull;
+            int who = lane;
+#pragma unroll
+            for (int o = 16; o; o >>= 1) {
+                const unsigned long long ok = __shfl_xor_sync(kFull, key, o);
+                const int ow = __shfl_xor_sync(kFull, who, o);
+                if (ok > key || (ok == key && ow < who)) { key = ok; who = ow; }
+            }
+            if (lane == who) x += err > 0.0 ? 4 : (err < 0.0 ? -4 : 4);
+        }
+        const double dd = __dsub_rn(u, (double)x);
+        const double d2 = seq_sum24(mine ? __dmul_rn(dd, dd) : 0.0);
+        if (d2 < best_d2 || (d2 == best_d2 && id < best_id)) { best_d2 = d2; best_id = id; best_x = x; }
+    }
+    norm2 = __reduce_add_sync(kFull, best_x * best_x);
+    __syncwarp();
+    return best_x;
 }
 
-// One warp per input vector.  EUCLIDEAN: the input is projected into the ball of radius sqrt(16 m_hi)
-// (App. E "Spherical shaping"); while the nearest lattice point lies beyond the last shell the working vector is
-// shrunk by 2 %; if it is the origin the input is scaled to the radius of the first shell.  ANGULAR: the input
-// direction is decoded at every shell radius sqrt(16 m); of the candidates inside the code the one with the
-// largest cosine wins (first radius on ties).  A zero input gives the point of index 0, (4, 4, 0^22), the first
-// point of the first class of Shell(2) (Sec. 2.3).  Needs m_lo == 2 and m_hi >= 6 (checked on the host).
+// One warp per input vector; inputs are binary32 values, all scoring runs in binary64 with one rounding per operation and
+// sums over the coordinates in order.  EUCLIDEAN: if the nearest lattice point of the input lies in the code it is the
+// answer (it is then also the nearest point of the cut, App. E "Spherical shaping").  Otherwise, and for ANGULAR always,
+// the input direction is decoded at every shell radius sqrt(16 m); of the candidates inside the code the one nearest to
+// the input (EUCLIDEAN) or with the largest cosine (ANGULAR) wins, the first radius on ties.  A zero input gives the
+// point of index 0, (4, 4, 0^22), the first point of the first class of Shell(2) (Sec. 2.3).  Needs m_lo == 2 and
+// m_hi >= 3 (checked on the host).
 __global__ void __launch_bounds__(kEncWarps * 32)
 encode_search_kernel(const uint32_t* __restrict__ golay, const float* __restrict__ v, uint64_t n, int metric, int m_lo, int m_hi,
                      int8_t* __restrict__ points, uint32_t* __restrict__ flags)
@@ -132,33 +169,43 @@ encode_search_kernel(const uint32_t* __restrict__ golay, const float* __restrict
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     WarpTables& W = tabs[warp];
     for (uint64_t vec = (uint64_t)blockIdx.x * kEncWarps + warp; vec < n; vec += (uint64_t)gridDim.x * kEncWarps) {
-        const float vi = lane < 24 ? __ldg(v + vec * 24 + lane) : 0.f;
-        const float n2 = warp_sum(vi * vi);
+        const double vi = lane < 24 ? (double)__ldg(v + vec * 24 + lane) : 0.0;
+        const double n2 = seq_sum24(__dmul_rn(vi, vi));
         int bestx = lane == 0 || lane == 1 ? 4 : 0;              // the point of index 0
-        bool ok = false;
-        if (n2 == 0.f) {
-            ok = true;
-        } else if (metric == LLVQ_EUCLIDEAN) {
-            const float r2 = 16.f * (float)m_hi;
-            float u = n2 > r2 ? vi * sqrtf(r2 / n2) : vi;
-            for (int it = 0; it < 64 && !ok; ++it) {
+        bool ok = false, direct = false;
+        const bool finite = n2 < 1.0e300;                        // false for NaN too
+        if (n2 == 0.0) {
+            ok = direct = true;
+        } else if (finite && metric == LLVQ_EUCLIDEAN) {
+            // no lattice point is farther than 4 from any input (covering radius): beyond radius sqrt(16 m_hi) + 4 the nearest
+            // point is certainly outside the code and the decode can be skipped
+            const double reach = sqrt(16.0 * (double)m_hi) + 4.01;
+            if (n2 <= reach * reach) {
                 int norm2;
-                const int x = lattice_nearest(W, golay_s, u, lane, norm2);
+                const int x = lattice_nearest(W, golay_s, vi, lane, norm2);
                 const int m = norm2 / 16;
-                if (m > m_hi) u *= 0.98f;
-                else if (m < 2) u = vi * sqrtf(32.f / n2);
-                else { ok = true; bestx = x; }
+                if (m >= m_lo && m <= m_hi) { ok = direct = true; bestx = x; }
             }
-        } else {
-            const float rn = 1.f / sqrtf(n2);
-            float best = -3.0e38f;
+        }
+        if (finite && !direct) {
+            const double rn = __ddiv_rn(1.0, __dsqrt_rn(n2));
+            double best = -1.0e300;
+            bool first = true;
             for (int m = m_lo; m <= m_hi; ++m) {
+                const double rad = __dsqrt_rn(__dmul_rn(16.0, (double)m));
                 int norm2;
-                const int x = lattice_nearest(W, golay_s, vi * rn * sqrtf(16.f * (float)m), lane, norm2);
+                const int x = lattice_nearest(W, golay_s, __dmul_rn(__dmul_rn(vi, rn), rad), lane, norm2);
                 const int mx = norm2 / 16;
                 if (mx < m_lo || mx > m_hi) continue;
-                const float score = warp_sum(vi * rn * (float)x) / sqrtf((float)norm2);
-                if (score > best) { best = score; bestx = x; ok = true; }
+                double score;
+                if (metric == LLVQ_EUCLIDEAN) {
+                    const double dd = __dsub_rn(vi, (double)x);
+                    score = -seq_sum24(lane < 24 ? __dmul_rn(dd, dd) : 0.0);
+                } else {
+                    const double dot = seq_sum24(lane < 24 ? __dmul_rn(__dmul_rn(vi, rn), (double)x) : 0.0);
+                    score = __ddiv_rn(dot, __dsqrt_rn((double)norm2));
+                }
+                if (first || score > best) { best = score; bestx = x; ok = true; first = false; }
             }
         }
         if (!ok) {

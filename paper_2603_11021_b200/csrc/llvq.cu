@@ -101,7 +101,7 @@ int llvq_create(llvq_ctx** out, int m_lo, int m_hi, int device)
     // encoder tables (point -> index), for codes the encoder supports
     std::vector<uint64_t> hkeys; std::vector<uint32_t> hcls;
     std::vector<uint16_t> pos12(4096, 0xffff);
-    ctx->can_encode = m_lo == 2 && m_hi >= 6 && h.W <= 64 && build_class_hash(h, hkeys, hcls);
+    ctx->can_encode = m_lo == 2 && m_hi >= 3 && h.W <= 64 && build_class_hash(h, hkeys, hcls);
     if (ctx->can_encode) {
         for (uint32_t j = 0; j < 4096; ++j) {
             uint16_t& slot = pos12[h.golay[j] & 0xfffu];
