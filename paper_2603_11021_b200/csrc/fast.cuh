@@ -90,15 +90,24 @@ __device__ __forceinline__ bool fast_load_image(uint8_t* dst, const uint8_t* __r
 }
 
 // Deposit the low bits of src into the set bits of mask, lowest first (24-bit masks, 6 bits per lookup).
+// r = a * b + c on the multiply-add pipe (the logic pipe is the busy one: sums of disjoint bit fields go here)
+__device__ __forceinline__ uint32_t mad_u32(uint32_t a, uint32_t b, uint32_t c)
+{
+    uint32_t r;
+    asm("mad.lo.u32 %0, %1, %2, %3;" : "=r"(r) : "r"(a), "r"(b), "r"(c));
+    return r;
+}
+
 __device__ __forceinline__ uint32_t deposit24(const uint8_t* pd6, uint32_t src, uint32_t mask)
 {
     // how many source bits the lower groups consume: known from the mask alone, so the four lookups are independent
     const uint32_t c1 = __popc(mask & 0x3fu), c2 = __popc(mask & 0xfffu), c3 = __popc(mask & 0x3ffffu);
-    const uint32_t r0 = pd6[((mask & 0x3fu) << 6) | (src & 63u)];
-    const uint32_t r1 = pd6[(((mask >> 6) & 0x3fu) << 6) | ((src >> c1) & 63u)];
-    const uint32_t r2 = pd6[(((mask >> 12) & 0x3fu) << 6) | ((src >> c2) & 63u)];
-    const uint32_t r3 = pd6[(((mask >> 18) & 0x3fu) << 6) | ((src >> c3) & 63u)];
-    return r0 | r1 << 6 | r2 << 12 | r3 << 18;
+    // row of a lookup = the group's 6 mask bits times 64: for groups 1..3 that is a masked (shifted) copy of the mask
+    const uint32_t r0 = pd6[mad_u32(mask & 0x3fu, 64u, src & 63u)];
+    const uint32_t r1 = pd6[(mask & 0xfc0u) + ((src >> c1) & 63u)];
+    const uint32_t r2 = pd6[((mask >> 6) & 0xfc0u) + ((src >> c2) & 63u)];
+    const uint32_t r3 = pd6[((mask >> 12) & 0xfc0u) + ((src >> c3) & 63u)];
+    return mad_u32(r3, 1u << 18, mad_u32(r2, 1u << 12, mad_u32(r1, 64u, r0)));
 }
 
 template <int kOff>
@@ -257,9 +266,9 @@ __device__ __forceinline__ void fast_decode_local(const FastSmem& T, uint32_t cl
             else if (kPar == 1 && l == 1 && __all_sync(mask, !active || nfree >= 22u)) a = deposit_two_holes(rel, freem);
             else a = deposit24(T.pd6, rel, freem);
             freem ^= a;
-            if (word & (1u << 27)) p0 |= a;
-            if (word & (1u << 28)) p1 |= a;
-            if (word & (1u << 29)) p2 |= a;
+            if ((l + 2) & 1) p0 |= a;                                   // the value id of level l is 2 + l
+            if ((l + 2) & 2) p1 |= a;
+            if ((l + 2) & 4) p2 |= a;
             if (kPar != 0 && (word & (1u << 30))) bit1 |= a;
             if (kPar != 1 && in_group0 && (word >> 31)) nz0 |= a;
         }
