@@ -180,10 +180,15 @@ int llvq_gemm_small_batch_sg(const llvq_ctx* ctx, const void* d_fields, int gain
  * llvq_gemv_sorted computes the same y = W x as llvq_gemv: all of App. A steps 1-4 still run in the kernel, but the
  * 32 lanes of a warp now execute one form with one trip count and read one class descriptor.
  * The sorted stream takes llvq_sorted_bytes() bytes (8 per block of the 8-row x 4-block units the matrix is padded
- * to; 0 if unsupported: the code must have its class tables in shared memory, at most 1023 classes and fewer than
- * 2^48 - 1 points, which holds for (2,2), (3,3) and (2,13), not for (2,53)).  The layout depends on the SM count of
- * the device; use it with the context that produced it.  d_sorted: device, 16-byte aligned.  Out-of-range fields
- * are counted when sorting and decode to zero.  Gains stay in their ROWWISE array.
+ * to; 0 if unsupported: a code with its class tables in shared memory needs at most 1023 classes and fewer than
+ * 2^48 - 1 points, which holds for (2,2), (3,3) and (2,13)).  The layout depends on the SM count of the device; use
+ * it with the context that produced it.  d_sorted: device, 16-byte aligned.  Out-of-range fields are counted when
+ * sorting and decode to zero.  Gains stay in their ROWWISE array.
+ * Codes whose class tables stay in global memory (the 72-bit code (2,53)): the three calls work on the layout of
+ * llvq_sort_blocks_gemm (96-bit entries in domains of 128 rows x 8 column blocks; llvq_sorted_bytes =
+ * llvq_sorted_gemm_bytes, llvq_sort_blocks = llvq_sort_blocks_gemm), which does not depend on the SM count, and
+ * llvq_gemv_sorted is the batch-1 case of the sorted small-batch product with the GEMV's output types; it asks for
+ * d_x_bf16 16-byte aligned and k_in % 8 == 0 (LLVQ_EALIGN otherwise) and n_out <= 65536.
  */
 size_t llvq_sorted_bytes(const llvq_ctx* ctx, int64_t n_out, int64_t k_in);
 int llvq_sort_blocks(const llvq_ctx* ctx, const void* d_idx, int64_t n_out, int64_t k_in, void* d_sorted, void* stream);
@@ -242,10 +247,12 @@ int llvq_gemm_small_batch(const llvq_ctx* ctx, const void* d_idx, const uint16_t
  * llvq_gemm_small_batch_sorted computes the same Y as llvq_gemm_small_batch from that stream and the unchanged
  * ROWWISE gains; all of App. A steps 1-4 run in the kernel.  llvq_sorted_gemm_bytes() gives the stream length (8 bytes
  * per block of the matrix padded to whole domains; 0 if unsupported: same codes as llvq_sort_blocks, plus the one below).
- * Codes whose class tables live in global memory (the 72-bit code, shells 2..53) take 128-bit entries, 16 bytes per
- * block: the stored index unchanged (72 bits), the number of its class (24 bits: App. A step 2 is then a table look-up
- * in the kernel instead of a search; steps 1, 3, 4 run there as before) and the position in the domain; the order is
- * by unranking steps, then class.  Out-of-range indices are counted by llvq_sort_blocks_gemm and stored as "no block".
+ * Codes whose class tables live in global memory (the 72-bit code, shells 2..53) take 96-bit entries, 12 bytes per
+ * block: the stored index unchanged (72 bits), the number of its class relative to the first class of the index's
+ * bucket in the table on the top 16 index bits (14 bits: App. A step 2 is then one table look-up in the kernel instead
+ * of a bisection over 128-bit offsets; steps 1, 3, 4 run there as before) and the position in the domain (10 bits); the
+ * order is by the shape of the unranking: parity (odd first), number of steps, which steps take at most three slots.
+ * Out-of-range indices are counted by llvq_sort_blocks_gemm and stored as "no block".
  * d_sorted: device, 16-byte aligned.  Other arguments and limits as in llvq_gemm_small_batch.
  */
 size_t llvq_sorted_gemm_bytes(const llvq_ctx* ctx, int64_t n_out, int64_t k_in);
@@ -293,15 +300,18 @@ int llvq_gemm_small_batch_noalloc(const llvq_ctx* ctx, const void* d_idx, const 
  * indices, ready for llvq_pack_fields).
  *
  * The paper defers the search itself to the literature.  Here the nearest point of the unbounded lattice is found
- * exactly by decoding all 2 x 4096 cosets (parity, Golay codeword) + 4 Z^24 under the sum rules of Sec. 2.4;
- * the restriction to the shells of the code is a policy:
- *   LLVQ_EUCLIDEAN (spherical shaping, App. E): the input is projected into the ball of radius sqrt(16 m_hi); while
- *     the nearest lattice point lies beyond the last shell the working vector is shrunk by 2 %; if it is the
- *     origin the input is scaled to the radius of the first shell and decoded again.
- *   LLVQ_ANGULAR (shape-gain, App. E): the input direction is decoded at every shell radius sqrt(16 m),
- *     m_lo <= m <= m_hi; of the candidates that lie in the code the one with the largest cosine wins.
+ * exactly by decoding all 2 x 4096 cosets (parity, Golay codeword) + 4 Z^24 under the sum rules of Sec. 2.4: a
+ * binary32 scan of all cosets, then every coset within rounding distance of the best one again in binary64 (one
+ * rounding per operation, sums over the coordinates in order; lowest parity, then lowest codeword position, among
+ * equal distances), so the result does not depend on the scan's rounding.  The restriction to the shells of the code:
+ *   LLVQ_EUCLIDEAN (spherical shaping, App. E): if the nearest lattice point of the input lies in the code it is the
+ *     answer (and then the nearest point of the cut as well).  Otherwise (input outside the ball, or next to the
+ *     origin) the input direction is decoded at every shell radius sqrt(16 m), m_lo <= m <= m_hi, and of the
+ *     candidates that lie in the code the one nearest to the input wins (first radius on ties): a candidate search,
+ *     not an exact one.
+ *   LLVQ_ANGULAR (shape-gain, App. E): the same candidates for every input; the one with the largest cosine wins.
  * A zero vector encodes to index 0.  Non-finite inputs encode to index 0 and set LLVQ_FLAG_SEARCH_GAVE_UP.
- * Supported codes: m_lo == 2, m_hi >= 6, indices of at most 64 bits; others return LLVQ_EUNSUPPORTED.
+ * Supported codes: m_lo == 2, m_hi >= 3, indices of at most 64 bits; others return LLVQ_EUNSUPPORTED.
  *
  * llvq_rank_blocks is the indexing step alone (point -> index, the inverse of llvq_decode_blocks): a point that
  * is not in the code gets index 0 and is counted like an out-of-range field (llvq_last_error).

@@ -24,7 +24,7 @@ __all__ = [
     "llvq_exchange_close", "llvq_signal_ranks", "llvq_wait_ranks", "LLVQ_EXCHANGE_HANDLE_BYTES",
     "llvq_gemm_small_batch_rowshard", "llvq_gemm_small_batch_sorted_rowshard",
     "llvq_sort_blocks_gemm_sg", "llvq_gemm_small_batch_sorted_sg",
-    "llvq_last_error", "LlvqError", "EXPORTS", "load_library",
+    "llvq_last_error", "LlvqError", "EXPORTS", "load_library", "llvq_gemv_multi", "llvq_gemv_sorted_multi", "GemvDesc",
     "LLVQ_LAYOUT_FLAT", "LLVQ_LAYOUT_ROWWISE", "LLVQ_F32", "LLVQ_BF16",
 ]
 
@@ -49,6 +49,7 @@ EXPORTS = [
     "llvq_exchange_close", "llvq_signal_ranks", "llvq_wait_ranks",
     "llvq_gemm_small_batch_rowshard", "llvq_gemm_small_batch_sorted_rowshard",
     "llvq_sort_blocks_gemm_sg", "llvq_gemm_small_batch_sorted_sg",
+    "llvq_gemv_multi", "llvq_gemv_sorted_multi",
 ]
 
 
