@@ -233,11 +233,13 @@ __device__ __forceinline__ void fast_decode_local(const FastSmem& T, uint32_t cl
                 if (kPar == -1 && (flags & 8u)) bit1 |= freem;
                 freem = F0; in_group0 = true;
             }
-            const bool active = (uint32_t)l < nlev;
+            // a lane whose class has fewer steps finds radix 1, k = 0 and all-ones reciprocals in its descriptor: the
+            // division returns remainder 0 and the rank unchanged, the empty subset is placed (lanes without a block run
+            // the steps of class 0, their result is dropped)
             const uint32_t word = lwords[l];
             const uint32_t radix = word & 0x3fffffu;
-            const uint32_t k = active ? (word >> 22) & 31u : 0u;
-            const uint32_t nfree = (mg.w >> (8 * l)) & 0xffu;            // slots free before this step
+            const uint32_t k = (word >> 22) & 31u;
+            const uint32_t nfree = (mg.w >> (8 * l)) & 0xffu;            // slots free before this step (0: no step)
             uint32_t rho;
             if (l == 0 && !rank32) {
                 uint64_t qq = __umul64hi(p, ((uint64_t)v.w << 32) | v.z);
@@ -250,7 +252,6 @@ __device__ __forceinline__ void fast_decode_local(const FastSmem& T, uint32_t cl
                 if (rem >= radix) { rem -= radix; ++qq; }
                 p32 = qq; rho = rem;
             }
-            if (!active) rho = 0u;
             uint32_t rel;
             if (T.sub3 != 0u && __all_sync(mask, k <= (uint32_t)kSmallSubsetMaxK)) {
                 rel = small_subset(T, k, rho);                          // few elements: one lookup whatever the number of slots
@@ -258,12 +259,12 @@ __device__ __forceinline__ void fast_decode_local(const FastSmem& T, uint32_t cl
                 int top;
                 if (kPar == 0) top = 16;
                 else if (kPar == 1 && l == 0) top = 24;
-                else top = __reduce_max_sync(mask, active ? nfree : 0u);
+                else top = __reduce_max_sync(mask, nfree);
                 rel = nth_subset(T, k, rho, top);
             }
             uint32_t a;
             if (kPar == 1 && l == 0) a = rel;                           // odd, first step: every position is free
-            else if (kPar == 1 && l == 1 && __all_sync(mask, !active || nfree >= 22u)) a = deposit_two_holes(rel, freem);
+            else if (kPar == 1 && l == 1 && __all_sync(mask, k == 0u || nfree >= 22u)) a = deposit_two_holes(rel, freem);
             else a = deposit24(T.pd6, rel, freem);
             freem ^= a;
             if ((l + 2) & 1) p0 |= a;                                   // the value id of level l is 2 + l

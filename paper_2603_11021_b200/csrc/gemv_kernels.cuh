@@ -309,9 +309,7 @@ sort_blocks_kernel(FastArgs fa, const uint32_t* __restrict__ stream, const uint1
 // lanes of a warp call this together; after sorting they almost always share the form (and the class).
 __device__ __forceinline__ void decode_known_class(const FastSmem& T, uint32_t cls, uint64_t local, bool valid, Decoded& r)
 {
-    const uint32_t h = T.desc[cls * kFastDescStride];
-    const uint32_t w8 = h & 0xffu;
-    const uint32_t kind = !valid ? kKindNull : ((h & (1u << 16)) ? kKindOdd : ((w8 == 8u || w8 == 12u || w8 == 16u) ? kKindEven : kKindOther));
+    const uint32_t kind = !valid ? kKindNull : (T.desc[cls * kFastDescStride] >> 22) & 3u;     // the form is part of the descriptor's flags
     r.p0 = r.p1 = r.p2 = r.neg = r.vals_lo = r.vals_hi = 0u;
     // every form writes r only for its own lanes
     if (__any_sync(kFullMask, kind == kKindOdd)) {

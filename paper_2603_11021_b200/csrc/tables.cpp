@@ -301,6 +301,8 @@ bool build_fast_image(const HostTables& t, FastLayout& L, std::vector<uint8_t>& 
         uint32_t flags = (d.parity ? 1u : 0u) | (d.signpar ? 2u : 0u) | (d.fill0 ? 4u : 0u) |
                          ((d.fill1 & 2) ? 8u : 0u) | ((d.fill0 & 2) ? 16u : 0u);
         if (!((t.info[j].card / ((u128)d.A << d.B)) >> 32)) flags |= kFastFlagRank32;
+        // decoder form of the class (bits 6-7): 0 even with Golay weight 8, 12 or 16, 1 odd, 2 any other
+        flags |= (d.parity ? 1u : ((d.w == 8 || d.w == 12 || d.w == 16) ? 0u : 2u)) << 6;
         w[0] = d.w | (uint32_t)d.B << 8 | flags << 16 | (uint32_t)d.nlev1 << 24 | (uint32_t)nlev << 28;
         w[1] = d.goff | (uint32_t)d.A << 16;
         w[2] = (uint32_t)d.magicA; w[3] = (uint32_t)(d.magicA >> 32);
@@ -321,6 +323,11 @@ bool build_fast_image(const HostTables& t, FastLayout& L, std::vector<uint8_t>& 
                 if (p_after >> 32) return false;                     // 32-bit quotient chain after the first step
                 w[11 + l] = (uint32_t)((1ull << 32) / lv.radix);
             }
+        }
+        for (int l = nlev; l < kFastMaxLevels; ++l) {          // steps the class does not have: radix 1 and the matching reciprocals, no slots:
+            w[8 + l] = 1u;                                      // the division by multiplication then returns the rank unchanged and
+            if (l == 0) { w[6] = w[7] = 0xffffffffu; w[kFastDescMagic0] = 0xffffffffu; }    // remainder 0, so a lane that runs such a
+            else w[11 + l] = 0xffffffffu;                       // step beside lanes with more steps needs no special case
         }
         std::memcpy(&w[4], vals, 8);
         w[15] = nbytes;

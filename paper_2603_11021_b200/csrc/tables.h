@@ -129,12 +129,13 @@ struct FastLayout {
 // Word layout of a fast descriptor:
 //  0: w | B << 8 | flags << 16 | nlev1 << 24 | nlev << 28
 //       flags: bit0 parity, bit1 signpar, bit2 fill0 is nonzero, bit3 fill1 has value bit 1, bit4 fill0 has value bit 1,
-//              bit5 the arrangement rank of the class fits 32 bits
+//              bit5 the arrangement rank of the class fits 32 bits, bits 6-7 decoder form (0 even with weight 8 / 12 / 16, 1 odd, 2 other)
 //  1: goff | A << 16
 //  2,3: magicA = floor((2^64-1)/A)
 //  4,5: absolute value of id 0..7 (one byte each): id 0 = fill0, id 1 = fill1, ids 2.. = levels in order
 //  6,7: magic of level 0 = floor((2^64-1)/radix0)
-//  8..11: level l: radix | k << 22 | id << 27 | (value bit 1) << 30 | (value nonzero) << 31
+//  8..11: level l: radix | k << 22 | id << 27 | (value bit 1) << 30 | (value nonzero) << 31; steps the class does not have:
+//         radix 1, k 0, reciprocals 0xffffffff (dividing by them leaves the rank unchanged and gives remainder 0)
 //  12..14: floor(2^32 / radix) of levels 1..3
 //  15: n (free slots before the step) of levels 0..3, one byte each
 //  16: binary32 bits of 1 / |x| = 1 / sqrt(16 m) (formed in binary64, rounded once), for the shape-gain form
