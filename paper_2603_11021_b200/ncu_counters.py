@@ -42,9 +42,9 @@ _SCALE = {"byte": 1.0, "Kbyte": 1e3, "Mbyte": 1e6, "Gbyte": 1e9, "ns": 1.0, "us"
 
 
 def source_hash() -> str:
-    """SHA-256 over the kernel sources (csrc and the public header), in a fixed order."""
+    """SHA-256 over the kernel sources (everything under csrc), in a fixed order."""
     h = hashlib.sha256()
-    files = sorted(glob.glob(os.path.join(PKG, "csrc", "*")) + glob.glob(os.path.join(ROOT, "include", "*.h")))
+    files = sorted(glob.glob(os.path.join(PKG, "csrc", "*")))
     for f in files:
         h.update(os.path.basename(f).encode())
         with open(f, "rb") as fh:
