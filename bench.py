@@ -706,7 +706,7 @@ def main() -> None:
 
     with ClockSampler(local_rank) as clocks:
         ms_per_step = timed(step, args.steps, args.warmup)
-        timed_launches = launches
+        timed_launches = launches - args.warmup              # the warm-up steps launch too; the timed region is args.steps launches
         # the same step for at least a quarter of a second, so that the clock samples cover a region of the headline kernel
         # that is long enough to mean something (the region above lasts a few milliseconds at small --steps)
         sustained_steps = max(args.steps, int(0.25 / (ms_per_step * 1e-3)))

@@ -99,16 +99,23 @@ __device__ int lattice_nearest(WarpTables& W, const uint32_t* __restrict__ golay
         const uint32_t c = golay_s[s * 32 + lane];
         best = fminf(best, fminf(coset_cost(W, c, 0u), coset_cost(W, c, 1u)));
     }
+    const float mine_best = best;                       // over this lane's 256 codewords
 #pragma unroll
     for (int o = 16; o; o >>= 1) best = fminf(best, __shfl_xor_sync(kFull, best, o));
     const float thr = best + (1.f / 4096.f + best * (1.f / 8192.f));
-    for (int s = 0; s < 128; ++s) {
-        const uint32_t j = (uint32_t)(s * 32 + lane), c = golay_s[j];
+    // only the lanes whose own minimum is within the margin can hold candidates (usually one lane): the warp goes through
+    // the 256 codewords of each such lane together, 8 per lane
+    for (uint32_t holders = __ballot_sync(kFull, mine_best <= thr); holders; holders &= holders - 1u) {
+        const uint32_t owner = (uint32_t)__ffs(holders) - 1u;
 #pragma unroll
-        for (uint32_t pi = 0; pi < 2; ++pi) {
-            if (coset_cost(W, c, pi) <= thr) {
-                const uint32_t slot = atomicAdd(&W.ncand, 1u);
-                if (slot < (uint32_t)kMaxCand) W.cand[slot] = pi << 12 | j;
+        for (int q = 0; q < 4; ++q) {
+            const uint32_t j = (uint32_t)((q * 32 + lane) * 32) + owner, c = golay_s[j];
+#pragma unroll
+            for (uint32_t pi = 0; pi < 2; ++pi) {
+                if (coset_cost(W, c, pi) <= thr) {
+                    const uint32_t slot = atomicAdd(&W.ncand, 1u);
+                    if (slot < (uint32_t)kMaxCand) W.cand[slot] = pi << 12 | j;
+                }
             }
         }
     }
