@@ -3,8 +3,8 @@
     ncu -i <capture>.ncu-rep --page raw --csv > raw.csv
     python -m paper_2603_11021_b200.ncu_counters raw.csv profiles/<name>_counters.json --blocks <blocks per launch>
 
-The counter file records, beside the counters of the first captured launch, the hash of the kernel sources at the
-time it is written (write it from the tree the capture ran on).  ``bench.py`` prints the counters only while
+The counter file records, beside the counters of the first captured launch, the names and the hash of the sources the
+captured kernel is compiled from at the time it is written (write it from the tree the capture ran on).  ``bench.py`` prints the counters only while
 that hash still matches the sources it runs: a kernel edited after its capture gets no stale numbers.
 """
 from __future__ import annotations
@@ -41,10 +41,15 @@ _SCALE = {"byte": 1.0, "Kbyte": 1e3, "Mbyte": 1e6, "Gbyte": 1e9, "ns": 1.0, "us"
           "msecond": 1e6, "second": 1e9}
 
 
-def source_hash() -> str:
-    """SHA-256 over the kernel sources (everything under csrc), in a fixed order."""
+# what the fused GEMV kernels are compiled from (the default set of sources a counter file vouches for)
+GEMV_SOURCES = ["tables.h", "tables.cpp", "ctx.h", "decode.cuh", "fast.cuh", "big.cuh", "umma.cuh", "kernels_common.cuh", "gemv_kernels.cuh",
+                "gemv.cu"]
+
+
+def source_hash(names=None) -> str:
+    """SHA-256 over the named files under csrc (default: everything there), in a fixed order."""
     h = hashlib.sha256()
-    files = sorted(glob.glob(os.path.join(PKG, "csrc", "*")))
+    files = sorted(glob.glob(os.path.join(PKG, "csrc", "*"))) if names is None else [os.path.join(PKG, "csrc", n) for n in sorted(names)]
     for f in files:
         h.update(os.path.basename(f).encode())
         with open(f, "rb") as fh:
@@ -53,13 +58,13 @@ def source_hash() -> str:
 
 
 def load(path: str) -> dict | None:
-    """The counter file, or None when it is missing or was written for other kernel sources."""
+    """The counter file, or None when it is missing or the sources it names have changed since it was written."""
     try:
         with open(path) as f:
             d = json.load(f)
+        return d if d.get("source_hash") == source_hash(d.get("sources")) else None
     except (OSError, ValueError):
         return None
-    return d if d.get("source_hash") == source_hash() else None
 
 
 def parse_raw_csv(path: str, kernel_filter: str | None = None) -> dict:
@@ -85,11 +90,13 @@ def main() -> None:
     ap.add_argument("--kernel", default=None, help="substring of the kernel name to pick (default: the first launch)")
     ap.add_argument("--blocks", type=int, required=True, help="blocks of 24 weights one launch processes")
     ap.add_argument("--workload", default="")
+    ap.add_argument("--sources", nargs="*", default=GEMV_SOURCES, help="files under csrc the captured kernel is compiled from")
     args = ap.parse_args()
     c = parse_raw_csv(args.raw_csv, args.kernel)
     c["blocks_per_launch"] = args.blocks
     c["workload"] = args.workload
-    c["source_hash"] = source_hash()
+    c["sources"] = sorted(args.sources)
+    c["source_hash"] = source_hash(args.sources)
     try:
         c["git_commit"] = subprocess.check_output(["git", "-C", ROOT, "rev-parse", "--short", "HEAD"], text=True).strip()
     except Exception:
