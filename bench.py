@@ -830,7 +830,7 @@ def main() -> None:
         counters = ncu_counters.load(COUNTER_FILE)               # None when the kernel sources changed after the capture
         roofline = {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
                     "traffic": counters["dram_traffic_bytes"] if counters else None,
-                    "kernel": "gemv_sorted_multi_kernel on the three layers of a step (one launch)",
+                    "kernel": "gemv_sorted_overlap_kernel on the three layers of a step (one launch)",
                     "algorithmic_bytes_per_launch": step_bytes, "peak_source": f"of {which}", "frac_of_nominal_8TBps": achieved / 8000.0,
                     "note": "the sorted layout stores 10 bytes per block (48-bit index, 16-bit position, fp16 gain) against the 8 algorithmic ones; "
                             "what binds the kernel is the integer pipe, see roofline_issue"}

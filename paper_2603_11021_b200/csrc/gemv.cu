@@ -294,6 +294,34 @@ static int gemv_multi_common(const llvq_ctx* ctx, const llvq_gemv_desc* descs, i
     cudaStream_t st = (cudaStream_t)stream;
     const FastArgs fa = fast_args(ctx, ext);
     const unsigned g = (unsigned)ctx->sm_count;
+    if (sorted && n_mats >= 2) {
+        // the kernel without a barrier between the matrices, when every CTA's share of every matrix is one segment and
+        // one pass and three sets of (x, row sums) fit beside the tables
+        int64_t max_groups = 0, max_nq = 0;
+        bool one_pass = true;
+        for (int i = 0; i < n_mats && one_pass; ++i) {
+            const int64_t nq = ((descs[i].k_in + 23) / 24 + 3) / 4;
+            const int64_t U = ((descs[i].n_out + kGemvGroupRows - 1) / kGemvGroupRows) * nq;
+            max_nq = std::max(max_nq, nq);
+            for (int64_t c = 0; c < g; ++c) {
+                const int64_t ub = c * U / g, ue = (c + 1) * U / g;
+                if (ue - ub > kSortSegUnits) { one_pass = false; break; }
+                max_groups = std::max(max_groups, (ue - 1) / nq - ub / nq + 1);
+            }
+        }
+        const int xs_words = (int)(max_nq * 48), acc_rows = (int)(max_groups * kGemvGroupRows);
+        const size_t smem_ov = fa.image_bytes + 16 + (size_t)kOverlapSets * ((size_t)xs_words + (size_t)kSortAccCopies * acc_rows) * 4 + kOverlapSets * sizeof(OverlapSet);
+        if (one_pass && max_groups <= kGemvGroupsPerPass && smem_ov <= kSmemLimit) {
+            if (y_dtype == LLVQ_BF16) {
+                if (!set_smem(gemv_sorted_overlap_kernel<true>, smem_ov)) return LLVQ_ECUDA;
+                if (launch_pdl(gemv_sorted_overlap_kernel<true>, g, (unsigned)kSortThreads, smem_ov, st, fa, mm, xs_words, acc_rows, ctx->d_scratch, ctx->d_counters) != cudaSuccess) return LLVQ_ECUDA;
+            } else {
+                if (!set_smem(gemv_sorted_overlap_kernel<false>, smem_ov)) return LLVQ_ECUDA;
+                if (launch_pdl(gemv_sorted_overlap_kernel<false>, g, (unsigned)kSortThreads, smem_ov, st, fa, mm, xs_words, acc_rows, ctx->d_scratch, ctx->d_counters) != cudaSuccess) return LLVQ_ECUDA;
+            }
+            return launch_status();
+        }
+    }
     if (sorted) {
         if (y_dtype == LLVQ_BF16) {
             if (!set_smem(gemv_sorted_multi_kernel<true>, smem)) return LLVQ_ECUDA;

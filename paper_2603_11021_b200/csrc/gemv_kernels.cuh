@@ -81,9 +81,11 @@ __device__ __forceinline__ void stage_x(uint32_t* xs, const uint16_t* __restrict
 template <bool kOutBf16, bool kShard, typename RowSum>
 __device__ __forceinline__ void finish_pass(const YOut& yo, int64_t rg0, int64_t rg1, int64_t nq, int64_t u_begin, int64_t u_end,
                                             int64_t U, int64_t G, int64_t n_out, float* __restrict__ scratch,
-                                            uint32_t* __restrict__ counters, RowSum row_sum, int64_t slot0 = 0)
+                                            uint32_t* __restrict__ counters, RowSum row_sum, int64_t slot0 = 0, int warp_of = -1, int nwarps_of = 0)
 {
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, nwarps = (int)(blockDim.x >> 5);
+    // by default the warps of the CTA share the row groups; warp_of / nwarps_of let a subset of the warps (one warp) do it
+    const int warp = warp_of >= 0 ? warp_of : (int)(threadIdx.x >> 5), lane = threadIdx.x & 31;
+    const int nwarps = warp_of >= 0 ? nwarps_of : (int)(blockDim.x >> 5);
     for (int64_t rg = rg0 + warp; rg <= rg1; rg += nwarps) {
         const bool whole = u_begin <= rg * nq && (rg + 1) * nq <= u_end;
         const int64_t row = rg * kGemvGroupRows + lane;
@@ -469,6 +471,146 @@ gemv_sorted_multi_kernel(FastArgs fa, const __grid_constant__ GemvMulti mm, floa
         gemv_sorted_body<kOutBf16, false, false>(fa, T, staging, static_cast<const unsigned long long*>(M.weights), M.gain, SgArgs{}, M.n_out, M.k_in,
                                                  (M.k_in + 23) / 24, M.nq_magic, M.x, yo, scratch, counters, M.slot0);
         __syncthreads();                                   // the next matrix restages x and clears the row sums
+    }
+}
+
+// The same, without a block barrier between the matrices: a warp that finds no chunk of matrix i left goes on to matrix
+// i + 1 while the others finish theirs, so the partly filled last round of chunks, the end of the pass and the staging of
+// x of one matrix run under the next matrix's work.  Three sets of (x, row sums, chunk counter) rotate: the warp that
+// completes matrix i (the last to run out of its chunks) ends the pass alone and then prepares set i % 3 for matrix
+// i + 3.  Taken when every CTA's share of every matrix is one segment and one pass (checked on the host).
+constexpr int kOverlapSets = 3;
+constexpr uint32_t kOverlapSpins = 1u << 22;         // polls of a shared-memory flag before a warp gives up (never in a correct run)
+
+struct OverlapSet {
+    uint32_t next_chunk;
+    uint32_t arrived;                                // warps that have run out of chunks of the set's matrix
+    uint32_t ready;                                  // index + 1 of the matrix the set is prepared for
+    uint32_t pad;
+};
+
+template <bool kOutBf16>
+__global__ void __launch_bounds__(kSortThreads, 1)
+gemv_sorted_overlap_kernel(FastArgs fa, const __grid_constant__ GemvMulti mm, int xs_words, int acc_rows, float* __restrict__ scratch,
+                           uint32_t* __restrict__ counters)
+{
+    prefetch_first_chunks(static_cast<const unsigned long long*>(mm.m[0].weights), mm.m[0].n_out, (mm.m[0].k_in + 23) / 24);
+    FAST_PROLOGUE();
+    // [kOverlapSets] x { x as packed pairs [xs_words] | row sums [kSortAccCopies][acc_rows] } | control words
+    const int set_words = xs_words + kSortAccCopies * acc_rows;
+    uint32_t* sets = reinterpret_cast<uint32_t*>(staging);
+    volatile OverlapSet* ctl = reinterpret_cast<volatile OverlapSet*>(sets + kOverlapSets * set_words);
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const uint32_t kWarps = blockDim.x >> 5;
+    const int64_t G = gridDim.x;
+
+    // what this CTA owns of matrix i
+    auto share = [&](int i, int64_t& nq, int64_t& U, int64_t& ub, int64_t& ue) {
+        const GemvMat& M = mm.m[i];
+        nq = ((M.k_in + 23) / 24 + 3) / 4;
+        U = ((M.n_out + kGemvGroupRows - 1) / kGemvGroupRows) * nq;
+        ub = blockIdx.x * U / G; ue = (blockIdx.x + 1) * U / G;
+    };
+    // prepare set i % kOverlapSets for matrix i with the calling threads (`nthreads` of them, numbered `tid`)
+    auto prepare = [&](int i, int tid, int nthreads) {
+        const GemvMat& M = mm.m[i];
+        uint32_t* xs = sets + (i % kOverlapSets) * set_words;
+        float* acc = reinterpret_cast<float*>(xs + xs_words);
+        const int64_t words = (int64_t)(((M.k_in + 23) / 24 + 3) / 4) * 48;
+        for (int64_t w = tid; w < words; w += nthreads) {
+            const int64_t e = 2 * w;
+            const uint32_t lo = e < M.k_in ? __ldg(M.x + e) : 0u, hi = e + 1 < M.k_in ? __ldg(M.x + e + 1) : 0u;
+            xs[w] = lo | hi << 16;
+        }
+        for (int r = tid; r < kSortAccCopies * acc_rows; r += nthreads) acc[r] = 0.f;
+    };
+
+    if (threadIdx.x < kOverlapSets) { ctl[threadIdx.x].next_chunk = 0u; ctl[threadIdx.x].arrived = 0u; ctl[threadIdx.x].ready = 0u; }
+    for (int i = 0; i < kOverlapSets && i < mm.n; ++i) prepare(i, (int)threadIdx.x, (int)blockDim.x);
+    __syncthreads();
+    if (threadIdx.x < kOverlapSets && (int)threadIdx.x < mm.n) ctl[threadIdx.x].ready = threadIdx.x + 1u;
+    __syncthreads();
+
+    for (int i = 0; i < mm.n; ++i) {
+        const GemvMat& M = mm.m[i];
+        const int set = i % kOverlapSets;
+        int64_t nq, U, ub, ue;
+        share(i, nq, U, ub, ue);
+        const int64_t bpr = (M.k_in + 23) / 24;
+        const int64_t rg0 = ub / nq, rg1 = ub < ue ? (ue - 1) / nq : rg0 - 1;
+        // the set is prepared for this matrix long before a warp gets here; a bounded wait all the same
+        {
+            uint32_t spins = 0;
+            while (ctl[set].ready != (uint32_t)i + 1u && ++spins < kOverlapSpins) {}
+            if (ctl[set].ready != (uint32_t)i + 1u) { if (lane == 0) atomicOr(fa.flags, 1u); return; }
+            __threadfence_block();
+        }
+        const uint32_t* xs = sets + set * set_words;
+        float* acc = reinterpret_cast<float*>(sets + set * set_words + xs_words);
+        const uint32_t nchunks = (uint32_t)(ue - ub), nq32 = (uint32_t)nq;
+        const uint32_t kq_a = (uint32_t)(ub - rg0 * nq);
+        const unsigned long long* seg = static_cast<const unsigned long long*>(M.weights) + ub * 32 + lane;
+        if (i + 1 < mm.n && warp == 0) {                    // ask for the next matrix's first chunks in L2
+            int64_t nq2, U2, ub2, ue2;
+            share(i + 1, nq2, U2, ub2, ue2);
+            const unsigned long long* nxt = static_cast<const unsigned long long*>(mm.m[i + 1].weights) + ub2 * 32;
+            for (int c = lane; c < 64 && ub2 + c / 2 < ue2; c += 32) asm volatile("prefetch.global.L2 [%0];" ::"l"(nxt + c * 16));
+        }
+        uint32_t ch = 0;
+        if (lane == 0) ch = atomicAdd(const_cast<uint32_t*>(&ctl[set].next_chunk), 1u);
+        ch = __shfl_sync(kFullMask, ch, 0);
+        unsigned long long e = ch < nchunks ? __ldg(seg + (uint64_t)ch * 32) : 0ull;
+        while (ch < nchunks) {
+            uint32_t nxt = 0;
+            if (lane == 0) nxt = atomicAdd(const_cast<uint32_t*>(&ctl[set].next_chunk), 1u);
+            nxt = __shfl_sync(kFullMask, nxt, 0);
+            const unsigned long long e_next = nxt < nchunks ? __ldg(seg + (uint64_t)nxt * 32) : 0ull;
+            const uint64_t I = e & kSortIndexMask;
+            const uint32_t pos = (uint32_t)(e >> 48);
+            const bool valid = I != kSortIndexMask && I < fa.n_points;
+            const uint32_t v = kq_a + (pos >> 5);
+            uint32_t q = __umulhi(v, M.nq_magic), kq = v - q * nq32;
+            if (kq >= nq32) { kq -= nq32; ++q; }
+            const uint32_t rloc = q * kGemvGroupRows + ((pos >> 2) & 7u);                 // row inside the CTA's share
+            const uint32_t cb = kq * 4u + (pos & 3u);
+            float gn = 0.f;
+            if (valid) gn = gain_to_float(__ldg(M.gain + ((int64_t)rg0 * kGemvGroupRows + rloc) * bpr + cb));
+            Decoded r;
+            decode_sorted_entry(fa, T, I, valid, r);
+            uint32_t w[12];
+            expand_bf16(r, gn, w);
+            const uint4* xb = reinterpret_cast<const uint4*>(xs + cb * 12u);
+            const uint4 x0 = xb[0], x1 = xb[1], x2 = xb[2];
+            const uint32_t xv[12] = {x0.x, x0.y, x0.z, x0.w, x1.x, x1.y, x1.z, x1.w, x2.x, x2.y, x2.z, x2.w};
+            const float dot = dot24_bf16(w, xv);
+            if (valid) atomicAdd(&acc[(warp & (kSortAccCopies - 1)) * acc_rows + rloc], dot);
+            ch = nxt; e = e_next;
+        }
+        // out of chunks: count this warp in; the last one ends the pass and hands the set on
+        __threadfence_block();
+        uint32_t last = 0;
+        if (lane == 0) last = atomicAdd(const_cast<uint32_t*>(&ctl[set].arrived), 1u) == kWarps - 1u;
+        last = __shfl_sync(kFullMask, last, 0);
+        if (last) {
+            __threadfence_block();
+            YOut yo{};
+            yo.y = M.y;
+            auto row_sum = [&](int64_t rr) {
+                float vv = 0.f;
+#pragma unroll
+                for (int c = 0; c < kSortAccCopies; ++c) vv += acc[c * acc_rows + rr];
+                return vv;
+            };
+            if (ub < ue) finish_pass<kOutBf16, false>(yo, rg0, rg1, nq, ub, ue, U, G, M.n_out, scratch, counters, row_sum, M.slot0, 0, 1);
+            __syncwarp();
+            if (i + kOverlapSets < mm.n) {
+                if (lane == 0) { ctl[set].next_chunk = 0u; ctl[set].arrived = 0u; }
+                prepare(i + kOverlapSets, lane, 32);
+                __threadfence_block();
+                __syncwarp();
+                if (lane == 0) ctl[set].ready = (uint32_t)(i + kOverlapSets) + 1u;
+            }
+        }
     }
 }
 

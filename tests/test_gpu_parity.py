@@ -835,3 +835,27 @@ def test_gemv_multi_full_size_step_and_limits(lib, ctxs, oracle_mod):
     with pytest.raises(lib.LlvqError):
         lib.llvq_gemv_sorted_multi(ctx, [tiny], y_dtype=torch.bfloat16)
     assert lib.llvq_last_error(ctx) == (0, 0)
+
+
+def test_gemv_sorted_multi_takes_the_kernel_with_barriers_where_a_share_needs_several_passes(lib, ctxs, oracle_mod):
+    # tall, narrow matrices: a thread block's share covers more row groups than it keeps sums for at a time, so the
+    # multi-matrix call cannot let its warps run ahead into the next matrix and uses the kernel with a block barrier
+    # between the matrices; a call with a single matrix does too
+    o = _oracle(oracle_mod)((2, 13))
+    ctx = ctxs[(2, 13)]
+    mats, refs = [], []
+    for i, (n, k) in enumerate([(8 * 140 * _sm_count() + 3, 24), (8 * 131 * _sm_count(), 48)]):
+        stream, gain, _ = gen.make_layer(o.N, o.W, n, k, 1, seed=90 + i)
+        x = gen.normal_bf16(k, seed=90 + i)
+        mats.append((lib.llvq_sort_blocks(ctx, to_dev_u8(stream), n, k), to_dev_f16(gain), n, k, to_dev_bf16(x),
+                     torch.full((n,), float("nan"), dtype=torch.float32, device="cuda")))
+        refs.append(o.gemv(stream, gain, n, k, x, threads=_threads()))
+    lib.llvq_gemv_sorted_multi(ctx, mats)
+    torch.cuda.synchronize()
+    for m, ref in zip(mats, refs):
+        assert gemv_error(m[5].cpu().numpy(), ref) <= TOL
+    mats[0][5].fill_(float("nan"))
+    lib.llvq_gemv_sorted_multi(ctx, mats[:1])
+    torch.cuda.synchronize()
+    assert gemv_error(mats[0][5].cpu().numpy(), refs[0]) <= TOL
+    assert lib.llvq_last_error(ctx) == (0, 0)
