@@ -53,12 +53,11 @@ __device__ __forceinline__ uint64_t lds_u64(uint32_t addr)
 // reciprocal comes from the tables beside it (64-bit while the arrangement rank needs it, 32-bit afterwards), steps that
 // take at most three slots are one lookup in the table of small subsets, and the point comes out as bit planes of value
 // ids.  All lanes of `mask` call this together; writes `out` only where `valid` (the caller presets it).
-__device__ __forceinline__ void big_decode_planes(const FastSmem& T, const DevCode& dc, int cls, uint64_t local, bool valid, uint32_t mask,
+// The class record arrives in registers (h0, h1 = its two 16-byte halves; zeros where !valid), so that a caller can
+// request it well before the block's turn.
+__device__ __forceinline__ void big_decode_record(const FastSmem& T, const uint4 h0, const uint4 h1, uint64_t local, bool valid, uint32_t mask,
                                                   DecodedBig& out)
 {
-    const uint4* cd = reinterpret_cast<const uint4*>(dc.big + (valid ? cls : 0));
-    const uint4 zero4 = make_uint4(0u, 0u, 0u, 0u);
-    const uint4 h0 = valid ? __ldg(cd) : zero4, h1 = valid ? __ldg(cd + 1) : zero4;
     const uint32_t w = h0.x & 0xff, B = (h0.x >> 8) & 0xff, flags = (h0.x >> 16) & 0xff;
     const uint32_t nlev1 = (h0.x >> 24) & 0xf, nlev = h0.x >> 28;
     const uint32_t goff = h0.y & 0xffff, A = h0.y >> 16;
@@ -151,6 +150,26 @@ __device__ __forceinline__ void big_decode_planes(const FastSmem& T, const DevCo
         out.d.vals_lo = h0.z; out.d.vals_hi = h0.w;
         out.p3 = p3; out.val8 = h1.z & 0xffu;
     }
+}
+
+// The 32-byte record of class `cls` (zeros where !valid), read from global memory / L2.  The loads are volatile
+// statements: they stay where the caller put them relative to its other volatile statements (the table reads of the decoder).
+__device__ __forceinline__ void big_load_record(const DevCode& dc, int cls, bool valid, uint4& h0, uint4& h1)
+{
+    h0 = h1 = make_uint4(0u, 0u, 0u, 0u);
+    if (valid) {
+        const BigDesc* rec = dc.big + cls;
+        asm volatile("ld.global.nc.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(h0.x), "=r"(h0.y), "=r"(h0.z), "=r"(h0.w) : "l"(rec));
+        asm volatile("ld.global.nc.v4.u32 {%0, %1, %2, %3}, [%4+16];" : "=r"(h1.x), "=r"(h1.y), "=r"(h1.z), "=r"(h1.w) : "l"(rec));
+    }
+}
+
+__device__ __forceinline__ void big_decode_planes(const FastSmem& T, const DevCode& dc, int cls, uint64_t local, bool valid, uint32_t mask,
+                                                  DecodedBig& out)
+{
+    uint4 h0, h1;
+    big_load_record(dc, cls, valid, h0, h1);
+    big_decode_record(T, h0, h1, local, valid, mask, out);
 }
 
 // Where the fourth plane is set the value id is 8: put bf16(gain * val8), signed, over what the three-plane expansion

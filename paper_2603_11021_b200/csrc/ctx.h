@@ -26,7 +26,6 @@ struct llvq_ctx {
     float* d_scratch = nullptr;      // split-K accumulation buffer of the small-batch GEMM, kept all-zero between calls
     uint32_t* d_counters = nullptr;  // per row tile arrival counters, kept zero between calls
     void* d_shard = nullptr;         // device copy of the destinations (peers' Y and flags) of the row-sharded GEMM in flight
-    int bucket_classes_max = 0;      // most classes that begin inside one bucket of the class table on the top 16 index bits
     bool fast = false;               // class tables fit the shared-memory image; otherwise they are read from global memory
     llvq::FastLayout fl{};
     const uint8_t* d_image = nullptr;

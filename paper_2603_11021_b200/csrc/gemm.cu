@@ -171,7 +171,7 @@ extern "C" {
 // Sorted layout of the small-batch GEMM (see the comment at sort_blocks_gemm_kernel).
 static bool gemm_sortable(const llvq_ctx* ctx)
 {
-    if (!ctx->fast) return ctx->host.W <= 72 && ctx->bucket_classes_max <= (int)kBigDeltaMask;   // 96-bit entries: 72-bit index + class within its bucket + position
+    if (!ctx->fast) return (int)ctx->host.desc.size() <= (1 << kBigClassBits);   // 96-bit entries: class-local index (63 bits) + class + position
     return ctx->d_sort_rank && ctx->host.W <= 48 && ctx->host.N < (u128)kSortIndexMask;
 }
 

@@ -258,18 +258,18 @@ sort_blocks_gemm_kernel(FastArgs fa, const uint32_t* __restrict__ stream, const 
 }
 
 // The same layout for codes whose class tables live in global memory (72-bit indices): 96-bit entries (three 32-bit
-// words): the stored index unchanged (bits 0..71), then 14 bits that name its class relative to the first class of
-// the index's bucket in the table on the top 16 index bits (so the kernel finds the class with one table read instead
-// of a bisection over 128-bit offsets), then the position in the domain (10 bits).  An index byte 64..71 of 0xff marks
-// "no block" (ragged edge or index out of range).  The blocks of a domain are ordered by the shape of their unranking:
-// parity (odd first), number of steps (most first), which of the steps take at most three slots, steps of the first
-// group; the lanes of a warp then run the same trip counts over similar slot counts and mostly agree on the cheap form
-// of a step.
-// Inside the kernels an entry travels as two 64-bit words: x = index bits 0..63, y = bits 64..71 | class << 8 |
-// position << 32, bit 63 = no block.
+// words).  An index is stored as its two digits in the mixed radix of the class table (App. A step 2, taken when the
+// layout is made): words 0-1 = the class-local index I - offset[class] (class sizes fit 63 bits; bit 63 set marks "no
+// block": ragged edge or index out of range), word 2 = class (17 bits) | position in the domain << 17 (10 bits).  The
+// kernel then needs neither the bucket table nor the 128-bit offsets, and the class record can be requested as soon as
+// the entry is there.  The blocks of a domain are ordered by the shape of their unranking: parity (odd first), number of
+// steps (most first), which of the steps take at most three slots, steps of the first group; the lanes of a warp then
+// run the same trip counts over similar slot counts and mostly agree on the cheap form of a step.
+// Inside the kernels an entry travels as two 64-bit words: x = the class-local index (stored stream: index bits 0..63),
+// y = class << 8 | position << 32, bit 63 = no block (stored stream: index bits 64..71 in the low byte).
 constexpr unsigned long long kBigNoBlock = 1ull << 63;
 constexpr int kBigEntryWords = 3;
-constexpr uint32_t kBigDeltaMask = 0x3fffu;
+constexpr int kBigClassBits = 17;
 
 // Top 16 bits of a W-bit index (hi:lo): the bucket of the class table.
 __device__ __forceinline__ uint32_t big_bucket(const DevCode& dc, uint64_t lo, uint64_t hi)
@@ -278,15 +278,14 @@ __device__ __forceinline__ uint32_t big_bucket(const DevCode& dc, uint64_t lo, u
     return (uint32_t)(sh >= 64 ? hi >> (sh - 64) : (sh ? (lo >> sh) | (hi << (64 - sh)) : lo)) & 0xffffu;
 }
 
-// Entry `at` of a sorted stream of 96-bit entries, in the two-word form the kernels use (one read of the bucket table).
-__device__ __forceinline__ ulonglong2 load_big_entry(const DevCode& dc, const void* sorted, int64_t at)
+// Entry `at` of a sorted stream of 96-bit entries, in the two-word form the kernels use.
+__device__ __forceinline__ ulonglong2 load_big_entry(const void* sorted, int64_t at)
 {
     const uint32_t* p = static_cast<const uint32_t*>(sorted) + at * kBigEntryWords;
     const uint32_t w0 = __ldg(p), w1 = __ldg(p + 1), w2 = __ldg(p + 2);
-    const unsigned long long lo = (unsigned long long)w1 << 32 | w0, hi = w2 & 0xffu, pos = w2 >> 22;
-    if (hi == 0xffull) return make_ulonglong2(0ull, kBigNoBlock | pos << 32);
-    const uint32_t cls = __ldg(dc.lut16 + big_bucket(dc, lo, hi)) + ((w2 >> 8) & kBigDeltaMask);
-    return make_ulonglong2(lo, hi | (unsigned long long)cls << 8 | pos << 32);
+    const unsigned long long pos = w2 >> kBigClassBits, cls = w2 & ((1u << kBigClassBits) - 1u);
+    return make_ulonglong2((unsigned long long)(w1 & 0x7fffffffu) << 32 | w0,
+                           ((unsigned long long)(w1 >> 31) << 63) | cls << 8 | pos << 32);
 }
 
 __global__ void __launch_bounds__(kDomEntries, 1)
@@ -300,7 +299,7 @@ sort_blocks_gemm_big_kernel(FastArgs fa, const uint32_t* __restrict__ stream, in
     for (int64_t dom = blockIdx.x; dom < ndomains; dom += gridDim.x) {
         const int64_t rt = dom / nd, d = dom - rt * nd;
         const int64_t row = rt * kGemmRows + (i >> 3), cb = d * kDomBlocks + (i & 7);
-        unsigned long long x = 0ull, y = 0xffull | (unsigned long long)i << 22;   // word 2 of an entry: index byte 0xff = no block
+        unsigned long long x = kBigNoBlock, y = (unsigned long long)i << kBigClassBits;   // words 0-1 and word 2 of an entry
         uint32_t key = 0x7ffffc00u | (uint32_t)i;                   // no block: after everything else
         if (row < n_out && cb < bpr) {
             uint64_t lo, hi;
@@ -311,9 +310,8 @@ sort_blocks_gemm_big_kernel(FastArgs fa, const uint32_t* __restrict__ stream, in
                 const uint32_t* rec = reinterpret_cast<const uint32_t*>(fa.dc.big + cls);
                 const uint32_t h = __ldg(rec), small_k = __ldg(rec + 6) >> 24;
                 const uint32_t nlev = h >> 28, nlev1 = (h >> 24) & 7u, parity = (h >> 16) & 1u;
-                const uint32_t delta = cls - __ldg(fa.dc.lut16 + big_bucket(fa.dc, lo, hi));      // < 2^14: checked when the context was made
-                x = lo;
-                y = (hi & 0xffull) | (unsigned long long)delta << 8 | (unsigned long long)i << 22;
+                x = local;
+                y = (unsigned long long)cls | (unsigned long long)i << kBigClassBits;
                 // odd classes first (their steps choose among up to 24 slots, the even classes' among at most 16), then by steps
                 key = (1u - parity) << 24 | (7u - min(nlev, 7u)) << 21 | (small_k & 0x7fu) << 14 | nlev1 << 11 | (uint32_t)i;
             } else {
@@ -393,7 +391,7 @@ gemm_sorted_kernel(FastArgs fa, const unsigned long long* __restrict__ sorted, c
             // warps pair chunk w - 1 of the first domain with chunk 31 - w of the second
             const int chunk = warp == 0 ? 31 : (q == 0 ? warp - 1 : 31 - warp);
             const int64_t at = (rt * nd + d + q) * kDomEntries + chunk * 32 + lane;
-            if (kBig) return load_big_entry(fa.dc, sorted, at);
+            if (kBig) return load_big_entry(sorted, at);
             return make_ulonglong2(__ldg(sorted + at), 0ull);
         };
         ulonglong2 e0 = entry_at(d_begin, 0), e1 = dpi > 1 ? entry_at(d_begin, 1) : no_entry;
@@ -417,9 +415,8 @@ gemm_sorted_kernel(FastArgs fa, const unsigned long long* __restrict__ sorted, c
                 uint32_t w[12];
                 if (kBig) {
                     const int cls = valid ? (int)((uint32_t)(e.y >> 8) & 0xffffffu) : 0;
-                    const uint64_t local = valid ? e.x - __ldg(fa.dc.off_lo + cls) : 0ull;     // class sizes fit 63 bits: exact mod 2^64
                     DecodedBig dec{};
-                    big_decode_planes(T, fa.dc, cls, local, valid, kFullMask, dec);
+                    big_decode_planes(T, fa.dc, cls, valid ? e.x : 0ull, valid, kFullMask, dec);
                     expand_bf16(dec.d, gn, w);
                     patch_id8_bf16(dec, gn, w);
                 } else {
@@ -648,11 +645,14 @@ gemm_pipe_kernel(FastArgs fa, const unsigned long long* __restrict__ sorted, con
                     return make_ulonglong2(f | (unsigned long long)pos << 48, 0ull);
                 }
                 const int64_t at = (rt * nd + d_begin + (int)(t >> 5)) * kDomEntries + (t & 31u) * 32u + lane;
-                if (kBig) return load_big_entry(fa.dc, sorted, at);
+                if (kBig) return load_big_entry(sorted, at);
                 return make_ulonglong2(__ldg(sorted + at), 0ull);
             };
             uint32_t tk = (uint32_t)warp - 1u;
             ulonglong2 e = entry_of(tk);
+            // sorted 96-bit entries name their class: its record is requested while the previous chunk is still being expanded
+            uint4 rec0 = make_uint4(0u, 0u, 0u, 0u), rec1 = rec0;
+            if (kBig && !kStored) big_load_record(fa.dc, (int)((uint32_t)(e.y >> 8) & 0xffffffu), !(e.y >> 63), rec0, rec1);
             while (tk < n_tickets) {
                 uint32_t tk_next = 0;
                 if (lane == 0) tk_next = atomicAdd(ticket, 1u);
@@ -676,13 +676,16 @@ gemm_pipe_kernel(FastArgs fa, const unsigned long long* __restrict__ sorted, con
                 if (kBig) {
                     int cls = 0;
                     uint64_t local = 0;
-                    if (kStored) { if (valid) cls = big_find_class(fa.dc, e.x, e.y & 0xffull, local); }
-                    else if (valid) {
-                        cls = (int)((uint32_t)(e.y >> 8) & 0xffffffu);
-                        local = e.x - __ldg(fa.dc.off_lo + cls);                 // class sizes fit 63 bits: exact mod 2^64
-                    }
                     DecodedBig dec{};
-                    big_decode_planes(T, fa.dc, cls, local, valid, kFullMask, dec);
+                    if (kStored) {
+                        if (valid) cls = big_find_class(fa.dc, e.x, e.y & 0xffull, local);
+                        big_decode_planes(T, fa.dc, cls, local, valid, kFullMask, dec);
+                    } else {
+                        big_decode_record(T, rec0, rec1, valid ? e.x : 0ull, valid, kFullMask, dec);
+                        // the next chunk's entries were requested a whole chunk ago: they are here, and their records have the
+                        // rest of this iteration to arrive
+                        big_load_record(fa.dc, (int)((uint32_t)(e_next.y >> 8) & 0xffffffu), !(e_next.y >> 63), rec0, rec1);
+                    }
                     expand_bf16(dec.d, gn, w);
                     patch_id8_bf16(dec, gn, w);
                 } else {

@@ -86,7 +86,6 @@ int llvq_create(llvq_ctx** out, int m_lo, int m_hi, int device)
     if (!ctx->fast && !build_fast_image(h, ctx->fl, image, false)) { delete ctx; return LLVQ_EUNSUPPORTED; }
     std::vector<uint32_t> lut16;
     build_bucket_table(h, lut16);
-    for (size_t b = 0; b + 1 < lut16.size(); ++b) ctx->bucket_classes_max = std::max(ctx->bucket_classes_max, (int)(lut16[b + 1] - lut16[b]));
     // class records in global memory: the full descriptors where the encoder's indexing kernel reads them (codes with their
     // tables in shared memory), the compact 32-byte records for the codes whose decoders read them from global memory
     std::vector<BigDesc> big;

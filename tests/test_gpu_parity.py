@@ -658,9 +658,9 @@ def test_sort_blocks_gemm_is_a_permutation_inside_every_domain(lib, ctxs, oracle
 
 
 def test_sort_blocks_gemm_72bit_entries(lib, ctxs, oracle_mod):
-    # 96-bit entries: the stored index unchanged, its class relative to the first class of its bucket (top 16 index bits),
-    # its position; a domain is ordered by the shape of the unranking (odd classes first, then by number of steps, most
-    # first); entries without a block come last
+    # 96-bit entries: the class-local index (bit 63 of its two words = no block), the class (17 bits) and the position; a
+    # domain is ordered by the shape of the unranking (odd classes first, then by number of steps, most first); entries
+    # without a block come last
     o = _oracle(oracle_mod)((2, 53))
     ctx = ctxs[(2, 53)]
     n_out, k_in = 200, 1000                                 # 2 row tiles, 42 blocks per row -> 6 domains per tile, ragged both ways
@@ -683,22 +683,21 @@ def test_sort_blocks_gemm_72bit_entries(lib, ctxs, oracle_mod):
         rt, d = divmod(dom, nd)
         positions, last_key, ended = set(), (-1, -99), False
         for w0, w1, w2 in e[dom].tolist():
-            pos = w2 >> 22
+            pos = w2 >> 17
             row, cb = rt * 128 + pos // 8, d * 8 + pos % 8
             assert pos not in positions
             positions.add(pos)
-            if (w2 & 0xff) == 0xff:
+            if w1 >> 31:
                 assert row >= n_out or cb >= bpr
                 ended = True                                # nothing with a block may follow
                 continue
             assert not ended
-            I = w0 | w1 << 32 | (w2 & 0xff) << 64
             b = row * bpr + cb
-            assert idx[b] == I and b not in seen
+            I = int(idx[b])
+            assert b not in seen
             seen.add(b)
             cls = bisect.bisect_right(offs, I) - 1
-            first_of_bucket = bisect.bisect_right(offs, (I >> 56) << 56) - 1
-            assert (w2 >> 8) & 0x3fff == cls - first_of_bucket
+            assert w2 & 0x1ffff == cls and (w0 | w1 << 32) == I - offs[cls]
             key = (1 - classes[cls]["parity"], -steps(classes[cls]))
             assert key >= last_key
             last_key = key
