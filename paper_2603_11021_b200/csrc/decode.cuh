@@ -103,6 +103,15 @@ __device__ __forceinline__ __nv_bfloat16 dequant(float gain, const Point& pt, in
     return __float2bfloat16_rn(gain * coord(pt, i));
 }
 
+// A 16-bit read-only load that stays where it is written among the other volatile statements (the decoders' table
+// reads): issued before a block is unranked, its result is first used when the weights are formed.
+__device__ __forceinline__ uint16_t ldg_u16_here(const uint16_t* p)
+{
+    uint16_t v;
+    asm volatile("ld.global.nc.u16 %0, [%1];" : "=h"(v) : "l"(p));
+    return v;
+}
+
 __device__ __forceinline__ float gain_to_float(uint16_t bits)
 {
     return __half2float(__ushort_as_half(bits));

@@ -671,7 +671,9 @@ gemm_pipe_kernel(FastArgs fa, const unsigned long long* __restrict__ sorted, con
                 }
                 const uint32_t r = pos >> 3, c = pos & 7u;
                 const int64_t row = rt * kGemmRows + r, cb = (int64_t)d * kDomBlocks + c;
-                float gn = (!kSg && valid) ? gain_to_float(__ldg(gain + row * ga.bpr + cb)) : 0.f;
+                uint16_t gbits = 0;
+                if (!kSg && valid) gbits = ldg_u16_here(gain + row * ga.bpr + cb);
+                float gn = 0.f;                                               // the gain is converted once the block is unranked
                 uint32_t w[12];
                 if (kBig) {
                     int cls = 0;
@@ -686,6 +688,7 @@ gemm_pipe_kernel(FastArgs fa, const unsigned long long* __restrict__ sorted, con
                         // rest of this iteration to arrive
                         big_load_record(fa.dc, (int)((uint32_t)(e_next.y >> 8) & 0xffffffu), !(e_next.y >> 63), rec0, rec1);
                     }
+                    gn = gain_to_float(gbits);
                     expand_bf16(dec.d, gn, w);
                     patch_id8_bf16(dec, gn, w);
                 } else {
@@ -699,6 +702,7 @@ gemm_pipe_kernel(FastArgs fa, const unsigned long long* __restrict__ sorted, con
                     } else {
                         cls = decode_sorted_entry(fa, T, I, valid, dec);
                     }
+                    if (!kSg) gn = gain_to_float(gbits);
                     if (kSg && valid) {
                         const float scale = sg.row_scale ? __ldg(sg.row_scale + row) : 1.f;
                         gn = __fmul_rn(__fmul_rn(scale, __ldg(sg.codebook + (uint32_t)(field >> fa.L.W))),

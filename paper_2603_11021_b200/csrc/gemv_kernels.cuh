@@ -411,9 +411,11 @@ __device__ __forceinline__ void gemv_sorted_body(const FastArgs& fa, const FastS
             const uint32_t rloc = (rg_off + q) * kGemvGroupRows + ((pos >> 2) & 7u);      // row inside the pass
             const uint32_t cb = kq * 4u + (pos & 3u);
             float gn = 0.f;
-            if (!kSg && valid) gn = gain_to_float(__ldg(gain + ((int64_t)rg0 * kGemvGroupRows + rloc) * bpr + cb));
+            uint16_t gbits = 0;
+            if (!kSg && valid) gbits = ldg_u16_here(gain + ((int64_t)rg0 * kGemvGroupRows + rloc) * bpr + cb);
             Decoded r;
             const uint32_t cls = decode_sorted_entry(fa, T, I, valid, r);
+            if (!kSg) gn = gain_to_float(gbits);
             if (kSg && valid) {
                 const float scale = sg.row_scale ? __ldg(sg.row_scale + (int64_t)rg0 * kGemvGroupRows + rloc) : 1.f;
                 gn = __fmul_rn(__fmul_rn(scale, __ldg(sg.codebook + (uint32_t)(field >> fa.L.W))),
@@ -574,9 +576,11 @@ gemv_sorted_overlap_kernel(FastArgs fa, const __grid_constant__ GemvMulti mm, in
             const uint32_t rloc = q * kGemvGroupRows + ((pos >> 2) & 7u);                 // row inside the CTA's share
             const uint32_t cb = kq * 4u + (pos & 3u);
             float gn = 0.f;
-            if (valid) gn = gain_to_float(__ldg(M.gain + ((int64_t)rg0 * kGemvGroupRows + rloc) * bpr + cb));
+            uint16_t gbits = 0;
+            if (valid) gbits = ldg_u16_here(M.gain + ((int64_t)rg0 * kGemvGroupRows + rloc) * bpr + cb);
             Decoded r;
             decode_sorted_entry(fa, T, I, valid, r);
+            gn = gain_to_float(gbits);
             uint32_t w[12];
             expand_bf16(r, gn, w);
             const uint4* xb = reinterpret_cast<const uint4*>(xs + cb * 12u);
@@ -745,16 +749,18 @@ __device__ __forceinline__ void gemv_bin_body(const FastArgs& fa, const FastSmem
             const uint32_t cb = kq * 4u + (pos & 3u);
             const uint32_t cls = valid ? (kSg ? cls16 & 1023u : cls16) : 0u;
             float gn = 0.f;
+            uint16_t gbits = 0;
             if (valid) {
                 if (kSg) {
                     const float scale = sg.row_scale ? __ldg(sg.row_scale + (int64_t)rg0 * kGemvGroupRows + rloc) : 1.f;
                     gn = __fmul_rn(__fmul_rn(scale, __ldg(sg.codebook + (cls16 >> 10))), __uint_as_float(T.desc[cls * kFastDescStride + kFastDescRnorm]));
                 } else {
-                    gn = gain_to_float(__ldg(gain_pass + (int64_t)rloc * bpr + cb));
+                    gbits = ldg_u16_here(gain_pass + (int64_t)rloc * bpr + cb);
                 }
             }
             Decoded r;
             decode_known_class(T, cls, e & ((1ull << 48) - 1ull), valid, r);
+            if (!kSg) gn = gain_to_float(gbits);
             uint32_t w[12];
             expand_bf16(r, gn, w);
             const uint4* xb = reinterpret_cast<const uint4*>(xs + cb * 12u);
