@@ -248,10 +248,11 @@ int llvq_gemm_small_batch(const llvq_ctx* ctx, const void* d_idx, const uint16_t
  * ROWWISE gains; all of App. A steps 1-4 run in the kernel.  llvq_sorted_gemm_bytes() gives the stream length (8 bytes
  * per block of the matrix padded to whole domains; 0 if unsupported: same codes as llvq_sort_blocks, plus the one below).
  * Codes whose class tables live in global memory (the 72-bit code, shells 2..53) take 96-bit entries, 12 bytes per
- * block: the stored index unchanged (72 bits), the number of its class relative to the first class of the index's
- * bucket in the table on the top 16 index bits (14 bits: App. A step 2 is then one table look-up in the kernel instead
- * of a bisection over 128-bit offsets; steps 1, 3, 4 run there as before) and the position in the domain (10 bits); the
- * order is by the shape of the unranking: parity (odd first), number of steps, which steps take at most three slots.
+ * block: the index as its two digits in the mixed radix of the class table, i.e. the class (17 bits) and the class-local
+ * index I - offset[class] (63 bits; bit 63 marks "no block"), and the position in the domain (10 bits).  App. A step 2
+ * (class look-up, a bisection over 128-bit offsets on the stored stream) is thus taken when the layout is made; steps 3-4
+ * (the unranking) run in the kernel as before.  The order is by the shape of the unranking: parity (odd first), number
+ * of steps, which steps take at most three slots.
  * Out-of-range indices are counted by llvq_sort_blocks_gemm and stored as "no block".
  * d_sorted: device, 16-byte aligned.  Other arguments and limits as in llvq_gemm_small_batch.
  */
