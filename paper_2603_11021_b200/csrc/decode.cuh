@@ -62,6 +62,28 @@ __device__ __forceinline__ uint64_t load_field(const uint32_t* __restrict__ stre
     return W < 64 ? v & ((1ull << W) - 1) : v;
 }
 
+// The same in two steps, for a caller that requests the words well before it needs the field: the words as they are
+// (x = words 0-1, y = word 2 | bit offset << 32), and the field from them.
+__device__ __forceinline__ ulonglong2 load_field_words(const uint32_t* __restrict__ stream, uint64_t b, int W)
+{
+    const uint64_t bp = b * (uint64_t)W;
+    const uint32_t* p = stream + (bp >> 5);
+    const int sh = (int)(bp & 31);
+    const int last = sh + W;
+    const uint32_t w0 = __ldg(p);
+    const uint32_t w1 = last > 32 ? __ldg(p + 1) : 0u;
+    const uint32_t w2 = last > 64 ? __ldg(p + 2) : 0u;
+    return make_ulonglong2(((unsigned long long)w1 << 32) | w0, (unsigned long long)w2 | (unsigned long long)sh << 32);
+}
+
+__device__ __forceinline__ uint64_t field_of_words(ulonglong2 w, int W)
+{
+    const int sh = (int)(w.y >> 32);
+    uint64_t v = w.x >> sh;
+    if (sh) v |= (w.y & 0xffffffffull) << (64 - sh);
+    return W < 64 ? v & ((1ull << W) - 1) : v;
+}
+
 // q = p / d, r = p % d with magic = floor((2^64 - 1) / d): the estimate is at most one too small.
 __device__ __forceinline__ void divmod_magic(uint64_t p, uint32_t d, uint64_t magic, uint64_t& q, uint32_t& r)
 {

@@ -32,6 +32,8 @@ struct GemmArgs {
     int64_t scratch_ld;        // row tiles * 128
     uint32_t* counters;        // [row tiles], zero on entry and on exit
     int y_f32;                 // Y holds binary32 instead of bf16 (the batch-1 product behind llvq_gemv_sorted of the 72-bit code)
+    const uint16_t* sort_rank; // stored stream ordered inside the kernel (gemm_sorted_kernel<.., kBin>): sort key of every class, else null
+    int nbins;                 // ... and the number of bins (a multiple of 32 above the largest key; the last bin is "no block")
 };
 
 __global__ void put_shard_kernel(YOut yo, YOut* dst)
@@ -336,10 +338,15 @@ sort_blocks_gemm_big_kernel(FastArgs fa, const uint32_t* __restrict__ stream, in
     }
 }
 
-template <bool kBig, bool kSg = false, bool kShard = false>
+// kBin: `sorted` points at the stored stream instead; at the start of an iteration every thread looks up the class of
+// one block per domain (S1-S2) and the CTA puts the 1024 fields of a domain into the order of the sorted layout with a
+// counting sort in shared memory (one bin per class), so that the unranking below runs on the same entries as with a
+// stream sorted at load time.  The fields of an iteration are requested one iteration ahead.
+template <bool kBig, bool kSg = false, bool kShard = false, bool kBin = false>
 __global__ void __launch_bounds__(kGemmThreads, 1)
 gemm_sorted_kernel(FastArgs fa, const unsigned long long* __restrict__ sorted, const uint16_t* __restrict__ gain, SgArgs sg, GemmArgs ga, int dpi)
 {
+    static_assert(!(kBin && kBig), "the in-kernel ordering is for the codes whose class tables sit in shared memory");
     extern __shared__ __align__(128) uint8_t smem[];
     const uint32_t img_bytes = fa.image_bytes;
     uint64_t* bar_img = reinterpret_cast<uint64_t*>(smem + img_bytes);
@@ -352,6 +359,11 @@ gemm_sorted_kernel(FastArgs fa, const unsigned long long* __restrict__ sorted, c
     uint8_t* a_buf = smem + a_off;                                        // [dpi * 2 stages] x 24576
     const uint32_t b_stage = (uint32_t)ga.npad * kStageK * 2;
     uint8_t* b_buf = a_buf + (uint32_t)dpi * kDomStages * kAStage;         // [dpi * 2 stages] x npad * 192
+    // kBin: per domain of the iteration the bins (then the next free slot of every bin), the warp totals of their prefix sum
+    // and the ordered entries
+    uint32_t* bin_hist = reinterpret_cast<uint32_t*>(b_buf + (uint32_t)dpi * kDomStages * b_stage);   // [dpi][nbins]
+    uint32_t* bin_wt = bin_hist + dpi * ga.nbins;                          // [dpi][32]
+    unsigned long long* bin_ent = reinterpret_cast<unsigned long long*>(bin_wt + dpi * 32);            // [dpi][1024]
 
     pdl_launch_dependents();
     const bool image_ok = fast_load_image(smem, fa.image, fa.image_bytes, bar_img, fa.flags);
@@ -362,6 +374,8 @@ gemm_sorted_kernel(FastArgs fa, const unsigned long long* __restrict__ sorted, c
     }
     const FastSmem T = fast_view(smem, fa.L);
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    if (kBin)
+        for (int i = threadIdx.x; i < dpi * ga.nbins; i += kGemmThreads) bin_hist[i] = 0u;
     if (threadIdx.x == 0) {
         mbar_init(bar_free, 1); mbar_init(bar_done, 1);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -387,6 +401,12 @@ gemm_sorted_kernel(FastArgs fa, const unsigned long long* __restrict__ sorted, c
         const ulonglong2 no_entry = make_ulonglong2(kSortIndexMask, kBigNoBlock);
         auto entry_at = [&](int d, int q) {
             if (d + q >= d_end) return no_entry;
+            if (kBin) {       // the stream words that hold the field of this thread's block of the domain (position = thread); y bit 63 = no block
+                const int64_t row = rt * kGemmRows + (threadIdx.x >> 3), cb = (int64_t)(d + q) * kDomBlocks + (threadIdx.x & 7u);
+                if (row < ga.n_out && cb < ga.bpr)
+                    return load_field_words(reinterpret_cast<const uint32_t*>(sorted), (uint64_t)(row * ga.bpr + cb), (int)fa.L.W + (kSg ? sg.bits : 0));
+                return no_entry;
+            }
             // warp 0 also issues the MMAs of every iteration: it takes the cheapest chunk of each domain (the last), the other
             // warps pair chunk w - 1 of the first domain with chunk 31 - w of the second
             const int chunk = warp == 0 ? 31 : (q == 0 ? warp - 1 : 31 - warp);
@@ -397,9 +417,65 @@ gemm_sorted_kernel(FastArgs fa, const unsigned long long* __restrict__ sorted, c
         ulonglong2 e0 = entry_at(d_begin, 0), e1 = dpi > 1 ? entry_at(d_begin, 1) : no_entry;
         for (int d0 = d_begin; d0 < d_end; d0 += dpi, ++uses) {
             const int nd_now = min(dpi, d_end - d0);
-            const ulonglong2 cur0 = e0, cur1 = e1;
+            ulonglong2 cur0 = e0, cur1 = e1;
             e0 = entry_at(d0 + dpi, 0);
             if (dpi > 1) e1 = entry_at(d0 + dpi, 1);
+            if (kBin) {
+                // ---- order the fields of each domain by the sort key of their class
+                const uint32_t nbins = (uint32_t)ga.nbins;
+                const int wbits = (int)fa.L.W + (kSg ? sg.bits : 0);
+                unsigned long long f[2] = {(cur0.y >> 63) ? kSortIndexMask : field_of_words(cur0, wbits),
+                                           (cur1.y >> 63) ? kSortIndexMask : field_of_words(cur1, wbits)};
+                uint32_t key[2] = {nbins - 1u, nbins - 1u}, cnt[2] = {0u, 0u}, incl[2] = {0u, 0u};
+#pragma unroll
+                for (int q = 0; q < 2; ++q) {
+                    if (q >= nd_now) break;
+                    if (f[q] != kSortIndexMask) {
+                        const uint64_t I = kSg ? f[q] & ((1ull << fa.L.W) - 1ull) : f[q];
+                        if (I < fa.n_points) {
+                            uint64_t local;
+                            key[q] = __ldg(ga.sort_rank + fast_find_class(T, I, local));
+                        } else {
+                            atomicAdd(fa.bad_index, 1ull);
+                            f[q] = kSortIndexMask;
+                        }
+                    }
+                    atomicAdd(&bin_hist[q * nbins + key[q]], 1u);
+                }
+                __syncthreads();
+#pragma unroll
+                for (int q = 0; q < 2; ++q) {
+                    if (q >= nd_now) break;
+                    cnt[q] = threadIdx.x < nbins ? bin_hist[q * nbins + threadIdx.x] : 0u;
+                    uint32_t v = cnt[q];
+#pragma unroll
+                    for (int o = 1; o < 32; o <<= 1) { const uint32_t t = __shfl_up_sync(kFullMask, v, o); if (lane >= o) v += t; }
+                    incl[q] = v;
+                    if (lane == 31) bin_wt[q * 32 + warp] = v;
+                }
+                __syncthreads();
+#pragma unroll
+                for (int q = 0; q < 2; ++q) {
+                    if (q >= nd_now) break;
+                    uint32_t v = bin_wt[q * 32 + lane];                    // every warp scans the 32 warp totals
+                    const uint32_t own = v;
+#pragma unroll
+                    for (int o = 1; o < 32; o <<= 1) { const uint32_t t = __shfl_up_sync(kFullMask, v, o); if (lane >= o) v += t; }
+                    const uint32_t before = __shfl_sync(kFullMask, v - own, warp);
+                    if (threadIdx.x < nbins) bin_hist[q * nbins + threadIdx.x] = before + incl[q] - cnt[q];
+                }
+                __syncthreads();
+#pragma unroll
+                for (int q = 0; q < 2; ++q) {
+                    if (q >= nd_now) break;
+                    const uint32_t slot = atomicAdd(&bin_hist[q * nbins + key[q]], 1u);
+                    bin_ent[q * kDomEntries + slot] = f[q] | (unsigned long long)threadIdx.x << 48;
+                }
+                __syncthreads();
+                for (int i = threadIdx.x; i < dpi * (int)nbins; i += kGemmThreads) bin_hist[i] = 0u;   // for the next iteration (a barrier follows below)
+                cur0 = make_ulonglong2(bin_ent[(warp == 0 ? 31 : warp - 1) * 32 + lane], 0ull);
+                if (nd_now > 1) cur1 = make_ulonglong2(bin_ent[kDomEntries + (warp == 0 ? 31 : 31 - warp) * 32 + lane], 0ull);
+            }
             // ---- A: every warp unranks one chunk of 32 sorted entries per domain
 #pragma unroll
             for (int q = 0; q < 2; ++q) {

@@ -273,6 +273,34 @@ def test_gemm_code_whose_tables_leave_no_room_for_two_buffer_sets(lib, oracle_mo
     _gemm_check(lib, ctx, _oracle(oracle_mod)((2, 16)), 300, 1000, batch, seed=9)
 
 
+@pytest.mark.parametrize("code", [(2, 13), (2, 53)])
+def test_products_on_a_stream_with_out_of_range_fields(lib, ctxs, oracle_mod, code):
+    # fields >= N decode to the zero block and are counted once per launch, whatever kernel serves the product
+    o = _oracle(oracle_mod)(code)
+    ctx = ctxs[code]
+    n_out, k_in = 300, 1000                                 # 42 blocks per row: ragged domains and units
+    stream, gain, nblocks = gen.make_layer(o.N, o.W, n_out, k_in, 1, seed=27)
+    idx = o.unpack(stream, nblocks)
+    for b in (0, 41, 42 * 128 + 5, 42 * 200 + 17, nblocks - 1):
+        idx[b] = o.N + b                                     # still below 2^W
+    lo, hi = gen.indices_to_arrays(idx)
+    stream = gen.pack_indices(lo, hi, o.W)
+    d_idx, d_gain = to_dev_u8(stream), to_dev_f16(gain)
+    x = gen.normal_bf16(k_in, seed=27)
+    y = lib.llvq_gemv(ctx, d_idx, d_gain, n_out, k_in, to_dev_bf16(x))
+    torch.cuda.synchronize()
+    assert lib.llvq_last_error(ctx) == (5, 0)
+    assert gemv_error(y.cpu().numpy(), o.gemv(stream, gain, n_out, k_in, x)) <= TOL
+    for batch in (16, 64):
+        X = gen.normal_bf16((batch, k_in), seed=batch)
+        want = o.gemm(stream, gain, n_out, k_in, X, threads=8)
+        Y = lib.llvq_gemm_small_batch(ctx, d_idx, d_gain, n_out, k_in, to_dev_bf16(X))
+        torch.cuda.synchronize()
+        assert lib.llvq_last_error(ctx) == (5, 0)
+        err = np.abs(Y.float().cpu().numpy() - want) / np.maximum(np.abs(want), 1e-3 * np.abs(want).max())
+        assert err.max() <= TOL_BF16_OUT
+
+
 def test_gemm_exact_integer_case(lib, ctxs, oracle_mod):
     # gains = 1, X = 0/1 patterns: every partial sum is a small integer, exact in binary32 and in bf16
     o = _oracle(oracle_mod)((2, 13))
