@@ -116,10 +116,11 @@ int launch_gemm(const llvq_ctx* ctx, const void* d_idx, const uint16_t* d_gain_f
     if (smem > 227 * 1024) return LLVQ_EUNSUPPORTED;
     const uint32_t* idx = static_cast<const uint32_t*>(d_idx);
     if (yo && sg) return LLVQ_EUNSUPPORTED;              // row-sharded: stored-gain form only
-    // codes with their class tables in shared memory and many classes (a warp of 32 unrelated blocks is what costs there):
-    // the kernel that puts every domain of 1024 blocks into the order of the sorted layout before unranking it
+    // codes with their class tables in shared memory and many classes (a warp of 32 unrelated blocks is what costs there),
+    // padded batch up to 32 (two domains per iteration fit; with one, the barriers of the ordering cost what it gains:
+    // measured): the kernel that puts every domain of 1024 blocks into the order of the sorted layout before unranking it
     const int ncls = (int)ctx->host.desc.size();
-    if (ctx->fast && ctx->d_sort_rank && ncls >= 64 && ncls < 1024 && ctx->host.W + (sg ? sg->bits : 0) <= 48) {
+    if (ctx->fast && ctx->d_sort_rank && ncls >= 64 && ncls < 1024 && ctx->host.W + (sg ? sg->bits : 0) <= 48 && ga.npad <= 32) {
         const size_t head = (img + 64 + 1023) & ~size_t(1023), a_set = (size_t)kDomStages * kGemmRows * kStageK * 2,
                      x_set = (size_t)kDomStages * ga.npad * kStageK * 2;
         GemmArgs gb = ga;
@@ -128,8 +129,7 @@ int launch_gemm(const llvq_ctx* ctx, const void* d_idx, const uint16_t* d_gain_f
         gb.sort_rank = ctx->d_sort_rank;
         gb.nbins = (ncls + 1 + 31) / 32 * 32;                                    // one bin per class and one for "no block"
         const size_t bins = (size_t)gb.nbins * 4 + 32 * 4 + (size_t)kDomEntries * 8;   // per domain of an iteration
-        int dpi = ga.npad <= 32 ? 2 : 1;
-        if (head + (size_t)dpi * (a_set + x_set + bins) > 227 * 1024) dpi = 1;
+        const int dpi = 2;
         const size_t smem_bin = head + (size_t)dpi * (a_set + x_set + bins);
         if (smem_bin <= 227 * 1024) {
             const unsigned grid_bin = (unsigned)std::min<int64_t>(row_tiles * gb.nstages, ctx->sm_count);

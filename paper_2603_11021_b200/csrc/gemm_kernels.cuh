@@ -359,9 +359,9 @@ gemm_sorted_kernel(FastArgs fa, const unsigned long long* __restrict__ sorted, c
     uint8_t* a_buf = smem + a_off;                                        // [dpi * 2 stages] x 24576
     const uint32_t b_stage = (uint32_t)ga.npad * kStageK * 2;
     uint8_t* b_buf = a_buf + (uint32_t)dpi * kDomStages * kAStage;         // [dpi * 2 stages] x npad * 192
-    // kBin: per domain of the iteration the bins (then the next free slot of every bin), the warp totals of their prefix sum
+    // kBin: per domain of the iteration the bins (block counts, then the first slot of every bin), the warp totals of their prefix sum
     // and the ordered entries
-    uint32_t* bin_hist = reinterpret_cast<uint32_t*>(b_buf + (uint32_t)dpi * kDomStages * b_stage);   // [dpi][nbins]
+    uint32_t* bin_hist = reinterpret_cast<uint32_t*>(b_buf + (uint32_t)dpi * kDomStages * b_stage);   // [dpi][nbins] counts, then first slots
     uint32_t* bin_wt = bin_hist + dpi * ga.nbins;                          // [dpi][32]
     unsigned long long* bin_ent = reinterpret_cast<unsigned long long*>(bin_wt + dpi * 32);            // [dpi][1024]
 
@@ -426,7 +426,7 @@ gemm_sorted_kernel(FastArgs fa, const unsigned long long* __restrict__ sorted, c
                 const int wbits = (int)fa.L.W + (kSg ? sg.bits : 0);
                 unsigned long long f[2] = {(cur0.y >> 63) ? kSortIndexMask : field_of_words(cur0, wbits),
                                            (cur1.y >> 63) ? kSortIndexMask : field_of_words(cur1, wbits)};
-                uint32_t key[2] = {nbins - 1u, nbins - 1u}, cnt[2] = {0u, 0u}, incl[2] = {0u, 0u};
+                uint32_t key[2] = {nbins - 1u, nbins - 1u}, rank[2] = {0u, 0u}, cnt[2] = {0u, 0u}, incl[2] = {0u, 0u};
 #pragma unroll
                 for (int q = 0; q < 2; ++q) {
                     if (q >= nd_now) break;
@@ -440,7 +440,7 @@ gemm_sorted_kernel(FastArgs fa, const unsigned long long* __restrict__ sorted, c
                             f[q] = kSortIndexMask;
                         }
                     }
-                    atomicAdd(&bin_hist[q * nbins + key[q]], 1u);
+                    rank[q] = atomicAdd(&bin_hist[q * nbins + key[q]], 1u);     // its place among the blocks of its bin
                 }
                 __syncthreads();
 #pragma unroll
@@ -468,7 +468,7 @@ gemm_sorted_kernel(FastArgs fa, const unsigned long long* __restrict__ sorted, c
 #pragma unroll
                 for (int q = 0; q < 2; ++q) {
                     if (q >= nd_now) break;
-                    const uint32_t slot = atomicAdd(&bin_hist[q * nbins + key[q]], 1u);
+                    const uint32_t slot = bin_hist[q * nbins + key[q]] + rank[q];
                     bin_ent[q * kDomEntries + slot] = f[q] | (unsigned long long)threadIdx.x << 48;
                 }
                 __syncthreads();
@@ -487,17 +487,21 @@ gemm_sorted_kernel(FastArgs fa, const unsigned long long* __restrict__ sorted, c
                 const bool valid = kBig ? !(e.y >> 63) : (field != kSortIndexMask && I < fa.n_points);
                 const uint32_t r = pos >> 3, c = pos & 7u;
                 const int64_t row = rt * kGemmRows + r, cb = (int64_t)(d0 + q) * kDomBlocks + c;
-                float gn = (!kSg && valid) ? gain_to_float(__ldg(gain + row * ga.bpr + cb)) : 0.f;
+                uint16_t gbits = 0;
+                if (!kSg && valid) gbits = ldg_u16_here(gain + row * ga.bpr + cb);
+                float gn = 0.f;                                               // the gain is converted once the block is unranked
                 uint32_t w[12];
                 if (kBig) {
                     const int cls = valid ? (int)((uint32_t)(e.y >> 8) & 0xffffffu) : 0;
                     DecodedBig dec{};
                     big_decode_planes(T, fa.dc, cls, valid ? e.x : 0ull, valid, kFullMask, dec);
+                    gn = gain_to_float(gbits);
                     expand_bf16(dec.d, gn, w);
                     patch_id8_bf16(dec, gn, w);
                 } else {
                     Decoded dec{};
                     const uint32_t cls = decode_sorted_entry(fa, T, I, valid, dec);
+                    if (!kSg) gn = gain_to_float(gbits);
                     if (kSg && valid) {
                         const float scale = sg.row_scale ? __ldg(sg.row_scale + row) : 1.f;
                         gn = __fmul_rn(__fmul_rn(scale, __ldg(sg.codebook + (uint32_t)(field >> fa.L.W))),
