@@ -267,9 +267,10 @@ __device__ __forceinline__ void fast_decode_local(const FastSmem& T, uint32_t cl
             else if (kPar == 1 && l == 1 && __all_sync(mask, k == 0u || nfree >= 22u)) a = deposit_two_holes(rel, freem);
             else a = deposit24(T.pd6, rel, freem);
             freem ^= a;
-            if ((l + 2) & 1) p0 |= a;                                   // the value id of level l is 2 + l
-            if ((l + 2) & 2) p1 |= a;
-            if ((l + 2) & 4) p2 |= a;
+            constexpr int kId0 = kPar == 1 ? 1 : 2;                     // the value id of level l is 2 + l (odd classes alone: 1 + l)
+            if ((l + kId0) & 1) p0 |= a;
+            if ((l + kId0) & 2) p1 |= a;
+            if ((l + kId0) & 4) p2 |= a;
             if (kPar != 0 && (word & (1u << 30))) bit1 |= a;
             if (kPar != 1 && in_group0 && (word >> 31)) nz0 |= a;
         }
@@ -295,7 +296,12 @@ __device__ __forceinline__ void fast_decode_local(const FastSmem& T, uint32_t cl
     }
     if (valid) {
         d.p0 = p0; d.p1 = p1; d.p2 = p2; d.neg = neg;
-        d.vals_lo = v.x; d.vals_hi = v.y;
+        if (kPar == 1) {
+            const uint2 vo = *reinterpret_cast<const uint2*>(T.desc + cls * kFastDescStride + kFastDescValsOdd);
+            d.vals_lo = vo.x; d.vals_hi = vo.y;
+        } else {
+            d.vals_lo = v.x; d.vals_hi = v.y;
+        }
     }
 }
 

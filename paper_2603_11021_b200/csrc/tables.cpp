@@ -330,6 +330,12 @@ bool build_fast_image(const HostTables& t, FastLayout& L, std::vector<uint8_t>& 
             else w[11 + l] = 0xffffffffu;                       // step beside lanes with more steps needs no special case
         }
         std::memcpy(&w[4], vals, 8);
+        // odd classes have no group 1: numbered without the gap at id 1, a class of four distinct values stays within ids 0..3
+        // (two bit planes) for the decoder form that handles odd classes alone
+        uint8_t vals_odd[8] = {d.fill0, 0, 0, 0, 0, 0, 0, 0};
+        if (d.parity)
+            for (int l = 0; l < nlev; ++l) vals_odd[1 + l] = d.lev[l].val;
+        std::memcpy(&w[kFastDescValsOdd], vals_odd, 8);
         w[15] = nbytes;
         const float rnorm = (float)(1.0 / std::sqrt(16.0 * (double)d.m));
         std::memcpy(&w[kFastDescRnorm], &rnorm, 4);

@@ -96,7 +96,8 @@ bool build_tables(int m_lo, int m_hi, HostTables& out);
 namespace llvq {
 
 constexpr int kFastMaxLevels = 4;      // unranking steps per class on the fast path
-constexpr int kFastDescWords = 18;     // words of a class descriptor that carry data
+constexpr int kFastDescWords = 20;     // words of a class descriptor that carry data
+constexpr int kFastDescValsOdd = 18;   // words 18, 19: absolute value of id 0..7 in the numbering of the odd-only decoder form
 constexpr int kFastDescRnorm = 16;     // word holding 1 / sqrt(16 m) as binary32
 constexpr int kFastDescMagic0 = 17;    // word holding floor(2^32 / radix) of level 0 (used when the arrangement rank fits 32 bits)
 constexpr uint32_t kFastFlagRank32 = 32u;   // descriptor flag: the class has fewer than 2^32 arrangements
@@ -140,6 +141,8 @@ struct FastLayout {
 //  15: n (free slots before the step) of levels 0..3, one byte each
 //  16: binary32 bits of 1 / |x| = 1 / sqrt(16 m) (formed in binary64, rounded once), for the shape-gain form
 //  17: floor(2^32 / radix) of level 0
+//  18,19: odd classes: absolute value of id 0..7 with id 0 = fill0 and ids 1.. = levels in order (the form that decodes odd
+//         classes alone numbers the levels from 1: there is no group 1 whose filler would take id 1)
 // with_classes = false builds only the class-independent tables (Golay, Pascal, subsets, deposit): codes whose class
 // tables do not fit shared memory keep those in global memory.
 bool build_fast_image(const HostTables& t, FastLayout& layout, std::vector<uint8_t>& image, bool with_classes = true);
