@@ -94,7 +94,6 @@ __device__ __forceinline__ void finish_pass(const YOut& yo, int64_t rg0, int64_t
         if (whole) {
             if (mine) {
                 store_y<kOutBf16, kShard>(yo, row, part);
-                if (kShard) __threadfence_system();
             }
             continue;
         }
@@ -109,7 +108,6 @@ __device__ __forceinline__ void finish_pass(const YOut& yo, int64_t rg0, int64_t
                 if (seen != 0ull) {
                     store_y<kOutBf16, kShard>(yo, row, __fadd_rn(__uint_as_float((uint32_t)seen), part));
                     __stcg(slot, 0ull);
-                    if (kShard) __threadfence_system();
                 }
             }
             continue;
@@ -128,7 +126,6 @@ __device__ __forceinline__ void finish_pass(const YOut& yo, int64_t rg0, int64_t
             if (mine) {
                 store_y<kOutBf16, kShard>(yo, row, __ldcg(scratch + slot0 + row));
                 __stcg(scratch + slot0 + row, 0.f);
-                if (kShard) __threadfence_system();
             }
             if (lane == 0) counters[slot0 / kGemvGroupRows + rg] = 0u;
         }
@@ -136,8 +133,9 @@ __device__ __forceinline__ void finish_pass(const YOut& yo, int64_t rg0, int64_t
 }
 
 // Last step of a row-sharded GEMV CTA (all threads call it, after their last store to y): counts the CTA in; the CTA
-// that completes the grid raises the epoch in every peer's flag word.  The remote stores of y are fenced at system
-// scope by the threads that made them (finish_pass) and once more, cumulatively, by the thread that counts.
+// that completes the grid raises the epoch in every peer's flag word.  The remote stores of y are plain stores; the block
+// barrier below orders them before the system-scope fence of the thread that counts the CTA in, which makes them visible,
+// cumulatively, before the flag (the usual barrier + fence + flag pattern: no fence per storing lane).
 __device__ __forceinline__ void shard_arrive(const YOut& yo)
 {
     if (yo.n_flag == 0) return;
@@ -146,10 +144,12 @@ __device__ __forceinline__ void shard_arrive(const YOut& yo)
     __threadfence_system();
     if (atomicAdd(yo.done, 1u) != gridDim.x - 1u) return;
     atomicExch(yo.done, 0u);
+    // one system-scope fence releases everything before it for all the flag words: the stores themselves are relaxed (a
+    // release store per word would pay the fence once per peer: measured 2 us each)
     __threadfence_system();
 #pragma unroll
     for (int p = 0; p < kMaxShardPeers; ++p)
-        if (p < yo.n_flag) asm volatile("st.release.sys.global.u32 [%0], %1;" ::"l"(yo.flag[p]), "r"(yo.epoch) : "memory");
+        if (p < yo.n_flag) asm volatile("st.relaxed.sys.global.u32 [%0], %1;" ::"l"(yo.flag[p]), "r"(yo.epoch) : "memory");
 }
 
 // sum_j w_j x_j over 12 packed bf16 pairs with binary32 accumulation: fma.rn.f32.bf16 takes the bf16 halves as they are
