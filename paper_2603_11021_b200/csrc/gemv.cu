@@ -57,7 +57,8 @@ int gemv_common(const llvq_ctx* ctx, const void* d_idx, const uint16_t* d_gain_f
     const int64_t nq = (bpr + 3) / 4;
     const size_t kSmemMax = 227 * 1024;
     const size_t rest = 16 + (size_t)nq * 48 * 4 + kGemvGroupsPerPass * kGemvGroupRows * 4 + 16;
-    const bool ext_direct = ctx->fl.total_ext + rest <= kSmemMax;      // room for the table of small subsets
+    // room for the table of small subsets (not for the 72-bit code: its warps hold 32 unrelated classes that almost never take it together)
+    const bool ext_direct = ctx->fast && ctx->fl.total_ext + rest <= kSmemMax;
     const size_t smem = (ext_direct ? ctx->fl.total_ext : ctx->fl.total) + rest;
     if (smem > kSmemMax || n_out > 64ll * kMaxScratchRows) return LLVQ_EUNSUPPORTED;
     const int64_t units = ((n_out + kGemvGroupRows - 1) / kGemvGroupRows) * nq;

@@ -253,17 +253,19 @@ int llvq_decode_blocks(const llvq_ctx* ctx, const void* d_idx, uint64_t nblocks,
     if (nblocks > (1ull << 40)) return LLVQ_EUNSUPPORTED;
     DeviceGuard guard(ctx->device);
     if (!guard.ok) return LLVQ_ECUDA;
-    const size_t smem = ctx->fl.total_ext + 16;
+    // a warp of these kernels holds 32 unrelated classes: the table of small subsets (FastLayout::sub3) would almost never be taken
+    // by all lanes of a step, and asking whether it can be costs more than it returns (measured), so the image goes without it
+    const size_t smem = ctx->fl.total + 16;
     const uint64_t tiles = (nblocks + kFastThreads - 1) / kFastThreads;
     const unsigned g = (unsigned)std::min<uint64_t>(tiles, (uint64_t)ctx->sm_count);
     const uint32_t* idx = static_cast<const uint32_t*>(d_idx);
     if (ctx->fast) {
         if (!set_smem(decode_blocks_fast_kernel<false>, smem)) return LLVQ_ECUDA;
-        if (launch_pdl(decode_blocks_fast_kernel<false>, g, (unsigned)kFastThreads, smem, (cudaStream_t)stream, fast_args(ctx, true), idx, nblocks,
+        if (launch_pdl(decode_blocks_fast_kernel<false>, g, (unsigned)kFastThreads, smem, (cudaStream_t)stream, fast_args(ctx, false), idx, nblocks,
                        reinterpret_cast<uint2*>(d_points)) != cudaSuccess) return LLVQ_ECUDA;
     } else {
         if (!set_smem(decode_blocks_fast_kernel<true>, smem)) return LLVQ_ECUDA;
-        if (launch_pdl(decode_blocks_fast_kernel<true>, g, (unsigned)kFastThreads, smem, (cudaStream_t)stream, fast_args(ctx, true), idx, nblocks,
+        if (launch_pdl(decode_blocks_fast_kernel<true>, g, (unsigned)kFastThreads, smem, (cudaStream_t)stream, fast_args(ctx, false), idx, nblocks,
                        reinterpret_cast<uint2*>(d_points)) != cudaSuccess) return LLVQ_ECUDA;
     }
     return launch_status();
@@ -285,18 +287,19 @@ int llvq_dequant_matrix(const llvq_ctx* ctx, const void* d_idx, const uint16_t* 
     if (layout == LLVQ_LAYOUT_FLAT && ld != cols) return LLVQ_EINVAL;
     const int64_t bpr = layout == LLVQ_LAYOUT_FLAT ? 0 : (cols + 23) / 24;
     const uint64_t nblocks = layout == LLVQ_LAYOUT_FLAT ? ((uint64_t)rows * (uint64_t)cols + 23) / 24 : (uint64_t)rows * (uint64_t)bpr;
-    const size_t smem = ctx->fl.total_ext + 16;
+    // (image without the table of small subsets, as in llvq_decode_blocks)
+    const size_t smem = ctx->fl.total + 16;
     const uint64_t tiles = (nblocks + kFastThreads - 1) / kFastThreads;
     const unsigned g = (unsigned)std::min<uint64_t>(tiles, (uint64_t)ctx->sm_count);
     const uint32_t* idx = static_cast<const uint32_t*>(d_idx);
     __nv_bfloat16* w = reinterpret_cast<__nv_bfloat16*>(d_w_bf16);
     if (ctx->fast) {
         if (!set_smem(dequant_fast_kernel<false>, smem)) return LLVQ_ECUDA;
-        if (launch_pdl(dequant_fast_kernel<false, false>, g, (unsigned)kFastThreads, smem, st, fast_args(ctx, true), idx, d_gain_f16, SgArgs{}, (uint64_t)nblocks,
+        if (launch_pdl(dequant_fast_kernel<false, false>, g, (unsigned)kFastThreads, smem, st, fast_args(ctx, false), idx, d_gain_f16, SgArgs{}, (uint64_t)nblocks,
                        rows, cols, bpr, w, ld) != cudaSuccess) return LLVQ_ECUDA;
     } else {
         if (!set_smem(dequant_fast_kernel<true>, smem)) return LLVQ_ECUDA;
-        if (launch_pdl(dequant_fast_kernel<true, false>, g, (unsigned)kFastThreads, smem, st, fast_args(ctx, true), idx, d_gain_f16, SgArgs{}, (uint64_t)nblocks,
+        if (launch_pdl(dequant_fast_kernel<true, false>, g, (unsigned)kFastThreads, smem, st, fast_args(ctx, false), idx, d_gain_f16, SgArgs{}, (uint64_t)nblocks,
                        rows, cols, bpr, w, ld) != cudaSuccess) return LLVQ_ECUDA;
     }
     return launch_status();
@@ -321,12 +324,13 @@ int llvq_dequant_matrix_sg(const llvq_ctx* ctx, const void* d_fields, int gain_b
     if (!guard.ok) return LLVQ_ECUDA;
     const int64_t bpr = (cols + 23) / 24;
     const uint64_t nblocks = (uint64_t)rows * (uint64_t)bpr;
-    const size_t smem = ctx->fl.total_ext + 16;
+    // (image without the table of small subsets, as in llvq_decode_blocks)
+    const size_t smem = ctx->fl.total + 16;
     const uint64_t tiles = (nblocks + kFastThreads - 1) / kFastThreads;
     const unsigned g = (unsigned)std::min<uint64_t>(tiles, (uint64_t)ctx->sm_count);
     if (!set_smem(dequant_fast_kernel<false, true>, smem)) return LLVQ_ECUDA;
     dequant_fast_kernel<false, true><<<g, kFastThreads, smem, (cudaStream_t)stream>>>(
-        fast_args(ctx, true), static_cast<const uint32_t*>(d_fields), nullptr, SgArgs{d_codebook_f32, d_row_scale_f32, gain_bits},
+        fast_args(ctx, false), static_cast<const uint32_t*>(d_fields), nullptr, SgArgs{d_codebook_f32, d_row_scale_f32, gain_bits},
         nblocks, rows, cols, bpr, reinterpret_cast<__nv_bfloat16*>(d_w_bf16), ld);
     return launch_status();
 }
