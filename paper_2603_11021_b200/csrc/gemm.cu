@@ -29,7 +29,7 @@ int launch_gemm_domains(const llvq_ctx* ctx, const void* p, const uint16_t* d_ga
     DeviceGuard guard(ctx->device);
     if (!guard.ok) return LLVQ_ECUDA;
     GemmArgs ga;
-    ga.y = d_y_bf16; ga.y_ld = n_out; ga.shard = nullptr; ga.y_f32 = y_f32; ga.sort_rank = nullptr; ga.nbins = 0;
+    ga.y = d_y_bf16; ga.y_ld = n_out; ga.shard = nullptr; ga.y_f32 = y_f32; ga.sort_rank = nullptr; ga.nbins = 0; ga.bin_round = 0;
     if (yo) {                                             // the description travels ahead of the kernel on the same stream
         ga.y = static_cast<uint16_t*>(yo->y); ga.y_ld = y_ld; ga.shard = static_cast<const YOut*>(ctx->d_shard);
         put_shard_kernel<<<1, 32, 0, (cudaStream_t)stream>>>(*yo, static_cast<YOut*>(ctx->d_shard));   // by value: safe under stream capture
@@ -90,7 +90,7 @@ int launch_gemm(const llvq_ctx* ctx, const void* d_idx, const uint16_t* d_gain_f
     cudaStream_t st = (cudaStream_t)stream;
     if (k_in == 0) return cudaMemsetAsync(d_y_bf16, 0, (size_t)n_out * batch * 2, st) == cudaSuccess ? LLVQ_OK : LLVQ_ECUDA;
     GemmArgs ga;
-    ga.y = d_y_bf16; ga.y_ld = n_out; ga.shard = nullptr; ga.y_f32 = 0; ga.sort_rank = nullptr; ga.nbins = 0;
+    ga.y = d_y_bf16; ga.y_ld = n_out; ga.shard = nullptr; ga.y_f32 = 0; ga.sort_rank = nullptr; ga.nbins = 0; ga.bin_round = 0;
     if (yo) {                                             // the description travels ahead of the kernel on the same stream
         ga.y = static_cast<uint16_t*>(yo->y); ga.y_ld = y_ld; ga.shard = static_cast<const YOut*>(ctx->d_shard);
         put_shard_kernel<<<1, 32, 0, (cudaStream_t)stream>>>(*yo, static_cast<YOut*>(ctx->d_shard));   // by value: safe under stream capture
@@ -116,11 +116,11 @@ int launch_gemm(const llvq_ctx* ctx, const void* d_idx, const uint16_t* d_gain_f
     if (smem > 227 * 1024) return LLVQ_EUNSUPPORTED;
     const uint32_t* idx = static_cast<const uint32_t*>(d_idx);
     if (yo && sg) return LLVQ_EUNSUPPORTED;              // row-sharded: stored-gain form only
-    // codes with their class tables in shared memory and many classes (a warp of 32 unrelated blocks is what costs there),
-    // padded batch up to 32 (two domains per iteration fit; with one, the barriers of the ordering cost what it gains:
-    // measured): the kernel that puts every domain of 1024 blocks into the order of the sorted layout before unranking it
+    // codes with their class tables in shared memory and many classes (a warp of 32 unrelated blocks is what costs there):
+    // the kernel that puts every domain of 1024 blocks into the order of the sorted layout before unranking it, as many
+    // domains at a time (up to 4) as shared memory has room for beside the operand buffers
     const int ncls = (int)ctx->host.desc.size();
-    if (ctx->fast && ctx->d_sort_rank && ncls >= 64 && ncls < 1024 && ctx->host.W + (sg ? sg->bits : 0) <= 48 && ga.npad <= 32) {
+    if (ctx->fast && ctx->d_sort_rank && ncls >= 64 && ncls < 1024 && ctx->host.W + (sg ? sg->bits : 0) <= 48) {
         const size_t head = (img + 64 + 1023) & ~size_t(1023), a_set = (size_t)kDomStages * kGemmRows * kStageK * 2,
                      x_set = (size_t)kDomStages * ga.npad * kStageK * 2;
         GemmArgs gb = ga;
@@ -128,22 +128,30 @@ int launch_gemm(const llvq_ctx* ctx, const void* d_idx, const uint16_t* d_gain_f
         gb.split = 1;
         gb.sort_rank = ctx->d_sort_rank;
         gb.nbins = (ncls + 1 + 31) / 32 * 32;                                    // one bin per class and one for "no block"
-        const size_t bins = (size_t)gb.nbins * 4 + 32 * 4 + (size_t)kDomEntries * 8;   // per domain of an iteration
-        const int dpi = 2;
-        const size_t smem_bin = head + (size_t)dpi * (a_set + x_set + bins);
+        const size_t bins = (size_t)gb.nbins * 4 + 32 * 4 + (size_t)kDomEntries * 8;   // per ordered domain
+        const int dpi = ga.npad <= 32 ? 2 : 1;
+        gb.bin_round = 4;
+        while (gb.bin_round > dpi && head + (size_t)dpi * (a_set + x_set) + (size_t)gb.bin_round * bins > 227 * 1024) gb.bin_round -= dpi;
+        const size_t smem_bin = head + (size_t)dpi * (a_set + x_set) + (size_t)gb.bin_round * bins;
         if (smem_bin <= 227 * 1024) {
             const unsigned grid_bin = (unsigned)std::min<int64_t>(row_tiles * gb.nstages, ctx->sm_count);
             const unsigned long long* words = static_cast<const unsigned long long*>(d_idx);
             const SgArgs sga = sg ? *sg : SgArgs{};
-#define LLVQ_LAUNCH_BINNED(SG, SH)                                                                                              \
+#define LLVQ_LAUNCH_BINNED(SG, SH, RD)                                                                                          \
     do {                                                                                                                        \
-        if (!set_smem(gemm_sorted_kernel<false, SG, SH, true>, smem_bin)) return LLVQ_ECUDA;                                     \
-        if (launch_pdl(gemm_sorted_kernel<false, SG, SH, true>, grid_bin, (unsigned)kGemmThreads, smem_bin, st, fast_args(ctx, false), words, \
+        if (!set_smem(gemm_sorted_kernel<false, SG, SH, true, RD>, smem_bin)) return LLVQ_ECUDA;                                 \
+        if (launch_pdl(gemm_sorted_kernel<false, SG, SH, true, RD>, grid_bin, (unsigned)kGemmThreads, smem_bin, st, fast_args(ctx, false), words, \
                        d_gain_f16, sga, gb, dpi) != cudaSuccess) return LLVQ_ECUDA;                                             \
     } while (0)
-            if (yo) LLVQ_LAUNCH_BINNED(false, true);
-            else if (sg) LLVQ_LAUNCH_BINNED(true, false);
-            else LLVQ_LAUNCH_BINNED(false, false);
+            if (gb.bin_round > dpi) {                    // rounds of several iterations
+                if (yo) LLVQ_LAUNCH_BINNED(false, true, true);
+                else if (sg) LLVQ_LAUNCH_BINNED(true, false, true);
+                else LLVQ_LAUNCH_BINNED(false, false, true);
+            } else {
+                if (yo) LLVQ_LAUNCH_BINNED(false, true, false);
+                else if (sg) LLVQ_LAUNCH_BINNED(true, false, false);
+                else LLVQ_LAUNCH_BINNED(false, false, false);
+            }
 #undef LLVQ_LAUNCH_BINNED
             return launch_status();
         }

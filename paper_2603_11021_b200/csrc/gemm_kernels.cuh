@@ -34,6 +34,7 @@ struct GemmArgs {
     int y_f32;                 // Y holds binary32 instead of bf16 (the batch-1 product behind llvq_gemv_sorted of the 72-bit code)
     const uint16_t* sort_rank; // stored stream ordered inside the kernel (gemm_sorted_kernel<.., kBin>): sort key of every class, else null
     int nbins;                 // ... and the number of bins (a multiple of 32 above the largest key; the last bin is "no block")
+    int bin_round;             // ... and how many domains are ordered at a time (a multiple of the domains per iteration, at most 4)
 };
 
 __global__ void put_shard_kernel(YOut yo, YOut* dst)
@@ -341,8 +342,10 @@ sort_blocks_gemm_big_kernel(FastArgs fa, const uint32_t* __restrict__ stream, in
 // kBin: `sorted` points at the stored stream instead; at the start of an iteration every thread looks up the class of
 // one block per domain (S1-S2) and the CTA puts the 1024 fields of a domain into the order of the sorted layout with a
 // counting sort in shared memory (one bin per class), so that the unranking below runs on the same entries as with a
-// stream sorted at load time.  The fields of an iteration are requested one iteration ahead.
-template <bool kBig, bool kSg = false, bool kShard = false, bool kBin = false>
+// stream sorted at load time.  ga.bin_round domains are ordered at a time (their four block barriers are then paid once per
+// round, not once per iteration); the stream words of the next round are requested in L2 a round ahead.
+// kRound (with kBin): a round is longer than an iteration; else it is one iteration and the words come through registers.
+template <bool kBig, bool kSg = false, bool kShard = false, bool kBin = false, bool kRound = false>
 __global__ void __launch_bounds__(kGemmThreads, 1)
 gemm_sorted_kernel(FastArgs fa, const unsigned long long* __restrict__ sorted, const uint16_t* __restrict__ gain, SgArgs sg, GemmArgs ga, int dpi)
 {
@@ -361,9 +364,11 @@ gemm_sorted_kernel(FastArgs fa, const unsigned long long* __restrict__ sorted, c
     uint8_t* b_buf = a_buf + (uint32_t)dpi * kDomStages * kAStage;         // [dpi * 2 stages] x npad * 192
     // kBin: per domain of the iteration the bins (block counts, then the first slot of every bin), the warp totals of their prefix sum
     // and the ordered entries
-    uint32_t* bin_hist = reinterpret_cast<uint32_t*>(b_buf + (uint32_t)dpi * kDomStages * b_stage);   // [dpi][nbins] counts, then first slots
-    uint32_t* bin_wt = bin_hist + dpi * ga.nbins;                          // [dpi][32]
-    unsigned long long* bin_ent = reinterpret_cast<unsigned long long*>(bin_wt + dpi * 32);            // [dpi][1024]
+    constexpr int kMaxRound = kRound ? 4 : 2;
+    const int nround = kBin ? ga.bin_round : 1;
+    uint32_t* bin_hist = reinterpret_cast<uint32_t*>(b_buf + (uint32_t)dpi * kDomStages * b_stage);   // [nround][nbins] counts, then first slots
+    uint32_t* bin_wt = bin_hist + nround * ga.nbins;                        // [nround][32]
+    unsigned long long* bin_ent = reinterpret_cast<unsigned long long*>(bin_wt + nround * 32);          // [nround][1024]
 
     pdl_launch_dependents();
     const bool image_ok = fast_load_image(smem, fa.image, fa.image_bytes, bar_img, fa.flags);
@@ -375,7 +380,7 @@ gemm_sorted_kernel(FastArgs fa, const unsigned long long* __restrict__ sorted, c
     const FastSmem T = fast_view(smem, fa.L);
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     if (kBin)
-        for (int i = threadIdx.x; i < dpi * ga.nbins; i += kGemmThreads) bin_hist[i] = 0u;
+        for (int i = threadIdx.x; i < nround * ga.nbins; i += kGemmThreads) bin_hist[i] = 0u;
     if (threadIdx.x == 0) {
         mbar_init(bar_free, 1); mbar_init(bar_done, 1);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -401,7 +406,9 @@ gemm_sorted_kernel(FastArgs fa, const unsigned long long* __restrict__ sorted, c
         const ulonglong2 no_entry = make_ulonglong2(kSortIndexMask, kBigNoBlock);
         auto entry_at = [&](int d, int q) {
             if (d + q >= d_end) return no_entry;
-            if (kBin) {       // the stream words that hold the field of this thread's block of the domain (position = thread); y bit 63 = no block
+            if (kBin) {       // a round is one iteration (no room for more): the stream words that hold the field of this thread's block
+                              // (position = thread) are requested an iteration ahead into registers; y bit 63 = no block
+                if (kRound) return no_entry;             // longer rounds ask for them in L2 instead, see below
                 const int64_t row = rt * kGemmRows + (threadIdx.x >> 3), cb = (int64_t)(d + q) * kDomBlocks + (threadIdx.x & 7u);
                 if (row < ga.n_out && cb < ga.bpr)
                     return load_field_words(reinterpret_cast<const uint32_t*>(sorted), (uint64_t)(row * ga.bpr + cb), (int)fa.L.W + (kSg ? sg.bits : 0));
@@ -421,60 +428,73 @@ gemm_sorted_kernel(FastArgs fa, const unsigned long long* __restrict__ sorted, c
             e0 = entry_at(d0 + dpi, 0);
             if (dpi > 1) e1 = entry_at(d0 + dpi, 1);
             if (kBin) {
-                // ---- order the fields of each domain by the sort key of their class
-                const uint32_t nbins = (uint32_t)ga.nbins;
-                const int wbits = (int)fa.L.W + (kSg ? sg.bits : 0);
-                unsigned long long f[2] = {(cur0.y >> 63) ? kSortIndexMask : field_of_words(cur0, wbits),
-                                           (cur1.y >> 63) ? kSortIndexMask : field_of_words(cur1, wbits)};
-                uint32_t key[2] = {nbins - 1u, nbins - 1u}, rank[2] = {0u, 0u}, cnt[2] = {0u, 0u}, incl[2] = {0u, 0u};
+                const int in_round = kRound ? (d0 - d_begin) % nround : 0;  // this iteration's first domain inside the round
+                if (in_round == 0) {
+                    // ---- order the fields of the round's domains, each by the sort key of its blocks' classes
+                    const uint32_t nbins = (uint32_t)ga.nbins;
+                    const int wbits = (int)fa.L.W + (kSg ? sg.bits : 0);
+                    const int nr = min(nround, d_end - d0);                  // domains in this round
+                    const uint32_t* words = reinterpret_cast<const uint32_t*>(sorted);
+                    const int64_t row = rt * kGemmRows + (threadIdx.x >> 3);
+                    unsigned long long f[kMaxRound];
+                    uint32_t key[kMaxRound], rank[kMaxRound], cnt[kMaxRound], incl[kMaxRound];
 #pragma unroll
-                for (int q = 0; q < 2; ++q) {
-                    if (q >= nd_now) break;
-                    if (f[q] != kSortIndexMask) {
-                        const uint64_t I = kSg ? f[q] & ((1ull << fa.L.W) - 1ull) : f[q];
-                        if (I < fa.n_points) {
-                            uint64_t local;
-                            key[q] = __ldg(ga.sort_rank + fast_find_class(T, I, local));
-                        } else {
-                            atomicAdd(fa.bad_index, 1ull);
-                            f[q] = kSortIndexMask;
+                    for (int r = 0; r < kMaxRound; ++r) {
+                        f[r] = kSortIndexMask; key[r] = nbins - 1u; rank[r] = cnt[r] = incl[r] = 0u;
+                        if (r >= nr) continue;
+                        const int64_t cb = (int64_t)(d0 + r) * kDomBlocks + (threadIdx.x & 7u);
+                        if (row < ga.n_out && cb < ga.bpr) {
+                            if (!kRound) f[r] = field_of_words(r == 0 ? cur0 : cur1, wbits);            // requested an iteration ago
+                            else f[r] = load_field(words, (uint64_t)(row * ga.bpr + cb), wbits);
+                            const uint64_t I = kSg ? f[r] & ((1ull << fa.L.W) - 1ull) : f[r];
+                            if (I < fa.n_points) {
+                                uint64_t local;
+                                key[r] = __ldg(ga.sort_rank + fast_find_class(T, I, local));
+                            } else {
+                                atomicAdd(fa.bad_index, 1ull);
+                                f[r] = kSortIndexMask;
+                            }
+                            // the same block of the next round: ask for its stream words in L2
+                            const int64_t cbn = cb + (int64_t)nround * kDomBlocks;
+                            if (kRound && d0 + r + nround < d_end && cbn < ga.bpr)
+                                asm volatile("prefetch.global.L2 [%0];" ::"l"(words + (((uint64_t)(row * ga.bpr + cbn) * (uint64_t)wbits) >> 5)));
                         }
+                        rank[r] = atomicAdd(&bin_hist[r * nbins + key[r]], 1u);   // its place among the blocks of its bin
                     }
-                    rank[q] = atomicAdd(&bin_hist[q * nbins + key[q]], 1u);     // its place among the blocks of its bin
+                    __syncthreads();
+#pragma unroll
+                    for (int r = 0; r < kMaxRound; ++r) {
+                        if (r >= nr) continue;
+                        cnt[r] = threadIdx.x < nbins ? bin_hist[r * nbins + threadIdx.x] : 0u;
+                        uint32_t v = cnt[r];
+#pragma unroll
+                        for (int o = 1; o < 32; o <<= 1) { const uint32_t t = __shfl_up_sync(kFullMask, v, o); if (lane >= o) v += t; }
+                        incl[r] = v;
+                        if (lane == 31) bin_wt[r * 32 + warp] = v;
+                    }
+                    __syncthreads();
+#pragma unroll
+                    for (int r = 0; r < kMaxRound; ++r) {
+                        if (r >= nr) continue;
+                        uint32_t v = bin_wt[r * 32 + lane];                  // every warp scans the 32 warp totals
+                        const uint32_t own = v;
+#pragma unroll
+                        for (int o = 1; o < 32; o <<= 1) { const uint32_t t = __shfl_up_sync(kFullMask, v, o); if (lane >= o) v += t; }
+                        const uint32_t before = __shfl_sync(kFullMask, v - own, warp);
+                        if (threadIdx.x < nbins) bin_hist[r * nbins + threadIdx.x] = before + incl[r] - cnt[r];
+                    }
+                    __syncthreads();
+#pragma unroll
+                    for (int r = 0; r < kMaxRound; ++r) {
+                        if (r >= nr) continue;
+                        const uint32_t slot = bin_hist[r * nbins + key[r]] + rank[r];
+                        bin_ent[r * kDomEntries + slot] = f[r] | (unsigned long long)threadIdx.x << 48;
+                    }
+                    __syncthreads();
+                    for (int i = threadIdx.x; i < nround * (int)nbins; i += kGemmThreads) bin_hist[i] = 0u;   // for the next round (barriers follow below)
                 }
-                __syncthreads();
-#pragma unroll
-                for (int q = 0; q < 2; ++q) {
-                    if (q >= nd_now) break;
-                    cnt[q] = threadIdx.x < nbins ? bin_hist[q * nbins + threadIdx.x] : 0u;
-                    uint32_t v = cnt[q];
-#pragma unroll
-                    for (int o = 1; o < 32; o <<= 1) { const uint32_t t = __shfl_up_sync(kFullMask, v, o); if (lane >= o) v += t; }
-                    incl[q] = v;
-                    if (lane == 31) bin_wt[q * 32 + warp] = v;
-                }
-                __syncthreads();
-#pragma unroll
-                for (int q = 0; q < 2; ++q) {
-                    if (q >= nd_now) break;
-                    uint32_t v = bin_wt[q * 32 + lane];                    // every warp scans the 32 warp totals
-                    const uint32_t own = v;
-#pragma unroll
-                    for (int o = 1; o < 32; o <<= 1) { const uint32_t t = __shfl_up_sync(kFullMask, v, o); if (lane >= o) v += t; }
-                    const uint32_t before = __shfl_sync(kFullMask, v - own, warp);
-                    if (threadIdx.x < nbins) bin_hist[q * nbins + threadIdx.x] = before + incl[q] - cnt[q];
-                }
-                __syncthreads();
-#pragma unroll
-                for (int q = 0; q < 2; ++q) {
-                    if (q >= nd_now) break;
-                    const uint32_t slot = bin_hist[q * nbins + key[q]] + rank[q];
-                    bin_ent[q * kDomEntries + slot] = f[q] | (unsigned long long)threadIdx.x << 48;
-                }
-                __syncthreads();
-                for (int i = threadIdx.x; i < dpi * (int)nbins; i += kGemmThreads) bin_hist[i] = 0u;   // for the next iteration (a barrier follows below)
-                cur0 = make_ulonglong2(bin_ent[(warp == 0 ? 31 : warp - 1) * 32 + lane], 0ull);
-                if (nd_now > 1) cur1 = make_ulonglong2(bin_ent[kDomEntries + (warp == 0 ? 31 : 31 - warp) * 32 + lane], 0ull);
+                cur0 = make_ulonglong2(bin_ent[in_round * kDomEntries + (warp == 0 ? 31 : warp - 1) * 32 + lane], 0ull);
+                if (nd_now > 1) cur1 = make_ulonglong2(bin_ent[(in_round + 1) * kDomEntries + (warp == 0 ? 31 : 31 - warp) * 32 + lane], 0ull);
             }
             // ---- A: every warp unranks one chunk of 32 sorted entries per domain
 #pragma unroll
