@@ -156,6 +156,34 @@ int launch_gemm(const llvq_ctx* ctx, const void* d_idx, const uint16_t* d_gain_f
             return launch_status();
         }
     }
+    // the 72-bit code at wide batches (one domain per iteration): the same with the coarse shape of the unranking as sort key,
+    // four domains ordered per round (at padded batch <= 32 the pipeline kernel on unordered chunks is faster: measured)
+    if (!ctx->fast && ctx->host.W > 64 && ctx->host.W <= 72 && ga.npad > 32 && !sg && (int)ctx->host.desc.size() <= (1 << kBigClassBits)) {
+        const size_t head = (img + 64 + 1023) & ~size_t(1023), a_set = (size_t)kDomStages * kGemmRows * kStageK * 2,
+                     x_set = (size_t)kDomStages * ga.npad * kStageK * 2;
+        GemmArgs gb = ga;
+        gb.nstages = (int)((ga.bpr + kDomBlocks - 1) / kDomBlocks);            // domains per row tile
+        gb.split = 1;
+        gb.nbins = 160;                                                         // 128 shapes; the last bin is "no block"
+        gb.bin_round = 4;
+        const size_t bins = (size_t)gb.nbins * 4 + 32 * 4 + (size_t)kDomEntries * (8 + 4);
+        const int dpi = 1;
+        const size_t smem_bin = head + (size_t)dpi * (a_set + x_set) + (size_t)gb.bin_round * bins;
+        if (smem_bin <= 227 * 1024) {
+            const unsigned grid_bin = (unsigned)std::min<int64_t>(row_tiles * gb.nstages, ctx->sm_count);
+            const unsigned long long* words = static_cast<const unsigned long long*>(d_idx);
+            if (yo) {
+                if (!set_smem(gemm_sorted_kernel<true, false, true, true, true>, smem_bin)) return LLVQ_ECUDA;
+                if (launch_pdl(gemm_sorted_kernel<true, false, true, true, true>, grid_bin, (unsigned)kGemmThreads, smem_bin, st, fast_args(ctx, true), words,
+                               d_gain_f16, SgArgs{}, gb, dpi) != cudaSuccess) return LLVQ_ECUDA;
+            } else {
+                if (!set_smem(gemm_sorted_kernel<true, false, false, true, true>, smem_bin)) return LLVQ_ECUDA;
+                if (launch_pdl(gemm_sorted_kernel<true, false, false, true, true>, grid_bin, (unsigned)kGemmThreads, smem_bin, st, fast_args(ctx, true), words,
+                               d_gain_f16, SgArgs{}, gb, dpi) != cudaSuccess) return LLVQ_ECUDA;
+            }
+            return launch_status();
+        }
+    }
     {
         // the kernel without a block barrier (see gemm_pipe_kernel), if its buffers fit
         const size_t head = (img + 64 + 1023) & ~size_t(1023), a_set = (size_t)kDomStages * kGemmRows * kStageK * 2,

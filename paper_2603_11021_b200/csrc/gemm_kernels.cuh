@@ -345,11 +345,15 @@ sort_blocks_gemm_big_kernel(FastArgs fa, const uint32_t* __restrict__ stream, in
 // stream sorted at load time.  ga.bin_round domains are ordered at a time (their four block barriers are then paid once per
 // round, not once per iteration); the stream words of the next round are requested in L2 a round ahead.
 // kRound (with kBin): a round is longer than an iteration; else it is one iteration and the words come through registers.
+// kBin with kBig (class tables in global memory; rounds only): the bins are the coarse shape of the unranking (parity,
+// number of steps, steps of the first group: 128 bins) instead of the full key of the sorted layout, the entries
+// (class-local index, class | position) as in the 96-bit layout; the class look-ups of a round's domains (dependent
+// reads from L2) run side by side.
 template <bool kBig, bool kSg = false, bool kShard = false, bool kBin = false, bool kRound = false>
 __global__ void __launch_bounds__(kGemmThreads, 1)
 gemm_sorted_kernel(FastArgs fa, const unsigned long long* __restrict__ sorted, const uint16_t* __restrict__ gain, SgArgs sg, GemmArgs ga, int dpi)
 {
-    static_assert(!(kBin && kBig), "the in-kernel ordering is for the codes whose class tables sit in shared memory");
+    static_assert(!(kBin && kBig && (kSg || !kRound)), "in-kernel ordering for the codes with tables in global memory: stored gains, rounds");
     extern __shared__ __align__(128) uint8_t smem[];
     const uint32_t img_bytes = fa.image_bytes;
     uint64_t* bar_img = reinterpret_cast<uint64_t*>(smem + img_bytes);
@@ -369,6 +373,7 @@ gemm_sorted_kernel(FastArgs fa, const unsigned long long* __restrict__ sorted, c
     uint32_t* bin_hist = reinterpret_cast<uint32_t*>(b_buf + (uint32_t)dpi * kDomStages * b_stage);   // [nround][nbins] counts, then first slots
     uint32_t* bin_wt = bin_hist + nround * ga.nbins;                        // [nround][32]
     unsigned long long* bin_ent = reinterpret_cast<unsigned long long*>(bin_wt + nround * 32);          // [nround][1024]
+    uint32_t* bin_ent2 = reinterpret_cast<uint32_t*>(bin_ent + nround * kDomEntries);                    // kBig: [nround][1024] class | position << 17
 
     pdl_launch_dependents();
     const bool image_ok = fast_load_image(smem, fa.image, fa.image_bytes, bar_img, fa.flags);
@@ -437,13 +442,34 @@ gemm_sorted_kernel(FastArgs fa, const unsigned long long* __restrict__ sorted, c
                     const uint32_t* words = reinterpret_cast<const uint32_t*>(sorted);
                     const int64_t row = rt * kGemmRows + (threadIdx.x >> 3);
                     unsigned long long f[kMaxRound];
+                    uint32_t f2[kMaxRound];                                  // kBig: class | position << 17
                     uint32_t key[kMaxRound], rank[kMaxRound], cnt[kMaxRound], incl[kMaxRound];
 #pragma unroll
                     for (int r = 0; r < kMaxRound; ++r) {
-                        f[r] = kSortIndexMask; key[r] = nbins - 1u; rank[r] = cnt[r] = incl[r] = 0u;
+                        f[r] = kBig ? kBigNoBlock : kSortIndexMask; f2[r] = threadIdx.x << kBigClassBits;
+                        key[r] = nbins - 1u; rank[r] = cnt[r] = incl[r] = 0u;
                         if (r >= nr) continue;
                         const int64_t cb = (int64_t)(d0 + r) * kDomBlocks + (threadIdx.x & 7u);
-                        if (row < ga.n_out && cb < ga.bpr) {
+                        if (kBig) {
+                            if (row < ga.n_out && cb < ga.bpr) {
+                                uint64_t lo, hi;
+                                load_index(words, (uint64_t)(row * ga.bpr + cb), fa.dc.W, lo, hi);
+                                if (hi < fa.dc.n_hi || (hi == fa.dc.n_hi && lo < fa.dc.n_lo)) {
+                                    uint64_t local;
+                                    const uint32_t cls = (uint32_t)big_find_class(fa.dc, lo, hi, local);
+                                    const uint32_t h = __ldg(reinterpret_cast<const uint32_t*>(fa.dc.big + cls));
+                                    const uint32_t nlev = h >> 28, nlev1 = (h >> 24) & 7u, parity = (h >> 16) & 1u;
+                                    key[r] = (1u - parity) << 6 | (7u - min(nlev, 7u)) << 3 | nlev1;
+                                    f[r] = local;
+                                    f2[r] |= cls;
+                                } else {
+                                    atomicAdd(fa.bad_index, 1ull);
+                                }
+                                const int64_t cbn = cb + (int64_t)nround * kDomBlocks;
+                                if (d0 + r + nround < d_end && cbn < ga.bpr)
+                                    asm volatile("prefetch.global.L2 [%0];" ::"l"(words + (((uint64_t)(row * ga.bpr + cbn) * (uint64_t)fa.dc.W) >> 5)));
+                            }
+                        } else if (row < ga.n_out && cb < ga.bpr) {
                             if (!kRound) f[r] = field_of_words(r == 0 ? cur0 : cur1, wbits);            // requested an iteration ago
                             else f[r] = load_field(words, (uint64_t)(row * ga.bpr + cb), wbits);
                             const uint64_t I = kSg ? f[r] & ((1ull << fa.L.W) - 1ull) : f[r];
@@ -488,13 +514,21 @@ gemm_sorted_kernel(FastArgs fa, const unsigned long long* __restrict__ sorted, c
                     for (int r = 0; r < kMaxRound; ++r) {
                         if (r >= nr) continue;
                         const uint32_t slot = bin_hist[r * nbins + key[r]] + rank[r];
-                        bin_ent[r * kDomEntries + slot] = f[r] | (unsigned long long)threadIdx.x << 48;
+                        if (kBig) { bin_ent[r * kDomEntries + slot] = f[r]; bin_ent2[r * kDomEntries + slot] = f2[r]; }
+                        else bin_ent[r * kDomEntries + slot] = f[r] | (unsigned long long)threadIdx.x << 48;
                     }
                     __syncthreads();
                     for (int i = threadIdx.x; i < nround * (int)nbins; i += kGemmThreads) bin_hist[i] = 0u;   // for the next round (barriers follow below)
                 }
-                cur0 = make_ulonglong2(bin_ent[in_round * kDomEntries + (warp == 0 ? 31 : warp - 1) * 32 + lane], 0ull);
-                if (nd_now > 1) cur1 = make_ulonglong2(bin_ent[(in_round + 1) * kDomEntries + (warp == 0 ? 31 : 31 - warp) * 32 + lane], 0ull);
+                auto ordered = [&](int at) {                               // entry `at` of the round's ordered domains in the form the unranking takes
+                    if (!kBig) return make_ulonglong2(bin_ent[at], 0ull);
+                    const unsigned long long x = bin_ent[at];
+                    const uint32_t y2 = bin_ent2[at];
+                    return make_ulonglong2(x & ~kBigNoBlock, (x & kBigNoBlock) | (unsigned long long)(y2 & ((1u << kBigClassBits) - 1u)) << 8 |
+                                                                  (unsigned long long)(y2 >> kBigClassBits) << 32);
+                };
+                cur0 = ordered(in_round * kDomEntries + (warp == 0 ? 31 : warp - 1) * 32 + lane);
+                if (nd_now > 1) cur1 = ordered((in_round + 1) * kDomEntries + (warp == 0 ? 31 : 31 - warp) * 32 + lane);
             }
             // ---- A: every warp unranks one chunk of 32 sorted entries per domain
 #pragma unroll
