@@ -301,6 +301,28 @@ def test_products_on_a_stream_with_out_of_range_fields(lib, ctxs, oracle_mod, co
         assert err.max() <= TOL_BF16_OUT
 
 
+@pytest.mark.parametrize("code", [(2, 13), (2, 53)])
+def test_gemm_stored_stream_and_sorted_layout_agree_on_random_shapes(lib, ctxs, code):
+    # the kernels that serve the stored stream (domains ordered inside the kernel, one, two or four per round, or unordered
+    # chunks) and the sorted layout unrank the same blocks: their products may differ by the accumulation order only.  Both
+    # are compared with the oracle elsewhere; this sweep runs through many ragged shapes and every padded batch cheaply.
+    ctx = ctxs[code]
+    rng = np.random.default_rng(31)
+    for case in range(14):
+        n_out, k_in = int(rng.integers(1, 900)), int(rng.integers(1, 260)) * 8
+        batch = [1, 16, 17, 32, 33, 48, 49, 64][case % 8]
+        stream, gain, _ = gen.make_layer(ctx.num_points, ctx.index_bits, n_out, k_in, 1, seed=100 + case)
+        X = to_dev_bf16(gen.normal_bf16((batch, k_in), seed=case))
+        d_idx, d_gain = to_dev_u8(stream), to_dev_f16(gain)
+        y1 = lib.llvq_gemm_small_batch(ctx, d_idx, d_gain, n_out, k_in, X).float()
+        y2 = lib.llvq_gemm_small_batch_sorted(ctx, lib.llvq_sort_blocks_gemm(ctx, d_idx, n_out, k_in), d_gain, n_out, k_in, X).float()
+        torch.cuda.synchronize()
+        assert lib.llvq_last_error(ctx) == (0, 0)
+        floor = 1e-3 * y2.abs().max().clamp_min(1e-30)
+        err = ((y1 - y2).abs() / y2.abs().clamp_min(floor)).max().item()
+        assert err <= 2.0 ** -7, (err, n_out, k_in, batch)          # one bf16 step at most
+
+
 def test_gemm_exact_integer_case(lib, ctxs, oracle_mod):
     # gains = 1, X = 0/1 patterns: every partial sum is a small integer, exact in binary32 and in bf16
     o = _oracle(oracle_mod)((2, 13))
