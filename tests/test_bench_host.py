@@ -95,3 +95,22 @@ def test_reference_arm_prints_on_rank0_only():
     line = json.loads(r.stdout.strip().splitlines()[-1])
     assert line["impl"] == "reference" and line["cpu_baseline"]["kind"] == "oracle" and line["value"] > 0
     assert line["e2e"]["h2d_bytes_per_step"] == 0 and line["unit"] == "GB/s"
+
+
+def test_counter_file_vouches_for_its_sources_only(tmp_path):
+    # the benchmark quotes profiler counters only while the sources the captured kernel is compiled from are unchanged
+    sys.path.insert(0, ROOT)
+    from paper_2603_11021_b200 import ncu_counters as nc
+    raw = tmp_path / "raw.csv"
+    raw.write_text('"ID","Kernel Name","gpu__time_duration.sum","dram__bytes_read.sum","smsp__inst_executed.sum"\n'
+                   '"","","us","Mbyte","inst"\n'
+                   '"0","void k<1>(int)","120.5","45.0","1000"\n')
+    d = nc.parse_raw_csv(str(raw))
+    assert d["kernel"] == "void k<1>" and d["duration_ns"] == 120500.0 and d["dram_bytes_read"] == 45e6 and d["warp_instructions"] == 1000.0
+    good = tmp_path / "good.json"
+    good.write_text(json.dumps({"duration_ns": 1.0, "sources": ["tables.h"], "source_hash": nc.source_hash(["tables.h"])}))
+    assert nc.load(str(good))["duration_ns"] == 1.0
+    stale = tmp_path / "stale.json"
+    stale.write_text(json.dumps({"duration_ns": 1.0, "sources": ["tables.h"], "source_hash": "0" * 16}))
+    assert nc.load(str(stale)) is None and nc.load(str(tmp_path / "missing.json")) is None
+    assert nc.source_hash(["tables.h"]) != nc.source_hash(["tables.h", "fast.cuh"])
