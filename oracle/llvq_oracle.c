@@ -459,10 +459,10 @@ static const oc_class* find_class(const oc_code* code, u128 I)
 /* Sign conventions (paper silent on which bit signs which coordinate):       */
 /*   odd:  x_i = -a_i iff c_i xor ((a_i >> 1) & 1), i.e. x_i = 1 mod 4 on F0  */
 /*         and 3 mod 4 on F1 (Sec. 2.4).                                      */
-/*   even: the F1 positions in ascending order take bits 0..w-2 of s (1 =     */
-/*         negative) and the last F1 position takes the sign that makes the   */
-/*         coordinate sum 0 mod 8; then the nonzero F0 positions in ascending */
-/*         order take the following bits of s.                                */
+/*   even: the positions that carry a sign -- all of F1 and the nonzero ones  */
+/*         of F0 -- take the bits of s in ascending order of position (1 =    */
+/*         negative), except the last F1 position, which takes the sign that  */
+/*         makes the coordinate sum 0 mod 8.                                  */
 /* ------------------------------------------------------------------------- */
 static int unrank_point(const oc_code* code, u128 I, int8_t x[OC_DIM])
 {
@@ -502,17 +502,18 @@ static int unrank_point(const oc_code* code, u128 I, int8_t x[OC_DIM])
     int a1[OC_DIM], a0[OC_DIM];
     if (n1) arrange(p1, v1, m1, nv1, n1, a1);
     if (n0) arrange(p0, v0, m0, nv0, n0, a0);
+    /* absolute values by position, then the signs in one pass over the positions */
+    int abs_at[OC_DIM];
+    for (int t = 0; t < n1; ++t) abs_at[F1[t]] = a1[t];
+    for (int t = 0; t < n0; ++t) abs_at[F0[t]] = a0[t];
+    const int last_f1 = n1 ? F1[n1 - 1] : -1;
     int bit = 0, negs = 0;
-    for (int t = 0; t < n1; ++t) {
-        int neg;
-        if (t < n1 - 1) { neg = (int)((s >> bit) & 1u); ++bit; negs += neg; }
-        else neg = (negs + n4 + n6) & 1;
-        x[F1[t]] = (int8_t)(neg ? -a1[t] : a1[t]);
-    }
-    for (int t = 0; t < n0; ++t) {
+    for (int i = 0; i < OC_DIM; ++i) {
+        const int in_f1 = (int)((c >> i) & 1u);
         int neg = 0;
-        if (a0[t] != 0) { neg = (int)((s >> bit) & 1u); ++bit; }
-        x[F0[t]] = (int8_t)(neg ? -a0[t] : a0[t]);
+        if (in_f1 && i == last_f1) neg = (negs + n4 + n6) & 1;          /* every other F1 sign is known by now */
+        else if (in_f1 || abs_at[i] != 0) { neg = (int)((s >> bit) & 1u); ++bit; negs += in_f1 ? neg : 0; }
+        x[i] = (int8_t)(neg ? -abs_at[i] : abs_at[i]);
     }
     return 0;
 }
@@ -565,9 +566,13 @@ static int rank_point(const oc_code* code, const int8_t x[OC_DIM], u128* I)
         u128 p1 = n1 ? arrange_rank(a1, v1, m1, nv1, n1) : 0;
         u128 p0 = n0 ? arrange_rank(a0, v0, m0, nv0, n0) : 0;
         p = p1 + k->P1 * p0;
+        const int last_f1 = n1 ? F1[n1 - 1] : -1;
         int bit = 0;
-        for (int t = 0; t + 1 < n1; ++t) { s |= (u128)(x[F1[t]] < 0) << bit; ++bit; }
-        for (int t = 0; t < n0; ++t) if (a0[t] != 0) { s |= (u128)(x[F0[t]] < 0) << bit; ++bit; }
+        for (int i = 0; i < OC_DIM; ++i) {
+            const int in_f1 = (int)((c >> i) & 1u);
+            if (in_f1 && i == last_f1) continue;                           /* fixed by the others */
+            if (in_f1 || a[i] != 0) { s |= (u128)(x[i] < 0) << bit; ++bit; }
+        }
     }
     *I = k->offset + r + (u128)k->A * (s + ((u128)1 << k->B) * p);
     return 0;

@@ -136,13 +136,14 @@ __device__ __forceinline__ void big_decode_record(const FastSmem& T, const uint4
     if (flags & 4u) nz0 |= freem;
 
     // S6: signs
-    const uint32_t nf1 = w ? w - 1u : 0u;                           // free sign bits on F1
-    const uint32_t s1 = s & ((1u << nf1) - 1u);
-    const uint32_t src1 = s1 | (((__popc(s1) + (flags >> 1)) & 1u) << nf1);     // last F1 position: sum = 0 mod 8
     uint32_t neg;
     if (__all_sync(mask, odd)) neg = c ^ bit1;                      // 1 mod 4 on F0, 3 mod 4 on F1
     else {
-        const uint32_t neg_even = deposit24(T.pd6, src1, F1) | deposit24(T.pd6, s >> nf1, odd ? 0u : nz0);
+        // the bits of s go to the positions that carry a sign (F1 and the nonzero ones of F0) in ascending order, except the
+        // last F1 position: its sign makes the sum 0 mod 8
+        const uint32_t last_f1 = F1 ? 0x80000000u >> __clz(F1) : 0u;
+        uint32_t neg_even = deposit24(T.pd6, s, (F1 | (odd ? 0u : nz0)) & ~last_f1);
+        if ((__popc(neg_even & F1) + (flags >> 1)) & 1u) neg_even |= last_f1;
         neg = odd ? (c ^ bit1) : neg_even;
     }
     if (valid) {

@@ -312,10 +312,11 @@ rank_kernel(DevCode dc, EncTables et, const uint32_t* __restrict__ golay, const 
         if (parity) {
             good &= neg == (c ^ bit1);                                     // 1 mod 4 on F0, 3 mod 4 on F1
         } else {
-            const uint32_t nf1 = d.w ? d.w - 1u : 0u;
-            const uint32_t s1_all = extract_bits(neg, F1), s1 = s1_all & ((1u << nf1) - 1u);
-            if (d.w) good &= ((s1_all >> nf1) & 1u) == ((__popc(s1) + d.signpar) & 1u);   // sum = 0 mod 8
-            s = s1 | (unsigned long long)extract_bits(neg, F0 & nonzero) << nf1;
+            // s = the signs of the positions that carry one (F1 and the nonzero ones of F0), ascending, without the last F1
+            // position, whose sign the others fix (sum = 0 mod 8)
+            const uint32_t last_f1 = F1 ? 0x80000000u >> __clz(F1) : 0u;
+            if (d.w) good &= ((neg & last_f1) != 0u) == (((__popc(neg & F1 & ~last_f1) + d.signpar) & 1u) != 0u);
+            s = extract_bits(neg, (F1 | (F0 & nonzero)) & ~last_f1);
         }
         I = dc.off_lo[cls] + r + (unsigned long long)d.A * (s + (p << d.B));
     }
