@@ -102,7 +102,11 @@ __device__ __forceinline__ void big_decode_record(const FastSmem& T, const uint4
             const uint32_t cell = nfree * 25u + k;                  // C(nfree, k) and its reciprocals
             const uint32_t radix = lds_u32(pascal_a + cell * 4u);
             uint32_t rho = 0u;
-            if (__any_sync(mask, (uint32_t)(p >> 32) != 0u)) {
+            if (l + 1 == maxlev) {
+                // the last step of the warp: what is left of the rank is the step's own digit (a lane without this step holds 0
+                // and places the empty subset), no division
+                rho = (uint32_t)p;
+            } else if (__any_sync(mask, (uint32_t)(p >> 32) != 0u)) {
                 const uint64_t qq0 = __umul64hi(p, lds_u64(r64_a + cell * 8u));
                 uint64_t qq = qq0, rem = p - qq * radix;
                 if (rem >= radix) { rem -= radix; ++qq; }

@@ -241,7 +241,11 @@ __device__ __forceinline__ void fast_decode_local(const FastSmem& T, uint32_t cl
             const uint32_t k = (word >> 22) & 31u;
             const uint32_t nfree = (mg.w >> (8 * l)) & 0xffu;            // slots free before this step (0: no step)
             uint32_t rho;
-            if (l == 0 && !rank32) {
+            if (l + 1 == maxlev) {
+                // the last step of the warp: what is left of the rank is the step's own digit (lanes whose class has fewer steps
+                // hold 0 here and place the empty subset), no division
+                rho = p32;
+            } else if (l == 0 && !rank32) {
                 uint64_t qq = __umul64hi(p, ((uint64_t)v.w << 32) | v.z);
                 uint64_t rem = p - qq * radix;
                 if (rem >= radix) { rem -= radix; ++qq; }
